@@ -1,0 +1,154 @@
+/*
+ * libcott -- cosine attention (Cottention, arXiv 2409.18747) for NVIDIA B200 (sm_100a).
+ *
+ * C ABI.  Plain pointers and sizes only.  Unless a parameter says "host", every
+ * tensor pointer is a DEVICE pointer owned by the caller; the library never
+ * allocates, frees or keeps caller memory.  Scratch memory comes from the
+ * caller-supplied workspace (size it with cott_workspace_bytes).
+ *
+ * Symbols: B batch, H heads, N sequence length, d per-head dimension (one d for
+ * keys and values).  q,k,v,o,d_o,dq,dk,dv are contiguous row-major [B,H,N,d] in
+ * the I/O dtype `dt`; decode tensors are [B,H,d]; `m`, `seq_len`, `state`, `dm`
+ * are always fp32.
+ *
+ * What is computed (paper equations):
+ *   x^      = x / max(||x||_2, 1e-12)            row normalisation of Q and K (Eq. 2, Eq. 3)
+ *   c[b,h]  = s_b ^ (-sigmoid(m_h))              stabilisation factor (Eq. 4); s_b >= 1
+ *   bidirectional: O = c * Q^ (K^^T V)           (Eq. 3 re-associated as in Eq. 5)
+ *   causal:        o_t = c * sum_{j<=t} (q^_t . k^_j) v_j     (Eq. 6, diagonal kept)
+ *                  computed through the running state of Eq. 7 / Eq. 8,
+ *                  S_t = S_{t-1} + k^_t (c v_t)^T ,  o_t = S_t^T q^_t
+ *   state layout: [B,H,d_key,d_value] fp32, S = sum_j k^_j (c v_j)^T
+ *                  (the paper's hidden state H_t transposed, scale included).
+ *
+ * All calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL is
+ * the legacy default stream).  The returned status covers argument validation and
+ * launch errors only.  Calls are thread-safe as long as concurrent calls use
+ * different workspaces.  Outputs must not alias inputs.
+ */
+#ifndef COTT_H_
+#define COTT_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    COTT_OK = 0,
+    COTT_ERR_INVALID_ARG = -1, /* NULL required pointer, non-positive size, s < 1, aliasing      */
+    COTT_ERR_UNSUPPORTED = -2, /* d not in {32,64,128}, unknown dtype, pointer not 16-B aligned  */
+    COTT_ERR_WORKSPACE = -3,   /* workspace NULL or smaller than cott_workspace_bytes()          */
+    COTT_ERR_CUDA = -4,        /* a CUDA runtime / driver call failed (see cott_last_cuda_error) */
+    COTT_ERR_TIMEOUT = -5      /* a bounded device-side wait expired (reported asynchronously)   */
+} cott_status;
+
+typedef enum { COTT_F32 = 0, COTT_BF16 = 1 } cott_dtype;
+
+typedef enum { COTT_OP_FWD = 0, COTT_OP_BWD = 1, COTT_OP_DECODE = 2 } cott_op;
+
+/* Parameters of the stabilisation factor of Eq. 4. */
+typedef struct {
+    const float* m;       /* device [H]: the learned per-head scalar; required                  */
+    const float* seq_len; /* device [B]: scaling base s_b per batch item, or NULL                */
+    float seq_len_scalar; /* used when seq_len == NULL: fwd/bwd take s_b = N if this is <= 0,    */
+                          /* otherwise this value; decode requires it (>= 1) when seq_len==NULL  */
+} cott_scale_params;
+
+/* Library version (major*10000 + minor*100 + patch). */
+int cott_version(void);
+
+/* Human-readable name of a status code (static string). */
+const char* cott_status_string(cott_status st);
+
+/* Text of the last CUDA error seen by this thread inside the library (static storage). */
+const char* cott_last_cuda_error(void);
+
+/*
+ * Bytes of device scratch the given call needs (0 is possible).  `op` is a cott_op.
+ * The workspace must be 256-byte aligned.  Returns (size_t)-1 for unsupported arguments.
+ */
+size_t cott_workspace_bytes(int op, cott_dtype dt, int B, int H, int N, int d, int causal);
+
+/*
+ * Reports how a call would be executed (for tests and tuning):
+ *   *path   0 = fp32 SIMT kernels, 1 = tcgen05 tensor-core kernels
+ *   *group  tokens per sequence group (the unit of sequence-level parallelism; the per-group
+ *           partial states are combined by an exclusive prefix scan, which is valid because
+ *           the cumulative sum of Eq. 7 is associative)
+ *   *chunk  tokens per chunk inside a group (tile of the masked Q^K^^T product, Eq. 6)
+ * Any output pointer may be NULL.  Host pointers.
+ */
+cott_status cott_query_plan(int op, cott_dtype dt, int B, int H, int N, int d, int causal,
+                            int* path, int* group, int* chunk);
+
+/*
+ * Forward pass: Eq. 3/4/5 (causal == 0) or Eq. 6/7/8 (causal != 0).
+ *   q,k,v   in : [B,H,N,d] dt
+ *   o       out: [B,H,N,d] dt
+ *   state_out  : NULL, or fp32 [B,H,d,d] receiving S_N = sum_j k^_j (c v_j)^T over all N tokens
+ *                (the state a following cott_decode_step continues from, Eq. 8)
+ * Rows of Q or K whose norm is <= 1e-12 normalise to (near) zero: a zero K row contributes
+ * nothing, a zero Q row yields a zero output row.  N need not be a multiple of any tile.
+ */
+cott_status cott_fwd(const void* q, const void* k, const void* v, void* o, float* state_out,
+                     int B, int H, int N, int d, int causal, cott_dtype dt,
+                     const cott_scale_params* sp, void* workspace, size_t workspace_bytes,
+                     void* stream);
+
+/*
+ * Backward pass of cott_fwd for L = sum(d_o * O): the gradient formulas printed after Eq. 7
+ * (dQ^ = (dO V'^T . M) K^, dK^ = (dO V'^T . M)^T Q^, dV' = (Q^ K^^T . M)^T dO; M all-ones when
+ * causal == 0), evaluated through a forward running state and a state that accumulates
+ * backward in time, followed by the chain rule through the row normalisation (Eq. 2/3) and
+ * the stabilisation factor (Eq. 4):
+ *   dq,dk,dv out: [B,H,N,d] dt, gradients w.r.t. the RAW q,k,v
+ *   dm       out: fp32 [H], gradient w.r.t. m summed over batch and positions; overwritten
+ * On a row with norm <= 1e-12 the gradient is that of the clamped formula, d x^ / 1e-12.
+ * There is no gradient for the scaling base s.
+ */
+cott_status cott_bwd(const void* q, const void* k, const void* v, const void* d_o, void* dq,
+                     void* dk, void* dv, float* dm, int B, int H, int N, int d, int causal,
+                     cott_dtype dt, const cott_scale_params* sp, void* workspace,
+                     size_t workspace_bytes, void* stream);
+
+/*
+ * One recurrent decode step, Eq. 8:  S <- S + k^ (c v)^T ;  o = S^T q^  (update, then read).
+ *   q,k,v  in    : [B,H,d] dt
+ *   state  in/out: fp32 [B,H,d,d], updated in place (constant-size inference memory)
+ *   o      out   : [B,H,d] dt
+ * The scaling base comes from sp->seq_len ([B]) or sp->seq_len_scalar (>= 1); keeping the
+ * prefill's value makes prefill + decode equal to one longer causal forward.
+ * Needs no workspace.
+ */
+cott_status cott_decode_step(const void* q, const void* k, const void* v, float* state, void* o,
+                             int B, int H, int d, cott_dtype dt, const cott_scale_params* sp,
+                             void* stream);
+
+/*
+ * Training step with HOST buffers (end-to-end path): copies q,k,v,d_o from host memory to the
+ * device arena, runs cott_fwd then cott_bwd, and copies o,dq,dk,dv,dm back, all on `stream`.
+ *   *_host  : host pointers ([B,H,N,d] dt; dm_host fp32 [H]); pinned memory makes the copies
+ *             asynchronous.  m_host fp32 [H], seq_len_host fp32 [B] or NULL (s_b = N).
+ *   arena   : device scratch of at least cott_host_step_arena_bytes() bytes, 256-B aligned.
+ * The caller synchronises `stream` before reading the host outputs.
+ */
+size_t cott_host_step_arena_bytes(cott_dtype dt, int B, int H, int N, int d, int causal);
+cott_status cott_fwd_bwd_host(const void* q_host, const void* k_host, const void* v_host,
+                              const void* d_o_host, void* o_host, void* dq_host, void* dk_host,
+                              void* dv_host, float* dm_host, const float* m_host,
+                              const float* seq_len_host, int B, int H, int N, int d, int causal,
+                              cott_dtype dt, void* arena, size_t arena_bytes, void* stream);
+
+/*
+ * Synchronises `stream`, then reads the status word the last call using `workspace` left
+ * there: COTT_OK, or COTT_ERR_TIMEOUT if a bounded device-side wait gave up, or COTT_ERR_CUDA
+ * if the stream reports an error.
+ */
+cott_status cott_last_async_status(const void* workspace, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* COTT_H_ */

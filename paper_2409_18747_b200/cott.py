@@ -1,0 +1,211 @@
+"""ctypes binding of the libcott C ABI: argument marshalling only.
+
+Function names and argument order follow ``include/cott.h``.  Tensors are torch CUDA
+tensors (contiguous ``[B,H,N,d]``, float32 or bfloat16); outputs and the workspace are
+allocated here with torch because the library itself never allocates.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_PKG, "libcott.so")
+_lib = None
+
+OP_FWD, OP_BWD, OP_DECODE = 0, 1, 2
+F32, BF16 = 0, 1
+_SIZE_MAX = ctypes.c_size_t(-1).value
+
+
+class CottError(RuntimeError):
+    """A libcott call returned a non-zero status."""
+
+    def __init__(self, status: int, where: str):
+        lib = _load()
+        msg = lib.cott_status_string(status).decode()
+        cuda = lib.cott_last_cuda_error().decode()
+        super().__init__(f"{where}: {msg} ({status})" + (f" [{cuda}]" if status == -4 and cuda else ""))
+        self.status = status
+
+
+class _ScaleParams(ctypes.Structure):
+    _fields_ = [("m", ctypes.c_void_p), ("seq_len", ctypes.c_void_p), ("seq_len_scalar", ctypes.c_float)]
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def _load():
+    """Loads libcott.so; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise RuntimeError(
+            f"{_LIB_PATH} is missing: build it with `python -m paper_2409_18747_b200._build` "
+            "(libcott has no CPU or PyTorch fallback)")
+    lib = ctypes.CDLL(_LIB_PATH)
+    vp, ci, cs = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    lib.cott_version.restype = ci
+    lib.cott_status_string.restype = ctypes.c_char_p
+    lib.cott_status_string.argtypes = [ci]
+    lib.cott_last_cuda_error.restype = ctypes.c_char_p
+    lib.cott_workspace_bytes.restype = cs
+    lib.cott_workspace_bytes.argtypes = [ci, ci, ci, ci, ci, ci, ci]
+    lib.cott_query_plan.restype = ci
+    lib.cott_query_plan.argtypes = [ci] * 7 + [ctypes.POINTER(ci)] * 3
+    lib.cott_fwd.restype = ci
+    lib.cott_fwd.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci,
+                             ctypes.POINTER(_ScaleParams), vp, cs, vp]
+    lib.cott_bwd.restype = ci
+    lib.cott_bwd.argtypes = [vp] * 8 + [ci, ci, ci, ci, ci, ci, ctypes.POINTER(_ScaleParams), vp, cs, vp]
+    lib.cott_decode_step.restype = ci
+    lib.cott_decode_step.argtypes = [vp] * 5 + [ci, ci, ci, ci, ctypes.POINTER(_ScaleParams), vp]
+    lib.cott_host_step_arena_bytes.restype = cs
+    lib.cott_host_step_arena_bytes.argtypes = [ci] * 6
+    lib.cott_fwd_bwd_host.restype = ci
+    lib.cott_fwd_bwd_host.argtypes = [vp] * 11 + [ci] * 6 + [vp, cs, vp]
+    lib.cott_last_async_status.restype = ci
+    lib.cott_last_async_status.argtypes = [vp, vp]
+    _lib = lib
+    return lib
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"libcott supports float32 and bfloat16 I/O, got {t.dtype}")
+
+
+def _check_dev(*ts):
+    for t in ts:
+        if t is None:
+            continue
+        if not t.is_cuda:
+            raise RuntimeError("libcott needs CUDA tensors (there is no CPU path)")
+        if not t.is_contiguous():
+            raise ValueError("libcott needs contiguous tensors")
+
+
+def _stream_ptr(stream) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return int(s.cuda_stream)
+
+
+def _scale(m: torch.Tensor, seq_len, scalar: float = 0.0) -> _ScaleParams:
+    sp = _ScaleParams()
+    sp.m = m.data_ptr()
+    sp.seq_len = seq_len.data_ptr() if isinstance(seq_len, torch.Tensor) else None
+    sp.seq_len_scalar = float(seq_len) if (seq_len is not None and not isinstance(seq_len, torch.Tensor)) else scalar
+    return sp
+
+
+def workspace_bytes(op: int, dt: int, B: int, H: int, N: int, d: int, causal: bool) -> int:
+    n = _load().cott_workspace_bytes(op, dt, B, H, N, d, int(bool(causal)))
+    if n == _SIZE_MAX:
+        raise CottError(-2, "cott_workspace_bytes")
+    return int(n)
+
+
+def query_plan(op: int, dt: int, B: int, H: int, N: int, d: int, causal: bool) -> dict:
+    path, group, chunk = ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
+    rc = _load().cott_query_plan(op, dt, B, H, N, d, int(bool(causal)), ctypes.byref(path),
+                                 ctypes.byref(group), ctypes.byref(chunk))
+    if rc != 0:
+        raise CottError(rc, "cott_query_plan")
+    return {"path": path.value, "group": group.value, "chunk": chunk.value}
+
+
+def _workspace(op, dt, B, H, N, d, causal, device, workspace):
+    need = workspace_bytes(op, dt, B, H, N, d, causal)
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=device)
+    return workspace, workspace.numel()
+
+
+def fwd(q, k, v, m, seq_len=None, causal=True, return_state=False, out=None, workspace=None,
+        stream=None):
+    """cott_fwd.  ``seq_len``: None (s_b = N), a float, or a float32 ``[B]`` CUDA tensor.
+    Returns ``o`` or ``(o, state[B,H,d,d] fp32)``."""
+    _check_dev(q, k, v, m, seq_len if isinstance(seq_len, torch.Tensor) else None)
+    B, H, N, d = q.shape
+    dt = _dt(q)
+    o = torch.empty_like(q) if out is None else out
+    state = torch.empty((B, H, d, d), dtype=torch.float32, device=q.device) if return_state else None
+    ws, ws_bytes = _workspace(OP_FWD, dt, B, H, N, d, causal, q.device, workspace)
+    sp = _scale(m, seq_len)
+    rc = _load().cott_fwd(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
+                          state.data_ptr() if state is not None else None, B, H, N, d,
+                          int(bool(causal)), dt, ctypes.byref(sp), ws.data_ptr(), ws_bytes,
+                          _stream_ptr(stream))
+    if rc != 0:
+        raise CottError(rc, "cott_fwd")
+    return (o, state) if return_state else o
+
+
+def bwd(q, k, v, d_o, m, seq_len=None, causal=True, workspace=None, stream=None):
+    """cott_bwd.  Returns ``(dq, dk, dv, dm[H] fp32)``."""
+    _check_dev(q, k, v, d_o, m, seq_len if isinstance(seq_len, torch.Tensor) else None)
+    B, H, N, d = q.shape
+    dt = _dt(q)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(q), torch.empty_like(q)
+    dm = torch.empty((H,), dtype=torch.float32, device=q.device)
+    ws, ws_bytes = _workspace(OP_BWD, dt, B, H, N, d, causal, q.device, workspace)
+    sp = _scale(m, seq_len)
+    rc = _load().cott_bwd(q.data_ptr(), k.data_ptr(), v.data_ptr(), d_o.data_ptr(), dq.data_ptr(),
+                          dk.data_ptr(), dv.data_ptr(), dm.data_ptr(), B, H, N, d,
+                          int(bool(causal)), dt, ctypes.byref(sp), ws.data_ptr(), ws_bytes,
+                          _stream_ptr(stream))
+    if rc != 0:
+        raise CottError(rc, "cott_bwd")
+    return dq, dk, dv, dm
+
+
+def decode_step(q, k, v, state, m, seq_len, out=None, stream=None):
+    """cott_decode_step.  q,k,v ``[B,H,d]``; ``state`` fp32 ``[B,H,d,d]`` updated in place;
+    ``seq_len`` a float (>= 1) or a float32 ``[B]`` CUDA tensor.  Returns ``o [B,H,d]``."""
+    _check_dev(q, k, v, state, m, seq_len if isinstance(seq_len, torch.Tensor) else None)
+    B, H, d = q.shape
+    if state.dtype != torch.float32 or tuple(state.shape) != (B, H, d, d):
+        raise ValueError("state must be float32 [B,H,d,d]")
+    o = torch.empty_like(q) if out is None else out
+    sp = _scale(m, seq_len)
+    rc = _load().cott_decode_step(q.data_ptr(), k.data_ptr(), v.data_ptr(), state.data_ptr(),
+                                  o.data_ptr(), B, H, d, _dt(q), ctypes.byref(sp),
+                                  _stream_ptr(stream))
+    if rc != 0:
+        raise CottError(rc, "cott_decode_step")
+    return o
+
+
+def fwd_bwd_host(q, k, v, d_o, m, o, dq, dk, dv, dm, causal=True, seq_len=None, arena=None,
+                 stream=None):
+    """cott_fwd_bwd_host: every tensor argument is a HOST tensor (pinned for async copies);
+    ``arena`` is a uint8 CUDA tensor (allocated here if None).  Returns the arena."""
+    B, H, N, d = q.shape
+    dt = _dt(q)
+    lib = _load()
+    need = lib.cott_host_step_arena_bytes(dt, B, H, N, d, int(bool(causal)))
+    if need == _SIZE_MAX:
+        raise CottError(-2, "cott_host_step_arena_bytes")
+    if arena is None:
+        arena = torch.empty(need, dtype=torch.uint8, device="cuda")
+    rc = lib.cott_fwd_bwd_host(q.data_ptr(), k.data_ptr(), v.data_ptr(), d_o.data_ptr(),
+                               o.data_ptr(), dq.data_ptr(), dk.data_ptr(), dv.data_ptr(),
+                               dm.data_ptr(), m.data_ptr(),
+                               seq_len.data_ptr() if seq_len is not None else None, B, H, N, d,
+                               int(bool(causal)), dt, arena.data_ptr(), arena.numel(),
+                               _stream_ptr(stream))
+    if rc != 0:
+        raise CottError(rc, "cott_fwd_bwd_host")
+    return arena
+
+
+def last_async_status(workspace: torch.Tensor, stream=None) -> int:
+    return int(_load().cott_last_async_status(workspace.data_ptr(), _stream_ptr(stream)))

@@ -1,0 +1,338 @@
+// C-ABI entry points of libcott: argument validation, execution plan, workspace layout and
+// the launch sequences.  All arithmetic of the method runs in the kernels.
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+#include "cott_internal.h"
+
+namespace cott {
+
+static thread_local char g_cuda_error[256] = "";
+
+static cott_status cuda_fail(cudaError_t e, const char* where) {
+    snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s", where, cudaGetErrorString(e));
+    return COTT_ERR_CUDA;
+}
+#define COTT_CUDA(expr)                                          \
+    do {                                                         \
+        cudaError_t e__ = (expr);                                \
+        if (e__ != cudaSuccess) return cuda_fail(e__, #expr);    \
+    } while (0)
+
+static int env_int(const char* name, int dflt) {
+    const char* v = getenv(name);
+    return (v && *v) ? atoi(v) : dflt;
+}
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static size_t dtype_size(cott_dtype dt) { return dt == COTT_F32 ? 4 : 2; }
+
+struct Plan {
+    int path;      // 0 SIMT, 1 tensor core
+    int group;     // tokens per sequence group
+    int chunk;     // tokens per chunk inside a group
+    int n_groups;
+};
+
+// Sequence groups give sequence-level parallelism when B*H alone cannot fill the GPU:
+// halve the group until there are enough CTAs, but never below a floor that keeps the
+// per-group state traffic (d*d fp32) small against the group's own q,k,v,o bytes.
+static bool make_plan(int op, cott_dtype dt, int B, int H, int N, int d, int causal, Plan* p) {
+    (void)op; (void)causal;
+    if (B < 1 || H < 1 || N < 1) return false;
+    if (d != 32 && d != 64 && d != 128) return false;
+    if (dt != COTT_F32 && dt != COTT_BF16) return false;
+    p->path = 0;
+    p->chunk = 16;
+    const long BH = (long)B * H;
+    int group = 1024;
+    const int floor_group = 128;
+    while (group > floor_group && BH * ((N + group - 1) / group) < 4 * 148) group >>= 1;
+    const int forced = env_int("COTT_FORCE_GROUP", 0);
+    if (forced > 0) group = (forced + p->chunk - 1) / p->chunk * p->chunk;
+    if (group >= N) group = (N + p->chunk - 1) / p->chunk * p->chunk;
+    p->group = group;
+    p->n_groups = (N + group - 1) / group;
+    return true;
+}
+
+static size_t states_bytes(const Plan& p, int B, int H, int d) {
+    return align_up((size_t)B * H * p.n_groups * d * d * sizeof(float), 256);
+}
+
+static size_t workspace_bytes_impl(int op, const Plan& p, int B, int H, int d) {
+    size_t total = kWsHeaderBytes;
+    if (op == COTT_OP_FWD) total += states_bytes(p, B, H, d);
+    else if (op == COTT_OP_BWD)
+        total += 3 * states_bytes(p, B, H, d) + align_up((size_t)B * H * p.n_groups * 4, 256);
+    return total;
+}
+
+static cott_status check_scale(const cott_scale_params* sp) {
+    if (!sp || !sp->m) return COTT_ERR_INVALID_ARG;
+    return COTT_OK;
+}
+
+static WalkArgs base_walk(const cott_scale_params* sp, int H, int N, const Plan& p) {
+    WalkArgs w;
+    memset(&w, 0, sizeof(w));
+    w.m = sp->m; w.seq_len = sp->seq_len; w.seq_len_scalar = sp->seq_len_scalar;
+    w.H = H; w.N = N; w.group = p.group; w.n_groups = p.n_groups;
+    return w;
+}
+
+// One gradient / output stream through the generic walk: (optional) per-group partial
+// states, their scan, then the walk that produces rows.
+static cott_status run_stream(WalkArgs w, const Plan& p, int BH, int d, cott_dtype dt, int causal,
+                              float* states, float* total_out, cudaStream_t st) {
+    const bool single = causal && p.n_groups == 1;
+    if (single) {
+        w.init = nullptr; w.update = 1; w.write_out = 1;
+        w.final_state = total_out; w.final_grouped = 0;
+        COTT_CUDA(launch_walk_simt(w, BH, d, dt, st));
+        return COTT_OK;
+    }
+    WalkArgs a = w;  // phase A: partial state of every group, no rows
+    a.init = nullptr; a.update = 1; a.write_out = 0; a.out = nullptr; a.proj = nullptr;
+    a.epilogue = EPI_PLAIN; a.dm_partial = nullptr;
+    a.final_state = states; a.final_grouped = 1;
+    COTT_CUDA(launch_walk_simt(a, BH, d, dt, st));
+    const int mode = !causal ? SCAN_TOTAL : (w.reverse ? SCAN_SUFFIX : SCAN_PREFIX);
+    COTT_CUDA(launch_scan(states, total_out, BH, p.n_groups, d, mode, st));
+    w.init = states; w.update = causal ? 1 : 0; w.write_out = 1; w.final_state = nullptr;
+    COTT_CUDA(launch_walk_simt(w, BH, d, dt, st));
+    return COTT_OK;
+}
+
+static cott_status fwd_impl(const void* q, const void* k, const void* v, void* o, float* state_out,
+                            int B, int H, int N, int d, int causal, cott_dtype dt,
+                            const cott_scale_params* sp, void* ws, const Plan& p,
+                            cudaStream_t st) {
+    COTT_CUDA(cudaMemsetAsync(ws, 0, kWsHeaderBytes, st));
+    float* states = reinterpret_cast<float*>(static_cast<char*>(ws) + kWsHeaderBytes);
+    WalkArgs w = base_walk(sp, H, N, p);
+    w.x = q; w.a = k; w.bv = v; w.out = o;
+    w.mode_x = ROW_NORM; w.mode_a = ROW_NORM; w.mode_b = ROW_SCALE;
+    w.epilogue = EPI_PLAIN; w.reverse = 0;
+    return run_stream(w, p, B * H, d, dt, causal, states, state_out, st);
+}
+
+static cott_status bwd_impl(const void* q, const void* k, const void* v, const void* d_o, void* dq,
+                            void* dk, void* dv, float* dm, int B, int H, int N, int d, int causal,
+                            cott_dtype dt, const cott_scale_params* sp, void* ws, const Plan& p,
+                            cudaStream_t st) {
+    COTT_CUDA(cudaMemsetAsync(ws, 0, kWsHeaderBytes, st));
+    char* base = static_cast<char*>(ws) + kWsHeaderBytes;
+    const size_t sb = states_bytes(p, B, H, d);
+    float* st0 = reinterpret_cast<float*>(base);
+    float* st1 = reinterpret_cast<float*>(base + sb);
+    float* st2 = reinterpret_cast<float*>(base + 2 * sb);
+    float* dm_partial = reinterpret_cast<float*>(base + 3 * sb);
+    const int BH = B * H;
+    cott_status rc;
+    {   // dQ^_t = S_t dO_t : the forward walk with (dO, V', K^) in the roles of (Q, K, V)
+        WalkArgs w = base_walk(sp, H, N, p);
+        w.x = d_o; w.a = v; w.bv = k; w.proj = q; w.out = dq;
+        w.mode_x = ROW_RAW; w.mode_a = ROW_SCALE; w.mode_b = ROW_NORM;
+        w.epilogue = EPI_PROJ; w.reverse = 0;
+        if ((rc = run_stream(w, p, BH, d, dt, causal, st0, nullptr, st)) != COTT_OK) return rc;
+    }
+    {   // dK^_j = R_j v'_j : running sum of dO_t q^_t^T accumulated backward in time
+        WalkArgs w = base_walk(sp, H, N, p);
+        w.x = v; w.a = d_o; w.bv = q; w.proj = k; w.out = dk;
+        w.mode_x = ROW_SCALE; w.mode_a = ROW_RAW; w.mode_b = ROW_NORM;
+        w.epilogue = EPI_PROJ; w.reverse = 1;
+        if ((rc = run_stream(w, p, BH, d, dt, causal, st1, nullptr, st)) != COTT_OK) return rc;
+    }
+    {   // dV'_j = R_j^T k^_j, dV = c dV', and <dV', V> for dm
+        WalkArgs w = base_walk(sp, H, N, p);
+        w.x = k; w.a = q; w.bv = d_o; w.proj = v; w.out = dv;
+        w.mode_x = ROW_NORM; w.mode_a = ROW_NORM; w.mode_b = ROW_RAW;
+        w.epilogue = EPI_DV; w.reverse = 1; w.dm_partial = dm_partial;
+        if ((rc = run_stream(w, p, BH, d, dt, causal, st2, nullptr, st)) != COTT_OK) return rc;
+    }
+    COTT_CUDA(launch_dm_finalize(dm_partial, dm, sp->m, sp->seq_len, sp->seq_len_scalar, B, H,
+                                 p.n_groups, N, st));
+    return COTT_OK;
+}
+
+}  // namespace cott
+
+using namespace cott;
+
+extern "C" {
+
+int cott_version(void) { return 100; }
+
+const char* cott_status_string(cott_status st) {
+    switch (st) {
+        case COTT_OK: return "ok";
+        case COTT_ERR_INVALID_ARG: return "invalid argument";
+        case COTT_ERR_UNSUPPORTED: return "unsupported shape, dtype or alignment";
+        case COTT_ERR_WORKSPACE: return "workspace missing or too small";
+        case COTT_ERR_CUDA: return "CUDA error";
+        case COTT_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+const char* cott_last_cuda_error(void) { return g_cuda_error; }
+
+size_t cott_workspace_bytes(int op, cott_dtype dt, int B, int H, int N, int d, int causal) {
+    if (op == COTT_OP_DECODE) return 0;
+    if (op != COTT_OP_FWD && op != COTT_OP_BWD) return (size_t)-1;
+    Plan p;
+    if (!make_plan(op, dt, B, H, N, d, causal, &p)) return (size_t)-1;
+    return workspace_bytes_impl(op, p, B, H, d);
+}
+
+cott_status cott_query_plan(int op, cott_dtype dt, int B, int H, int N, int d, int causal,
+                            int* path, int* group, int* chunk) {
+    Plan p;
+    if (op == COTT_OP_DECODE) { p.path = 0; p.group = 1; p.chunk = 1; }
+    else if (!make_plan(op, dt, B, H, N, d, causal, &p)) return COTT_ERR_UNSUPPORTED;
+    if (path) *path = p.path;
+    if (group) *group = p.group;
+    if (chunk) *chunk = p.chunk;
+    return COTT_OK;
+}
+
+cott_status cott_fwd(const void* q, const void* k, const void* v, void* o, float* state_out,
+                     int B, int H, int N, int d, int causal, cott_dtype dt,
+                     const cott_scale_params* sp, void* workspace, size_t workspace_bytes,
+                     void* stream) {
+    if (!q || !k || !v || !o || B < 1 || H < 1 || N < 1) return COTT_ERR_INVALID_ARG;
+    if (check_scale(sp) != COTT_OK) return COTT_ERR_INVALID_ARG;
+    if (o == q || o == k || o == v) return COTT_ERR_INVALID_ARG;
+    if (!sp->seq_len && sp->seq_len_scalar > 0.f && sp->seq_len_scalar < 1.f)
+        return COTT_ERR_INVALID_ARG;
+    Plan p;
+    if (!make_plan(COTT_OP_FWD, dt, B, H, N, d, causal, &p)) return COTT_ERR_UNSUPPORTED;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) ||
+        (state_out && !aligned16(state_out)))
+        return COTT_ERR_UNSUPPORTED;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
+        workspace_bytes < workspace_bytes_impl(COTT_OP_FWD, p, B, H, d))
+        return COTT_ERR_WORKSPACE;
+    return fwd_impl(q, k, v, o, state_out, B, H, N, d, causal, dt, sp, workspace, p,
+                    static_cast<cudaStream_t>(stream));
+}
+
+cott_status cott_bwd(const void* q, const void* k, const void* v, const void* d_o, void* dq,
+                     void* dk, void* dv, float* dm, int B, int H, int N, int d, int causal,
+                     cott_dtype dt, const cott_scale_params* sp, void* workspace,
+                     size_t workspace_bytes, void* stream) {
+    if (!q || !k || !v || !d_o || !dq || !dk || !dv || !dm || B < 1 || H < 1 || N < 1)
+        return COTT_ERR_INVALID_ARG;
+    if (check_scale(sp) != COTT_OK) return COTT_ERR_INVALID_ARG;
+    const void* ins[4] = {q, k, v, d_o};
+    void* outs[3] = {dq, dk, dv};
+    for (int i = 0; i < 3; ++i) {
+        for (int j = 0; j < 4; ++j)
+            if (outs[i] == ins[j]) return COTT_ERR_INVALID_ARG;
+        for (int j = i + 1; j < 3; ++j)
+            if (outs[i] == outs[j]) return COTT_ERR_INVALID_ARG;
+    }
+    if (!sp->seq_len && sp->seq_len_scalar > 0.f && sp->seq_len_scalar < 1.f)
+        return COTT_ERR_INVALID_ARG;
+    Plan p;
+    if (!make_plan(COTT_OP_BWD, dt, B, H, N, d, causal, &p)) return COTT_ERR_UNSUPPORTED;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(d_o) || !aligned16(dq) ||
+        !aligned16(dk) || !aligned16(dv))
+        return COTT_ERR_UNSUPPORTED;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
+        workspace_bytes < workspace_bytes_impl(COTT_OP_BWD, p, B, H, d))
+        return COTT_ERR_WORKSPACE;
+    return bwd_impl(q, k, v, d_o, dq, dk, dv, dm, B, H, N, d, causal, dt, sp, workspace, p,
+                    static_cast<cudaStream_t>(stream));
+}
+
+cott_status cott_decode_step(const void* q, const void* k, const void* v, float* state, void* o,
+                             int B, int H, int d, cott_dtype dt, const cott_scale_params* sp,
+                             void* stream) {
+    if (!q || !k || !v || !state || !o || B < 1 || H < 1) return COTT_ERR_INVALID_ARG;
+    if (check_scale(sp) != COTT_OK) return COTT_ERR_INVALID_ARG;
+    if (!sp->seq_len && !(sp->seq_len_scalar >= 1.f)) return COTT_ERR_INVALID_ARG;
+    if (d != 32 && d != 64 && d != 128) return COTT_ERR_UNSUPPORTED;
+    if (dt != COTT_F32 && dt != COTT_BF16) return COTT_ERR_UNSUPPORTED;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(state) || !aligned16(o))
+        return COTT_ERR_UNSUPPORTED;
+    COTT_CUDA(launch_decode(q, k, v, state, o, B, H, d, dt, sp->m, sp->seq_len,
+                            sp->seq_len_scalar, static_cast<cudaStream_t>(stream)));
+    return COTT_OK;
+}
+
+// Arena layout of the host-buffer training step: 8 tensors, m, seq_len, dm, workspace.
+static size_t host_step_layout(cott_dtype dt, int B, int H, int N, int d, int causal,
+                               size_t* tensor_bytes, size_t* ws_bytes) {
+    const size_t tb = align_up((size_t)B * H * N * d * dtype_size(dt), 256);
+    const size_t wf = cott_workspace_bytes(COTT_OP_FWD, dt, B, H, N, d, causal);
+    const size_t wb = cott_workspace_bytes(COTT_OP_BWD, dt, B, H, N, d, causal);
+    if (wf == (size_t)-1 || wb == (size_t)-1) return (size_t)-1;
+    const size_t wsz = align_up(wf > wb ? wf : wb, 256);
+    if (tensor_bytes) *tensor_bytes = tb;
+    if (ws_bytes) *ws_bytes = wsz;
+    return 8 * tb + 3 * align_up((size_t)(B > H ? B : H) * 4, 256) + wsz;
+}
+
+size_t cott_host_step_arena_bytes(cott_dtype dt, int B, int H, int N, int d, int causal) {
+    if (B < 1 || H < 1 || N < 1) return (size_t)-1;
+    return host_step_layout(dt, B, H, N, d, causal, nullptr, nullptr);
+}
+
+cott_status cott_fwd_bwd_host(const void* q_host, const void* k_host, const void* v_host,
+                              const void* d_o_host, void* o_host, void* dq_host, void* dk_host,
+                              void* dv_host, float* dm_host, const float* m_host,
+                              const float* seq_len_host, int B, int H, int N, int d, int causal,
+                              cott_dtype dt, void* arena, size_t arena_bytes, void* stream) {
+    if (!q_host || !k_host || !v_host || !d_o_host || !o_host || !dq_host || !dk_host ||
+        !dv_host || !dm_host || !m_host || B < 1 || H < 1 || N < 1)
+        return COTT_ERR_INVALID_ARG;
+    size_t tb = 0, wsz = 0;
+    const size_t need = host_step_layout(dt, B, H, N, d, causal, &tb, &wsz);
+    if (need == (size_t)-1) return COTT_ERR_UNSUPPORTED;
+    if (!arena || (reinterpret_cast<uintptr_t>(arena) & 255u) || arena_bytes < need)
+        return COTT_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char* p = static_cast<char*>(arena);
+    void* dq_ = p;           void* dk_ = p + tb;      void* dv_ = p + 2 * tb;
+    void* q_ = p + 3 * tb;   void* k_ = p + 4 * tb;   void* v_ = p + 5 * tb;
+    void* do_ = p + 6 * tb;  void* o_ = p + 7 * tb;
+    const size_t small = align_up((size_t)(B > H ? B : H) * 4, 256);
+    float* m_ = reinterpret_cast<float*>(p + 8 * tb);
+    float* sl_ = reinterpret_cast<float*>(p + 8 * tb + small);
+    float* dm_ = reinterpret_cast<float*>(p + 8 * tb + 2 * small);
+    void* ws = p + 8 * tb + 3 * small;
+    const size_t nbytes = (size_t)B * H * N * d * dtype_size(dt);
+    COTT_CUDA(cudaMemcpyAsync(q_, q_host, nbytes, cudaMemcpyHostToDevice, st));
+    COTT_CUDA(cudaMemcpyAsync(k_, k_host, nbytes, cudaMemcpyHostToDevice, st));
+    COTT_CUDA(cudaMemcpyAsync(v_, v_host, nbytes, cudaMemcpyHostToDevice, st));
+    COTT_CUDA(cudaMemcpyAsync(do_, d_o_host, nbytes, cudaMemcpyHostToDevice, st));
+    COTT_CUDA(cudaMemcpyAsync(m_, m_host, (size_t)H * 4, cudaMemcpyHostToDevice, st));
+    if (seq_len_host)
+        COTT_CUDA(cudaMemcpyAsync(sl_, seq_len_host, (size_t)B * 4, cudaMemcpyHostToDevice, st));
+    cott_scale_params sp;
+    sp.m = m_; sp.seq_len = seq_len_host ? sl_ : nullptr; sp.seq_len_scalar = 0.f;
+    cott_status rc = cott_fwd(q_, k_, v_, o_, nullptr, B, H, N, d, causal, dt, &sp, ws, wsz, stream);
+    if (rc != COTT_OK) return rc;
+    rc = cott_bwd(q_, k_, v_, do_, dq_, dk_, dv_, dm_, B, H, N, d, causal, dt, &sp, ws, wsz, stream);
+    if (rc != COTT_OK) return rc;
+    COTT_CUDA(cudaMemcpyAsync(o_host, o_, nbytes, cudaMemcpyDeviceToHost, st));
+    COTT_CUDA(cudaMemcpyAsync(dq_host, dq_, nbytes, cudaMemcpyDeviceToHost, st));
+    COTT_CUDA(cudaMemcpyAsync(dk_host, dk_, nbytes, cudaMemcpyDeviceToHost, st));
+    COTT_CUDA(cudaMemcpyAsync(dv_host, dv_, nbytes, cudaMemcpyDeviceToHost, st));
+    COTT_CUDA(cudaMemcpyAsync(dm_host, dm_, (size_t)H * 4, cudaMemcpyDeviceToHost, st));
+    return COTT_OK;
+}
+
+cott_status cott_last_async_status(const void* workspace, void* stream) {
+    if (!workspace) return COTT_ERR_INVALID_ARG;
+    COTT_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+    int word = 0;
+    COTT_CUDA(cudaMemcpy(&word, workspace, sizeof(int), cudaMemcpyDeviceToHost));
+    return word == 0 ? COTT_OK : COTT_ERR_TIMEOUT;
+}
+
+}  // extern "C"

@@ -1,0 +1,63 @@
+// Internal declarations shared by the translation units of libcott.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include "cott.h"
+
+namespace cott {
+
+constexpr float kEps = 1e-12f;        // denominator floor of the row normalisation (Eq. 2/3)
+constexpr int kWsHeaderBytes = 256;   // workspace header: word 0 = asynchronous status
+
+// Row treatment applied to a tile row when it is staged in shared memory.
+enum RowMode : int {
+    ROW_RAW = 0,    // use as is (dO)
+    ROW_NORM = 1,   // x / max(||x||, eps)     (Q and K, Eq. 3)
+    ROW_SCALE = 2   // c * x                   (V, Eq. 4)
+};
+
+// What happens to the rows a walk produces before they are stored.
+enum Epilogue : int {
+    EPI_PLAIN = 0,  // store
+    EPI_PROJ = 1,   // chain rule through the row normalisation of `proj` (raw q or k)
+    EPI_DV = 2      // multiply by c, and accumulate <row, proj row> for dm (proj = raw v)
+};
+
+// How the scan kernel combines the per-group partial states.
+enum ScanMode : int { SCAN_PREFIX = 0, SCAN_SUFFIX = 1, SCAN_TOTAL = 2 };
+
+// One pass of the generic running-sum walk (Eq. 7 / Eq. 8 with operand roles):
+//   state[a][b] += A_t[a] * Bv_t[b]   (if update)      out_t[b] = sum_a X_t[a] * state[a][b]
+// Forward:  (X,A,Bv) = (q^, k^, c v).      dQ^: (dO, c v, k^)  -> state is S^T.
+// dK^: (c v, dO, q^) reversed in time.     dV': (k^, q^, dO) reversed in time.
+struct WalkArgs {
+    const void* x; const void* a; const void* bv; const void* proj;
+    void* out;
+    const float* init;   // [BH, n_groups, d*d] or NULL (zero initial state)
+    float* final_state;  // NULL, or [BH, n_groups, d*d] (final_grouped) / [BH, d*d] (one group)
+    int final_grouped;
+    float* dm_partial;   // [BH, n_groups] or NULL
+    const float* m; const float* seq_len; float seq_len_scalar;
+    int H; int N; int group; int n_groups;
+    int mode_x, mode_a, mode_b;
+    int epilogue; int reverse; int update; int write_out;
+};
+
+cudaError_t launch_walk_simt(const WalkArgs& w, int BH, int d, cott_dtype dt, cudaStream_t st);
+cudaError_t launch_scan(float* states, float* total_out, int BH, int n_groups, int d, int mode,
+                        cudaStream_t st);
+cudaError_t launch_dm_finalize(const float* dm_partial, float* dm, const float* m,
+                               const float* seq_len, float seq_len_scalar, int B, int H,
+                               int n_groups, int N, cudaStream_t st);
+cudaError_t launch_decode(const void* q, const void* k, const void* v, float* state, void* o,
+                          int B, int H, int d, cott_dtype dt, const float* m,
+                          const float* seq_len, float seq_len_scalar, cudaStream_t st);
+
+// Stabilisation factor of Eq. 4 in fp32: c = exp(-sigmoid(m) * ln s).
+__device__ __forceinline__ float stab_factor(float m, float s) {
+    float sg = 1.0f / (1.0f + expf(-m));
+    return expf(-sg * logf(s));
+}
+
+}  // namespace cott

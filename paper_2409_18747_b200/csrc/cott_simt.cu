@@ -1,0 +1,385 @@
+// fp32 SIMT kernels: the running-sum walk (Eq. 7 / Eq. 8), the scan over per-group partial
+// states, the dm reduction and the recurrent decode step.  These serve fp32 I/O (tensor
+// cores in TF32 cannot meet the fp32 tolerance) and every shape the tensor-core kernels do
+// not cover.
+#include "cott_internal.h"
+
+namespace cott {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kTile = 16;  // tokens staged per shared-memory tile
+
+template <typename T> __device__ __forceinline__ void load4(const T* p, float (&f)[4]);
+template <> __device__ __forceinline__ void load4<float>(const float* p, float (&f)[4]) {
+    float4 v = *reinterpret_cast<const float4*>(p);
+    f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;
+}
+template <> __device__ __forceinline__ void load4<__nv_bfloat16>(const __nv_bfloat16* p,
+                                                                 float (&f)[4]) {
+    uint2 v = *reinterpret_cast<const uint2*>(p);
+    __nv_bfloat162 lo = *reinterpret_cast<__nv_bfloat162*>(&v.x);
+    __nv_bfloat162 hi = *reinterpret_cast<__nv_bfloat162*>(&v.y);
+    f[0] = __low2float(lo); f[1] = __high2float(lo);
+    f[2] = __low2float(hi); f[3] = __high2float(hi);
+}
+template <typename T> __device__ __forceinline__ float to_f32(T v);
+template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) {
+    return __bfloat162float(v);
+}
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) {
+    return __float2bfloat16_rn(v);
+}
+template <typename T> __device__ __forceinline__ void store4(T* p, const float (&f)[4]);
+template <> __device__ __forceinline__ void store4<float>(float* p, const float (&f)[4]) {
+    *reinterpret_cast<float4*>(p) = make_float4(f[0], f[1], f[2], f[3]);
+}
+template <> __device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16* p,
+                                                                  const float (&f)[4]) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(f[0], f[1]);
+    __nv_bfloat162 hi = __floats2bfloat162_rn(f[2], f[3]);
+    uint2 v;
+    v.x = *reinterpret_cast<uint32_t*>(&lo);
+    v.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(p) = v;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Stage rows [t0, t0+kTile) of one [N,D] slice as fp32; rows outside [lo,hi) become zero.
+template <int D, typename T>
+__device__ __forceinline__ void stage_tile(float (*dst)[D], const T* src, int t0, int lo, int hi,
+                                           int tid) {
+    constexpr int V4 = D / 4;
+    for (int i = tid; i < kTile * V4; i += kThreads) {
+        int r = i / V4, c4 = i % V4;
+        int t = t0 + r;
+        float f[4] = {0.f, 0.f, 0.f, 0.f};
+        if (t >= lo && t < hi) load4<T>(src + (size_t)t * D + c4 * 4, f);
+        *reinterpret_cast<float4*>(&dst[r][c4 * 4]) = make_float4(f[0], f[1], f[2], f[3]);
+    }
+}
+
+// Apply the row treatment to a staged tile: one warp per row.
+template <int D>
+__device__ __forceinline__ void treat_rows(float (*tile)[D], int mode, float c, int warp,
+                                           int lane) {
+    if (mode == ROW_RAW) return;
+    for (int r = warp; r < kTile; r += kThreads / 32) {
+        float scale = c;
+        if (mode == ROW_NORM) {
+            float ss = 0.f;
+            for (int e = lane; e < D; e += 32) ss += tile[r][e] * tile[r][e];
+            ss = warp_sum(ss);
+            scale = 1.0f / fmaxf(sqrtf(ss), kEps);
+        }
+        for (int e = lane; e < D; e += 32) tile[r][e] *= scale;
+    }
+}
+
+template <int D, typename T>
+__global__ void __launch_bounds__(kThreads) walk_kernel(WalkArgs w) {
+    constexpr int NSPLIT = kThreads / D;  // threads sharing one state column
+    constexpr int AR = D / NSPLIT;        // state rows owned by one thread
+    __shared__ __align__(16) float xs[kTile][D];
+    __shared__ __align__(16) float as[kTile][D];
+    __shared__ __align__(16) float bs[kTile][D];
+    __shared__ __align__(16) float part[kTile][NSPLIT][D];
+    __shared__ float dm_red[kThreads / 32];
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int g = blockIdx.x % w.n_groups;
+    const int bh = blockIdx.x / w.n_groups;
+    const int b = bh / w.H, h = bh % w.H;
+    const int lo = g * w.group;
+    const int hi = min(w.N, lo + w.group);
+    const size_t slice = (size_t)bh * w.N * D;
+    const T* X = static_cast<const T*>(w.x) + slice;
+    const T* A = static_cast<const T*>(w.a) + slice;
+    const T* Bv = static_cast<const T*>(w.bv) + slice;
+    const T* P = w.proj ? static_cast<const T*>(w.proj) + slice : nullptr;
+    T* O = w.out ? static_cast<T*>(w.out) + slice : nullptr;
+
+    const float s_b = w.seq_len ? w.seq_len[b]
+                                : (w.seq_len_scalar > 0.f ? w.seq_len_scalar : (float)w.N);
+    const float c = stab_factor(w.m[h], s_b);
+
+    const int col = tid % D, split = tid / D, a0 = split * AR;
+    float S[AR];
+    if (w.init) {
+        const float* src = w.init + ((size_t)bh * w.n_groups + g) * D * D;
+#pragma unroll
+        for (int i = 0; i < AR; ++i) S[i] = src[(size_t)(a0 + i) * D + col];
+    } else {
+#pragma unroll
+        for (int i = 0; i < AR; ++i) S[i] = 0.f;
+    }
+
+    float dm_acc = 0.f;
+    const int n_tiles = (hi - lo + kTile - 1) / kTile;
+    for (int it = 0; it < n_tiles; ++it) {
+        const int tile_idx = w.reverse ? (n_tiles - 1 - it) : it;
+        const int t0 = lo + tile_idx * kTile;
+        __syncthreads();  // previous tile fully consumed
+        stage_tile<D, T>(xs, X, t0, lo, hi, tid);
+        stage_tile<D, T>(as, A, t0, lo, hi, tid);
+        stage_tile<D, T>(bs, Bv, t0, lo, hi, tid);
+        __syncthreads();
+        treat_rows<D>(xs, w.mode_x, c, warp, lane);
+        treat_rows<D>(as, w.mode_a, c, warp, lane);
+        treat_rows<D>(bs, w.mode_b, c, warp, lane);
+        __syncthreads();
+
+        for (int s = 0; s < kTile; ++s) {
+            const int tt = w.reverse ? (kTile - 1 - s) : s;
+            const float bval = bs[tt][col];
+            float acc = 0.f;
+            if (w.update) {
+#pragma unroll
+                for (int i = 0; i < AR; i += 4) {
+                    float4 av = *reinterpret_cast<const float4*>(&as[tt][a0 + i]);
+                    S[i] += av.x * bval; S[i + 1] += av.y * bval;
+                    S[i + 2] += av.z * bval; S[i + 3] += av.w * bval;
+                }
+            }
+            if (w.write_out) {
+#pragma unroll
+                for (int i = 0; i < AR; i += 4) {
+                    float4 xv = *reinterpret_cast<const float4*>(&xs[tt][a0 + i]);
+                    acc += xv.x * S[i]; acc += xv.y * S[i + 1];
+                    acc += xv.z * S[i + 2]; acc += xv.w * S[i + 3];
+                }
+                part[tt][split][col] = acc;
+            }
+        }
+        if (!w.write_out) continue;
+        __syncthreads();
+        // Sum the partial read-outs of the NSPLIT thread groups into part[.][0][.].
+        for (int i = tid; i < kTile * D; i += kThreads) {
+            int r = i / D, e = i % D;
+            float v = part[r][0][e];
+#pragma unroll
+            for (int sp = 1; sp < NSPLIT; ++sp) v += part[r][sp][e];
+            part[r][0][e] = v;
+        }
+        if (w.epilogue != EPI_PLAIN) stage_tile<D, T>(xs, P, t0, lo, hi, tid);  // xs is dead now
+        __syncthreads();
+        // Epilogue: one warp per row.
+        for (int r = warp; r < kTile; r += kThreads / 32) {
+            const int t = t0 + r;
+            if (t >= hi) continue;
+            float* row = part[r][0];
+            if (w.epilogue == EPI_PROJ) {
+                // dx = (dx^ - x^ <x^, dx^>) / ||x||, or dx^ / eps on the clamped branch
+                float ss = 0.f, dp = 0.f;
+                for (int e = lane; e < D; e += 32) {
+                    ss += xs[r][e] * xs[r][e];
+                    dp += xs[r][e] * row[e];
+                }
+                ss = warp_sum(ss); dp = warp_sum(dp);
+                const float nrm = sqrtf(ss);
+                const float rinv = 1.0f / fmaxf(nrm, kEps);
+                const float coef = nrm > kEps ? dp * rinv * rinv : 0.f;  // <x^,dx^> * rinv
+                for (int e = lane; e < D; e += 32) row[e] = (row[e] - xs[r][e] * coef) * rinv;
+            } else if (w.epilogue == EPI_DV) {
+                float dp = 0.f;
+                for (int e = lane; e < D; e += 32) {
+                    dp += xs[r][e] * row[e];
+                    row[e] *= c;
+                }
+                dm_acc += dp;  // per-lane partial; summed over the warp at the end
+            }
+            __syncwarp();
+            for (int e4 = lane; e4 < D / 4; e4 += 32) {
+                float f[4] = {row[e4 * 4], row[e4 * 4 + 1], row[e4 * 4 + 2], row[e4 * 4 + 3]};
+                store4<T>(O + (size_t)t * D + e4 * 4, f);
+            }
+        }
+    }
+
+    if (w.final_state) {
+        float* dst = w.final_state +
+                     (w.final_grouped ? ((size_t)bh * w.n_groups + g) : (size_t)bh) * D * D;
+#pragma unroll
+        for (int i = 0; i < AR; ++i) dst[(size_t)(a0 + i) * D + col] = S[i];
+    }
+    if (w.dm_partial) {
+        dm_acc = warp_sum(dm_acc);
+        if (lane == 0) dm_red[warp] = dm_acc;
+        __syncthreads();
+        if (tid == 0) {
+            float t = 0.f;
+            for (int i = 0; i < kThreads / 32; ++i) t += dm_red[i];
+            w.dm_partial[(size_t)bh * w.n_groups + g] = t;
+        }
+    }
+}
+
+// Combine per-group partial states: exclusive prefix (forward), exclusive suffix (reverse
+// time) or the total written to every group.  One thread per state element.
+__global__ void scan_kernel(float* states, float* total_out, int n_groups, int dd, int mode) {
+    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    const int bh = blockIdx.y;
+    if (e >= dd) return;
+    float* base = states + (size_t)bh * n_groups * dd + e;
+    float run = 0.f;
+    if (mode == SCAN_PREFIX) {
+        for (int g = 0; g < n_groups; ++g) {
+            float v = base[(size_t)g * dd];
+            base[(size_t)g * dd] = run;
+            run += v;
+        }
+    } else if (mode == SCAN_SUFFIX) {
+        for (int g = n_groups - 1; g >= 0; --g) {
+            float v = base[(size_t)g * dd];
+            base[(size_t)g * dd] = run;
+            run += v;
+        }
+    } else {
+        for (int g = 0; g < n_groups; ++g) run += base[(size_t)g * dd];
+        for (int g = 0; g < n_groups; ++g) base[(size_t)g * dd] = run;
+    }
+    if (total_out) total_out[(size_t)bh * dd + e] = run;
+}
+
+// dm_h = sum_b dc/dm * <dV', V>_{b,h},  dc/dm = -ln(s_b) sigma(m_h)(1-sigma(m_h)) c_{b,h}.
+// Fixed summation order (deterministic).
+__global__ void dm_finalize_kernel(const float* dm_partial, float* dm, const float* m,
+                                   const float* seq_len, float seq_len_scalar, int B, int H,
+                                   int n_groups, int N) {
+    const int h = blockIdx.x * blockDim.x + threadIdx.x;
+    if (h >= H) return;
+    const float sg = 1.0f / (1.0f + expf(-m[h]));
+    float total = 0.f;
+    for (int b = 0; b < B; ++b) {
+        const float s_b = seq_len ? seq_len[b] : (seq_len_scalar > 0.f ? seq_len_scalar : (float)N);
+        const float ls = logf(s_b);
+        const float c = expf(-sg * ls);
+        float acc = 0.f;
+        for (int g = 0; g < n_groups; ++g) acc += dm_partial[((size_t)b * H + h) * n_groups + g];
+        total += acc * (-ls * sg * (1.0f - sg) * c);
+    }
+    dm[h] = total;
+}
+
+// Recurrent decode step (Eq. 8): one CTA per (b,h); the fp32 state streams through once with
+// 128-bit loads and stores, update and read-out fused.
+template <int D, typename T>
+__global__ void __launch_bounds__(kThreads) decode_kernel(const T* q, const T* k, const T* v,
+                                                          float* state, T* o, int H,
+                                                          const float* m, const float* seq_len,
+                                                          float seq_len_scalar) {
+    constexpr int V4 = D / 4;             // float4 per state row
+    constexpr int RG = kThreads / V4;     // rows covered per sweep
+    __shared__ float qh[D], kh[D], vp[D];
+    __shared__ __align__(16) float red[RG][D];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int bh = blockIdx.x, b = bh / H, h = bh % H;
+    const float s_b = seq_len ? seq_len[b] : seq_len_scalar;
+    const float c = stab_factor(m[h], s_b);
+    if (tid < D) {
+        qh[tid] = to_f32<T>(q[(size_t)bh * D + tid]);
+        kh[tid] = to_f32<T>(k[(size_t)bh * D + tid]);
+        vp[tid] = to_f32<T>(v[(size_t)bh * D + tid]) * c;
+    }
+    __syncthreads();
+    if (warp < 2) {
+        float* row = warp == 0 ? qh : kh;
+        float ss = 0.f;
+        for (int e = lane; e < D; e += 32) ss += row[e] * row[e];
+        ss = warp_sum(ss);
+        const float r = 1.0f / fmaxf(sqrtf(ss), kEps);
+        for (int e = lane; e < D; e += 32) row[e] *= r;
+    }
+    __syncthreads();
+    const int c4 = tid % V4, r0 = tid / V4;
+    const float4 vv = *reinterpret_cast<const float4*>(&vp[c4 * 4]);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float4* S = reinterpret_cast<float4*>(state + (size_t)bh * D * D);
+#pragma unroll 4
+    for (int a = r0; a < D; a += RG) {
+        float4 sv = S[(size_t)a * V4 + c4];
+        const float ka = kh[a], qa = qh[a];
+        sv.x += ka * vv.x; sv.y += ka * vv.y; sv.z += ka * vv.z; sv.w += ka * vv.w;
+        S[(size_t)a * V4 + c4] = sv;
+        acc.x += qa * sv.x; acc.y += qa * sv.y; acc.z += qa * sv.z; acc.w += qa * sv.w;
+    }
+    *reinterpret_cast<float4*>(&red[r0][c4 * 4]) = acc;
+    __syncthreads();
+    if (tid < D) {
+        float t = 0.f;
+#pragma unroll
+        for (int r = 0; r < RG; ++r) t += red[r][tid];
+        o[(size_t)bh * D + tid] = from_f32<T>(t);
+    }
+}
+
+template <typename T>
+cudaError_t launch_walk_t(const WalkArgs& w, int BH, int d, cudaStream_t st) {
+    dim3 grid((unsigned)(BH * w.n_groups));
+    switch (d) {
+        case 32: walk_kernel<32, T><<<grid, kThreads, 0, st>>>(w); break;
+        case 64: walk_kernel<64, T><<<grid, kThreads, 0, st>>>(w); break;
+        case 128: walk_kernel<128, T><<<grid, kThreads, 0, st>>>(w); break;
+        default: return cudaErrorInvalidValue;
+    }
+    return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t launch_decode_t(const void* q, const void* k, const void* v, float* state, void* o,
+                            int B, int H, int d, const float* m, const float* seq_len,
+                            float seq_len_scalar, cudaStream_t st) {
+    dim3 grid((unsigned)(B * H));
+    const T *qq = (const T*)q, *kk = (const T*)k, *vv = (const T*)v;
+    T* oo = (T*)o;
+    switch (d) {
+        case 32: decode_kernel<32, T><<<grid, kThreads, 0, st>>>(qq, kk, vv, state, oo, H, m, seq_len, seq_len_scalar); break;
+        case 64: decode_kernel<64, T><<<grid, kThreads, 0, st>>>(qq, kk, vv, state, oo, H, m, seq_len, seq_len_scalar); break;
+        case 128: decode_kernel<128, T><<<grid, kThreads, 0, st>>>(qq, kk, vv, state, oo, H, m, seq_len, seq_len_scalar); break;
+        default: return cudaErrorInvalidValue;
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_walk_simt(const WalkArgs& w, int BH, int d, cott_dtype dt, cudaStream_t st) {
+    return dt == COTT_F32 ? launch_walk_t<float>(w, BH, d, st)
+                          : launch_walk_t<__nv_bfloat16>(w, BH, d, st);
+}
+
+cudaError_t launch_scan(float* states, float* total_out, int BH, int n_groups, int d, int mode,
+                        cudaStream_t st) {
+    const int dd = d * d;
+    dim3 grid((unsigned)((dd + 255) / 256), (unsigned)BH);
+    scan_kernel<<<grid, 256, 0, st>>>(states, total_out, n_groups, dd, mode);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_dm_finalize(const float* dm_partial, float* dm, const float* m,
+                               const float* seq_len, float seq_len_scalar, int B, int H,
+                               int n_groups, int N, cudaStream_t st) {
+    dm_finalize_kernel<<<(H + 127) / 128, 128, 0, st>>>(dm_partial, dm, m, seq_len,
+                                                        seq_len_scalar, B, H, n_groups, N);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_decode(const void* q, const void* k, const void* v, float* state, void* o,
+                          int B, int H, int d, cott_dtype dt, const float* m,
+                          const float* seq_len, float seq_len_scalar, cudaStream_t st) {
+    return dt == COTT_F32
+               ? launch_decode_t<float>(q, k, v, state, o, B, H, d, m, seq_len, seq_len_scalar, st)
+               : launch_decode_t<__nv_bfloat16>(q, k, v, state, o, B, H, d, m, seq_len,
+                                                seq_len_scalar, st);
+}
+
+}  // namespace cott

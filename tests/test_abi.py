@@ -1,0 +1,100 @@
+"""The C-ABI library loads, exports every symbol the header declares, and its host-only
+entry points behave.  No kernel is launched here (runs without a GPU)."""
+import ctypes
+import os
+import re
+
+import paper_2409_18747_b200 as cott_pkg
+from paper_2409_18747_b200 import cott
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "cott.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(cott_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_exports_every_declared_symbol():
+    lib = ctypes.CDLL(cott_pkg.library_path())
+    names = declared_symbols()
+    assert {"cott_fwd", "cott_bwd", "cott_decode_step", "cott_workspace_bytes"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def test_version_and_status_strings():
+    lib = cott._load()
+    assert lib.cott_version() >= 100
+    seen = {lib.cott_status_string(s).decode() for s in (0, -1, -2, -3, -4, -5)}
+    assert len(seen) == 6
+
+
+def test_workspace_and_plan_are_host_only():
+    for (B, H, N, d, causal) in [(1, 2, 256, 32, True), (32, 12, 512, 64, False), (4, 16, 4096, 64, True),
+                                 (1, 16, 131072, 128, True)]:
+        for dt in (cott.F32, cott.BF16):
+            plan = cott.query_plan(cott.OP_FWD, dt, B, H, N, d, causal)
+            assert plan["group"] % plan["chunk"] == 0 and plan["group"] >= 1
+            wf = cott.workspace_bytes(cott.OP_FWD, dt, B, H, N, d, causal)
+            wb = cott.workspace_bytes(cott.OP_BWD, dt, B, H, N, d, causal)
+            assert 256 <= wf <= wb < (8 << 30)
+    assert cott.workspace_bytes(cott.OP_DECODE, cott.BF16, 64, 16, 1, 128, True) == 0
+    lib = cott._load()
+    assert lib.cott_workspace_bytes(0, cott.BF16, 1, 1, 16, 48, 1) == ctypes.c_size_t(-1).value  # d unsupported
+    assert lib.cott_workspace_bytes(0, cott.BF16, 0, 1, 16, 64, 1) == ctypes.c_size_t(-1).value
+
+
+def test_argument_validation_returns_before_any_launch():
+    lib = cott._load()
+    sp = cott._ScaleParams()
+    sp.m, sp.seq_len, sp.seq_len_scalar = 256, None, 0.0  # fake non-NULL address: never dereferenced on host
+    a = 4096  # fake 16-byte aligned device address; validation must fail before it is used
+    null = None
+    # NULL tensor
+    assert lib.cott_fwd(null, a, a, a, null, 1, 1, 16, 64, 1, cott.BF16, ctypes.byref(sp), a, 1 << 20, null) == -1
+    # NULL scale params / NULL m
+    assert lib.cott_fwd(a, a, a, a + 65536, null, 1, 1, 16, 64, 1, cott.BF16, None, a, 1 << 20, null) == -1
+    # output aliases an input
+    assert lib.cott_fwd(a, a, a, a, null, 1, 1, 16, 64, 1, cott.BF16, ctypes.byref(sp), a, 1 << 20, null) == -1
+    # unsupported head dimension, misaligned pointer
+    assert lib.cott_fwd(a, a, a, a + 65536, null, 1, 1, 16, 48, 1, cott.BF16, ctypes.byref(sp), a, 1 << 20, null) == -2
+    assert lib.cott_fwd(a + 2, a, a, a + 65536, null, 1, 1, 16, 64, 1, cott.BF16, ctypes.byref(sp), a, 1 << 20, null) == -2
+    # workspace missing / too small
+    assert lib.cott_fwd(a, a, a, a + 65536, null, 1, 1, 16, 64, 1, cott.BF16, ctypes.byref(sp), null, 0, null) == -3
+    assert lib.cott_fwd(a, a, a, a + 65536, null, 1, 1, 16, 64, 1, cott.BF16, ctypes.byref(sp), a, 8, null) == -3
+    # scaling base below one
+    sp.seq_len_scalar = 0.5
+    assert lib.cott_fwd(a, a, a, a + 65536, null, 1, 1, 16, 64, 1, cott.BF16, ctypes.byref(sp), a, 1 << 20, null) == -1
+    assert lib.cott_decode_step(a, a, a, a, a + 65536, 1, 1, 64, cott.BF16, ctypes.byref(sp), null) == -1
+    sp.seq_len_scalar = 0.0
+    assert lib.cott_decode_step(a, a, a, a, a + 65536, 1, 1, 64, cott.BF16, ctypes.byref(sp), null) == -1
+    # backward: NULL dm, aliasing outputs
+    assert lib.cott_bwd(a, a, a, a, a + 65536, a + 131072, a + 196608, null, 1, 1, 16, 64, 1, cott.BF16,
+                        ctypes.byref(sp), a, 1 << 24, null) == -1
+    assert lib.cott_bwd(a, a, a, a, a + 65536, a + 65536, a + 196608, a, 1, 1, 16, 64, 1, cott.BF16,
+                        ctypes.byref(sp), a, 1 << 24, null) == -1
+
+
+def test_missing_library_fails_loudly(monkeypatch):
+    monkeypatch.setattr(cott, "_lib", None)
+    monkeypatch.setattr(cott, "_LIB_PATH", "/nonexistent/libcott.so")
+    try:
+        cott._load()
+    except RuntimeError as e:
+        assert "no CPU" in str(e)
+    else:
+        raise AssertionError("loading a missing library must raise")
+
+
+def test_cpu_tensors_are_rejected():
+    import torch
+    q = torch.zeros((1, 1, 16, 64), dtype=torch.bfloat16)
+    m = torch.zeros((1,))
+    try:
+        cott.fwd(q, q, q, m)
+    except RuntimeError as e:
+        assert "CUDA" in str(e)
+    else:
+        raise AssertionError("CPU tensors must be rejected")

@@ -1,0 +1,308 @@
+"""GPU parity: libcott (through the C ABI) against the fp64 CPU oracle on the same seeded
+inputs.  Tolerances: fp32 I/O max relative error (floored, see _metrics) <= 1e-4; bf16 I/O
+normalised max error <= 1e-2; integer-valued index/mask cases bit-exact."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2409_18747_b200 as cott
+from paper_2409_18747_b200 import synth
+from _metrics import norm_max_err, rel_err_floor
+
+pytestmark = pytest.mark.gpu
+
+TOL_F32 = 1e-4
+TOL_BF16 = 1e-2
+
+
+def dev(x):
+    return x.cuda() if isinstance(x, torch.Tensor) else x
+
+
+def gate(x, ref, dtype):
+    if dtype == torch.float32:
+        e = rel_err_floor(x, ref)
+        assert e <= TOL_F32, f"fp32 relative error {e:.3e} > {TOL_F32}"
+    else:
+        e = norm_max_err(x, ref)
+        assert e <= TOL_BF16, f"bf16 normalised max error {e:.3e} > {TOL_BF16}"
+    return e
+
+
+def gate_dm(dm, ref, tol):
+    dm, ref = dm.double().cpu().numpy(), np.asarray(ref)
+    den = np.maximum(np.abs(ref), 0.1 * np.abs(ref).max())
+    e = float((np.abs(dm - ref) / den).max())
+    assert e <= tol, f"dm relative error {e:.3e} > {tol}"
+
+
+@pytest.fixture
+def force_group(monkeypatch):
+    def _set(g):
+        if g is None:
+            monkeypatch.delenv("COTT_FORCE_GROUP", raising=False)
+        else:
+            monkeypatch.setenv("COTT_FORCE_GROUP", str(g))
+    return _set
+
+
+# ------------------------------------------------------------------ the five workloads
+def test_config1_tiny_causal_fp32():
+    c = synth.make_config(1)
+    o = cott.fwd(dev(c["q"]), dev(c["k"]), dev(c["v"]), dev(c["m"]), causal=True)
+    ref = oracle.fwd_quadratic(c["q"], c["k"], c["v"], c["m"], None, True)
+    ref_rec, _ = oracle.fwd_recurrent(c["q"], c["k"], c["v"], c["m"], None)
+    np.testing.assert_allclose(ref_rec, ref, rtol=1e-11, atol=1e-12)
+    gate(o, ref, torch.float32)
+    # cosine similarity ignores row lengths: dividing out the lognormal factors changes nothing
+    qn = c["q"] / c["q"].norm(dim=-1, keepdim=True)
+    kn = c["k"] / c["k"].norm(dim=-1, keepdim=True)
+    o2 = cott.fwd(dev(qn), dev(kn), dev(c["v"]), dev(c["m"]), causal=True)
+    gate(o2, ref, torch.float32)
+
+
+def test_config2_bidirectional_bf16():
+    c = synth.make_config(2)
+    o, st = cott.fwd(dev(c["q"]), dev(c["k"]), dev(c["v"]), dev(c["m"]), causal=False, return_state=True)
+    ref, ref_state = oracle.fwd_bidir_assoc(c["q"], c["k"], c["v"], c["m"], None)
+    gate(o, ref, torch.bfloat16)
+    rows = [0, 1, 127, 128, 255, 256, 511]
+    ref_rows = oracle.fwd_rows(c["q"], c["k"], c["v"], c["m"], rows, None, False)  # the definition itself
+    gate(o[:, :, rows], ref_rows, torch.bfloat16)
+    assert norm_max_err(st, ref_state) <= 1e-5  # exported state = c K^^T V (fp32 accumulate)
+    sub = slice(0, 2)
+    ref_q = oracle.fwd_quadratic(c["q"][sub], c["k"][sub], c["v"][sub], c["m"], None, False)
+    gate(o[sub], ref_q, torch.bfloat16)
+
+
+def test_config3_causal_bf16_zero_keys():
+    c = synth.make_config(3)
+    o = cott.fwd(dev(c["q"]), dev(c["k"]), dev(c["v"]), dev(c["m"]), causal=True)
+    ref, _ = oracle.fwd_recurrent(c["q"], c["k"], c["v"], c["m"], None)
+    gate(o, ref, torch.bfloat16)
+    sub = slice(0, 1)
+    ref_q = oracle.fwd_quadratic(c["q"][sub], c["k"][sub], c["v"][sub], c["m"], None, True)
+    gate(o[sub], ref_q, torch.bfloat16)
+    # a zero key contributes nothing: replacing its value row by junk must not change a bit
+    v2 = c["v"].clone()
+    zero = (c["k"].float().abs().sum(-1) == 0)
+    v2[zero] = 1000.0
+    o2 = cott.fwd(dev(c["q"]), dev(c["k"]), dev(v2), dev(c["m"]), causal=True)
+    assert torch.equal(o2, o)
+
+
+def test_config4_causal_fwd_bwd_bf16():
+    c = synth.make_config(4)
+    q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
+    o = cott.fwd(q, k, v, m, causal=True)
+    dq, dk, dv, dm = cott.bwd(q, k, v, d_o, m, causal=True)
+    ref_o, _ = oracle.fwd_recurrent(c["q"], c["k"], c["v"], c["m"], None)
+    gate(o, ref_o, torch.bfloat16)
+    rq, rk, rv, rm = oracle.bwd_recurrent(c["q"], c["k"], c["v"], c["d_o"], c["m"], None)
+    gate(dq, rq, torch.bfloat16); gate(dk, rk, torch.bfloat16); gate(dv, rv, torch.bfloat16)
+    gate_dm(dm, rm, 1e-2)
+    # second route to dm:  dm_h = <dO,O>_h * (-ln s) sigma(1-sigma), from the oracle's forward
+    sg = 1.0 / (1.0 + np.exp(-c["m"].double().numpy()))
+    dm2 = (c["d_o"].double().numpy() * ref_o).sum(axis=(0, 2, 3)) * (-np.log(4096.0)) * sg * (1 - sg)
+    np.testing.assert_allclose(rm, dm2, rtol=1e-9)
+
+
+def test_config4_reduced_against_quadratic_definition():
+    c = synth.make_qkv(1, 2, 1024, 64, torch.bfloat16, 2004, with_do=True)
+    q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
+    dq, dk, dv, dm = cott.bwd(q, k, v, d_o, m, causal=True)
+    rq, rk, rv, rm = oracle.bwd_quadratic(c["q"], c["k"], c["v"], c["d_o"], c["m"], None, True)
+    gate(dq, rq, torch.bfloat16); gate(dk, rk, torch.bfloat16); gate(dv, rv, torch.bfloat16)
+    gate_dm(dm, rm, 1e-2)
+
+
+@pytest.mark.parametrize("N", synth.C5_SWEEP_N)
+def test_config5_long_causal_bf16(N):
+    c = synth.make_config(5, N=N)
+    o = cott.fwd(dev(c["q"]), dev(c["k"]), dev(c["v"]), dev(c["m"]), causal=True)
+    heads = slice(0, 16) if N <= 16384 else slice(3, 7)
+    ref, _ = oracle.fwd_recurrent(c["q"][:, heads], c["k"][:, heads], c["v"][:, heads], c["m"][heads], np.array([float(N)]))
+    e = gate(o[:, heads], ref, torch.bfloat16)
+    print(f"config5 N={N}: normalised max error {e:.3e}")
+    plan = cott.query_plan(cott.cott.OP_FWD, cott.cott.BF16, 1, 16, N, 128, True)
+    G, C = plan["group"], plan["chunk"]
+    rows = sorted({0, 1, C - 1, C, C + 1, G - 1, G, min(G + 1, N - 1), N // 2, N - 2, N - 1} |
+                  set(np.random.default_rng(N).integers(0, N, 245).tolist()))
+    rows = [r for r in rows if 0 <= r < N]
+    ref_rows = oracle.fwd_rows(c["q"], c["k"], c["v"], c["m"], rows, None, True)
+    den = np.abs(ref).max()
+    err = np.abs(o[:, :, rows].double().cpu().numpy() - ref_rows).max() / den
+    assert err <= TOL_BF16
+
+
+def test_config5_decode_after_prefill():
+    """B=64,H=16,d=128: prefill N=8192 through cott_fwd, then 1024 single-token steps.  The
+    oracle follows a seeded subset of 16 (b,h) pairs through all 8192+1024 tokens."""
+    cfg = synth.C5_DECODE
+    B, H, d, N, T = cfg["B"], cfg["H"], cfg["d"], cfg["prefill"], cfg["steps"]
+    g = torch.Generator(device="cuda"); g.manual_seed(1005)
+    q, k, v = (torch.randn((B, H, N, d), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+               for _ in range(3))
+    m = torch.randn((H,), generator=g, device="cuda", dtype=torch.float32)
+    o, state = cott.fwd(q, k, v, m, causal=True, return_state=True)
+    sq, sk, sv = synth.make_decode_steps(B, H, d, T, torch.bfloat16, 1006)
+    rng = np.random.default_rng(1007)
+    pairs = [(int(rng.integers(0, B)), int(rng.integers(0, H))) for _ in range(16)]
+    state0 = state.clone()
+    outs = []
+    dq_, dk_, dv_ = sq.cuda(), sk.cuda(), sv.cuda()
+    for t in range(T):
+        outs.append(cott.decode_step(dq_[t], dk_[t], dv_[t], state, m, float(N)))
+    outs = torch.stack(outs)  # [T,B,H,d]
+    for (b, h) in pairs:
+        qq = torch.cat([q[b, h].cpu(), sq[:, b, h]])[None, None]
+        kk = torch.cat([k[b, h].cpu(), sk[:, b, h]])[None, None]
+        vv = torch.cat([v[b, h].cpu(), sv[:, b, h]])[None, None]
+        mm = m[h:h + 1].cpu()
+        ref, ref_state = oracle.fwd_recurrent(qq, kk, vv, mm, np.array([float(N)]))
+        assert norm_max_err(o[b, h], ref[0, 0, :N]) <= TOL_BF16
+        assert norm_max_err(outs[:, b, h], ref[0, 0, N:]) <= TOL_BF16
+        _, ref_state0 = oracle.fwd_recurrent(qq[:, :, :N], kk[:, :, :N], vv[:, :, :N], mm, np.array([float(N)]))
+        assert norm_max_err(state0[b, h], ref_state0[0, 0]) <= 1e-5
+        assert norm_max_err(state[b, h], ref_state[0, 0]) <= 1e-5
+
+
+# ------------------------------------------------------------------ bit-exact index / mask logic
+@pytest.mark.parametrize("dtype,d", [(torch.bfloat16, 64), (torch.bfloat16, 128), (torch.float32, 32)])
+def test_exact_integer_boundaries(dtype, d, force_group):
+    dt = cott.cott.BF16 if dtype == torch.bfloat16 else cott.cott.F32
+    force_group(256)
+    plan = cott.query_plan(cott.cott.OP_FWD, dt, 1, 2, 4096, d, True)
+    G, C = plan["group"], plan["chunk"]
+    one = torch.tensor([1.0], device="cuda")
+    for N in sorted({1, 2, C - 1, C, C + 1, G - 1, G, G + 1, 2 * G, 3 * G + 5}):
+        c = synth.make_onehot_case(1, 2, N, d, dtype, 3000 + N)
+        for causal in (True, False):
+            o = cott.fwd(dev(c["q"]), dev(c["k"]), dev(c["v"]), dev(c["m"]), seq_len=one, causal=causal)
+            ref = oracle.fwd_quadratic(c["q"], c["k"], c["v"], c["m"], np.array([1.0]), causal)
+            assert np.array_equal(ref, np.round(ref))
+            assert np.array_equal(o.double().cpu().numpy(), ref), (N, causal)
+
+
+def test_staircase_shows_inclusive_diagonal():
+    N, d = 40, 32
+    q = torch.zeros((1, 1, N, d)); q[..., 0] = 1.0
+    k = q.clone()
+    v = torch.zeros((1, 1, N, d))
+    v[0, 0, torch.arange(N), torch.arange(N) % d] = 1.0
+    m = torch.zeros((1,))
+    o = cott.fwd(dev(q), dev(k), dev(v), dev(m), seq_len=1.0, causal=True).cpu()
+    expect = torch.cumsum(v, dim=2)  # token t sees itself: o_0 = e_0
+    assert torch.equal(o, expect)
+
+
+# ------------------------------------------------------------------ small shapes, every path
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("d", [32, 64, 128])
+@pytest.mark.parametrize("causal", [True, False])
+def test_forward_backward_small(dtype, d, causal, force_group):
+    force_group(64)  # several groups: exercises the partial-state scan
+    B, H, N = 2, 3, 203  # ragged: not a multiple of any tile
+    c = synth.make_qkv(B, H, N, d, dtype, 4000 + d, row_lognormal=True, with_do=True)
+    s = torch.tensor([float(N), 150.0])
+    args = [dev(c[x]) for x in ("q", "k", "v")]
+    o, st = cott.fwd(*args, dev(c["m"]), seq_len=dev(s), causal=causal, return_state=True)
+    ref = oracle.fwd_quadratic(c["q"], c["k"], c["v"], c["m"], s, causal)
+    gate(o, ref, dtype)
+    _, ref_state = oracle.fwd_bidir_assoc(c["q"], c["k"], c["v"], c["m"], s)
+    assert norm_max_err(st, ref_state) <= 1e-5
+    dq, dk, dv, dm = cott.bwd(*args, dev(c["d_o"]), dev(c["m"]), seq_len=dev(s), causal=causal)
+    rq, rk, rv, rm = oracle.bwd_quadratic(c["q"], c["k"], c["v"], c["d_o"], c["m"], s, causal)
+    gate(dq, rq, dtype); gate(dk, rk, dtype); gate(dv, rv, dtype)
+    gate_dm(dm, rm, 1e-4 if dtype == torch.float32 else 1e-2)
+
+
+def test_single_token_and_single_head():
+    c = synth.make_qkv(1, 1, 1, 64, torch.float32, 4100, with_do=True)
+    o = cott.fwd(dev(c["q"]), dev(c["k"]), dev(c["v"]), dev(c["m"]), causal=True)
+    ref = oracle.fwd_quadratic(c["q"], c["k"], c["v"], c["m"], None, True)  # o_0 = c (q^.k^) v_0
+    gate(o, ref, torch.float32)
+
+
+def test_zero_query_rows_and_clamped_gradient():
+    c = synth.make_qkv(1, 2, 50, 32, torch.float32, 4200, with_do=True)
+    c["q"][0, 0, 7] = 0.0
+    c["k"][0, 1, 9] = 0.0
+    args = [dev(c[x]) for x in ("q", "k", "v")]
+    o = cott.fwd(*args, dev(c["m"]), causal=True)
+    assert torch.equal(o[0, 0, 7], torch.zeros(32, device="cuda"))
+    dq, dk, dv, dm = cott.bwd(*args, dev(c["d_o"]), dev(c["m"]), causal=True)
+    rq, rk, rv, rm = oracle.bwd_quadratic(c["q"], c["k"], c["v"], c["d_o"], c["m"], None, True)
+    # clamped rows carry gradients of order 1e12: compare them relatively, the rest with the gate
+    np.testing.assert_allclose(dq[0, 0, 7].cpu().numpy(), rq[0, 0, 7], rtol=1e-4)
+    np.testing.assert_allclose(dk[0, 1, 9].cpu().numpy(), rk[0, 1, 9], rtol=1e-4)
+    mask = torch.ones((1, 2, 50), dtype=torch.bool); mask[0, 0, 7] = False
+    gate(dq.cpu()[mask], rq[mask.numpy()], torch.float32)
+    mask = torch.ones((1, 2, 50), dtype=torch.bool); mask[0, 1, 9] = False
+    gate(dk.cpu()[mask], rk[mask.numpy()], torch.float32)
+    gate(dv, rv, torch.float32)
+
+
+def test_causality_bitwise(force_group):
+    force_group(128)
+    c = synth.make_qkv(1, 2, 300, 64, torch.bfloat16, 4300)
+    o = cott.fwd(dev(c["q"]), dev(c["k"]), dev(c["v"]), dev(c["m"]), seq_len=300.0, causal=True)
+    c2 = {x: c[x].clone() for x in ("q", "k", "v")}
+    for x in c2.values():
+        x[:, :, 200:] = 3.0
+    o2 = cott.fwd(dev(c2["q"]), dev(c2["k"]), dev(c2["v"]), dev(c["m"]), seq_len=300.0, causal=True)
+    assert torch.equal(o[:, :, :200], o2[:, :, :200])  # later tokens cannot change earlier rows
+
+
+def test_run_to_run_determinism():
+    c = synth.make_config(4, B=1)
+    q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
+    a = cott.bwd(q, k, v, d_o, m, causal=True)
+    b = cott.bwd(q, k, v, d_o, m, causal=True)
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)
+
+
+# ------------------------------------------------------------------ decode step
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("d", [32, 64, 128])
+def test_decode_matches_longer_forward(dtype, d):
+    B, H, N, T = 2, 3, 70, 9
+    c = synth.make_qkv(B, H, N + T, d, dtype, 5000 + d)
+    q, k, v, m = (dev(c[x]) for x in ("q", "k", "v", "m"))
+    s = torch.tensor([100.0, 64.0], device="cuda")
+    full = oracle.fwd_quadratic(c["q"], c["k"], c["v"], c["m"], s.cpu(), True)
+    _, state = cott.fwd(q[:, :, :N].contiguous(), k[:, :, :N].contiguous(), v[:, :, :N].contiguous(), m,
+                        seq_len=s, causal=True, return_state=True)
+    saved = None
+    for t in range(N, N + T):
+        o = cott.decode_step(q[:, :, t].contiguous(), k[:, :, t].contiguous(), v[:, :, t].contiguous(), state, m, s)
+        gate(o, full[:, :, t], dtype)
+        if t == N + 3:
+            saved = state.clone()
+    # checkpoint / resume: restoring a saved state and replaying gives identical bits
+    resumed = saved.clone()
+    for t in range(N + 4, N + T):
+        o2 = cott.decode_step(q[:, :, t].contiguous(), k[:, :, t].contiguous(), v[:, :, t].contiguous(), resumed, m, s)
+    assert torch.equal(resumed, state) and torch.equal(o2, o)
+    _, ref_state = oracle.fwd_recurrent(c["q"], c["k"], c["v"], c["m"], s.cpu())
+    assert norm_max_err(state, ref_state) <= 1e-5
+
+
+# ------------------------------------------------------------------ host-buffer entry point
+def test_fwd_bwd_host_matches_device_calls():
+    c = synth.make_config(4, B=1, N=512)
+    host = {x: c[x].pin_memory() for x in ("q", "k", "v", "d_o", "m")}
+    outs = {x: torch.empty_like(c["q"]).pin_memory() for x in ("o", "dq", "dk", "dv")}
+    dm = torch.empty(16, dtype=torch.float32).pin_memory()
+    cott.fwd_bwd_host(host["q"], host["k"], host["v"], host["d_o"], host["m"], outs["o"], outs["dq"],
+                      outs["dk"], outs["dv"], dm, causal=True)
+    torch.cuda.synchronize()
+    q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
+    o = cott.fwd(q, k, v, m, causal=True)
+    dq, dk, dv, dm2 = cott.bwd(q, k, v, d_o, m, causal=True)
+    assert torch.equal(outs["o"], o.cpu()) and torch.equal(outs["dq"], dq.cpu())
+    assert torch.equal(outs["dk"], dk.cpu()) and torch.equal(outs["dv"], dv.cpu()) and torch.equal(dm, dm2.cpu())
