@@ -1,0 +1,367 @@
+#!/usr/bin/env python
+"""Benchmark of the libcott hot path.
+
+Default workload (the one the headline metric is quoted on): causal cosine attention
+forward + backward, bf16 I/O with fp32 state, B=4 H=16 N=4096 d=64, synthetic N(0,1)
+tensors.  A step is one cott_fwd followed by one cott_bwd over one batch.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload c4|c2|c3|c5:<N>|decode]
+
+Prints ONE JSON line.  `value` is tokens/s with inputs resident in HBM; `e2e` is the same
+metric through the host-buffer entry point (host<->device copies inside the timed region);
+`roofline` compares the dominant call with the HBM roofline; `cpu_baseline` times the fp64
+oracle on a bounded sample on the host cores.  With N > 1 (torchrun) every rank runs an
+independent replica of the workload (heads and batch items are independent: there is no
+data-path collective), and the time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "causal Cottention fwd+bwd tokens/s"
+L2_FLUSH_BYTES = 256 << 20  # larger than the 126 MB L2
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "source": "fallback"}
+
+
+WORKLOADS = {
+    "c4": dict(name="C4 causal fwd+bwd", B=4, H=16, N=4096, d=64, causal=True, bwd=True),
+    "c3": dict(name="C3 causal fwd", B=8, H=12, N=1024, d=64, causal=True, bwd=False),
+    "c2": dict(name="C2 bidirectional fwd", B=32, H=12, N=512, d=64, causal=False, bwd=False),
+}
+
+
+def get_workload(spec: str) -> dict:
+    if spec in WORKLOADS:
+        return dict(WORKLOADS[spec])
+    if spec.startswith("c5:"):
+        n = int(spec.split(":")[1])
+        return dict(name=f"C5 causal fwd N={n}", B=1, H=16, N=n, d=128, causal=True, bwd=False)
+    if spec == "decode":
+        return dict(name="C5 decode step", B=64, H=16, N=1, d=128, causal=True, bwd=False, decode=True)
+    raise SystemExit(f"unknown workload {spec}")
+
+
+def algorithmic_bytes(w: dict) -> dict:
+    """Bytes the method must move per step (bf16 I/O): forward reads q,k,v and writes o
+    (4 tensors), backward reads q,k,v,dO and writes dq,dk,dv (7 tensors); a decode step
+    reads and writes the fp32 state once."""
+    th = w["B"] * w["H"] * w["N"] * w["d"] * 2
+    if w.get("decode"):
+        st = w["B"] * w["H"] * w["d"] * w["d"] * 4
+        return {"fwd": 2 * st + 4 * w["B"] * w["H"] * w["d"] * 2, "bwd": 0}
+    return {"fwd": 4 * th, "bwd": 7 * th if w["bwd"] else 0}
+
+
+class ClockSampler:
+    """Samples nvidia-smi SM clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.proc = None
+        self.gpu_index = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def max_over_ranks(value: float, world: int) -> float:
+    """Max of a per-rank scalar (device time) over all ranks; identity for one rank."""
+    if world == 1:
+        return value
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device="cuda" if dist.get_backend() == "nccl" else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_tokens_per_s(tokens_per_rank_step: int, world: int, ms_per_step_max: float) -> float:
+    """Whole-job throughput: every rank processes its own replica batch (weak scaling)."""
+    return tokens_per_rank_step * world / (ms_per_step_max * 1e-3)
+
+
+# ----------------------------------------------------------------------------- CPU oracle arm
+def oracle_sample_step(w: dict, sample_heads: int):
+    """Returns (callable running the oracle once on the bounded sample, tokens it covers).
+    The sample keeps N and d and takes `sample_heads` heads of one batch item; tokens are
+    scaled by the fraction of (b,h) pairs covered."""
+    import torch
+    import oracle
+    from paper_2409_18747_b200 import synth
+    H = min(sample_heads, w["H"])
+    if w.get("decode"):
+        c = synth.make_qkv(1, H, 1, w["d"], torch.bfloat16, 99)
+        import numpy as np
+        state = np.zeros((1, H, w["d"], w["d"]))
+        run = lambda: oracle.decode_step(c["q"][:, :, 0], c["k"][:, :, 0], c["v"][:, :, 0], c["m"], 8192.0, state)
+        return run, w["B"] * (H / (w["B"] * w["H"])), f"decode step on {H} of {w['B'] * w['H']} (b,h) states"
+    c = synth.make_qkv(1, H, w["N"], w["d"], torch.bfloat16, 99, with_do=True)
+
+    def run():
+        oracle.fwd_quadratic(c["q"], c["k"], c["v"], c["m"], None, w["causal"])
+        if w["bwd"]:
+            oracle.bwd_quadratic(c["q"], c["k"], c["v"], c["d_o"], c["m"], None, w["causal"])
+    frac = H / (w["B"] * w["H"])
+    what = "fwd+bwd" if w["bwd"] else "fwd"
+    return run, w["B"] * w["N"] * frac, (f"fp64 quadratic definition {what} on {H} of {w['B'] * w['H']} (b,h) "
+                                         f"pairs at N={w['N']}, d={w['d']}")
+
+
+def run_reference(args, w):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    import oracle
+    # bounded sample: fewer (b,h) pairs per step when more steps are asked for, so the whole
+    # run stays within a few minutes (one pair at N=4096, d=64 is about 4 core-seconds)
+    heads = max(1, min(16, 48 // max(args.steps, 1)))
+    if w["N"] > 4096:
+        heads = 1
+    run, tokens, what = oracle_sample_step(w, heads)
+    for _ in range(max(1, min(args.warmup, 1))):
+        run()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        run()
+    dt = (time.perf_counter() - t0) / args.steps
+    value = tokens / dt
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w["name"], "B": w["B"], "H": w["H"], "N": w["N"], "d": w["d"]},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": min(oracle.num_threads(), heads), "kind": "oracle",
+                         "sample": what},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------- GPU arm
+def run_ours(args, w):
+    import torch
+    import paper_2409_18747_b200 as cott
+    from paper_2409_18747_b200 import synth
+
+    rank, world, local = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: libcott has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    peaks = load_peaks()
+    B, H, N, d = w["B"], w["H"], w["N"], w["d"]
+    dev = torch.device("cuda", local)
+    g = torch.Generator(device=dev); g.manual_seed(1004 + rank)
+    mk = lambda *shape: torch.randn(shape, generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    m = torch.randn((H,), generator=g, device=dev, dtype=torch.float32)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+    dt_code = cott.cott.BF16
+
+    if w.get("decode"):
+        q, k, v = mk(B, H, d), mk(B, H, d), mk(B, H, d)
+        state = torch.randn((B, H, d, d), generator=g, device=dev, dtype=torch.float32)
+        o = torch.empty_like(q)
+        fwd_call = lambda: cott.decode_step(q, k, v, state, m, 8192.0, out=o)
+        bwd_call = None
+        tokens_per_step = B
+    else:
+        q, k, v = mk(B, H, N, d), mk(B, H, N, d), mk(B, H, N, d)
+        d_o = mk(B, H, N, d) if w["bwd"] else None
+        o = torch.empty_like(q)
+        ws_f = torch.empty(cott.workspace_bytes(cott.cott.OP_FWD, dt_code, B, H, N, d, w["causal"]),
+                           dtype=torch.uint8, device=dev)
+        fwd_call = lambda: cott.fwd(q, k, v, m, causal=w["causal"], out=o, workspace=ws_f)
+        bwd_call = None
+        if w["bwd"]:
+            ws_b = torch.empty(cott.workspace_bytes(cott.cott.OP_BWD, dt_code, B, H, N, d, w["causal"]),
+                               dtype=torch.uint8, device=dev)
+            bwd_call = lambda: cott.bwd(q, k, v, d_o, m, causal=w["causal"], workspace=ws_b)
+        tokens_per_step = B * N
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed_steps(n_steps, record):
+        """Runs n_steps; returns per-step (fwd_ms, bwd_ms) lists measured with CUDA events on
+        the launching stream; L2 is flushed before every step (outside the timed spans)."""
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(n_steps)]
+        for i in range(n_steps):
+            flush.fill_(i & 0xFF)
+            ev[i][0].record(stream)
+            fwd_call()
+            ev[i][1].record(stream)
+            if bwd_call is not None:
+                bwd_call()
+            ev[i][2].record(stream)
+        torch.cuda.synchronize()
+        if not record:
+            return [], []
+        return ([e[0].elapsed_time(e[1]) for e in ev], [e[1].elapsed_time(e[2]) for e in ev])
+
+    timed_steps(max(args.warmup, 3), record=False)
+    sampler = ClockSampler(local)
+    barrier()
+    launches0 = cott.cott.launch_count()
+    sampler.start()
+    fwd_ms, bwd_ms = timed_steps(args.steps, record=True)
+    barrier()
+    clocks = sampler.stop()
+    launches = cott.cott.launch_count() - launches0
+    step_ms_local = (sum(fwd_ms) + sum(bwd_ms)) / args.steps
+    step_ms = max_over_ranks(step_ms_local, world)
+    value = aggregate_tokens_per_s(tokens_per_step, world, step_ms)
+
+    # ---- end to end: host buffers in, host buffers out, through cott_fwd_bwd_host
+    e2e = None
+    if w.get("bwd") and not w.get("decode"):
+        host_in = [t.cpu().pin_memory() for t in (q, k, v, d_o)]
+        host_m = m.cpu().pin_memory()
+        host_out = [torch.empty_like(host_in[0]).pin_memory() for _ in range(4)]
+        host_dm = torch.empty((H,), dtype=torch.float32).pin_memory()
+        arena = None
+        n_e2e = max(3, min(args.steps, 10))
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(n_e2e)]
+        for it in range(2 + n_e2e):
+            if it >= 2:
+                evs[it - 2][0].record(stream)
+            arena = cott.fwd_bwd_host(*host_in, host_m, *host_out, host_dm, causal=w["causal"], arena=arena)
+            if it >= 2:
+                evs[it - 2][1].record(stream)
+            torch.cuda.synchronize()
+        e2e_ms = max_over_ranks(sum(a.elapsed_time(b) for a, b in evs) / n_e2e, world)
+        nbytes = q.numel() * 2
+        e2e = {"value": aggregate_tokens_per_s(tokens_per_step, world, e2e_ms), "unit": "tokens/s",
+               "ms_per_step": e2e_ms, "h2d_bytes_per_step": 4 * nbytes + H * 4,
+               "d2h_bytes_per_step": 4 * nbytes + H * 4}
+
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank != 0:
+        return
+    ab = algorithmic_bytes(w)
+    dom = "bwd" if w.get("bwd") else "fwd"
+    dom_ms = statistics.mean(bwd_ms if dom == "bwd" else fwd_ms)
+    achieved = ab[dom] / (dom_ms * 1e-3) / 1e9
+    plan = cott.query_plan(cott.cott.OP_BWD if dom == "bwd" else cott.cott.OP_FWD, dt_code, B, H, max(N, 1), d,
+                           w["causal"]) if not w.get("decode") else {"path": 0, "group": 1, "chunk": 1}
+    roofline = {
+        "bound": "hbm", "kernel": f"cott_{dom} call ({'tcgen05' if plan['path'] == 1 else 'simt'} path)",
+        "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+        "peak_source": peaks["source"], "traffic": None, "algorithmic_bytes": ab[dom], "ms": dom_ms,
+        "frac_of_nominal_8TBs": achieved / 8000.0,
+    }
+    fwd_mean = statistics.mean(fwd_ms)
+    extra = {"fwd_ms": fwd_mean, "fwd_gbs": ab["fwd"] / (fwd_mean * 1e-3) / 1e9,
+             "fwd_frac": ab["fwd"] / (fwd_mean * 1e-3) / 1e9 / peaks["hbm_gbs"],
+             "step_frac": (ab["fwd"] + ab["bwd"]) / (step_ms_local * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    if bwd_ms:
+        extra["bwd_ms"] = statistics.mean(bwd_ms)
+
+    cpu = None
+    if world == 1 or rank == 0:
+        import oracle
+        n_pairs = 16 if N <= 4096 else 1
+        run, tokens, what = oracle_sample_step(w, n_pairs)
+        t0 = time.perf_counter(); run(); dt = time.perf_counter() - t0
+        cpu = {"value": tokens / dt, "unit": "tokens/s", "cores": min(oracle.num_threads(), n_pairs, H),
+               "kind": "oracle",
+               "sample": what, "seconds": dt}
+
+    line = {
+        "metric": METRIC if w.get("bwd") else f"{w['name']} tokens/s", "value": value, "unit": "tokens/s",
+        "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": step_ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w["name"], "B": B, "H": H, "N": N, "d": d, "causal": w["causal"],
+                   "io": "bf16, fp32 state and accumulators", "parallelism": f"replicas x{world}",
+                   "l2": "flushed between steps (256 MB write); working set also exceeds L2",
+                   "plan": plan},
+        "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+        "detail": extra,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c4")
+    args = ap.parse_args()
+    w = get_workload(args.workload)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -65,6 +65,9 @@ const char* cott_status_string(cott_status st);
 /* Text of the last CUDA error seen by this thread inside the library (static storage). */
 const char* cott_last_cuda_error(void);
 
+/* Number of kernels this process has launched through the library so far (all threads). */
+unsigned long long cott_launch_count(void);
+
 /*
  * Bytes of device scratch the given call needs (0 is possible).  `op` is a cott_op.
  * The workspace must be 256-byte aligned.  Returns (size_t)-1 for unsupported arguments.

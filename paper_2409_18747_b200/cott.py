@@ -54,6 +54,7 @@ def _load():
     lib.cott_status_string.restype = ctypes.c_char_p
     lib.cott_status_string.argtypes = [ci]
     lib.cott_last_cuda_error.restype = ctypes.c_char_p
+    lib.cott_launch_count.restype = ctypes.c_ulonglong
     lib.cott_workspace_bytes.restype = cs
     lib.cott_workspace_bytes.argtypes = [ci, ci, ci, ci, ci, ci, ci]
     lib.cott_query_plan.restype = ci
@@ -205,6 +206,10 @@ def fwd_bwd_host(q, k, v, d_o, m, o, dq, dk, dv, dm, causal=True, seq_len=None, 
     if rc != 0:
         raise CottError(rc, "cott_fwd_bwd_host")
     return arena
+
+
+def launch_count() -> int:
+    return int(_load().cott_launch_count())
 
 
 def last_async_status(workspace: torch.Tensor, stream=None) -> int:

@@ -3,11 +3,14 @@
 #include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
+#include <atomic>
 #include "cott_internal.h"
 
 namespace cott {
 
 static thread_local char g_cuda_error[256] = "";
+static std::atomic<unsigned long long> g_launches{0};
+void note_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
 
 static cott_status cuda_fail(cudaError_t e, const char* where) {
     snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s", where, cudaGetErrorString(e));
@@ -179,6 +182,8 @@ const char* cott_status_string(cott_status st) {
 }
 
 const char* cott_last_cuda_error(void) { return g_cuda_error; }
+
+unsigned long long cott_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 size_t cott_workspace_bytes(int op, cott_dtype dt, int B, int H, int N, int d, int causal) {
     if (op == COTT_OP_DECODE) return 0;

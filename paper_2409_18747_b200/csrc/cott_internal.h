@@ -54,6 +54,9 @@ cudaError_t launch_decode(const void* q, const void* k, const void* v, float* st
                           int B, int H, int d, cott_dtype dt, const float* m,
                           const float* seq_len, float seq_len_scalar, cudaStream_t st);
 
+// Counts kernel launches issued by this process (reported by cott_launch_count).
+void note_launch(int n = 1);
+
 // Stabilisation factor of Eq. 4 in fp32: c = exp(-sigmoid(m) * ln s).
 __device__ __forceinline__ float stab_factor(float m, float s) {
     float sg = 1.0f / (1.0f + expf(-m));

@@ -331,6 +331,7 @@ cudaError_t launch_walk_t(const WalkArgs& w, int BH, int d, cudaStream_t st) {
         case 128: walk_kernel<128, T><<<grid, kThreads, 0, st>>>(w); break;
         default: return cudaErrorInvalidValue;
     }
+    note_launch();
     return cudaGetLastError();
 }
 
@@ -347,6 +348,7 @@ cudaError_t launch_decode_t(const void* q, const void* k, const void* v, float* 
         case 128: decode_kernel<128, T><<<grid, kThreads, 0, st>>>(qq, kk, vv, state, oo, H, m, seq_len, seq_len_scalar); break;
         default: return cudaErrorInvalidValue;
     }
+    note_launch();
     return cudaGetLastError();
 }
 
@@ -362,6 +364,7 @@ cudaError_t launch_scan(float* states, float* total_out, int BH, int n_groups, i
     const int dd = d * d;
     dim3 grid((unsigned)((dd + 255) / 256), (unsigned)BH);
     scan_kernel<<<grid, 256, 0, st>>>(states, total_out, n_groups, dd, mode);
+    note_launch();
     return cudaGetLastError();
 }
 
@@ -370,6 +373,7 @@ cudaError_t launch_dm_finalize(const float* dm_partial, float* dm, const float* 
                                int n_groups, int N, cudaStream_t st) {
     dm_finalize_kernel<<<(H + 127) / 128, 128, 0, st>>>(dm_partial, dm, m, seq_len,
                                                         seq_len_scalar, B, H, n_groups, N);
+    note_launch();
     return cudaGetLastError();
 }
 
