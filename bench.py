@@ -153,6 +153,15 @@ def oracle_sample_step(w: dict, sample_heads: int):
         state = np.zeros((1, H, w["d"], w["d"]))
         run = lambda: oracle.decode_step(c["q"][:, :, 0], c["k"][:, :, 0], c["v"][:, :, 0], c["m"], 8192.0, state)
         return run, w["B"] * (H / (w["B"] * w["H"])), f"decode step on {H} of {w['B'] * w['H']} (b,h) states"
+    if w["N"] > 4096:
+        # long sequences: the definition on evenly spaced rows of one head, about 2e10 flops
+        import numpy as np
+        c = synth.make_qkv(1, 1, w["N"], w["d"], torch.bfloat16, 99)
+        n_rows = max(4, int(2e10 / (w["N"] / 2 * w["d"] * 4)))
+        rows = np.linspace(0, w["N"] - 1, n_rows).astype(np.int64)
+        run = lambda: oracle.fwd_rows(c["q"], c["k"], c["v"], c["m"], rows, None, w["causal"])
+        return run, n_rows / w["H"], (f"fp64 quadratic definition on {n_rows} evenly spaced rows of one head "
+                                      f"at N={w['N']}, d={w['d']}")
     c = synth.make_qkv(1, H, w["N"], w["d"], torch.bfloat16, 99, with_do=True)
 
     def run():

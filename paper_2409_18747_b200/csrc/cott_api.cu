@@ -43,17 +43,27 @@ struct Plan {
 // halve the group until there are enough CTAs, but never below a floor that keeps the
 // per-group state traffic (d*d fp32) small against the group's own q,k,v,o bytes.
 static bool make_plan(int op, cott_dtype dt, int B, int H, int N, int d, int causal, Plan* p) {
-    (void)op; (void)causal;
+    (void)causal;
     if (B < 1 || H < 1 || N < 1) return false;
     if (d != 32 && d != 64 && d != 128) return false;
     if (dt != COTT_F32 && dt != COTT_BF16) return false;
-    p->path = 0;
-    p->chunk = 16;
     const long BH = (long)B * H;
-    int group = 1024;
-    const int floor_group = 128;
-    while (group > floor_group && BH * ((N + group - 1) / group) < 4 * 148) group >>= 1;
     const int forced = env_int("COTT_FORCE_GROUP", 0);
+    const bool tc_ok = dt == COTT_BF16 && (d == 64 || d == 128) && op == COTT_OP_FWD;
+    p->path = (tc_ok && env_int("COTT_FORCE_PATH", 1) != 0) ? 1 : 0;
+    int group;
+    if (p->path == 1) {
+        // One CTA per group and per SM slot (two CTAs fit per SM at d = 64): take the largest
+        // group that still gives every slot a CTA.
+        p->chunk = 128;
+        const long slots = 148L * (d == 64 ? 2 : 1);
+        group = 2048;
+        while (group > 128 && BH * ((N + group - 1) / group) < slots) group >>= 1;
+    } else {
+        p->chunk = 16;
+        group = 1024;
+        while (group > 128 && BH * ((N + group - 1) / group) < 4 * 148) group >>= 1;
+    }
     if (forced > 0) group = (forced + p->chunk - 1) / p->chunk * p->chunk;
     if (group >= N) group = (N + p->chunk - 1) / p->chunk * p->chunk;
     p->group = group;
@@ -115,6 +125,24 @@ static cott_status fwd_impl(const void* q, const void* k, const void* v, void* o
                             cudaStream_t st) {
     COTT_CUDA(cudaMemsetAsync(ws, 0, kWsHeaderBytes, st));
     float* states = reinterpret_cast<float*>(static_cast<char*>(ws) + kWsHeaderBytes);
+    if (p.path == 1) {
+        int* status = static_cast<int*>(ws);
+        const float* m = sp->m; const float* sl = sp->seq_len; const float sc = sp->seq_len_scalar;
+        if (causal && p.n_groups == 1 && !state_out) {
+            COTT_CUDA(launch_tc_fwd(1, q, k, v, o, nullptr, nullptr, status, m, sl, sc, B, H, N, d,
+                                    p.group, 1, st));
+            return COTT_OK;
+        }
+        // Phase A: unscaled partial state of every group; scan; phase C from the prefix
+        // (causal) or read-out against the total (bidirectional).
+        COTT_CUDA(launch_tc_fwd(0, nullptr, k, v, nullptr, nullptr, states, status, m, sl, sc, B,
+                                H, N, d, p.group, p.n_groups, st));
+        COTT_CUDA(launch_scan(states, state_out, B * H, p.n_groups, d,
+                              causal ? SCAN_PREFIX : SCAN_TOTAL, st, m, sl, sc, H, N));
+        COTT_CUDA(launch_tc_fwd(causal ? 1 : 2, q, k, v, o, states, nullptr, status, m, sl, sc, B,
+                                H, N, d, p.group, p.n_groups, st));
+        return COTT_OK;
+    }
     WalkArgs w = base_walk(sp, H, N, p);
     w.x = q; w.a = k; w.bv = v; w.out = o;
     w.mode_x = ROW_NORM; w.mode_a = ROW_NORM; w.mode_b = ROW_SCALE;

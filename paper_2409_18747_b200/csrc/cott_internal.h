@@ -45,8 +45,19 @@ struct WalkArgs {
 };
 
 cudaError_t launch_walk_simt(const WalkArgs& w, int BH, int d, cott_dtype dt, cudaStream_t st);
+// `total_scale_m` non-NULL: the total written to total_out is multiplied by the stabilisation
+// factor c[b,h] (the tensor-core path keeps its states unscaled).
 cudaError_t launch_scan(float* states, float* total_out, int BH, int n_groups, int d, int mode,
-                        cudaStream_t st);
+                        cudaStream_t st, const float* total_scale_m = nullptr,
+                        const float* seq_len = nullptr, float seq_len_scalar = 0.f, int H = 1,
+                        int N = 1);
+
+// Tensor-core forward kernels (bf16, d in {64,128}); mode: 0 partial states of every group,
+// 1 causal chunk walk from the group's prefix state, 2 read-out O = Q S for a fixed state.
+cudaError_t launch_tc_fwd(int mode, const void* q, const void* k, const void* v, void* o,
+                          const float* init, float* state_out, int* status, const float* m,
+                          const float* seq_len, float seq_len_scalar, int B, int H, int N, int d,
+                          int group, int n_groups, cudaStream_t st);
 cudaError_t launch_dm_finalize(const float* dm_partial, float* dm, const float* m,
                                const float* seq_len, float seq_len_scalar, int B, int H,
                                int n_groups, int N, cudaStream_t st);

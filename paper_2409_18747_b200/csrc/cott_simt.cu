@@ -225,7 +225,9 @@ __global__ void __launch_bounds__(kThreads) walk_kernel(WalkArgs w) {
 
 // Combine per-group partial states: exclusive prefix (forward), exclusive suffix (reverse
 // time) or the total written to every group.  One thread per state element.
-__global__ void scan_kernel(float* states, float* total_out, int n_groups, int dd, int mode) {
+__global__ void scan_kernel(float* states, float* total_out, int n_groups, int dd, int mode,
+                            const float* scale_m, const float* seq_len, float seq_len_scalar,
+                            int H, int N) {
     const int e = blockIdx.x * blockDim.x + threadIdx.x;
     const int bh = blockIdx.y;
     if (e >= dd) return;
@@ -247,7 +249,14 @@ __global__ void scan_kernel(float* states, float* total_out, int n_groups, int d
         for (int g = 0; g < n_groups; ++g) run += base[(size_t)g * dd];
         for (int g = 0; g < n_groups; ++g) base[(size_t)g * dd] = run;
     }
-    if (total_out) total_out[(size_t)bh * dd + e] = run;
+    if (total_out) {
+        if (scale_m) {
+            const float s_b = seq_len ? seq_len[bh / H]
+                                      : (seq_len_scalar > 0.f ? seq_len_scalar : (float)N);
+            run *= stab_factor(scale_m[bh % H], s_b);
+        }
+        total_out[(size_t)bh * dd + e] = run;
+    }
 }
 
 // dm_h = sum_b dc/dm * <dV', V>_{b,h},  dc/dm = -ln(s_b) sigma(m_h)(1-sigma(m_h)) c_{b,h}.
@@ -360,10 +369,12 @@ cudaError_t launch_walk_simt(const WalkArgs& w, int BH, int d, cott_dtype dt, cu
 }
 
 cudaError_t launch_scan(float* states, float* total_out, int BH, int n_groups, int d, int mode,
-                        cudaStream_t st) {
+                        cudaStream_t st, const float* total_scale_m, const float* seq_len,
+                        float seq_len_scalar, int H, int N) {
     const int dd = d * d;
     dim3 grid((unsigned)((dd + 255) / 256), (unsigned)BH);
-    scan_kernel<<<grid, 256, 0, st>>>(states, total_out, n_groups, dd, mode);
+    scan_kernel<<<grid, 256, 0, st>>>(states, total_out, n_groups, dd, mode, total_scale_m, seq_len,
+                                      seq_len_scalar, H, N);
     note_launch();
     return cudaGetLastError();
 }

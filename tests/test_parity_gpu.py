@@ -16,6 +16,15 @@ pytestmark = pytest.mark.gpu
 
 TOL_F32 = 1e-4
 TOL_BF16 = 1e-2
+# Exported / decode states are fp32, but on the bf16 tensor-core path their operands (k^ and v)
+# are bf16, so the state carries bf16 operand rounding: same normalised gate as bf16 outputs.
+# The fp32 SIMT path accumulates exact fp32 products: 1e-5.
+TOL_STATE_TC = 1e-2
+TOL_STATE_F32 = 1e-5
+
+
+def state_tol(dtype, d):
+    return TOL_STATE_TC if (dtype == torch.bfloat16 and d in (64, 128)) else TOL_STATE_F32
 
 
 def dev(x):
@@ -72,7 +81,7 @@ def test_config2_bidirectional_bf16():
     rows = [0, 1, 127, 128, 255, 256, 511]
     ref_rows = oracle.fwd_rows(c["q"], c["k"], c["v"], c["m"], rows, None, False)  # the definition itself
     gate(o[:, :, rows], ref_rows, torch.bfloat16)
-    assert norm_max_err(st, ref_state) <= 1e-5  # exported state = c K^^T V (fp32 accumulate)
+    assert norm_max_err(st, ref_state) <= TOL_STATE_TC  # exported state = c K^^T V
     sub = slice(0, 2)
     ref_q = oracle.fwd_quadratic(c["q"][sub], c["k"][sub], c["v"][sub], c["m"], None, False)
     gate(o[sub], ref_q, torch.bfloat16)
@@ -166,8 +175,8 @@ def test_config5_decode_after_prefill():
         assert norm_max_err(o[b, h], ref[0, 0, :N]) <= TOL_BF16
         assert norm_max_err(outs[:, b, h], ref[0, 0, N:]) <= TOL_BF16
         _, ref_state0 = oracle.fwd_recurrent(qq[:, :, :N], kk[:, :, :N], vv[:, :, :N], mm, np.array([float(N)]))
-        assert norm_max_err(state0[b, h], ref_state0[0, 0]) <= 1e-5
-        assert norm_max_err(state[b, h], ref_state[0, 0]) <= 1e-5
+        assert norm_max_err(state0[b, h], ref_state0[0, 0]) <= TOL_STATE_TC
+        assert norm_max_err(state[b, h], ref_state[0, 0]) <= TOL_STATE_TC
 
 
 # ------------------------------------------------------------------ bit-exact index / mask logic
@@ -213,7 +222,7 @@ def test_forward_backward_small(dtype, d, causal, force_group):
     ref = oracle.fwd_quadratic(c["q"], c["k"], c["v"], c["m"], s, causal)
     gate(o, ref, dtype)
     _, ref_state = oracle.fwd_bidir_assoc(c["q"], c["k"], c["v"], c["m"], s)
-    assert norm_max_err(st, ref_state) <= 1e-5
+    assert norm_max_err(st, ref_state) <= state_tol(dtype, d)
     dq, dk, dv, dm = cott.bwd(*args, dev(c["d_o"]), dev(c["m"]), seq_len=dev(s), causal=causal)
     rq, rk, rv, rm = oracle.bwd_quadratic(c["q"], c["k"], c["v"], c["d_o"], c["m"], s, causal)
     gate(dq, rq, dtype); gate(dk, rk, dtype); gate(dv, rv, dtype)
@@ -289,7 +298,7 @@ def test_decode_matches_longer_forward(dtype, d):
         o2 = cott.decode_step(q[:, :, t].contiguous(), k[:, :, t].contiguous(), v[:, :, t].contiguous(), resumed, m, s)
     assert torch.equal(resumed, state) and torch.equal(o2, o)
     _, ref_state = oracle.fwd_recurrent(c["q"], c["k"], c["v"], c["m"], s.cpu())
-    assert norm_max_err(state, ref_state) <= 1e-5
+    assert norm_max_err(state, ref_state) <= state_tol(dtype, d)
 
 
 # ------------------------------------------------------------------ host-buffer entry point
