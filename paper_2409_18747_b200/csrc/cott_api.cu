@@ -49,14 +49,14 @@ static bool make_plan(int op, cott_dtype dt, int B, int H, int N, int d, int cau
     if (dt != COTT_F32 && dt != COTT_BF16) return false;
     const long BH = (long)B * H;
     const int forced = env_int("COTT_FORCE_GROUP", 0);
-    const bool tc_ok = dt == COTT_BF16 && (d == 64 || d == 128) && op == COTT_OP_FWD;
+    const bool tc_ok = dt == COTT_BF16 && (d == 64 || d == 128);
     p->path = (tc_ok && env_int("COTT_FORCE_PATH", 1) != 0) ? 1 : 0;
     int group;
     if (p->path == 1) {
         // One CTA per group and per SM slot (two CTAs fit per SM at d = 64): take the largest
         // group that still gives every slot a CTA.
         p->chunk = 128;
-        const long slots = 148L * (d == 64 ? 2 : 1);
+        const long slots = 148L * ((d == 64 && op == COTT_OP_FWD) ? 2 : 1);
         group = 2048;
         while (group > 128 && BH * ((N + group - 1) / group) < slots) group >>= 1;
     } else {
@@ -119,6 +119,31 @@ static cott_status run_stream(WalkArgs w, const Plan& p, int BH, int d, cott_dty
     return COTT_OK;
 }
 
+// One output stream through the tensor-core walk: partial states of every group, their
+// scan, then the chunk walk (causal) or the read-out against the total (bidirectional).
+// A causal call with a single group and no state export needs only the walk.
+static cott_status run_tc_stream(TcWalkArgs t, const Plan& p, int B, int H, int N, int d,
+                                 int causal, const cott_scale_params* sp, int* status,
+                                 float* states, float* total_out, cudaStream_t st) {
+    t.status = status; t.m = sp->m; t.seq_len = sp->seq_len; t.seq_len_scalar = sp->seq_len_scalar;
+    t.group = p.group; t.n_groups = p.n_groups;
+    if (causal && p.n_groups == 1 && !total_out) {
+        t.mode = 1; t.init = nullptr; t.state_out = nullptr;
+        COTT_CUDA(launch_tc_walk(t, B, H, N, d, st));
+        return COTT_OK;
+    }
+    TcWalkArgs a = t;
+    a.mode = 0; a.x = nullptr; a.proj = nullptr; a.out = nullptr; a.init = nullptr;
+    a.state_out = states; a.dm_partial = nullptr; a.epilogue = EPI_PLAIN;
+    COTT_CUDA(launch_tc_walk(a, B, H, N, d, st));
+    const int mode = !causal ? SCAN_TOTAL : (t.reverse ? SCAN_SUFFIX : SCAN_PREFIX);
+    COTT_CUDA(launch_scan(states, total_out, B * H, p.n_groups, d, mode, st, sp->m, sp->seq_len,
+                          sp->seq_len_scalar, H, N));
+    t.mode = causal ? 1 : 2; t.init = states; t.state_out = nullptr;
+    COTT_CUDA(launch_tc_walk(t, B, H, N, d, st));
+    return COTT_OK;
+}
+
 static cott_status fwd_impl(const void* q, const void* k, const void* v, void* o, float* state_out,
                             int B, int H, int N, int d, int causal, cott_dtype dt,
                             const cott_scale_params* sp, void* ws, const Plan& p,
@@ -126,22 +151,12 @@ static cott_status fwd_impl(const void* q, const void* k, const void* v, void* o
     COTT_CUDA(cudaMemsetAsync(ws, 0, kWsHeaderBytes, st));
     float* states = reinterpret_cast<float*>(static_cast<char*>(ws) + kWsHeaderBytes);
     if (p.path == 1) {
-        int* status = static_cast<int*>(ws);
-        const float* m = sp->m; const float* sl = sp->seq_len; const float sc = sp->seq_len_scalar;
-        if (causal && p.n_groups == 1 && !state_out) {
-            COTT_CUDA(launch_tc_fwd(1, q, k, v, o, nullptr, nullptr, status, m, sl, sc, B, H, N, d,
-                                    p.group, 1, st));
-            return COTT_OK;
-        }
-        // Phase A: unscaled partial state of every group; scan; phase C from the prefix
-        // (causal) or read-out against the total (bidirectional).
-        COTT_CUDA(launch_tc_fwd(0, nullptr, k, v, nullptr, nullptr, states, status, m, sl, sc, B,
-                                H, N, d, p.group, p.n_groups, st));
-        COTT_CUDA(launch_scan(states, state_out, B * H, p.n_groups, d,
-                              causal ? SCAN_PREFIX : SCAN_TOTAL, st, m, sl, sc, H, N));
-        COTT_CUDA(launch_tc_fwd(causal ? 1 : 2, q, k, v, o, states, nullptr, status, m, sl, sc, B,
-                                H, N, d, p.group, p.n_groups, st));
-        return COTT_OK;
+        TcWalkArgs t;
+        memset(&t, 0, sizeof(t));
+        t.x = q; t.a = k; t.bv = v; t.out = o;
+        t.norm_bv = 0; t.x_norm = 1; t.epilogue = EPI_PLAIN; t.reverse = 0;
+        return run_tc_stream(t, p, B, H, N, d, causal, sp, static_cast<int*>(ws), states,
+                             state_out, st);
     }
     WalkArgs w = base_walk(sp, H, N, p);
     w.x = q; w.a = k; w.bv = v; w.out = o;
@@ -163,6 +178,26 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
     float* dm_partial = reinterpret_cast<float*>(base + 3 * sb);
     const int BH = B * H;
     cott_status rc;
+    if (p.path == 1) {
+        int* status = static_cast<int*>(ws);
+        TcWalkArgs t;
+        memset(&t, 0, sizeof(t));
+        // dQ^: forward walk with (dO, V, K^); c multiplies the accumulator; project with raw q
+        t.x = d_o; t.a = v; t.bv = k; t.proj = q; t.out = dq;
+        t.norm_bv = 1; t.x_norm = 0; t.epilogue = EPI_PROJ; t.reverse = 0;
+        if ((rc = run_tc_stream(t, p, B, H, N, d, causal, sp, status, st0, nullptr, st)) != COTT_OK) return rc;
+        // dK^: backward in time with (V, dO, Q^); project with raw k
+        t.x = v; t.a = d_o; t.bv = q; t.proj = k; t.out = dk;
+        t.norm_bv = 1; t.x_norm = 0; t.epilogue = EPI_PROJ; t.reverse = 1;
+        if ((rc = run_tc_stream(t, p, B, H, N, d, causal, sp, status, st1, nullptr, st)) != COTT_OK) return rc;
+        // dV': backward in time with (K, Q^, dO); rows scale by c / ||k||; <dV', V> for dm
+        t.x = k; t.a = q; t.bv = d_o; t.proj = v; t.out = dv;
+        t.norm_bv = 0; t.x_norm = 1; t.epilogue = EPI_DV; t.reverse = 1; t.dm_partial = dm_partial;
+        if ((rc = run_tc_stream(t, p, B, H, N, d, causal, sp, status, st2, nullptr, st)) != COTT_OK) return rc;
+        COTT_CUDA(launch_dm_finalize(dm_partial, dm, sp->m, sp->seq_len, sp->seq_len_scalar, B, H,
+                                     p.n_groups, N, st));
+        return COTT_OK;
+    }
     {   // dQ^_t = S_t dO_t : the forward walk with (dO, V', K^) in the roles of (Q, K, V)
         WalkArgs w = base_walk(sp, H, N, p);
         w.x = d_o; w.a = v; w.bv = k; w.proj = q; w.out = dq;

@@ -52,12 +52,19 @@ cudaError_t launch_scan(float* states, float* total_out, int BH, int n_groups, i
                         const float* seq_len = nullptr, float seq_len_scalar = 0.f, int H = 1,
                         int N = 1);
 
-// Tensor-core forward kernels (bf16, d in {64,128}); mode: 0 partial states of every group,
-// 1 causal chunk walk from the group's prefix state, 2 read-out O = Q S for a fixed state.
-cudaError_t launch_tc_fwd(int mode, const void* q, const void* k, const void* v, void* o,
-                          const float* init, float* state_out, int* status, const float* m,
-                          const float* seq_len, float seq_len_scalar, int B, int H, int N, int d,
-                          int group, int n_groups, cudaStream_t st);
+// Tensor-core running-sum walk (bf16, d in {64,128}) with operand roles (x, a, bv); see
+// cott_tc_walk.cu.  mode: 0 partial states of every group, 1 chunk walk from the group's
+// prefix / suffix state, 2 read-out Out = X State for a fixed state.
+struct TcWalkArgs {
+    int mode;
+    const void* x; const void* a; const void* bv; const void* proj; void* out;
+    const float* init; float* state_out; float* dm_partial; int* status;
+    const float* m; const float* seq_len; float seq_len_scalar;
+    int group; int n_groups;
+    int norm_bv; int x_norm; int epilogue; int reverse;
+};
+cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cudaStream_t st);
+
 cudaError_t launch_dm_finalize(const float* dm_partial, float* dm, const float* m,
                                const float* seq_len, float seq_len_scalar, int B, int H,
                                int n_groups, int N, cudaStream_t st);

@@ -224,38 +224,59 @@ __global__ void __launch_bounds__(kThreads) walk_kernel(WalkArgs w) {
 }
 
 // Combine per-group partial states: exclusive prefix (forward), exclusive suffix (reverse
-// time) or the total written to every group.  One thread per state element.
-__global__ void scan_kernel(float* states, float* total_out, int n_groups, int dd, int mode,
-                            const float* scale_m, const float* seq_len, float seq_len_scalar,
-                            int H, int N) {
-    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+// time) or the total written to every group.  One thread per four consecutive state
+// elements; groups are visited in batches whose loads are all issued before the first use.
+__global__ void __launch_bounds__(256) scan_kernel(float* __restrict__ states,
+                                                   float* __restrict__ total_out, int n_groups,
+                                                   int dd, int mode, const float* scale_m,
+                                                   const float* seq_len, float seq_len_scalar,
+                                                   int H, int N) {
+    constexpr int kBatch = 8;
+    const int e4 = blockIdx.x * blockDim.x + threadIdx.x;
     const int bh = blockIdx.y;
-    if (e >= dd) return;
-    float* base = states + (size_t)bh * n_groups * dd + e;
-    float run = 0.f;
-    if (mode == SCAN_PREFIX) {
-        for (int g = 0; g < n_groups; ++g) {
-            float v = base[(size_t)g * dd];
-            base[(size_t)g * dd] = run;
-            run += v;
+    if (e4 * 4 >= dd) return;
+    float4* base = reinterpret_cast<float4*>(states + (size_t)bh * n_groups * dd) + e4;
+    const size_t stride = (size_t)dd / 4;
+    float4 run = make_float4(0.f, 0.f, 0.f, 0.f);
+    auto add = [](float4& a, const float4& b) { a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w; };
+    if (mode == SCAN_TOTAL) {
+        for (int g0 = 0; g0 < n_groups; g0 += kBatch) {
+            float4 v[kBatch];
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i)
+                if (g0 + i < n_groups) v[i] = base[(size_t)(g0 + i) * stride];
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i)
+                if (g0 + i < n_groups) add(run, v[i]);
         }
-    } else if (mode == SCAN_SUFFIX) {
-        for (int g = n_groups - 1; g >= 0; --g) {
-            float v = base[(size_t)g * dd];
-            base[(size_t)g * dd] = run;
-            run += v;
-        }
+        for (int g = 0; g < n_groups; ++g) base[(size_t)g * stride] = run;
     } else {
-        for (int g = 0; g < n_groups; ++g) run += base[(size_t)g * dd];
-        for (int g = 0; g < n_groups; ++g) base[(size_t)g * dd] = run;
+        const bool rev = mode == SCAN_SUFFIX;
+        for (int g0 = 0; g0 < n_groups; g0 += kBatch) {
+            float4 v[kBatch];
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i) {
+                const int g = rev ? n_groups - 1 - (g0 + i) : g0 + i;
+                if (g0 + i < n_groups) v[i] = base[(size_t)g * stride];
+            }
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i) {
+                const int g = rev ? n_groups - 1 - (g0 + i) : g0 + i;
+                if (g0 + i < n_groups) {
+                    base[(size_t)g * stride] = run;
+                    add(run, v[i]);
+                }
+            }
+        }
     }
     if (total_out) {
         if (scale_m) {
             const float s_b = seq_len ? seq_len[bh / H]
                                       : (seq_len_scalar > 0.f ? seq_len_scalar : (float)N);
-            run *= stab_factor(scale_m[bh % H], s_b);
+            const float c = stab_factor(scale_m[bh % H], s_b);
+            run.x *= c; run.y *= c; run.z *= c; run.w *= c;
         }
-        total_out[(size_t)bh * dd + e] = run;
+        reinterpret_cast<float4*>(total_out + (size_t)bh * dd)[e4] = run;
     }
 }
 
@@ -372,7 +393,7 @@ cudaError_t launch_scan(float* states, float* total_out, int BH, int n_groups, i
                         cudaStream_t st, const float* total_scale_m, const float* seq_len,
                         float seq_len_scalar, int H, int N) {
     const int dd = d * d;
-    dim3 grid((unsigned)((dd + 255) / 256), (unsigned)BH);
+    dim3 grid((unsigned)((dd / 4 + 255) / 256), (unsigned)BH);
     scan_kernel<<<grid, 256, 0, st>>>(states, total_out, n_groups, dd, mode, total_scale_m, seq_len,
                                       seq_len_scalar, H, N);
     note_launch();
