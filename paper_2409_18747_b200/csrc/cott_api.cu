@@ -53,10 +53,9 @@ static bool make_plan(int op, cott_dtype dt, int B, int H, int N, int d, int cau
     p->path = (tc_ok && env_int("COTT_FORCE_PATH", 1) != 0) ? 1 : 0;
     int group;
     if (p->path == 1) {
-        // One CTA per group and per SM slot (two CTAs fit per SM at d = 64): take the largest
-        // group that still gives every slot a CTA.
+        // One CTA per group and per SM: take the largest group that still gives every SM a CTA.
         p->chunk = 128;
-        const long slots = 148L * ((d == 64 && op == COTT_OP_FWD) ? 2 : 1);
+        const long slots = 148L;
         group = 2048;
         while (group > 128 && BH * ((N + group - 1) / group) < slots) group >>= 1;
     } else {

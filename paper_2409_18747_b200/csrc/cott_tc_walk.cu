@@ -26,7 +26,7 @@ using namespace sm100;
 namespace {
 
 constexpr int kChunk = 128;
-constexpr int kTcThreads = 128;
+constexpr int kTcThreads = 288;   // 8 row-worker warps + 1 control warp
 constexpr uint64_t kWaitTimeoutNs = 2000000000ull;  // 2 s: far above any legitimate wait
 
 struct TcWalkParams {
@@ -43,16 +43,23 @@ struct TcWalkParams {
 };
 
 template <int D> struct Smem {
+    static constexpr int kStages = (D == 128) ? 2 : 3;    // TMA ring depth
     static constexpr int kTile = kChunk * D * 2;          // one 128 x D bf16 tile
     static constexpr int kStage = 3 * kTile;              // X, A, Bv
     static constexpr int kSb = D * D * 2;                 // bf16 copy of the state
-    static constexpr int kOffSb = 2 * kStage;
-    static constexpr int kOffBar = kOffSb + kSb;          // full[2], mma, proj, tmem slot, dm scratch
+    static constexpr int kOffSb = kStages * kStage;
+    // Masked-score operand P~ (128 x 128 bf16): d = 128 reuses the X slot (same size, and X
+    // is dead by then); d = 64 has a buffer of its own.
+    static constexpr int kOffPt = kOffSb + kSb;
+    static constexpr int kPt = (D == 64) ? kChunk * kChunk * 2 : 0;
+    static constexpr int kOffBar = kOffPt + kPt;          // mbarriers, TMEM slot, abort flag
+    static constexpr int kOffRx = kOffBar + 160;          // rx[kStages][128] floats, dm scratch
+    static constexpr int kCtlBytes = 160 + kStages * 512 + 32;
     // d = 64 only, and only for launches whose epilogue needs a fourth tile: a dedicated
     // buffer behind everything else (d = 128 reuses the A slot instead).
-    static constexpr int kOffProj = (kOffBar + 128 + 1023) / 1024 * 1024;
+    static constexpr int kOffProj = (kOffBar + kCtlBytes + 1023) / 1024 * 1024;
     static constexpr int dyn_bytes(bool with_proj) {
-        return ((with_proj && D == 64) ? kOffProj + kTile : kOffBar + 128) + 1024;  // + align slack
+        return ((with_proj && D == 64) ? kOffProj + kTile : kOffBar + kCtlBytes) + 1024;  // + align slack
     }
 };
 
@@ -96,71 +103,67 @@ __device__ __forceinline__ void issue_atb(uint32_t tS, uint32_t a, uint32_t bv, 
                idesc, (kk > 0) || acc_first);
 }
 
-// Sum of squares of a 128-byte-swizzled tile row held by this thread.
-template <int D>
-__device__ __forceinline__ float row_sumsq(const uint8_t* tile, int row) {
+// Bounded wait that also gives up as soon as any thread of the CTA has given up.
+__device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = globaltimer_ns();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 15u) == 0) {
+            if (*abort_flag) return false;
+            if (globaltimer_ns() - t0 > kWaitTimeoutNs) { *abort_flag = 1; return false; }
+        }
+    }
+}
+
+__device__ __forceinline__ float sumsq8(const uint4& w) {
+    const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&w);
     float ss = 0.f;
 #pragma unroll
-    for (int ch = 0; ch < D / 8; ++ch) {
-        uint4 w = *reinterpret_cast<const uint4*>(tile + (ch >> 3) * 16384 + swz(row, ch & 7));
-        const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&w);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            float2 f = __bfloat1622float2(e[i]);
-            ss += f.x * f.x + f.y * f.y;
-        }
+    for (int i = 0; i < 4; ++i) {
+        float2 f = __bfloat1622float2(e[i]);
+        ss += f.x * f.x + f.y * f.y;
     }
     return ss;
 }
 
-// x^ = x / max(||x||, eps) on this thread's row, in place, rounded to bf16.
-template <int D>
-__device__ __forceinline__ void normalise_row_inplace(uint8_t* tile, int row) {
-    uint4 w[D / 8];
-    float ss = 0.f;
-#pragma unroll
-    for (int ch = 0; ch < D / 8; ++ch) {
-        w[ch] = *reinterpret_cast<const uint4*>(tile + (ch >> 3) * 16384 + swz(row, ch & 7));
-        const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&w[ch]);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            float2 f = __bfloat1622float2(e[i]);
-            ss += f.x * f.x + f.y * f.y;
-        }
-    }
-    const float r = 1.0f / fmaxf(sqrtf(ss), kEps);
-#pragma unroll
-    for (int ch = 0; ch < D / 8; ++ch) {
-        const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&w[ch]);
-        uint4 o;
-        uint32_t* ow = reinterpret_cast<uint32_t*>(&o);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            float2 f = __bfloat1622float2(e[i]);
-            ow[i] = pack_bf16(f.x * r, f.y * r);
-        }
-        *reinterpret_cast<uint4*>(tile + (ch >> 3) * 16384 + swz(row, ch & 7)) = o;
-    }
-}
-
 enum { MODE_STATE = 0, MODE_CAUSAL = 1, MODE_READOUT = 2 };
 
+// Thread roles: warps 0-7 are the row workers (norms, score masking, state and output
+// epilogues); warp 8 lane 0 is the control thread (TMA loads / stores and all tcgen05.mma).
+// The roles meet only through mbarriers, every wait bounded.
 template <int D, int MODE>
 __global__ void __launch_bounds__(kTcThreads, 1)
 tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmA,
                const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmP,
                const __grid_constant__ CUtensorMap tmO, TcWalkParams p) {
     using L = Smem<D>;
+    constexpr int NST = L::kStages;
     constexpr int NH = D / 64;                       // 64-column half tiles per row
-    constexpr uint32_t kTmemCols = (D == 128) ? 512 : 256;
-    constexpr uint32_t colS = 0, colO = D, colP = 2 * D;
+    constexpr uint32_t kTmemCols = 512;
+    constexpr uint32_t colS = 0, colP = D, colO0 = D + 128;   // O double-buffered: colO0, colO0 + D
+    constexpr int HW = D / 2;                        // accumulator columns per worker thread
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* gbase = smem_raw + (base - smem_u32(smem_raw));
-    const uint32_t bar_full0 = base + L::kOffBar, bar_full1 = bar_full0 + 8, bar_mma = bar_full0 + 16;
-    const uint32_t bar_proj = bar_full0 + 24, tmem_slot = bar_full0 + 32;
-    volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(gbase + L::kOffBar + 32);
-    float* dm_red = reinterpret_cast<float*>(gbase + L::kOffBar + 64);
+    const uint32_t bars = base + L::kOffBar;
+    // Barriers that a fast role could otherwise lap are arrays indexed by stage or by chunk
+    // parity, so a phase parity always names one chunk.
+    const uint32_t bar_full = bars;            // [NST] (<= 3) TMA landed
+    const uint32_t bar_a_ready = bars + 24;    // [NST] rows normalised (256 arrivals)
+    const uint32_t bar_p_full = bars + 48;     //       scores and X State done (commit)
+    const uint32_t bar_s_full = bars + 56;     // [2]   state update done (commit)
+    const uint32_t bar_pt_ready = bars + 72;   //       masked scores in shared memory (256)
+    const uint32_t bar_sb_ready = bars + 80;   //       bf16 state copy written (256)
+    const uint32_t bar_o_full = bars + 88;     // [2]   output accumulator complete (commit)
+    const uint32_t bar_o_free = bars + 104;    // [2]   output accumulator drained (256)
+    const uint32_t bar_proj = bars + 120;      //       epilogue tile landed
+    const uint32_t bar_o_staged = bars + 128;  // [2]   output rows staged (256)
+    const uint32_t tmem_slot = bars + 144;
+    volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(gbase + L::kOffBar + 144);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + L::kOffBar + 148);
+    float* rx_buf = reinterpret_cast<float*>(gbase + L::kOffRx);                 // [NST][128]
+    float* dm_red = reinterpret_cast<float*>(gbase + L::kOffRx + NST * 512);     // [8]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = blockIdx.x % p.n_groups, bh = blockIdx.x / p.n_groups;
@@ -169,16 +172,24 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     const int tok1 = min(p.N, tok0 + p.group);
     const int n_chunks = (tok1 - tok0 + kChunk - 1) / kChunk;
     const bool with_proj = (MODE != MODE_STATE) && (p.epilogue != EPI_PLAIN);
+    const bool is_ctrl = warp == 8;
 
-    if (warp == 0) {
+    if (warp == 8) {
         tmem_alloc(tmem_slot, kTmemCols);
         tmem_relinquish();
     }
     if (tid == 0) {
-        mbar_init(bar_full0, 1); mbar_init(bar_full1, 1); mbar_init(bar_mma, 1);
-        mbar_init(bar_proj, 1);
+        for (int i = 0; i < NST; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_a_ready + 8 * i, 256); }
+        mbar_init(bar_p_full, 1); mbar_init(bar_s_full, 1); mbar_init(bar_s_full + 8, 1);
+        mbar_init(bar_pt_ready, 256); mbar_init(bar_sb_ready, 256);
+        mbar_init(bar_o_full, 1); mbar_init(bar_o_full + 8, 1);
+        mbar_init(bar_o_free, 256); mbar_init(bar_o_free + 8, 256);
+        mbar_init(bar_proj, 1); mbar_init(bar_o_staged, 256); mbar_init(bar_o_staged + 8, 256);
+        *abort_flag = 0;
         mbar_fence_init();
         fence_proxy_async();
+    }
+    if (is_ctrl && lane == 0) {
         tma_prefetch_desc(&tmX); tma_prefetch_desc(&tmA); tma_prefetch_desc(&tmB);
         tma_prefetch_desc(&tmP); tma_prefetch_desc(&tmO);
     }
@@ -186,213 +197,289 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot_g;
-    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
 
     const float s_b = p.seq_len ? p.seq_len[b] : (p.seq_len_scalar > 0.f ? p.seq_len_scalar : (float)p.N);
     const float cfac = stab_factor(p.m[h], s_b);
 
-    // State row held by this thread: with M = 128 accumulator rows map to lanes one to one;
-    // with M = 64 row r sits in lane (r % 16) + 32 * (r / 16).
-    const bool owns_row = (D == 128) || (lane < 16);
-    const int srow = (D == 128) ? tid : warp * 16 + (lane & 15);
+    // Accumulator mapping of a worker thread: TMEM lane quadrant q, column half hf, row.
+    const int q = warp & 3, hf = (warp >> 2) & 1;
+    const uint32_t lane_base = (uint32_t)(q * 32) << 16;
+    const int arow = q * 32 + lane;                   // row of P / Out held by this thread
+    // State rows: M = 128 maps row r to lane r; M = 64 maps row r to lane (r%16) + 32*(r/16).
+    const bool owns_srow = (D == 128) || (lane < 16);
+    const int srow = (D == 128) ? arow : q * 16 + (lane & 15);
     const uint32_t sb = base + L::kOffSb;
 
-    bool has_state = false;
-    if (p.init != nullptr) {
-        // Load the group's initial state into TMEM (fp32) and its bf16 copy into shared memory.
+    auto stage_x = [&](int s) { return base + s * L::kStage; };
+    auto stage_a = [&](int s) { return base + s * L::kStage + L::kTile; };
+    auto stage_b = [&](int s) { return base + s * L::kStage + 2 * L::kTile; };
+    auto stage_pt = [&](int s) { return (D == 128) ? stage_x(s) : base + L::kOffPt; };
+    auto chunk_row = [&](int c) { return tok0 + (p.reverse ? (n_chunks - 1 - c) : c) * kChunk; };
+
+    // bf16 copy of this thread's HW state columns into the MN-major state tile.
+    auto write_sb = [&](const uint32_t (&r)[32], int c0) {
+#pragma unroll
+        for (int i = 0; i < 32; i += 8) {
+            uint4 w;
+            w.x = pack_bf16(__uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+            w.y = pack_bf16(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+            w.z = pack_bf16(__uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
+            w.w = pack_bf16(__uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
+            const int col = c0 + i;
+            const uint32_t off = (col >> 6) * (D * 128u) + swz(srow, (col & 63) >> 3);
+            *reinterpret_cast<uint4*>(gbase + L::kOffSb + off) = w;
+        }
+    };
+
+    const bool init_state = p.init != nullptr;
+    if (init_state && !is_ctrl) {
+        // Initial state of the group: fp32 into TMEM, bf16 copy into shared memory.
         const float* src = p.init + ((size_t)bh * p.n_groups + g) * D * D + (size_t)srow * D;
 #pragma unroll
-        for (int c0 = 0; c0 < D; c0 += 32) {
+        for (int c0 = hf * HW; c0 < (hf + 1) * HW; c0 += 32) {
             uint32_t r[32];
 #pragma unroll
             for (int i = 0; i < 32; i += 4) {
-                float4 v = owns_row ? *reinterpret_cast<const float4*>(src + c0 + i)
-                                    : make_float4(0.f, 0.f, 0.f, 0.f);
+                float4 v = owns_srow ? *reinterpret_cast<const float4*>(src + c0 + i)
+                                     : make_float4(0.f, 0.f, 0.f, 0.f);
                 r[i] = __float_as_uint(v.x); r[i + 1] = __float_as_uint(v.y);
                 r[i + 2] = __float_as_uint(v.z); r[i + 3] = __float_as_uint(v.w);
             }
             if (MODE == MODE_CAUSAL) tmem_st32(tmem + lane_base + colS + c0, r);
-            if (owns_row) {
-#pragma unroll
-                for (int i = 0; i < 32; i += 8) {
-                    uint4 w;
-                    w.x = pack_bf16(__uint_as_float(r[i]), __uint_as_float(r[i + 1]));
-                    w.y = pack_bf16(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
-                    w.z = pack_bf16(__uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
-                    w.w = pack_bf16(__uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
-                    const int col = c0 + i;  // first of 8 columns
-                    const uint32_t off = (col >> 6) * (D * 128u) + swz(srow, (col & 63) >> 3);
-                    *reinterpret_cast<uint4*>(gbase + L::kOffSb + off) = w;
-                }
-            }
+            if (owns_srow) write_sb(r, c0);
         }
         if (MODE == MODE_CAUSAL) tmem_wait_st();
         fence_proxy_async();
-        has_state = true;
     }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
 
-    bool failed = false;
-    uint32_t mma_phase = 0;
     float dm_acc = 0.f;
-    auto stage_x = [&](int s) { return base + s * L::kStage; };
-    auto stage_a = [&](int s) { return base + s * L::kStage + L::kTile; };
-    auto stage_b = [&](int s) { return base + s * L::kStage + 2 * L::kTile; };
-    // Chunk visited at step c (time runs backward when p.reverse).
-    auto chunk_row = [&](int c) { return tok0 + (p.reverse ? (n_chunks - 1 - c) : c) * kChunk; };
 
-    auto issue_loads = [&](int c) {
-        const int s = c & 1;
-        const uint32_t bar = s ? bar_full1 : bar_full0;
-        const int row = chunk_row(c);
-        constexpr uint32_t n_tiles = (MODE == MODE_STATE) ? 2 : (MODE == MODE_CAUSAL ? 3 : 1);
-        mbar_expect_tx(bar, n_tiles * L::kTile);
+    if (is_ctrl) {
+        // ------------------------------------------------------------------ control thread
+        if (lane == 0 && n_chunks > 0) {
+            bool alive = true;
+            auto issue_loads = [&](int c) {
+                const int s = c % NST;
+                const uint32_t bar = bar_full + 8 * s;
+                const int row = chunk_row(c);
+                constexpr uint32_t n_tiles = (MODE == MODE_STATE) ? 2 : (MODE == MODE_CAUSAL ? 3 : 1);
+                mbar_expect_tx(bar, n_tiles * L::kTile);
 #pragma unroll
-        for (int hh = 0; hh < NH; ++hh) {
-            if (MODE != MODE_STATE) tma_load_3d(stage_x(s) + hh * 16384, &tmX, bar, hh * 64, row, bh);
+                for (int hh = 0; hh < NH; ++hh) {
+                    if (MODE != MODE_STATE) tma_load_3d(stage_x(s) + hh * 16384, &tmX, bar, hh * 64, row, bh);
+                    if (MODE != MODE_READOUT) {
+                        tma_load_3d(stage_a(s) + hh * 16384, &tmA, bar, hh * 64, row, bh);
+                        tma_load_3d(stage_b(s) + hh * 16384, &tmB, bar, hh * 64, row, bh);
+                    }
+                }
+            };
+            // First MMA batch of chunk c: scores, X State (needs the previous chunk's state
+            // copy and a drained output buffer), state update.
+            auto batch1 = [&](int c) {
+                const int s = c % NST;
+                if (!wait_or_abort(bar_a_ready + 8 * s, (c / NST) & 1, abort_flag)) { alive = false; return; }
+                const bool acc = init_state || c > 0;
+                if (MODE != MODE_STATE) {
+                    if (MODE == MODE_CAUSAL && c >= 1 &&
+                        !wait_or_abort(bar_sb_ready, (c - 1) & 1, abort_flag)) { alive = false; return; }
+                    if (c >= 2 && !wait_or_abort(bar_o_free + 8 * (c & 1), ((c >> 1) & 1) ^ 1, abort_flag)) {
+                        alive = false; return;
+                    }
+                }
+                tc_fence_after();
+                const uint32_t tO = tmem + colO0 + (c & 1) * D;
+                if (MODE == MODE_CAUSAL) {
+                    issue_p<D>(tmem + colP, stage_x(s), stage_a(s));
+                    if (acc) issue_xs<D>(tO, stage_x(s), sb);
+                    tc_commit(bar_p_full);
+                    issue_atb<D>(tmem + colS, stage_a(s), stage_b(s), acc);
+                    tc_commit(bar_s_full + 8 * (c & 1));
+                } else if (MODE == MODE_STATE) {
+                    issue_atb<D>(tmem + colS, stage_a(s), stage_b(s), acc);
+                    tc_commit(bar_s_full + 8 * (c & 1));
+                } else {
+                    issue_xs<D>(tO, stage_x(s), sb);
+                    tc_commit(bar_o_full + 8 * (c & 1));
+                }
+            };
+            for (int c = 0; c < NST && c < n_chunks; ++c) issue_loads(c);
+            batch1(0);
+            for (int c = 0; c < n_chunks && alive; ++c) {
+                const int s = c % NST;
+                if (with_proj) {
+                    // d = 128: the A slot is free once the state update has read it.
+                    if (MODE == MODE_CAUSAL && D == 128 &&
+                        !wait_or_abort(bar_s_full + 8 * (c & 1), (c >> 1) & 1, abort_flag)) { alive = false; break; }
+                    const uint32_t proj_u = (D == 128) ? stage_a(s) : base + L::kOffProj;
+                    mbar_expect_tx(bar_proj, L::kTile);
+#pragma unroll
+                    for (int hh = 0; hh < NH; ++hh)
+                        tma_load_3d(proj_u + hh * 16384, &tmP, bar_proj, hh * 64, chunk_row(c), bh);
+                }
+                if (MODE == MODE_CAUSAL) {
+                    if (!wait_or_abort(bar_pt_ready, c & 1, abort_flag)) { alive = false; break; }
+                    tc_fence_after();
+                    issue_pb<D>(tmem + colO0 + (c & 1) * D, stage_pt(s), stage_b(s), init_state || c > 0);
+                    tc_commit(bar_o_full + 8 * (c & 1));
+                }
+                if (c + 1 < n_chunks) { batch1(c + 1); if (!alive) break; }
+                if (MODE != MODE_STATE) {
+                    if (!wait_or_abort(bar_o_staged + 8 * (c & 1), (c >> 1) & 1, abort_flag)) { alive = false; break; }
+#pragma unroll
+                    for (int hh = 0; hh < NH; ++hh)
+                        tma_store_3d(&tmO, stage_b(s) + hh * 16384, hh * 64, chunk_row(c), bh);
+                    tma_store_commit();
+                } else {
+                    if (!wait_or_abort(bar_s_full + 8 * (c & 1), (c >> 1) & 1, abort_flag)) { alive = false; break; }
+                }
+                if (c + NST < n_chunks) {
+                    if (MODE != MODE_STATE) tma_store_wait_read0();
+                    issue_loads(c + NST);
+                }
+            }
+            tma_store_wait_all0();
+        }
+    } else {
+        // ------------------------------------------------------------------ row workers
+        bool alive = n_chunks > 0;
+        // Norm-phase mapping: lanes l and l^16 share a row (two column halves).
+        const int nrow = warp * 16 + (lane & 15), nhalf = lane >> 4;
+        constexpr int NC = D / 16;                    // 16-byte chunks in half a row
+        auto tile_half_ptr = [&](uint8_t* tile, int j) {
+            const int ch = nhalf * NC + j;            // chunk index within the row
+            return tile + (ch >> 3) * 16384 + swz(nrow, ch & 7);
+        };
+        // Row norms of chunk c: the contraction-side operand is normalised in place; the X
+        // row scale (times c) is left in rx_buf[c&1] for the output epilogue.
+        auto norm_phase = [&](int c) {
+            const int s = c % NST;
+            if (!wait_or_abort(bar_full + 8 * s, (c / NST) & 1, abort_flag)) { alive = false; return; }
+            uint8_t* xs = gbase + s * L::kStage;
+            if (MODE != MODE_STATE) {
+                float rx = cfac;
+                if (p.x_norm) {
+                    float ss = 0.f;
+#pragma unroll
+                    for (int j = 0; j < NC; ++j)
+                        ss += sumsq8(*reinterpret_cast<const uint4*>(tile_half_ptr(xs, j)));
+                    ss += __shfl_xor_sync(0xffffffffu, ss, 16);
+                    rx = cfac / fmaxf(sqrtf(ss), kEps);
+                }
+                if (nhalf == 0) rx_buf[(c % NST) * 128 + nrow] = rx;
+            }
             if (MODE != MODE_READOUT) {
-                tma_load_3d(stage_a(s) + hh * 16384, &tmA, bar, hh * 64, row, bh);
-                tma_load_3d(stage_b(s) + hh * 16384, &tmB, bar, hh * 64, row, bh);
+                uint8_t* nt = xs + (p.norm_bv ? 2 : 1) * L::kTile;
+                uint4 w[NC];
+                float ss = 0.f;
+#pragma unroll
+                for (int j = 0; j < NC; ++j) {
+                    w[j] = *reinterpret_cast<const uint4*>(tile_half_ptr(nt, j));
+                    ss += sumsq8(w[j]);
+                }
+                ss += __shfl_xor_sync(0xffffffffu, ss, 16);
+                const float r = 1.0f / fmaxf(sqrtf(ss), kEps);
+#pragma unroll
+                for (int j = 0; j < NC; ++j) {
+                    const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&w[j]);
+                    uint4 o;
+                    uint32_t* ow = reinterpret_cast<uint32_t*>(&o);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        float2 f = __bfloat1622float2(e[i]);
+                        ow[i] = pack_bf16(f.x * r, f.y * r);
+                    }
+                    *reinterpret_cast<uint4*>(tile_half_ptr(nt, j)) = o;
+                }
+                fence_proxy_async();
             }
-        }
-    };
+            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_a_ready + 8 * s) : "memory");
+        };
+        auto arrive = [&](uint32_t bar) {
+            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+        };
 
-    if (tid == 0 && n_chunks > 0) issue_loads(0);
-
-    for (int c = 0; c < n_chunks; ++c) {
-        const int s = c & 1;
-        if (tid == 0 && c + 1 < n_chunks) {
-            tma_store_wait_read0();  // the store that read a slot of stage s^1 has drained
-            issue_loads(c + 1);
-        }
-        bool ok = mbar_wait(s ? bar_full1 : bar_full0, (uint32_t)((c >> 1) & 1), kWaitTimeoutNs);
-        if (__syncthreads_or(!ok)) { failed = true; break; }
-
-        uint8_t* xs = gbase + s * L::kStage;
-        uint8_t* as = xs + L::kTile;
-        uint8_t* bs = xs + 2 * L::kTile;
-        // Row scale of X (thread t owns token row t of the chunk), applied in the epilogue.
-        float rx = cfac;
-        if (MODE != MODE_STATE && p.x_norm) rx = cfac / fmaxf(sqrtf(row_sumsq<D>(xs, tid)), kEps);
-        if (MODE != MODE_READOUT) {
-            normalise_row_inplace<D>(p.norm_bv ? bs : as, tid);
-            fence_proxy_async();
-        }
-        tc_fence_before();
-        __syncthreads();
-
-        if (tid == 0) {
-            tc_fence_after();
+        if (alive) norm_phase(0);
+        for (int c = 0; c < n_chunks && alive; ++c) {
+            const int s = c % NST;
+            uint8_t* xs = gbase + s * L::kStage;
+            uint8_t* bs = xs + 2 * L::kTile;
+            uint8_t* pt = (D == 128) ? xs : gbase + L::kOffPt;
             if (MODE == MODE_CAUSAL) {
-                issue_p<D>(tmem + colP, stage_x(s), stage_a(s));
-                if (has_state) issue_xs<D>(tmem + colO, stage_x(s), sb);
-                issue_atb<D>(tmem + colS, stage_a(s), stage_b(s), has_state);
-            } else if (MODE == MODE_STATE) {
-                issue_atb<D>(tmem + colS, stage_a(s), stage_b(s), has_state);
-            } else {
-                issue_xs<D>(tmem + colO, stage_x(s), sb);
-            }
-            tc_commit(bar_mma);
-        }
-        ok = mbar_wait(bar_mma, mma_phase, kWaitTimeoutNs);
-        mma_phase ^= 1;
-        if (__syncthreads_or(!ok)) { failed = true; break; }
-        tc_fence_after();
-
-        // The tile the epilogue needs besides the accumulator (raw q, k or v rows): fetched
-        // now so that it lands while the scores are processed.  d = 128 reuses the A slot
-        // (both MMAs that read A have completed); d = 64 has a dedicated buffer.
-        uint8_t* proj = (D == 128) ? as : gbase + L::kOffProj;
-        const uint32_t proj_u = (D == 128) ? stage_a(s) : base + L::kOffProj;
-        if (with_proj && tid == 0) {
-            if (D == 64) tma_store_wait_read0();  // previous chunk's store out of this buffer
-            mbar_expect_tx(bar_proj, L::kTile);
-#pragma unroll
-            for (int hh = 0; hh < NH; ++hh)
-                tma_load_3d(proj_u + hh * 16384, &tmP, bar_proj, hh * 64, chunk_row(c), bh);
-        }
-
-        if (MODE == MODE_CAUSAL) {
-            // Masked scores -> bf16 operand in the X slot (X is dead: both MMAs that read it
-            // have completed).  Forward: row i keeps columns j <= i (the diagonal stays,
-            // Eq. 6); backward in time: columns j >= i.
-#pragma unroll
-            for (int c0 = 0; c0 < kChunk; c0 += 32) {
-                uint32_t r[32];
-                tmem_ld32(tmem + lane_base + colP + c0, r);
+                // Masked scores -> bf16 operand in the X slot (both MMAs that read X are done).
+                // Forward: row i keeps columns j <= i (diagonal kept, Eq. 6); backward in time:
+                // columns j >= i.
+                if (!wait_or_abort(bar_p_full, c & 1, abort_flag)) { alive = false; break; }
+                tc_fence_after();
+                uint32_t r0[32], r1[32];
+                tmem_ld32(tmem + lane_base + colP + hf * 64, r0);
+                tmem_ld32(tmem + lane_base + colP + hf * 64 + 32, r1);
                 tmem_wait_ld();
 #pragma unroll
-                for (int i = 0; i < 32; i += 8) {
-                    uint4 w;
-                    uint32_t* ww = reinterpret_cast<uint32_t*>(&w);
+                for (int part = 0; part < 2; ++part) {
+                    const uint32_t* r = part ? r1 : r0;
 #pragma unroll
-                    for (int j = 0; j < 8; j += 2) {
-                        const int col = c0 + i + j;
-                        const bool k0 = p.reverse ? (col >= tid) : (col <= tid);
-                        const bool k1 = p.reverse ? (col + 1 >= tid) : (col + 1 <= tid);
-                        ww[j >> 1] = pack_bf16(k0 ? __uint_as_float(r[i + j]) : 0.f,
-                                               k1 ? __uint_as_float(r[i + j + 1]) : 0.f);
-                    }
-                    const int col = c0 + i;
-                    *reinterpret_cast<uint4*>(xs + (col >> 6) * 16384 + swz(tid, (col & 63) >> 3)) = w;
-                }
-            }
-            // bf16 copy of the updated state for the next chunk's X State product.
-            if (c + 1 < n_chunks) {
+                    for (int i = 0; i < 32; i += 8) {
+                        uint4 w;
+                        uint32_t* ww = reinterpret_cast<uint32_t*>(&w);
 #pragma unroll
-                for (int c0 = 0; c0 < D; c0 += 32) {
-                    uint32_t r[32];
-                    tmem_ld32(tmem + lane_base + colS + c0, r);
-                    tmem_wait_ld();
-                    if (owns_row) {
-#pragma unroll
-                        for (int i = 0; i < 32; i += 8) {
-                            uint4 w;
-                            w.x = pack_bf16(__uint_as_float(r[i]), __uint_as_float(r[i + 1]));
-                            w.y = pack_bf16(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
-                            w.z = pack_bf16(__uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
-                            w.w = pack_bf16(__uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
-                            const int col = c0 + i;
-                            const uint32_t off = (col >> 6) * (D * 128u) + swz(srow, (col & 63) >> 3);
-                            *reinterpret_cast<uint4*>(gbase + L::kOffSb + off) = w;
+                        for (int j = 0; j < 8; j += 2) {
+                            const int col = hf * 64 + part * 32 + i + j;
+                            const bool k0 = p.reverse ? (col >= arow) : (col <= arow);
+                            const bool k1 = p.reverse ? (col + 1 >= arow) : (col + 1 <= arow);
+                            ww[j >> 1] = pack_bf16(k0 ? __uint_as_float(r[i + j]) : 0.f,
+                                                   k1 ? __uint_as_float(r[i + j + 1]) : 0.f);
                         }
+                        const int ch = (part * 32 + i) >> 3;   // chunk within this thread's half
+                        *reinterpret_cast<uint4*>(pt + hf * 16384 + swz(arow, ch)) = w;
                     }
                 }
+                fence_proxy_async();
+                tc_fence_before();
+                arrive(bar_pt_ready);
+                // bf16 copy of the updated state for the next chunk's X State product.
+                if (c + 1 < n_chunks) {
+                    if (!wait_or_abort(bar_s_full + 8 * (c & 1), (c >> 1) & 1, abort_flag)) { alive = false; break; }
+                    tc_fence_after();
+#pragma unroll
+                    for (int c0 = hf * HW; c0 < (hf + 1) * HW; c0 += 32) {
+                        uint32_t r[32];
+                        tmem_ld32(tmem + lane_base + colS + c0, r);
+                        tmem_wait_ld();
+                        if (owns_srow) write_sb(r, c0);
+                    }
+                    fence_proxy_async();
+                    tc_fence_before();
+                    arrive(bar_sb_ready);
+                }
             }
-            fence_proxy_async();
-            tc_fence_before();
-            __syncthreads();
-            if (tid == 0) {
-                tc_fence_after();
-                issue_pb<D>(tmem + colO, stage_x(s), stage_b(s), has_state);
-                tc_commit(bar_mma);
-            }
-            ok = mbar_wait(bar_mma, mma_phase, kWaitTimeoutNs);
-            mma_phase ^= 1;
-            if (__syncthreads_or(!ok)) { failed = true; break; }
-            tc_fence_after();
-        }
-        has_state = true;
+            if (c + 1 < n_chunks) { norm_phase(c + 1); if (!alive) break; }
+            if (MODE == MODE_STATE) continue;
 
-        if (MODE != MODE_STATE) {
-            uint8_t* stage_out = bs;
-            uint32_t stage_out_u = stage_b(s);
+            // ---- output epilogue of chunk c
+            if (!wait_or_abort(bar_o_full + 8 * (c & 1), (c >> 1) & 1, abort_flag)) { alive = false; break; }
+            tc_fence_after();
+            const uint32_t tO = tmem + lane_base + colO0 + (c & 1) * D;
+            const float rx = rx_buf[(c % NST) * 128 + arow];
             float coef = 0.f, rp = 1.f;
+            const uint8_t* proj = (D == 128) ? (xs + L::kTile) : (gbase + L::kOffProj);
             if (with_proj) {
-                ok = mbar_wait(bar_proj, (uint32_t)(c & 1), kWaitTimeoutNs);
-                if (__syncthreads_or(!ok)) { failed = true; break; }
-                stage_out = proj; stage_out_u = proj_u;
-                // First pass over the accumulator row: <p, g> and ||p||^2.
+                if (!wait_or_abort(bar_proj, c & 1, abort_flag)) { alive = false; break; }
+                // <p, acc> and ||p||^2 over the whole row (both column-half threads compute
+                // the same sums; the proj tile is read-only).
                 float ss = 0.f, dp = 0.f;
 #pragma unroll
                 for (int c0 = 0; c0 < D; c0 += 32) {
                     uint32_t r[32];
-                    tmem_ld32(tmem + lane_base + colO + c0, r);
+                    tmem_ld32(tO + c0, r);
                     tmem_wait_ld();
 #pragma unroll
                     for (int i = 0; i < 32; i += 8) {
                         const int col = c0 + i;
                         uint4 w = *reinterpret_cast<const uint4*>(proj + (col >> 6) * 16384 +
-                                                                  swz(tid, (col & 63) >> 3));
+                                                                  swz(arow, (col & 63) >> 3));
                         const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&w);
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
@@ -403,29 +490,29 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     }
                 }
                 if (p.epilogue == EPI_PROJ) {
-                    // g = rx * acc;  out = (g - p^ <p^, g>) / max(||p||, eps), clamped branch: g / eps
+                    // g = rx * acc;  out = (g - p^ <p^, g>) / max(||p||, eps); clamped branch: g / eps
                     const float nrm = sqrtf(ss);
                     rp = 1.0f / fmaxf(nrm, kEps);
                     coef = nrm > kEps ? dp * rx * rp * rp : 0.f;
-                } else {
-                    dm_acc += dp * rx / cfac;  // <dV', v> with dV' = (rx / c) * acc
+                } else if (hf == 0) {
+                    dm_acc += dp * rx / cfac;  // <dV', v> with dV' = (rx / c) * acc, once per row
                 }
             }
-            // Output rows: scale, (project,) round to bf16, stage, TMA store.
+            // This thread's HW columns: scale, (project,) round to bf16, stage in the Bv slot.
 #pragma unroll
-            for (int c0 = 0; c0 < D; c0 += 32) {
+            for (int c0 = hf * HW; c0 < (hf + 1) * HW; c0 += 32) {
                 uint32_t r[32];
-                tmem_ld32(tmem + lane_base + colO + c0, r);
+                tmem_ld32(tO + c0, r);
                 tmem_wait_ld();
 #pragma unroll
                 for (int i = 0; i < 32; i += 8) {
                     const int col = c0 + i;
-                    uint8_t* dst = stage_out + (col >> 6) * 16384 + swz(tid, (col & 63) >> 3);
+                    const uint32_t off = (col >> 6) * 16384 + swz(arow, (col & 63) >> 3);
                     float v[8];
 #pragma unroll
                     for (int j = 0; j < 8; ++j) v[j] = __uint_as_float(r[i + j]) * rx;
                     if (with_proj && p.epilogue == EPI_PROJ) {
-                        uint4 w = *reinterpret_cast<const uint4*>(dst);
+                        uint4 w = *reinterpret_cast<const uint4*>(proj + off);
                         const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&w);
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
@@ -437,60 +524,52 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     uint4 w;
                     w.x = pack_bf16(v[0], v[1]); w.y = pack_bf16(v[2], v[3]);
                     w.z = pack_bf16(v[4], v[5]); w.w = pack_bf16(v[6], v[7]);
-                    *reinterpret_cast<uint4*>(dst) = w;
+                    *reinterpret_cast<uint4*>(bs + off) = w;
                 }
             }
-            fence_proxy_async();
             tc_fence_before();
-            __syncthreads();
-            if (tid == 0) {
+            arrive(bar_o_free + 8 * (c & 1));
+            fence_proxy_async();
+            arrive(bar_o_staged + 8 * (c & 1));
+        }
+
+        if (MODE == MODE_STATE && alive && p.state_out != nullptr) {
+            // Partial state of this group, fp32, unscaled.
+            if (wait_or_abort(bar_s_full + 8 * ((n_chunks - 1) & 1), ((n_chunks - 1) >> 1) & 1, abort_flag)) {
+                tc_fence_after();
+                float* dst = p.state_out + ((size_t)bh * p.n_groups + g) * D * D + (size_t)srow * D;
 #pragma unroll
-                for (int hh = 0; hh < NH; ++hh)
-                    tma_store_3d(&tmO, stage_out_u + hh * 16384, hh * 64, chunk_row(c), bh);
-                tma_store_commit();
+                for (int c0 = hf * HW; c0 < (hf + 1) * HW; c0 += 32) {
+                    uint32_t r[32];
+                    tmem_ld32(tmem + lane_base + colS + c0, r);
+                    tmem_wait_ld();
+                    if (owns_srow) {
+#pragma unroll
+                        for (int i = 0; i < 32; i += 4)
+                            *reinterpret_cast<float4*>(dst + c0 + i) =
+                                make_float4(__uint_as_float(r[i]), __uint_as_float(r[i + 1]),
+                                            __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+                    }
+                }
             }
+        }
+        if (MODE != MODE_STATE && p.dm_partial != nullptr) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) dm_acc += __shfl_xor_sync(0xffffffffu, dm_acc, o);
+            if (lane == 0) dm_red[warp] = dm_acc;
         }
     }
 
-    if (MODE == MODE_STATE && !failed && p.state_out != nullptr) {
-        // Partial state of this group, fp32, unscaled.
-        float* dst = p.state_out + ((size_t)bh * p.n_groups + g) * D * D + (size_t)srow * D;
-#pragma unroll
-        for (int c0 = 0; c0 < D; c0 += 32) {
-            uint32_t r[32];
-            tmem_ld32(tmem + lane_base + colS + c0, r);
-            tmem_wait_ld();
-            if (owns_row) {
-#pragma unroll
-                for (int i = 0; i < 32; i += 4)
-                    *reinterpret_cast<float4*>(dst + c0 + i) =
-                        make_float4(__uint_as_float(r[i]), __uint_as_float(r[i + 1]),
-                                    __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
-            }
-        }
-    }
-    if (MODE != MODE_STATE && p.dm_partial != nullptr && !failed) {
-        // Fixed-order reduction of <dV', V> over the CTA.
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) dm_acc += __shfl_xor_sync(0xffffffffu, dm_acc, o);
-        if (lane == 0) dm_red[warp] = dm_acc;
-        __syncthreads();
-        if (tid == 0)
-            p.dm_partial[(size_t)bh * p.n_groups + g] = (dm_red[0] + dm_red[1]) + (dm_red[2] + dm_red[3]);
-    }
-
-    if (failed) {
-        if (tid == 0) {
-            atomicExch(p.status, 1);
-            // Give outstanding loads a bounded chance to land before shared memory is released.
-            mbar_wait(bar_full0, 0, 1000000ull);
-            mbar_wait(bar_full1, 0, 1000000ull);
-        }
-    }
-    if (tid == 0) tma_store_wait_all0();
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+    if (MODE != MODE_STATE && p.dm_partial != nullptr && tid == 0 && !*abort_flag) {
+        // Fixed-order reduction of <dV', V> over the CTA.
+        p.dm_partial[(size_t)bh * p.n_groups + g] =
+            ((dm_red[0] + dm_red[1]) + (dm_red[2] + dm_red[3])) +
+            ((dm_red[4] + dm_red[5]) + (dm_red[6] + dm_red[7]));
+    }
+    if (tid == 0 && *abort_flag) atomicExch(p.status, 1);
+    if (warp == 8) tmem_dealloc(tmem, kTmemCols);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
