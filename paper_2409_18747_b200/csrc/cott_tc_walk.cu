@@ -33,6 +33,7 @@ struct TcWalkParams {
     const float* init;      // [BH, n_groups, d*d] unscaled prefix / suffix / total states, or NULL
     float* state_out;       // MODE_STATE: [BH, n_groups, d*d] partial states (unscaled)
     float* dm_partial;      // EPI_DV: [BH, n_groups]
+    void* out;              // [BH, N, d] bf16 output rows (written straight from registers)
     int* status;            // workspace status word
     const float* m; const float* seq_len; float seq_len_scalar;
     int H; int N; int group; int n_groups;
@@ -42,24 +43,37 @@ struct TcWalkParams {
     int reverse;            // 1: walk backward in time, mask keeps columns >= row
 };
 
-template <int D> struct Smem {
-    static constexpr int kStages = (D == 128) ? 2 : 3;    // TMA ring depth
+enum { MODE_STATE = 0, MODE_CAUSAL = 1, MODE_READOUT = 2 };
+
+// Shared-memory plan.  A stage holds the tiles one chunk needs from TMA: (A, Bv) for the
+// state-only pass, (X, A, Bv) for the causal walk, (X) for the read-out.
+template <int D, int MODE> struct Smem {
     static constexpr int kTile = kChunk * D * 2;          // one 128 x D bf16 tile
-    static constexpr int kStage = 3 * kTile;              // X, A, Bv
-    static constexpr int kSb = D * D * 2;                 // bf16 copy of the state
+    static constexpr bool kHasX = MODE != MODE_STATE;
+    static constexpr bool kHasAB = MODE != MODE_READOUT;
+    static constexpr int kTilesPerStage = (kHasX ? 1 : 0) + (kHasAB ? 2 : 0);
+    static constexpr int kStages = MODE == MODE_CAUSAL ? (D == 128 ? 2 : 3)
+                                 : MODE == MODE_STATE ? (D == 128 ? 3 : 4) : 4;
+    static constexpr int kStage = kTilesPerStage * kTile;
+    static constexpr int kOffX = 0;
+    static constexpr int kOffA = kHasX ? kTile : 0;
+    static constexpr int kOffB = kOffA + kTile;
+    static constexpr int kSb = (MODE == MODE_STATE) ? 0 : D * D * 2;   // bf16 copy of the state
     static constexpr int kOffSb = kStages * kStage;
     // Masked-score operand P~ (128 x 128 bf16): d = 128 reuses the X slot (same size, and X
     // is dead by then); d = 64 has a buffer of its own.
     static constexpr int kOffPt = kOffSb + kSb;
-    static constexpr int kPt = (D == 64) ? kChunk * kChunk * 2 : 0;
+    static constexpr int kPt = (MODE == MODE_CAUSAL && D == 64) ? kChunk * kChunk * 2 : 0;
     static constexpr int kOffBar = kOffPt + kPt;          // mbarriers, TMEM slot, abort flag
-    static constexpr int kOffRx = kOffBar + 160;          // rx[kStages][128] floats, dm scratch
-    static constexpr int kCtlBytes = 160 + kStages * 512 + 32;
-    // d = 64 only, and only for launches whose epilogue needs a fourth tile: a dedicated
-    // buffer behind everything else (d = 128 reuses the A slot instead).
+    static constexpr int kOffRx = kOffBar + 192;          // rx[kStages][128] floats, dm scratch
+    static constexpr int kCtlBytes = 192 + kStages * 512 + 32;
+    // Fourth tile for the gradient epilogues (raw q, k or v rows).  The causal walk at
+    // d = 128 reuses the A slot; every other case has a buffer behind the control block,
+    // allocated only for launches that need it.
+    static constexpr bool kProjInA = (MODE == MODE_CAUSAL && D == 128);
     static constexpr int kOffProj = (kOffBar + kCtlBytes + 1023) / 1024 * 1024;
     static constexpr int dyn_bytes(bool with_proj) {
-        return ((with_proj && D == 64) ? kOffProj + kTile : kOffBar + kCtlBytes) + 1024;  // + align slack
+        return ((with_proj && !kProjInA) ? kOffProj + kTile : kOffBar + kCtlBytes) + 1024;  // + align slack
     }
 };
 
@@ -116,28 +130,52 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, vol
     }
 }
 
-__device__ __forceinline__ float sumsq8(const uint4& w) {
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+// Sum of squares of eight bf16 values, on two independent accumulators.
+__device__ __forceinline__ void sumsq8(const uint4& w, float& a0, float& a1) {
     const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&w);
-    float ss = 0.f;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         float2 f = __bfloat1622float2(e[i]);
-        ss += f.x * f.x + f.y * f.y;
+        a0 = fmaf(f.x, f.x, a0);
+        a1 = fmaf(f.y, f.y, a1);
     }
-    return ss;
 }
 
-enum { MODE_STATE = 0, MODE_CAUSAL = 1, MODE_READOUT = 2 };
+__device__ __forceinline__ uint4 pack8(const uint32_t* r) {
+    uint4 w;
+    w.x = pack_bf16(__uint_as_float(r[0]), __uint_as_float(r[1]));
+    w.y = pack_bf16(__uint_as_float(r[2]), __uint_as_float(r[3]));
+    w.z = pack_bf16(__uint_as_float(r[4]), __uint_as_float(r[5]));
+    w.w = pack_bf16(__uint_as_float(r[6]), __uint_as_float(r[7]));
+    return w;
+}
+
+#ifdef COTT_TIMING
+// Debug build only: phase timestamps of CTA 0 for chunks 2 and 3, written behind the status
+// word of the workspace header.
+#define COTT_STAMP(slot)                                                              \
+    do {                                                                              \
+        if (blockIdx.x == 0 && (threadIdx.x == 0 || threadIdx.x == 256) && (c == 2 || c == 3)) \
+            reinterpret_cast<unsigned long long*>(p.status)[1 + (threadIdx.x == 256 ? 14 : 0) + (c - 2) * 7 + (slot)] = \
+                globaltimer_ns();                                                     \
+    } while (0)
+#else
+#define COTT_STAMP(slot) do {} while (0)
+#endif
 
 // Thread roles: warps 0-7 are the row workers (norms, score masking, state and output
-// epilogues); warp 8 lane 0 is the control thread (TMA loads / stores and all tcgen05.mma).
+// epilogues); warp 8 lane 0 is the control thread (TMA loads and all tcgen05.mma).
 // The roles meet only through mbarriers, every wait bounded.
 template <int D, int MODE>
 __global__ void __launch_bounds__(kTcThreads, 1)
 tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmA,
                const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmP,
-               const __grid_constant__ CUtensorMap tmO, TcWalkParams p) {
-    using L = Smem<D>;
+               TcWalkParams p) {
+    using L = Smem<D, MODE>;
     constexpr int NST = L::kStages;
     constexpr int NH = D / 64;                       // 64-column half tiles per row
     constexpr uint32_t kTmemCols = 512;
@@ -149,19 +187,19 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     const uint32_t bars = base + L::kOffBar;
     // Barriers that a fast role could otherwise lap are arrays indexed by stage or by chunk
     // parity, so a phase parity always names one chunk.
-    const uint32_t bar_full = bars;            // [NST] (<= 3) TMA landed
-    const uint32_t bar_a_ready = bars + 24;    // [NST] rows normalised (256 arrivals)
-    const uint32_t bar_p_full = bars + 48;     //       scores and X State done (commit)
-    const uint32_t bar_s_full = bars + 56;     // [2]   state update done (commit)
-    const uint32_t bar_pt_ready = bars + 72;   //       masked scores in shared memory (256)
-    const uint32_t bar_sb_ready = bars + 80;   //       bf16 state copy written (256)
-    const uint32_t bar_o_full = bars + 88;     // [2]   output accumulator complete (commit)
-    const uint32_t bar_o_free = bars + 104;    // [2]   output accumulator drained (256)
-    const uint32_t bar_proj = bars + 120;      //       epilogue tile landed
-    const uint32_t bar_o_staged = bars + 128;  // [2]   output rows staged (256)
-    const uint32_t tmem_slot = bars + 144;
-    volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(gbase + L::kOffBar + 144);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + L::kOffBar + 148);
+    const uint32_t bar_full = bars;            // [NST] (<= 4) TMA landed
+    const uint32_t bar_a_ready = bars + 32;    // [NST] rows normalised (256 arrivals)
+    const uint32_t bar_p_full = bars + 64;     //       scores and X State done (commit)
+    const uint32_t bar_s_full = bars + 72;     // [2]   state update done (commit)
+    const uint32_t bar_pt_ready = bars + 88;   //       masked scores in shared memory (256)
+    const uint32_t bar_sb_ready = bars + 96;   //       bf16 state copy written (256)
+    const uint32_t bar_o_full = bars + 104;    // [2]   output accumulator complete (commit)
+    const uint32_t bar_o_free = bars + 120;    // [2]   output accumulator drained (256)
+    const uint32_t bar_proj = bars + 136;      //       epilogue tile landed
+    const uint32_t bar_e_done = bars + 144;    // [2]   output rows of the chunk written (256)
+    const uint32_t tmem_slot = bars + 160;
+    volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(gbase + L::kOffBar + 160);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + L::kOffBar + 164);
     float* rx_buf = reinterpret_cast<float*>(gbase + L::kOffRx);                 // [NST][128]
     float* dm_red = reinterpret_cast<float*>(gbase + L::kOffRx + NST * 512);     // [8]
 
@@ -184,14 +222,14 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         mbar_init(bar_pt_ready, 256); mbar_init(bar_sb_ready, 256);
         mbar_init(bar_o_full, 1); mbar_init(bar_o_full + 8, 1);
         mbar_init(bar_o_free, 256); mbar_init(bar_o_free + 8, 256);
-        mbar_init(bar_proj, 1); mbar_init(bar_o_staged, 256); mbar_init(bar_o_staged + 8, 256);
+        mbar_init(bar_proj, 1); mbar_init(bar_e_done, 256); mbar_init(bar_e_done + 8, 256);
         *abort_flag = 0;
         mbar_fence_init();
         fence_proxy_async();
     }
     if (is_ctrl && lane == 0) {
         tma_prefetch_desc(&tmX); tma_prefetch_desc(&tmA); tma_prefetch_desc(&tmB);
-        tma_prefetch_desc(&tmP); tma_prefetch_desc(&tmO);
+        tma_prefetch_desc(&tmP);
     }
     tc_fence_before();
     __syncthreads();
@@ -210,24 +248,19 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     const int srow = (D == 128) ? arow : q * 16 + (lane & 15);
     const uint32_t sb = base + L::kOffSb;
 
-    auto stage_x = [&](int s) { return base + s * L::kStage; };
-    auto stage_a = [&](int s) { return base + s * L::kStage + L::kTile; };
-    auto stage_b = [&](int s) { return base + s * L::kStage + 2 * L::kTile; };
+    auto stage_x = [&](int s) { return base + s * L::kStage + L::kOffX; };
+    auto stage_a = [&](int s) { return base + s * L::kStage + L::kOffA; };
+    auto stage_b = [&](int s) { return base + s * L::kStage + L::kOffB; };
     auto stage_pt = [&](int s) { return (D == 128) ? stage_x(s) : base + L::kOffPt; };
     auto chunk_row = [&](int c) { return tok0 + (p.reverse ? (n_chunks - 1 - c) : c) * kChunk; };
 
-    // bf16 copy of this thread's HW state columns into the MN-major state tile.
+    // bf16 copy of 32 state columns of this thread's row into the MN-major state tile.
     auto write_sb = [&](const uint32_t (&r)[32], int c0) {
 #pragma unroll
         for (int i = 0; i < 32; i += 8) {
-            uint4 w;
-            w.x = pack_bf16(__uint_as_float(r[i]), __uint_as_float(r[i + 1]));
-            w.y = pack_bf16(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
-            w.z = pack_bf16(__uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
-            w.w = pack_bf16(__uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
             const int col = c0 + i;
             const uint32_t off = (col >> 6) * (D * 128u) + swz(srow, (col & 63) >> 3);
-            *reinterpret_cast<uint4*>(gbase + L::kOffSb + off) = w;
+            *reinterpret_cast<uint4*>(gbase + L::kOffSb + off) = pack8(&r[i]);
         }
     };
 
@@ -246,7 +279,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 r[i + 2] = __float_as_uint(v.z); r[i + 3] = __float_as_uint(v.w);
             }
             if (MODE == MODE_CAUSAL) tmem_st32(tmem + lane_base + colS + c0, r);
-            if (owns_srow) write_sb(r, c0);
+            if (MODE != MODE_STATE && owns_srow) write_sb(r, c0);
         }
         if (MODE == MODE_CAUSAL) tmem_wait_st();
         fence_proxy_async();
@@ -265,29 +298,29 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 const int s = c % NST;
                 const uint32_t bar = bar_full + 8 * s;
                 const int row = chunk_row(c);
-                constexpr uint32_t n_tiles = (MODE == MODE_STATE) ? 2 : (MODE == MODE_CAUSAL ? 3 : 1);
-                mbar_expect_tx(bar, n_tiles * L::kTile);
+                mbar_expect_tx(bar, L::kTilesPerStage * L::kTile);
 #pragma unroll
                 for (int hh = 0; hh < NH; ++hh) {
-                    if (MODE != MODE_STATE) tma_load_3d(stage_x(s) + hh * 16384, &tmX, bar, hh * 64, row, bh);
-                    if (MODE != MODE_READOUT) {
+                    if (L::kHasX) tma_load_3d(stage_x(s) + hh * 16384, &tmX, bar, hh * 64, row, bh);
+                    if (L::kHasAB) {
                         tma_load_3d(stage_a(s) + hh * 16384, &tmA, bar, hh * 64, row, bh);
                         tma_load_3d(stage_b(s) + hh * 16384, &tmB, bar, hh * 64, row, bh);
                     }
                 }
             };
+            auto wait = [&](uint32_t bar, uint32_t parity) {
+                if (alive && !wait_or_abort(bar, parity, abort_flag)) alive = false;
+                return alive;
+            };
             // First MMA batch of chunk c: scores, X State (needs the previous chunk's state
             // copy and a drained output buffer), state update.
             auto batch1 = [&](int c) {
                 const int s = c % NST;
-                if (!wait_or_abort(bar_a_ready + 8 * s, (c / NST) & 1, abort_flag)) { alive = false; return; }
+                if (!wait(bar_a_ready + 8 * s, (c / NST) & 1)) return;
                 const bool acc = init_state || c > 0;
                 if (MODE != MODE_STATE) {
-                    if (MODE == MODE_CAUSAL && c >= 1 &&
-                        !wait_or_abort(bar_sb_ready, (c - 1) & 1, abort_flag)) { alive = false; return; }
-                    if (c >= 2 && !wait_or_abort(bar_o_free + 8 * (c & 1), ((c >> 1) & 1) ^ 1, abort_flag)) {
-                        alive = false; return;
-                    }
+                    if (MODE == MODE_CAUSAL && c >= 1 && !wait(bar_sb_ready, (c - 1) & 1)) return;
+                    if (c >= 2 && !wait(bar_o_free + 8 * (c & 1), ((c >> 1) & 1) ^ 1)) return;
                 }
                 tc_fence_after();
                 const uint32_t tO = tmem + colO0 + (c & 1) * D;
@@ -305,46 +338,57 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     tc_commit(bar_o_full + 8 * (c & 1));
                 }
             };
+            // Reload the stage of chunk c with chunk c + NST once nothing reads it any more.
+            auto refill = [&](int c) {
+                if (c + NST >= n_chunks) return;
+                if (MODE == MODE_STATE) {
+                    if (!wait(bar_s_full + 8 * (c & 1), (c >> 1) & 1)) return;
+                } else {
+                    if (!wait(bar_o_full + 8 * (c & 1), (c >> 1) & 1)) return;
+                    if (with_proj && L::kProjInA && !wait(bar_e_done + 8 * (c & 1), (c >> 1) & 1)) return;
+                }
+                issue_loads(c + NST);
+            };
             for (int c = 0; c < NST && c < n_chunks; ++c) issue_loads(c);
             batch1(0);
             for (int c = 0; c < n_chunks && alive; ++c) {
                 const int s = c % NST;
+                COTT_STAMP(0);
                 if (with_proj) {
-                    // d = 128: the A slot is free once the state update has read it.
-                    if (MODE == MODE_CAUSAL && D == 128 &&
-                        !wait_or_abort(bar_s_full + 8 * (c & 1), (c >> 1) & 1, abort_flag)) { alive = false; break; }
-                    const uint32_t proj_u = (D == 128) ? stage_a(s) : base + L::kOffProj;
+                    // The buffer is free once the state update has read the A slot (d = 128
+                    // causal walk) or the previous chunk's epilogue has finished (dedicated).
+                    if (L::kProjInA) { if (!wait(bar_s_full + 8 * (c & 1), (c >> 1) & 1)) break; }
+                    else if (c >= 1) { if (!wait(bar_e_done + 8 * ((c - 1) & 1), ((c - 1) >> 1) & 1)) break; }
+                    const uint32_t proj_u = L::kProjInA ? stage_a(s) : base + L::kOffProj;
                     mbar_expect_tx(bar_proj, L::kTile);
 #pragma unroll
                     for (int hh = 0; hh < NH; ++hh)
                         tma_load_3d(proj_u + hh * 16384, &tmP, bar_proj, hh * 64, chunk_row(c), bh);
                 }
                 if (MODE == MODE_CAUSAL) {
-                    if (!wait_or_abort(bar_pt_ready, c & 1, abort_flag)) { alive = false; break; }
+                    if (!wait(bar_pt_ready, c & 1)) break;
+                    COTT_STAMP(1);
                     tc_fence_after();
                     issue_pb<D>(tmem + colO0 + (c & 1) * D, stage_pt(s), stage_b(s), init_state || c > 0);
                     tc_commit(bar_o_full + 8 * (c & 1));
                 }
-                if (c + 1 < n_chunks) { batch1(c + 1); if (!alive) break; }
-                if (MODE != MODE_STATE) {
-                    if (!wait_or_abort(bar_o_staged + 8 * (c & 1), (c >> 1) & 1, abort_flag)) { alive = false; break; }
-#pragma unroll
-                    for (int hh = 0; hh < NH; ++hh)
-                        tma_store_3d(&tmO, stage_b(s) + hh * 16384, hh * 64, chunk_row(c), bh);
-                    tma_store_commit();
-                } else {
-                    if (!wait_or_abort(bar_s_full + 8 * (c & 1), (c >> 1) & 1, abort_flag)) { alive = false; break; }
-                }
-                if (c + NST < n_chunks) {
-                    if (MODE != MODE_STATE) tma_store_wait_read0();
-                    issue_loads(c + NST);
-                }
+                COTT_STAMP(2);
+                const bool refill_late = with_proj && L::kProjInA;   // stage holds the proj tile
+                if (!refill_late) refill(c);
+                COTT_STAMP(3);
+                if (c + 1 < n_chunks) batch1(c + 1);
+                COTT_STAMP(4);
+                if (refill_late) refill(c);
+                COTT_STAMP(5);
             }
-            tma_store_wait_all0();
         }
     } else {
         // ------------------------------------------------------------------ row workers
         bool alive = n_chunks > 0;
+        auto wait = [&](uint32_t bar, uint32_t parity) {
+            if (alive && !wait_or_abort(bar, parity, abort_flag)) alive = false;
+            return alive;
+        };
         // Norm-phase mapping: lanes l and l^16 share a row (two column halves).
         const int nrow = warp * 16 + (lane & 15), nhalf = lane >> 4;
         constexpr int NC = D / 16;                    // 16-byte chunks in half a row
@@ -353,37 +397,43 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             return tile + (ch >> 3) * 16384 + swz(nrow, ch & 7);
         };
         // Row norms of chunk c: the contraction-side operand is normalised in place; the X
-        // row scale (times c) is left in rx_buf[c&1] for the output epilogue.
+        // row scale (times c) is left in rx_buf[c % NST] for the output epilogue.
         auto norm_phase = [&](int c) {
             const int s = c % NST;
-            if (!wait_or_abort(bar_full + 8 * s, (c / NST) & 1, abort_flag)) { alive = false; return; }
-            uint8_t* xs = gbase + s * L::kStage;
-            if (MODE != MODE_STATE) {
+            if (!wait(bar_full + 8 * s, (c / NST) & 1)) return;
+            uint8_t* st = gbase + s * L::kStage;
+            uint4 wx[NC], wn[NC];
+            if (L::kHasX && p.x_norm) {
+#pragma unroll
+                for (int j = 0; j < NC; ++j) wx[j] = *reinterpret_cast<const uint4*>(tile_half_ptr(st + L::kOffX, j));
+            }
+            uint8_t* nt = st + (p.norm_bv ? L::kOffB : L::kOffA);
+            if (L::kHasAB) {
+#pragma unroll
+                for (int j = 0; j < NC; ++j) wn[j] = *reinterpret_cast<const uint4*>(tile_half_ptr(nt, j));
+            }
+            if (L::kHasX) {
                 float rx = cfac;
                 if (p.x_norm) {
-                    float ss = 0.f;
+                    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
-                    for (int j = 0; j < NC; ++j)
-                        ss += sumsq8(*reinterpret_cast<const uint4*>(tile_half_ptr(xs, j)));
+                    for (int j = 0; j < NC; j += 2) { sumsq8(wx[j], a0, a1); sumsq8(wx[j + 1], a2, a3); }
+                    float ss = (a0 + a1) + (a2 + a3);
                     ss += __shfl_xor_sync(0xffffffffu, ss, 16);
                     rx = cfac / fmaxf(sqrtf(ss), kEps);
                 }
                 if (nhalf == 0) rx_buf[(c % NST) * 128 + nrow] = rx;
             }
-            if (MODE != MODE_READOUT) {
-                uint8_t* nt = xs + (p.norm_bv ? 2 : 1) * L::kTile;
-                uint4 w[NC];
-                float ss = 0.f;
+            if (L::kHasAB) {
+                float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
-                for (int j = 0; j < NC; ++j) {
-                    w[j] = *reinterpret_cast<const uint4*>(tile_half_ptr(nt, j));
-                    ss += sumsq8(w[j]);
-                }
+                for (int j = 0; j < NC; j += 2) { sumsq8(wn[j], a0, a1); sumsq8(wn[j + 1], a2, a3); }
+                float ss = (a0 + a1) + (a2 + a3);
                 ss += __shfl_xor_sync(0xffffffffu, ss, 16);
                 const float r = 1.0f / fmaxf(sqrtf(ss), kEps);
 #pragma unroll
                 for (int j = 0; j < NC; ++j) {
-                    const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&w[j]);
+                    const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&wn[j]);
                     uint4 o;
                     uint32_t* ow = reinterpret_cast<uint32_t*>(&o);
 #pragma unroll
@@ -395,53 +445,54 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 }
                 fence_proxy_async();
             }
-            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_a_ready + 8 * s) : "memory");
-        };
-        auto arrive = [&](uint32_t bar) {
-            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+            mbar_arrive(bar_a_ready + 8 * s);
         };
 
         if (alive) norm_phase(0);
         for (int c = 0; c < n_chunks && alive; ++c) {
             const int s = c % NST;
-            uint8_t* xs = gbase + s * L::kStage;
-            uint8_t* bs = xs + 2 * L::kTile;
-            uint8_t* pt = (D == 128) ? xs : gbase + L::kOffPt;
+            uint8_t* st = gbase + s * L::kStage;
+            uint8_t* pt = (D == 128) ? st + L::kOffX : gbase + L::kOffPt;
             if (MODE == MODE_CAUSAL) {
-                // Masked scores -> bf16 operand in the X slot (both MMAs that read X are done).
-                // Forward: row i keeps columns j <= i (diagonal kept, Eq. 6); backward in time:
-                // columns j >= i.
-                if (!wait_or_abort(bar_p_full, c & 1, abort_flag)) { alive = false; break; }
+                // Masked scores -> bf16 operand P~ (both MMAs that read X are done).  Forward:
+                // row i keeps columns j <= i (diagonal kept, Eq. 6); backward in time: j >= i.
+                // Per 32 x 32 block of this warp the mask is all-keep, all-zero, or (on the
+                // diagonal) a triangle: the first two cases are warp-uniform.
+                COTT_STAMP(0);
+                if (!wait(bar_p_full, c & 1)) break;
                 tc_fence_after();
-                uint32_t r0[32], r1[32];
-                tmem_ld32(tmem + lane_base + colP + hf * 64, r0);
-                tmem_ld32(tmem + lane_base + colP + hf * 64 + 32, r1);
-                tmem_wait_ld();
+                COTT_STAMP(1);
 #pragma unroll
-                for (int part = 0; part < 2; ++part) {
-                    const uint32_t* r = part ? r1 : r0;
+                for (int sbk = 0; sbk < 2; ++sbk) {
+                    const int cb = 2 * hf + sbk;      // 32-column block index; row block index is q
+                    const bool keep_all = p.reverse ? (cb > q) : (cb < q);
+                    const bool diag = cb == q;
+                    uint32_t r[32];
+                    if (keep_all || diag) {
+                        tmem_ld32(tmem + lane_base + colP + cb * 32, r);
+                        tmem_wait_ld();
+                        if (diag) {
 #pragma unroll
-                    for (int i = 0; i < 32; i += 8) {
-                        uint4 w;
-                        uint32_t* ww = reinterpret_cast<uint32_t*>(&w);
-#pragma unroll
-                        for (int j = 0; j < 8; j += 2) {
-                            const int col = hf * 64 + part * 32 + i + j;
-                            const bool k0 = p.reverse ? (col >= arow) : (col <= arow);
-                            const bool k1 = p.reverse ? (col + 1 >= arow) : (col + 1 <= arow);
-                            ww[j >> 1] = pack_bf16(k0 ? __uint_as_float(r[i + j]) : 0.f,
-                                                   k1 ? __uint_as_float(r[i + j + 1]) : 0.f);
+                            for (int j = 0; j < 32; ++j) {
+                                const bool keep = p.reverse ? (j >= lane) : (j <= lane);
+                                r[j] = keep ? r[j] : 0u;
+                            }
                         }
-                        const int ch = (part * 32 + i) >> 3;   // chunk within this thread's half
-                        *reinterpret_cast<uint4*>(pt + hf * 16384 + swz(arow, ch)) = w;
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) r[j] = 0u;
                     }
+#pragma unroll
+                    for (int i = 0; i < 32; i += 8)
+                        *reinterpret_cast<uint4*>(pt + hf * 16384 + swz(arow, sbk * 4 + (i >> 3))) = pack8(&r[i]);
                 }
+                COTT_STAMP(2);
                 fence_proxy_async();
                 tc_fence_before();
-                arrive(bar_pt_ready);
+                mbar_arrive(bar_pt_ready);
                 // bf16 copy of the updated state for the next chunk's X State product.
                 if (c + 1 < n_chunks) {
-                    if (!wait_or_abort(bar_s_full + 8 * (c & 1), (c >> 1) & 1, abort_flag)) { alive = false; break; }
+                    if (!wait(bar_s_full + 8 * (c & 1), (c >> 1) & 1)) break;
                     tc_fence_after();
 #pragma unroll
                     for (int c0 = hf * HW; c0 < (hf + 1) * HW; c0 += 32) {
@@ -452,24 +503,32 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     }
                     fence_proxy_async();
                     tc_fence_before();
-                    arrive(bar_sb_ready);
+                    mbar_arrive(bar_sb_ready);
                 }
+                COTT_STAMP(3);
             }
             if (c + 1 < n_chunks) { norm_phase(c + 1); if (!alive) break; }
-            if (MODE == MODE_STATE) continue;
+            COTT_STAMP(4);
+            if (MODE == MODE_STATE) {
+                // Follow every state update (a parity names one chunk only if no phase is
+                // skipped); after the last one the accumulator holds the group's state.
+                if (!wait(bar_s_full + 8 * (c & 1), (c >> 1) & 1)) break;
+                continue;
+            }
 
-            // ---- output epilogue of chunk c
-            if (!wait_or_abort(bar_o_full + 8 * (c & 1), (c >> 1) & 1, abort_flag)) { alive = false; break; }
+            // ---- output epilogue of chunk c: straight from the accumulator to global memory
+            if (!wait(bar_o_full + 8 * (c & 1), (c >> 1) & 1)) break;
             tc_fence_after();
+            COTT_STAMP(5);
             const uint32_t tO = tmem + lane_base + colO0 + (c & 1) * D;
             const float rx = rx_buf[(c % NST) * 128 + arow];
             float coef = 0.f, rp = 1.f;
-            const uint8_t* proj = (D == 128) ? (xs + L::kTile) : (gbase + L::kOffProj);
+            const uint8_t* proj = L::kProjInA ? (st + L::kOffA) : (gbase + L::kOffProj);
             if (with_proj) {
-                if (!wait_or_abort(bar_proj, c & 1, abort_flag)) { alive = false; break; }
+                if (!wait(bar_proj, c & 1)) break;
                 // <p, acc> and ||p||^2 over the whole row (both column-half threads compute
                 // the same sums; the proj tile is read-only).
-                float ss = 0.f, dp = 0.f;
+                float ss0 = 0.f, ss1 = 0.f, dp0 = 0.f, dp1 = 0.f;
 #pragma unroll
                 for (int c0 = 0; c0 < D; c0 += 32) {
                     uint32_t r[32];
@@ -484,11 +543,13 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
                             float2 f = __bfloat1622float2(e[j]);
-                            ss += f.x * f.x + f.y * f.y;
-                            dp += f.x * __uint_as_float(r[i + 2 * j]) + f.y * __uint_as_float(r[i + 2 * j + 1]);
+                            ss0 = fmaf(f.x, f.x, ss0); ss1 = fmaf(f.y, f.y, ss1);
+                            dp0 = fmaf(f.x, __uint_as_float(r[i + 2 * j]), dp0);
+                            dp1 = fmaf(f.y, __uint_as_float(r[i + 2 * j + 1]), dp1);
                         }
                     }
                 }
+                const float ss = ss0 + ss1, dp = dp0 + dp1;
                 if (p.epilogue == EPI_PROJ) {
                     // g = rx * acc;  out = (g - p^ <p^, g>) / max(||p||, eps); clamped branch: g / eps
                     const float nrm = sqrtf(ss);
@@ -498,7 +559,10 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     dm_acc += dp * rx / cfac;  // <dV', v> with dV' = (rx / c) * acc, once per row
                 }
             }
-            // This thread's HW columns: scale, (project,) round to bf16, stage in the Bv slot.
+            // This thread's HW columns: scale, (project,) round to bf16, store (one full
+            // 64-byte or 128-byte run of the output row per thread).
+            const int grow = chunk_row(c) + arow;
+            __nv_bfloat16* orow = static_cast<__nv_bfloat16*>(p.out) + ((size_t)bh * p.N + grow) * D;
 #pragma unroll
             for (int c0 = hf * HW; c0 < (hf + 1) * HW; c0 += 32) {
                 uint32_t r[32];
@@ -507,12 +571,12 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
 #pragma unroll
                 for (int i = 0; i < 32; i += 8) {
                     const int col = c0 + i;
-                    const uint32_t off = (col >> 6) * 16384 + swz(arow, (col & 63) >> 3);
                     float v[8];
 #pragma unroll
                     for (int j = 0; j < 8; ++j) v[j] = __uint_as_float(r[i + j]) * rx;
                     if (with_proj && p.epilogue == EPI_PROJ) {
-                        uint4 w = *reinterpret_cast<const uint4*>(proj + off);
+                        uint4 w = *reinterpret_cast<const uint4*>(proj + (col >> 6) * 16384 +
+                                                                  swz(arow, (col & 63) >> 3));
                         const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&w);
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
@@ -524,18 +588,18 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     uint4 w;
                     w.x = pack_bf16(v[0], v[1]); w.y = pack_bf16(v[2], v[3]);
                     w.z = pack_bf16(v[4], v[5]); w.w = pack_bf16(v[6], v[7]);
-                    *reinterpret_cast<uint4*>(bs + off) = w;
+                    if (grow < p.N) *reinterpret_cast<uint4*>(orow + col) = w;
                 }
             }
             tc_fence_before();
-            arrive(bar_o_free + 8 * (c & 1));
-            fence_proxy_async();
-            arrive(bar_o_staged + 8 * (c & 1));
+            mbar_arrive(bar_o_free + 8 * (c & 1));
+            mbar_arrive(bar_e_done + 8 * (c & 1));
+            COTT_STAMP(6);
         }
 
         if (MODE == MODE_STATE && alive && p.state_out != nullptr) {
             // Partial state of this group, fp32, unscaled.
-            if (wait_or_abort(bar_s_full + 8 * ((n_chunks - 1) & 1), ((n_chunks - 1) >> 1) & 1, abort_flag)) {
+            {
                 tc_fence_after();
                 float* dst = p.state_out + ((size_t)bh * p.n_groups + g) * D * D + (size_t)srow * D;
 #pragma unroll
@@ -612,13 +676,13 @@ cudaError_t launch_mode(const CUtensorMap* tm, const TcWalkParams& p, int BH, cu
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             Smem<D>::dyn_bytes(true));
+                                             Smem<D, MODE>::dyn_bytes(true));
         if (e != cudaSuccess) return e;
         configured = true;
     }
     const bool with_proj = (MODE != MODE_STATE) && (p.epilogue != EPI_PLAIN);
-    kern<<<dim3((unsigned)(BH * p.n_groups)), kTcThreads, Smem<D>::dyn_bytes(with_proj), st>>>(
-        tm[0], tm[1], tm[2], tm[3], tm[4], p);
+    kern<<<dim3((unsigned)(BH * p.n_groups)), kTcThreads, Smem<D, MODE>::dyn_bytes(with_proj), st>>>(
+        tm[0], tm[1], tm[2], tm[3], p);
     note_launch();
     return cudaGetLastError();
 }
@@ -629,13 +693,14 @@ cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cuda
     const int BH = B * H;
     // Unused operands still need a valid map: point them at a tensor that exists.
     const void* any = a.x ? a.x : a.a;
-    const void* ptrs[5] = {a.x ? a.x : any, a.a ? a.a : any, a.bv ? a.bv : any,
-                           a.proj ? a.proj : any, a.out ? a.out : any};
-    CUtensorMap tm[5];
-    for (int i = 0; i < 5; ++i)
+    const void* ptrs[4] = {a.x ? a.x : any, a.a ? a.a : any, a.bv ? a.bv : any,
+                           a.proj ? a.proj : any};
+    CUtensorMap tm[4];
+    for (int i = 0; i < 4; ++i)
         if (!make_tile_map(&tm[i], ptrs[i], BH, N, d)) return cudaErrorInvalidValue;
     TcWalkParams p;
     p.init = a.init; p.state_out = a.state_out; p.dm_partial = a.dm_partial; p.status = a.status;
+    p.out = a.out;
     p.m = a.m; p.seq_len = a.seq_len; p.seq_len_scalar = a.seq_len_scalar;
     p.H = H; p.N = N; p.group = a.group; p.n_groups = a.n_groups;
     p.norm_bv = a.norm_bv; p.x_norm = a.x_norm; p.epilogue = a.epilogue; p.reverse = a.reverse;
