@@ -26,14 +26,13 @@ using namespace sm100;
 namespace {
 
 constexpr int kChunk = 128;
-constexpr int kTcThreads = 288;   // 8 row-worker warps + 1 control warp
+constexpr int kTcThreads = 544;   // 16 row-worker warps + 1 control warp
 constexpr uint64_t kWaitTimeoutNs = 2000000000ull;  // 2 s: far above any legitimate wait
 
 struct TcWalkParams {
     const float* init;      // [BH, n_groups, d*d] unscaled prefix / suffix / total states, or NULL
     float* state_out;       // MODE_STATE: [BH, n_groups, d*d] partial states (unscaled)
     float* dm_partial;      // EPI_DV: [BH, n_groups]
-    void* out;              // [BH, N, d] bf16 output rows (written straight from registers)
     int* status;            // workspace status word
     const float* m; const float* seq_len; float seq_len_scalar;
     int H; int N; int group; int n_groups;
@@ -44,6 +43,9 @@ struct TcWalkParams {
 };
 
 enum { MODE_STATE = 0, MODE_CAUSAL = 1, MODE_READOUT = 2 };
+
+constexpr int kWorkerWarps = 16;                      // row-worker warps (4 per TMEM lane quadrant)
+constexpr int kWorkers = kWorkerWarps * 32;
 
 // Shared-memory plan.  A stage holds the tiles one chunk needs from TMA: (A, Bv) for the
 // state-only pass, (X, A, Bv) for the causal walk, (X) for the read-out.
@@ -58,6 +60,7 @@ template <int D, int MODE> struct Smem {
     static constexpr int kOffX = 0;
     static constexpr int kOffA = kHasX ? kTile : 0;
     static constexpr int kOffB = kOffA + kTile;
+    static constexpr int kOffOut = kHasAB ? kOffB : kOffX;             // output staging slot
     static constexpr int kSb = (MODE == MODE_STATE) ? 0 : D * D * 2;   // bf16 copy of the state
     static constexpr int kOffSb = kStages * kStage;
     // Masked-score operand P~ (128 x 128 bf16): d = 128 reuses the X slot (same size, and X
@@ -66,14 +69,16 @@ template <int D, int MODE> struct Smem {
     static constexpr int kPt = (MODE == MODE_CAUSAL && D == 64) ? kChunk * kChunk * 2 : 0;
     static constexpr int kOffBar = kOffPt + kPt;          // mbarriers, TMEM slot, abort flag
     static constexpr int kOffRx = kOffBar + 192;          // rx[kStages][128] floats, dm scratch
-    static constexpr int kCtlBytes = 192 + kStages * 512 + 32;
-    // Fourth tile for the gradient epilogues (raw q, k or v rows).  The causal walk at
-    // d = 128 reuses the A slot; every other case has a buffer behind the control block,
-    // allocated only for launches that need it.
+    static constexpr int kCtlBytes = 192 + kStages * 512 + 64;
+    // Gradient epilogues need a fourth tile (raw q, k or v rows) and a 4 KB exchange area
+    // for per-row partial sums.  The causal walk at d = 128 has no room for either: it puts
+    // the tile in the A slot and the exchange area in the X slot, both dead by then.  Every
+    // other case has a buffer behind the control block, allocated only when needed.
     static constexpr bool kProjInA = (MODE == MODE_CAUSAL && D == 128);
     static constexpr int kOffProj = (kOffBar + kCtlBytes + 1023) / 1024 * 1024;
+    static constexpr int kXch = 4096;
     static constexpr int dyn_bytes(bool with_proj) {
-        return ((with_proj && !kProjInA) ? kOffProj + kTile : kOffBar + kCtlBytes) + 1024;  // + align slack
+        return ((with_proj && !kProjInA) ? kOffProj + kTile + kXch : kOffBar + kCtlBytes) + 1024;  // + align slack
     }
 };
 
@@ -154,54 +159,64 @@ __device__ __forceinline__ uint4 pack8(const uint32_t* r) {
     return w;
 }
 
+// QW (16 or 32) consecutive accumulator columns of this thread's TMEM lane.
+template <int QW> __device__ __forceinline__ void tmem_ldq(uint32_t taddr, uint32_t (&r)[QW]);
+template <> __device__ __forceinline__ void tmem_ldq<32>(uint32_t taddr, uint32_t (&r)[32]) { tmem_ld32(taddr, r); }
+template <> __device__ __forceinline__ void tmem_ldq<16>(uint32_t taddr, uint32_t (&r)[16]) { tmem_ld16(taddr, r); }
+template <int QW> __device__ __forceinline__ void tmem_stq(uint32_t taddr, const uint32_t (&r)[QW]);
+template <> __device__ __forceinline__ void tmem_stq<32>(uint32_t taddr, const uint32_t (&r)[32]) { tmem_st32(taddr, r); }
+template <> __device__ __forceinline__ void tmem_stq<16>(uint32_t taddr, const uint32_t (&r)[16]) { tmem_st16(taddr, r); }
+
 #ifdef COTT_TIMING
 // Debug build only: phase timestamps of CTA 0 for chunks 2 and 3, written behind the status
 // word of the workspace header.
 #define COTT_STAMP(slot)                                                              \
     do {                                                                              \
-        if (blockIdx.x == 0 && (threadIdx.x == 0 || threadIdx.x == 256) && (c == 2 || c == 3)) \
-            reinterpret_cast<unsigned long long*>(p.status)[1 + (threadIdx.x == 256 ? 14 : 0) + (c - 2) * 7 + (slot)] = \
+        if (blockIdx.x == 0 && (threadIdx.x == 0 || threadIdx.x == kWorkers) && (c == 2 || c == 3)) \
+            reinterpret_cast<unsigned long long*>(p.status)[1 + (threadIdx.x == kWorkers ? 14 : 0) + (c - 2) * 7 + (slot)] = \
                 globaltimer_ns();                                                     \
     } while (0)
 #else
 #define COTT_STAMP(slot) do {} while (0)
 #endif
 
-// Thread roles: warps 0-7 are the row workers (norms, score masking, state and output
-// epilogues); warp 8 lane 0 is the control thread (TMA loads and all tcgen05.mma).
+// Thread roles: warps 0-15 are the row workers (norms, score masking, state and output
+// epilogues; four warps per TMEM lane quadrant, each owning a quarter of the columns);
+// warp 16 lane 0 is the control thread (TMA loads / stores and all tcgen05.mma).
 // The roles meet only through mbarriers, every wait bounded.
 template <int D, int MODE>
 __global__ void __launch_bounds__(kTcThreads, 1)
 tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmA,
                const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmP,
-               TcWalkParams p) {
+               const __grid_constant__ CUtensorMap tmO, TcWalkParams p) {
     using L = Smem<D, MODE>;
     constexpr int NST = L::kStages;
     constexpr int NH = D / 64;                       // 64-column half tiles per row
     constexpr uint32_t kTmemCols = 512;
     constexpr uint32_t colS = 0, colP = D, colO0 = D + 128;   // O double-buffered: colO0, colO0 + D
-    constexpr int HW = D / 2;                        // accumulator columns per worker thread
+    constexpr int QW = D / 4;                        // accumulator columns per worker thread
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* gbase = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t bars = base + L::kOffBar;
     // Barriers that a fast role could otherwise lap are arrays indexed by stage or by chunk
-    // parity, so a phase parity always names one chunk.
+    // parity, so a phase parity always names one chunk; no waiter ever skips a phase.
     const uint32_t bar_full = bars;            // [NST] (<= 4) TMA landed
-    const uint32_t bar_a_ready = bars + 32;    // [NST] rows normalised (256 arrivals)
+    const uint32_t bar_a_ready = bars + 32;    // [NST] rows normalised (all workers)
     const uint32_t bar_p_full = bars + 64;     //       scores and X State done (commit)
     const uint32_t bar_s_full = bars + 72;     // [2]   state update done (commit)
-    const uint32_t bar_pt_ready = bars + 88;   //       masked scores in shared memory (256)
-    const uint32_t bar_sb_ready = bars + 96;   //       bf16 state copy written (256)
+    const uint32_t bar_pt_ready = bars + 88;   //       masked scores in shared memory (all workers)
+    const uint32_t bar_sb_ready = bars + 96;   //       bf16 state copy written (all workers)
     const uint32_t bar_o_full = bars + 104;    // [2]   output accumulator complete (commit)
-    const uint32_t bar_o_free = bars + 120;    // [2]   output accumulator drained (256)
+    const uint32_t bar_o_free = bars + 120;    // [2]   output accumulator drained (all workers)
     const uint32_t bar_proj = bars + 136;      //       epilogue tile landed
-    const uint32_t bar_e_done = bars + 144;    // [2]   output rows of the chunk written (256)
-    const uint32_t tmem_slot = bars + 160;
-    volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(gbase + L::kOffBar + 160);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + L::kOffBar + 164);
+    const uint32_t bar_e_done = bars + 144;    // [2]   output rows of the chunk staged (all workers)
+    const uint32_t bar_xch = bars + 160;       //       per-row partial sums exchanged (all workers)
+    const uint32_t tmem_slot = bars + 168;
+    volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(gbase + L::kOffBar + 168);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + L::kOffBar + 172);
     float* rx_buf = reinterpret_cast<float*>(gbase + L::kOffRx);                 // [NST][128]
-    float* dm_red = reinterpret_cast<float*>(gbase + L::kOffRx + NST * 512);     // [8]
+    float* dm_red = reinterpret_cast<float*>(gbase + L::kOffRx + NST * 512);     // [16]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = blockIdx.x % p.n_groups, bh = blockIdx.x / p.n_groups;
@@ -210,26 +225,27 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     const int tok1 = min(p.N, tok0 + p.group);
     const int n_chunks = (tok1 - tok0 + kChunk - 1) / kChunk;
     const bool with_proj = (MODE != MODE_STATE) && (p.epilogue != EPI_PLAIN);
-    const bool is_ctrl = warp == 8;
+    const bool is_ctrl = warp == kWorkerWarps;
 
-    if (warp == 8) {
+    if (is_ctrl) {
         tmem_alloc(tmem_slot, kTmemCols);
         tmem_relinquish();
     }
     if (tid == 0) {
-        for (int i = 0; i < NST; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_a_ready + 8 * i, 256); }
+        for (int i = 0; i < NST; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_a_ready + 8 * i, kWorkers); }
         mbar_init(bar_p_full, 1); mbar_init(bar_s_full, 1); mbar_init(bar_s_full + 8, 1);
-        mbar_init(bar_pt_ready, 256); mbar_init(bar_sb_ready, 256);
+        mbar_init(bar_pt_ready, kWorkers); mbar_init(bar_sb_ready, kWorkers);
         mbar_init(bar_o_full, 1); mbar_init(bar_o_full + 8, 1);
-        mbar_init(bar_o_free, 256); mbar_init(bar_o_free + 8, 256);
-        mbar_init(bar_proj, 1); mbar_init(bar_e_done, 256); mbar_init(bar_e_done + 8, 256);
+        mbar_init(bar_o_free, kWorkers); mbar_init(bar_o_free + 8, kWorkers);
+        mbar_init(bar_proj, 1); mbar_init(bar_e_done, kWorkers); mbar_init(bar_e_done + 8, kWorkers);
+        mbar_init(bar_xch, kWorkers);
         *abort_flag = 0;
         mbar_fence_init();
         fence_proxy_async();
     }
     if (is_ctrl && lane == 0) {
         tma_prefetch_desc(&tmX); tma_prefetch_desc(&tmA); tma_prefetch_desc(&tmB);
-        tma_prefetch_desc(&tmP);
+        tma_prefetch_desc(&tmP); tma_prefetch_desc(&tmO);
     }
     tc_fence_before();
     __syncthreads();
@@ -239,8 +255,8 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     const float s_b = p.seq_len ? p.seq_len[b] : (p.seq_len_scalar > 0.f ? p.seq_len_scalar : (float)p.N);
     const float cfac = stab_factor(p.m[h], s_b);
 
-    // Accumulator mapping of a worker thread: TMEM lane quadrant q, column half hf, row.
-    const int q = warp & 3, hf = (warp >> 2) & 1;
+    // Accumulator mapping of a worker thread: TMEM lane quadrant q, column quarter cq, row.
+    const int q = warp & 3, cq = (warp >> 2) & 3;
     const uint32_t lane_base = (uint32_t)(q * 32) << 16;
     const int arow = q * 32 + lane;                   // row of P / Out held by this thread
     // State rows: M = 128 maps row r to lane r; M = 64 maps row r to lane (r%16) + 32*(r/16).
@@ -254,10 +270,10 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     auto stage_pt = [&](int s) { return (D == 128) ? stage_x(s) : base + L::kOffPt; };
     auto chunk_row = [&](int c) { return tok0 + (p.reverse ? (n_chunks - 1 - c) : c) * kChunk; };
 
-    // bf16 copy of 32 state columns of this thread's row into the MN-major state tile.
-    auto write_sb = [&](const uint32_t (&r)[32], int c0) {
+    // bf16 copy of QW state columns of this thread's row into the MN-major state tile.
+    auto write_sb = [&](const uint32_t (&r)[QW], int c0) {
 #pragma unroll
-        for (int i = 0; i < 32; i += 8) {
+        for (int i = 0; i < QW; i += 8) {
             const int col = c0 + i;
             const uint32_t off = (col >> 6) * (D * 128u) + swz(srow, (col & 63) >> 3);
             *reinterpret_cast<uint4*>(gbase + L::kOffSb + off) = pack8(&r[i]);
@@ -267,21 +283,16 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     const bool init_state = p.init != nullptr;
     if (init_state && !is_ctrl) {
         // Initial state of the group: fp32 into TMEM, bf16 copy into shared memory.
-        const float* src = p.init + ((size_t)bh * p.n_groups + g) * D * D + (size_t)srow * D;
+        const float* src = p.init + ((size_t)bh * p.n_groups + g) * D * D + (size_t)srow * D + cq * QW;
+        uint32_t r[QW];
 #pragma unroll
-        for (int c0 = hf * HW; c0 < (hf + 1) * HW; c0 += 32) {
-            uint32_t r[32];
-#pragma unroll
-            for (int i = 0; i < 32; i += 4) {
-                float4 v = owns_srow ? *reinterpret_cast<const float4*>(src + c0 + i)
-                                     : make_float4(0.f, 0.f, 0.f, 0.f);
-                r[i] = __float_as_uint(v.x); r[i + 1] = __float_as_uint(v.y);
-                r[i + 2] = __float_as_uint(v.z); r[i + 3] = __float_as_uint(v.w);
-            }
-            if (MODE == MODE_CAUSAL) tmem_st32(tmem + lane_base + colS + c0, r);
-            if (MODE != MODE_STATE && owns_srow) write_sb(r, c0);
+        for (int i = 0; i < QW; i += 4) {
+            float4 v = owns_srow ? *reinterpret_cast<const float4*>(src + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+            r[i] = __float_as_uint(v.x); r[i + 1] = __float_as_uint(v.y);
+            r[i + 2] = __float_as_uint(v.z); r[i + 3] = __float_as_uint(v.w);
         }
-        if (MODE == MODE_CAUSAL) tmem_wait_st();
+        if (MODE == MODE_CAUSAL) { tmem_stq<QW>(tmem + lane_base + colS + cq * QW, r); tmem_wait_st(); }
+        if (MODE != MODE_STATE && owns_srow) write_sb(r, cq * QW);
         fence_proxy_async();
     }
     tc_fence_before();
@@ -294,18 +305,25 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         // ------------------------------------------------------------------ control thread
         if (lane == 0 && n_chunks > 0) {
             bool alive = true;
-            auto issue_loads = [&](int c) {
+            auto load_tile = [&](uint32_t dst, const CUtensorMap* tm, uint32_t bar, int row) {
+#pragma unroll
+                for (int hh = 0; hh < NH; ++hh) tma_load_3d(dst + hh * 16384, tm, bar, hh * 64, row, bh);
+            };
+            // Loads of chunk c: part 1 = X and A (and the byte count of the whole stage),
+            // part 2 = Bv (or everything when the stage was not split).
+            auto issue_loads = [&](int c, bool part1, bool part2) {
                 const int s = c % NST;
                 const uint32_t bar = bar_full + 8 * s;
                 const int row = chunk_row(c);
-                mbar_expect_tx(bar, L::kTilesPerStage * L::kTile);
-#pragma unroll
-                for (int hh = 0; hh < NH; ++hh) {
-                    if (L::kHasX) tma_load_3d(stage_x(s) + hh * 16384, &tmX, bar, hh * 64, row, bh);
-                    if (L::kHasAB) {
-                        tma_load_3d(stage_a(s) + hh * 16384, &tmA, bar, hh * 64, row, bh);
-                        tma_load_3d(stage_b(s) + hh * 16384, &tmB, bar, hh * 64, row, bh);
+                if (part1) mbar_expect_tx(bar, L::kTilesPerStage * L::kTile);
+                if (L::kHasAB) {
+                    if (part1) {
+                        if (L::kHasX) load_tile(stage_x(s), &tmX, bar, row);
+                        load_tile(stage_a(s), &tmA, bar, row);
                     }
+                    if (part2) load_tile(stage_b(s), &tmB, bar, row);
+                } else if (part2) {
+                    load_tile(stage_x(s), &tmX, bar, row);
                 }
             };
             auto wait = [&](uint32_t bar, uint32_t parity) {
@@ -338,21 +356,15 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     tc_commit(bar_o_full + 8 * (c & 1));
                 }
             };
-            // Reload the stage of chunk c with chunk c + NST once nothing reads it any more.
-            auto refill = [&](int c) {
-                if (c + NST >= n_chunks) return;
-                if (MODE == MODE_STATE) {
-                    if (!wait(bar_s_full + 8 * (c & 1), (c >> 1) & 1)) return;
-                } else {
-                    if (!wait(bar_o_full + 8 * (c & 1), (c >> 1) & 1)) return;
-                    if (with_proj && L::kProjInA && !wait(bar_e_done + 8 * (c & 1), (c >> 1) & 1)) return;
-                }
-                issue_loads(c + NST);
-            };
-            for (int c = 0; c < NST && c < n_chunks; ++c) issue_loads(c);
+            // The stage of chunk c is refilled with chunk c + NST in two steps when possible:
+            // X and A as soon as the last MMA that reads the stage has completed, Bv (the
+            // output staging slot) after the chunk's output store has drained.
+            const bool split_refill = MODE == MODE_CAUSAL && !(with_proj && L::kProjInA);
+            for (int c = 0; c < NST && c < n_chunks; ++c) issue_loads(c, true, true);
             batch1(0);
             for (int c = 0; c < n_chunks && alive; ++c) {
                 const int s = c % NST;
+                const bool more = c + NST < n_chunks;
                 COTT_STAMP(0);
                 if (with_proj) {
                     // The buffer is free once the state update has read the A slot (d = 128
@@ -361,9 +373,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     else if (c >= 1) { if (!wait(bar_e_done + 8 * ((c - 1) & 1), ((c - 1) >> 1) & 1)) break; }
                     const uint32_t proj_u = L::kProjInA ? stage_a(s) : base + L::kOffProj;
                     mbar_expect_tx(bar_proj, L::kTile);
-#pragma unroll
-                    for (int hh = 0; hh < NH; ++hh)
-                        tma_load_3d(proj_u + hh * 16384, &tmP, bar_proj, hh * 64, chunk_row(c), bh);
+                    load_tile(proj_u, &tmP, bar_proj, chunk_row(c));
                 }
                 if (MODE == MODE_CAUSAL) {
                     if (!wait(bar_pt_ready, c & 1)) break;
@@ -373,14 +383,35 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     tc_commit(bar_o_full + 8 * (c & 1));
                 }
                 COTT_STAMP(2);
-                const bool refill_late = with_proj && L::kProjInA;   // stage holds the proj tile
-                if (!refill_late) refill(c);
+                if (MODE == MODE_STATE) {
+                    if (more) { if (!wait(bar_s_full + 8 * (c & 1), (c >> 1) & 1)) break; issue_loads(c + NST, true, true); }
+                    if (c + 1 < n_chunks) batch1(c + 1);
+                    continue;
+                }
+                if (split_refill && more) {
+                    if (!wait(bar_o_full + 8 * (c & 1), (c >> 1) & 1)) break;
+                    issue_loads(c + NST, true, false);
+                }
                 COTT_STAMP(3);
-                if (c + 1 < n_chunks) batch1(c + 1);
+                if (c + 1 < n_chunks) { batch1(c + 1); if (!alive) break; }
                 COTT_STAMP(4);
-                if (refill_late) refill(c);
+                // Output rows staged by the workers: store them, then finish the refill.
+                if (!wait(bar_e_done + 8 * (c & 1), (c >> 1) & 1)) break;
+                {
+                    const uint32_t src = base + s * L::kStage + L::kOffOut;
+#pragma unroll
+                    for (int hh = 0; hh < NH; ++hh)
+                        tma_store_3d(&tmO, src + hh * 16384, hh * 64, chunk_row(c), bh);
+                    tma_store_commit();
+                }
                 COTT_STAMP(5);
+                if (more) {
+                    tma_store_wait_read0();
+                    issue_loads(c + NST, !split_refill, true);
+                }
+                COTT_STAMP(6);
             }
+            tma_store_wait_all0();
         }
     } else {
         // ------------------------------------------------------------------ row workers
@@ -389,12 +420,17 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             if (alive && !wait_or_abort(bar, parity, abort_flag)) alive = false;
             return alive;
         };
-        // Norm-phase mapping: lanes l and l^16 share a row (two column halves).
-        const int nrow = warp * 16 + (lane & 15), nhalf = lane >> 4;
-        constexpr int NC = D / 16;                    // 16-byte chunks in half a row
-        auto tile_half_ptr = [&](uint8_t* tile, int j) {
-            const int ch = nhalf * NC + j;            // chunk index within the row
+        // Norm-phase mapping: lanes l, l^8, l^16, l^24 share a row (four column quarters).
+        const int nrow = warp * 8 + (lane & 7), nq = lane >> 3;
+        constexpr int NC = D / 32;                    // 16-byte chunks in a quarter row
+        auto tile_q_ptr = [&](uint8_t* tile, int j) {
+            const int ch = nq * NC + j;               // chunk index within the row
             return tile + (ch >> 3) * 16384 + swz(nrow, ch & 7);
+        };
+        auto quad_sum = [&](float v) {
+            v += __shfl_xor_sync(0xffffffffu, v, 8);
+            v += __shfl_xor_sync(0xffffffffu, v, 16);
+            return v;
         };
         // Row norms of chunk c: the contraction-side operand is normalised in place; the X
         // row scale (times c) is left in rx_buf[c % NST] for the output epilogue.
@@ -405,12 +441,12 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             uint4 wx[NC], wn[NC];
             if (L::kHasX && p.x_norm) {
 #pragma unroll
-                for (int j = 0; j < NC; ++j) wx[j] = *reinterpret_cast<const uint4*>(tile_half_ptr(st + L::kOffX, j));
+                for (int j = 0; j < NC; ++j) wx[j] = *reinterpret_cast<const uint4*>(tile_q_ptr(st + L::kOffX, j));
             }
             uint8_t* nt = st + (p.norm_bv ? L::kOffB : L::kOffA);
             if (L::kHasAB) {
 #pragma unroll
-                for (int j = 0; j < NC; ++j) wn[j] = *reinterpret_cast<const uint4*>(tile_half_ptr(nt, j));
+                for (int j = 0; j < NC; ++j) wn[j] = *reinterpret_cast<const uint4*>(tile_q_ptr(nt, j));
             }
             if (L::kHasX) {
                 float rx = cfac;
@@ -418,18 +454,16 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
                     for (int j = 0; j < NC; j += 2) { sumsq8(wx[j], a0, a1); sumsq8(wx[j + 1], a2, a3); }
-                    float ss = (a0 + a1) + (a2 + a3);
-                    ss += __shfl_xor_sync(0xffffffffu, ss, 16);
+                    const float ss = quad_sum((a0 + a1) + (a2 + a3));
                     rx = cfac / fmaxf(sqrtf(ss), kEps);
                 }
-                if (nhalf == 0) rx_buf[(c % NST) * 128 + nrow] = rx;
+                if (nq == 0) rx_buf[(c % NST) * 128 + nrow] = rx;
             }
             if (L::kHasAB) {
                 float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
                 for (int j = 0; j < NC; j += 2) { sumsq8(wn[j], a0, a1); sumsq8(wn[j + 1], a2, a3); }
-                float ss = (a0 + a1) + (a2 + a3);
-                ss += __shfl_xor_sync(0xffffffffu, ss, 16);
+                const float ss = quad_sum((a0 + a1) + (a2 + a3));
                 const float r = 1.0f / fmaxf(sqrtf(ss), kEps);
 #pragma unroll
                 for (int j = 0; j < NC; ++j) {
@@ -441,7 +475,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                         float2 f = __bfloat1622float2(e[i]);
                         ow[i] = pack_bf16(f.x * r, f.y * r);
                     }
-                    *reinterpret_cast<uint4*>(tile_half_ptr(nt, j)) = o;
+                    *reinterpret_cast<uint4*>(tile_q_ptr(nt, j)) = o;
                 }
                 fence_proxy_async();
             }
@@ -456,20 +490,18 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             if (MODE == MODE_CAUSAL) {
                 // Masked scores -> bf16 operand P~ (both MMAs that read X are done).  Forward:
                 // row i keeps columns j <= i (diagonal kept, Eq. 6); backward in time: j >= i.
-                // Per 32 x 32 block of this warp the mask is all-keep, all-zero, or (on the
-                // diagonal) a triangle: the first two cases are warp-uniform.
+                // This warp owns the 32 x 32 block (row block q, column block cq): all-keep,
+                // all-zero, or (q == cq) a triangle; the first two cases are warp-uniform.
                 COTT_STAMP(0);
                 if (!wait(bar_p_full, c & 1)) break;
                 tc_fence_after();
                 COTT_STAMP(1);
-#pragma unroll
-                for (int sbk = 0; sbk < 2; ++sbk) {
-                    const int cb = 2 * hf + sbk;      // 32-column block index; row block index is q
-                    const bool keep_all = p.reverse ? (cb > q) : (cb < q);
-                    const bool diag = cb == q;
+                {
+                    const bool keep_all = p.reverse ? (cq > q) : (cq < q);
+                    const bool diag = cq == q;
                     uint32_t r[32];
                     if (keep_all || diag) {
-                        tmem_ld32(tmem + lane_base + colP + cb * 32, r);
+                        tmem_ld32(tmem + lane_base + colP + cq * 32, r);
                         tmem_wait_ld();
                         if (diag) {
 #pragma unroll
@@ -484,7 +516,8 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     }
 #pragma unroll
                     for (int i = 0; i < 32; i += 8)
-                        *reinterpret_cast<uint4*>(pt + hf * 16384 + swz(arow, sbk * 4 + (i >> 3))) = pack8(&r[i]);
+                        *reinterpret_cast<uint4*>(pt + (cq >> 1) * 16384 + swz(arow, (cq & 1) * 4 + (i >> 3))) =
+                            pack8(&r[i]);
                 }
                 COTT_STAMP(2);
                 fence_proxy_async();
@@ -494,13 +527,10 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 if (c + 1 < n_chunks) {
                     if (!wait(bar_s_full + 8 * (c & 1), (c >> 1) & 1)) break;
                     tc_fence_after();
-#pragma unroll
-                    for (int c0 = hf * HW; c0 < (hf + 1) * HW; c0 += 32) {
-                        uint32_t r[32];
-                        tmem_ld32(tmem + lane_base + colS + c0, r);
-                        tmem_wait_ld();
-                        if (owns_srow) write_sb(r, c0);
-                    }
+                    uint32_t r[QW];
+                    tmem_ldq<QW>(tmem + lane_base + colS + cq * QW, r);
+                    tmem_wait_ld();
+                    if (owns_srow) write_sb(r, cq * QW);
                     fence_proxy_async();
                     tc_fence_before();
                     mbar_arrive(bar_sb_ready);
@@ -516,105 +546,95 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 continue;
             }
 
-            // ---- output epilogue of chunk c: straight from the accumulator to global memory
+            // ---- output epilogue of chunk c: accumulator -> bf16 rows in the staging slot
             if (!wait(bar_o_full + 8 * (c & 1), (c >> 1) & 1)) break;
             tc_fence_after();
             COTT_STAMP(5);
-            const uint32_t tO = tmem + lane_base + colO0 + (c & 1) * D;
+            const uint32_t tO = tmem + lane_base + colO0 + (c & 1) * D + cq * QW;
             const float rx = rx_buf[(c % NST) * 128 + arow];
+            uint32_t r[QW];
+            tmem_ldq<QW>(tO, r);
+            tmem_wait_ld();
+            tc_fence_before();
+            mbar_arrive(bar_o_free + 8 * (c & 1));
             float coef = 0.f, rp = 1.f;
             const uint8_t* proj = L::kProjInA ? (st + L::kOffA) : (gbase + L::kOffProj);
+            uint4 pw[QW / 8];
             if (with_proj) {
                 if (!wait(bar_proj, c & 1)) break;
-                // <p, acc> and ||p||^2 over the whole row (both column-half threads compute
-                // the same sums; the proj tile is read-only).
+                // Per-row <p, acc> and ||p||^2: each of the four column-quarter threads sums its
+                // part; the parts meet in shared memory.
+                float2* xch = reinterpret_cast<float2*>(L::kProjInA ? (st + L::kOffX)
+                                                                    : (gbase + L::kOffProj + L::kTile));
                 float ss0 = 0.f, ss1 = 0.f, dp0 = 0.f, dp1 = 0.f;
 #pragma unroll
-                for (int c0 = 0; c0 < D; c0 += 32) {
-                    uint32_t r[32];
-                    tmem_ld32(tO + c0, r);
-                    tmem_wait_ld();
+                for (int i = 0; i < QW; i += 8) {
+                    const int col = cq * QW + i;
+                    pw[i >> 3] = *reinterpret_cast<const uint4*>(proj + (col >> 6) * 16384 +
+                                                                 swz(arow, (col & 63) >> 3));
+                    const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&pw[i >> 3]);
 #pragma unroll
-                    for (int i = 0; i < 32; i += 8) {
-                        const int col = c0 + i;
-                        uint4 w = *reinterpret_cast<const uint4*>(proj + (col >> 6) * 16384 +
-                                                                  swz(arow, (col & 63) >> 3));
-                        const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&w);
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            float2 f = __bfloat1622float2(e[j]);
-                            ss0 = fmaf(f.x, f.x, ss0); ss1 = fmaf(f.y, f.y, ss1);
-                            dp0 = fmaf(f.x, __uint_as_float(r[i + 2 * j]), dp0);
-                            dp1 = fmaf(f.y, __uint_as_float(r[i + 2 * j + 1]), dp1);
-                        }
+                    for (int j = 0; j < 4; ++j) {
+                        float2 f = __bfloat1622float2(e[j]);
+                        ss0 = fmaf(f.x, f.x, ss0); ss1 = fmaf(f.y, f.y, ss1);
+                        dp0 = fmaf(f.x, __uint_as_float(r[i + 2 * j]), dp0);
+                        dp1 = fmaf(f.y, __uint_as_float(r[i + 2 * j + 1]), dp1);
                     }
                 }
-                const float ss = ss0 + ss1, dp = dp0 + dp1;
+                xch[cq * 128 + arow] = make_float2(ss0 + ss1, dp0 + dp1);
+                mbar_arrive(bar_xch);
+                if (!wait(bar_xch, c & 1)) break;
+                const float2 e0 = xch[arow], e1 = xch[128 + arow], e2 = xch[256 + arow], e3 = xch[384 + arow];
+                const float ss = (e0.x + e1.x) + (e2.x + e3.x), dp = (e0.y + e1.y) + (e2.y + e3.y);
                 if (p.epilogue == EPI_PROJ) {
                     // g = rx * acc;  out = (g - p^ <p^, g>) / max(||p||, eps); clamped branch: g / eps
                     const float nrm = sqrtf(ss);
                     rp = 1.0f / fmaxf(nrm, kEps);
                     coef = nrm > kEps ? dp * rx * rp * rp : 0.f;
-                } else if (hf == 0) {
+                } else if (cq == 0) {
                     dm_acc += dp * rx / cfac;  // <dV', v> with dV' = (rx / c) * acc, once per row
                 }
             }
-            // This thread's HW columns: scale, (project,) round to bf16, store (one full
-            // 64-byte or 128-byte run of the output row per thread).
-            const int grow = chunk_row(c) + arow;
-            __nv_bfloat16* orow = static_cast<__nv_bfloat16*>(p.out) + ((size_t)bh * p.N + grow) * D;
+            // Scale, (project,) round to bf16, stage for the TMA store.
+            uint8_t* so = st + L::kOffOut;
 #pragma unroll
-            for (int c0 = hf * HW; c0 < (hf + 1) * HW; c0 += 32) {
-                uint32_t r[32];
-                tmem_ld32(tO + c0, r);
-                tmem_wait_ld();
+            for (int i = 0; i < QW; i += 8) {
+                const int col = cq * QW + i;
+                float v[8];
 #pragma unroll
-                for (int i = 0; i < 32; i += 8) {
-                    const int col = c0 + i;
-                    float v[8];
+                for (int j = 0; j < 8; ++j) v[j] = __uint_as_float(r[i + j]) * rx;
+                if (with_proj && p.epilogue == EPI_PROJ) {
+                    const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&pw[i >> 3]);
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) v[j] = __uint_as_float(r[i + j]) * rx;
-                    if (with_proj && p.epilogue == EPI_PROJ) {
-                        uint4 w = *reinterpret_cast<const uint4*>(proj + (col >> 6) * 16384 +
-                                                                  swz(arow, (col & 63) >> 3));
-                        const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&w);
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            float2 f = __bfloat1622float2(e[j]);
-                            v[2 * j] = (v[2 * j] - f.x * coef) * rp;
-                            v[2 * j + 1] = (v[2 * j + 1] - f.y * coef) * rp;
-                        }
+                    for (int j = 0; j < 4; ++j) {
+                        float2 f = __bfloat1622float2(e[j]);
+                        v[2 * j] = (v[2 * j] - f.x * coef) * rp;
+                        v[2 * j + 1] = (v[2 * j + 1] - f.y * coef) * rp;
                     }
-                    uint4 w;
-                    w.x = pack_bf16(v[0], v[1]); w.y = pack_bf16(v[2], v[3]);
-                    w.z = pack_bf16(v[4], v[5]); w.w = pack_bf16(v[6], v[7]);
-                    if (grow < p.N) *reinterpret_cast<uint4*>(orow + col) = w;
                 }
+                uint4 w;
+                w.x = pack_bf16(v[0], v[1]); w.y = pack_bf16(v[2], v[3]);
+                w.z = pack_bf16(v[4], v[5]); w.w = pack_bf16(v[6], v[7]);
+                *reinterpret_cast<uint4*>(so + (col >> 6) * 16384 + swz(arow, (col & 63) >> 3)) = w;
             }
-            tc_fence_before();
-            mbar_arrive(bar_o_free + 8 * (c & 1));
+            fence_proxy_async();
             mbar_arrive(bar_e_done + 8 * (c & 1));
             COTT_STAMP(6);
         }
 
         if (MODE == MODE_STATE && alive && p.state_out != nullptr) {
-            // Partial state of this group, fp32, unscaled.
-            {
-                tc_fence_after();
-                float* dst = p.state_out + ((size_t)bh * p.n_groups + g) * D * D + (size_t)srow * D;
+            // Partial state of this group, fp32, unscaled (every state update was waited for).
+            tc_fence_after();
+            float* dst = p.state_out + ((size_t)bh * p.n_groups + g) * D * D + (size_t)srow * D + cq * QW;
+            uint32_t r[QW];
+            tmem_ldq<QW>(tmem + lane_base + colS + cq * QW, r);
+            tmem_wait_ld();
+            if (owns_srow) {
 #pragma unroll
-                for (int c0 = hf * HW; c0 < (hf + 1) * HW; c0 += 32) {
-                    uint32_t r[32];
-                    tmem_ld32(tmem + lane_base + colS + c0, r);
-                    tmem_wait_ld();
-                    if (owns_srow) {
-#pragma unroll
-                        for (int i = 0; i < 32; i += 4)
-                            *reinterpret_cast<float4*>(dst + c0 + i) =
-                                make_float4(__uint_as_float(r[i]), __uint_as_float(r[i + 1]),
-                                            __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
-                    }
-                }
+                for (int i = 0; i < QW; i += 4)
+                    *reinterpret_cast<float4*>(dst + i) =
+                        make_float4(__uint_as_float(r[i]), __uint_as_float(r[i + 1]),
+                                    __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
             }
         }
         if (MODE != MODE_STATE && p.dm_partial != nullptr) {
@@ -627,13 +647,11 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     tc_fence_before();
     __syncthreads();
     if (MODE != MODE_STATE && p.dm_partial != nullptr && tid == 0 && !*abort_flag) {
-        // Fixed-order reduction of <dV', V> over the CTA.
-        p.dm_partial[(size_t)bh * p.n_groups + g] =
-            ((dm_red[0] + dm_red[1]) + (dm_red[2] + dm_red[3])) +
-            ((dm_red[4] + dm_red[5]) + (dm_red[6] + dm_red[7]));
+        // Fixed-order reduction of <dV', V> over the CTA (only the cq == 0 warps hold sums).
+        p.dm_partial[(size_t)bh * p.n_groups + g] = (dm_red[0] + dm_red[1]) + (dm_red[2] + dm_red[3]);
     }
     if (tid == 0 && *abort_flag) atomicExch(p.status, 1);
-    if (warp == 8) tmem_dealloc(tmem, kTmemCols);
+    if (is_ctrl) tmem_dealloc(tmem, kTmemCols);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
@@ -676,13 +694,13 @@ cudaError_t launch_mode(const CUtensorMap* tm, const TcWalkParams& p, int BH, cu
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             Smem<D, MODE>::dyn_bytes(true));
+                                             Smem<D, MODE>::dyn_bytes(MODE != MODE_STATE));
         if (e != cudaSuccess) return e;
         configured = true;
     }
     const bool with_proj = (MODE != MODE_STATE) && (p.epilogue != EPI_PLAIN);
     kern<<<dim3((unsigned)(BH * p.n_groups)), kTcThreads, Smem<D, MODE>::dyn_bytes(with_proj), st>>>(
-        tm[0], tm[1], tm[2], tm[3], p);
+        tm[0], tm[1], tm[2], tm[3], tm[4], p);
     note_launch();
     return cudaGetLastError();
 }
@@ -693,14 +711,13 @@ cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cuda
     const int BH = B * H;
     // Unused operands still need a valid map: point them at a tensor that exists.
     const void* any = a.x ? a.x : a.a;
-    const void* ptrs[4] = {a.x ? a.x : any, a.a ? a.a : any, a.bv ? a.bv : any,
-                           a.proj ? a.proj : any};
-    CUtensorMap tm[4];
-    for (int i = 0; i < 4; ++i)
+    const void* ptrs[5] = {a.x ? a.x : any, a.a ? a.a : any, a.bv ? a.bv : any,
+                           a.proj ? a.proj : any, a.out ? a.out : any};
+    CUtensorMap tm[5];
+    for (int i = 0; i < 5; ++i)
         if (!make_tile_map(&tm[i], ptrs[i], BH, N, d)) return cudaErrorInvalidValue;
     TcWalkParams p;
     p.init = a.init; p.state_out = a.state_out; p.dm_partial = a.dm_partial; p.status = a.status;
-    p.out = a.out;
     p.m = a.m; p.seq_len = a.seq_len; p.seq_len_scalar = a.seq_len_scalar;
     p.H = H; p.N = N; p.group = a.group; p.n_groups = a.n_groups;
     p.norm_bv = a.norm_bv; p.x_norm = a.x_norm; p.epilogue = a.epilogue; p.reverse = a.reverse;
