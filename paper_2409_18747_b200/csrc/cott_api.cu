@@ -53,11 +53,16 @@ static bool make_plan(int op, cott_dtype dt, int B, int H, int N, int d, int cau
     p->path = (tc_ok && env_int("COTT_FORCE_PATH", 1) != 0) ? 1 : 0;
     int group;
     if (p->path == 1) {
-        // One CTA per group and per SM: take the largest group that still gives every SM a CTA.
+        // One CTA per (b,h) and group, one CTA per SM.  Measured on B200: fewer, longer
+        // groups win (per-CTA set-up and the per-group state traffic shrink) as long as
+        // about every SM still gets a CTA, and a single group per (b,h) needs no partial-state
+        // pass at all.  So: as many groups per (b,h) as fit in one wave (rounded down), each a
+        // multiple of the 128-token chunk, at most 4096 tokens.
         p->chunk = 128;
-        const long slots = 148L;
-        group = 2048;
-        while (group > 128 && BH * ((N + group - 1) / group) < slots) group >>= 1;
+        const long per_head = BH >= 148 ? 1 : 148 / BH;
+        long g = (N + per_head - 1) / per_head;
+        g = (g + 127) / 128 * 128;
+        group = (int)(g > 4096 ? 4096 : g);
     } else {
         p->chunk = 16;
         group = 1024;
@@ -136,8 +141,9 @@ static cott_status run_tc_stream(TcWalkArgs t, const Plan& p, int B, int H, int 
     a.state_out = states; a.dm_partial = nullptr; a.epilogue = EPI_PLAIN;
     COTT_CUDA(launch_tc_walk(a, B, H, N, d, st));
     const int mode = !causal ? SCAN_TOTAL : (t.reverse ? SCAN_SUFFIX : SCAN_PREFIX);
-    COTT_CUDA(launch_scan(states, total_out, B * H, p.n_groups, d, mode, st, sp->m, sp->seq_len,
-                          sp->seq_len_scalar, H, N));
+    if (causal || p.n_groups > 1 || total_out)  // one bidirectional group: its partial is the total
+        COTT_CUDA(launch_scan(states, total_out, B * H, p.n_groups, d, mode, st, sp->m, sp->seq_len,
+                              sp->seq_len_scalar, H, N));
     t.mode = causal ? 1 : 2; t.init = states; t.state_out = nullptr;
     COTT_CUDA(launch_tc_walk(t, B, H, N, d, st));
     return COTT_OK;

@@ -334,13 +334,19 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(const T* q, const T* k
     const float4 vv = *reinterpret_cast<const float4*>(&vp[c4 * 4]);
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float4* S = reinterpret_cast<float4*>(state + (size_t)bh * D * D);
-#pragma unroll 4
-    for (int a = r0; a < D; a += RG) {
-        float4 sv = S[(size_t)a * V4 + c4];
+    // All loads of this thread's state elements are issued before the first use, so the
+    // whole 16 KB - 64 KB state of the (b,h) pair is in flight at once.
+    constexpr int NIT = D / RG;
+    float4 sv[NIT];
+#pragma unroll
+    for (int i = 0; i < NIT; ++i) sv[i] = S[(size_t)(r0 + i * RG) * V4 + c4];
+#pragma unroll
+    for (int i = 0; i < NIT; ++i) {
+        const int a = r0 + i * RG;
         const float ka = kh[a], qa = qh[a];
-        sv.x += ka * vv.x; sv.y += ka * vv.y; sv.z += ka * vv.z; sv.w += ka * vv.w;
-        S[(size_t)a * V4 + c4] = sv;
-        acc.x += qa * sv.x; acc.y += qa * sv.y; acc.z += qa * sv.z; acc.w += qa * sv.w;
+        sv[i].x += ka * vv.x; sv[i].y += ka * vv.y; sv[i].z += ka * vv.z; sv[i].w += ka * vv.w;
+        S[(size_t)a * V4 + c4] = sv[i];
+        acc.x += qa * sv[i].x; acc.y += qa * sv[i].y; acc.z += qa * sv[i].z; acc.w += qa * sv[i].w;
     }
     *reinterpret_cast<float4*>(&red[r0][c4 * 4]) = acc;
     __syncthreads();

@@ -437,6 +437,10 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         auto norm_phase = [&](int c) {
             const int s = c % NST;
             if (!wait(bar_full + 8 * s, (c / NST) & 1)) return;
+#ifdef COTT_TIMING
+            if (blockIdx.x == 0 && threadIdx.x == 0 && (c == 3 || c == 4))
+                reinterpret_cast<unsigned long long*>(p.status)[1 + (c - 3) * 7 + 4] = globaltimer_ns();
+#endif
             uint8_t* st = gbase + s * L::kStage;
             uint4 wx[NC], wn[NC];
             if (L::kHasX && p.x_norm) {
@@ -538,7 +542,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 COTT_STAMP(3);
             }
             if (c + 1 < n_chunks) { norm_phase(c + 1); if (!alive) break; }
-            COTT_STAMP(4);
+            COTT_STAMP(5);
             if (MODE == MODE_STATE) {
                 // Follow every state update (a parity names one chunk only if no phase is
                 // skipped); after the last one the accumulator holds the group's state.
@@ -549,7 +553,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             // ---- output epilogue of chunk c: accumulator -> bf16 rows in the staging slot
             if (!wait(bar_o_full + 8 * (c & 1), (c >> 1) & 1)) break;
             tc_fence_after();
-            COTT_STAMP(5);
+            COTT_STAMP(6);
             const uint32_t tO = tmem + lane_base + colO0 + (c & 1) * D + cq * QW;
             const float rx = rx_buf[(c % NST) * 128 + arow];
             uint32_t r[QW];
@@ -619,7 +623,6 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             }
             fence_proxy_async();
             mbar_arrive(bar_e_done + 8 * (c & 1));
-            COTT_STAMP(6);
         }
 
         if (MODE == MODE_STATE && alive && p.state_out != nullptr) {
