@@ -69,6 +69,18 @@ const char* cott_last_cuda_error(void);
 unsigned long long cott_launch_count(void);
 
 /*
+ * Per-launch timing of the tensor-core walk kernels, for benchmarks.  cott_profile_enable(n)
+ * with n > 0 starts recording a pair of library-owned CUDA events around each of the next n
+ * (at most 256) walk-kernel launches; n <= 0 stops.  cott_profile_read waits for the recorded
+ * launches and writes their durations in milliseconds to ms[] and their kind to kinds[]
+ * (0 = partial-state pass, 1 = causal walk, 2 = read-out); both are host arrays of `cap`
+ * entries.  Returns the number of entries written, or -1 on a CUDA error.  Not thread-safe
+ * against concurrent library calls; leave it off outside measurements.
+ */
+cott_status cott_profile_enable(int max_launches);
+int cott_profile_read(float* ms, int* kinds, int cap);
+
+/*
  * Bytes of device scratch the given call needs (0 is possible).  `op` is a cott_op.
  * The workspace must be 256-byte aligned.  Returns (size_t)-1 for unsupported arguments.
  */

@@ -55,6 +55,10 @@ def _load():
     lib.cott_status_string.argtypes = [ci]
     lib.cott_last_cuda_error.restype = ctypes.c_char_p
     lib.cott_launch_count.restype = ctypes.c_ulonglong
+    lib.cott_profile_enable.restype = ci
+    lib.cott_profile_enable.argtypes = [ci]
+    lib.cott_profile_read.restype = ci
+    lib.cott_profile_read.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ci), ci]
     lib.cott_workspace_bytes.restype = cs
     lib.cott_workspace_bytes.argtypes = [ci, ci, ci, ci, ci, ci, ci]
     lib.cott_query_plan.restype = ci
@@ -210,6 +214,22 @@ def fwd_bwd_host(q, k, v, d_o, m, o, dq, dk, dv, dm, causal=True, seq_len=None, 
 
 def launch_count() -> int:
     return int(_load().cott_launch_count())
+
+
+def profile_enable(max_launches: int) -> None:
+    rc = _load().cott_profile_enable(int(max_launches))
+    if rc != 0:
+        raise CottError(rc, "cott_profile_enable")
+
+
+def profile_read(cap: int = 256):
+    """Returns [(kind, milliseconds), ...] of the walk-kernel launches recorded so far."""
+    ms = (ctypes.c_float * cap)()
+    kinds = (ctypes.c_int * cap)()
+    n = _load().cott_profile_read(ms, kinds, cap)
+    if n < 0:
+        raise CottError(-4, "cott_profile_read")
+    return [(int(kinds[i]), float(ms[i])) for i in range(n)]
 
 
 def last_async_status(workspace: torch.Tensor, stream=None) -> int:

@@ -12,6 +12,27 @@ static thread_local char g_cuda_error[256] = "";
 static std::atomic<unsigned long long> g_launches{0};
 void note_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
 
+// ---- optional per-launch timing (library-owned CUDA events; created on first use)
+static constexpr int kProfMax = 256;
+static cudaEvent_t g_prof_ev[2 * kProfMax];
+static int g_prof_kind[kProfMax];
+static bool g_prof_created = false;
+static std::atomic<int> g_prof_n{-1};   // -1: disabled
+static int g_prof_cap = 0;
+
+int profile_begin_launch(int kind, cudaStream_t st) {
+    int n = g_prof_n.load(std::memory_order_relaxed);
+    if (n < 0 || n >= g_prof_cap) return -1;
+    n = g_prof_n.fetch_add(1);
+    if (n >= g_prof_cap) return -1;
+    g_prof_kind[n] = kind;
+    cudaEventRecord(g_prof_ev[2 * n], st);
+    return n;
+}
+void profile_end_launch(int idx, cudaStream_t st) {
+    if (idx >= 0) cudaEventRecord(g_prof_ev[2 * idx + 1], st);
+}
+
 static cott_status cuda_fail(cudaError_t e, const char* where) {
     snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s", where, cudaGetErrorString(e));
     return COTT_ERR_CUDA;
@@ -250,6 +271,31 @@ const char* cott_status_string(cott_status st) {
 }
 
 const char* cott_last_cuda_error(void) { return g_cuda_error; }
+
+cott_status cott_profile_enable(int max_launches) {
+    if (max_launches <= 0) { g_prof_n.store(-1); return COTT_OK; }
+    if (!g_prof_created) {
+        for (int i = 0; i < 2 * kProfMax; ++i)
+            if (cudaEventCreate(&g_prof_ev[i]) != cudaSuccess) return COTT_ERR_CUDA;
+        g_prof_created = true;
+    }
+    g_prof_cap = max_launches < kProfMax ? max_launches : kProfMax;
+    g_prof_n.store(0);
+    return COTT_OK;
+}
+
+int cott_profile_read(float* ms, int* kinds, int cap) {
+    int n = g_prof_n.load();
+    if (n < 0) return 0;
+    if (n > g_prof_cap) n = g_prof_cap;
+    if (n > cap) n = cap;
+    for (int i = 0; i < n; ++i) {
+        if (cudaEventSynchronize(g_prof_ev[2 * i + 1]) != cudaSuccess) return -1;
+        if (cudaEventElapsedTime(&ms[i], g_prof_ev[2 * i], g_prof_ev[2 * i + 1]) != cudaSuccess) return -1;
+        kinds[i] = g_prof_kind[i];
+    }
+    return n;
+}
 
 unsigned long long cott_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 

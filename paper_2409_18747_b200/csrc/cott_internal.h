@@ -72,6 +72,11 @@ cudaError_t launch_decode(const void* q, const void* k, const void* v, float* st
                           int B, int H, int d, cott_dtype dt, const float* m,
                           const float* seq_len, float seq_len_scalar, cudaStream_t st);
 
+// Optional per-launch timing of the tensor-core walk kernels (cott_profile_enable): returns
+// the index of the event pair to record around the next launch, or -1 when disabled / full.
+int profile_begin_launch(int kind, cudaStream_t st);
+void profile_end_launch(int idx, cudaStream_t st);
+
 // Counts kernel launches issued by this process (reported by cott_launch_count).
 void note_launch(int n = 1);
 

@@ -301,7 +301,9 @@ __global__ void dm_finalize_kernel(const float* dm_partial, float* dm, const flo
 }
 
 // Recurrent decode step (Eq. 8): one CTA per (b,h); the fp32 state streams through once with
-// 128-bit loads and stores, update and read-out fused.
+// 128-bit loads and stores, update and read-out fused.  Every thread first issues all loads
+// of its state elements (the whole state of the pair is then in flight), and only then
+// normalises q and k, so the row norms hide behind the memory latency.
 template <int D, typename T>
 __global__ void __launch_bounds__(kThreads) decode_kernel(const T* q, const T* k, const T* v,
                                                           float* state, T* o, int H,
@@ -309,10 +311,17 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(const T* q, const T* k
                                                           float seq_len_scalar) {
     constexpr int V4 = D / 4;             // float4 per state row
     constexpr int RG = kThreads / V4;     // rows covered per sweep
+    constexpr int NIT = D / RG;
     __shared__ float qh[D], kh[D], vp[D];
     __shared__ __align__(16) float red[RG][D];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int bh = blockIdx.x, b = bh / H, h = bh % H;
+    const int c4 = tid % V4, r0 = tid / V4;
+    float4* S = reinterpret_cast<float4*>(state + (size_t)bh * D * D);
+    float4 sv[NIT];
+#pragma unroll
+    for (int i = 0; i < NIT; ++i) sv[i] = S[(size_t)(r0 + i * RG) * V4 + c4];
+
     const float s_b = seq_len ? seq_len[b] : seq_len_scalar;
     const float c = stab_factor(m[h], s_b);
     if (tid < D) {
@@ -330,16 +339,8 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(const T* q, const T* k
         for (int e = lane; e < D; e += 32) row[e] *= r;
     }
     __syncthreads();
-    const int c4 = tid % V4, r0 = tid / V4;
     const float4 vv = *reinterpret_cast<const float4*>(&vp[c4 * 4]);
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    float4* S = reinterpret_cast<float4*>(state + (size_t)bh * D * D);
-    // All loads of this thread's state elements are issued before the first use, so the
-    // whole 16 KB - 64 KB state of the (b,h) pair is in flight at once.
-    constexpr int NIT = D / RG;
-    float4 sv[NIT];
-#pragma unroll
-    for (int i = 0; i < NIT; ++i) sv[i] = S[(size_t)(r0 + i * RG) * V4 + c4];
 #pragma unroll
     for (int i = 0; i < NIT; ++i) {
         const int a = r0 + i * RG;

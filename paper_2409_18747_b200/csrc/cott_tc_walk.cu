@@ -702,8 +702,10 @@ cudaError_t launch_mode(const CUtensorMap* tm, const TcWalkParams& p, int BH, cu
         configured = true;
     }
     const bool with_proj = (MODE != MODE_STATE) && (p.epilogue != EPI_PLAIN);
+    const int prof = profile_begin_launch(MODE, st);
     kern<<<dim3((unsigned)(BH * p.n_groups)), kTcThreads, Smem<D, MODE>::dyn_bytes(with_proj), st>>>(
         tm[0], tm[1], tm[2], tm[3], tm[4], p);
+    profile_end_launch(prof, st);
     note_launch();
     return cudaGetLastError();
 }
