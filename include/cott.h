@@ -157,6 +157,28 @@ cott_status cott_fwd_bwd_host(const void* q_host, const void* k_host, const void
                               cott_dtype dt, void* arena, size_t arena_bytes, void* stream);
 
 /*
+ * cott_fwd without a caller workspace (the paper has no counterpart: this exists for the way
+ * the library is embedded, not for the method).  It serves callers that cannot obtain device
+ * memory at call time, e.g. a server whose own pool already holds all of HBM, or a loop that
+ * cannot afford the device-wide synchronisation of cudaMalloc / cudaFree.  The scratch is a
+ * fixed 8 MiB array (cott_fwd_noalloc_max_bytes()) compiled into the library, so every GPU
+ * that loads the library gives up that much memory until the process exits.  The call itself
+ * allocates and frees nothing.
+ *   - Arguments as for cott_fwd (no state export); inputs and outputs are still the caller's.
+ *   - Returns COTT_ERR_WORKSPACE when cott_workspace_bytes(COTT_OP_FWD, ...) for this problem
+ *     exceeds the 8 MiB; use cott_fwd with your own workspace then.
+ *   - The first call on each device looks up the array's device address (a host-side set-up
+ *     step); make that first call before starting any stream capture.
+ *   - All calls on a device share the one array: two calls whose kernels may overlap on the
+ *     GPU (different streams, no ordering) race on it.  Calls ordered on one stream are safe;
+ *     nothing needs to be cleared between them.
+ */
+size_t cott_fwd_noalloc_max_bytes(void);
+cott_status cott_fwd_noalloc(const void* q, const void* k, const void* v, void* o, int B, int H,
+                             int N, int d, int causal, cott_dtype dt, const cott_scale_params* sp,
+                             void* stream);
+
+/*
  * Synchronises `stream`, then reads the status word the last call using `workspace` left
  * there: COTT_OK, or COTT_ERR_TIMEOUT if a bounded device-side wait gave up, or COTT_ERR_CUDA
  * if the stream reports an error.

@@ -74,6 +74,9 @@ def _load():
     lib.cott_host_step_arena_bytes.argtypes = [ci] * 6
     lib.cott_fwd_bwd_host.restype = ci
     lib.cott_fwd_bwd_host.argtypes = [vp] * 11 + [ci] * 6 + [vp, cs, vp]
+    lib.cott_fwd_noalloc_max_bytes.restype = cs
+    lib.cott_fwd_noalloc.restype = ci
+    lib.cott_fwd_noalloc.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ctypes.POINTER(_ScaleParams), vp]
     lib.cott_last_async_status.restype = ci
     lib.cott_last_async_status.argtypes = [vp, vp]
     _lib = lib
@@ -152,6 +155,20 @@ def fwd(q, k, v, m, seq_len=None, causal=True, return_state=False, out=None, wor
     if rc != 0:
         raise CottError(rc, "cott_fwd")
     return (o, state) if return_state else o
+
+
+def fwd_noalloc(q, k, v, m, seq_len=None, causal=True, out=None, stream=None):
+    """cott_fwd_noalloc: the forward pass on the library's built-in 8 MiB scratch, for callers
+    that cannot supply a workspace.  Raises CottError(-3) when the problem needs more."""
+    _check_dev(q, k, v, m, seq_len if isinstance(seq_len, torch.Tensor) else None)
+    B, H, N, d = q.shape
+    o = torch.empty_like(q) if out is None else out
+    sp = _scale(m, seq_len)
+    rc = _load().cott_fwd_noalloc(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, H, N, d,
+                                  int(bool(causal)), _dt(q), ctypes.byref(sp), _stream_ptr(stream))
+    if rc != 0:
+        raise CottError(rc, "cott_fwd_noalloc")
+    return o
 
 
 def bwd(q, k, v, d_o, m, seq_len=None, causal=True, workspace=None, stream=None):
