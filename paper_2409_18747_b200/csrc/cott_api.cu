@@ -161,10 +161,15 @@ static cott_status run_tc_stream(TcWalkArgs t, const Plan& p, int B, int H, int 
     a.mode = 0; a.x = nullptr; a.proj = nullptr; a.out = nullptr; a.init = nullptr;
     a.state_out = states; a.dm_partial = nullptr; a.epilogue = EPI_PLAIN;
     COTT_CUDA(launch_tc_walk(a, B, H, N, d, st));
+    // Few groups and no state export: every walk CTA sums the partial states it needs itself
+    // and the scan launch is dropped -- as long as those extra d x d reads (n_groups / 2 of
+    // them on average) stay small against the group's own q, k, v, o bytes.
+    const bool fused_scan = !total_out && p.n_groups <= 8 && (long)p.n_groups * d * 8 <= p.group;
     const int mode = !causal ? SCAN_TOTAL : (t.reverse ? SCAN_SUFFIX : SCAN_PREFIX);
-    if (causal || p.n_groups > 1 || total_out)  // one bidirectional group: its partial is the total
+    if (!fused_scan)
         COTT_CUDA(launch_scan(states, total_out, B * H, p.n_groups, d, mode, st, sp->m, sp->seq_len,
                               sp->seq_len_scalar, H, N));
+    t.init_sum = fused_scan ? 1 : 0;
     t.mode = causal ? 1 : 2; t.init = states; t.state_out = nullptr;
     COTT_CUDA(launch_tc_walk(t, B, H, N, d, st));
     return COTT_OK;

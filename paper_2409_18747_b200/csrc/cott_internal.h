@@ -62,6 +62,7 @@ struct TcWalkArgs {
     const float* m; const float* seq_len; float seq_len_scalar;
     int group; int n_groups;
     int norm_bv; int x_norm; int epilogue; int reverse;
+    int init_sum;   // 1: `init` holds raw partial states; the walk forms its own prefix / suffix / total
 };
 cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cudaStream_t st);
 

@@ -30,7 +30,10 @@ constexpr int kTcThreads = 544;   // 16 row-worker warps + 1 control warp
 constexpr uint64_t kWaitTimeoutNs = 2000000000ull;  // 2 s: far above any legitimate wait
 
 struct TcWalkParams {
-    const float* init;      // [BH, n_groups, d*d] unscaled prefix / suffix / total states, or NULL
+    const float* init;      // [BH, n_groups, d*d] unscaled group states, or NULL
+    int init_sum;           // 0: init holds this group's start state; 1: it holds raw partial
+                            // states, to be summed here over the groups before (after, when
+                            // time runs backward; all, for the read-out) this one
     float* state_out;       // MODE_STATE: [BH, n_groups, d*d] partial states (unscaled)
     float* dm_partial;      // EPI_DV: [BH, n_groups]
     int* status;            // workspace status word
@@ -282,14 +285,37 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
 
     const bool init_state = p.init != nullptr;
     if (init_state && !is_ctrl) {
-        // Initial state of the group: fp32 into TMEM, bf16 copy into shared memory.
-        const float* src = p.init + ((size_t)bh * p.n_groups + g) * D * D + (size_t)srow * D + cq * QW;
+        // Initial state of the group: fp32 into TMEM, bf16 copy into shared memory.  With
+        // init_sum the exclusive prefix (suffix / total) over the groups' partial states is
+        // formed here, in group order, instead of by a separate scan launch.
+        const float* src = p.init + (size_t)bh * p.n_groups * D * D + (size_t)srow * D + cq * QW;
         uint32_t r[QW];
+        if (!p.init_sum) {
+            const float* s0 = src + (size_t)g * D * D;
 #pragma unroll
-        for (int i = 0; i < QW; i += 4) {
-            float4 v = owns_srow ? *reinterpret_cast<const float4*>(src + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-            r[i] = __float_as_uint(v.x); r[i + 1] = __float_as_uint(v.y);
-            r[i + 2] = __float_as_uint(v.z); r[i + 3] = __float_as_uint(v.w);
+            for (int i = 0; i < QW; i += 4) {
+                float4 v = owns_srow ? *reinterpret_cast<const float4*>(s0 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+                r[i] = __float_as_uint(v.x); r[i + 1] = __float_as_uint(v.y);
+                r[i + 2] = __float_as_uint(v.z); r[i + 3] = __float_as_uint(v.w);
+            }
+        } else {
+            float acc[QW];
+#pragma unroll
+            for (int i = 0; i < QW; ++i) acc[i] = 0.f;
+            const int g_lo = (MODE == MODE_READOUT) ? 0 : (p.reverse ? g + 1 : 0);
+            const int g_hi = (MODE == MODE_READOUT) ? p.n_groups : (p.reverse ? p.n_groups : g);
+            if (owns_srow) {
+                for (int gg = g_lo; gg < g_hi; ++gg) {
+                    const float* sg = src + (size_t)gg * D * D;
+#pragma unroll
+                    for (int i = 0; i < QW; i += 4) {
+                        const float4 v = *reinterpret_cast<const float4*>(sg + i);
+                        acc[i] += v.x; acc[i + 1] += v.y; acc[i + 2] += v.z; acc[i + 3] += v.w;
+                    }
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < QW; ++i) r[i] = __float_as_uint(acc[i]);
         }
         if (MODE == MODE_CAUSAL) { tmem_stq<QW>(tmem + lane_base + colS + cq * QW, r); tmem_wait_st(); }
         if (MODE != MODE_STATE && owns_srow) write_sb(r, cq * QW);
@@ -726,6 +752,7 @@ cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cuda
     p.m = a.m; p.seq_len = a.seq_len; p.seq_len_scalar = a.seq_len_scalar;
     p.H = H; p.N = N; p.group = a.group; p.n_groups = a.n_groups;
     p.norm_bv = a.norm_bv; p.x_norm = a.x_norm; p.epilogue = a.epilogue; p.reverse = a.reverse;
+    p.init_sum = a.init_sum;
     if (d == 128) {
         if (a.mode == MODE_STATE) return launch_mode<128, MODE_STATE>(tm, p, BH, st);
         if (a.mode == MODE_CAUSAL) return launch_mode<128, MODE_CAUSAL>(tm, p, BH, st);
