@@ -254,6 +254,10 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot_g;
+    // Everything above touched only this CTA's own resources.  From here on global memory
+    // written by the previous kernel of the stream is read (and its inputs overwritten).
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     const float s_b = p.seq_len ? p.seq_len[b] : (p.seq_len_scalar > 0.f ? p.seq_len_scalar : (float)p.N);
     const float cfac = stab_factor(p.m[h], s_b);
@@ -729,11 +733,23 @@ cudaError_t launch_mode(const CUtensorMap* tm, const TcWalkParams& p, int BH, cu
     }
     const bool with_proj = (MODE != MODE_STATE) && (p.epilogue != EPI_PLAIN);
     const int prof = profile_begin_launch(MODE, st);
-    kern<<<dim3((unsigned)(BH * p.n_groups)), kTcThreads, Smem<D, MODE>::dyn_bytes(with_proj), st>>>(
-        tm[0], tm[1], tm[2], tm[3], tm[4], p);
+    // Programmatic dependent launch: this kernel may start (allocate TMEM, set up barriers,
+    // prefetch tensor maps) while the previous kernel of the stream drains; it waits for that
+    // kernel's memory with griddepcontrol.wait before touching any global data.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(BH * p.n_groups));
+    cfg.blockDim = dim3(kTcThreads);
+    cfg.dynamicSmemBytes = Smem<D, MODE>::dyn_bytes(with_proj);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t le = cudaLaunchKernelEx(&cfg, kern, tm[0], tm[1], tm[2], tm[3], tm[4], p);
     profile_end_launch(prof, st);
     note_launch();
-    return cudaGetLastError();
+    return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 }  // namespace
