@@ -149,7 +149,8 @@ static cott_status run_stream(WalkArgs w, const Plan& p, int BH, int d, cott_dty
 // A causal call with a single group and no state export needs only the walk.
 static cott_status run_tc_stream(TcWalkArgs t, const Plan& p, int B, int H, int N, int d,
                                  int causal, const cott_scale_params* sp, int* status,
-                                 float* states, float* total_out, cudaStream_t st) {
+                                 float* states, float* total_out, cudaStream_t st,
+                                 bool reuse_transposed = false) {
     t.status = status; t.m = sp->m; t.seq_len = sp->seq_len; t.seq_len_scalar = sp->seq_len_scalar;
     t.group = p.group; t.n_groups = p.n_groups;
     if (causal && p.n_groups == 1 && !total_out) {
@@ -157,19 +158,25 @@ static cott_status run_tc_stream(TcWalkArgs t, const Plan& p, int B, int H, int 
         COTT_CUDA(launch_tc_walk(t, B, H, N, d, st));
         return COTT_OK;
     }
-    TcWalkArgs a = t;
-    a.mode = 0; a.x = nullptr; a.proj = nullptr; a.out = nullptr; a.init = nullptr;
-    a.state_out = states; a.dm_partial = nullptr; a.epilogue = EPI_PLAIN;
-    COTT_CUDA(launch_tc_walk(a, B, H, N, d, st));
     // Few groups and no state export: every walk CTA sums the partial states it needs itself
     // and the scan launch is dropped -- as long as those extra d x d reads (n_groups / 2 of
     // them on average) stay small against the group's own q, k, v, o bytes.
     const bool fused_scan = !total_out && p.n_groups <= 8 && (long)p.n_groups * d * 8 <= p.group;
-    const int mode = !causal ? SCAN_TOTAL : (t.reverse ? SCAN_SUFFIX : SCAN_PREFIX);
-    if (!fused_scan)
-        COTT_CUDA(launch_scan(states, total_out, B * H, p.n_groups, d, mode, st, sp->m, sp->seq_len,
-                              sp->seq_len_scalar, H, N));
+    if (!reuse_transposed) {
+        TcWalkArgs a = t;
+        a.mode = 0; a.x = nullptr; a.proj = nullptr; a.out = nullptr; a.init = nullptr;
+        a.state_out = states; a.dm_partial = nullptr; a.epilogue = EPI_PLAIN;
+        COTT_CUDA(launch_tc_walk(a, B, H, N, d, st));
+        const int mode = !causal ? SCAN_TOTAL : (t.reverse ? SCAN_SUFFIX : SCAN_PREFIX);
+        if (!fused_scan)
+            COTT_CUDA(launch_scan(states, total_out, B * H, p.n_groups, d, mode, st, sp->m, sp->seq_len,
+                                  sp->seq_len_scalar, H, N));
+    }
+    // reuse_transposed: `states` already holds, transposed, what this stream needs (raw
+    // partials when the scan is fused, scanned states otherwise) from a sibling stream that
+    // walks in the same direction.
     t.init_sum = fused_scan ? 1 : 0;
+    t.init_transposed = reuse_transposed ? 1 : 0;
     t.mode = causal ? 1 : 2; t.init = states; t.state_out = nullptr;
     COTT_CUDA(launch_tc_walk(t, B, H, N, d, st));
     return COTT_OK;
@@ -223,8 +230,10 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
         if ((rc = run_tc_stream(t, p, B, H, N, d, causal, sp, status, st1, nullptr, st)) != COTT_OK) return rc;
         // dV': backward in time with (K, Q^, dO); rows scale by c / ||k||; <dV', V> for dm
         t.x = k; t.a = q; t.bv = d_o; t.proj = v; t.out = dv;
+        // Its state sum_t q^_t dO_t^T is the transpose of the dK^ stream's sum_t dO_t q^_t^T,
+        // accumulated in the same direction: reuse those group states instead of a third pass.
         t.norm_bv = 0; t.x_norm = 1; t.epilogue = EPI_DV; t.reverse = 1; t.dm_partial = dm_partial;
-        if ((rc = run_tc_stream(t, p, B, H, N, d, causal, sp, status, st2, nullptr, st)) != COTT_OK) return rc;
+        if ((rc = run_tc_stream(t, p, B, H, N, d, causal, sp, status, st1, nullptr, st, true)) != COTT_OK) return rc;
         COTT_CUDA(launch_dm_finalize(dm_partial, dm, sp->m, sp->seq_len, sp->seq_len_scalar, B, H,
                                      p.n_groups, N, st));
         return COTT_OK;

@@ -63,6 +63,7 @@ struct TcWalkArgs {
     int group; int n_groups;
     int norm_bv; int x_norm; int epilogue; int reverse;
     int init_sum;   // 1: `init` holds raw partial states; the walk forms its own prefix / suffix / total
+    int init_transposed;  // 1: `init` holds the transposes of the states this walk starts from
 };
 cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cudaStream_t st);
 

@@ -31,6 +31,7 @@ constexpr uint64_t kWaitTimeoutNs = 2000000000ull;  // 2 s: far above any legiti
 
 struct TcWalkParams {
     const float* init;      // [BH, n_groups, d*d] unscaled group states, or NULL
+    int init_transposed;    // 1: init holds the transposes of the states this walk needs
     int init_sum;           // 0: init holds this group's start state; 1: it holds raw partial
                             // states, to be summed here over the groups before (after, when
                             // time runs backward; all, for the read-out) this one
@@ -292,13 +293,20 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         // Initial state of the group: fp32 into TMEM, bf16 copy into shared memory.  With
         // init_sum the exclusive prefix (suffix / total) over the groups' partial states is
         // formed here, in group order, instead of by a separate scan launch.
-        const float* src = p.init + (size_t)bh * p.n_groups * D * D + (size_t)srow * D + cq * QW;
+        // Element (srow, cq*QW + i) of group gg's state; a transposed source (the state of a
+        // sibling gradient stream, which is this stream's state transposed) is read by columns.
+        const float* src = p.init + (size_t)bh * p.n_groups * D * D;
+        auto load4 = [&](int gg, int i) -> float4 {
+            const float* sg = src + (size_t)gg * D * D;
+            if (!p.init_transposed) return *reinterpret_cast<const float4*>(sg + (size_t)srow * D + cq * QW + i);
+            const float* col = sg + (size_t)(cq * QW + i) * D + srow;
+            return make_float4(col[0], col[D], col[2 * D], col[3 * D]);
+        };
         uint32_t r[QW];
         if (!p.init_sum) {
-            const float* s0 = src + (size_t)g * D * D;
 #pragma unroll
             for (int i = 0; i < QW; i += 4) {
-                float4 v = owns_srow ? *reinterpret_cast<const float4*>(s0 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+                float4 v = owns_srow ? load4(g, i) : make_float4(0.f, 0.f, 0.f, 0.f);
                 r[i] = __float_as_uint(v.x); r[i + 1] = __float_as_uint(v.y);
                 r[i + 2] = __float_as_uint(v.z); r[i + 3] = __float_as_uint(v.w);
             }
@@ -310,10 +318,9 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             const int g_hi = (MODE == MODE_READOUT) ? p.n_groups : (p.reverse ? p.n_groups : g);
             if (owns_srow) {
                 for (int gg = g_lo; gg < g_hi; ++gg) {
-                    const float* sg = src + (size_t)gg * D * D;
 #pragma unroll
                     for (int i = 0; i < QW; i += 4) {
-                        const float4 v = *reinterpret_cast<const float4*>(sg + i);
+                        const float4 v = load4(gg, i);
                         acc[i] += v.x; acc[i + 1] += v.y; acc[i + 2] += v.z; acc[i + 3] += v.w;
                     }
                 }
@@ -373,11 +380,12 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 tc_fence_after();
                 const uint32_t tO = tmem + colO0 + (c & 1) * D;
                 if (MODE == MODE_CAUSAL) {
+                    // The state update of this chunk is issued later, behind P~ Bv, so that
+                    // the workers mask the scores without the tensor core hammering shared
+                    // memory and TMEM at the same time.
                     issue_p<D>(tmem + colP, stage_x(s), stage_a(s));
                     if (acc) issue_xs<D>(tO, stage_x(s), sb);
                     tc_commit(bar_p_full);
-                    issue_atb<D>(tmem + colS, stage_a(s), stage_b(s), acc);
-                    tc_commit(bar_s_full + 8 * (c & 1));
                 } else if (MODE == MODE_STATE) {
                     issue_atb<D>(tmem + colS, stage_a(s), stage_b(s), acc);
                     tc_commit(bar_s_full + 8 * (c & 1));
@@ -396,21 +404,30 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 const int s = c % NST;
                 const bool more = c + NST < n_chunks;
                 COTT_STAMP(0);
-                if (with_proj) {
-                    // The buffer is free once the state update has read the A slot (d = 128
-                    // causal walk) or the previous chunk's epilogue has finished (dedicated).
-                    if (L::kProjInA) { if (!wait(bar_s_full + 8 * (c & 1), (c >> 1) & 1)) break; }
-                    else if (c >= 1) { if (!wait(bar_e_done + 8 * ((c - 1) & 1), ((c - 1) >> 1) & 1)) break; }
+                auto load_proj = [&]() {
                     const uint32_t proj_u = L::kProjInA ? stage_a(s) : base + L::kOffProj;
                     mbar_expect_tx(bar_proj, L::kTile);
                     load_tile(proj_u, &tmP, bar_proj, chunk_row(c));
+                };
+                if (with_proj && !L::kProjInA) {
+                    // Dedicated buffer: free once the previous chunk's epilogue has finished.
+                    if (c >= 1 && !wait(bar_e_done + 8 * ((c - 1) & 1), ((c - 1) >> 1) & 1)) break;
+                    load_proj();
                 }
                 if (MODE == MODE_CAUSAL) {
                     if (!wait(bar_pt_ready, c & 1)) break;
                     COTT_STAMP(1);
                     tc_fence_after();
-                    issue_pb<D>(tmem + colO0 + (c & 1) * D, stage_pt(s), stage_b(s), init_state || c > 0);
+                    const bool acc = init_state || c > 0;
+                    issue_pb<D>(tmem + colO0 + (c & 1) * D, stage_pt(s), stage_b(s), acc);
                     tc_commit(bar_o_full + 8 * (c & 1));
+                    issue_atb<D>(tmem + colS, stage_a(s), stage_b(s), acc);
+                    tc_commit(bar_s_full + 8 * (c & 1));
+                    if (with_proj && L::kProjInA) {
+                        // The A slot is free once the state update has read it.
+                        if (!wait(bar_s_full + 8 * (c & 1), (c >> 1) & 1)) break;
+                        load_proj();
+                    }
                 }
                 COTT_STAMP(2);
                 if (MODE == MODE_STATE) {
@@ -419,7 +436,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     continue;
                 }
                 if (split_refill && more) {
-                    if (!wait(bar_o_full + 8 * (c & 1), (c >> 1) & 1)) break;
+                    if (!wait(bar_s_full + 8 * (c & 1), (c >> 1) & 1)) break;   // covers P~ Bv too
                     issue_loads(c + NST, true, false);
                 }
                 COTT_STAMP(3);
@@ -557,6 +574,8 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 fence_proxy_async();
                 tc_fence_before();
                 mbar_arrive(bar_pt_ready);
+                // Next chunk's norms while the tensor core runs P~ Bv and the state update.
+                if (c + 1 < n_chunks) { norm_phase(c + 1); if (!alive) break; }
                 // bf16 copy of the updated state for the next chunk's X State product.
                 if (c + 1 < n_chunks) {
                     if (!wait(bar_s_full + 8 * (c & 1), (c >> 1) & 1)) break;
@@ -571,7 +590,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 }
                 COTT_STAMP(3);
             }
-            if (c + 1 < n_chunks) { norm_phase(c + 1); if (!alive) break; }
+            if (MODE != MODE_CAUSAL && c + 1 < n_chunks) { norm_phase(c + 1); if (!alive) break; }
             COTT_STAMP(5);
             if (MODE == MODE_STATE) {
                 // Follow every state update (a parity names one chunk only if no phase is
@@ -768,7 +787,7 @@ cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cuda
     p.m = a.m; p.seq_len = a.seq_len; p.seq_len_scalar = a.seq_len_scalar;
     p.H = H; p.N = N; p.group = a.group; p.n_groups = a.n_groups;
     p.norm_bv = a.norm_bv; p.x_norm = a.x_norm; p.epilogue = a.epilogue; p.reverse = a.reverse;
-    p.init_sum = a.init_sum;
+    p.init_sum = a.init_sum; p.init_transposed = a.init_transposed;
     if (d == 128) {
         if (a.mode == MODE_STATE) return launch_mode<128, MODE_STATE>(tm, p, BH, st);
         if (a.mode == MODE_CAUSAL) return launch_mode<128, MODE_CAUSAL>(tm, p, BH, st);
