@@ -77,13 +77,12 @@ static bool make_plan(int op, cott_dtype dt, int B, int H, int N, int d, int cau
         // One CTA per (b,h) and group, one CTA per SM.  Measured on B200: fewer, longer
         // groups win (per-CTA set-up and the per-group state traffic shrink) as long as
         // about every SM still gets a CTA, and a single group per (b,h) needs no partial-state
-        // pass at all.  So: as many groups per (b,h) as fit in one wave (rounded down), each a
-        // multiple of the 128-token chunk, at most 4096 tokens.
+        // pass at all.  So: as many groups per (b,h) as fit in ONE wave of CTAs (rounded
+        // down), each a multiple of the 128-token chunk.
         p->chunk = 128;
         const long per_head = BH >= 148 ? 1 : 148 / BH;
         long g = (N + per_head - 1) / per_head;
-        g = (g + 127) / 128 * 128;
-        group = (int)(g > 4096 ? 4096 : g);
+        group = (int)((g + 127) / 128 * 128);
     } else {
         p->chunk = 16;
         group = 1024;
