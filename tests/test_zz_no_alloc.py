@@ -30,7 +30,7 @@ def test_noalloc_matches_cott_fwd_twice_in_a_row():
 
 def test_noalloc_rejects_problems_beyond_its_scratch():
     lib = cott.cott._load()
-    B, H, N, d = 1, 16, 131072, 128
+    B, H, N, d = 64, 16, 8192, 128   # the decode prefill: 64 MB of group states
     assert cott.workspace_bytes(cott.cott.OP_FWD, cott.cott.BF16, B, H, N, d, True) > lib.cott_fwd_noalloc_max_bytes()
     sp = cott.cott._ScaleParams()
     sp.m, sp.seq_len, sp.seq_len_scalar = 256, None, 0.0   # never dereferenced: the size check comes first
