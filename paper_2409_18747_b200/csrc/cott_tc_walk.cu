@@ -67,10 +67,8 @@ template <int D, int MODE> struct Smem {
     static constexpr int kOffOut = kHasAB ? kOffB : kOffX;             // output staging slot
     static constexpr int kSb = (MODE == MODE_STATE) ? 0 : D * D * 2;   // bf16 copy of the state
     static constexpr int kOffSb = kStages * kStage;
-    // Masked-score operand P~ (128 x 128 bf16): d = 128 reuses the X slot (same size, and X
-    // is dead by then); d = 64 has a buffer of its own.
     static constexpr int kOffPt = kOffSb + kSb;
-    static constexpr int kPt = (MODE == MODE_CAUSAL && D == 64) ? kChunk * kChunk * 2 : 0;
+    static constexpr int kPt = 0;   // the masked scores live in tensor memory
     static constexpr int kOffBar = kOffPt + kPt;          // mbarriers, TMEM slot, abort flag
     static constexpr int kOffRx = kOffBar + 192;          // rx[kStages][128] floats, dm scratch
     static constexpr int kCtlBytes = 192 + kStages * 512 + 64;
@@ -108,14 +106,12 @@ __device__ __forceinline__ void issue_xs(uint32_t tO, uint32_t x, uint32_t sb) {
     }
 }
 template <int D>
-__device__ __forceinline__ void issue_pb(uint32_t tO, uint32_t p, uint32_t bv, bool acc_first) {
+__device__ __forceinline__ void issue_pb(uint32_t tO, uint32_t tPt, uint32_t bv, bool acc_first) {
+    // P~ (bf16, packed two per column) is the A operand in tensor memory: 8 columns per K = 16.
     constexpr uint32_t idesc = instr_desc_bf16(128, D, false, true);
 #pragma unroll
-    for (int kk = 0; kk < kChunk / 16; ++kk) {
-        const uint32_t off = (kk >> 2) * 16384u + (kk & 3) * 32u;
-        mma_ss(tO, smem_desc(p + off, 16, 1024), smem_desc(bv + kk * 2048u, 16384, 1024), idesc,
-               (kk > 0) || acc_first);
-    }
+    for (int kk = 0; kk < kChunk / 16; ++kk)
+        mma_ts(tO, tPt + kk * 8u, smem_desc(bv + kk * 2048u, 16384, 1024), idesc, (kk > 0) || acc_first);
 }
 template <int D>
 __device__ __forceinline__ void issue_atb(uint32_t tS, uint32_t a, uint32_t bv, bool acc_first) {
@@ -197,7 +193,10 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     constexpr int NST = L::kStages;
     constexpr int NH = D / 64;                       // 64-column half tiles per row
     constexpr uint32_t kTmemCols = 512;
-    constexpr uint32_t colS = 0, colP = D, colO0 = D + 128;   // O double-buffered: colO0, colO0 + D
+    // Columns: State d | P 128 (fp32 scores) | P~ 64 (bf16 masked scores, packed) | Out.
+    // d = 64 double-buffers Out; at d = 128 only one Out buffer fits in the 512 columns.
+    constexpr uint32_t colS = 0, colP = D, colPt = D + 128, colO0 = D + 192;
+    constexpr int kOBufs = (D == 64) ? 2 : 1;
     constexpr int QW = D / 4;                        // accumulator columns per worker thread
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -275,7 +274,6 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     auto stage_x = [&](int s) { return base + s * L::kStage + L::kOffX; };
     auto stage_a = [&](int s) { return base + s * L::kStage + L::kOffA; };
     auto stage_b = [&](int s) { return base + s * L::kStage + L::kOffB; };
-    auto stage_pt = [&](int s) { return (D == 128) ? stage_x(s) : base + L::kOffPt; };
     auto chunk_row = [&](int c) { return tok0 + (p.reverse ? (n_chunks - 1 - c) : c) * kChunk; };
 
     // bf16 copy of QW state columns of this thread's row into the MN-major state tile.
@@ -373,19 +371,26 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 const int s = c % NST;
                 if (!wait(bar_a_ready + 8 * s, (c / NST) & 1)) return;
                 const bool acc = init_state || c > 0;
+                if (MODE == MODE_CAUSAL) {
+                    // Scores first: they need neither the state copy nor the output buffer.
+                    tc_fence_after();
+                    issue_p<D>(tmem + colP, stage_x(s), stage_a(s));
+                    tc_commit(bar_p_full);
+                }
                 if (MODE != MODE_STATE) {
                     if (MODE == MODE_CAUSAL && c >= 1 && !wait(bar_sb_ready, (c - 1) & 1)) return;
-                    if (c >= 2 && !wait(bar_o_free + 8 * (c & 1), ((c >> 1) & 1) ^ 1)) return;
+                    // The output accumulator this chunk writes must have been drained: by chunk
+                    // c - 2 with two buffers, by chunk c - 1 with one.
+                    if (kOBufs == 2) { if (c >= 2 && !wait(bar_o_free + 8 * (c & 1), ((c >> 1) & 1) ^ 1)) return; }
+                    else if (c >= 1 && !wait(bar_o_free + 8 * ((c - 1) & 1), ((c - 1) >> 1) & 1)) return;
                 }
                 tc_fence_after();
-                const uint32_t tO = tmem + colO0 + (c & 1) * D;
+                const uint32_t tO = tmem + colO0 + (c % kOBufs) * D;
                 if (MODE == MODE_CAUSAL) {
                     // The state update of this chunk is issued later, behind P~ Bv, so that
                     // the workers mask the scores without the tensor core hammering shared
                     // memory and TMEM at the same time.
-                    issue_p<D>(tmem + colP, stage_x(s), stage_a(s));
                     if (acc) issue_xs<D>(tO, stage_x(s), sb);
-                    tc_commit(bar_p_full);
                 } else if (MODE == MODE_STATE) {
                     issue_atb<D>(tmem + colS, stage_a(s), stage_b(s), acc);
                     tc_commit(bar_s_full + 8 * (c & 1));
@@ -419,7 +424,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     COTT_STAMP(1);
                     tc_fence_after();
                     const bool acc = init_state || c > 0;
-                    issue_pb<D>(tmem + colO0 + (c & 1) * D, stage_pt(s), stage_b(s), acc);
+                    issue_pb<D>(tmem + colO0 + (c % kOBufs) * D, tmem + colPt, stage_b(s), acc);
                     tc_commit(bar_o_full + 8 * (c & 1));
                     issue_atb<D>(tmem + colS, stage_a(s), stage_b(s), acc);
                     tc_commit(bar_s_full + 8 * (c & 1));
@@ -537,7 +542,6 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         for (int c = 0; c < n_chunks && alive; ++c) {
             const int s = c % NST;
             uint8_t* st = gbase + s * L::kStage;
-            uint8_t* pt = (D == 128) ? st + L::kOffX : gbase + L::kOffPt;
             if (MODE == MODE_CAUSAL) {
                 // Masked scores -> bf16 operand P~ (both MMAs that read X are done).  Forward:
                 // row i keeps columns j <= i (diagonal kept, Eq. 6); backward in time: j >= i.
@@ -565,13 +569,16 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
 #pragma unroll
                         for (int j = 0; j < 32; ++j) r[j] = 0u;
                     }
+                    // bf16, two scores per column (even column index in the low half), into the
+                    // A-operand region of tensor memory: this block's 32 k-values are 16 columns.
+                    uint32_t pk[16];
 #pragma unroll
-                    for (int i = 0; i < 32; i += 8)
-                        *reinterpret_cast<uint4*>(pt + (cq >> 1) * 16384 + swz(arow, (cq & 1) * 4 + (i >> 3))) =
-                            pack8(&r[i]);
+                    for (int j = 0; j < 16; ++j)
+                        pk[j] = pack_bf16(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
+                    tmem_st16(tmem + lane_base + colPt + cq * 16, pk);
+                    tmem_wait_st();
                 }
                 COTT_STAMP(2);
-                fence_proxy_async();
                 tc_fence_before();
                 mbar_arrive(bar_pt_ready);
                 // Next chunk's norms while the tensor core runs P~ Bv and the state update.
@@ -603,7 +610,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             if (!wait(bar_o_full + 8 * (c & 1), (c >> 1) & 1)) break;
             tc_fence_after();
             COTT_STAMP(6);
-            const uint32_t tO = tmem + lane_base + colO0 + (c & 1) * D + cq * QW;
+            const uint32_t tO = tmem + lane_base + colO0 + (c % kOBufs) * D + cq * QW;
             const float rx = rx_buf[(c % NST) * 128 + arow];
             uint32_t r[QW];
             tmem_ldq<QW>(tO, r);
