@@ -70,13 +70,21 @@ template <int D, int MODE> struct Smem {
     static constexpr int kOffPt = kOffSb + kSb;
     static constexpr int kPt = 0;   // the masked scores live in tensor memory
     static constexpr int kOffBar = kOffPt + kPt;          // mbarriers, TMEM slot, abort flag
-    static constexpr int kOffRx = kOffBar + 192;          // rx[kStages][128] floats, dm scratch
-    static constexpr int kCtlBytes = 192 + kStages * 512 + 64;
+    // Row scales of X wait in rx[kRx][128] from the norm phase of a chunk to its output
+    // epilogue; three buffers are needed because X and A of chunk c+2 can land (and be
+    // normalised) before every worker has finished the epilogue of chunk c.
+    static constexpr int kRx = kStages < 3 ? 3 : kStages;
+    static constexpr int kOffRx = kOffBar + 256;          // rx[kRx][128] floats, dm scratch
+    static constexpr int kCtlBytes = 256 + kRx * 512 + 64;
     // Gradient epilogues need a fourth tile (raw q, k or v rows) and a 4 KB exchange area
     // for per-row partial sums.  The causal walk at d = 128 has no room for either: it puts
     // the tile in the A slot and the exchange area in the X slot, both dead by then.  Every
     // other case has a buffer behind the control block, allocated only when needed.
     static constexpr bool kProjInA = (MODE == MODE_CAUSAL && D == 128);
+    // Causal walk at d = 128 (two-stage ring): Bv, loaded last and needed last, has a barrier
+    // of its own so that the scores of a chunk do not wait for it.  Measured: helps the
+    // two-stage ring, costs a little with the three stages of d = 64.
+    static constexpr bool kSplitB = (MODE == MODE_CAUSAL && D == 128);
     static constexpr int kOffProj = (kOffBar + kCtlBytes + 1023) / 1024 * 1024;
     static constexpr int kXch = 4096;
     static constexpr int dyn_bytes(bool with_proj) {
@@ -204,22 +212,25 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     const uint32_t bars = base + L::kOffBar;
     // Barriers that a fast role could otherwise lap are arrays indexed by stage or by chunk
     // parity, so a phase parity always names one chunk; no waiter ever skips a phase.
-    const uint32_t bar_full = bars;            // [NST] (<= 4) TMA landed
-    const uint32_t bar_a_ready = bars + 32;    // [NST] rows normalised (all workers)
-    const uint32_t bar_p_full = bars + 64;     //       scores and X State done (commit)
+    const uint32_t bar_full = bars;            // [NST] (<= 4) TMA landed: X and A (causal walk), all tiles otherwise
+    const uint32_t bar_a_ready = bars + 32;    // [NST] X scale known, A normalised (all workers)
+    const uint32_t bar_p_full = bars + 64;     //       scores done (commit)
     const uint32_t bar_s_full = bars + 72;     // [2]   state update done (commit)
-    const uint32_t bar_pt_ready = bars + 88;   //       masked scores in shared memory (all workers)
+    const uint32_t bar_pt_ready = bars + 88;   //       masked scores in tensor memory (all workers)
     const uint32_t bar_sb_ready = bars + 96;   //       bf16 state copy written (all workers)
     const uint32_t bar_o_full = bars + 104;    // [2]   output accumulator complete (commit)
     const uint32_t bar_o_free = bars + 120;    // [2]   output accumulator drained (all workers)
     const uint32_t bar_proj = bars + 136;      //       epilogue tile landed
     const uint32_t bar_e_done = bars + 144;    // [2]   output rows of the chunk staged (all workers)
     const uint32_t bar_xch = bars + 160;       //       per-row partial sums exchanged (all workers)
-    const uint32_t tmem_slot = bars + 168;
-    volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(gbase + L::kOffBar + 168);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + L::kOffBar + 172);
-    float* rx_buf = reinterpret_cast<float*>(gbase + L::kOffRx);                 // [NST][128]
-    float* dm_red = reinterpret_cast<float*>(gbase + L::kOffRx + NST * 512);     // [16]
+    const uint32_t bar_full_b = bars + 168;    // [NST] causal walk: Bv landed (it is loaded last and needed last)
+    const uint32_t bar_b_ready = bars + 200;   // [NST] causal walk: Bv normalised, when it is the one (all workers)
+    const uint32_t tmem_slot = bars + 232;
+    volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(gbase + L::kOffBar + 232);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + L::kOffBar + 236);
+    constexpr int NRX = L::kRx;
+    float* rx_buf = reinterpret_cast<float*>(gbase + L::kOffRx);                 // [NRX][128]
+    float* dm_red = reinterpret_cast<float*>(gbase + L::kOffRx + NRX * 512);     // [16]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = blockIdx.x % p.n_groups, bh = blockIdx.x / p.n_groups;
@@ -235,7 +246,8 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         tmem_relinquish();
     }
     if (tid == 0) {
-        for (int i = 0; i < NST; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_a_ready + 8 * i, kWorkers); }
+        for (int i = 0; i < NST; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_a_ready + 8 * i, kWorkers);
+                                        mbar_init(bar_full_b + 8 * i, 1); mbar_init(bar_b_ready + 8 * i, kWorkers); }
         mbar_init(bar_p_full, 1); mbar_init(bar_s_full, 1); mbar_init(bar_s_full + 8, 1);
         mbar_init(bar_pt_ready, kWorkers); mbar_init(bar_sb_ready, kWorkers);
         mbar_init(bar_o_full, 1); mbar_init(bar_o_full + 8, 1);
@@ -350,15 +362,28 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 const int s = c % NST;
                 const uint32_t bar = bar_full + 8 * s;
                 const int row = chunk_row(c);
-                if (part1) mbar_expect_tx(bar, L::kTilesPerStage * L::kTile);
-                if (L::kHasAB) {
+                if (L::kSplitB) {
                     if (part1) {
-                        if (L::kHasX) load_tile(stage_x(s), &tmX, bar, row);
+                        mbar_expect_tx(bar, 2 * L::kTile);
+                        load_tile(stage_x(s), &tmX, bar, row);
                         load_tile(stage_a(s), &tmA, bar, row);
                     }
-                    if (part2) load_tile(stage_b(s), &tmB, bar, row);
-                } else if (part2) {
-                    load_tile(stage_x(s), &tmX, bar, row);
+                    if (part2) {
+                        mbar_expect_tx(bar_full_b + 8 * s, L::kTile);
+                        load_tile(stage_b(s), &tmB, bar_full_b + 8 * s, row);
+                    }
+                } else {
+                    // One barrier for the stage: its byte count is armed with the first part.
+                    if (part1) mbar_expect_tx(bar, L::kTilesPerStage * L::kTile);
+                    if (L::kHasAB) {
+                        if (part1) {
+                            if (L::kHasX) load_tile(stage_x(s), &tmX, bar, row);
+                            load_tile(stage_a(s), &tmA, bar, row);
+                        }
+                        if (part2) load_tile(stage_b(s), &tmB, bar, row);
+                    } else if (part2) {
+                        load_tile(stage_x(s), &tmX, bar, row);
+                    }
                 }
             };
             auto wait = [&](uint32_t bar, uint32_t parity) {
@@ -421,6 +446,12 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 }
                 if (MODE == MODE_CAUSAL) {
                     if (!wait(bar_pt_ready, c & 1)) break;
+                    // Bv is needed from here on: landed, and normalised if it is the operand
+                    // whose row scale sits on the contraction index.
+                    if (L::kSplitB) {
+                        if (!wait(bar_full_b + 8 * s, (c / NST) & 1)) break;
+                        if (p.norm_bv && !wait(bar_b_ready + 8 * s, (c / NST) & 1)) break;
+                    }
                     COTT_STAMP(1);
                     tc_fence_after();
                     const bool acc = init_state || c > 0;
@@ -491,7 +522,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             if (!wait(bar_full + 8 * s, (c / NST) & 1)) return;
 #ifdef COTT_TIMING
             if (blockIdx.x == 0 && threadIdx.x == 0 && (c == 3 || c == 4))
-                reinterpret_cast<unsigned long long*>(p.status)[1 + (c - 3) * 7 + 4] = globaltimer_ns();
+                reinterpret_cast<unsigned long long*>(p.status)[1 + (c - 3) * 7 + 3] = globaltimer_ns();
 #endif
             uint8_t* st = gbase + s * L::kStage;
             uint4 wx[NC], wn[NC];
@@ -500,7 +531,9 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 for (int j = 0; j < NC; ++j) wx[j] = *reinterpret_cast<const uint4*>(tile_q_ptr(st + L::kOffX, j));
             }
             uint8_t* nt = st + (p.norm_bv ? L::kOffB : L::kOffA);
-            if (L::kHasAB) {
+            // In the causal walk Bv arrives on its own barrier and is normalised later (norm_b).
+            const bool norm_here = L::kHasAB && !(L::kSplitB && p.norm_bv);
+            if (norm_here) {
 #pragma unroll
                 for (int j = 0; j < NC; ++j) wn[j] = *reinterpret_cast<const uint4*>(tile_q_ptr(nt, j));
             }
@@ -513,9 +546,9 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     const float ss = quad_sum((a0 + a1) + (a2 + a3));
                     rx = cfac / fmaxf(sqrtf(ss), kEps);
                 }
-                if (nq == 0) rx_buf[(c % NST) * 128 + nrow] = rx;
+                if (nq == 0) rx_buf[(c % NRX) * 128 + nrow] = rx;
             }
-            if (L::kHasAB) {
+            if (norm_here) {
                 float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
                 for (int j = 0; j < NC; j += 2) { sumsq8(wn[j], a0, a1); sumsq8(wn[j + 1], a2, a3); }
@@ -538,10 +571,49 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             mbar_arrive(bar_a_ready + 8 * s);
         };
 
+        // Causal walk, Bv is the normalised operand (dQ^ and dK^ streams): done once Bv has
+        // landed, just before the tensor core needs it.
+        auto norm_b = [&](int c) {
+            const int s = c % NST;
+            if (!wait(bar_full_b + 8 * s, (c / NST) & 1)) return;
+            uint8_t* nt = gbase + s * L::kStage + L::kOffB;
+            uint4 wn[NC];
+            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+            for (int j = 0; j < NC; ++j) wn[j] = *reinterpret_cast<const uint4*>(tile_q_ptr(nt, j));
+#pragma unroll
+            for (int j = 0; j < NC; j += 2) { sumsq8(wn[j], a0, a1); sumsq8(wn[j + 1], a2, a3); }
+            const float ss = quad_sum((a0 + a1) + (a2 + a3));
+            const float r = 1.0f / fmaxf(sqrtf(ss), kEps);
+#pragma unroll
+            for (int j = 0; j < NC; ++j) {
+                const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&wn[j]);
+                uint4 o;
+                uint32_t* ow = reinterpret_cast<uint32_t*>(&o);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    float2 f = __bfloat1622float2(e[i]);
+                    ow[i] = pack_bf16(f.x * r, f.y * r);
+                }
+                *reinterpret_cast<uint4*>(tile_q_ptr(nt, j)) = o;
+            }
+            fence_proxy_async();
+            mbar_arrive(bar_b_ready + 8 * s);
+        };
+
         if (alive) norm_phase(0);
         for (int c = 0; c < n_chunks && alive; ++c) {
             const int s = c % NST;
             uint8_t* st = gbase + s * L::kStage;
+            bool bv_normed = false;
+            if (L::kSplitB && p.norm_bv) {
+                // Bv of this chunk usually landed long ago: normalise it now, in the shadow of
+                // the score MMA, rather than between the masking and P~ Bv (decided per warp).
+                int ready = 0;
+                if (lane == 0) ready = mbar_try_wait(bar_full_b + 8 * s, (c / NST) & 1) ? 1 : 0;
+                ready = __shfl_sync(0xffffffffu, ready, 0);
+                if (ready) { norm_b(c); bv_normed = true; if (!alive) break; }
+            }
             if (MODE == MODE_CAUSAL) {
                 // Masked scores -> bf16 operand P~ (both MMAs that read X are done).  Forward:
                 // row i keeps columns j <= i (diagonal kept, Eq. 6); backward in time: j >= i.
@@ -581,8 +653,10 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 COTT_STAMP(2);
                 tc_fence_before();
                 mbar_arrive(bar_pt_ready);
+                if (L::kSplitB && p.norm_bv && !bv_normed) { norm_b(c); if (!alive) break; }
                 // Next chunk's norms while the tensor core runs P~ Bv and the state update.
                 if (c + 1 < n_chunks) { norm_phase(c + 1); if (!alive) break; }
+                COTT_STAMP(4);
                 // bf16 copy of the updated state for the next chunk's X State product.
                 if (c + 1 < n_chunks) {
                     if (!wait(bar_s_full + 8 * (c & 1), (c >> 1) & 1)) break;
@@ -595,10 +669,9 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     tc_fence_before();
                     mbar_arrive(bar_sb_ready);
                 }
-                COTT_STAMP(3);
+                COTT_STAMP(5);
             }
             if (MODE != MODE_CAUSAL && c + 1 < n_chunks) { norm_phase(c + 1); if (!alive) break; }
-            COTT_STAMP(5);
             if (MODE == MODE_STATE) {
                 // Follow every state update (a parity names one chunk only if no phase is
                 // skipped); after the last one the accumulator holds the group's state.
@@ -611,7 +684,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             tc_fence_after();
             COTT_STAMP(6);
             const uint32_t tO = tmem + lane_base + colO0 + (c % kOBufs) * D + cq * QW;
-            const float rx = rx_buf[(c % NST) * 128 + arow];
+            const float rx = rx_buf[(c % NRX) * 128 + arow];
             uint32_t r[QW];
             tmem_ldq<QW>(tO, r);
             tmem_wait_ld();
