@@ -50,6 +50,7 @@ enum { MODE_STATE = 0, MODE_CAUSAL = 1, MODE_READOUT = 2 };
 
 constexpr int kWorkerWarps = 16;                      // row-worker warps (4 per TMEM lane quadrant)
 constexpr int kWorkers = kWorkerWarps * 32;
+constexpr int kGroupThreads = kWorkers / 2;           // the workers act as two groups of eight warps
 
 // Shared-memory plan.  A stage holds the tiles one chunk needs from TMA: (A, Bv) for the
 // state-only pass, (X, A, Bv) for the causal walk, (X) for the read-out.
@@ -86,7 +87,7 @@ template <int D, int MODE> struct Smem {
     // two-stage ring, costs a little with the three stages of d = 64.
     static constexpr bool kSplitB = (MODE == MODE_CAUSAL && D == 128);
     static constexpr int kOffProj = (kOffBar + kCtlBytes + 1023) / 1024 * 1024;
-    static constexpr int kXch = 4096;
+    static constexpr int kXch = 2048;
     static constexpr int dyn_bytes(bool with_proj) {
         return ((with_proj && !kProjInA) ? kOffProj + kTile + kXch : kOffBar + kCtlBytes) + 1024;  // + align slack
     }
@@ -188,10 +189,10 @@ template <> __device__ __forceinline__ void tmem_stq<16>(uint32_t taddr, const u
 #define COTT_STAMP(slot) do {} while (0)
 #endif
 
-// Thread roles: warps 0-15 are the row workers (norms, score masking, state and output
-// epilogues; four warps per TMEM lane quadrant, each owning a quarter of the columns);
-// warp 16 lane 0 is the control thread (TMA loads / stores and all tcgen05.mma).
-// The roles meet only through mbarriers, every wait bounded.
+// Thread roles: warps 0-15 are the row workers, in two groups of eight that work on different
+// chunks at once (score masking + state copy / row norms + output epilogue); warp 16 lane 0
+// is the control thread (TMA loads / stores and all tcgen05.mma).  The roles meet only
+// through mbarriers, every wait bounded.
 template <int D, int MODE>
 __global__ void __launch_bounds__(kTcThreads, 1)
 tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmA,
@@ -228,6 +229,11 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     const uint32_t tmem_slot = bars + 232;
     volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(gbase + L::kOffBar + 232);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + L::kOffBar + 236);
+    // State-update barrier of chunk c.  The state-only pass, whose two worker groups may drift
+    // apart by more than one chunk, cycles through four barriers (bars + 64 .. + 88; the
+    // score barriers are unused there); the other modes use two.
+    auto sfull_bar = [&](int c) { return MODE == MODE_STATE ? bars + 64 + 8 * (c & 3) : bar_s_full + 8 * (c & 1); };
+    auto sfull_par = [&](int c) { return (uint32_t)(MODE == MODE_STATE ? (c >> 2) & 1 : (c >> 1) & 1); };
     constexpr int NRX = L::kRx;
     float* rx_buf = reinterpret_cast<float*>(gbase + L::kOffRx);                 // [NRX][128]
     float* dm_red = reinterpret_cast<float*>(gbase + L::kOffRx + NRX * 512);     // [16]
@@ -246,14 +252,16 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         tmem_relinquish();
     }
     if (tid == 0) {
-        for (int i = 0; i < NST; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_a_ready + 8 * i, kWorkers);
-                                        mbar_init(bar_full_b + 8 * i, 1); mbar_init(bar_b_ready + 8 * i, kWorkers); }
+        for (int i = 0; i < NST; ++i) {
+            mbar_init(bar_full + 8 * i, 1); mbar_init(bar_a_ready + 8 * i, kGroupThreads);
+            mbar_init(bar_full_b + 8 * i, 1); mbar_init(bar_b_ready + 8 * i, kGroupThreads);
+        }
         mbar_init(bar_p_full, 1); mbar_init(bar_s_full, 1); mbar_init(bar_s_full + 8, 1);
-        mbar_init(bar_pt_ready, kWorkers); mbar_init(bar_sb_ready, kWorkers);
+        mbar_init(bar_pt_ready, MODE == MODE_STATE ? 1 : kGroupThreads); mbar_init(bar_sb_ready, kGroupThreads);
         mbar_init(bar_o_full, 1); mbar_init(bar_o_full + 8, 1);
-        mbar_init(bar_o_free, kWorkers); mbar_init(bar_o_free + 8, kWorkers);
-        mbar_init(bar_proj, 1); mbar_init(bar_e_done, kWorkers); mbar_init(bar_e_done + 8, kWorkers);
-        mbar_init(bar_xch, kWorkers);
+        mbar_init(bar_o_free, kGroupThreads); mbar_init(bar_o_free + 8, kGroupThreads);
+        mbar_init(bar_proj, 1); mbar_init(bar_e_done, kGroupThreads); mbar_init(bar_e_done + 8, kGroupThreads);
+        mbar_init(bar_xch, kGroupThreads);
         *abort_flag = 0;
         mbar_fence_init();
         fence_proxy_async();
@@ -418,7 +426,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     if (acc) issue_xs<D>(tO, stage_x(s), sb);
                 } else if (MODE == MODE_STATE) {
                     issue_atb<D>(tmem + colS, stage_a(s), stage_b(s), acc);
-                    tc_commit(bar_s_full + 8 * (c & 1));
+                    tc_commit(sfull_bar(c));
                 } else {
                     issue_xs<D>(tO, stage_x(s), sb);
                     tc_commit(bar_o_full + 8 * (c & 1));
@@ -458,21 +466,21 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     issue_pb<D>(tmem + colO0 + (c % kOBufs) * D, tmem + colPt, stage_b(s), acc);
                     tc_commit(bar_o_full + 8 * (c & 1));
                     issue_atb<D>(tmem + colS, stage_a(s), stage_b(s), acc);
-                    tc_commit(bar_s_full + 8 * (c & 1));
+                    tc_commit(sfull_bar(c));
                     if (with_proj && L::kProjInA) {
                         // The A slot is free once the state update has read it.
-                        if (!wait(bar_s_full + 8 * (c & 1), (c >> 1) & 1)) break;
+                        if (!wait(sfull_bar(c), sfull_par(c))) break;
                         load_proj();
                     }
                 }
                 COTT_STAMP(2);
                 if (MODE == MODE_STATE) {
-                    if (more) { if (!wait(bar_s_full + 8 * (c & 1), (c >> 1) & 1)) break; issue_loads(c + NST, true, true); }
+                    if (more) { if (!wait(sfull_bar(c), sfull_par(c))) break; issue_loads(c + NST, true, true); }
                     if (c + 1 < n_chunks) batch1(c + 1);
                     continue;
                 }
                 if (split_refill && more) {
-                    if (!wait(bar_s_full + 8 * (c & 1), (c >> 1) & 1)) break;   // covers P~ Bv too
+                    if (!wait(sfull_bar(c), sfull_par(c))) break;   // covers P~ Bv too
                     issue_loads(c + NST, true, false);
                 }
                 COTT_STAMP(3);
@@ -498,93 +506,38 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         }
     } else {
         // ------------------------------------------------------------------ row workers
+        // Two groups of eight warps work on different chunks at the same time, so that the
+        // long-latency steps of one (TMEM loads, shared-memory round trips) hide behind the
+        // other:  group P (warps 0-7)  masks the scores and refreshes the bf16 state copy;
+        //         group O (warps 8-15) computes the row norms of the next chunk and runs the
+        //         output epilogue of the current one.
+        // Each group covers all four TMEM lane quadrants with two warps (column halves).  In
+        // the state-only pass both groups normalise, on alternate chunks.
         bool alive = n_chunks > 0;
         auto wait = [&](uint32_t bar, uint32_t parity) {
             if (alive && !wait_or_abort(bar, parity, abort_flag)) alive = false;
             return alive;
         };
-        // Norm-phase mapping: lanes l, l^8, l^16, l^24 share a row (four column quarters).
-        const int nrow = warp * 8 + (lane & 7), nq = lane >> 3;
-        constexpr int NC = D / 32;                    // 16-byte chunks in a quarter row
-        auto tile_q_ptr = [&](uint8_t* tile, int j) {
-            const int ch = nq * NC + j;               // chunk index within the row
+        const int grp = warp >> 3, w8 = warp & 7, hf = w8 >> 2;
+        constexpr int HW = D / 2;                     // accumulator columns per thread in the chunk loops
+        constexpr int NPIECE = HW / 32;               // 32-column pieces of that range
+        // Norm mapping inside a group: lanes l and l^16 share a row (two column halves).
+        const int nrow = w8 * 16 + (lane & 15), nhalf = lane >> 4;
+        constexpr int NC = D / 16;                    // 16-byte chunks in half a row
+        auto tile_h_ptr = [&](uint8_t* tile, int j) {
+            const int ch = nhalf * NC + j;            // chunk index within the row
             return tile + (ch >> 3) * 16384 + swz(nrow, ch & 7);
         };
-        auto quad_sum = [&](float v) {
-            v += __shfl_xor_sync(0xffffffffu, v, 8);
-            v += __shfl_xor_sync(0xffffffffu, v, 16);
-            return v;
-        };
-        // Row norms of chunk c: the contraction-side operand is normalised in place; the X
-        // row scale (times c) is left in rx_buf[c % NST] for the output epilogue.
-        auto norm_phase = [&](int c) {
-            const int s = c % NST;
-            if (!wait(bar_full + 8 * s, (c / NST) & 1)) return;
-#ifdef COTT_TIMING
-            if (blockIdx.x == 0 && threadIdx.x == 0 && (c == 3 || c == 4))
-                reinterpret_cast<unsigned long long*>(p.status)[1 + (c - 3) * 7 + 3] = globaltimer_ns();
-#endif
-            uint8_t* st = gbase + s * L::kStage;
-            uint4 wx[NC], wn[NC];
-            if (L::kHasX && p.x_norm) {
-#pragma unroll
-                for (int j = 0; j < NC; ++j) wx[j] = *reinterpret_cast<const uint4*>(tile_q_ptr(st + L::kOffX, j));
-            }
-            uint8_t* nt = st + (p.norm_bv ? L::kOffB : L::kOffA);
-            // In the causal walk Bv arrives on its own barrier and is normalised later (norm_b).
-            const bool norm_here = L::kHasAB && !(L::kSplitB && p.norm_bv);
-            if (norm_here) {
-#pragma unroll
-                for (int j = 0; j < NC; ++j) wn[j] = *reinterpret_cast<const uint4*>(tile_q_ptr(nt, j));
-            }
-            if (L::kHasX) {
-                float rx = cfac;
-                if (p.x_norm) {
-                    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll
-                    for (int j = 0; j < NC; j += 2) { sumsq8(wx[j], a0, a1); sumsq8(wx[j + 1], a2, a3); }
-                    const float ss = quad_sum((a0 + a1) + (a2 + a3));
-                    rx = cfac / fmaxf(sqrtf(ss), kEps);
-                }
-                if (nq == 0) rx_buf[(c % NRX) * 128 + nrow] = rx;
-            }
-            if (norm_here) {
-                float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll
-                for (int j = 0; j < NC; j += 2) { sumsq8(wn[j], a0, a1); sumsq8(wn[j + 1], a2, a3); }
-                const float ss = quad_sum((a0 + a1) + (a2 + a3));
-                const float r = 1.0f / fmaxf(sqrtf(ss), kEps);
-#pragma unroll
-                for (int j = 0; j < NC; ++j) {
-                    const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&wn[j]);
-                    uint4 o;
-                    uint32_t* ow = reinterpret_cast<uint32_t*>(&o);
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        float2 f = __bfloat1622float2(e[i]);
-                        ow[i] = pack_bf16(f.x * r, f.y * r);
-                    }
-                    *reinterpret_cast<uint4*>(tile_q_ptr(nt, j)) = o;
-                }
-                fence_proxy_async();
-            }
-            mbar_arrive(bar_a_ready + 8 * s);
-        };
-
-        // Causal walk, Bv is the normalised operand (dQ^ and dK^ streams): done once Bv has
-        // landed, just before the tensor core needs it.
-        auto norm_b = [&](int c) {
-            const int s = c % NST;
-            if (!wait(bar_full_b + 8 * s, (c / NST) & 1)) return;
-            uint8_t* nt = gbase + s * L::kStage + L::kOffB;
+        auto pair_sum = [&](float v) { return v + __shfl_xor_sync(0xffffffffu, v, 16); };
+        // x^ = x / max(||x||, eps) on this thread's half row, in place, rounded to bf16.
+        auto normalise_half_row = [&](uint8_t* nt) {
             uint4 wn[NC];
             float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
-            for (int j = 0; j < NC; ++j) wn[j] = *reinterpret_cast<const uint4*>(tile_q_ptr(nt, j));
+            for (int j = 0; j < NC; ++j) wn[j] = *reinterpret_cast<const uint4*>(tile_h_ptr(nt, j));
 #pragma unroll
             for (int j = 0; j < NC; j += 2) { sumsq8(wn[j], a0, a1); sumsq8(wn[j + 1], a2, a3); }
-            const float ss = quad_sum((a0 + a1) + (a2 + a3));
-            const float r = 1.0f / fmaxf(sqrtf(ss), kEps);
+            const float r = 1.0f / fmaxf(sqrtf(pair_sum((a0 + a1) + (a2 + a3))), kEps);
 #pragma unroll
             for (int j = 0; j < NC; ++j) {
                 const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&wn[j]);
@@ -595,40 +548,78 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     float2 f = __bfloat1622float2(e[i]);
                     ow[i] = pack_bf16(f.x * r, f.y * r);
                 }
-                *reinterpret_cast<uint4*>(tile_q_ptr(nt, j)) = o;
+                *reinterpret_cast<uint4*>(tile_h_ptr(nt, j)) = o;
             }
             fence_proxy_async();
+        };
+        // Row norms of chunk c: the contraction-side operand is normalised in place; the X
+        // row scale (times c) is left in rx_buf[c % NRX] for the output epilogue.
+        auto norm_phase = [&](int c) {
+            const int s = c % NST;
+            if (!wait(bar_full + 8 * s, (c / NST) & 1)) return;
+            uint8_t* st = gbase + s * L::kStage;
+            if (L::kHasX) {
+                float rx = cfac;
+                if (p.x_norm) {
+                    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+                    for (int j = 0; j < NC; j += 2) {
+                        sumsq8(*reinterpret_cast<const uint4*>(tile_h_ptr(st + L::kOffX, j)), a0, a1);
+                        sumsq8(*reinterpret_cast<const uint4*>(tile_h_ptr(st + L::kOffX, j + 1)), a2, a3);
+                    }
+                    rx = cfac / fmaxf(sqrtf(pair_sum((a0 + a1) + (a2 + a3))), kEps);
+                }
+                if (nhalf == 0) rx_buf[(c % NRX) * 128 + nrow] = rx;
+            }
+            // In the split causal walk Bv arrives on its own barrier and is normalised later.
+            if (L::kHasAB && !(L::kSplitB && p.norm_bv))
+                normalise_half_row(st + (p.norm_bv ? L::kOffB : L::kOffA));
+            mbar_arrive(bar_a_ready + 8 * s);
+        };
+        // Split causal walk, Bv is the normalised operand (dQ^ and dK^ streams).
+        auto norm_b = [&](int c) {
+            const int s = c % NST;
+            if (!wait(bar_full_b + 8 * s, (c / NST) & 1)) return;
+            normalise_half_row(gbase + s * L::kStage + L::kOffB);
             mbar_arrive(bar_b_ready + 8 * s);
         };
-
-        if (alive) norm_phase(0);
-        for (int c = 0; c < n_chunks && alive; ++c) {
-            const int s = c % NST;
-            uint8_t* st = gbase + s * L::kStage;
-            bool bv_normed = false;
-            if (L::kSplitB && p.norm_bv) {
-                // Bv of this chunk usually landed long ago: normalise it now, in the shadow of
-                // the score MMA, rather than between the masking and P~ Bv (decided per warp).
-                int ready = 0;
-                if (lane == 0) ready = mbar_try_wait(bar_full_b + 8 * s, (c / NST) & 1) ? 1 : 0;
-                ready = __shfl_sync(0xffffffffu, ready, 0);
-                if (ready) { norm_b(c); bv_normed = true; if (!alive) break; }
+        // bf16 copy of 32 state columns of this thread's row into the MN-major state tile.
+        auto write_sb32 = [&](const uint32_t (&r)[32], int c0) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 8) {
+                const int col = c0 + i;
+                const uint32_t off = (col >> 6) * (D * 128u) + swz(srow, (col & 63) >> 3);
+                *reinterpret_cast<uint4*>(gbase + L::kOffSb + off) = pack8(&r[i]);
             }
-            if (MODE == MODE_CAUSAL) {
-                // Masked scores -> bf16 operand P~ (both MMAs that read X are done).  Forward:
-                // row i keeps columns j <= i (diagonal kept, Eq. 6); backward in time: j >= i.
-                // This warp owns the 32 x 32 block (row block q, column block cq): all-keep,
-                // all-zero, or (q == cq) a triangle; the first two cases are warp-uniform.
+        };
+
+        if (MODE == MODE_STATE) {
+            // Both groups normalise, on alternate chunks, and follow every state update (a
+            // parity names one chunk only if no phase is skipped).
+            for (int c = 0; c < n_chunks && alive; ++c) {
+                if ((c & 1) == grp) norm_phase(c);
+                if (c >= 1 && !wait(sfull_bar(c - 1), sfull_par(c - 1))) break;
+            }
+            if (alive) wait(sfull_bar(n_chunks - 1), sfull_par(n_chunks - 1));
+        } else if (grp == 0) {
+            // -------------------------------------------------------------- group P
+            for (int c = 0; MODE == MODE_CAUSAL && c < n_chunks && alive; ++c) {
+                // Masked scores -> bf16 operand P~ in tensor memory.  Forward: row i keeps
+                // columns j <= i (diagonal kept, Eq. 6); backward in time: j >= i.  Per
+                // 32 x 32 block (row block q, column block cb) the mask is all-keep, all-zero
+                // or, on the diagonal, a triangle; the first two cases are warp-uniform.
                 COTT_STAMP(0);
                 if (!wait(bar_p_full, c & 1)) break;
                 tc_fence_after();
                 COTT_STAMP(1);
-                {
-                    const bool keep_all = p.reverse ? (cq > q) : (cq < q);
-                    const bool diag = cq == q;
+#pragma unroll
+                for (int sbk = 0; sbk < 2; ++sbk) {
+                    const int cb = 2 * hf + sbk;
+                    const bool keep_all = p.reverse ? (cb > q) : (cb < q);
+                    const bool diag = cb == q;
                     uint32_t r[32];
                     if (keep_all || diag) {
-                        tmem_ld32(tmem + lane_base + colP + cq * 32, r);
+                        tmem_ld32(tmem + lane_base + colP + cb * 32, r);
                         tmem_wait_ld();
                         if (diag) {
 #pragma unroll
@@ -641,117 +632,126 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
 #pragma unroll
                         for (int j = 0; j < 32; ++j) r[j] = 0u;
                     }
-                    // bf16, two scores per column (even column index in the low half), into the
-                    // A-operand region of tensor memory: this block's 32 k-values are 16 columns.
+                    // bf16, two scores per column (even column index in the low half): this
+                    // block's 32 k-values are 16 columns of the A-operand region.
                     uint32_t pk[16];
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
                         pk[j] = pack_bf16(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
-                    tmem_st16(tmem + lane_base + colPt + cq * 16, pk);
-                    tmem_wait_st();
+                    tmem_st16(tmem + lane_base + colPt + cb * 16, pk);
                 }
+                tmem_wait_st();
                 COTT_STAMP(2);
                 tc_fence_before();
                 mbar_arrive(bar_pt_ready);
-                if (L::kSplitB && p.norm_bv && !bv_normed) { norm_b(c); if (!alive) break; }
-                // Next chunk's norms while the tensor core runs P~ Bv and the state update.
-                if (c + 1 < n_chunks) { norm_phase(c + 1); if (!alive) break; }
-                COTT_STAMP(4);
                 // bf16 copy of the updated state for the next chunk's X State product.
                 if (c + 1 < n_chunks) {
-                    if (!wait(bar_s_full + 8 * (c & 1), (c >> 1) & 1)) break;
+                    if (!wait(sfull_bar(c), sfull_par(c))) break;
                     tc_fence_after();
-                    uint32_t r[QW];
-                    tmem_ldq<QW>(tmem + lane_base + colS + cq * QW, r);
-                    tmem_wait_ld();
-                    if (owns_srow) write_sb(r, cq * QW);
+#pragma unroll
+                    for (int pc = 0; pc < NPIECE; ++pc) {
+                        uint32_t r[32];
+                        tmem_ld32(tmem + lane_base + colS + hf * HW + pc * 32, r);
+                        tmem_wait_ld();
+                        if (owns_srow) write_sb32(r, hf * HW + pc * 32);
+                    }
                     fence_proxy_async();
                     tc_fence_before();
                     mbar_arrive(bar_sb_ready);
                 }
-                COTT_STAMP(5);
+                COTT_STAMP(3);
             }
-            if (MODE != MODE_CAUSAL && c + 1 < n_chunks) { norm_phase(c + 1); if (!alive) break; }
-            if (MODE == MODE_STATE) {
-                // Follow every state update (a parity names one chunk only if no phase is
-                // skipped); after the last one the accumulator holds the group's state.
-                if (!wait(bar_s_full + 8 * (c & 1), (c >> 1) & 1)) break;
-                continue;
-            }
-
-            // ---- output epilogue of chunk c: accumulator -> bf16 rows in the staging slot
-            if (!wait(bar_o_full + 8 * (c & 1), (c >> 1) & 1)) break;
-            tc_fence_after();
-            COTT_STAMP(6);
-            const uint32_t tO = tmem + lane_base + colO0 + (c % kOBufs) * D + cq * QW;
-            const float rx = rx_buf[(c % NRX) * 128 + arow];
-            uint32_t r[QW];
-            tmem_ldq<QW>(tO, r);
-            tmem_wait_ld();
-            tc_fence_before();
-            mbar_arrive(bar_o_free + 8 * (c & 1));
-            float coef = 0.f, rp = 1.f;
-            const uint8_t* proj = L::kProjInA ? (st + L::kOffA) : (gbase + L::kOffProj);
-            uint4 pw[QW / 8];
-            if (with_proj) {
-                if (!wait(bar_proj, c & 1)) break;
-                // Per-row <p, acc> and ||p||^2: each of the four column-quarter threads sums its
-                // part; the parts meet in shared memory.
-                float2* xch = reinterpret_cast<float2*>(L::kProjInA ? (st + L::kOffX)
-                                                                    : (gbase + L::kOffProj + L::kTile));
-                float ss0 = 0.f, ss1 = 0.f, dp0 = 0.f, dp1 = 0.f;
+        } else {
+            // -------------------------------------------------------------- group O
+            norm_phase(0);
+            if (L::kSplitB && p.norm_bv && alive) norm_b(0);
+            for (int c = 0; c < n_chunks && alive; ++c) {
+                const int s = c % NST;
+                uint8_t* st = gbase + s * L::kStage;
+                if (c + 1 < n_chunks) { norm_phase(c + 1); if (!alive) break; }
+                // ---- output epilogue of chunk c: accumulator -> bf16 rows in the staging slot
+                if (!wait(bar_o_full + 8 * (c & 1), (c >> 1) & 1)) break;
+                tc_fence_after();
+                const uint32_t tO = tmem + lane_base + colO0 + (c % kOBufs) * D + hf * HW;
+                const float rx = rx_buf[(c % NRX) * 128 + arow];
+                uint32_t r[HW];
 #pragma unroll
-                for (int i = 0; i < QW; i += 8) {
-                    const int col = cq * QW + i;
-                    pw[i >> 3] = *reinterpret_cast<const uint4*>(proj + (col >> 6) * 16384 +
-                                                                 swz(arow, (col & 63) >> 3));
-                    const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&pw[i >> 3]);
+                for (int pc = 0; pc < NPIECE; ++pc)
+                    tmem_ld32(tO + pc * 32, *reinterpret_cast<uint32_t(*)[32]>(&r[pc * 32]));
+                tmem_wait_ld();
+                tc_fence_before();
+                mbar_arrive(bar_o_free + 8 * (c & 1));
+                float coef = 0.f, rp = 1.f;
+                const uint8_t* proj = L::kProjInA ? (st + L::kOffA) : (gbase + L::kOffProj);
+                auto proj_chunk = [&](int i) {       // 8 raw values next to accumulator columns hf*HW + i ..
+                    const int col = hf * HW + i;
+                    return *reinterpret_cast<const uint4*>(proj + (col >> 6) * 16384 + swz(arow, (col & 63) >> 3));
+                };
+                if (with_proj) {
+                    if (!wait(bar_proj, c & 1)) break;
+                    // Per-row <p, acc> and ||p||^2: each of the two column-half threads sums its
+                    // part; the parts meet in shared memory.
+                    float2* xch = reinterpret_cast<float2*>(L::kProjInA ? (st + L::kOffX)
+                                                                        : (gbase + L::kOffProj + L::kTile));
+                    float ss0 = 0.f, ss1 = 0.f, dp0 = 0.f, dp1 = 0.f;
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        float2 f = __bfloat1622float2(e[j]);
-                        ss0 = fmaf(f.x, f.x, ss0); ss1 = fmaf(f.y, f.y, ss1);
-                        dp0 = fmaf(f.x, __uint_as_float(r[i + 2 * j]), dp0);
-                        dp1 = fmaf(f.y, __uint_as_float(r[i + 2 * j + 1]), dp1);
+                    for (int i = 0; i < HW; i += 8) {
+                        const uint4 w = proj_chunk(i);
+                        const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&w);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            float2 f = __bfloat1622float2(e[j]);
+                            ss0 = fmaf(f.x, f.x, ss0); ss1 = fmaf(f.y, f.y, ss1);
+                            dp0 = fmaf(f.x, __uint_as_float(r[i + 2 * j]), dp0);
+                            dp1 = fmaf(f.y, __uint_as_float(r[i + 2 * j + 1]), dp1);
+                        }
+                    }
+                    xch[hf * 128 + arow] = make_float2(ss0 + ss1, dp0 + dp1);
+                    mbar_arrive(bar_xch);
+                    if (!wait(bar_xch, c & 1)) break;
+                    const float2 e0 = xch[arow], e1 = xch[128 + arow];
+                    const float ss = e0.x + e1.x, dp = e0.y + e1.y;
+                    if (p.epilogue == EPI_PROJ) {
+                        // g = rx * acc;  out = (g - p^ <p^, g>) / max(||p||, eps); clamped branch: g / eps
+                        const float nrm = sqrtf(ss);
+                        rp = 1.0f / fmaxf(nrm, kEps);
+                        coef = nrm > kEps ? dp * rx * rp * rp : 0.f;
+                    } else if (hf == 0) {
+                        dm_acc += dp * rx / cfac;  // <dV', v> with dV' = (rx / c) * acc, once per row
                     }
                 }
-                xch[cq * 128 + arow] = make_float2(ss0 + ss1, dp0 + dp1);
-                mbar_arrive(bar_xch);
-                if (!wait(bar_xch, c & 1)) break;
-                const float2 e0 = xch[arow], e1 = xch[128 + arow], e2 = xch[256 + arow], e3 = xch[384 + arow];
-                const float ss = (e0.x + e1.x) + (e2.x + e3.x), dp = (e0.y + e1.y) + (e2.y + e3.y);
-                if (p.epilogue == EPI_PROJ) {
-                    // g = rx * acc;  out = (g - p^ <p^, g>) / max(||p||, eps); clamped branch: g / eps
-                    const float nrm = sqrtf(ss);
-                    rp = 1.0f / fmaxf(nrm, kEps);
-                    coef = nrm > kEps ? dp * rx * rp * rp : 0.f;
-                } else if (cq == 0) {
-                    dm_acc += dp * rx / cfac;  // <dV', v> with dV' = (rx / c) * acc, once per row
-                }
-            }
-            // Scale, (project,) round to bf16, stage for the TMA store.
-            uint8_t* so = st + L::kOffOut;
+                // Scale, (project,) round to bf16, stage for the TMA store.  The staging slot is
+                // the Bv slot, which the state update (issued behind P~ Bv) still reads: wait for it.
+                if (MODE == MODE_CAUSAL && !wait(sfull_bar(c), sfull_par(c))) break;
+                uint8_t* so = st + L::kOffOut;
 #pragma unroll
-            for (int i = 0; i < QW; i += 8) {
-                const int col = cq * QW + i;
-                float v[8];
+                for (int i = 0; i < HW; i += 8) {
+                    const int col = hf * HW + i;
+                    float v[8];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) v[j] = __uint_as_float(r[i + j]) * rx;
-                if (with_proj && p.epilogue == EPI_PROJ) {
-                    const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&pw[i >> 3]);
+                    for (int j = 0; j < 8; ++j) v[j] = __uint_as_float(r[i + j]) * rx;
+                    if (with_proj && p.epilogue == EPI_PROJ) {
+                        const uint4 w = proj_chunk(i);
+                        const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&w);
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        float2 f = __bfloat1622float2(e[j]);
-                        v[2 * j] = (v[2 * j] - f.x * coef) * rp;
-                        v[2 * j + 1] = (v[2 * j + 1] - f.y * coef) * rp;
+                        for (int j = 0; j < 4; ++j) {
+                            float2 f = __bfloat1622float2(e[j]);
+                            v[2 * j] = (v[2 * j] - f.x * coef) * rp;
+                            v[2 * j + 1] = (v[2 * j + 1] - f.y * coef) * rp;
+                        }
                     }
+                    uint4 w;
+                    w.x = pack_bf16(v[0], v[1]); w.y = pack_bf16(v[2], v[3]);
+                    w.z = pack_bf16(v[4], v[5]); w.w = pack_bf16(v[6], v[7]);
+                    *reinterpret_cast<uint4*>(so + (col >> 6) * 16384 + swz(arow, (col & 63) >> 3)) = w;
                 }
-                uint4 w;
-                w.x = pack_bf16(v[0], v[1]); w.y = pack_bf16(v[2], v[3]);
-                w.z = pack_bf16(v[4], v[5]); w.w = pack_bf16(v[6], v[7]);
-                *reinterpret_cast<uint4*>(so + (col >> 6) * 16384 + swz(arow, (col & 63) >> 3)) = w;
+                fence_proxy_async();
+                mbar_arrive(bar_e_done + 8 * (c & 1));
+                // Bv of the next chunk lands last; normalise it (when it is the one) after this
+                // chunk's epilogue, before the tensor core needs it.
+                if (L::kSplitB && p.norm_bv && c + 1 < n_chunks) { norm_b(c + 1); if (!alive) break; }
+                COTT_STAMP(6);
             }
-            fence_proxy_async();
-            mbar_arrive(bar_e_done + 8 * (c & 1));
         }
 
         if (MODE == MODE_STATE && alive && p.state_out != nullptr) {
@@ -779,8 +779,8 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     tc_fence_before();
     __syncthreads();
     if (MODE != MODE_STATE && p.dm_partial != nullptr && tid == 0 && !*abort_flag) {
-        // Fixed-order reduction of <dV', V> over the CTA (only the cq == 0 warps hold sums).
-        p.dm_partial[(size_t)bh * p.n_groups + g] = (dm_red[0] + dm_red[1]) + (dm_red[2] + dm_red[3]);
+        // Fixed-order reduction of <dV', V> over the CTA (the first-half warps of group O hold sums).
+        p.dm_partial[(size_t)bh * p.n_groups + g] = (dm_red[8] + dm_red[9]) + (dm_red[10] + dm_red[11]);
     }
     if (tid == 0 && *abort_flag) atomicExch(p.status, 1);
     if (is_ctrl) tmem_dealloc(tmem, kTmemCols);
