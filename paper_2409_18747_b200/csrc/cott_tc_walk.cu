@@ -105,13 +105,13 @@ __device__ __forceinline__ void issue_p(uint32_t tP, uint32_t x, uint32_t a) {
     }
 }
 template <int D>
-__device__ __forceinline__ void issue_xs(uint32_t tO, uint32_t x, uint32_t sb, bool acc_first = false) {
+__device__ __forceinline__ void issue_xs(uint32_t tO, uint32_t x, uint32_t sb) {
     constexpr uint32_t idesc = instr_desc_bf16(128, D, false, true);
 #pragma unroll
     for (int kk = 0; kk < D / 16; ++kk) {
         const uint32_t off = (kk >> 2) * 16384u + (kk & 3) * 32u;
         mma_ss(tO, smem_desc(x + off, 16, 1024), smem_desc(sb + kk * 2048u, D * 128u, 1024), idesc,
-               (kk > 0) || acc_first);
+               kk > 0);
     }
 }
 template <int D>
@@ -202,9 +202,9 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     constexpr int NST = L::kStages;
     constexpr int NH = D / 64;                       // 64-column half tiles per row
     constexpr uint32_t kTmemCols = 512;
-    // Columns: State d | P 128 (fp32 scores) | P~ 2 x 64 (bf16 masked scores, packed, double-
-    // buffered) | Out.  d = 64 double-buffers Out; at d = 128 one Out buffer fills the 512.
-    constexpr uint32_t colS = 0, colP = D, colPt = D + 128, colO0 = D + 256;
+    // Columns: State d | P 128 (fp32 scores) | P~ 64 (bf16 masked scores, packed) | Out.
+    // d = 64 double-buffers Out; at d = 128 only one Out buffer fits in the 512 columns.
+    constexpr uint32_t colS = 0, colP = D, colPt = D + 128, colO0 = D + 192;
     constexpr int kOBufs = (D == 64) ? 2 : 1;
     constexpr int QW = D / 4;                        // accumulator columns per worker thread
     extern __shared__ uint8_t smem_raw[];
@@ -404,7 +404,14 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 const int s = c % NST;
                 if (!wait(bar_a_ready + 8 * s, (c / NST) & 1)) return;
                 const bool acc = init_state || c > 0;
+                if (MODE == MODE_CAUSAL) {
+                    // Scores first: they need neither the state copy nor the output buffer.
+                    tc_fence_after();
+                    issue_p<D>(tmem + colP, stage_x(s), stage_a(s));
+                    tc_commit(bar_p_full);
+                }
                 if (MODE != MODE_STATE) {
+                    if (MODE == MODE_CAUSAL && c >= 1 && !wait(bar_sb_ready, (c - 1) & 1)) return;
                     // The output accumulator this chunk writes must have been drained: by chunk
                     // c - 2 with two buffers, by chunk c - 1 with one.
                     if (kOBufs == 2) { if (c >= 2 && !wait(bar_o_free + 8 * (c & 1), ((c >> 1) & 1) ^ 1)) return; }
@@ -413,7 +420,10 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 tc_fence_after();
                 const uint32_t tO = tmem + colO0 + (c % kOBufs) * D;
                 if (MODE == MODE_CAUSAL) {
-                    // (the causal walk has its own schedule below)
+                    // The state update of this chunk is issued later, behind P~ Bv, so that
+                    // the workers mask the scores without the tensor core hammering shared
+                    // memory and TMEM at the same time.
+                    if (acc) issue_xs<D>(tO, stage_x(s), sb);
                 } else if (MODE == MODE_STATE) {
                     issue_atb<D>(tmem + colS, stage_a(s), stage_b(s), acc);
                     tc_commit(sfull_bar(c));
@@ -427,122 +437,70 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             // output staging slot) after the chunk's output store has drained.
             const bool split_refill = MODE == MODE_CAUSAL && !(with_proj && L::kProjInA);
             for (int c = 0; c < NST && c < n_chunks; ++c) issue_loads(c, true, true);
-            if (MODE == MODE_CAUSAL) {
-                // ---- causal walk.  Tensor-pipe order per chunk c: scores of chunk c+1 (they
-                // only need the next tiles and a free score buffer), then P~ Bv and X State of
-                // chunk c into its output accumulator, then the state update.  So the workers
-                // mask chunk c+1 while the tensor core finishes chunk c.
-                int p_next = 0;   // first chunk whose score MMA has not been issued yet
-                auto issue_scores = [&](int c, bool blocking) {
-                    const int s = c % NST;
-                    if (blocking) { if (!wait(bar_a_ready + 8 * s, (c / NST) & 1)) return; }
-                    else if (!mbar_try_wait(bar_a_ready + 8 * s, (c / NST) & 1)) return;
-                    tc_fence_after();
-                    issue_p<D>(tmem + colP, stage_x(s), stage_a(s));
-                    tc_commit(bar_p_full);
-                    p_next = c + 1;
+            batch1(0);
+            for (int c = 0; c < n_chunks && alive; ++c) {
+                const int s = c % NST;
+                const bool more = c + NST < n_chunks;
+                COTT_STAMP(0);
+                auto load_proj = [&]() {
+                    const uint32_t proj_u = L::kProjInA ? stage_a(s) : base + L::kOffProj;
+                    mbar_expect_tx(bar_proj, L::kTile);
+                    load_tile(proj_u, &tmP, bar_proj, chunk_row(c));
                 };
-                issue_scores(0, true);
-                for (int c = 0; c < n_chunks && alive; ++c) {
-                    const int s = c % NST;
-                    const bool more = c + NST < n_chunks;
-                    auto load_proj = [&]() {
-                        const uint32_t proj_u = L::kProjInA ? stage_a(s) : base + L::kOffProj;
-                        mbar_expect_tx(bar_proj, L::kTile);
-                        load_tile(proj_u, &tmP, bar_proj, chunk_row(c));
-                    };
-                    if (with_proj && !L::kProjInA) {
-                        // Dedicated buffer: free once the previous chunk's epilogue has finished.
-                        if (c >= 1 && !wait(bar_e_done + 8 * ((c - 1) & 1), ((c - 1) >> 1) & 1)) break;
-                        load_proj();
-                    }
-                    COTT_STAMP(0);
-                    if (!wait(bar_pt_ready, c & 1)) break;     // P~(c) written, score buffer free
-                    COTT_STAMP(1);
-                    if (c + 1 < n_chunks && p_next == c + 1) issue_scores(c + 1, false);
-                    // The output accumulator of this chunk must have been drained: by chunk
-                    // c - 2 with two buffers, by chunk c - 1 with one.
-                    if (kOBufs == 2) { if (c >= 2 && !wait(bar_o_free + 8 * (c & 1), ((c >> 1) & 1) ^ 1)) break; }
-                    else if (c >= 1 && !wait(bar_o_free + 8 * ((c - 1) & 1), ((c - 1) >> 1) & 1)) break;
-                    // Bv: landed, and normalised if it is the operand whose row scale sits on
-                    // the contraction index.
+                if (with_proj && !L::kProjInA) {
+                    // Dedicated buffer: free once the previous chunk's epilogue has finished.
+                    if (c >= 1 && !wait(bar_e_done + 8 * ((c - 1) & 1), ((c - 1) >> 1) & 1)) break;
+                    load_proj();
+                }
+                if (MODE == MODE_CAUSAL) {
+                    if (!wait(bar_pt_ready, c & 1)) break;
+                    // Bv is needed from here on: landed, and normalised if it is the operand
+                    // whose row scale sits on the contraction index.
                     if (L::kSplitB) {
                         if (!wait(bar_full_b + 8 * s, (c / NST) & 1)) break;
                         if (p.norm_bv && !wait(bar_b_ready + 8 * s, (c / NST) & 1)) break;
                     }
+                    COTT_STAMP(1);
                     tc_fence_after();
                     const bool acc = init_state || c > 0;
-                    const uint32_t tO = tmem + colO0 + (c % kOBufs) * D;
-                    issue_pb<D>(tO, tmem + colPt + (c & 1) * 64, stage_b(s), false);
-                    if (acc) {
-                        // X State needs the bf16 copy of the previous chunk's state; the same
-                        // hand-off says the workers are done reading the fp32 state.
-                        if (c >= 1 && !wait(bar_sb_ready, (c - 1) & 1)) break;
-                        tc_fence_after();
-                        issue_xs<D>(tO, stage_x(s), sb, true);
-                    }
+                    issue_pb<D>(tmem + colO0 + (c % kOBufs) * D, tmem + colPt, stage_b(s), acc);
                     tc_commit(bar_o_full + 8 * (c & 1));
                     issue_atb<D>(tmem + colS, stage_a(s), stage_b(s), acc);
                     tc_commit(sfull_bar(c));
-                    COTT_STAMP(2);
-                    if (c + 1 < n_chunks && p_next == c + 1) { issue_scores(c + 1, true); if (!alive) break; }
-                    COTT_STAMP(3);
                     if (with_proj && L::kProjInA) {
                         // The A slot is free once the state update has read it.
                         if (!wait(sfull_bar(c), sfull_par(c))) break;
                         load_proj();
                     }
-                    if (split_refill && more) {
-                        if (!wait(sfull_bar(c), sfull_par(c))) break;   // covers every MMA of the chunk
-                        issue_loads(c + NST, true, false);
-                    }
-                    COTT_STAMP(4);
-                    // Output rows staged by the workers: store them, then finish the refill.
-                    if (!wait(bar_e_done + 8 * (c & 1), (c >> 1) & 1)) break;
-                    {
-                        const uint32_t src = base + s * L::kStage + L::kOffOut;
-#pragma unroll
-                        for (int hh = 0; hh < NH; ++hh)
-                            tma_store_3d(&tmO, src + hh * 16384, hh * 64, chunk_row(c), bh);
-                        tma_store_commit();
-                    }
-                    COTT_STAMP(5);
-                    if (more) {
-                        tma_store_wait_read0();
-                        issue_loads(c + NST, !split_refill, true);
-                    }
-                    COTT_STAMP(6);
                 }
-            } else {
-                batch1(0);
-                for (int c = 0; c < n_chunks && alive; ++c) {
-                    const int s = c % NST;
-                    const bool more = c + NST < n_chunks;
-                    if (MODE == MODE_STATE) {
-                        if (more) { if (!wait(sfull_bar(c), sfull_par(c))) break; issue_loads(c + NST, true, true); }
-                        if (c + 1 < n_chunks) batch1(c + 1);
-                        continue;
-                    }
-                    // ---- read-out: one X State product per chunk
-                    if (with_proj) {
-                        if (c >= 1 && !wait(bar_e_done + 8 * ((c - 1) & 1), ((c - 1) >> 1) & 1)) break;
-                        mbar_expect_tx(bar_proj, L::kTile);
-                        load_tile(base + L::kOffProj, &tmP, bar_proj, chunk_row(c));
-                    }
-                    if (c + 1 < n_chunks) { batch1(c + 1); if (!alive) break; }
-                    if (!wait(bar_e_done + 8 * (c & 1), (c >> 1) & 1)) break;
-                    {
-                        const uint32_t src = base + s * L::kStage + L::kOffOut;
-#pragma unroll
-                        for (int hh = 0; hh < NH; ++hh)
-                            tma_store_3d(&tmO, src + hh * 16384, hh * 64, chunk_row(c), bh);
-                        tma_store_commit();
-                    }
-                    if (more) {
-                        tma_store_wait_read0();
-                        issue_loads(c + NST, true, true);
-                    }
+                COTT_STAMP(2);
+                if (MODE == MODE_STATE) {
+                    if (more) { if (!wait(sfull_bar(c), sfull_par(c))) break; issue_loads(c + NST, true, true); }
+                    if (c + 1 < n_chunks) batch1(c + 1);
+                    continue;
                 }
+                if (split_refill && more) {
+                    if (!wait(sfull_bar(c), sfull_par(c))) break;   // covers P~ Bv too
+                    issue_loads(c + NST, true, false);
+                }
+                COTT_STAMP(3);
+                if (c + 1 < n_chunks) { batch1(c + 1); if (!alive) break; }
+                COTT_STAMP(4);
+                // Output rows staged by the workers: store them, then finish the refill.
+                if (!wait(bar_e_done + 8 * (c & 1), (c >> 1) & 1)) break;
+                {
+                    const uint32_t src = base + s * L::kStage + L::kOffOut;
+#pragma unroll
+                    for (int hh = 0; hh < NH; ++hh)
+                        tma_store_3d(&tmO, src + hh * 16384, hh * 64, chunk_row(c), bh);
+                    tma_store_commit();
+                }
+                COTT_STAMP(5);
+                if (more) {
+                    tma_store_wait_read0();
+                    issue_loads(c + NST, !split_refill, true);
+                }
+                COTT_STAMP(6);
             }
             tma_store_wait_all0();
         }
@@ -645,13 +603,15 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             if (alive) wait(sfull_bar(n_chunks - 1), sfull_par(n_chunks - 1));
         } else if (grp == 0) {
             // -------------------------------------------------------------- group P
-            // Masked scores -> bf16 operand P~ in tensor memory.  Forward: row i keeps columns
-            // j <= i (diagonal kept, Eq. 6); backward in time: j >= i.  Per 32 x 32 block (row
-            // block q, column block cb) the mask is all-keep, all-zero or, on the diagonal, a
-            // triangle; the first two cases are warp-uniform.
-            auto mask_scores = [&](int c) {
-                if (!wait(bar_p_full, c & 1)) return;
+            for (int c = 0; MODE == MODE_CAUSAL && c < n_chunks && alive; ++c) {
+                // Masked scores -> bf16 operand P~ in tensor memory.  Forward: row i keeps
+                // columns j <= i (diagonal kept, Eq. 6); backward in time: j >= i.  Per
+                // 32 x 32 block (row block q, column block cb) the mask is all-keep, all-zero
+                // or, on the diagonal, a triangle; the first two cases are warp-uniform.
+                COTT_STAMP(0);
+                if (!wait(bar_p_full, c & 1)) break;
                 tc_fence_after();
+                COTT_STAMP(1);
 #pragma unroll
                 for (int sbk = 0; sbk < 2; ++sbk) {
                     const int cb = 2 * hf + sbk;
@@ -673,38 +633,32 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                         for (int j = 0; j < 32; ++j) r[j] = 0u;
                     }
                     // bf16, two scores per column (even column index in the low half): this
-                    // block's 32 k-values are 16 columns of the A-operand buffer of this chunk.
+                    // block's 32 k-values are 16 columns of the A-operand region.
                     uint32_t pk[16];
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
                         pk[j] = pack_bf16(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
-                    tmem_st16(tmem + lane_base + colPt + (c & 1) * 64 + cb * 16, pk);
+                    tmem_st16(tmem + lane_base + colPt + cb * 16, pk);
                 }
                 tmem_wait_st();
+                COTT_STAMP(2);
                 tc_fence_before();
                 mbar_arrive(bar_pt_ready);
-            };
-            if (MODE == MODE_CAUSAL && alive) mask_scores(0);
-            for (int c = 0; MODE == MODE_CAUSAL && c + 1 < n_chunks && alive; ++c) {
-                COTT_STAMP(0);
-                // Scores of the next chunk first (the tensor core computed them ahead) ...
-                mask_scores(c + 1);
-                if (!alive) break;
-                COTT_STAMP(1);
-                // ... then the bf16 copy of this chunk's updated state for the next X State.
-                if (!wait(sfull_bar(c), sfull_par(c))) break;
-                tc_fence_after();
-                COTT_STAMP(2);
+                // bf16 copy of the updated state for the next chunk's X State product.
+                if (c + 1 < n_chunks) {
+                    if (!wait(sfull_bar(c), sfull_par(c))) break;
+                    tc_fence_after();
 #pragma unroll
-                for (int pc = 0; pc < NPIECE; ++pc) {
-                    uint32_t r[32];
-                    tmem_ld32(tmem + lane_base + colS + hf * HW + pc * 32, r);
-                    tmem_wait_ld();
-                    if (owns_srow) write_sb32(r, hf * HW + pc * 32);
+                    for (int pc = 0; pc < NPIECE; ++pc) {
+                        uint32_t r[32];
+                        tmem_ld32(tmem + lane_base + colS + hf * HW + pc * 32, r);
+                        tmem_wait_ld();
+                        if (owns_srow) write_sb32(r, hf * HW + pc * 32);
+                    }
+                    fence_proxy_async();
+                    tc_fence_before();
+                    mbar_arrive(bar_sb_ready);
                 }
-                fence_proxy_async();
-                tc_fence_before();
-                mbar_arrive(bar_sb_ready);
                 COTT_STAMP(3);
             }
         } else {
