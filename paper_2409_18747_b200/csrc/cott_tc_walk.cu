@@ -40,13 +40,19 @@ struct TcWalkParams {
     int* status;            // workspace status word
     const float* m; const float* seq_len; float seq_len_scalar;
     int H; int N; int group; int n_groups;
-    int norm_bv;            // 1: Bv is normalised in shared memory, 0: A is
-    int x_norm;             // 1: rows of X are normalised (scale applied in the epilogue)
-    int epilogue;           // Epilogue enum
-    int reverse;            // 1: walk backward in time, mask keeps columns >= row
 };
 
 enum { MODE_STATE = 0, MODE_CAUSAL = 1, MODE_READOUT = 2 };
+
+// Output stream a kernel instance serves.  The operand roles, the direction of time and the
+// epilogue are compile-time properties, so that every instance carries only its own code (the
+// walk is sensitive to instruction-cache misses: ncu showed 'no instruction' as the top stall
+// of the d = 128 causal walk when all variants shared one body).
+//   S_FWD: X rows normalised in the epilogue, A normalised in shared memory, plain store
+//   S_DQ : Bv normalised, projection epilogue
+//   S_DK : as S_DQ, time reversed
+//   S_DV : as S_FWD, time reversed, scale + <dV', V> epilogue
+enum { S_FWD = 0, S_DQ = 1, S_DK = 2, S_DV = 3 };
 
 constexpr int kWorkerWarps = 16;                      // row-worker warps (4 per TMEM lane quadrant)
 constexpr int kWorkers = kWorkerWarps * 32;
@@ -193,7 +199,7 @@ template <> __device__ __forceinline__ void tmem_stq<16>(uint32_t taddr, const u
 // chunks at once (score masking + state copy / row norms + output epilogue); warp 16 lane 0
 // is the control thread (TMA loads / stores and all tcgen05.mma).  The roles meet only
 // through mbarriers, every wait bounded.
-template <int D, int MODE>
+template <int D, int MODE, int STREAM>
 __global__ void __launch_bounds__(kTcThreads, 1)
 tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmA,
                const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmP,
@@ -244,7 +250,11 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     const int tok0 = g * p.group;
     const int tok1 = min(p.N, tok0 + p.group);
     const int n_chunks = (tok1 - tok0 + kChunk - 1) / kChunk;
-    const bool with_proj = (MODE != MODE_STATE) && (p.epilogue != EPI_PLAIN);
+    constexpr bool kNormBv = STREAM == S_DQ || STREAM == S_DK;
+    constexpr bool kXNorm = STREAM == S_FWD || STREAM == S_DV;
+    constexpr bool kReverse = STREAM == S_DK || STREAM == S_DV;
+    constexpr int kEpi = STREAM == S_FWD ? EPI_PLAIN : (STREAM == S_DV ? EPI_DV : EPI_PROJ);
+    constexpr bool with_proj = (MODE != MODE_STATE) && (kEpi != EPI_PLAIN);
     const bool is_ctrl = warp == kWorkerWarps;
 
     if (is_ctrl) {
@@ -294,7 +304,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     auto stage_x = [&](int s) { return base + s * L::kStage + L::kOffX; };
     auto stage_a = [&](int s) { return base + s * L::kStage + L::kOffA; };
     auto stage_b = [&](int s) { return base + s * L::kStage + L::kOffB; };
-    auto chunk_row = [&](int c) { return tok0 + (p.reverse ? (n_chunks - 1 - c) : c) * kChunk; };
+    auto chunk_row = [&](int c) { return tok0 + (kReverse ? (n_chunks - 1 - c) : c) * kChunk; };
 
     // bf16 copy of QW state columns of this thread's row into the MN-major state tile.
     auto write_sb = [&](const uint32_t (&r)[QW], int c0) {
@@ -332,8 +342,8 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             float acc[QW];
 #pragma unroll
             for (int i = 0; i < QW; ++i) acc[i] = 0.f;
-            const int g_lo = (MODE == MODE_READOUT) ? 0 : (p.reverse ? g + 1 : 0);
-            const int g_hi = (MODE == MODE_READOUT) ? p.n_groups : (p.reverse ? p.n_groups : g);
+            const int g_lo = (MODE == MODE_READOUT) ? 0 : (kReverse ? g + 1 : 0);
+            const int g_hi = (MODE == MODE_READOUT) ? p.n_groups : (kReverse ? p.n_groups : g);
             if (owns_srow) {
                 for (int gg = g_lo; gg < g_hi; ++gg) {
 #pragma unroll
@@ -458,7 +468,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     // whose row scale sits on the contraction index.
                     if (L::kSplitB) {
                         if (!wait(bar_full_b + 8 * s, (c / NST) & 1)) break;
-                        if (p.norm_bv && !wait(bar_b_ready + 8 * s, (c / NST) & 1)) break;
+                        if (kNormBv && !wait(bar_b_ready + 8 * s, (c / NST) & 1)) break;
                     }
                     COTT_STAMP(1);
                     tc_fence_after();
@@ -560,7 +570,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             uint8_t* st = gbase + s * L::kStage;
             if (L::kHasX) {
                 float rx = cfac;
-                if (p.x_norm) {
+                if (kXNorm) {
                     float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
                     for (int j = 0; j < NC; j += 2) {
@@ -572,8 +582,8 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 if (nhalf == 0) rx_buf[(c % NRX) * 128 + nrow] = rx;
             }
             // In the split causal walk Bv arrives on its own barrier and is normalised later.
-            if (L::kHasAB && !(L::kSplitB && p.norm_bv))
-                normalise_half_row(st + (p.norm_bv ? L::kOffB : L::kOffA));
+            if (L::kHasAB && !(L::kSplitB && kNormBv))
+                normalise_half_row(st + (kNormBv ? L::kOffB : L::kOffA));
             mbar_arrive(bar_a_ready + 8 * s);
         };
         // Split causal walk, Bv is the normalised operand (dQ^ and dK^ streams).
@@ -615,7 +625,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
 #pragma unroll
                 for (int sbk = 0; sbk < 2; ++sbk) {
                     const int cb = 2 * hf + sbk;
-                    const bool keep_all = p.reverse ? (cb > q) : (cb < q);
+                    const bool keep_all = kReverse ? (cb > q) : (cb < q);
                     const bool diag = cb == q;
                     uint32_t r[32];
                     if (keep_all || diag) {
@@ -624,7 +634,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                         if (diag) {
 #pragma unroll
                             for (int j = 0; j < 32; ++j) {
-                                const bool keep = p.reverse ? (j >= lane) : (j <= lane);
+                                const bool keep = kReverse ? (j >= lane) : (j <= lane);
                                 r[j] = keep ? r[j] : 0u;
                             }
                         }
@@ -664,7 +674,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         } else {
             // -------------------------------------------------------------- group O
             norm_phase(0);
-            if (L::kSplitB && p.norm_bv && alive) norm_b(0);
+            if (L::kSplitB && kNormBv && alive) norm_b(0);
             for (int c = 0; c < n_chunks && alive; ++c) {
                 const int s = c % NST;
                 uint8_t* st = gbase + s * L::kStage;
@@ -711,7 +721,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     if (!wait(bar_xch, c & 1)) break;
                     const float2 e0 = xch[arow], e1 = xch[128 + arow];
                     const float ss = e0.x + e1.x, dp = e0.y + e1.y;
-                    if (p.epilogue == EPI_PROJ) {
+                    if (kEpi == EPI_PROJ) {
                         // g = rx * acc;  out = (g - p^ <p^, g>) / max(||p||, eps); clamped branch: g / eps
                         const float nrm = sqrtf(ss);
                         rp = 1.0f / fmaxf(nrm, kEps);
@@ -730,7 +740,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     float v[8];
 #pragma unroll
                     for (int j = 0; j < 8; ++j) v[j] = __uint_as_float(r[i + j]) * rx;
-                    if (with_proj && p.epilogue == EPI_PROJ) {
+                    if (with_proj && kEpi == EPI_PROJ) {
                         const uint4 w = proj_chunk(i);
                         const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&w);
 #pragma unroll
@@ -749,7 +759,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 mbar_arrive(bar_e_done + 8 * (c & 1));
                 // Bv of the next chunk lands last; normalise it (when it is the one) after this
                 // chunk's epilogue, before the tensor core needs it.
-                if (L::kSplitB && p.norm_bv && c + 1 < n_chunks) { norm_b(c + 1); if (!alive) break; }
+                if (L::kSplitB && kNormBv && c + 1 < n_chunks) { norm_b(c + 1); if (!alive) break; }
                 COTT_STAMP(6);
             }
         }
@@ -820,17 +830,17 @@ bool make_tile_map(CUtensorMap* map, const void* ptr, int BH, int N, int d) {
     return r == CUDA_SUCCESS;
 }
 
-template <int D, int MODE>
+template <int D, int MODE, int STREAM>
 cudaError_t launch_mode(const CUtensorMap* tm, const TcWalkParams& p, int BH, cudaStream_t st) {
-    auto kern = tc_walk_kernel<D, MODE>;
+    auto kern = tc_walk_kernel<D, MODE, STREAM>;
+    constexpr bool with_proj = (MODE != MODE_STATE) && (STREAM != S_FWD);
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             Smem<D, MODE>::dyn_bytes(MODE != MODE_STATE));
+                                             Smem<D, MODE>::dyn_bytes(with_proj));
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    const bool with_proj = (MODE != MODE_STATE) && (p.epilogue != EPI_PLAIN);
     const int prof = profile_begin_launch(MODE, st);
     // Programmatic dependent launch: this kernel may start (allocate TMEM, set up barriers,
     // prefetch tensor maps) while the previous kernel of the stream drains; it waits for that
@@ -851,6 +861,28 @@ cudaError_t launch_mode(const CUtensorMap* tm, const TcWalkParams& p, int BH, cu
     return le != cudaSuccess ? le : cudaGetLastError();
 }
 
+template <int D>
+cudaError_t launch_d(int mode, int stream_kind, const CUtensorMap* tm, const TcWalkParams& p, int BH,
+                     cudaStream_t st) {
+    if (mode == MODE_STATE)   // only the operand that is normalised distinguishes the instances
+        return (stream_kind == S_DQ || stream_kind == S_DK) ? launch_mode<D, MODE_STATE, S_DQ>(tm, p, BH, st)
+                                                            : launch_mode<D, MODE_STATE, S_FWD>(tm, p, BH, st);
+    if (mode == MODE_CAUSAL) {
+        switch (stream_kind) {
+            case S_FWD: return launch_mode<D, MODE_CAUSAL, S_FWD>(tm, p, BH, st);
+            case S_DQ: return launch_mode<D, MODE_CAUSAL, S_DQ>(tm, p, BH, st);
+            case S_DK: return launch_mode<D, MODE_CAUSAL, S_DK>(tm, p, BH, st);
+            default: return launch_mode<D, MODE_CAUSAL, S_DV>(tm, p, BH, st);
+        }
+    }
+    switch (stream_kind) {
+        case S_FWD: return launch_mode<D, MODE_READOUT, S_FWD>(tm, p, BH, st);
+        case S_DQ: return launch_mode<D, MODE_READOUT, S_DQ>(tm, p, BH, st);
+        case S_DK: return launch_mode<D, MODE_READOUT, S_DK>(tm, p, BH, st);
+        default: return launch_mode<D, MODE_READOUT, S_DV>(tm, p, BH, st);
+    }
+}
+
 }  // namespace
 
 cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cudaStream_t st) {
@@ -866,18 +898,17 @@ cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cuda
     p.init = a.init; p.state_out = a.state_out; p.dm_partial = a.dm_partial; p.status = a.status;
     p.m = a.m; p.seq_len = a.seq_len; p.seq_len_scalar = a.seq_len_scalar;
     p.H = H; p.N = N; p.group = a.group; p.n_groups = a.n_groups;
-    p.norm_bv = a.norm_bv; p.x_norm = a.x_norm; p.epilogue = a.epilogue; p.reverse = a.reverse;
     p.init_sum = a.init_sum; p.init_transposed = a.init_transposed;
-    if (d == 128) {
-        if (a.mode == MODE_STATE) return launch_mode<128, MODE_STATE>(tm, p, BH, st);
-        if (a.mode == MODE_CAUSAL) return launch_mode<128, MODE_CAUSAL>(tm, p, BH, st);
-        return launch_mode<128, MODE_READOUT>(tm, p, BH, st);
-    }
-    if (d == 64) {
-        if (a.mode == MODE_STATE) return launch_mode<64, MODE_STATE>(tm, p, BH, st);
-        if (a.mode == MODE_CAUSAL) return launch_mode<64, MODE_CAUSAL>(tm, p, BH, st);
-        return launch_mode<64, MODE_READOUT>(tm, p, BH, st);
-    }
+    // The four combinations of roles the library uses, as compile-time kernel variants.
+    int kind;
+    if (a.epilogue == EPI_PLAIN && !a.norm_bv && a.x_norm && !a.reverse) kind = S_FWD;
+    else if (a.epilogue == EPI_PROJ && a.norm_bv && !a.x_norm && !a.reverse) kind = S_DQ;
+    else if (a.epilogue == EPI_PROJ && a.norm_bv && !a.x_norm && a.reverse) kind = S_DK;
+    else if (a.epilogue == EPI_DV && !a.norm_bv && a.x_norm && a.reverse) kind = S_DV;
+    else if (a.mode == MODE_STATE) kind = a.norm_bv ? S_DQ : S_FWD;
+    else return cudaErrorInvalidValue;
+    if (d == 128) return launch_d<128>(a.mode, kind, tm, p, BH, st);
+    if (d == 64) return launch_d<64>(a.mode, kind, tm, p, BH, st);
     return cudaErrorInvalidValue;
 }
 
