@@ -622,7 +622,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 if (!wait(bar_p_full, c & 1)) break;
                 tc_fence_after();
                 COTT_STAMP(1);
-#pragma unroll
+#pragma unroll 1
                 for (int sbk = 0; sbk < 2; ++sbk) {
                     const int cb = 2 * hf + sbk;
                     const bool keep_all = kReverse ? (cb > q) : (cb < q);
@@ -658,7 +658,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 if (c + 1 < n_chunks) {
                     if (!wait(sfull_bar(c), sfull_par(c))) break;
                     tc_fence_after();
-#pragma unroll
+#pragma unroll 1
                     for (int pc = 0; pc < NPIECE; ++pc) {
                         uint32_t r[32];
                         tmem_ld32(tmem + lane_base + colS + hf * HW + pc * 32, r);
