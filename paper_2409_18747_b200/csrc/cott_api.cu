@@ -165,6 +165,7 @@ static cott_status run_tc_stream(TcWalkArgs t, const Plan& p, int B, int H, int 
         TcWalkArgs a = t;
         a.mode = 0; a.x = nullptr; a.proj = nullptr; a.out = nullptr; a.init = nullptr;
         a.state_out = states; a.dm_partial = nullptr; a.epilogue = EPI_PLAIN;
+        a.reverse = t.reverse ? 0 : 1;   // chunk order opposite to the walk's: L2 reuse of its tiles
         COTT_CUDA(launch_tc_walk(a, B, H, N, d, st));
         const int mode = !causal ? SCAN_TOTAL : (t.reverse ? SCAN_SUFFIX : SCAN_PREFIX);
         if (!fused_scan)

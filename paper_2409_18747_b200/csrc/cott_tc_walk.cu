@@ -32,6 +32,7 @@ constexpr uint64_t kWaitTimeoutNs = 2000000000ull;  // 2 s: far above any legiti
 struct TcWalkParams {
     const float* init;      // [BH, n_groups, d*d] unscaled group states, or NULL
     int init_transposed;    // 1: init holds the transposes of the states this walk needs
+    int state_rev;          // state-only pass: visit the chunks of a group last to first
     int init_sum;           // 0: init holds this group's start state; 1: it holds raw partial
                             // states, to be summed here over the groups before (after, when
                             // time runs backward; all, for the read-out) this one
@@ -304,7 +305,11 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     auto stage_x = [&](int s) { return base + s * L::kStage + L::kOffX; };
     auto stage_a = [&](int s) { return base + s * L::kStage + L::kOffA; };
     auto stage_b = [&](int s) { return base + s * L::kStage + L::kOffB; };
-    auto chunk_row = [&](int c) { return tok0 + (kReverse ? (n_chunks - 1 - c) : c) * kChunk; };
+    // Chunk visited at step c.  The state-only pass may take either order (its result does not
+    // depend on it): it takes the opposite of the walk that follows, so that the tiles it
+    // read last -- still in L2 -- are the ones the walk needs first.
+    const bool backward = (MODE == MODE_STATE) ? (p.state_rev != 0) : kReverse;
+    auto chunk_row = [&](int c) { return tok0 + (backward ? (n_chunks - 1 - c) : c) * kChunk; };
 
     // bf16 copy of QW state columns of this thread's row into the MN-major state tile.
     auto write_sb = [&](const uint32_t (&r)[QW], int c0) {
@@ -899,6 +904,7 @@ cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cuda
     p.m = a.m; p.seq_len = a.seq_len; p.seq_len_scalar = a.seq_len_scalar;
     p.H = H; p.N = N; p.group = a.group; p.n_groups = a.n_groups;
     p.init_sum = a.init_sum; p.init_transposed = a.init_transposed;
+    p.state_rev = (a.mode == MODE_STATE) ? a.reverse : 0;
     // The four combinations of roles the library uses, as compile-time kernel variants.
     int kind;
     if (a.epilogue == EPI_PLAIN && !a.norm_bv && a.x_norm && !a.reverse) kind = S_FWD;
