@@ -166,6 +166,11 @@ static cott_status run_tc_stream(TcWalkArgs t, const Plan& p, int B, int H, int 
         a.mode = 0; a.x = nullptr; a.proj = nullptr; a.out = nullptr; a.init = nullptr;
         a.state_out = states; a.dm_partial = nullptr; a.epilogue = EPI_PLAIN;
         a.reverse = t.reverse ? 0 : 1;   // chunk order opposite to the walk's: L2 reuse of its tiles
+        if (causal && !total_out) {
+            // Nobody reads the partial state of the group the walk visits last.
+            a.grid_groups = p.n_groups - 1;
+            a.first_group = t.reverse ? 1 : 0;
+        }
         COTT_CUDA(launch_tc_walk(a, B, H, N, d, st));
         const int mode = !causal ? SCAN_TOTAL : (t.reverse ? SCAN_SUFFIX : SCAN_PREFIX);
         if (!fused_scan)

@@ -64,6 +64,10 @@ struct TcWalkArgs {
     int norm_bv; int x_norm; int epilogue; int reverse;
     int init_sum;   // 1: `init` holds raw partial states; the walk forms its own prefix / suffix / total
     int init_transposed;  // 1: `init` holds the transposes of the states this walk starts from
+    // State-only pass: groups first_group .. first_group + grid_groups - 1 are computed
+    // (grid_groups == 0 means all of them).  A causal walk never reads the partial state of
+    // the group it visits last, so that group is left out unless the total is exported.
+    int first_group; int grid_groups;
 };
 cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cudaStream_t st);
 

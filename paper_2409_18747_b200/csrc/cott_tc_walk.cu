@@ -41,6 +41,7 @@ struct TcWalkParams {
     int* status;            // workspace status word
     const float* m; const float* seq_len; float seq_len_scalar;
     int H; int N; int group; int n_groups;
+    int first_group; int grid_groups;   // groups this launch covers: one CTA per (b, h, group)
 };
 
 enum { MODE_STATE = 0, MODE_CAUSAL = 1, MODE_READOUT = 2 };
@@ -246,7 +247,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     float* dm_red = reinterpret_cast<float*>(gbase + L::kOffRx + NRX * 512);     // [16]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int g = blockIdx.x % p.n_groups, bh = blockIdx.x / p.n_groups;
+    const int g = p.first_group + blockIdx.x % p.grid_groups, bh = blockIdx.x / p.grid_groups;
     const int b = bh / p.H, h = bh % p.H;
     const int tok0 = g * p.group;
     const int tok1 = min(p.N, tok0 + p.group);
@@ -851,7 +852,7 @@ cudaError_t launch_mode(const CUtensorMap* tm, const TcWalkParams& p, int BH, cu
     // prefetch tensor maps) while the previous kernel of the stream drains; it waits for that
     // kernel's memory with griddepcontrol.wait before touching any global data.
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(BH * p.n_groups));
+    cfg.gridDim = dim3((unsigned)(BH * p.grid_groups));
     cfg.blockDim = dim3(kTcThreads);
     cfg.dynamicSmemBytes = Smem<D, MODE>::dyn_bytes(with_proj);
     cfg.stream = st;
@@ -905,6 +906,10 @@ cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cuda
     p.H = H; p.N = N; p.group = a.group; p.n_groups = a.n_groups;
     p.init_sum = a.init_sum; p.init_transposed = a.init_transposed;
     p.state_rev = (a.mode == MODE_STATE) ? a.reverse : 0;
+    const bool subset = a.mode == MODE_STATE && a.grid_groups > 0;
+    p.first_group = subset ? a.first_group : 0;
+    p.grid_groups = subset ? a.grid_groups : a.n_groups;
+    if (p.first_group < 0 || p.first_group + p.grid_groups > a.n_groups) return cudaErrorInvalidValue;
     // The four combinations of roles the library uses, as compile-time kernel variants.
     int kind;
     if (a.epilogue == EPI_PLAIN && !a.norm_bv && a.x_norm && !a.reverse) kind = S_FWD;
