@@ -26,7 +26,7 @@ using namespace sm100;
 namespace {
 
 constexpr int kChunk = 128;
-constexpr int kTcThreads = 544;   // 16 row-worker warps + 1 control warp
+constexpr int kTcThreads = 576;   // 16 row-worker warps + control (MMA / load) warp + store warp
 constexpr uint64_t kWaitTimeoutNs = 2000000000ull;  // 2 s: far above any legitimate wait
 
 struct TcWalkParams {
@@ -258,6 +258,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     constexpr int kEpi = STREAM == S_FWD ? EPI_PLAIN : (STREAM == S_DV ? EPI_DV : EPI_PROJ);
     constexpr bool with_proj = (MODE != MODE_STATE) && (kEpi != EPI_PLAIN);
     const bool is_ctrl = warp == kWorkerWarps;
+    const bool is_store = warp == kWorkerWarps + 1;
 
     if (is_ctrl) {
         tmem_alloc(tmem_slot, kTmemCols);
@@ -265,7 +266,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     }
     if (tid == 0) {
         for (int i = 0; i < NST; ++i) {
-            mbar_init(bar_full + 8 * i, 1); mbar_init(bar_a_ready + 8 * i, kGroupThreads);
+            mbar_init(bar_full + 8 * i, L::kSplitB ? 1 : 2); mbar_init(bar_a_ready + 8 * i, kGroupThreads);
             mbar_init(bar_full_b + 8 * i, 1); mbar_init(bar_b_ready + 8 * i, kGroupThreads);
         }
         mbar_init(bar_p_full, 1); mbar_init(bar_s_full, 1); mbar_init(bar_s_full + 8, 1);
@@ -323,7 +324,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     };
 
     const bool init_state = p.init != nullptr;
-    if (init_state && !is_ctrl) {
+    if (init_state && warp < kWorkerWarps) {
         // Initial state of the group: fp32 into TMEM, bf16 copy into shared memory.  With
         // init_sum the exclusive prefix (suffix / total) over the groups' partial states is
         // formed here, in group order, instead of by a separate scan launch.
@@ -372,44 +373,53 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
 
     float dm_acc = 0.f;
 
+    // TMA loads (issued by single threads of the control and the store warp).
+    auto load_tile = [&](uint32_t dst, const CUtensorMap* tm, uint32_t bar, int row) {
+#pragma unroll
+        for (int hh = 0; hh < NH; ++hh) tma_load_3d(dst + hh * 16384, tm, bar, hh * 64, row, bh);
+    };
+    // Loads of chunk c: part 1 = X and A, part 2 = Bv (X alone in the read-out pass).
+    auto issue_loads = [&](int c, bool part1, bool part2) {
+        const int s = c % NST;
+        const uint32_t bar = bar_full + 8 * s;
+        const int row = chunk_row(c);
+        if (L::kSplitB) {
+            if (part1) {
+                mbar_expect_tx(bar, 2 * L::kTile);
+                load_tile(stage_x(s), &tmX, bar, row);
+                load_tile(stage_a(s), &tmA, bar, row);
+            }
+            if (part2) {
+                mbar_expect_tx(bar_full_b + 8 * s, L::kTile);
+                load_tile(stage_b(s), &tmB, bar_full_b + 8 * s, row);
+            }
+        } else {
+            // One barrier for the stage, two arrivals: each part arms its own byte count
+            // before its copies (the parts may come from different threads).
+            constexpr int kPart1Tiles = L::kHasAB ? (L::kHasX ? 2 : 1) : 0;
+            if (part1) {
+                mbar_expect_tx(bar, kPart1Tiles * L::kTile);
+                if (L::kHasAB) {
+                    if (L::kHasX) load_tile(stage_x(s), &tmX, bar, row);
+                    load_tile(stage_a(s), &tmA, bar, row);
+                }
+            }
+            if (part2) {
+                mbar_expect_tx(bar, L::kTile);
+                if (L::kHasAB) load_tile(stage_b(s), &tmB, bar, row);
+                else load_tile(stage_x(s), &tmX, bar, row);
+            }
+        }
+    };
+    // The stage of chunk c is refilled with chunk c + NST in two steps when possible: X and A
+    // as soon as the last MMA that reads the stage has completed (control thread), Bv -- the
+    // output staging slot -- after the chunk's output store has drained (store thread).
+    constexpr bool split_refill = MODE == MODE_CAUSAL && !(with_proj && L::kProjInA);
+
     if (is_ctrl) {
         // ------------------------------------------------------------------ control thread
         if (lane == 0 && n_chunks > 0) {
             bool alive = true;
-            auto load_tile = [&](uint32_t dst, const CUtensorMap* tm, uint32_t bar, int row) {
-#pragma unroll
-                for (int hh = 0; hh < NH; ++hh) tma_load_3d(dst + hh * 16384, tm, bar, hh * 64, row, bh);
-            };
-            // Loads of chunk c: part 1 = X and A (and the byte count of the whole stage),
-            // part 2 = Bv (or everything when the stage was not split).
-            auto issue_loads = [&](int c, bool part1, bool part2) {
-                const int s = c % NST;
-                const uint32_t bar = bar_full + 8 * s;
-                const int row = chunk_row(c);
-                if (L::kSplitB) {
-                    if (part1) {
-                        mbar_expect_tx(bar, 2 * L::kTile);
-                        load_tile(stage_x(s), &tmX, bar, row);
-                        load_tile(stage_a(s), &tmA, bar, row);
-                    }
-                    if (part2) {
-                        mbar_expect_tx(bar_full_b + 8 * s, L::kTile);
-                        load_tile(stage_b(s), &tmB, bar_full_b + 8 * s, row);
-                    }
-                } else {
-                    // One barrier for the stage: its byte count is armed with the first part.
-                    if (part1) mbar_expect_tx(bar, L::kTilesPerStage * L::kTile);
-                    if (L::kHasAB) {
-                        if (part1) {
-                            if (L::kHasX) load_tile(stage_x(s), &tmX, bar, row);
-                            load_tile(stage_a(s), &tmA, bar, row);
-                        }
-                        if (part2) load_tile(stage_b(s), &tmB, bar, row);
-                    } else if (part2) {
-                        load_tile(stage_x(s), &tmX, bar, row);
-                    }
-                }
-            };
             auto wait = [&](uint32_t bar, uint32_t parity) {
                 if (alive && !wait_or_abort(bar, parity, abort_flag)) alive = false;
                 return alive;
@@ -448,10 +458,6 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     tc_commit(bar_o_full + 8 * (c & 1));
                 }
             };
-            // The stage of chunk c is refilled with chunk c + NST in two steps when possible:
-            // X and A as soon as the last MMA that reads the stage has completed, Bv (the
-            // output staging slot) after the chunk's output store has drained.
-            const bool split_refill = MODE == MODE_CAUSAL && !(with_proj && L::kProjInA);
             for (int c = 0; c < NST && c < n_chunks; ++c) issue_loads(c, true, true);
             batch1(0);
             for (int c = 0; c < n_chunks && alive; ++c) {
@@ -502,21 +508,27 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 COTT_STAMP(3);
                 if (c + 1 < n_chunks) { batch1(c + 1); if (!alive) break; }
                 COTT_STAMP(4);
-                // Output rows staged by the workers: store them, then finish the refill.
-                if (!wait(bar_e_done + 8 * (c & 1), (c >> 1) & 1)) break;
-                {
-                    const uint32_t src = base + s * L::kStage + L::kOffOut;
+            }
+        }
+    } else if (is_store) {
+        // ------------------------------------------------------------------ store thread
+        // Output rows staged by the workers go out by TMA; once the store has read the
+        // staging slot the stage's refill is finished.  Kept off the control thread, whose
+        // MMA issue would otherwise stall behind the store's shared-memory read.
+        if (lane == 0 && MODE != MODE_STATE) {
+            bool alive = n_chunks > 0;
+            for (int c = 0; c < n_chunks && alive; ++c) {
+                const int s = c % NST;
+                if (!wait_or_abort(bar_e_done + 8 * (c & 1), (c >> 1) & 1, abort_flag)) { alive = false; break; }
+                const uint32_t src = base + s * L::kStage + L::kOffOut;
 #pragma unroll
-                    for (int hh = 0; hh < NH; ++hh)
-                        tma_store_3d(&tmO, src + hh * 16384, hh * 64, chunk_row(c), bh);
-                    tma_store_commit();
-                }
-                COTT_STAMP(5);
-                if (more) {
+                for (int hh = 0; hh < NH; ++hh)
+                    tma_store_3d(&tmO, src + hh * 16384, hh * 64, chunk_row(c), bh);
+                tma_store_commit();
+                if (c + NST < n_chunks) {
                     tma_store_wait_read0();
                     issue_loads(c + NST, !split_refill, true);
                 }
-                COTT_STAMP(6);
             }
             tma_store_wait_all0();
         }
