@@ -27,7 +27,7 @@ namespace {
 
 constexpr int kChunk = 128;
 constexpr int kTcThreads = 576;   // 16 row-worker warps + control (MMA / load) warp + store warp
-constexpr uint64_t kWaitTimeoutNs = 2000000000ull;  // 2 s: far above any legitimate wait
+constexpr long long kWaitTimeoutCycles = 4000000000ll;  // about 2 s of SM clock: far above any legitimate wait
 
 struct TcWalkParams {
     const float* init;      // [BH, n_groups, d*d] unscaled group states, or NULL
@@ -60,6 +60,22 @@ constexpr int kWorkerWarps = 16;                      // row-worker warps (4 per
 constexpr int kWorkers = kWorkerWarps * 32;
 constexpr int kGroupThreads = kWorkers / 2;           // the workers act as two groups of eight warps
 
+#ifdef COTT_TIMING
+// Debug build only (d = 64): SM-clock timestamps of CTA 0 for chunks 2 and 3 -- 7 slots per
+// chunk for thread 0 (group P), the control thread and thread 256 (group O) -- kept in shared
+// memory and written behind the status word of the workspace header when the kernel ends.
+#define COTT_STAMP(slot)                                                              \
+    do {                                                                              \
+        if (D == 64 && blockIdx.x == 0 && (c == 2 || c == 3) &&                       \
+            (threadIdx.x == 0 || threadIdx.x == kWorkers || threadIdx.x == 256))      \
+            stamps[(threadIdx.x == kWorkers ? 14 : (threadIdx.x == 256 ? 28 : 0)) + (c - 2) * 7 + (slot)] = clock64(); \
+    } while (0)
+constexpr int kStampBytes = 384;
+#else
+#define COTT_STAMP(slot) do {} while (0)
+constexpr int kStampBytes = 0;
+#endif
+
 // Shared-memory plan.  A stage holds the tiles one chunk needs from TMA: (A, Bv) for the
 // state-only pass, (X, A, Bv) for the causal walk, (X) for the read-out.
 template <int D, int MODE> struct Smem {
@@ -84,7 +100,7 @@ template <int D, int MODE> struct Smem {
     // normalised) before every worker has finished the epilogue of chunk c.
     static constexpr int kRx = kStages < 3 ? 3 : kStages;
     static constexpr int kOffRx = kOffBar + 256;          // rx[kRx][128] floats, dm scratch
-    static constexpr int kCtlBytes = 256 + kRx * 512 + 64;
+    static constexpr int kCtlBytes = 256 + kRx * 512 + 64 + (D == 64 ? kStampBytes : 0);
     // Gradient epilogues need a fourth tile (raw q, k or v rows) and a 4 KB exchange area
     // for per-row partial sums.  The causal walk at d = 128 has no room for either: it puts
     // the tile in the A slot and the exchange area in the X slot, both dead by then.  Every
@@ -142,12 +158,12 @@ __device__ __forceinline__ void issue_atb(uint32_t tS, uint32_t a, uint32_t bv, 
 // Bounded wait that also gives up as soon as any thread of the CTA has given up.
 __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = globaltimer_ns();
+    const long long t0 = clock64();   // SM cycle counter: far cheaper to read than the global timer
     for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 15u) == 0) {
             if (*abort_flag) return false;
-            if (globaltimer_ns() - t0 > kWaitTimeoutNs) { *abort_flag = 1; return false; }
+            if (clock64() - t0 > kWaitTimeoutCycles) { *abort_flag = 1; return false; }
         }
     }
 }
@@ -184,18 +200,6 @@ template <int QW> __device__ __forceinline__ void tmem_stq(uint32_t taddr, const
 template <> __device__ __forceinline__ void tmem_stq<32>(uint32_t taddr, const uint32_t (&r)[32]) { tmem_st32(taddr, r); }
 template <> __device__ __forceinline__ void tmem_stq<16>(uint32_t taddr, const uint32_t (&r)[16]) { tmem_st16(taddr, r); }
 
-#ifdef COTT_TIMING
-// Debug build only: phase timestamps of CTA 0 for chunks 2 and 3, written behind the status
-// word of the workspace header.
-#define COTT_STAMP(slot)                                                              \
-    do {                                                                              \
-        if (blockIdx.x == 0 && (threadIdx.x == 0 || threadIdx.x == kWorkers) && (c == 2 || c == 3)) \
-            reinterpret_cast<unsigned long long*>(p.status)[1 + (threadIdx.x == kWorkers ? 14 : 0) + (c - 2) * 7 + (slot)] = \
-                globaltimer_ns();                                                     \
-    } while (0)
-#else
-#define COTT_STAMP(slot) do {} while (0)
-#endif
 
 // Thread roles: warps 0-15 are the row workers, in two groups of eight that work on different
 // chunks at once (score masking + state copy / row norms + output epilogue); warp 16 lane 0
@@ -245,6 +249,9 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     constexpr int NRX = L::kRx;
     float* rx_buf = reinterpret_cast<float*>(gbase + L::kOffRx);                 // [NRX][128]
     float* dm_red = reinterpret_cast<float*>(gbase + L::kOffRx + NRX * 512);     // [16]
+#ifdef COTT_TIMING
+    long long* stamps = reinterpret_cast<long long*>(gbase + L::kOffRx + NRX * 512 + 64);
+#endif
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = p.first_group + blockIdx.x % p.grid_groups, bh = blockIdx.x / p.grid_groups;
@@ -436,6 +443,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     issue_p<D>(tmem + colP, stage_x(s), stage_a(s));
                     tc_commit(bar_p_full);
                 }
+                { const int cn = c; { const int c = cn - 1; COTT_STAMP(5); } }   // stamped with the loop's chunk
                 if (MODE != MODE_STATE) {
                     if (MODE == MODE_CAUSAL && c >= 1 && !wait(bar_sb_ready, (c - 1) & 1)) return;
                     // The output accumulator this chunk writes must have been drained: by chunk
@@ -462,7 +470,6 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             batch1(0);
             for (int c = 0; c < n_chunks && alive; ++c) {
                 const int s = c % NST;
-                const bool more = c + NST < n_chunks;
                 COTT_STAMP(0);
                 auto load_proj = [&]() {
                     const uint32_t proj_u = L::kProjInA ? stage_a(s) : base + L::kOffProj;
@@ -487,6 +494,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     const bool acc = init_state || c > 0;
                     issue_pb<D>(tmem + colO0 + (c % kOBufs) * D, tmem + colPt, stage_b(s), acc);
                     tc_commit(bar_o_full + 8 * (c & 1));
+                    COTT_STAMP(2);
                     issue_atb<D>(tmem + colS, stage_a(s), stage_b(s), acc);
                     tc_commit(sfull_bar(c));
                     if (with_proj && L::kProjInA) {
@@ -495,42 +503,41 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                         load_proj();
                     }
                 }
-                COTT_STAMP(2);
-                if (MODE == MODE_STATE) {
-                    if (more) { if (!wait(sfull_bar(c), sfull_par(c))) break; issue_loads(c + NST, true, true); }
-                    if (c + 1 < n_chunks) batch1(c + 1);
-                    continue;
-                }
-                if (split_refill && more) {
-                    if (!wait(sfull_bar(c), sfull_par(c))) break;   // covers P~ Bv too
-                    issue_loads(c + NST, true, false);
-                }
                 COTT_STAMP(3);
-                if (c + 1 < n_chunks) { batch1(c + 1); if (!alive) break; }
                 COTT_STAMP(4);
+                if (c + 1 < n_chunks) { batch1(c + 1); if (!alive) break; }
+                COTT_STAMP(6);
             }
         }
     } else if (is_store) {
         // ------------------------------------------------------------------ store thread
-        // Output rows staged by the workers go out by TMA; once the store has read the
-        // staging slot the stage's refill is finished.  Kept off the control thread, whose
-        // MMA issue would otherwise stall behind the store's shared-memory read.
-        if (lane == 0 && MODE != MODE_STATE) {
+        // Refills the stages and stores the output rows the workers staged.  Kept off the
+        // control thread: issuing a TMA copy costs it about as much as several MMAs, and the
+        // wait for a store's shared-memory read would stall the MMA issue.
+        if (lane == 0) {
             bool alive = n_chunks > 0;
             for (int c = 0; c < n_chunks && alive; ++c) {
                 const int s = c % NST;
+                const bool more = c + NST < n_chunks;
+                // X and A (everything in the state-only pass) as soon as the chunk's last MMA,
+                // the state update, has completed.
+                if ((MODE == MODE_STATE || split_refill) && more) {
+                    if (!wait_or_abort(sfull_bar(c), sfull_par(c), abort_flag)) { alive = false; break; }
+                    issue_loads(c + NST, true, MODE == MODE_STATE);
+                }
+                if (MODE == MODE_STATE) continue;
                 if (!wait_or_abort(bar_e_done + 8 * (c & 1), (c >> 1) & 1, abort_flag)) { alive = false; break; }
                 const uint32_t src = base + s * L::kStage + L::kOffOut;
 #pragma unroll
                 for (int hh = 0; hh < NH; ++hh)
                     tma_store_3d(&tmO, src + hh * 16384, hh * 64, chunk_row(c), bh);
                 tma_store_commit();
-                if (c + NST < n_chunks) {
+                if (more) {
                     tma_store_wait_read0();
                     issue_loads(c + NST, !split_refill, true);
                 }
             }
-            tma_store_wait_all0();
+            if (MODE != MODE_STATE) tma_store_wait_all0();
         }
     } else {
         // ------------------------------------------------------------------ row workers
@@ -696,10 +703,13 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             for (int c = 0; c < n_chunks && alive; ++c) {
                 const int s = c % NST;
                 uint8_t* st = gbase + s * L::kStage;
+                COTT_STAMP(0);
                 if (c + 1 < n_chunks) { norm_phase(c + 1); if (!alive) break; }
+                COTT_STAMP(1);
                 // ---- output epilogue of chunk c: accumulator -> bf16 rows in the staging slot
                 if (!wait(bar_o_full + 8 * (c & 1), (c >> 1) & 1)) break;
                 tc_fence_after();
+                COTT_STAMP(2);
                 const uint32_t tO = tmem + lane_base + colO0 + (c % kOBufs) * D + hf * HW;
                 const float rx = rx_buf[(c % NRX) * 128 + arow];
                 uint32_t r[HW];
@@ -750,7 +760,9 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 }
                 // Scale, (project,) round to bf16, stage for the TMA store.  The staging slot is
                 // the Bv slot, which the state update (issued behind P~ Bv) still reads: wait for it.
+                COTT_STAMP(3);
                 if (MODE == MODE_CAUSAL && !wait(sfull_bar(c), sfull_par(c))) break;
+                COTT_STAMP(4);
                 uint8_t* so = st + L::kOffOut;
 #pragma unroll
                 for (int i = 0; i < HW; i += 8) {
@@ -775,6 +787,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 }
                 fence_proxy_async();
                 mbar_arrive(bar_e_done + 8 * (c & 1));
+                COTT_STAMP(5);
                 // Bv of the next chunk lands last; normalise it (when it is the one) after this
                 // chunk's epilogue, before the tensor core needs it.
                 if (L::kSplitB && kNormBv && c + 1 < n_chunks) { norm_b(c + 1); if (!alive) break; }
@@ -811,6 +824,9 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         p.dm_partial[(size_t)bh * p.n_groups + g] = (dm_red[8] + dm_red[9]) + (dm_red[10] + dm_red[11]);
     }
     if (tid == 0 && *abort_flag) atomicExch(p.status, 1);
+#ifdef COTT_TIMING
+    if (D == 64 && blockIdx.x == 0 && tid < 42) reinterpret_cast<long long*>(p.status)[1 + tid] = stamps[tid];
+#endif
     if (is_ctrl) tmem_dealloc(tmem, kTmemCols);
 }
 
