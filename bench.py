@@ -33,8 +33,13 @@ METRIC = "causal Cottention fwd+bwd tokens/s"
 L2_FLUSH_BYTES = 256 << 20  # larger than the 126 MB L2
 # DRAM bytes (read + write) per token-head of one causal-walk launch, from the ncu captures
 # summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum divided by the
-# token-heads of the captured launch); keyed by (d, causal).  None: no capture yet.
-KERNEL_DRAM_TRAFFIC = {}
+# token-heads of the captured launch); keyed by (d, causal).  Missing key: no capture yet.
+#   (64, causal):  mean of the four walk launches of a C4 step, 141.8 MB / 262144 token-heads
+#                  (profiles/tc_walk_kernel_c4_d64.md)
+#   (128, causal): forward walk at B=1 H=16 N=16384, 252.5 MB / 262144 token-heads
+#                  (profiles/tc_walk_kernel_c5_n16384_d128.md); traffic grows with the number
+#                  of tokens, so the figure is scaled to the launch that was timed.
+KERNEL_DRAM_TRAFFIC = {(64, True): 541.0, (128, True): 963.0}
 
 
 def load_peaks():
@@ -76,16 +81,54 @@ def algorithmic_bytes(w: dict) -> dict:
 
 
 class ClockSampler:
-    """Samples nvidia-smi SM clocks and throttle reasons while the timed region runs."""
+    """Samples SM clock and clock-event (throttle) reasons while the timed region runs.
+
+    Read-only NVML queries from a background thread every 2 ms (the timed region of a default
+    run lasts tens of milliseconds); falls back to an `nvidia-smi -lms` child process when the
+    NVML binding is missing."""
     FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    PERIOD_S = 0.002
 
-    def __init__(self, gpu_index: int):
+    def __init__(self, gpu_index: int, uuid: str | None = None):
         self.proc = None
+        self.thread = None
         self.gpu_index = gpu_index
+        self.uuid = uuid
+        self.sm, self.bits = [], 0
+        self.max_mhz = None
+        self._stop = False
+
+    def _nvml_loop(self, nv, handle):
+        while not self._stop:
+            try:
+                self.sm.append(float(nv.nvmlDeviceGetClockInfo(handle, nv.NVML_CLOCK_SM)))
+                self.bits |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(handle))
+            except Exception:       # a failed read is a missing sample, not a failed run
+                pass
+            time.sleep(self.PERIOD_S)
 
     def start(self):
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            handle = None
+            if self.uuid:
+                try:
+                    handle = nv.nvmlDeviceGetHandleByUUID(self.uuid)
+                except Exception:
+                    handle = None
+            if handle is None:
+                handle = nv.nvmlDeviceGetHandleByIndex(self.gpu_index)
+            self.max_mhz = float(nv.nvmlDeviceGetMaxClockInfo(handle, nv.NVML_CLOCK_SM))
+            self._nv = nv
+            import threading
+            self.thread = threading.Thread(target=self._nvml_loop, args=(nv, handle), daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.thread = None
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
@@ -94,6 +137,17 @@ class ClockSampler:
             self.proc = None
 
     def stop(self) -> dict:
+        if self.thread is not None:
+            self._stop = True
+            self.thread.join(timeout=2)
+            nv = self._nv
+            names = (("hw_slowdown", nv.nvmlClocksEventReasonHwSlowdown),
+                     ("hw_thermal_slowdown", nv.nvmlClocksEventReasonHwThermalSlowdown),
+                     ("sw_thermal_slowdown", nv.nvmlClocksEventReasonSwThermalSlowdown),
+                     ("sw_power_cap", nv.nvmlClocksEventReasonSwPowerCap))
+            reasons = sorted(n for n, bit in names if self.bits & bit)
+            return {"sm_mhz": statistics.median(self.sm) if self.sm else None, "sm_max_mhz": self.max_mhz,
+                    "samples": len(self.sm), "source": "nvml, 2 ms period", "reasons": reasons}
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         time.sleep(0.15)
@@ -116,7 +170,7 @@ class ClockSampler:
                 if val.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "source": "nvidia-smi, 100 ms period", "reasons": sorted(reasons)}
 
 
 def dist_env():
@@ -277,7 +331,11 @@ def run_ours(args, w):
         return ([e[0].elapsed_time(e[1]) for e in ev], [e[1].elapsed_time(e[2]) for e in ev])
 
     timed_steps(max(args.warmup, 3), record=False)
-    sampler = ClockSampler(local)
+    try:
+        gpu_uuid = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
+    except Exception:
+        gpu_uuid = None
+    sampler = ClockSampler(local, gpu_uuid)
     barrier()
     launches0 = cott.cott.launch_count()
     sampler.start()
@@ -393,7 +451,7 @@ def run_ours(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c4")
