@@ -38,6 +38,9 @@ def gate(x, ref, dtype):
     else:
         e = norm_max_err(x, ref)
         assert e <= TOL_BF16, f"bf16 normalised max error {e:.3e} > {TOL_BF16}"
+    # shown with `pytest -s`: the measured error of every gated tensor
+    print(f"[{os.environ.get('PYTEST_CURRENT_TEST', '').split('::')[-1].split(' ')[0]}] "
+          f"{'fp32 rel' if dtype == torch.float32 else 'bf16 norm'} err {e:.3e}")
     return e
 
 
