@@ -383,7 +383,7 @@ def run_ours(args, w):
             if bwd_call is not None:
                 bwd_call()
         torch.cuda.synchronize()
-        walk_ms = [ms for kind, ms in cott.cott.profile_read() if kind in (1, 2)]
+        walk_ms = [ms for kind, ms in cott.cott.profile_read() if kind in (1, 2, 17)]   # 17: see cott.h
         cott.cott.profile_enable(0)
 
     if world > 1:

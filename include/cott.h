@@ -73,8 +73,10 @@ unsigned long long cott_launch_count(void);
  * with n > 0 starts recording a pair of library-owned CUDA events around each of the next n
  * (at most 256) walk-kernel launches; n <= 0 stops.  cott_profile_read waits for the recorded
  * launches and writes their durations in milliseconds to ms[] and their kind to kinds[]
- * (0 = partial-state pass, 1 = causal walk, 2 = read-out); both are host arrays of `cap`
- * entries.  Returns the number of entries written, or -1 on a CUDA error.  Not thread-safe
+ * (0 = partial-state pass, 1 = causal walk, 2 = read-out; 17 = a causal walk that ran side by
+ * side with a sibling walk of the same size on another stream of the library, in which case
+ * its ms is half of the span the pair occupied, first start to last end); both are host
+ * arrays of `cap` entries.  Returns the number of entries written, or -1 on a CUDA error.  Not thread-safe
  * against concurrent library calls; leave it off outside measurements.
  */
 cott_status cott_profile_enable(int max_launches);

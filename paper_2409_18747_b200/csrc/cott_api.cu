@@ -4,6 +4,7 @@
 #include <stdlib.h>
 #include <string.h>
 #include <atomic>
+#include <mutex>
 #include "cott_internal.h"
 
 namespace cott {
@@ -16,6 +17,9 @@ void note_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memor
 static constexpr int kProfMax = 256;
 static cudaEvent_t g_prof_ev[2 * kProfMax];
 static int g_prof_kind[kProfMax];
+static int g_prof_tag[kProfMax];        // non-zero: launches with the same tag ran side by side
+static thread_local int g_prof_cur_tag = 0;
+static std::atomic<int> g_prof_next_tag{1};
 static bool g_prof_created = false;
 static std::atomic<int> g_prof_n{-1};   // -1: disabled
 static int g_prof_cap = 0;
@@ -26,6 +30,7 @@ int profile_begin_launch(int kind, cudaStream_t st) {
     n = g_prof_n.fetch_add(1);
     if (n >= g_prof_cap) return -1;
     g_prof_kind[n] = kind;
+    g_prof_tag[n] = g_prof_cur_tag;
     cudaEventRecord(g_prof_ev[2 * n], st);
     return n;
 }
@@ -149,7 +154,9 @@ static cott_status run_stream(WalkArgs w, const Plan& p, int BH, int d, cott_dty
 static cott_status run_tc_stream(TcWalkArgs t, const Plan& p, int B, int H, int N, int d,
                                  int causal, const cott_scale_params* sp, int* status,
                                  float* states, float* total_out, cudaStream_t st,
-                                 bool reuse_transposed = false) {
+                                 bool reuse_states = false, bool states_only = false,
+                                 bool states_transposed = true) {
+    const bool reuse_transposed = reuse_states;
     t.status = status; t.m = sp->m; t.seq_len = sp->seq_len; t.seq_len_scalar = sp->seq_len_scalar;
     t.group = p.group; t.n_groups = p.n_groups;
     if (causal && p.n_groups == 1 && !total_out) {
@@ -180,8 +187,9 @@ static cott_status run_tc_stream(TcWalkArgs t, const Plan& p, int B, int H, int 
     // reuse_transposed: `states` already holds, transposed, what this stream needs (raw
     // partials when the scan is fused, scanned states otherwise) from a sibling stream that
     // walks in the same direction.
+    if (states_only) return COTT_OK;
     t.init_sum = fused_scan ? 1 : 0;
-    t.init_transposed = reuse_transposed ? 1 : 0;
+    t.init_transposed = (reuse_states && states_transposed) ? 1 : 0;
     t.mode = causal ? 1 : 2; t.init = states; t.state_out = nullptr;
     COTT_CUDA(launch_tc_walk(t, B, H, N, d, st));
     return COTT_OK;
@@ -208,6 +216,31 @@ static cott_status fwd_impl(const void* q, const void* k, const void* v, void* o
     return run_stream(w, p, B * H, d, dt, causal, states, state_out, st);
 }
 
+// Side streams and events for launches of one call that run next to each other on the GPU
+// (created once per device, on the first call that needs them; never destroyed).
+struct SideStreams {
+    bool ready = false;
+    cudaStream_t s[2];
+    cudaEvent_t fork, join[2];
+};
+static SideStreams* side_streams() {
+    static SideStreams per_device[64];
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    SideStreams& ss = per_device[dev];
+    if (!ss.ready) {
+        for (int i = 0; i < 2; ++i) {
+            if (cudaStreamCreateWithFlags(&ss.s[i], cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+            if (cudaEventCreateWithFlags(&ss.join[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        }
+        if (cudaEventCreateWithFlags(&ss.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        ss.ready = true;
+    }
+    return &ss;
+}
+
 static cott_status bwd_impl(const void* q, const void* k, const void* v, const void* d_o, void* dq,
                             void* dk, void* dv, float* dm, int B, int H, int N, int d, int causal,
                             cott_dtype dt, const cott_scale_params* sp, void* ws, const Plan& p,
@@ -225,20 +258,55 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
         int* status = static_cast<int*>(ws);
         TcWalkArgs t;
         memset(&t, 0, sizeof(t));
+        // When two walks with one CTA per (b, h) fit on the GPU side by side but not two per
+        // (b, h) (74 / 2 < B*H <= 74), the dQ^ and dK^ streams run next to each other, each
+        // over the whole sequence as a single group (no partial-state pass, no scan), with the
+        // dV' stream's partial-state pass filling the SMs that are left; the dV' walk follows on
+        // the whole GPU.  Each side stream then carries one tensor-core kernel per call.
+        SideStreams* ss = nullptr;
+        Plan pp = p;                       // plan of the two side-by-side streams
+        if (causal && p.n_groups >= 2 && 2 * BH <= 148 && 74 / BH == 1 && env_int("COTT_PAIR", 1) != 0) {
+            pp.group = (N + 127) / 128 * 128;
+            pp.n_groups = 1;
+            ss = side_streams();
+        }
         // dQ^: forward walk with (dO, V, K^); c multiplies the accumulator; project with raw q
-        t.x = d_o; t.a = v; t.bv = k; t.proj = q; t.out = dq;
-        t.norm_bv = 1; t.x_norm = 0; t.epilogue = EPI_PROJ; t.reverse = 0;
-        if ((rc = run_tc_stream(t, p, B, H, N, d, causal, sp, status, st0, nullptr, st)) != COTT_OK) return rc;
+        TcWalkArgs tq = t;
+        tq.x = d_o; tq.a = v; tq.bv = k; tq.proj = q; tq.out = dq;
+        tq.norm_bv = 1; tq.x_norm = 0; tq.epilogue = EPI_PROJ; tq.reverse = 0;
         // dK^: backward in time with (V, dO, Q^); project with raw k
-        t.x = v; t.a = d_o; t.bv = q; t.proj = k; t.out = dk;
-        t.norm_bv = 1; t.x_norm = 0; t.epilogue = EPI_PROJ; t.reverse = 1;
-        if ((rc = run_tc_stream(t, p, B, H, N, d, causal, sp, status, st1, nullptr, st)) != COTT_OK) return rc;
+        TcWalkArgs tk = t;
+        tk.x = v; tk.a = d_o; tk.bv = q; tk.proj = k; tk.out = dk;
+        tk.norm_bv = 1; tk.x_norm = 0; tk.epilogue = EPI_PROJ; tk.reverse = 1;
         // dV': backward in time with (K, Q^, dO); rows scale by c / ||k||; <dV', V> for dm
-        t.x = k; t.a = q; t.bv = d_o; t.proj = v; t.out = dv;
-        // Its state sum_t q^_t dO_t^T is the transpose of the dK^ stream's sum_t dO_t q^_t^T,
-        // accumulated in the same direction: reuse those group states instead of a third pass.
-        t.norm_bv = 0; t.x_norm = 1; t.epilogue = EPI_DV; t.reverse = 1; t.dm_partial = dm_partial;
-        if ((rc = run_tc_stream(t, p, B, H, N, d, causal, sp, status, st1, nullptr, st, true)) != COTT_OK) return rc;
+        TcWalkArgs tv = t;
+        tv.x = k; tv.a = q; tv.bv = d_o; tv.proj = v; tv.out = dv;
+        tv.norm_bv = 0; tv.x_norm = 1; tv.epilogue = EPI_DV; tv.reverse = 1; tv.dm_partial = dm_partial;
+        if (ss) {
+            struct TagScope { ~TagScope() { g_prof_cur_tag = 0; } } tag_scope;
+            // Everything that follows a cross-stream event wait is a plain launch.
+            tk.plain_launch = 1; tv.plain_launch = 1;
+            g_prof_cur_tag = g_prof_next_tag.fetch_add(1);
+            COTT_CUDA(cudaEventRecord(ss->fork, st));
+            COTT_CUDA(cudaStreamWaitEvent(ss->s[0], ss->fork, 0));
+            COTT_CUDA(cudaStreamWaitEvent(ss->s[1], ss->fork, 0));
+            if ((rc = run_tc_stream(tq, pp, B, H, N, d, causal, sp, status, st0, nullptr, st)) != COTT_OK) return rc;
+            if ((rc = run_tc_stream(tk, pp, B, H, N, d, causal, sp, status, st1, nullptr, ss->s[0])) != COTT_OK) return rc;
+            g_prof_cur_tag = 0;
+            if ((rc = run_tc_stream(tv, p, B, H, N, d, causal, sp, status, st2, nullptr, ss->s[1], false, true)) != COTT_OK) return rc;
+            COTT_CUDA(cudaEventRecord(ss->join[0], ss->s[0]));
+            COTT_CUDA(cudaEventRecord(ss->join[1], ss->s[1]));
+            COTT_CUDA(cudaStreamWaitEvent(st, ss->join[0], 0));
+            COTT_CUDA(cudaStreamWaitEvent(st, ss->join[1], 0));
+            if ((rc = run_tc_stream(tv, p, B, H, N, d, causal, sp, status, st2, nullptr, st, true, false, false)) != COTT_OK) return rc;
+        } else {
+            if ((rc = run_tc_stream(tq, p, B, H, N, d, causal, sp, status, st0, nullptr, st)) != COTT_OK) return rc;
+            if ((rc = run_tc_stream(tk, p, B, H, N, d, causal, sp, status, st1, nullptr, st)) != COTT_OK) return rc;
+            // The dV' state sum_t q^_t dO_t^T is the transpose of the dK^ stream's
+            // sum_t dO_t q^_t^T, accumulated in the same direction: reuse those group states
+            // instead of a third pass.
+            if ((rc = run_tc_stream(tv, p, B, H, N, d, causal, sp, status, st1, nullptr, st, true)) != COTT_OK) return rc;
+        }
         COTT_CUDA(launch_dm_finalize(dm_partial, dm, sp->m, sp->seq_len, sp->seq_len_scalar, B, H,
                                      p.n_groups, N, st));
         return COTT_OK;
@@ -308,10 +376,24 @@ int cott_profile_read(float* ms, int* kinds, int cap) {
     if (n < 0) return 0;
     if (n > g_prof_cap) n = g_prof_cap;
     if (n > cap) n = cap;
-    for (int i = 0; i < n; ++i) {
+    for (int i = 0; i < n; ++i)
         if (cudaEventSynchronize(g_prof_ev[2 * i + 1]) != cudaSuccess) return -1;
+    for (int i = 0; i < n; ++i) {
         if (cudaEventElapsedTime(&ms[i], g_prof_ev[2 * i], g_prof_ev[2 * i + 1]) != cudaSuccess) return -1;
         kinds[i] = g_prof_kind[i];
+        if (g_prof_tag[i] == 0 || g_prof_kind[i] != 1) continue;
+        // A causal walk that ran side by side with a sibling walk of the same size: report
+        // half of the span the pair occupied (first start to last end).
+        for (int j = 0; j < n; ++j) {
+            if (j == i || g_prof_tag[j] != g_prof_tag[i] || g_prof_kind[j] != 1) continue;
+            float span = ms[i], t;
+            if (cudaEventElapsedTime(&t, g_prof_ev[2 * j], g_prof_ev[2 * j + 1]) == cudaSuccess && t > span) span = t;
+            if (cudaEventElapsedTime(&t, g_prof_ev[2 * i], g_prof_ev[2 * j + 1]) == cudaSuccess && t > span) span = t;
+            if (cudaEventElapsedTime(&t, g_prof_ev[2 * j], g_prof_ev[2 * i + 1]) == cudaSuccess && t > span) span = t;
+            ms[i] = 0.5f * span;
+            kinds[i] = g_prof_kind[i] | 16;
+            break;
+        }
     }
     return n;
 }

@@ -68,6 +68,10 @@ struct TcWalkArgs {
     // (grid_groups == 0 means all of them).  A causal walk never reads the partial state of
     // the group it visits last, so that group is left out unless the total is exported.
     int first_group; int grid_groups;
+    // 1: plain stream-ordered launch.  Default (0) is a programmatic dependent launch, whose
+    // prologue overlaps the tail of the previous kernel of the same stream; launches that
+    // follow a cross-stream event wait are made plain.
+    int plain_launch;
 };
 cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cudaStream_t st);
 

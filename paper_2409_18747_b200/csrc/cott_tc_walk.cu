@@ -42,6 +42,7 @@ struct TcWalkParams {
     const float* m; const float* seq_len; float seq_len_scalar;
     int H; int N; int group; int n_groups;
     int first_group; int grid_groups;   // groups this launch covers: one CTA per (b, h, group)
+    int plain_launch;                   // host side only: launch without programmatic serialization
 };
 
 enum { MODE_STATE = 0, MODE_CAUSAL = 1, MODE_READOUT = 2 };
@@ -156,6 +157,9 @@ __device__ __forceinline__ void issue_atb(uint32_t tS, uint32_t a, uint32_t bv, 
 }
 
 // Bounded wait that also gives up as soon as any thread of the CTA has given up.
+// The thread that gives up first leaves a record of where: bit 31 set, warp index in bits
+// 16-20, byte offset of the barrier inside the barrier block in bits 4-11, parity in bit 0.
+// (The abort flag sits 236 bytes into the barrier block.)
 __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();   // SM cycle counter: far cheaper to read than the global timer
@@ -163,7 +167,12 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, vol
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 15u) == 0) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitTimeoutCycles) { *abort_flag = 1; return false; }
+            if (clock64() - t0 > kWaitTimeoutCycles) {
+                const uint32_t bars = (uint32_t)__cvta_generic_to_shared((const void*)abort_flag) - 236u;
+                const uint32_t where = 0x80000000u | ((threadIdx.x >> 5) << 16) | (((bar - bars) & 0xFFu) << 4) | (parity & 1u);
+                atomicCAS(const_cast<int*>(abort_flag), 0, (int)where);
+                return false;
+            }
         }
     }
 }
@@ -823,7 +832,18 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         // Fixed-order reduction of <dV', V> over the CTA (the first-half warps of group O hold sums).
         p.dm_partial[(size_t)bh * p.n_groups + g] = (dm_red[8] + dm_red[9]) + (dm_red[10] + dm_red[11]);
     }
-    if (tid == 0 && *abort_flag) atomicExch(p.status, 1);
+    if (*abort_flag) {
+        // A wait gave up.  Before the CTA's shared memory and tensor memory go away, give the
+        // copies and MMAs still in flight time to land (they need microseconds; nothing here
+        // waits without a limit), then report: status word 0 = 1, word 1 = where the first
+        // wait gave up, word 2 = the CTA.
+        for (int i = 0; i < 100; ++i) __nanosleep(1000);
+        __syncthreads();
+        if (tid == 0 && atomicCAS(p.status, 0, 1) == 0) {
+            p.status[1] = *abort_flag;
+            p.status[2] = (int)blockIdx.x | (MODE << 24) | (STREAM << 28);
+        }
+    }
 #ifdef COTT_TIMING
     if (D == 64 && blockIdx.x == 0 && tid < 42) reinterpret_cast<long long*>(p.status)[1 + tid] = stamps[tid];
 #endif
@@ -888,7 +908,7 @@ cudaError_t launch_mode(const CUtensorMap* tm, const TcWalkParams& p, int BH, cu
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = p.plain_launch ? 0 : 1;
     cudaError_t le = cudaLaunchKernelEx(&cfg, kern, tm[0], tm[1], tm[2], tm[3], tm[4], p);
     profile_end_launch(prof, st);
     note_launch();
@@ -937,6 +957,7 @@ cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cuda
     const bool subset = a.mode == MODE_STATE && a.grid_groups > 0;
     p.first_group = subset ? a.first_group : 0;
     p.grid_groups = subset ? a.grid_groups : a.n_groups;
+    p.plain_launch = a.plain_launch;
     if (p.first_group < 0 || p.first_group + p.grid_groups > a.n_groups) return cudaErrorInvalidValue;
     // The four combinations of roles the library uses, as compile-time kernel variants.
     int kind;

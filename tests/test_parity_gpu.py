@@ -252,6 +252,21 @@ def test_forward_backward_small(dtype, d, causal, force_group):
     gate_dm(dm, rm, 1e-4 if f32 else 1e-2, dm_condition(rv, c["v"], c["m"], s), DM_COND_F32 if f32 else DM_COND_BF16)
 
 
+def test_backward_d128_several_chunks_per_group(force_group):
+    """d = 128 gradient streams with groups of several chunks and a ragged tail: the two-stage
+    ring, the projection tile in the A slot and the separate Bv barrier all cycle."""
+    force_group(512)
+    B, H, N, d = 1, 2, 1061, 128
+    c = synth.make_qkv(B, H, N, d, torch.bfloat16, 4500, with_do=True)
+    args = [dev(c[x]) for x in ("q", "k", "v")]
+    o = cott.fwd(*args, dev(c["m"]), causal=True)
+    gate(o, oracle.fwd_quadratic(c["q"], c["k"], c["v"], c["m"], None, True), torch.bfloat16)
+    dq, dk, dv, dm = cott.bwd(*args, dev(c["d_o"]), dev(c["m"]), causal=True)
+    rq, rk, rv, rm = oracle.bwd_quadratic(c["q"], c["k"], c["v"], c["d_o"], c["m"], None, True)
+    gate(dq, rq, torch.bfloat16); gate(dk, rk, torch.bfloat16); gate(dv, rv, torch.bfloat16)
+    gate_dm(dm, rm, 1e-2, dm_condition(rv, c["v"], c["m"], None), DM_COND_BF16)
+
+
 def test_single_token_and_single_head():
     c = synth.make_qkv(1, 1, 1, 64, torch.float32, 4100, with_do=True)
     o = cott.fwd(dev(c["q"]), dev(c["k"]), dev(c["v"]), dev(c["m"]), causal=True)
@@ -289,8 +304,9 @@ def test_causality_bitwise(force_group):
     assert torch.equal(o[:, :, :200], o2[:, :, :200])  # later tokens cannot change earlier rows
 
 
-def test_run_to_run_determinism():
-    c = synth.make_config(4, B=1)
+@pytest.mark.parametrize("B", [1, 4])   # B = 4: the dQ and dK streams run side by side
+def test_run_to_run_determinism(B):
+    c = synth.make_config(4, B=B)
     q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
     a = cott.bwd(q, k, v, d_o, m, causal=True)
     b = cott.bwd(q, k, v, d_o, m, causal=True)
