@@ -147,7 +147,7 @@ class ClockSampler:
                      ("sw_power_cap", nv.nvmlClocksEventReasonSwPowerCap))
             reasons = sorted(n for n, bit in names if self.bits & bit)
             return {"sm_mhz": statistics.median(self.sm) if self.sm else None, "sm_max_mhz": self.max_mhz,
-                    "samples": len(self.sm), "source": "nvml, 2 ms period", "reasons": reasons}
+                    "samples": len(self.sm), "source": "nvml, read back to back with 2 ms sleeps", "reasons": reasons}
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         time.sleep(0.15)

@@ -159,6 +159,7 @@ static cott_status run_tc_stream(TcWalkArgs t, const Plan& p, int B, int H, int 
     const bool reuse_transposed = reuse_states;
     t.status = status; t.m = sp->m; t.seq_len = sp->seq_len; t.seq_len_scalar = sp->seq_len_scalar;
     t.group = p.group; t.n_groups = p.n_groups;
+    // t.clear_status (first stream of a call) applies to the first kernel launched here only.
     if (causal && p.n_groups == 1 && !total_out) {
         t.mode = 1; t.init = nullptr; t.state_out = nullptr;
         COTT_CUDA(launch_tc_walk(t, B, H, N, d, st));
@@ -172,6 +173,7 @@ static cott_status run_tc_stream(TcWalkArgs t, const Plan& p, int B, int H, int 
         TcWalkArgs a = t;
         a.mode = 0; a.x = nullptr; a.proj = nullptr; a.out = nullptr; a.init = nullptr;
         a.state_out = states; a.dm_partial = nullptr; a.epilogue = EPI_PLAIN;
+        t.clear_status = 0;              // the state pass, launched first, does it
         a.reverse = t.reverse ? 0 : 1;   // chunk order opposite to the walk's: L2 reuse of its tiles
         if (causal && !total_out) {
             // Nobody reads the partial state of the group the walk visits last.
@@ -199,13 +201,15 @@ static cott_status fwd_impl(const void* q, const void* k, const void* v, void* o
                             int B, int H, int N, int d, int causal, cott_dtype dt,
                             const cott_scale_params* sp, void* ws, const Plan& p,
                             cudaStream_t st) {
-    COTT_CUDA(cudaMemsetAsync(ws, 0, kWsHeaderBytes, st));
+    // The tensor-core path clears the status words in its first kernel.
+    if (p.path != 1) COTT_CUDA(cudaMemsetAsync(ws, 0, kWsHeaderBytes, st));
     float* states = reinterpret_cast<float*>(static_cast<char*>(ws) + kWsHeaderBytes);
     if (p.path == 1) {
         TcWalkArgs t;
         memset(&t, 0, sizeof(t));
         t.x = q; t.a = k; t.bv = v; t.out = o;
         t.norm_bv = 0; t.x_norm = 1; t.epilogue = EPI_PLAIN; t.reverse = 0;
+        t.clear_status = 1;
         return run_tc_stream(t, p, B, H, N, d, causal, sp, static_cast<int*>(ws), states,
                              state_out, st);
     }
@@ -245,7 +249,8 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
                             void* dk, void* dv, float* dm, int B, int H, int N, int d, int causal,
                             cott_dtype dt, const cott_scale_params* sp, void* ws, const Plan& p,
                             cudaStream_t st) {
-    COTT_CUDA(cudaMemsetAsync(ws, 0, kWsHeaderBytes, st));
+    // The tensor-core path clears the status words in its first kernel.
+    if (p.path != 1) COTT_CUDA(cudaMemsetAsync(ws, 0, kWsHeaderBytes, st));
     char* base = static_cast<char*>(ws) + kWsHeaderBytes;
     const size_t sb = states_bytes(p, B, H, d);
     float* st0 = reinterpret_cast<float*>(base);
@@ -274,6 +279,7 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
         TcWalkArgs tq = t;
         tq.x = d_o; tq.a = v; tq.bv = k; tq.proj = q; tq.out = dq;
         tq.norm_bv = 1; tq.x_norm = 0; tq.epilogue = EPI_PROJ; tq.reverse = 0;
+        tq.clear_status = 1;             // the dQ^ stream is launched first
         // dK^: backward in time with (V, dO, Q^); project with raw k
         TcWalkArgs tk = t;
         tk.x = v; tk.a = d_o; tk.bv = q; tk.proj = k; tk.out = dk;

@@ -72,6 +72,10 @@ struct TcWalkArgs {
     // prologue overlaps the tail of the previous kernel of the same stream; launches that
     // follow a cross-stream event wait are made plain.
     int plain_launch;
+    // 1: this is the first kernel of a library call; its first CTA clears the status words of
+    // the workspace header (a wait that gives up writes them two seconds later at the earliest),
+    // which saves a separate memset in front of every call.
+    int clear_status;
 };
 cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cudaStream_t st);
 

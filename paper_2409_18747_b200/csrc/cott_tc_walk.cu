@@ -43,6 +43,7 @@ struct TcWalkParams {
     int H; int N; int group; int n_groups;
     int first_group; int grid_groups;   // groups this launch covers: one CTA per (b, h, group)
     int plain_launch;                   // host side only: launch without programmatic serialization
+    int clear_status;                   // first kernel of a call: CTA 0 zeroes the status words
 };
 
 enum { MODE_STATE = 0, MODE_CAUSAL = 1, MODE_READOUT = 2 };
@@ -303,10 +304,64 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot_g;
+    auto stage_x = [&](int s) { return base + s * L::kStage + L::kOffX; };
+    auto stage_a = [&](int s) { return base + s * L::kStage + L::kOffA; };
+    auto stage_b = [&](int s) { return base + s * L::kStage + L::kOffB; };
+    // Chunk visited at step c.  The state-only pass may take either order (its result does not
+    // depend on it): it takes the opposite of the walk that follows, so that the tiles it
+    // read last -- still in L2 -- are the ones the walk needs first.
+    const bool backward = (MODE == MODE_STATE) ? (p.state_rev != 0) : kReverse;
+    auto chunk_row = [&](int c) { return tok0 + (backward ? (n_chunks - 1 - c) : c) * kChunk; };
+
+    // TMA loads (issued by single threads of the control and the store warp).
+    auto load_tile = [&](uint32_t dst, const CUtensorMap* tm, uint32_t bar, int row) {
+#pragma unroll
+        for (int hh = 0; hh < NH; ++hh) tma_load_3d(dst + hh * 16384, tm, bar, hh * 64, row, bh);
+    };
+    // Loads of chunk c: part 1 = X and A, part 2 = Bv (X alone in the read-out pass).
+    auto issue_loads = [&](int c, bool part1, bool part2) {
+        const int s = c % NST;
+        const uint32_t bar = bar_full + 8 * s;
+        const int row = chunk_row(c);
+        if (L::kSplitB) {
+            if (part1) {
+                mbar_expect_tx(bar, 2 * L::kTile);
+                load_tile(stage_x(s), &tmX, bar, row);
+                load_tile(stage_a(s), &tmA, bar, row);
+            }
+            if (part2) {
+                mbar_expect_tx(bar_full_b + 8 * s, L::kTile);
+                load_tile(stage_b(s), &tmB, bar_full_b + 8 * s, row);
+            }
+        } else {
+            // One barrier for the stage, two arrivals: each part arms its own byte count
+            // before its copies (the parts may come from different threads).
+            constexpr int kPart1Tiles = L::kHasAB ? (L::kHasX ? 2 : 1) : 0;
+            if (part1) {
+                mbar_expect_tx(bar, kPart1Tiles * L::kTile);
+                if (L::kHasAB) {
+                    if (L::kHasX) load_tile(stage_x(s), &tmX, bar, row);
+                    load_tile(stage_a(s), &tmA, bar, row);
+                }
+            }
+            if (part2) {
+                mbar_expect_tx(bar, L::kTile);
+                if (L::kHasAB) load_tile(stage_b(s), &tmB, bar, row);
+                else load_tile(stage_x(s), &tmX, bar, row);
+            }
+        }
+    };
+    // Every kernel but the first of a library call follows a kernel of the same call, which
+    // writes none of the tensors loaded here: its first tiles are requested before the wait
+    // for that kernel, so their HBM latency overlaps its tail.
+    const bool early_loads = p.clear_status == 0 && n_chunks > 0;
+    if (early_loads && is_ctrl && lane == 0)
+        for (int c = 0; c < NST && c < n_chunks; ++c) issue_loads(c, true, true);
     // Everything above touched only this CTA's own resources.  From here on global memory
     // written by the previous kernel of the stream is read (and its inputs overwritten).
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (p.clear_status && blockIdx.x == 0 && tid == 0) { p.status[0] = 0; p.status[1] = 0; p.status[2] = 0; }
 
     const float s_b = p.seq_len ? p.seq_len[b] : (p.seq_len_scalar > 0.f ? p.seq_len_scalar : (float)p.N);
     const float cfac = stab_factor(p.m[h], s_b);
@@ -319,15 +374,6 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     const bool owns_srow = (D == 128) || (lane < 16);
     const int srow = (D == 128) ? arow : q * 16 + (lane & 15);
     const uint32_t sb = base + L::kOffSb;
-
-    auto stage_x = [&](int s) { return base + s * L::kStage + L::kOffX; };
-    auto stage_a = [&](int s) { return base + s * L::kStage + L::kOffA; };
-    auto stage_b = [&](int s) { return base + s * L::kStage + L::kOffB; };
-    // Chunk visited at step c.  The state-only pass may take either order (its result does not
-    // depend on it): it takes the opposite of the walk that follows, so that the tiles it
-    // read last -- still in L2 -- are the ones the walk needs first.
-    const bool backward = (MODE == MODE_STATE) ? (p.state_rev != 0) : kReverse;
-    auto chunk_row = [&](int c) { return tok0 + (backward ? (n_chunks - 1 - c) : c) * kChunk; };
 
     // bf16 copy of QW state columns of this thread's row into the MN-major state tile.
     auto write_sb = [&](const uint32_t (&r)[QW], int c0) {
@@ -389,44 +435,6 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
 
     float dm_acc = 0.f;
 
-    // TMA loads (issued by single threads of the control and the store warp).
-    auto load_tile = [&](uint32_t dst, const CUtensorMap* tm, uint32_t bar, int row) {
-#pragma unroll
-        for (int hh = 0; hh < NH; ++hh) tma_load_3d(dst + hh * 16384, tm, bar, hh * 64, row, bh);
-    };
-    // Loads of chunk c: part 1 = X and A, part 2 = Bv (X alone in the read-out pass).
-    auto issue_loads = [&](int c, bool part1, bool part2) {
-        const int s = c % NST;
-        const uint32_t bar = bar_full + 8 * s;
-        const int row = chunk_row(c);
-        if (L::kSplitB) {
-            if (part1) {
-                mbar_expect_tx(bar, 2 * L::kTile);
-                load_tile(stage_x(s), &tmX, bar, row);
-                load_tile(stage_a(s), &tmA, bar, row);
-            }
-            if (part2) {
-                mbar_expect_tx(bar_full_b + 8 * s, L::kTile);
-                load_tile(stage_b(s), &tmB, bar_full_b + 8 * s, row);
-            }
-        } else {
-            // One barrier for the stage, two arrivals: each part arms its own byte count
-            // before its copies (the parts may come from different threads).
-            constexpr int kPart1Tiles = L::kHasAB ? (L::kHasX ? 2 : 1) : 0;
-            if (part1) {
-                mbar_expect_tx(bar, kPart1Tiles * L::kTile);
-                if (L::kHasAB) {
-                    if (L::kHasX) load_tile(stage_x(s), &tmX, bar, row);
-                    load_tile(stage_a(s), &tmA, bar, row);
-                }
-            }
-            if (part2) {
-                mbar_expect_tx(bar, L::kTile);
-                if (L::kHasAB) load_tile(stage_b(s), &tmB, bar, row);
-                else load_tile(stage_x(s), &tmX, bar, row);
-            }
-        }
-    };
     // The stage of chunk c is refilled with chunk c + NST in two steps when possible: X and A
     // as soon as the last MMA that reads the stage has completed (control thread), Bv -- the
     // output staging slot -- after the chunk's output store has drained (store thread).
@@ -475,7 +483,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     tc_commit(bar_o_full + 8 * (c & 1));
                 }
             };
-            for (int c = 0; c < NST && c < n_chunks; ++c) issue_loads(c, true, true);
+            if (!early_loads) for (int c = 0; c < NST && c < n_chunks; ++c) issue_loads(c, true, true);
             batch1(0);
             for (int c = 0; c < n_chunks && alive; ++c) {
                 const int s = c % NST;
@@ -958,6 +966,7 @@ cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cuda
     p.first_group = subset ? a.first_group : 0;
     p.grid_groups = subset ? a.grid_groups : a.n_groups;
     p.plain_launch = a.plain_launch;
+    p.clear_status = a.clear_status;
     if (p.first_group < 0 || p.first_group + p.grid_groups > a.n_groups) return cudaErrorInvalidValue;
     // The four combinations of roles the library uses, as compile-time kernel variants.
     int kind;
