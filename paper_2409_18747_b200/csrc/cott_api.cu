@@ -63,13 +63,13 @@ struct Plan {
     int group;     // tokens per sequence group
     int chunk;     // tokens per chunk inside a group
     int n_groups;
+    int split;   // partial-state pass: parts per group when the walk sums the prefix itself
 };
 
 // Sequence groups give sequence-level parallelism when B*H alone cannot fill the GPU:
 // halve the group until there are enough CTAs, but never below a floor that keeps the
 // per-group state traffic (d*d fp32) small against the group's own q,k,v,o bytes.
 static bool make_plan(int op, cott_dtype dt, int B, int H, int N, int d, int causal, Plan* p) {
-    (void)causal;
     if (B < 1 || H < 1 || N < 1) return false;
     if (d != 32 && d != 64 && d != 128) return false;
     if (dt != COTT_F32 && dt != COTT_BF16) return false;
@@ -97,11 +97,23 @@ static bool make_plan(int op, cott_dtype dt, int B, int H, int N, int d, int cau
     if (group >= N) group = (N + p->chunk - 1) / p->chunk * p->chunk;
     p->group = group;
     p->n_groups = (N + group - 1) / group;
+    // With the prefix summed inside the walk (few groups, see run_tc_stream), the state pass
+    // may use a finer partition than the walk -- each group cut into `split` equal parts of
+    // whole chunks -- when that still fits in one wave of CTAs: its CTAs get shorter, the walk
+    // sums `split` times as many states.
+    p->split = 1;
+    if (p->path == 1 && causal && p->n_groups >= 2 && p->n_groups <= 8 &&
+        (long)p->n_groups * d * 8 <= group && N % group == 0) {
+        const long ctas = BH * (p->n_groups - 1);
+        const int chunks = group / p->chunk;
+        for (int s2 = 4; s2 >= 2; s2 >>= 1)
+            if (ctas * s2 <= 148 && chunks % s2 == 0 && chunks / s2 >= 4) { p->split = s2; break; }
+    }
     return true;
 }
 
 static size_t states_bytes(const Plan& p, int B, int H, int d) {
-    return align_up((size_t)B * H * p.n_groups * d * d * sizeof(float), 256);
+    return align_up((size_t)B * H * p.n_groups * p.split * d * d * sizeof(float), 256);
 }
 
 static size_t workspace_bytes_impl(int op, const Plan& p, int B, int H, int d) {
@@ -169,16 +181,18 @@ static cott_status run_tc_stream(TcWalkArgs t, const Plan& p, int B, int H, int 
     // and the scan launch is dropped -- as long as those extra d x d reads (n_groups / 2 of
     // them on average) stay small against the group's own q, k, v, o bytes.
     const bool fused_scan = !total_out && p.n_groups <= 8 && (long)p.n_groups * d * 8 <= p.group;
+    const int split = (fused_scan && causal) ? p.split : 1;
     if (!reuse_transposed) {
         TcWalkArgs a = t;
+        a.group = p.group / split; a.n_groups = p.n_groups * split;
         a.mode = 0; a.x = nullptr; a.proj = nullptr; a.out = nullptr; a.init = nullptr;
         a.state_out = states; a.dm_partial = nullptr; a.epilogue = EPI_PLAIN;
         t.clear_status = 0;              // the state pass, launched first, does it
         a.reverse = t.reverse ? 0 : 1;   // chunk order opposite to the walk's: L2 reuse of its tiles
         if (causal && !total_out) {
             // Nobody reads the partial state of the group the walk visits last.
-            a.grid_groups = p.n_groups - 1;
-            a.first_group = t.reverse ? 1 : 0;
+            a.grid_groups = (p.n_groups - 1) * split;
+            a.first_group = t.reverse ? split : 0;
         }
         COTT_CUDA(launch_tc_walk(a, B, H, N, d, st));
         const int mode = !causal ? SCAN_TOTAL : (t.reverse ? SCAN_SUFFIX : SCAN_PREFIX);
@@ -191,6 +205,7 @@ static cott_status run_tc_stream(TcWalkArgs t, const Plan& p, int B, int H, int 
     // walks in the same direction.
     if (states_only) return COTT_OK;
     t.init_sum = fused_scan ? 1 : 0;
+    t.init_split = split;
     t.init_transposed = (reuse_states && states_transposed) ? 1 : 0;
     t.mode = causal ? 1 : 2; t.init = states; t.state_out = nullptr;
     COTT_CUDA(launch_tc_walk(t, B, H, N, d, st));
@@ -272,7 +287,7 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
         Plan pp = p;                       // plan of the two side-by-side streams
         if (causal && p.n_groups >= 2 && 2 * BH <= 148 && 74 / BH == 1 && env_int("COTT_PAIR", 1) != 0) {
             pp.group = (N + 127) / 128 * 128;
-            pp.n_groups = 1;
+            pp.n_groups = 1; pp.split = 1;
             ss = side_streams();
         }
         // dQ^: forward walk with (dO, V, K^); c multiplies the accumulator; project with raw q

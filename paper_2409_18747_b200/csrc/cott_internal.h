@@ -63,6 +63,9 @@ struct TcWalkArgs {
     int group; int n_groups;
     int norm_bv; int x_norm; int epilogue; int reverse;
     int init_sum;   // 1: `init` holds raw partial states; the walk forms its own prefix / suffix / total
+    // With init_sum the partial states may come from a finer partition than the walk's groups:
+    // init_split consecutive entries of `init` per group (0 or 1: one entry per group).
+    int init_split;
     int init_transposed;  // 1: `init` holds the transposes of the states this walk starts from
     // State-only pass: groups first_group .. first_group + grid_groups - 1 are computed
     // (grid_groups == 0 means all of them).  A causal walk never reads the partial state of

@@ -33,6 +33,7 @@ struct TcWalkParams {
     const float* init;      // [BH, n_groups, d*d] unscaled group states, or NULL
     int init_transposed;    // 1: init holds the transposes of the states this walk needs
     int state_rev;          // state-only pass: visit the chunks of a group last to first
+    int init_split;         // init_sum: entries of `init` per group (a finer state-pass partition)
     int init_sum;           // 0: init holds this group's start state; 1: it holds raw partial
                             // states, to be summed here over the groups before (after, when
                             // time runs backward; all, for the read-out) this one
@@ -392,7 +393,8 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         // formed here, in group order, instead of by a separate scan launch.
         // Element (srow, cq*QW + i) of group gg's state; a transposed source (the state of a
         // sibling gradient stream, which is this stream's state transposed) is read by columns.
-        const float* src = p.init + (size_t)bh * p.n_groups * D * D;
+        const int n_init = p.n_groups * p.init_split;     // entries of `init` per (b, h)
+        const float* src = p.init + (size_t)bh * n_init * D * D;
         auto load4 = [&](int gg, int i) -> float4 {
             const float* sg = src + (size_t)gg * D * D;
             if (!p.init_transposed) return *reinterpret_cast<const float4*>(sg + (size_t)srow * D + cq * QW + i);
@@ -411,8 +413,8 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             float acc[QW];
 #pragma unroll
             for (int i = 0; i < QW; ++i) acc[i] = 0.f;
-            const int g_lo = (MODE == MODE_READOUT) ? 0 : (kReverse ? g + 1 : 0);
-            const int g_hi = (MODE == MODE_READOUT) ? p.n_groups : (kReverse ? p.n_groups : g);
+            const int g_lo = (MODE == MODE_READOUT) ? 0 : (kReverse ? (g + 1) * p.init_split : 0);
+            const int g_hi = (MODE == MODE_READOUT) ? n_init : (kReverse ? n_init : g * p.init_split);
             if (owns_srow) {
                 for (int gg = g_lo; gg < g_hi; ++gg) {
 #pragma unroll
@@ -961,6 +963,7 @@ cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cuda
     p.m = a.m; p.seq_len = a.seq_len; p.seq_len_scalar = a.seq_len_scalar;
     p.H = H; p.N = N; p.group = a.group; p.n_groups = a.n_groups;
     p.init_sum = a.init_sum; p.init_transposed = a.init_transposed;
+    p.init_split = (a.init_sum && a.init_split > 1) ? a.init_split : 1;
     p.state_rev = (a.mode == MODE_STATE) ? a.reverse : 0;
     const bool subset = a.mode == MODE_STATE && a.grid_groups > 0;
     p.first_group = subset ? a.first_group : 0;
