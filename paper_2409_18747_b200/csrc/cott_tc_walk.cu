@@ -352,6 +352,14 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             }
         }
     };
+    // Raw q, k or v rows of chunk c for the gradient epilogues: into the A slot of the chunk's
+    // stage once the state update has read it (d = 128 causal walk, control thread), else into
+    // a buffer of its own once the previous chunk's epilogue is done (store thread).
+    auto load_proj = [&](int c) {
+        const uint32_t proj_u = L::kProjInA ? stage_a(c % NST) : base + L::kOffProj;
+        mbar_expect_tx(bar_proj, L::kTile);
+        load_tile(proj_u, &tmP, bar_proj, chunk_row(c));
+    };
     // Every kernel but the first of a library call follows a kernel of the same call, which
     // writes none of the tensors loaded here: its first tiles are requested before the wait
     // for that kernel, so their HBM latency overlaps its tail.
@@ -490,16 +498,6 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             for (int c = 0; c < n_chunks && alive; ++c) {
                 const int s = c % NST;
                 COTT_STAMP(0);
-                auto load_proj = [&]() {
-                    const uint32_t proj_u = L::kProjInA ? stage_a(s) : base + L::kOffProj;
-                    mbar_expect_tx(bar_proj, L::kTile);
-                    load_tile(proj_u, &tmP, bar_proj, chunk_row(c));
-                };
-                if (with_proj && !L::kProjInA) {
-                    // Dedicated buffer: free once the previous chunk's epilogue has finished.
-                    if (c >= 1 && !wait(bar_e_done + 8 * ((c - 1) & 1), ((c - 1) >> 1) & 1)) break;
-                    load_proj();
-                }
                 if (MODE == MODE_CAUSAL) {
                     if (!wait(bar_pt_ready, c & 1)) break;
                     // Bv is needed from here on: landed, and normalised if it is the operand
@@ -519,7 +517,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     if (with_proj && L::kProjInA) {
                         // The A slot is free once the state update has read it.
                         if (!wait(sfull_bar(c), sfull_par(c))) break;
-                        load_proj();
+                        load_proj(c);
                     }
                 }
                 COTT_STAMP(3);
@@ -535,6 +533,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         // wait for a store's shared-memory read would stall the MMA issue.
         if (lane == 0) {
             bool alive = n_chunks > 0;
+            if (alive && with_proj && !L::kProjInA) load_proj(0);
             for (int c = 0; c < n_chunks && alive; ++c) {
                 const int s = c % NST;
                 const bool more = c + NST < n_chunks;
@@ -546,6 +545,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 }
                 if (MODE == MODE_STATE) continue;
                 if (!wait_or_abort(bar_e_done + 8 * (c & 1), (c >> 1) & 1, abort_flag)) { alive = false; break; }
+                if (with_proj && !L::kProjInA && c + 1 < n_chunks) load_proj(c + 1);   // its buffer is free now
                 const uint32_t src = base + s * L::kStage + L::kOffOut;
 #pragma unroll
                 for (int hh = 0; hh < NH; ++hh)
