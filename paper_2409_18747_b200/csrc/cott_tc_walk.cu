@@ -26,7 +26,7 @@ using namespace sm100;
 namespace {
 
 constexpr int kChunk = 128;
-constexpr int kTcThreads = 576;   // 16 row-worker warps + control (MMA / load) warp + store warp
+constexpr int kTcThreads = 608;   // 16 row-worker warps + control warp + store warp + state-update warp
 constexpr long long kWaitTimeoutCycles = 4000000000ll;  // about 2 s of SM clock: far above any legitimate wait
 
 struct TcWalkParams {
@@ -93,7 +93,11 @@ template <int D, int MODE> struct Smem {
     static constexpr int kOffA = kHasX ? kTile : 0;
     static constexpr int kOffB = kOffA + kTile;
     static constexpr int kOffOut = kHasAB ? kOffB : kOffX;             // output staging slot
-    static constexpr int kSb = (MODE == MODE_STATE) ? 0 : D * D * 2;   // bf16 copy of the state
+    // bf16 copy of the state for the X State product.  The d = 64 causal walk keeps two copies
+    // (chunk parity), so that the copy of chunk c can be written while X State of chunk c
+    // still reads the previous one; at d = 128 there is room for one.
+    static constexpr int kSbBufs = (MODE == MODE_CAUSAL && D == 64) ? 2 : 1;
+    static constexpr int kSb = (MODE == MODE_STATE) ? 0 : D * D * 2 * kSbBufs;
     static constexpr int kOffSb = kStages * kStage;
     static constexpr int kOffPt = kOffSb + kSb;
     static constexpr int kPt = 0;   // the masked scores live in tensor memory
@@ -241,7 +245,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     const uint32_t bar_p_full = bars + 64;     //       scores done (commit)
     const uint32_t bar_s_full = bars + 72;     // [2]   state update done (commit)
     const uint32_t bar_pt_ready = bars + 88;   //       masked scores in tensor memory (all workers)
-    const uint32_t bar_sb_ready = bars + 96;   //       bf16 state copy written (all workers)
+    const uint32_t bar_sb_ready = bars + 96;   // [2]   bf16 state copy written (all workers); the second one sits at bars + 240
     const uint32_t bar_o_full = bars + 104;    // [2]   output accumulator complete (commit)
     const uint32_t bar_o_free = bars + 120;    // [2]   output accumulator drained (all workers)
     const uint32_t bar_proj = bars + 136;      //       epilogue tile landed
@@ -257,6 +261,11 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     // score barriers are unused there); the other modes use two.
     auto sfull_bar = [&](int c) { return MODE == MODE_STATE ? bars + 64 + 8 * (c & 3) : bar_s_full + 8 * (c & 1); };
     auto sfull_par = [&](int c) { return (uint32_t)(MODE == MODE_STATE ? (c >> 2) & 1 : (c >> 1) & 1); };
+    auto sb_bar = [&](int c) { return (c & 1) ? bars + 240 : bar_sb_ready; };
+    auto sb_par = [&](int c) { return (uint32_t)((c >> 1) & 1); };
+    // Byte offset of the state copy X State of chunk c reads (written after chunk c - 1, or by
+    // the prologue for c = 0).
+    auto sb_off = [&](int c) { return (uint32_t)(L::kSbBufs == 2 ? ((c + 1) & 1) * (D * D * 2) : 0); };
     constexpr int NRX = L::kRx;
     float* rx_buf = reinterpret_cast<float*>(gbase + L::kOffRx);                 // [NRX][128]
     float* dm_red = reinterpret_cast<float*>(gbase + L::kOffRx + NRX * 512);     // [16]
@@ -277,6 +286,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     constexpr bool with_proj = (MODE != MODE_STATE) && (kEpi != EPI_PLAIN);
     const bool is_ctrl = warp == kWorkerWarps;
     const bool is_store = warp == kWorkerWarps + 1;
+    const bool is_upd = warp == kWorkerWarps + 2;
 
     if (is_ctrl) {
         tmem_alloc(tmem_slot, kTmemCols);
@@ -289,6 +299,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         }
         mbar_init(bar_p_full, 1); mbar_init(bar_s_full, 1); mbar_init(bar_s_full + 8, 1);
         mbar_init(bar_pt_ready, MODE == MODE_STATE ? 1 : kGroupThreads); mbar_init(bar_sb_ready, kGroupThreads);
+        mbar_init(bars + 240, kGroupThreads);
         mbar_init(bar_o_full, 1); mbar_init(bar_o_full + 8, 1);
         mbar_init(bar_o_free, kGroupThreads); mbar_init(bar_o_free + 8, kGroupThreads);
         mbar_init(bar_proj, 1); mbar_init(bar_e_done, kGroupThreads); mbar_init(bar_e_done + 8, kGroupThreads);
@@ -390,7 +401,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         for (int i = 0; i < QW; i += 8) {
             const int col = c0 + i;
             const uint32_t off = (col >> 6) * (D * 128u) + swz(srow, (col & 63) >> 3);
-            *reinterpret_cast<uint4*>(gbase + L::kOffSb + off) = pack8(&r[i]);
+            *reinterpret_cast<uint4*>(gbase + L::kOffSb + sb_off(0) + off) = pack8(&r[i]);
         }
     };
 
@@ -472,7 +483,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 }
                 { const int cn = c; { const int c = cn - 1; COTT_STAMP(5); } }   // stamped with the loop's chunk
                 if (MODE != MODE_STATE) {
-                    if (MODE == MODE_CAUSAL && c >= 1 && !wait(bar_sb_ready, (c - 1) & 1)) return;
+                    if (MODE == MODE_CAUSAL && c >= 1 && !wait(sb_bar(c - 1), sb_par(c - 1))) return;
                     // The output accumulator this chunk writes must have been drained: by chunk
                     // c - 2 with two buffers, by chunk c - 1 with one.
                     if (kOBufs == 2) { if (c >= 2 && !wait(bar_o_free + 8 * (c & 1), ((c >> 1) & 1) ^ 1)) return; }
@@ -481,10 +492,8 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 tc_fence_after();
                 const uint32_t tO = tmem + colO0 + (c % kOBufs) * D;
                 if (MODE == MODE_CAUSAL) {
-                    // The state update of this chunk is issued later, behind P~ Bv, so that
-                    // the workers mask the scores without the tensor core hammering shared
-                    // memory and TMEM at the same time.
-                    if (acc) issue_xs<D>(tO, stage_x(s), sb);
+                    // (The state update of the chunk is issued by the state-update thread.)
+                    if (acc) issue_xs<D>(tO, stage_x(s), sb + sb_off(c));
                 } else if (MODE == MODE_STATE) {
                     issue_atb<D>(tmem + colS, stage_a(s), stage_b(s), acc);
                     tc_commit(sfull_bar(c));
@@ -512,8 +521,6 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     issue_pb<D>(tmem + colO0 + (c % kOBufs) * D, tmem + colPt, stage_b(s), acc);
                     tc_commit(bar_o_full + 8 * (c & 1));
                     COTT_STAMP(2);
-                    issue_atb<D>(tmem + colS, stage_a(s), stage_b(s), acc);
-                    tc_commit(sfull_bar(c));
                     if (with_proj && L::kProjInA) {
                         // The A slot is free once the state update has read it.
                         if (!wait(sfull_bar(c), sfull_par(c))) break;
@@ -524,6 +531,26 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 COTT_STAMP(4);
                 if (c + 1 < n_chunks) { batch1(c + 1); if (!alive) break; }
                 COTT_STAMP(6);
+            }
+        }
+    } else if (is_upd) {
+        // ------------------------------------------------------------------ state-update thread
+        // Causal walk: State += A^T Bv of chunk c depends on the chunk's tiles and on the
+        // workers having copied the previous state, not on the scores; issued from a thread of
+        // its own it neither waits behind the masked scores nor holds up their MMAs.
+        if (lane == 0 && MODE == MODE_CAUSAL) {
+            for (int c = 0; c < n_chunks; ++c) {
+                const int s = c % NST;
+                if (!wait_or_abort(bar_a_ready + 8 * s, (c / NST) & 1, abort_flag)) break;
+                if (L::kSplitB) {
+                    if (!wait_or_abort(bar_full_b + 8 * s, (c / NST) & 1, abort_flag)) break;
+                    if (kNormBv && !wait_or_abort(bar_b_ready + 8 * s, (c / NST) & 1, abort_flag)) break;
+                }
+                // the workers have read the fp32 state of the previous chunk
+                if (c >= 1 && !wait_or_abort(sb_bar(c - 1), sb_par(c - 1), abort_flag)) break;
+                tc_fence_after();
+                issue_atb<D>(tmem + colS, stage_a(s), stage_b(s), init_state || c > 0);
+                tc_commit(sfull_bar(c));
             }
         }
     } else if (is_store) {
@@ -541,6 +568,9 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 // the state update, has completed.
                 if ((MODE == MODE_STATE || split_refill) && more) {
                     if (!wait_or_abort(sfull_bar(c), sfull_par(c), abort_flag)) { alive = false; break; }
+                    // (causal walk: the other MMAs of the chunk come from another thread)
+                    if (MODE == MODE_CAUSAL &&
+                        !wait_or_abort(bar_o_full + 8 * (c & 1), (c >> 1) & 1, abort_flag)) { alive = false; break; }
                     issue_loads(c + NST, true, MODE == MODE_STATE);
                 }
                 if (MODE == MODE_STATE) continue;
@@ -638,12 +668,12 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             mbar_arrive(bar_b_ready + 8 * s);
         };
         // bf16 copy of 32 state columns of this thread's row into the MN-major state tile.
-        auto write_sb32 = [&](const uint32_t (&r)[32], int c0) {
+        auto write_sb32 = [&](const uint32_t (&r)[32], int c0, uint32_t buf) {
 #pragma unroll
             for (int i = 0; i < 32; i += 8) {
                 const int col = c0 + i;
                 const uint32_t off = (col >> 6) * (D * 128u) + swz(srow, (col & 63) >> 3);
-                *reinterpret_cast<uint4*>(gbase + L::kOffSb + off) = pack8(&r[i]);
+                *reinterpret_cast<uint4*>(gbase + L::kOffSb + buf + off) = pack8(&r[i]);
             }
         };
 
@@ -701,17 +731,19 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 // bf16 copy of the updated state for the next chunk's X State product.
                 if (c + 1 < n_chunks) {
                     if (!wait(sfull_bar(c), sfull_par(c))) break;
+                    // A single copy is still being read by this chunk's X State product.
+                    if (L::kSbBufs == 1 && !wait(bar_o_full + 8 * (c & 1), (c >> 1) & 1)) break;
                     tc_fence_after();
 #pragma unroll 1
                     for (int pc = 0; pc < NPIECE; ++pc) {
                         uint32_t r[32];
                         tmem_ld32(tmem + lane_base + colS + hf * HW + pc * 32, r);
                         tmem_wait_ld();
-                        if (owns_srow) write_sb32(r, hf * HW + pc * 32);
+                        if (owns_srow) write_sb32(r, hf * HW + pc * 32, sb_off(c + 1));
                     }
                     fence_proxy_async();
                     tc_fence_before();
-                    mbar_arrive(bar_sb_ready);
+                    mbar_arrive(sb_bar(c));
                 }
                 COTT_STAMP(3);
             }
