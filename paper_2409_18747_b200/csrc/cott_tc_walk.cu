@@ -106,8 +106,9 @@ template <int D, int MODE> struct Smem {
     // epilogue; three buffers are needed because X and A of chunk c+2 can land (and be
     // normalised) before every worker has finished the epilogue of chunk c.
     static constexpr int kRx = kStages < 3 ? 3 : kStages;
-    static constexpr int kOffRx = kOffBar + 256;          // rx[kRx][128] floats, dm scratch
-    static constexpr int kCtlBytes = 256 + kRx * 512 + 64 + (D == 64 ? kStampBytes : 0);
+    static constexpr int kBarBytes = 384;                 // mbarriers, TMEM slot, abort flag
+    static constexpr int kOffRx = kOffBar + kBarBytes;    // rx[kRx][128] floats, dm scratch
+    static constexpr int kCtlBytes = kBarBytes + kRx * 512 + 64 + (D == 64 ? kStampBytes : 0);
     // Gradient epilogues need a fourth tile (raw q, k or v rows) and a 4 KB exchange area
     // for per-row partial sums.  The causal walk at d = 128 has no room for either: it puts
     // the tile in the A slot and the exchange area in the X slot, both dead by then.  Every
@@ -164,7 +165,7 @@ __device__ __forceinline__ void issue_atb(uint32_t tS, uint32_t a, uint32_t bv, 
 
 // Bounded wait that also gives up as soon as any thread of the CTA has given up.
 // The thread that gives up first leaves a record of where: bit 31 set, warp index in bits
-// 16-20, byte offset of the barrier inside the barrier block in bits 4-11, parity in bit 0.
+// 16-20, byte offset of the barrier inside the barrier block in bits 4-13, parity in bit 0.
 // (The abort flag sits 236 bytes into the barrier block.)
 __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -175,7 +176,7 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, vol
             if (*abort_flag) return false;
             if (clock64() - t0 > kWaitTimeoutCycles) {
                 const uint32_t bars = (uint32_t)__cvta_generic_to_shared((const void*)abort_flag) - 236u;
-                const uint32_t where = 0x80000000u | ((threadIdx.x >> 5) << 16) | (((bar - bars) & 0xFFu) << 4) | (parity & 1u);
+                const uint32_t where = 0x80000000u | ((threadIdx.x >> 5) << 16) | (((bar - bars) & 0x3FFu) << 4) | (parity & 1u);
                 atomicCAS(const_cast<int*>(abort_flag), 0, (int)where);
                 return false;
             }
@@ -243,24 +244,29 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     const uint32_t bar_full = bars;            // [NST] (<= 4) TMA landed: X and A (causal walk), all tiles otherwise
     const uint32_t bar_a_ready = bars + 32;    // [NST] X scale known, A normalised (all workers)
     const uint32_t bar_p_full = bars + 64;     //       scores done (commit)
-    const uint32_t bar_s_full = bars + 72;     // [2]   state update done (commit)
+    const uint32_t bar_s_full = bars + 256;    // [4]   state update done (commit)
     const uint32_t bar_pt_ready = bars + 88;   //       masked scores in tensor memory (all workers)
     const uint32_t bar_sb_ready = bars + 96;   // [2]   bf16 state copy written (all workers); the second one sits at bars + 240
-    const uint32_t bar_o_full = bars + 104;    // [2]   output accumulator complete (commit)
+    const uint32_t bar_o_full = bars + 288;    // [4]   output accumulator complete (commit)
     const uint32_t bar_o_free = bars + 120;    // [2]   output accumulator drained (all workers)
     const uint32_t bar_proj = bars + 136;      //       epilogue tile landed
-    const uint32_t bar_e_done = bars + 144;    // [2]   output rows of the chunk staged (all workers)
+    const uint32_t bar_e_done = bars + 320;    // [4]   output rows of the chunk staged (all workers)
     const uint32_t bar_xch = bars + 160;       //       per-row partial sums exchanged (all workers)
     const uint32_t bar_full_b = bars + 168;    // [NST] causal walk: Bv landed (it is loaded last and needed last)
     const uint32_t bar_b_ready = bars + 200;   // [NST] causal walk: Bv normalised, when it is the one (all workers)
     const uint32_t tmem_slot = bars + 232;
     volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(gbase + L::kOffBar + 232);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + L::kOffBar + 236);
-    // State-update barrier of chunk c.  The state-only pass, whose two worker groups may drift
-    // apart by more than one chunk, cycles through four barriers (bars + 64 .. + 88; the
-    // score barriers are unused there); the other modes use two.
-    auto sfull_bar = [&](int c) { return MODE == MODE_STATE ? bars + 64 + 8 * (c & 3) : bar_s_full + 8 * (c & 1); };
-    auto sfull_par = [&](int c) { return (uint32_t)(MODE == MODE_STATE ? (c >> 2) & 1 : (c >> 1) & 1); };
+    // Barriers with waiters that only the data flow holds back (the store thread, the
+    // state-update thread, a worker group behind the other) are rings of four indexed by
+    // chunk: the stage ring (at most four deep) keeps every role within three chunks of the
+    // others, so a phase parity always names one chunk.
+    auto sfull_bar = [&](int c) { return bar_s_full + 8 * (c & 3); };
+    auto sfull_par = [&](int c) { return (uint32_t)((c >> 2) & 1); };
+    auto ofull_bar = [&](int c) { return bar_o_full + 8 * (c & 3); };
+    auto ofull_par = [&](int c) { return (uint32_t)((c >> 2) & 1); };
+    auto edone_bar = [&](int c) { return bar_e_done + 8 * (c & 3); };
+    auto edone_par = [&](int c) { return (uint32_t)((c >> 2) & 1); };
     auto sb_bar = [&](int c) { return (c & 1) ? bars + 240 : bar_sb_ready; };
     auto sb_par = [&](int c) { return (uint32_t)((c >> 1) & 1); };
     // Byte offset of the state copy X State of chunk c reads (written after chunk c - 1, or by
@@ -297,12 +303,12 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             mbar_init(bar_full + 8 * i, L::kSplitB ? 1 : 2); mbar_init(bar_a_ready + 8 * i, kGroupThreads);
             mbar_init(bar_full_b + 8 * i, 1); mbar_init(bar_b_ready + 8 * i, kGroupThreads);
         }
-        mbar_init(bar_p_full, 1); mbar_init(bar_s_full, 1); mbar_init(bar_s_full + 8, 1);
-        mbar_init(bar_pt_ready, MODE == MODE_STATE ? 1 : kGroupThreads); mbar_init(bar_sb_ready, kGroupThreads);
+        mbar_init(bar_p_full, 1);
+        for (int i = 0; i < 4; ++i) { mbar_init(bar_s_full + 8 * i, 1); mbar_init(bar_o_full + 8 * i, 1); mbar_init(bar_e_done + 8 * i, kGroupThreads); }
+        mbar_init(bar_pt_ready, kGroupThreads); mbar_init(bar_sb_ready, kGroupThreads);
         mbar_init(bars + 240, kGroupThreads);
-        mbar_init(bar_o_full, 1); mbar_init(bar_o_full + 8, 1);
         mbar_init(bar_o_free, kGroupThreads); mbar_init(bar_o_free + 8, kGroupThreads);
-        mbar_init(bar_proj, 1); mbar_init(bar_e_done, kGroupThreads); mbar_init(bar_e_done + 8, kGroupThreads);
+        mbar_init(bar_proj, 1);
         mbar_init(bar_xch, kGroupThreads);
         *abort_flag = 0;
         mbar_fence_init();
@@ -499,7 +505,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     tc_commit(sfull_bar(c));
                 } else {
                     issue_xs<D>(tO, stage_x(s), sb);
-                    tc_commit(bar_o_full + 8 * (c & 1));
+                    tc_commit(ofull_bar(c));
                 }
             };
             if (!early_loads) for (int c = 0; c < NST && c < n_chunks; ++c) issue_loads(c, true, true);
@@ -519,7 +525,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     tc_fence_after();
                     const bool acc = init_state || c > 0;
                     issue_pb<D>(tmem + colO0 + (c % kOBufs) * D, tmem + colPt, stage_b(s), acc);
-                    tc_commit(bar_o_full + 8 * (c & 1));
+                    tc_commit(ofull_bar(c));
                     COTT_STAMP(2);
                     if (with_proj && L::kProjInA) {
                         // The A slot is free once the state update has read it.
@@ -548,6 +554,9 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 }
                 // the workers have read the fp32 state of the previous chunk
                 if (c >= 1 && !wait_or_abort(sb_bar(c - 1), sb_par(c - 1), abort_flag)) break;
+                // Nothing else ties this thread to group O: stay within two chunks of its
+                // epilogue, so that the ring of state-update barriers cannot lap it.
+                if (c >= 2 && !wait_or_abort(edone_bar(c - 2), edone_par(c - 2), abort_flag)) break;
                 tc_fence_after();
                 issue_atb<D>(tmem + colS, stage_a(s), stage_b(s), init_state || c > 0);
                 tc_commit(sfull_bar(c));
@@ -570,11 +579,11 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     if (!wait_or_abort(sfull_bar(c), sfull_par(c), abort_flag)) { alive = false; break; }
                     // (causal walk: the other MMAs of the chunk come from another thread)
                     if (MODE == MODE_CAUSAL &&
-                        !wait_or_abort(bar_o_full + 8 * (c & 1), (c >> 1) & 1, abort_flag)) { alive = false; break; }
+                        !wait_or_abort(ofull_bar(c), ofull_par(c), abort_flag)) { alive = false; break; }
                     issue_loads(c + NST, true, MODE == MODE_STATE);
                 }
                 if (MODE == MODE_STATE) continue;
-                if (!wait_or_abort(bar_e_done + 8 * (c & 1), (c >> 1) & 1, abort_flag)) { alive = false; break; }
+                if (!wait_or_abort(edone_bar(c), edone_par(c), abort_flag)) { alive = false; break; }
                 if (with_proj && !L::kProjInA && c + 1 < n_chunks) load_proj(c + 1);   // its buffer is free now
                 const uint32_t src = base + s * L::kStage + L::kOffOut;
 #pragma unroll
@@ -732,7 +741,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 if (c + 1 < n_chunks) {
                     if (!wait(sfull_bar(c), sfull_par(c))) break;
                     // A single copy is still being read by this chunk's X State product.
-                    if (L::kSbBufs == 1 && !wait(bar_o_full + 8 * (c & 1), (c >> 1) & 1)) break;
+                    if (L::kSbBufs == 1 && !wait(ofull_bar(c), ofull_par(c))) break;
                     tc_fence_after();
 #pragma unroll 1
                     for (int pc = 0; pc < NPIECE; ++pc) {
@@ -758,7 +767,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 if (c + 1 < n_chunks) { norm_phase(c + 1); if (!alive) break; }
                 COTT_STAMP(1);
                 // ---- output epilogue of chunk c: accumulator -> bf16 rows in the staging slot
-                if (!wait(bar_o_full + 8 * (c & 1), (c >> 1) & 1)) break;
+                if (!wait(ofull_bar(c), ofull_par(c))) break;
                 tc_fence_after();
                 COTT_STAMP(2);
                 const uint32_t tO = tmem + lane_base + colO0 + (c % kOBufs) * D + hf * HW;
@@ -837,7 +846,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     *reinterpret_cast<uint4*>(so + (col >> 6) * 16384 + swz(arow, (col & 63) >> 3)) = w;
                 }
                 fence_proxy_async();
-                mbar_arrive(bar_e_done + 8 * (c & 1));
+                mbar_arrive(edone_bar(c));
                 COTT_STAMP(5);
                 // Bv of the next chunk lands last; normalise it (when it is the one) after this
                 // chunk's epilogue, before the tensor core needs it.
