@@ -300,34 +300,38 @@ __global__ void dm_finalize_kernel(const float* dm_partial, float* dm, const flo
     dm[h] = total;
 }
 
-// Recurrent decode step (Eq. 8): one CTA per (b,h); the fp32 state streams through once with
-// 128-bit loads and stores, update and read-out fused.  Every thread first issues all loads
-// of its state elements (the whole state of the pair is then in flight), and only then
-// normalises q and k, so the row norms hide behind the memory latency.
-template <int D, typename T>
+// Recurrent decode step (Eq. 8): SPLIT CTAs per (b,h), each owning D / SPLIT value columns of
+// the fp32 state, which streams through once with 128-bit loads and stores, update and
+// read-out fused.  Every thread first issues all loads of its state elements (the CTA's whole
+// share is then in flight), and only then normalises q and k, so the row norms hide behind
+// the memory latency.  The column split keeps the per-thread share small (more CTAs resident,
+// a shorter last wave); every CTA normalises q and k for itself and owns its columns of o.
+template <int D, int SPLIT, typename T>
 __global__ void __launch_bounds__(kThreads) decode_kernel(const T* q, const T* k, const T* v,
                                                           float* state, T* o, int H,
                                                           const float* m, const float* seq_len,
                                                           float seq_len_scalar) {
-    constexpr int V4 = D / 4;             // float4 per state row
+    constexpr int DC = D / SPLIT;         // value columns of this CTA
+    constexpr int V4 = DC / 4;            // float4 per state row share
     constexpr int RG = kThreads / V4;     // rows covered per sweep
     constexpr int NIT = D / RG;
-    __shared__ float qh[D], kh[D], vp[D];
-    __shared__ __align__(16) float red[RG][D];
+    __shared__ float qh[D], kh[D], vp[DC];
+    __shared__ __align__(16) float red[RG][DC];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int bh = blockIdx.x, b = bh / H, h = bh % H;
+    const int bh = blockIdx.x / SPLIT, col0 = (blockIdx.x % SPLIT) * DC;
+    const int b = bh / H, h = bh % H;
     const int c4 = tid % V4, r0 = tid / V4;
-    float4* S = reinterpret_cast<float4*>(state + (size_t)bh * D * D);
+    float4* S = reinterpret_cast<float4*>(state + (size_t)bh * D * D + col0);   // row stride D / 4
     float4 sv[NIT];
 #pragma unroll
-    for (int i = 0; i < NIT; ++i) sv[i] = S[(size_t)(r0 + i * RG) * V4 + c4];
+    for (int i = 0; i < NIT; ++i) sv[i] = S[(size_t)(r0 + i * RG) * (D / 4) + c4];
 
     const float s_b = seq_len ? seq_len[b] : seq_len_scalar;
     const float c = stab_factor(m[h], s_b);
     if (tid < D) {
         qh[tid] = to_f32<T>(q[(size_t)bh * D + tid]);
         kh[tid] = to_f32<T>(k[(size_t)bh * D + tid]);
-        vp[tid] = to_f32<T>(v[(size_t)bh * D + tid]) * c;
+        if (tid < DC) vp[tid] = to_f32<T>(v[(size_t)bh * D + col0 + tid]) * c;
     }
     __syncthreads();
     if (warp < 2) {
@@ -346,16 +350,16 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(const T* q, const T* k
         const int a = r0 + i * RG;
         const float ka = kh[a], qa = qh[a];
         sv[i].x += ka * vv.x; sv[i].y += ka * vv.y; sv[i].z += ka * vv.z; sv[i].w += ka * vv.w;
-        S[(size_t)a * V4 + c4] = sv[i];
+        S[(size_t)a * (D / 4) + c4] = sv[i];
         acc.x += qa * sv[i].x; acc.y += qa * sv[i].y; acc.z += qa * sv[i].z; acc.w += qa * sv[i].w;
     }
     *reinterpret_cast<float4*>(&red[r0][c4 * 4]) = acc;
     __syncthreads();
-    if (tid < D) {
+    if (tid < DC) {
         float t = 0.f;
 #pragma unroll
         for (int r = 0; r < RG; ++r) t += red[r][tid];
-        o[(size_t)bh * D + tid] = from_f32<T>(t);
+        o[(size_t)bh * D + col0 + tid] = from_f32<T>(t);
     }
 }
 
@@ -376,13 +380,13 @@ template <typename T>
 cudaError_t launch_decode_t(const void* q, const void* k, const void* v, float* state, void* o,
                             int B, int H, int d, const float* m, const float* seq_len,
                             float seq_len_scalar, cudaStream_t st) {
-    dim3 grid((unsigned)(B * H));
+    const unsigned BH = (unsigned)(B * H);
     const T *qq = (const T*)q, *kk = (const T*)k, *vv = (const T*)v;
     T* oo = (T*)o;
     switch (d) {
-        case 32: decode_kernel<32, T><<<grid, kThreads, 0, st>>>(qq, kk, vv, state, oo, H, m, seq_len, seq_len_scalar); break;
-        case 64: decode_kernel<64, T><<<grid, kThreads, 0, st>>>(qq, kk, vv, state, oo, H, m, seq_len, seq_len_scalar); break;
-        case 128: decode_kernel<128, T><<<grid, kThreads, 0, st>>>(qq, kk, vv, state, oo, H, m, seq_len, seq_len_scalar); break;
+        case 32: decode_kernel<32, 1, T><<<BH, kThreads, 0, st>>>(qq, kk, vv, state, oo, H, m, seq_len, seq_len_scalar); break;
+        case 64: decode_kernel<64, 1, T><<<BH, kThreads, 0, st>>>(qq, kk, vv, state, oo, H, m, seq_len, seq_len_scalar); break;
+        case 128: decode_kernel<128, 2, T><<<2 * BH, kThreads, 0, st>>>(qq, kk, vv, state, oo, H, m, seq_len, seq_len_scalar); break;
         default: return cudaErrorInvalidValue;
     }
     note_launch();
