@@ -69,11 +69,14 @@ constexpr int kGroupThreads = kWorkers / 2;           // the workers act as two 
 // memory and written behind the status word of the workspace header when the kernel ends.
 #define COTT_STAMP(slot)                                                              \
     do {                                                                              \
-        if (D == 64 && blockIdx.x == 0 && (c == 2 || c == 3) &&                       \
+        if (D == 64 && STREAM == COTT_STAMP_STREAM && blockIdx.x == 0 && (c == 2 || c == 3) && \
             (threadIdx.x == 0 || threadIdx.x == kWorkers || threadIdx.x == 256))      \
             stamps[(threadIdx.x == kWorkers ? 14 : (threadIdx.x == 256 ? 28 : 0)) + (c - 2) * 7 + (slot)] = clock64(); \
     } while (0)
 constexpr int kStampBytes = 384;
+#ifndef COTT_STAMP_STREAM
+#define COTT_STAMP_STREAM 0   // which output stream's walk is stamped (0 forward, 1 dQ, 2 dK, 3 dV)
+#endif
 #else
 #define COTT_STAMP(slot) do {} while (0)
 constexpr int kStampBytes = 0;
@@ -896,7 +899,8 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         }
     }
 #ifdef COTT_TIMING
-    if (D == 64 && blockIdx.x == 0 && tid < 42) reinterpret_cast<long long*>(p.status)[1 + tid] = stamps[tid];
+    if (D == 64 && STREAM == COTT_STAMP_STREAM && MODE == MODE_CAUSAL && blockIdx.x == 0 && tid < 42)
+        reinterpret_cast<long long*>(p.status)[1 + tid] = stamps[tid];
 #endif
     if (is_ctrl) tmem_dealloc(tmem, kTmemCols);
 }
