@@ -124,6 +124,11 @@ cott_status cott_fwd(const void* q, const void* k, const void* v, void* o, float
  *   dm       out: fp32 [H], gradient w.r.t. m summed over batch and positions; overwritten
  * On a row with norm <= 1e-12 the gradient is that of the clamped formula, d x^ / 1e-12.
  * There is no gradient for the scaling base s.
+ * No output tensor may overlap an input tensor.  The call is ordered on `stream` as a whole:
+ * work issued to `stream` before it has finished when it starts, and work issued after it
+ * sees all its results; inside, the library may run independent gradient streams on two
+ * streams of its own (created once per device on first use), forked from and joined back
+ * into `stream` with events.
  */
 cott_status cott_bwd(const void* q, const void* k, const void* v, const void* d_o, void* dq,
                      void* dk, void* dv, float* dm, int B, int H, int N, int d, int causal,
@@ -183,7 +188,10 @@ cott_status cott_fwd_noalloc(const void* q, const void* k, const void* v, void* 
 /*
  * Synchronises `stream`, then reads the status word the last call using `workspace` left
  * there: COTT_OK, or COTT_ERR_TIMEOUT if a bounded device-side wait gave up, or COTT_ERR_CUDA
- * if the stream reports an error.
+ * if the stream reports an error.  After a timeout the next two 32-bit words of the workspace
+ * say where the first wait gave up: word 1 = bit 31 set, warp index in bits 16-20, byte offset
+ * of the barrier in the kernel's barrier block in bits 4-13, phase parity in bit 0; word 2 =
+ * CTA index in bits 0-23, kernel mode in bits 24-27, output stream in bits 28-31.
  */
 cott_status cott_last_async_status(const void* workspace, void* stream);
 

@@ -221,9 +221,11 @@ template <> __device__ __forceinline__ void tmem_stq<16>(uint32_t taddr, const u
 
 
 // Thread roles: warps 0-15 are the row workers, in two groups of eight that work on different
-// chunks at once (score masking + state copy / row norms + output epilogue); warp 16 lane 0
-// is the control thread (TMA loads / stores and all tcgen05.mma).  The roles meet only
-// through mbarriers, every wait bounded.
+// chunks at once (score masking + state copy / row norms + output epilogue).  Lane 0 of
+// warp 16 is the control thread (scores, P~ Bv and X State MMAs), of warp 17 the store thread
+// (output stores, stage refills, epilogue-tile loads), of warp 18 the state-update thread
+// (State += A^T Bv in the causal walk).  The roles meet only through mbarriers, every wait
+// bounded.
 template <int D, int MODE, int STREAM>
 __global__ void __launch_bounds__(kTcThreads, 1)
 tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmA,
