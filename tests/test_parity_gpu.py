@@ -354,3 +354,50 @@ def test_fwd_bwd_host_matches_device_calls():
     dq, dk, dv, dm2 = cott.bwd(q, k, v, d_o, m, causal=True)
     assert torch.equal(outs["o"], o.cpu()) and torch.equal(outs["dq"], dq.cpu())
     assert torch.equal(outs["dk"], dk.cpu()) and torch.equal(outs["dv"], dv.cpu()) and torch.equal(dm, dm2.cpu())
+
+
+# ------------------------------------------------------------------ library services
+def test_profile_and_status_words():
+    """Per-launch timing of the walk kernels, the launch counter and the status read-back."""
+    c = synth.make_config(4, B=1)
+    q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
+    B, H, N, d = q.shape
+    ws = torch.zeros(cott.workspace_bytes(cott.cott.OP_BWD, cott.cott.BF16, B, H, N, d, True),
+                     dtype=torch.uint8, device="cuda")
+    ws[:16] = 0xFF        # stale status words from "an earlier user" of the memory
+    n0 = cott.cott.launch_count()
+    cott.cott.profile_enable(64)
+    cott.fwd(q, k, v, m, causal=True, workspace=ws)
+    cott.bwd(q, k, v, d_o, m, causal=True, workspace=ws)
+    rec = cott.cott.profile_read()
+    cott.cott.profile_enable(0)
+    kinds = [kd for kd, _ in rec]
+    assert kinds.count(1) + kinds.count(17) == 4          # forward walk + three gradient walks
+    assert 0 in kinds                                      # at least one partial-state pass
+    assert all(0.0 < ms < 50.0 for _, ms in rec)
+    assert cott.cott.launch_count() - n0 >= len(rec) + 1   # + dm
+    assert cott.cott.last_async_status(ws) == 0            # the first kernel of a call clears the words
+    assert int(ws[:12].view(torch.int32).abs().sum()) == 0
+    assert cott.cott.profile_read() == []                  # disabled
+
+
+def test_side_by_side_backward_matches_one_after_the_other(monkeypatch):
+    """B*H = 64: the dQ and dK streams run side by side, each over the whole sequence.  Same
+    gradients (up to the rounding of a different grouping) as the three streams in sequence,
+    also with a ragged last chunk."""
+    for N in (4096, 1000):
+        c = synth.make_qkv(4, 16, N, 64, torch.bfloat16, 4600 + N, with_do=True)
+        q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
+        monkeypatch.setenv("COTT_PAIR", "1")
+        a = cott.bwd(q, k, v, d_o, m, causal=True)
+        monkeypatch.setenv("COTT_PAIR", "0")
+        b = cott.bwd(q, k, v, d_o, m, causal=True)
+        for x, y in zip(a[:3], b[:3]):
+            assert norm_max_err(x, y.double().cpu().numpy()) <= TOL_BF16
+        torch.testing.assert_close(a[3], b[3], rtol=2e-2, atol=2e-2 * float(b[3].abs().max()))
+    # and against the definition on a slice of the ragged case
+    sub = slice(0, 1)
+    rq, rk, rv, _ = oracle.bwd_quadratic(c["q"][sub], c["k"][sub], c["v"][sub], c["d_o"][sub], c["m"], None, True)
+    monkeypatch.setenv("COTT_PAIR", "1")
+    dq, dk, dv, _ = cott.bwd(q, k, v, d_o, m, causal=True)
+    gate(dq[sub], rq, torch.bfloat16); gate(dk[sub], rk, torch.bfloat16); gate(dv[sub], rv, torch.bfloat16)
