@@ -393,6 +393,10 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (p.clear_status && blockIdx.x == 0 && tid == 0) { p.status[0] = 0; p.status[1] = 0; p.status[2] = 0; }
+    // The first kernel of a call may follow a kernel that produced its inputs: its first tiles
+    // are requested here, right behind the wait.
+    if (!early_loads && is_ctrl && lane == 0)
+        for (int c = 0; c < NST && c < n_chunks; ++c) issue_loads(c, true, true);
 
     const float s_b = p.seq_len ? p.seq_len[b] : (p.seq_len_scalar > 0.f ? p.seq_len_scalar : (float)p.N);
     const float cfac = stab_factor(p.m[h], s_b);
@@ -513,7 +517,6 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     tc_commit(ofull_bar(c));
                 }
             };
-            if (!early_loads) for (int c = 0; c < NST && c < n_chunks; ++c) issue_loads(c, true, true);
             batch1(0);
             for (int c = 0; c < n_chunks && alive; ++c) {
                 const int s = c % NST;
