@@ -4,7 +4,6 @@
 #include <stdlib.h>
 #include <string.h>
 #include <atomic>
-#include <mutex>
 #include "cott_internal.h"
 
 namespace cott {
@@ -235,19 +234,18 @@ static cott_status fwd_impl(const void* q, const void* k, const void* v, void* o
     return run_stream(w, p, B * H, d, dt, causal, states, state_out, st);
 }
 
-// Side streams and events for launches of one call that run next to each other on the GPU
-// (created once per device, on the first call that needs them; never destroyed).
+// Side streams and events for launches of one call that run next to each other on the GPU:
+// one set per host thread and device (two calls from different threads must not share events),
+// created on the first call that needs them and kept until the process ends.
 struct SideStreams {
     bool ready = false;
     cudaStream_t s[2];
     cudaEvent_t fork, join[2];
 };
 static SideStreams* side_streams() {
-    static SideStreams per_device[64];
-    static std::mutex mu;
+    static thread_local SideStreams per_device[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-    std::lock_guard<std::mutex> lock(mu);
     SideStreams& ss = per_device[dev];
     if (!ss.ready) {
         for (int i = 0; i < 2; ++i) {
@@ -303,6 +301,7 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
         TcWalkArgs tv = t;
         tv.x = k; tv.a = q; tv.bv = d_o; tv.proj = v; tv.out = dv;
         tv.norm_bv = 0; tv.x_norm = 1; tv.epilogue = EPI_DV; tv.reverse = 1; tv.dm_partial = dm_partial;
+        tv.dm_out = dm;                  // finalised by the last CTA of the dV' walk
         if (ss) {
             struct TagScope { ~TagScope() { g_prof_cur_tag = 0; } } tag_scope;
             // Everything that follows a cross-stream event wait is a plain launch.
@@ -328,8 +327,6 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
             // instead of a third pass.
             if ((rc = run_tc_stream(tv, p, B, H, N, d, causal, sp, status, st1, nullptr, st, true)) != COTT_OK) return rc;
         }
-        COTT_CUDA(launch_dm_finalize(dm_partial, dm, sp->m, sp->seq_len, sp->seq_len_scalar, B, H,
-                                     p.n_groups, N, st));
         return COTT_OK;
     }
     {   // dQ^_t = S_t dO_t : the forward walk with (dO, V', K^) in the roles of (Q, K, V)

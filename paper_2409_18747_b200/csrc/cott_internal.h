@@ -79,6 +79,9 @@ struct TcWalkArgs {
     // the workspace header (a wait that gives up writes them two seconds later at the earliest),
     // which saves a separate memset in front of every call.
     int clear_status;
+    // EPI_DV: when set, the CTA that finishes last turns the [BH, n_groups] partial sums of
+    // <dV', V> into dm[H] (fixed summation order), so no separate launch is needed.
+    float* dm_out;
 };
 cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cudaStream_t st);
 

@@ -39,6 +39,7 @@ struct TcWalkParams {
                             // time runs backward; all, for the read-out) this one
     float* state_out;       // MODE_STATE: [BH, n_groups, d*d] partial states (unscaled)
     float* dm_partial;      // EPI_DV: [BH, n_groups]
+    float* dm_out;          // EPI_DV: dm[H], written by the CTA that finishes last (or NULL)
     int* status;            // workspace status word
     const float* m; const float* seq_len; float seq_len_scalar;
     int H; int N; int group; int n_groups;
@@ -392,7 +393,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     // written by the previous kernel of the stream is read (and its inputs overwritten).
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (p.clear_status && blockIdx.x == 0 && tid == 0) { p.status[0] = 0; p.status[1] = 0; p.status[2] = 0; }
+    if (p.clear_status && blockIdx.x == 0 && tid < 8) p.status[tid] = 0;   // status words and the dm counter
     // The first kernel of a call may follow a kernel that produced its inputs: its first tiles
     // are requested here, right behind the wait.
     if (!early_loads && is_ctrl && lane == 0)
@@ -887,9 +888,39 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
 
     tc_fence_before();
     __syncthreads();
-    if (MODE != MODE_STATE && p.dm_partial != nullptr && tid == 0 && !*abort_flag) {
-        // Fixed-order reduction of <dV', V> over the CTA (the first-half warps of group O hold sums).
-        p.dm_partial[(size_t)bh * p.n_groups + g] = (dm_red[8] + dm_red[9]) + (dm_red[10] + dm_red[11]);
+    if (MODE != MODE_STATE && p.dm_partial != nullptr) {
+        int* last_flag = reinterpret_cast<int*>(&dm_red[15]);
+        if (tid == 0) {
+            // Fixed-order reduction of <dV', V> over the CTA (the first-half warps of group O hold sums).
+            if (!*abort_flag)
+                p.dm_partial[(size_t)bh * p.n_groups + g] = (dm_red[8] + dm_red[9]) + (dm_red[10] + dm_red[11]);
+            *last_flag = 0;
+            if (p.dm_out != nullptr) {
+                __threadfence();
+                *last_flag = atomicAdd(&p.status[4], 1) == (int)gridDim.x - 1;
+            }
+        }
+        __syncthreads();
+        if (*last_flag) {
+            // Every CTA's partial sum is visible: dm_h = sum_b dc/dm(b,h) * sum_g <dV', V>_{b,h,g},
+            // dc/dm = -ln(s_b) sigma(m_h) (1 - sigma(m_h)) c_{b,h}; fixed order, so deterministic.
+            __threadfence();
+            const int n_b = (int)gridDim.x / (p.n_groups * p.H);
+            for (int hh = tid; hh < p.H; hh += kTcThreads) {
+                const float sg = 1.0f / (1.0f + expf(-p.m[hh]));
+                float total = 0.f;
+                for (int bb = 0; bb < n_b; ++bb) {
+                    const float sb2 = p.seq_len ? p.seq_len[bb] : (p.seq_len_scalar > 0.f ? p.seq_len_scalar : (float)p.N);
+                    const float ls = logf(sb2);
+                    float acc = 0.f;
+                    for (int gg = 0; gg < p.n_groups; ++gg)
+                        acc += __ldcg(&p.dm_partial[((size_t)bb * p.H + hh) * p.n_groups + gg]);
+                    total += acc * (-ls * sg * (1.0f - sg) * expf(-sg * ls));
+                }
+                p.dm_out[hh] = total;
+            }
+            if (tid == 0) p.status[4] = 0;
+        }
     }
     if (*abort_flag) {
         // A wait gave up.  Before the CTA's shared memory and tensor memory go away, give the
@@ -1009,7 +1040,7 @@ cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cuda
     for (int i = 0; i < 5; ++i)
         if (!make_tile_map(&tm[i], ptrs[i], BH, N, d)) return cudaErrorInvalidValue;
     TcWalkParams p;
-    p.init = a.init; p.state_out = a.state_out; p.dm_partial = a.dm_partial; p.status = a.status;
+    p.init = a.init; p.state_out = a.state_out; p.dm_partial = a.dm_partial; p.dm_out = a.dm_out; p.status = a.status;
     p.m = a.m; p.seq_len = a.seq_len; p.seq_len_scalar = a.seq_len_scalar;
     p.H = H; p.N = N; p.group = a.group; p.n_groups = a.n_groups;
     p.init_sum = a.init_sum; p.init_transposed = a.init_transposed;
