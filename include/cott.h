@@ -115,6 +115,24 @@ cott_status cott_fwd(const void* q, const void* k, const void* v, void* o, float
                      void* stream);
 
 /*
+ * Causal forward over one SEGMENT of a longer sequence (chunked prefill; blocks of several
+ * tokens between decode steps): the running state of Eq. 8 carried across calls.
+ *   state_in  : NULL (the sequence starts here) or fp32 [B,H,d,d], the state left by the previous
+ *               segment, by cott_fwd (state_out) or by cott_decode_step; it contains c
+ *   state_out : NULL or fp32 [B,H,d,d] receiving state_in + sum_j k^_j (c v_j)^T over this segment;
+ *               must not be the same buffer as state_in
+ *   o         : rows of this segment, o_t = S_t^T q^_t with S_t including state_in
+ * The scaling base of Eq. 4 has to be the caller's and the same for every segment of one
+ * sequence: sp->seq_len ([B]) or sp->seq_len_scalar (>= 1); with that, the segments together
+ * give the rows of one cott_fwd over the whole sequence.  Other arguments as for cott_fwd
+ * (workspace: cott_workspace_bytes(COTT_OP_FWD, ..., causal = 1)).
+ */
+cott_status cott_fwd_stateful(const void* q, const void* k, const void* v, void* o,
+                              const float* state_in, float* state_out, int B, int H, int N, int d,
+                              cott_dtype dt, const cott_scale_params* sp, void* workspace,
+                              size_t workspace_bytes, void* stream);
+
+/*
  * Backward pass of cott_fwd for L = sum(d_o * O): the gradient formulas printed after Eq. 7
  * (dQ^ = (dO V'^T . M) K^, dK^ = (dO V'^T . M)^T Q^, dV' = (Q^ K^^T . M)^T dO; M all-ones when
  * causal == 0), evaluated through a forward running state and a state that accumulates

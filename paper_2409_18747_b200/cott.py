@@ -66,6 +66,9 @@ def _load():
     lib.cott_fwd.restype = ci
     lib.cott_fwd.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci,
                              ctypes.POINTER(_ScaleParams), vp, cs, vp]
+    lib.cott_fwd_stateful.restype = ci
+    lib.cott_fwd_stateful.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci,
+                                      ctypes.POINTER(_ScaleParams), vp, cs, vp]
     lib.cott_bwd.restype = ci
     lib.cott_bwd.argtypes = [vp] * 8 + [ci, ci, ci, ci, ci, ci, ctypes.POINTER(_ScaleParams), vp, cs, vp]
     lib.cott_decode_step.restype = ci
@@ -154,6 +157,32 @@ def fwd(q, k, v, m, seq_len=None, causal=True, return_state=False, out=None, wor
                           _stream_ptr(stream))
     if rc != 0:
         raise CottError(rc, "cott_fwd")
+    return (o, state) if return_state else o
+
+
+def fwd_stateful(q, k, v, m, seq_len, state_in=None, return_state=True, out=None, workspace=None,
+                 stream=None):
+    """cott_fwd_stateful: causal forward over one segment of a longer sequence.  ``state_in``
+    (fp32 ``[B,H,d,d]`` or None) is the state the previous segment (or a decode step) left;
+    ``seq_len`` (a float >= 1 or a float32 ``[B]`` CUDA tensor) is the scaling base of the WHOLE
+    sequence and must be the same for all its segments.  Returns ``(o, state)`` or ``o``."""
+    _check_dev(q, k, v, m, state_in, seq_len if isinstance(seq_len, torch.Tensor) else None)
+    if seq_len is None:
+        raise ValueError("fwd_stateful needs the scaling base of the whole sequence")
+    B, H, N, d = q.shape
+    dt = _dt(q)
+    if state_in is not None and (state_in.dtype != torch.float32 or tuple(state_in.shape) != (B, H, d, d)):
+        raise ValueError("state_in must be float32 [B,H,d,d]")
+    o = torch.empty_like(q) if out is None else out
+    state = torch.empty((B, H, d, d), dtype=torch.float32, device=q.device) if return_state else None
+    ws, ws_bytes = _workspace(OP_FWD, dt, B, H, N, d, True, q.device, workspace)
+    sp = _scale(m, seq_len)
+    rc = _load().cott_fwd_stateful(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
+                                   state_in.data_ptr() if state_in is not None else None,
+                                   state.data_ptr() if state is not None else None, B, H, N, d, dt,
+                                   ctypes.byref(sp), ws.data_ptr(), ws_bytes, _stream_ptr(stream))
+    if rc != 0:
+        raise CottError(rc, "cott_fwd_stateful")
     return (o, state) if return_state else o
 
 

@@ -139,8 +139,9 @@ static WalkArgs base_walk(const cott_scale_params* sp, int H, int N, const Plan&
 // One gradient / output stream through the generic walk: (optional) per-group partial
 // states, their scan, then the walk that produces rows.
 static cott_status run_stream(WalkArgs w, const Plan& p, int BH, int d, cott_dtype dt, int causal,
-                              float* states, float* total_out, cudaStream_t st) {
-    const bool single = causal && p.n_groups == 1;
+                              float* states, float* total_out, cudaStream_t st,
+                              const float* state_in = nullptr) {
+    const bool single = causal && p.n_groups == 1 && !state_in;
     if (single) {
         w.init = nullptr; w.update = 1; w.write_out = 1;
         w.final_state = total_out; w.final_grouped = 0;
@@ -153,7 +154,9 @@ static cott_status run_stream(WalkArgs w, const Plan& p, int BH, int d, cott_dty
     a.final_state = states; a.final_grouped = 1;
     COTT_CUDA(launch_walk_simt(a, BH, d, dt, st));
     const int mode = !causal ? SCAN_TOTAL : (w.reverse ? SCAN_SUFFIX : SCAN_PREFIX);
-    COTT_CUDA(launch_scan(states, total_out, BH, p.n_groups, d, mode, st));
+    // (these states contain c, like a caller's initial state, which the scan starts from)
+    COTT_CUDA(launch_scan(states, total_out, BH, p.n_groups, d, mode, st, nullptr, nullptr, 0.f, 1, 1,
+                          state_in));
     w.init = states; w.update = causal ? 1 : 0; w.write_out = 1; w.final_state = nullptr;
     COTT_CUDA(launch_walk_simt(w, BH, d, dt, st));
     return COTT_OK;
@@ -166,12 +169,12 @@ static cott_status run_tc_stream(TcWalkArgs t, const Plan& p, int B, int H, int 
                                  int causal, const cott_scale_params* sp, int* status,
                                  float* states, float* total_out, cudaStream_t st,
                                  bool reuse_states = false, bool states_only = false,
-                                 bool states_transposed = true) {
+                                 bool states_transposed = true, const float* state_in = nullptr) {
     const bool reuse_transposed = reuse_states;
     t.status = status; t.m = sp->m; t.seq_len = sp->seq_len; t.seq_len_scalar = sp->seq_len_scalar;
     t.group = p.group; t.n_groups = p.n_groups;
     // t.clear_status (first stream of a call) applies to the first kernel launched here only.
-    if (causal && p.n_groups == 1 && !total_out) {
+    if (causal && p.n_groups == 1 && !total_out && !state_in) {
         t.mode = 1; t.init = nullptr; t.state_out = nullptr;
         COTT_CUDA(launch_tc_walk(t, B, H, N, d, st));
         return COTT_OK;
@@ -179,7 +182,8 @@ static cott_status run_tc_stream(TcWalkArgs t, const Plan& p, int B, int H, int 
     // Few groups and no state export: every walk CTA sums the partial states it needs itself
     // and the scan launch is dropped -- as long as those extra d x d reads (n_groups / 2 of
     // them on average) stay small against the group's own q, k, v, o bytes.
-    const bool fused_scan = !total_out && p.n_groups <= 8 && (long)p.n_groups * d * 8 <= p.group;
+    // (A caller's initial state enters through the scan kernel.)
+    const bool fused_scan = !total_out && !state_in && p.n_groups <= 8 && (long)p.n_groups * d * 8 <= p.group;
     const int split = (fused_scan && causal) ? p.split : 1;
     if (!reuse_transposed) {
         TcWalkArgs a = t;
@@ -193,11 +197,13 @@ static cott_status run_tc_stream(TcWalkArgs t, const Plan& p, int B, int H, int 
             a.grid_groups = (p.n_groups - 1) * split;
             a.first_group = t.reverse ? split : 0;
         }
-        COTT_CUDA(launch_tc_walk(a, B, H, N, d, st));
+        const bool no_state_ctas = causal && !total_out && p.n_groups == 1;   // nothing to accumulate
+        if (!no_state_ctas) COTT_CUDA(launch_tc_walk(a, B, H, N, d, st));
+        else t.clear_status = a.clear_status;                                 // the walk is first, then
         const int mode = !causal ? SCAN_TOTAL : (t.reverse ? SCAN_SUFFIX : SCAN_PREFIX);
         if (!fused_scan)
             COTT_CUDA(launch_scan(states, total_out, B * H, p.n_groups, d, mode, st, sp->m, sp->seq_len,
-                                  sp->seq_len_scalar, H, N));
+                                  sp->seq_len_scalar, H, N, state_in));
     }
     // reuse_transposed: `states` already holds, transposed, what this stream needs (raw
     // partials when the scan is fused, scanned states otherwise) from a sibling stream that
@@ -214,7 +220,7 @@ static cott_status run_tc_stream(TcWalkArgs t, const Plan& p, int B, int H, int 
 static cott_status fwd_impl(const void* q, const void* k, const void* v, void* o, float* state_out,
                             int B, int H, int N, int d, int causal, cott_dtype dt,
                             const cott_scale_params* sp, void* ws, const Plan& p,
-                            cudaStream_t st) {
+                            cudaStream_t st, const float* state_in = nullptr) {
     // The tensor-core path clears the status words in its first kernel.
     if (p.path != 1) COTT_CUDA(cudaMemsetAsync(ws, 0, kWsHeaderBytes, st));
     float* states = reinterpret_cast<float*>(static_cast<char*>(ws) + kWsHeaderBytes);
@@ -225,13 +231,13 @@ static cott_status fwd_impl(const void* q, const void* k, const void* v, void* o
         t.norm_bv = 0; t.x_norm = 1; t.epilogue = EPI_PLAIN; t.reverse = 0;
         t.clear_status = 1;
         return run_tc_stream(t, p, B, H, N, d, causal, sp, static_cast<int*>(ws), states,
-                             state_out, st);
+                             state_out, st, false, false, true, state_in);
     }
     WalkArgs w = base_walk(sp, H, N, p);
     w.x = q; w.a = k; w.bv = v; w.out = o;
     w.mode_x = ROW_NORM; w.mode_a = ROW_NORM; w.mode_b = ROW_SCALE;
     w.epilogue = EPI_PLAIN; w.reverse = 0;
-    return run_stream(w, p, B * H, d, dt, causal, states, state_out, st);
+    return run_stream(w, p, B * H, d, dt, causal, states, state_out, st, state_in);
 }
 
 // Side streams and events for launches of one call that run next to each other on the GPU:
@@ -456,6 +462,28 @@ cott_status cott_fwd(const void* q, const void* k, const void* v, void* o, float
         return COTT_ERR_WORKSPACE;
     return fwd_impl(q, k, v, o, state_out, B, H, N, d, causal, dt, sp, workspace, p,
                     static_cast<cudaStream_t>(stream));
+}
+
+cott_status cott_fwd_stateful(const void* q, const void* k, const void* v, void* o,
+                              const float* state_in, float* state_out, int B, int H, int N, int d,
+                              cott_dtype dt, const cott_scale_params* sp, void* workspace,
+                              size_t workspace_bytes, void* stream) {
+    if (!q || !k || !v || !o || B < 1 || H < 1 || N < 1) return COTT_ERR_INVALID_ARG;
+    if (check_scale(sp) != COTT_OK) return COTT_ERR_INVALID_ARG;
+    if (o == q || o == k || o == v) return COTT_ERR_INVALID_ARG;
+    if (state_in && state_in == state_out) return COTT_ERR_INVALID_ARG;
+    // the scaling base must be the caller's (the same for every segment of a sequence)
+    if (!sp->seq_len && !(sp->seq_len_scalar >= 1.f)) return COTT_ERR_INVALID_ARG;
+    Plan p;
+    if (!make_plan(COTT_OP_FWD, dt, B, H, N, d, 1, &p)) return COTT_ERR_UNSUPPORTED;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) ||
+        (state_in && !aligned16(state_in)) || (state_out && !aligned16(state_out)))
+        return COTT_ERR_UNSUPPORTED;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
+        workspace_bytes < workspace_bytes_impl(COTT_OP_FWD, p, B, H, d))
+        return COTT_ERR_WORKSPACE;
+    return fwd_impl(q, k, v, o, state_out, B, H, N, d, 1, dt, sp, workspace, p,
+                    static_cast<cudaStream_t>(stream), state_in);
 }
 
 cott_status cott_bwd(const void* q, const void* k, const void* v, const void* d_o, void* dq,

@@ -50,7 +50,7 @@ cudaError_t launch_walk_simt(const WalkArgs& w, int BH, int d, cott_dtype dt, cu
 cudaError_t launch_scan(float* states, float* total_out, int BH, int n_groups, int d, int mode,
                         cudaStream_t st, const float* total_scale_m = nullptr,
                         const float* seq_len = nullptr, float seq_len_scalar = 0.f, int H = 1,
-                        int N = 1);
+                        int N = 1, const float* init_in = nullptr);
 
 // Tensor-core running-sum walk (bf16, d in {64,128}) with operand roles (x, a, bv); see
 // cott_tc_walk.cu.  mode: 0 partial states of every group, 1 chunk walk from the group's

@@ -230,7 +230,7 @@ __global__ void __launch_bounds__(256) scan_kernel(float* __restrict__ states,
                                                    float* __restrict__ total_out, int n_groups,
                                                    int dd, int mode, const float* scale_m,
                                                    const float* seq_len, float seq_len_scalar,
-                                                   int H, int N) {
+                                                   int H, int N, const float* __restrict__ init_in) {
     constexpr int kBatch = 8;
     const int e4 = blockIdx.x * blockDim.x + threadIdx.x;
     const int bh = blockIdx.y;
@@ -238,6 +238,19 @@ __global__ void __launch_bounds__(256) scan_kernel(float* __restrict__ states,
     float4* base = reinterpret_cast<float4*>(states + (size_t)bh * n_groups * dd) + e4;
     const size_t stride = (size_t)dd / 4;
     float4 run = make_float4(0.f, 0.f, 0.f, 0.f);
+    // With scale_m the states being scanned are unscaled and the total is multiplied by c on
+    // the way out; a caller's initial state (which contains c) enters divided by c.
+    float c = 1.f;
+    if (scale_m) {
+        const float s_b = seq_len ? seq_len[bh / H]
+                                  : (seq_len_scalar > 0.f ? seq_len_scalar : (float)N);
+        c = stab_factor(scale_m[bh % H], s_b);
+    }
+    if (init_in) {
+        const float4 v0 = reinterpret_cast<const float4*>(init_in + (size_t)bh * dd)[e4];
+        const float ic = 1.0f / c;
+        run = make_float4(v0.x * ic, v0.y * ic, v0.z * ic, v0.w * ic);
+    }
     auto add = [](float4& a, const float4& b) { a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w; };
     if (mode == SCAN_TOTAL) {
         for (int g0 = 0; g0 < n_groups; g0 += kBatch) {
@@ -270,12 +283,7 @@ __global__ void __launch_bounds__(256) scan_kernel(float* __restrict__ states,
         }
     }
     if (total_out) {
-        if (scale_m) {
-            const float s_b = seq_len ? seq_len[bh / H]
-                                      : (seq_len_scalar > 0.f ? seq_len_scalar : (float)N);
-            const float c = stab_factor(scale_m[bh % H], s_b);
-            run.x *= c; run.y *= c; run.z *= c; run.w *= c;
-        }
+        if (scale_m) { run.x *= c; run.y *= c; run.z *= c; run.w *= c; }
         reinterpret_cast<float4*>(total_out + (size_t)bh * dd)[e4] = run;
     }
 }
@@ -402,11 +410,11 @@ cudaError_t launch_walk_simt(const WalkArgs& w, int BH, int d, cott_dtype dt, cu
 
 cudaError_t launch_scan(float* states, float* total_out, int BH, int n_groups, int d, int mode,
                         cudaStream_t st, const float* total_scale_m, const float* seq_len,
-                        float seq_len_scalar, int H, int N) {
+                        float seq_len_scalar, int H, int N, const float* init_in) {
     const int dd = d * d;
     dim3 grid((unsigned)((dd / 4 + 255) / 256), (unsigned)BH);
     scan_kernel<<<grid, 256, 0, st>>>(states, total_out, n_groups, dd, mode, total_scale_m, seq_len,
-                                      seq_len_scalar, H, N);
+                                      seq_len_scalar, H, N, init_in);
     note_launch();
     return cudaGetLastError();
 }

@@ -401,3 +401,57 @@ def test_side_by_side_backward_matches_one_after_the_other(monkeypatch):
     monkeypatch.setenv("COTT_PAIR", "1")
     dq, dk, dv, _ = cott.bwd(q, k, v, d_o, m, causal=True)
     gate(dq[sub], rq, torch.bfloat16); gate(dk[sub], rk, torch.bfloat16); gate(dv[sub], rv, torch.bfloat16)
+
+
+# ------------------------------------------------------------------ stateful continuation (Eq. 8 across calls)
+@pytest.mark.parametrize("dtype,d", [(torch.bfloat16, 64), (torch.bfloat16, 128), (torch.float32, 32)])
+def test_segments_equal_one_long_forward(dtype, d, force_group):
+    """A sequence fed in segments through cott_fwd_stateful -- cuts at chunk and group
+    boundaries, next to them, and a ragged tail -- gives the rows of the definition over the
+    whole sequence, and the state left by the last segment is c K^^T V of all of it."""
+    force_group(256)
+    B, H, N = 2, 2, 1000
+    c = synth.make_qkv(B, H, N, d, dtype, 4700 + d)
+    s_b = torch.tensor([float(N), 600.0])
+    ref = oracle.fwd_quadratic(c["q"], c["k"], c["v"], c["m"], s_b, True)
+    _, ref_state = oracle.fwd_bidir_assoc(c["q"], c["k"], c["v"], c["m"], s_b)
+    q, k, v, m, s_dev = (dev(x) for x in (c["q"], c["k"], c["v"], c["m"], s_b))
+    for cuts in ([0, 1000], [0, 128, 256, 257, 511, 900, 1000], [0, 1, 2, 129, 1000]):
+        state, outs = None, []
+        for a, b in zip(cuts[:-1], cuts[1:]):
+            o, state = cott.fwd_stateful(q[:, :, a:b].contiguous(), k[:, :, a:b].contiguous(),
+                                         v[:, :, a:b].contiguous(), m, s_dev, state_in=state)
+            outs.append(o)
+        gate(torch.cat(outs, dim=2), ref, dtype)
+        assert norm_max_err(state, ref_state) <= state_tol(dtype, d)
+
+
+def test_segment_continues_decode_state():
+    """prefill (cott_fwd) -> a few decode steps -> a segment (cott_fwd_stateful) -> decode
+    again: every row equals the row of one long causal forward."""
+    B, H, d, N = 2, 3, 64, 640
+    c = synth.make_qkv(B, H, N, d, torch.bfloat16, 4800)
+    ref = oracle.fwd_quadratic(c["q"], c["k"], c["v"], c["m"], np.full((B,), float(N)), True)
+    q, k, v, m = (dev(c[x]) for x in ("q", "k", "v", "m"))
+    rows = []
+    o, state = cott.fwd(q[:, :, :300].contiguous(), k[:, :, :300].contiguous(), v[:, :, :300].contiguous(),
+                        m, seq_len=float(N), causal=True, return_state=True)
+    rows.append(o)
+    for t in range(300, 303):
+        rows.append(cott.decode_step(q[:, :, t].contiguous(), k[:, :, t].contiguous(), v[:, :, t].contiguous(),
+                                     state, m, float(N)).unsqueeze(2))
+    o, state = cott.fwd_stateful(q[:, :, 303:639].contiguous(), k[:, :, 303:639].contiguous(),
+                                 v[:, :, 303:639].contiguous(), m, float(N), state_in=state)
+    rows.append(o)
+    rows.append(cott.decode_step(q[:, :, 639].contiguous(), k[:, :, 639].contiguous(), v[:, :, 639].contiguous(),
+                                 state, m, float(N)).unsqueeze(2))
+    gate(torch.cat(rows, dim=2), ref, torch.bfloat16)
+
+
+def test_stateful_argument_checks():
+    c = synth.make_qkv(1, 1, 64, 64, torch.bfloat16, 4900)
+    q, k, v, m = (dev(c[x]) for x in ("q", "k", "v", "m"))
+    with pytest.raises(ValueError):
+        cott.fwd_stateful(q, k, v, m, None)
+    with pytest.raises(cott.CottError):
+        cott.fwd_stateful(q, k, v, m, 0.5)           # scaling base below 1
