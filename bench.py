@@ -426,6 +426,24 @@ def run_ours(args, w):
         e1.record(stream)
         torch.cuda.synchronize()
         loop_detail["loop_1024_graph_us_per_step"] = e0.elapsed_time(e1) * 1e3 / n_loop
+        # ---- blocks of T tokens through cott_fwd_stateful: the state is read and written once
+        # per block instead of once per token (L2 flushed before every block)
+        for T in (16, 128):
+            qb, kb, vb = mk(B, H, T, d), mk(B, H, T, d), mk(B, H, T, d)
+            ob = torch.empty_like(qb)
+            st_a = state.clone()
+            ws_blk = torch.empty(cott.workspace_bytes(cott.cott.OP_FWD, dt_code, B, H, T, d, True),
+                                 dtype=torch.uint8, device=dev)
+            ts = []
+            for i in range(8):
+                flush_l2(i)
+                e0.record(stream)
+                _, st_b = cott.fwd_stateful(qb, kb, vb, m, 8192.0, state_in=st_a, out=ob, workspace=ws_blk)
+                e1.record(stream)
+                torch.cuda.synchronize()
+                ts.append(e0.elapsed_time(e1))
+                st_a = st_b
+            loop_detail[f"block_T{T}_us_per_token"] = statistics.median(ts[2:]) * 1e3 / T
 
     if world > 1:
         import torch.distributed as dist

@@ -164,7 +164,7 @@ static cott_status run_stream(WalkArgs w, const Plan& p, int BH, int d, cott_dty
 
 // One output stream through the tensor-core walk: partial states of every group, their
 // scan, then the chunk walk (causal) or the read-out against the total (bidirectional).
-// A causal call with a single group and no state export needs only the walk.
+// A causal call with a single group needs only the walk.
 static cott_status run_tc_stream(TcWalkArgs t, const Plan& p, int B, int H, int N, int d,
                                  int causal, const cott_scale_params* sp, int* status,
                                  float* states, float* total_out, cudaStream_t st,
@@ -174,8 +174,11 @@ static cott_status run_tc_stream(TcWalkArgs t, const Plan& p, int B, int H, int 
     t.status = status; t.m = sp->m; t.seq_len = sp->seq_len; t.seq_len_scalar = sp->seq_len_scalar;
     t.group = p.group; t.n_groups = p.n_groups;
     // t.clear_status (first stream of a call) applies to the first kernel launched here only.
-    if (causal && p.n_groups == 1 && !total_out && !state_in) {
-        t.mode = 1; t.init = nullptr; t.state_out = nullptr;
+    if (causal && p.n_groups == 1) {
+        // One group: the walk alone, starting from the caller's state (if any) and leaving the
+        // final state (if asked for).
+        t.mode = 1; t.init = state_in; t.init_has_scale = state_in ? 1 : 0; t.state_out = nullptr;
+        t.state_final = total_out;
         COTT_CUDA(launch_tc_walk(t, B, H, N, d, st));
         return COTT_OK;
     }
@@ -197,9 +200,7 @@ static cott_status run_tc_stream(TcWalkArgs t, const Plan& p, int B, int H, int 
             a.grid_groups = (p.n_groups - 1) * split;
             a.first_group = t.reverse ? split : 0;
         }
-        const bool no_state_ctas = causal && !total_out && p.n_groups == 1;   // nothing to accumulate
-        if (!no_state_ctas) COTT_CUDA(launch_tc_walk(a, B, H, N, d, st));
-        else t.clear_status = a.clear_status;                                 // the walk is first, then
+        COTT_CUDA(launch_tc_walk(a, B, H, N, d, st));
         const int mode = !causal ? SCAN_TOTAL : (t.reverse ? SCAN_SUFFIX : SCAN_PREFIX);
         if (!fused_scan)
             COTT_CUDA(launch_scan(states, total_out, B * H, p.n_groups, d, mode, st, sp->m, sp->seq_len,

@@ -82,6 +82,10 @@ struct TcWalkArgs {
     // EPI_DV: when set, the CTA that finishes last turns the [BH, n_groups] partial sums of
     // <dV', V> into dm[H] (fixed summation order), so no separate launch is needed.
     float* dm_out;
+    // Causal walk of a single group: `init` is a caller's state (it contains c and is divided
+    // by c on the way in), and the state after the last token goes to state_final, times c.
+    int init_has_scale;
+    float* state_final;
 };
 cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cudaStream_t st);
 

@@ -40,6 +40,8 @@ struct TcWalkParams {
     float* state_out;       // MODE_STATE: [BH, n_groups, d*d] partial states (unscaled)
     float* dm_partial;      // EPI_DV: [BH, n_groups]
     float* dm_out;          // EPI_DV: dm[H], written by the CTA that finishes last (or NULL)
+    int init_has_scale;     // init is a caller's state (contains c): divide by c on the way in
+    float* state_final;     // causal walk, one group: [BH, d*d] state after the last token, times c (or NULL)
     int* status;            // workspace status word
     const float* m; const float* seq_len; float seq_len_scalar;
     int H; int N; int group; int n_groups;
@@ -441,6 +443,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
 #pragma unroll
             for (int i = 0; i < QW; i += 4) {
                 float4 v = owns_srow ? load4(g, i) : make_float4(0.f, 0.f, 0.f, 0.f);
+                if (p.init_has_scale) { const float ic = 1.0f / cfac; v.x *= ic; v.y *= ic; v.z *= ic; v.w *= ic; }
                 r[i] = __float_as_uint(v.x); r[i + 1] = __float_as_uint(v.y);
                 r[i + 2] = __float_as_uint(v.z); r[i + 3] = __float_as_uint(v.w);
             }
@@ -879,6 +882,23 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                                     __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
             }
         }
+        if (MODE == MODE_CAUSAL && p.state_final != nullptr && alive) {
+            // State after the last token of the (single) group, times c: the caller's Eq. 8 state.
+            if (wait(sfull_bar(n_chunks - 1), sfull_par(n_chunks - 1))) {
+                tc_fence_after();
+                float* dst = p.state_final + (size_t)bh * D * D + (size_t)srow * D + cq * QW;
+                uint32_t r[QW];
+                tmem_ldq<QW>(tmem + lane_base + colS + cq * QW, r);
+                tmem_wait_ld();
+                if (owns_srow) {
+#pragma unroll
+                    for (int i = 0; i < QW; i += 4)
+                        *reinterpret_cast<float4*>(dst + i) =
+                            make_float4(__uint_as_float(r[i]) * cfac, __uint_as_float(r[i + 1]) * cfac,
+                                        __uint_as_float(r[i + 2]) * cfac, __uint_as_float(r[i + 3]) * cfac);
+                }
+            }
+        }
         if (MODE != MODE_STATE && p.dm_partial != nullptr) {
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) dm_acc += __shfl_xor_sync(0xffffffffu, dm_acc, o);
@@ -1041,6 +1061,7 @@ cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cuda
         if (!make_tile_map(&tm[i], ptrs[i], BH, N, d)) return cudaErrorInvalidValue;
     TcWalkParams p;
     p.init = a.init; p.state_out = a.state_out; p.dm_partial = a.dm_partial; p.dm_out = a.dm_out; p.status = a.status;
+    p.init_has_scale = a.init_has_scale; p.state_final = a.state_final;
     p.m = a.m; p.seq_len = a.seq_len; p.seq_len_scalar = a.seq_len_scalar;
     p.H = H; p.N = N; p.group = a.group; p.n_groups = a.n_groups;
     p.init_sum = a.init_sum; p.init_transposed = a.init_transposed;
