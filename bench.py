@@ -286,13 +286,16 @@ def run_ours(args, w):
     flush_sink = torch.zeros(1, dtype=torch.int32, device=dev)
 
     def flush_l2(i):
-        """Evicts the step's tensors from L2 by READING a buffer twice the size of L2.  (A
-        write would leave the L2 full of dirty lines whose write-back would then be charged to
-        the timed kernels.)"""
-        if os.environ.get("COTT_BENCH_FLUSH", "read") == "write":
-            flush.fill_(i & 0xFF)
-        else:
+        """Evicts the step's tensors from L2 by writing a buffer twice the size of L2.  The L2
+        is then full of dirty lines of that buffer, whose write-back the timed kernels pay for
+        as they bring in their own data -- about what a steady-state step pays for evicting
+        the outputs of the step before it.  COTT_BENCH_FLUSH=read evicts by reading instead
+        (clean lines; the kernels' own output write-back then falls partly outside the timed
+        region, which flatters short kernels)."""
+        if os.environ.get("COTT_BENCH_FLUSH", "write") == "read":
             torch.amax(flush, dim=0, keepdim=True, out=flush_sink)
+        else:
+            flush.fill_(i & 0xFF)
 
     stream = torch.cuda.current_stream()
     dt_code = cott.cott.BF16
@@ -354,6 +357,18 @@ def run_ours(args, w):
     barrier()
     clocks = sampler.stop()
     launches = cott.cott.launch_count() - launches0
+    # the same steps without the flush: part of the tensors (all of them, for the small
+    # workloads) is then served from L2 -- reported beside the flushed figure, never instead
+    ev_u = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    n_unfl = max(3, min(args.steps, 50))
+    ev_u[0].record(stream)
+    for _ in range(n_unfl):
+        fwd_call()
+        if bwd_call is not None:
+            bwd_call()
+    ev_u[1].record(stream)
+    torch.cuda.synchronize()
+    unflushed_ms = ev_u[0].elapsed_time(ev_u[1]) / n_unfl
     step_ms_local = (sum(fwd_ms) + sum(bwd_ms)) / args.steps
     step_ms = max_over_ranks(step_ms_local, world)
     value = aggregate_tokens_per_s(tokens_per_step, world, step_ms)
@@ -479,6 +494,7 @@ def run_ours(args, w):
     extra = {"fwd_ms": fwd_mean, "fwd_gbs": ab["fwd"] / (fwd_mean * 1e-3) / 1e9,
              "fwd_frac": ab["fwd"] / (fwd_mean * 1e-3) / 1e9 / peaks["hbm_gbs"],
              "step_frac": (ab["fwd"] + ab["bwd"]) / (step_ms_local * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    extra["step_ms_unflushed_back_to_back"] = unflushed_ms
     extra.update(loop_detail)
     if bwd_call is not None:
         extra["bwd_ms"] = statistics.mean(bwd_ms)
@@ -500,7 +516,7 @@ def run_ours(args, w):
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w["name"], "B": B, "H": H, "N": N, "d": d, "causal": w["causal"],
                    "io": "bf16, fp32 state and accumulators", "parallelism": f"replicas x{world}",
-                   "l2": "flushed before every step (256 MB read); working set also exceeds L2",
+                   "l2": "flushed before every step (256 MB " + os.environ.get("COTT_BENCH_FLUSH", "write") + "); working set also exceeds L2",
                    "plan": plan},
         "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
         "detail": extra,

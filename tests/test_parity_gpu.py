@@ -483,3 +483,20 @@ def test_repeated_calls_are_bit_identical(shape):
     assert cott.cott.last_async_status(ws_f) == 0 and cott.cott.last_async_status(ws_b) == 0
     assert acc.tolist() == [0, 0, 0, 0, 0]
     assert all(torch.isfinite(x.float()).all() for x in first)
+
+
+def test_bidirectional_backward_many_heads():
+    """Bidirectional gradients at a BERT-like shape with more (b,h) pairs than SMs: one group of
+    four chunks per CTA through the read-out form of every gradient stream."""
+    B, H, N, d = 13, 12, 512, 64
+    c = synth.make_qkv(B, H, N, d, torch.bfloat16, 5100, with_do=True)
+    q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
+    dq, dk, dv, dm = cott.bwd(q, k, v, d_o, m, causal=False)
+    sub = slice(0, 2)        # the definition on the first two batch items
+    rq, rk, rv, _ = oracle.bwd_quadratic(c["q"][sub], c["k"][sub], c["v"][sub], c["d_o"][sub], c["m"], None, False)
+    gate(dq[sub], rq, torch.bfloat16); gate(dk[sub], rk, torch.bfloat16); gate(dv[sub], rv, torch.bfloat16)
+    # dm sums over the batch: both routes on the GPU result (dm_h = sum_b <dO,O> dc/dm / c)
+    o = cott.fwd(q, k, v, m, causal=False)
+    sg = torch.sigmoid(m.double())
+    route2 = (d_o.double() * o.double()).sum(dim=(0, 2, 3)) * (-np.log(float(N))) * sg * (1 - sg)
+    torch.testing.assert_close(dm.double(), route2, rtol=5e-2, atol=5e-2 * float(route2.abs().max()))
