@@ -361,6 +361,10 @@ def run_ours(args, w):
     # workloads) is then served from L2 -- reported beside the flushed figure, never instead
     ev_u = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
     n_unfl = max(3, min(args.steps, 50))
+    for _ in range(5):                       # the GPU has idled for a moment: steps to get back up to speed
+        fwd_call()
+        if bwd_call is not None:
+            bwd_call()
     ev_u[0].record(stream)
     for _ in range(n_unfl):
         fwd_call()
