@@ -168,7 +168,9 @@ cott_status cott_decode_step(const void* q, const void* k, const void* v, float*
 
 /*
  * Training step with HOST buffers (end-to-end path): copies q,k,v,d_o from host memory to the
- * device arena, runs cott_fwd then cott_bwd, and copies o,dq,dk,dv,dm back, all on `stream`.
+ * device arena, runs cott_fwd then cott_bwd, and copies o,dq,dk,dv,dm back.  The call is ordered
+ * on `stream` as a whole; inside, o travels back on a stream of the library while d_o comes in
+ * (the link is full duplex), joined into `stream` before the call's last copy.
  *   *_host  : host pointers ([B,H,N,d] dt; dm_host fp32 [H]); pinned memory makes the copies
  *             asynchronous.  m_host fp32 [H], seq_len_host fp32 [B] or NULL (s_b = N).
  *   arena   : device scratch of at least cott_host_step_arena_bytes() bytes, 256-B aligned.

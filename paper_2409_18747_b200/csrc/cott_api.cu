@@ -246,8 +246,8 @@ static cott_status fwd_impl(const void* q, const void* k, const void* v, void* o
 // created on the first call that needs them and kept until the process ends.
 struct SideStreams {
     bool ready = false;
-    cudaStream_t s[2];
-    cudaEvent_t fork, join[2];
+    cudaStream_t s[3];            // [0], [1]: gradient streams of cott_bwd; [2]: copies of the host step
+    cudaEvent_t fork, join[3], fork_copy;
 };
 static SideStreams* side_streams() {
     static thread_local SideStreams per_device[64];
@@ -255,11 +255,12 @@ static SideStreams* side_streams() {
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
     SideStreams& ss = per_device[dev];
     if (!ss.ready) {
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < 3; ++i) {
             if (cudaStreamCreateWithFlags(&ss.s[i], cudaStreamNonBlocking) != cudaSuccess) return nullptr;
             if (cudaEventCreateWithFlags(&ss.join[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
         }
         if (cudaEventCreateWithFlags(&ss.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        if (cudaEventCreateWithFlags(&ss.fork_copy, cudaEventDisableTiming) != cudaSuccess) return nullptr;
         ss.ready = true;
     }
     return &ss;
@@ -580,7 +581,6 @@ cott_status cott_fwd_bwd_host(const void* q_host, const void* k_host, const void
     COTT_CUDA(cudaMemcpyAsync(q_, q_host, nbytes, cudaMemcpyHostToDevice, st));
     COTT_CUDA(cudaMemcpyAsync(k_, k_host, nbytes, cudaMemcpyHostToDevice, st));
     COTT_CUDA(cudaMemcpyAsync(v_, v_host, nbytes, cudaMemcpyHostToDevice, st));
-    COTT_CUDA(cudaMemcpyAsync(do_, d_o_host, nbytes, cudaMemcpyHostToDevice, st));
     COTT_CUDA(cudaMemcpyAsync(m_, m_host, (size_t)H * 4, cudaMemcpyHostToDevice, st));
     if (seq_len_host)
         COTT_CUDA(cudaMemcpyAsync(sl_, seq_len_host, (size_t)B * 4, cudaMemcpyHostToDevice, st));
@@ -588,9 +588,19 @@ cott_status cott_fwd_bwd_host(const void* q_host, const void* k_host, const void
     sp.m = m_; sp.seq_len = seq_len_host ? sl_ : nullptr; sp.seq_len_scalar = 0.f;
     cott_status rc = cott_fwd(q_, k_, v_, o_, nullptr, B, H, N, d, causal, dt, &sp, ws, wsz, stream);
     if (rc != COTT_OK) return rc;
+    // The link is full duplex: o goes back to the host on a side stream while dO comes in.
+    SideStreams* ss = side_streams();
+    if (ss) {
+        COTT_CUDA(cudaEventRecord(ss->fork_copy, st));
+        COTT_CUDA(cudaStreamWaitEvent(ss->s[2], ss->fork_copy, 0));
+        COTT_CUDA(cudaMemcpyAsync(o_host, o_, nbytes, cudaMemcpyDeviceToHost, ss->s[2]));
+        COTT_CUDA(cudaEventRecord(ss->join[2], ss->s[2]));
+    }
+    COTT_CUDA(cudaMemcpyAsync(do_, d_o_host, nbytes, cudaMemcpyHostToDevice, st));
     rc = cott_bwd(q_, k_, v_, do_, dq_, dk_, dv_, dm_, B, H, N, d, causal, dt, &sp, ws, wsz, stream);
     if (rc != COTT_OK) return rc;
-    COTT_CUDA(cudaMemcpyAsync(o_host, o_, nbytes, cudaMemcpyDeviceToHost, st));
+    if (ss) COTT_CUDA(cudaStreamWaitEvent(st, ss->join[2], 0));
+    else COTT_CUDA(cudaMemcpyAsync(o_host, o_, nbytes, cudaMemcpyDeviceToHost, st));
     COTT_CUDA(cudaMemcpyAsync(dq_host, dq_, nbytes, cudaMemcpyDeviceToHost, st));
     COTT_CUDA(cudaMemcpyAsync(dk_host, dk_, nbytes, cudaMemcpyDeviceToHost, st));
     COTT_CUDA(cudaMemcpyAsync(dv_host, dv_, nbytes, cudaMemcpyDeviceToHost, st));
