@@ -239,7 +239,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     constexpr int NH = D / 64;                       // 64-column half tiles per row
     constexpr uint32_t kTmemCols = 512;
     // Columns: State d | P 128 (fp32 scores) | P~ 64 (bf16 masked scores, packed) | Out.
-    // d = 64 double-buffers Out; at d = 128 only one Out buffer fits in the 512 columns.
+    // d = 64 double-buffers Out; at d = 128 one Out buffer is used (448 of the 512 columns).
     constexpr uint32_t colS = 0, colP = D, colPt = D + 128, colO0 = D + 192;
     constexpr int kOBufs = (D == 64) ? 2 : 1;
     constexpr int QW = D / 4;                        // accumulator columns per worker thread
@@ -475,9 +475,9 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
 
     float dm_acc = 0.f;
 
-    // The stage of chunk c is refilled with chunk c + NST in two steps when possible: X and A
-    // as soon as the last MMA that reads the stage has completed (control thread), Bv -- the
-    // output staging slot -- after the chunk's output store has drained (store thread).
+    // The stage of chunk c is refilled with chunk c + NST by the store thread, in two steps
+    // when possible: X and A as soon as the last MMAs that read the stage have completed, Bv
+    // -- the output staging slot -- after the chunk's output store has drained.
     constexpr bool split_refill = MODE == MODE_CAUSAL && !(with_proj && L::kProjInA);
 
     if (is_ctrl) {
@@ -500,7 +500,6 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     issue_p<D>(tmem + colP, stage_x(s), stage_a(s));
                     tc_commit(bar_p_full);
                 }
-                { const int cn = c; { const int c = cn - 1; COTT_STAMP(5); } }   // stamped with the loop's chunk
                 if (MODE != MODE_STATE) {
                     if (MODE == MODE_CAUSAL && c >= 1 && !wait(sb_bar(c - 1), sb_par(c - 1))) return;
                     // The output accumulator this chunk writes must have been drained: by chunk
