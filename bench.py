@@ -197,7 +197,7 @@ def aggregate_tokens_per_s(tokens_per_rank_step: int, world: int, ms_per_step_ma
 
 
 # ----------------------------------------------------------------------------- CPU oracle arm
-def oracle_sample_step(w: dict, sample_heads: int):
+def oracle_sample_step(w: dict, sample_heads: int, form: str = "quadratic"):
     """Returns (callable running the oracle once on the bounded sample, tokens it covers).
     The sample keeps N and d and takes `sample_heads` heads of one batch item; tokens are
     scaled by the fraction of (b,h) pairs covered."""
@@ -222,13 +222,21 @@ def oracle_sample_step(w: dict, sample_heads: int):
                                       f"at N={w['N']}, d={w['d']}")
     c = synth.make_qkv(1, H, w["N"], w["d"], torch.bfloat16, 99, with_do=True)
 
+    recurrent = form == "recurrent" and w["causal"]
+
     def run():
+        if recurrent:
+            oracle.fwd_recurrent(c["q"], c["k"], c["v"], c["m"], None)
+            if w["bwd"]:
+                oracle.bwd_recurrent(c["q"], c["k"], c["v"], c["d_o"], c["m"], None)
+            return
         oracle.fwd_quadratic(c["q"], c["k"], c["v"], c["m"], None, w["causal"])
         if w["bwd"]:
             oracle.bwd_quadratic(c["q"], c["k"], c["v"], c["d_o"], c["m"], None, w["causal"])
     frac = H / (w["B"] * w["H"])
     what = "fwd+bwd" if w["bwd"] else "fwd"
-    return run, w["B"] * w["N"] * frac, (f"fp64 quadratic definition {what} on {H} of {w['B'] * w['H']} (b,h) "
+    name = "recurrence (Eq. 8, running state)" if recurrent else "quadratic definition"
+    return run, w["B"] * w["N"] * frac, (f"fp64 {name} {what} on {H} of {w['B'] * w['H']} (b,h) "
                                          f"pairs at N={w['N']}, d={w['d']}")
 
 
@@ -239,10 +247,16 @@ def run_reference(args, w):
     import oracle
     # bounded sample: fewer (b,h) pairs per step when more steps are asked for, so the whole
     # run stays within a few minutes (one pair at N=4096, d=64 is about 4 core-seconds)
+    n_runs = args.steps + max(1, min(args.warmup, 1))
     heads = max(1, min(16, 48 // max(args.steps, 1)))
+    form = "quadratic"
     if w["N"] > 4096:
         heads = 1
-    run, tokens, what = oracle_sample_step(w, heads)
+    elif n_runs > 60 and w["causal"] and not w.get("decode"):
+        # many steps: even one pair per step of the quadratic definition (about 1.6 s) would run
+        # for many minutes; the oracle's linear-time recurrence on 16 pairs takes a fraction of that
+        form, heads = "recurrent", 16
+    run, tokens, what = oracle_sample_step(w, heads, form)
     for _ in range(max(1, min(args.warmup, 1))):
         run()
     t0 = time.perf_counter()
