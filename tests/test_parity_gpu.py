@@ -500,3 +500,35 @@ def test_bidirectional_backward_many_heads():
     sg = torch.sigmoid(m.double())
     route2 = (d_o.double() * o.double()).sum(dim=(0, 2, 3)) * (-np.log(float(N))) * sg * (1 - sg)
     torch.testing.assert_close(dm.double(), route2, rtol=5e-2, atol=5e-2 * float(route2.abs().max()))
+
+
+# ------------------------------------------------------------------ seeded sweep over shapes
+def _sweep_cases():
+    rng = np.random.RandomState(77)
+    cases = []
+    for i in range(14):
+        d = int(rng.choice([32, 64, 128]))
+        dtype = torch.float32 if d == 32 and rng.rand() < 0.7 else torch.bfloat16
+        B = int(rng.randint(1, 5)); H = int(rng.randint(1, 20))
+        N = int(rng.choice([1, 2, 63, 127, 128, 129, 255, 300, 511, 640, 777]))
+        cases.append((B, H, N, d, dtype, bool(rng.rand() < 0.75), i))
+    return cases
+
+
+@pytest.mark.parametrize("case", _sweep_cases(), ids=lambda c: f"B{c[0]}H{c[1]}N{c[2]}d{c[3]}{'bf16' if c[4] == torch.bfloat16 else 'f32'}{'c' if c[5] else 'b'}")
+def test_shape_sweep_forward_backward(case):
+    """Seeded sweep over batch, heads, length, head size, dtype and masking with the library's
+    own plan (no forced group): forward, exported state and all gradients against the
+    definition."""
+    B, H, N, d, dtype, causal, i = case
+    c = synth.make_qkv(B, H, N, d, dtype, 5200 + i, with_do=True)
+    args = [dev(c[x]) for x in ("q", "k", "v")]
+    o, st = cott.fwd(*args, dev(c["m"]), causal=causal, return_state=True)
+    gate(o, oracle.fwd_quadratic(c["q"], c["k"], c["v"], c["m"], None, causal), dtype)
+    _, ref_state = oracle.fwd_bidir_assoc(c["q"], c["k"], c["v"], c["m"], None)
+    assert norm_max_err(st, ref_state) <= state_tol(dtype, d)
+    dq, dk, dv, dm = cott.bwd(*args, dev(c["d_o"]), dev(c["m"]), causal=causal)
+    rq, rk, rv, rm = oracle.bwd_quadratic(c["q"], c["k"], c["v"], c["d_o"], c["m"], None, causal)
+    gate(dq, rq, dtype); gate(dk, rk, dtype); gate(dv, rv, dtype)
+    f32 = dtype == torch.float32
+    gate_dm(dm, rm, 1e-4 if f32 else 1e-2, dm_condition(rv, c["v"], c["m"], None), DM_COND_F32 if f32 else DM_COND_BF16)
