@@ -255,8 +255,14 @@ static SideStreams* side_streams() {
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
     SideStreams& ss = per_device[dev];
     if (!ss.ready) {
+        // s[0] carries a walk that should start together with the one on the caller's stream;
+        // it gets the highest priority, so that its CTAs are placed ahead of the state pass on
+        // s[1] when both become ready on the same event.
+        int prio_lo = 0, prio_hi = 0;
+        if (cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi) != cudaSuccess) return nullptr;
         for (int i = 0; i < 3; ++i) {
-            if (cudaStreamCreateWithFlags(&ss.s[i], cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+            if (cudaStreamCreateWithPriority(&ss.s[i], cudaStreamNonBlocking, i == 0 ? prio_hi : prio_lo) != cudaSuccess)
+                return nullptr;
             if (cudaEventCreateWithFlags(&ss.join[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
         }
         if (cudaEventCreateWithFlags(&ss.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
