@@ -532,3 +532,28 @@ def test_shape_sweep_forward_backward(case):
     gate(dq, rq, dtype); gate(dk, rk, dtype); gate(dv, rv, dtype)
     f32 = dtype == torch.float32
     gate_dm(dm, rm, 1e-4 if f32 else 1e-2, dm_condition(rv, c["v"], c["m"], None), DM_COND_F32 if f32 else DM_COND_BF16)
+
+
+@pytest.mark.parametrize("dtype,d", [(torch.bfloat16, 128), (torch.bfloat16, 64), (torch.float32, 32)])
+def test_short_blocks_many_heads(dtype, d):
+    """More (b,h) pairs than SMs and blocks of a few tokens (the shape of tokens between decode
+    steps): prefill, then blocks of 1, 7, 32 and 20 tokens through cott_fwd_stateful; every row
+    equals the row of one long causal forward."""
+    B, H, N0 = 10, 16, 100
+    cuts = [N0, N0 + 1, N0 + 8, N0 + 40, N0 + 60]
+    N = cuts[-1]
+    c = synth.make_qkv(B, H, N, d, dtype, 5300 + d)
+    ref = oracle.fwd_quadratic(c["q"], c["k"], c["v"], c["m"], np.full((B,), float(N)), True)
+    _, ref_state = oracle.fwd_bidir_assoc(c["q"], c["k"], c["v"], c["m"], np.full((B,), float(N)))
+    q, k, v, m = (dev(c[x]) for x in ("q", "k", "v", "m"))
+    seg = lambda x, a, b: x[:, :, a:b].contiguous()
+    o, state = cott.fwd(seg(q, 0, N0), seg(k, 0, N0), seg(v, 0, N0), m, seq_len=float(N), causal=True, return_state=True)
+    rows = [o]
+    for a, b in zip(cuts[:-1], cuts[1:]):
+        o, state = cott.fwd_stateful(seg(q, a, b), seg(k, a, b), seg(v, a, b), m, float(N), state_in=state)
+        rows.append(o)
+    gate(torch.cat(rows, dim=2), ref, dtype)
+    assert norm_max_err(state, ref_state) <= state_tol(dtype, d)
+    # a block with no state to start from is a short causal forward
+    o0 = cott.fwd_stateful(seg(q, 0, 9), seg(k, 0, 9), seg(v, 0, 9), m, float(N), return_state=False)
+    gate(o0, ref[:, :, :9], dtype)
