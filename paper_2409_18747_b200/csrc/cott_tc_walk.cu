@@ -16,6 +16,7 @@
 // Modes:  MODE_STATE   only accumulates the group's partial state and writes it (phase A);
 //         MODE_CAUSAL  the chunk walk starting from the group's prefix / suffix state;
 //         MODE_READOUT Out = X State for a fixed state (bidirectional form, Eq. 5).
+#include <stdlib.h>
 #include "cott_internal.h"
 #include "cott_sm100.cuh"
 
@@ -27,7 +28,7 @@ namespace {
 
 constexpr int kChunk = 128;
 constexpr int kTcThreads = 608;   // 16 row-worker warps + control warp + store warp + state-update warp
-constexpr long long kWaitTimeoutCycles = 4000000000ll;  // about 2 s of SM clock: far above any legitimate wait
+constexpr int kWaitLimitMsDefault = 2000;   // bound of every device-side wait: far above any legitimate one
 
 struct TcWalkParams {
     const float* init;      // [BH, n_groups, d*d] unscaled group states, or NULL
@@ -48,6 +49,8 @@ struct TcWalkParams {
     int first_group; int grid_groups;   // groups this launch covers: one CTA per (b, h, group)
     int plain_launch;                   // host side only: launch without programmatic serialization
     int clear_status;                   // first kernel of a call: CTA 0 zeroes the status words
+    int wait_limit_kcycles;             // bound of every wait, in units of 1024 SM cycles
+    int debug_drop_commit;              // test hook: the scores of chunk 1 are never reported complete
 };
 
 enum { MODE_STATE = 0, MODE_CAUSAL = 1, MODE_READOUT = 2 };
@@ -180,7 +183,8 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, vol
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 15u) == 0) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitTimeoutCycles) {
+            // the limit (in units of 1024 SM cycles) sits three words behind the abort flag
+            if (clock64() - t0 > ((long long)abort_flag[3] << 10)) {
                 const uint32_t bars = (uint32_t)__cvta_generic_to_shared((const void*)abort_flag) - 236u;
                 const uint32_t where = 0x80000000u | ((threadIdx.x >> 5) << 16) | (((bar - bars) & 0x3FFu) << 4) | (parity & 1u);
                 atomicCAS(const_cast<int*>(abort_flag), 0, (int)where);
@@ -319,6 +323,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         mbar_init(bar_proj, 1);
         mbar_init(bar_xch, kGroupThreads);
         *abort_flag = 0;
+        abort_flag[3] = p.wait_limit_kcycles;
         mbar_fence_init();
         fence_proxy_async();
     }
@@ -498,7 +503,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     // Scores first: they need neither the state copy nor the output buffer.
                     tc_fence_after();
                     issue_p<D>(tmem + colP, stage_x(s), stage_a(s));
-                    tc_commit(bar_p_full);
+                    if (!(p.debug_drop_commit && c == 1)) tc_commit(bar_p_full);
                 }
                 if (MODE != MODE_STATE) {
                     if (MODE == MODE_CAUSAL && c >= 1 && !wait(sb_bar(c - 1), sb_par(c - 1))) return;
@@ -1071,6 +1076,13 @@ cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cuda
     p.grid_groups = subset ? a.grid_groups : a.n_groups;
     p.plain_launch = a.plain_launch;
     p.clear_status = a.clear_status;
+    {   // knobs for the test of the timeout path: a short bound, and a hand-off that never comes
+        const char* e = getenv("COTT_WAIT_LIMIT_MS");
+        const long ms = (e && *e) ? atol(e) : kWaitLimitMsDefault;
+        p.wait_limit_kcycles = (int)((ms < 1 ? 1 : (ms > 100000 ? 100000 : ms)) * 2000);   // <= 2 GHz
+        e = getenv("COTT_DEBUG_DROP_COMMIT");
+        p.debug_drop_commit = (e && *e == '1') ? 1 : 0;
+    }
     if (p.first_group < 0 || p.first_group + p.grid_groups > a.n_groups) return cudaErrorInvalidValue;
     // The four combinations of roles the library uses, as compile-time kernel variants.
     int kind;

@@ -557,3 +557,28 @@ def test_short_blocks_many_heads(dtype, d):
     # a block with no state to start from is a short causal forward
     o0 = cott.fwd_stateful(seg(q, 0, 9), seg(k, 0, 9), seg(v, 0, 9), m, float(N), return_state=False)
     gate(o0, ref[:, :, :9], dtype)
+
+
+# ------------------------------------------------------------------ a wait that runs out
+def test_bounded_wait_runs_out_and_reports(monkeypatch, force_group):
+    """Every device-side wait has a bound.  With the bound set to 20 ms and one hand-off
+    withheld (the scores of chunk 1 are never reported complete -- a flag that nothing sets),
+    the kernel gives up, reports where, frees its tensor memory and returns; the context stays
+    usable and the next call is correct."""
+    force_group(512)
+    c = synth.make_qkv(1, 2, 512, 64, torch.bfloat16, 5400)
+    q, k, v, m = (dev(c[x]) for x in ("q", "k", "v", "m"))
+    ws = torch.zeros(cott.workspace_bytes(cott.cott.OP_FWD, cott.cott.BF16, 1, 2, 512, 64, True),
+                     dtype=torch.uint8, device="cuda")
+    monkeypatch.setenv("COTT_WAIT_LIMIT_MS", "20")
+    monkeypatch.setenv("COTT_DEBUG_DROP_COMMIT", "1")
+    cott.fwd(q, k, v, m, causal=True, workspace=ws)
+    assert cott.cott.last_async_status(ws) == -5                 # COTT_ERR_TIMEOUT
+    words = ws[:12].view(torch.int32).cpu().numpy().view(np.uint32)
+    assert words[0] == 1 and (words[1] >> 31) == 1               # where the first wait gave up
+    assert ((words[1] >> 4) & 0x3FF) < 384                       # a barrier of the kernel's block
+    monkeypatch.delenv("COTT_DEBUG_DROP_COMMIT")
+    monkeypatch.delenv("COTT_WAIT_LIMIT_MS")
+    o = cott.fwd(q, k, v, m, causal=True, workspace=ws)
+    assert cott.cott.last_async_status(ws) == 0
+    gate(o, oracle.fwd_quadratic(c["q"], c["k"], c["v"], c["m"], None, True), torch.bfloat16)
