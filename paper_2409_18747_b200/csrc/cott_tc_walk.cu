@@ -70,23 +70,37 @@ constexpr int kWorkers = kWorkerWarps * 32;
 constexpr int kGroupThreads = kWorkers / 2;           // the workers act as two groups of eight warps
 
 #ifdef COTT_TIMING
-// Debug build only (d = 64): SM-clock timestamps of CTA 0 for chunks 2 and 3 -- 7 slots per
-// chunk for thread 0 (group P), the control thread and thread 256 (group O) -- kept in shared
-// memory and written behind the status word of the workspace header when the kernel ends.
-#define COTT_STAMP(slot)                                                              \
-    do {                                                                              \
-        if (D == 64 && STREAM == COTT_STAMP_STREAM && blockIdx.x == 0 && (c == 2 || c == 3) && \
-            (threadIdx.x == 0 || threadIdx.x == kWorkers || threadIdx.x == 256))      \
-            stamps[(threadIdx.x == kWorkers ? 14 : (threadIdx.x == 256 ? 28 : 0)) + (c - 2) * 7 + (slot)] = clock64(); \
-    } while (0)
-constexpr int kStampBytes = 384;
+// Debug build only: SM-clock timestamps of one CTA of the causal walk of one output stream,
+// chunks kStampC0 .. kStampC0 + 3, eight slots per chunk for each of five roles (0 = thread 0
+// of group P, 1 = thread 256 of group O, 2 = control, 3 = state update, 4 = store thread),
+// written straight to a device array that cott_debug_stamps copies out.  Slots 5-7 of role 0 in
+// the first stamped chunk hold: kernel entry, the return of the wait for the previous kernel,
+// the end of the prologue.
 #ifndef COTT_STAMP_STREAM
 #define COTT_STAMP_STREAM 0   // which output stream's walk is stamped (0 forward, 1 dQ, 2 dK, 3 dV)
 #endif
-#else
-#define COTT_STAMP(slot) do {} while (0)
-constexpr int kStampBytes = 0;
+#ifndef COTT_STAMP_CTA
+#define COTT_STAMP_CTA 0
 #endif
+#ifndef COTT_STAMP_D
+#define COTT_STAMP_D 64
+#endif
+#ifndef COTT_STAMP_C0
+#define COTT_STAMP_C0 4
+#endif
+constexpr int kStampC0 = COTT_STAMP_C0;
+__device__ long long g_cott_stamps[5 * 4 * 8];
+#define COTT_STAMP_AT(role, cc, slot)                                                          \
+    do {                                                                                       \
+        if (D == COTT_STAMP_D && MODE == MODE_CAUSAL && STREAM == COTT_STAMP_STREAM &&         \
+            blockIdx.x == COTT_STAMP_CTA && (cc) >= kStampC0 && (cc) < kStampC0 + 4 &&         \
+            ((role) == 0 ? threadIdx.x == 0 : (role) == 1 ? threadIdx.x == 256 : true))        \
+            g_cott_stamps[((role) * 4 + ((cc) - kStampC0)) * 8 + (slot)] = clock64();          \
+    } while (0)
+#else
+#define COTT_STAMP_AT(role, cc, slot) do {} while (0)
+#endif
+constexpr int kStampBytes = 0;
 
 // Shared-memory plan.  A stage holds the tiles one chunk needs from TMA: (A, Bv) for the
 // state-only pass, (X, A, Bv) for the causal walk, (X) for the read-out.
@@ -108,13 +122,20 @@ template <int D, int MODE> struct Smem {
     static constexpr int kSbBufs = (MODE == MODE_CAUSAL && D == 64) ? 2 : 1;
     static constexpr int kSb = (MODE == MODE_STATE) ? 0 : D * D * 2 * kSbBufs;
     static constexpr int kOffSb = kStages * kStage;
-    static constexpr int kOffPt = kOffSb + kSb;
-    static constexpr int kPt = 0;   // the masked scores live in tensor memory
-    static constexpr int kOffBar = kOffPt + kPt;          // mbarriers, TMEM slot, abort flag
+    // Output staging.  The d = 64 causal walk has room for two buffers of its own (chunk
+    // parity): the whole stage of chunk c can then be refilled as soon as the chunk's last MMA
+    // has read it, instead of after its epilogue and output store -- with a ring of three
+    // stages the refill latency, not the arithmetic, sets the pace of the walk.  Every other
+    // case stages the output in a slot of the chunk's stage that is dead by then.
+    static constexpr int kOutBufs = (MODE == MODE_CAUSAL && D == 64) ? 2 : 0;
+    static constexpr int kOffOutBuf = kOffSb + kSb;
+    static constexpr int kOffBar = kOffOutBuf + kOutBufs * kTile;   // mbarriers, TMEM slot, abort flag
     // Row scales of X wait in rx[kRx][128] from the norm phase of a chunk to its output
     // epilogue; three buffers are needed because X and A of chunk c+2 can land (and be
     // normalised) before every worker has finished the epilogue of chunk c.
-    static constexpr int kRx = kStages < 3 ? 3 : kStages;
+    // (Four in the d = 64 causal walk, where group P may compute the scale of chunk c + 1
+    // while group O has not yet begun the epilogue of chunk c - 2.)
+    static constexpr int kRx = (MODE == MODE_CAUSAL && D == 64) ? 4 : (kStages < 3 ? 3 : kStages);
     static constexpr int kBarBytes = 384;                 // mbarriers, TMEM slot, abort flag
     static constexpr int kOffRx = kOffBar + kBarBytes;    // rx[kRx][128] floats, dm scratch
     static constexpr int kCtlBytes = kBarBytes + kRx * 512 + 64 + (D == 64 ? kStampBytes : 0);
@@ -139,37 +160,45 @@ template <int D, int MODE> struct Smem {
 template <int D>
 __device__ __forceinline__ void issue_p(uint32_t tP, uint32_t x, uint32_t a) {
     constexpr uint32_t idesc = instr_desc_bf16(128, 128, false, false);
+    constexpr uint32_t hi = smem_desc_hi(1024);
+    const uint32_t xl = smem_desc_lo(x, 16), al = smem_desc_lo(a, 16);
 #pragma unroll
     for (int kk = 0; kk < D / 16; ++kk) {
-        const uint32_t off = (kk >> 2) * 16384u + (kk & 3) * 32u;
-        mma_ss(tP, smem_desc(x + off, 16, 1024), smem_desc(a + off, 16, 1024), idesc, kk > 0);
+        const uint32_t off = ((kk >> 2) * 16384u + (kk & 3) * 32u) >> 4;
+        mma_ss_w(tP, xl + off, hi, al + off, hi, idesc, kk > 0);
     }
 }
 template <int D>
 __device__ __forceinline__ void issue_xs(uint32_t tO, uint32_t x, uint32_t sb) {
     constexpr uint32_t idesc = instr_desc_bf16(128, D, false, true);
+    constexpr uint32_t hi = smem_desc_hi(1024);
+    const uint32_t xl = smem_desc_lo(x, 16), sl = smem_desc_lo(sb, D * 128u);
 #pragma unroll
     for (int kk = 0; kk < D / 16; ++kk) {
-        const uint32_t off = (kk >> 2) * 16384u + (kk & 3) * 32u;
-        mma_ss(tO, smem_desc(x + off, 16, 1024), smem_desc(sb + kk * 2048u, D * 128u, 1024), idesc,
-               kk > 0);
+        const uint32_t off = ((kk >> 2) * 16384u + (kk & 3) * 32u) >> 4;
+        mma_ss_w(tO, xl + off, hi, sl + kk * 128u, hi, idesc, kk > 0);
     }
 }
 template <int D>
 __device__ __forceinline__ void issue_pb(uint32_t tO, uint32_t tPt, uint32_t bv, bool acc_first) {
     // P~ (bf16, packed two per column) is the A operand in tensor memory: 8 columns per K = 16.
     constexpr uint32_t idesc = instr_desc_bf16(128, D, false, true);
+    constexpr uint32_t hi = smem_desc_hi(1024);
+    const uint32_t bl = smem_desc_lo(bv, 16384);
+    mma_ts_w(tO, tPt, bl, hi, idesc, acc_first);
 #pragma unroll
-    for (int kk = 0; kk < kChunk / 16; ++kk)
-        mma_ts(tO, tPt + kk * 8u, smem_desc(bv + kk * 2048u, 16384, 1024), idesc, (kk > 0) || acc_first);
+    for (int kk = 1; kk < kChunk / 16; ++kk)
+        mma_ts_w(tO, tPt + kk * 8u, bl + kk * 128u, hi, idesc, 1u);
 }
 template <int D>
 __device__ __forceinline__ void issue_atb(uint32_t tS, uint32_t a, uint32_t bv, bool acc_first) {
     constexpr uint32_t idesc = instr_desc_bf16(D, D, true, true);
+    constexpr uint32_t hi = smem_desc_hi(1024);
+    const uint32_t al = smem_desc_lo(a, 16384), bl = smem_desc_lo(bv, 16384);
+    mma_ss_w(tS, al, hi, bl, hi, idesc, acc_first);
 #pragma unroll
-    for (int kk = 0; kk < kChunk / 16; ++kk)
-        mma_ss(tS, smem_desc(a + kk * 2048u, 16384, 1024), smem_desc(bv + kk * 2048u, 16384, 1024),
-               idesc, (kk > 0) || acc_first);
+    for (int kk = 1; kk < kChunk / 16; ++kk)
+        mma_ss_w(tS, al + kk * 128u, hi, bl + kk * 128u, hi, idesc, 1u);
 }
 
 // Bounded wait that also gives up as soon as any thread of the CTA has given up.
@@ -242,9 +271,13 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     constexpr int NST = L::kStages;
     constexpr int NH = D / 64;                       // 64-column half tiles per row
     constexpr uint32_t kTmemCols = 512;
-    // Columns: State d | P 128 (fp32 scores) | P~ 64 (bf16 masked scores, packed) | Out.
-    // d = 64 double-buffers Out; at d = 128 one Out buffer is used (448 of the 512 columns).
-    constexpr uint32_t colS = 0, colP = D, colPt = D + 128, colO0 = D + 192;
+    // Columns: State d | P 128 (fp32 scores) | P~ 64 (bf16 masked scores, packed) | Out | P~.
+    // d = 64 double-buffers Out.  P~ has two buffers (chunk parity; the second one takes the
+    // last 64 columns): the scores of chunk c + 1 may be issued ahead of P~ Bv of chunk c, so
+    // the mask of chunk c + 1 can finish while that product still reads P~ of chunk c.
+    constexpr uint32_t colS = 0, colP = D, colPt0 = D + 128, colPt1 = 448, colO0 = D + 192;
+    static_assert(D + 192 + (D == 64 ? 2 : 1) * D <= 448, "tensor-memory columns overlap");
+    auto colPt = [&](int c) { return (c & 1) ? colPt1 : colPt0; };
     constexpr int kOBufs = (D == 64) ? 2 : 1;
     constexpr int QW = D / 4;                        // accumulator columns per worker thread
     extern __shared__ uint8_t smem_raw[];
@@ -261,11 +294,12 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     const uint32_t bar_sb_ready = bars + 96;   // [2]   bf16 state copy written (all workers); the second one sits at bars + 240
     const uint32_t bar_o_full = bars + 288;    // [4]   output accumulator complete (commit)
     const uint32_t bar_o_free = bars + 120;    // [2]   output accumulator drained (all workers)
-    const uint32_t bar_proj = bars + 136;      //       epilogue tile landed
+    const uint32_t bar_proj = bars + 136;      // [2]   epilogue tile landed (second one only with two tile buffers)
     const uint32_t bar_e_done = bars + 320;    // [4]   output rows of the chunk staged (all workers)
     const uint32_t bar_xch = bars + 160;       //       per-row partial sums exchanged (all workers)
     const uint32_t bar_full_b = bars + 168;    // [NST] causal walk: Bv landed (it is loaded last and needed last)
     const uint32_t bar_b_ready = bars + 200;   // [NST] causal walk: Bv normalised, when it is the one (all workers)
+    const uint32_t bar_out_free = bars + 352;  // [2]   own output buffers: the store of the chunk has read its buffer
     const uint32_t tmem_slot = bars + 232;
     volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(gbase + L::kOffBar + 232);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + L::kOffBar + 236);
@@ -287,11 +321,9 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     constexpr int NRX = L::kRx;
     float* rx_buf = reinterpret_cast<float*>(gbase + L::kOffRx);                 // [NRX][128]
     float* dm_red = reinterpret_cast<float*>(gbase + L::kOffRx + NRX * 512);     // [16]
-#ifdef COTT_TIMING
-    long long* stamps = reinterpret_cast<long long*>(gbase + L::kOffRx + NRX * 512 + 64);
-#endif
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    COTT_STAMP_AT(0, kStampC0, 5);
     const int g = p.first_group + blockIdx.x % p.grid_groups, bh = blockIdx.x / p.grid_groups;
     const int b = bh / p.H, h = bh % p.H;
     const int tok0 = g * p.group;
@@ -320,8 +352,9 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         mbar_init(bar_pt_ready, kGroupThreads); mbar_init(bar_sb_ready, kGroupThreads);
         mbar_init(bars + 240, kGroupThreads);
         mbar_init(bar_o_free, kGroupThreads); mbar_init(bar_o_free + 8, kGroupThreads);
-        mbar_init(bar_proj, 1);
+        mbar_init(bar_proj, 1); mbar_init(bar_proj + 8, 1);
         mbar_init(bar_xch, kGroupThreads);
+        mbar_init(bar_out_free, 1); mbar_init(bar_out_free + 8, 1);
         *abort_flag = 0;
         abort_flag[3] = p.wait_limit_kcycles;
         mbar_fence_init();
@@ -386,9 +419,12 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     // stage once the state update has read it (d = 128 causal walk, control thread), else into
     // a buffer of its own once the previous chunk's epilogue is done (store thread).
     auto load_proj = [&](int c) {
-        const uint32_t proj_u = L::kProjInA ? stage_a(c % NST) : base + L::kOffProj;
-        mbar_expect_tx(bar_proj, L::kTile);
-        load_tile(proj_u, &tmP, bar_proj, chunk_row(c));
+        constexpr bool two = L::kOutBufs > 0 && !L::kProjInA;   // two tile buffers (see below)
+        const uint32_t proj_u = L::kProjInA ? stage_a(c % NST)
+                                            : base + ((two && (c & 1)) ? L::kOffOutBuf + L::kTile : L::kOffProj);
+        const uint32_t pbar = two ? bar_proj + 8 * (c & 1) : bar_proj;
+        mbar_expect_tx(pbar, L::kTile);
+        load_tile(proj_u, &tmP, pbar, chunk_row(c));
     };
     // Every kernel but the first of a library call follows a kernel of the same call, which
     // writes none of the tensors loaded here: its first tiles are requested before the wait
@@ -399,6 +435,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     // Everything above touched only this CTA's own resources.  From here on global memory
     // written by the previous kernel of the stream is read (and its inputs overwritten).
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    COTT_STAMP_AT(0, kStampC0, 6);
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (p.clear_status && blockIdx.x == 0 && tid < 8) p.status[tid] = 0;   // status words and the dm counter
     // The first kernel of a call may follow a kernel that produced its inputs: its first tiles
@@ -479,11 +516,32 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     tc_fence_after();
 
     float dm_acc = 0.f;
+    COTT_STAMP_AT(0, kStampC0, 7);
 
     // The stage of chunk c is refilled with chunk c + NST by the store thread, in two steps
     // when possible: X and A as soon as the last MMAs that read the stage have completed, Bv
     // -- the output staging slot -- after the chunk's output store has drained.
     constexpr bool split_refill = MODE == MODE_CAUSAL && !(with_proj && L::kProjInA);
+    constexpr bool own_out = L::kOutBufs > 0;     // output staged outside the stage ring
+    // Gradient epilogues of that walk: one output buffer, and the other 16 KB hold a second
+    // buffer for the raw rows, so that the rows of chunk c + 2 are requested when the epilogue
+    // of chunk c is done and their latency is not part of any epilogue.
+    constexpr bool proj2 = own_out && with_proj && !L::kProjInA;
+    constexpr bool out_pair = own_out && !proj2;  // two output buffers (chunk parity)
+    // Which worker group normalises the contraction-side tile / computes the X row scales in
+    // the d = 64 causal walk.  Group O is the busy one (it has the epilogue), so: the forward
+    // walk gives the X scales to group P; the gradient walks, whose epilogues are longer and
+    // whose scores leave group P idle most of the time, give it the tile.
+    constexpr bool kTileNormInP = own_out && STREAM != S_FWD;
+    constexpr bool kXScaleInP = own_out && STREAM == S_FWD;
+    // Where the normalised operand is Bv (dQ^ and dK^ streams) the scores need only the raw X
+    // and A tiles: they are issued as soon as the tiles have landed, and the normalisation is
+    // waited for before P~ Bv and the state update.
+    constexpr bool kScoresOnFull = own_out && kNormBv;
+    auto proj_bar = [&](int c) { return proj2 ? bar_proj + 8 * (c & 1) : bar_proj; };
+    auto proj_par = [&](int c) { return (uint32_t)((proj2 ? (c >> 1) : c) & 1); };
+    auto proj_off = [&](int c) { return (proj2 && (c & 1)) ? L::kOffOutBuf + L::kTile : L::kOffProj; };
+    auto out_off = [&](int c) { return L::kOffOutBuf + (out_pair ? (c & 1) * L::kTile : 0); };
 
     if (is_ctrl) {
         // ------------------------------------------------------------------ control thread
@@ -495,28 +553,34 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             };
             // First MMA batch of chunk c: scores, X State (needs the previous chunk's state
             // copy and a drained output buffer), state update.
-            auto batch1 = [&](int c) {
+            auto scores = [&](int c) {
                 const int s = c % NST;
-                if (!wait(bar_a_ready + 8 * s, (c / NST) & 1)) return;
+                tc_fence_after();
+                issue_p<D>(tmem + colP, stage_x(s), stage_a(s));
+                if (!(p.debug_drop_commit && c == 1)) tc_commit(bar_p_full);
+            };
+            auto batch1 = [&](int c, bool scores_issued) {
+                const int s = c % NST;
+                if (!wait((kScoresOnFull ? bar_full : bar_a_ready) + 8 * s, (c / NST) & 1)) return;
+                COTT_STAMP_AT(2, c - 1, 4);
                 const bool acc = init_state || c > 0;
-                if (MODE == MODE_CAUSAL) {
-                    // Scores first: they need neither the state copy nor the output buffer.
-                    tc_fence_after();
-                    issue_p<D>(tmem + colP, stage_x(s), stage_a(s));
-                    if (!(p.debug_drop_commit && c == 1)) tc_commit(bar_p_full);
-                }
+                // Scores first: they need neither the state copy nor the output buffer.
+                if (MODE == MODE_CAUSAL && !scores_issued) scores(c);
                 if (MODE != MODE_STATE) {
                     if (MODE == MODE_CAUSAL && c >= 1 && !wait(sb_bar(c - 1), sb_par(c - 1))) return;
+                    COTT_STAMP_AT(2, c - 1, 5);
                     // The output accumulator this chunk writes must have been drained: by chunk
                     // c - 2 with two buffers, by chunk c - 1 with one.
                     if (kOBufs == 2) { if (c >= 2 && !wait(bar_o_free + 8 * (c & 1), ((c >> 1) & 1) ^ 1)) return; }
                     else if (c >= 1 && !wait(bar_o_free + 8 * ((c - 1) & 1), ((c - 1) >> 1) & 1)) return;
                 }
                 tc_fence_after();
+                COTT_STAMP_AT(2, c - 1, 6);
                 const uint32_t tO = tmem + colO0 + (c % kOBufs) * D;
                 if (MODE == MODE_CAUSAL) {
                     // (The state update of the chunk is issued by the state-update thread.)
                     if (acc) issue_xs<D>(tO, stage_x(s), sb + sb_off(c));
+                    COTT_STAMP_AT(2, c - 1, 7);
                 } else if (MODE == MODE_STATE) {
                     issue_atb<D>(tmem + colS, stage_a(s), stage_b(s), acc);
                     tc_commit(sfull_bar(c));
@@ -525,34 +589,44 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     tc_commit(ofull_bar(c));
                 }
             };
-            batch1(0);
+            batch1(0, false);
             for (int c = 0; c < n_chunks && alive; ++c) {
                 const int s = c % NST;
-                COTT_STAMP(0);
+                bool next_scores = false;
+                COTT_STAMP_AT(2, c, 0);
                 if (MODE == MODE_CAUSAL) {
                     if (!wait(bar_pt_ready, c & 1)) break;
+                    COTT_STAMP_AT(2, c, 1);
+                    // The masked scores of chunk c have left the score columns.  If the next
+                    // chunk's tiles are ready its scores go in ahead of P~ Bv of this one: the
+                    // mask of the next chunk, not the epilogue of this one, waits on the tensor
+                    // core here.
+                    if (c + 1 < n_chunks &&
+                        mbar_try_wait((kScoresOnFull ? bar_full : bar_a_ready) + 8 * ((c + 1) % NST),
+                                      ((c + 1) / NST) & 1)) {
+                        scores(c + 1);
+                        next_scores = true;
+                    }
+                    COTT_STAMP_AT(2, c, 2);
                     // Bv is needed from here on: landed, and normalised if it is the operand
                     // whose row scale sits on the contraction index.
                     if (L::kSplitB) {
                         if (!wait(bar_full_b + 8 * s, (c / NST) & 1)) break;
                         if (kNormBv && !wait(bar_b_ready + 8 * s, (c / NST) & 1)) break;
                     }
-                    COTT_STAMP(1);
+                    if (kScoresOnFull && !wait(bar_a_ready + 8 * s, (c / NST) & 1)) break;
                     tc_fence_after();
                     const bool acc = init_state || c > 0;
-                    issue_pb<D>(tmem + colO0 + (c % kOBufs) * D, tmem + colPt, stage_b(s), acc);
+                    issue_pb<D>(tmem + colO0 + (c % kOBufs) * D, tmem + colPt(c), stage_b(s), acc);
                     tc_commit(ofull_bar(c));
-                    COTT_STAMP(2);
+                    COTT_STAMP_AT(2, c, 3);
                     if (with_proj && L::kProjInA) {
                         // The A slot is free once the state update has read it.
                         if (!wait(sfull_bar(c), sfull_par(c))) break;
                         load_proj(c);
                     }
                 }
-                COTT_STAMP(3);
-                COTT_STAMP(4);
-                if (c + 1 < n_chunks) { batch1(c + 1); if (!alive) break; }
-                COTT_STAMP(6);
+                if (c + 1 < n_chunks) { batch1(c + 1, next_scores); if (!alive) break; }
             }
         }
     } else if (is_upd) {
@@ -563,19 +637,24 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         if (lane == 0 && MODE == MODE_CAUSAL) {
             for (int c = 0; c < n_chunks; ++c) {
                 const int s = c % NST;
+                COTT_STAMP_AT(3, c, 0);
                 if (!wait_or_abort(bar_a_ready + 8 * s, (c / NST) & 1, abort_flag)) break;
+                COTT_STAMP_AT(3, c, 1);
                 if (L::kSplitB) {
                     if (!wait_or_abort(bar_full_b + 8 * s, (c / NST) & 1, abort_flag)) break;
                     if (kNormBv && !wait_or_abort(bar_b_ready + 8 * s, (c / NST) & 1, abort_flag)) break;
                 }
                 // the workers have read the fp32 state of the previous chunk
                 if (c >= 1 && !wait_or_abort(sb_bar(c - 1), sb_par(c - 1), abort_flag)) break;
+                COTT_STAMP_AT(3, c, 2);
                 // Nothing else ties this thread to group O: stay within two chunks of its
                 // epilogue, so that the ring of state-update barriers cannot lap it.
                 if (c >= 2 && !wait_or_abort(edone_bar(c - 2), edone_par(c - 2), abort_flag)) break;
+                COTT_STAMP_AT(3, c, 3);
                 tc_fence_after();
                 issue_atb<D>(tmem + colS, stage_a(s), stage_b(s), init_state || c > 0);
                 tc_commit(sfull_bar(c));
+                COTT_STAMP_AT(3, c, 4);
             }
         }
     } else if (is_store) {
@@ -585,10 +664,14 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         // wait for a store's shared-memory read would stall the MMA issue.
         if (lane == 0) {
             bool alive = n_chunks > 0;
-            if (alive && with_proj && !L::kProjInA) load_proj(0);
+            if (alive && with_proj && !L::kProjInA) {
+                load_proj(0);
+                if (proj2 && n_chunks > 1) load_proj(1);
+            }
             for (int c = 0; c < n_chunks && alive; ++c) {
                 const int s = c % NST;
                 const bool more = c + NST < n_chunks;
+                COTT_STAMP_AT(4, c, 0);
                 // X and A (everything in the state-only pass) as soon as the chunk's last MMA,
                 // the state update, has completed.
                 if ((MODE == MODE_STATE || split_refill) && more) {
@@ -596,20 +679,35 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     // (causal walk: the other MMAs of the chunk come from another thread)
                     if (MODE == MODE_CAUSAL &&
                         !wait_or_abort(ofull_bar(c), ofull_par(c), abort_flag)) { alive = false; break; }
-                    issue_loads(c + NST, true, MODE == MODE_STATE);
+                    COTT_STAMP_AT(4, c, 1);
+                    issue_loads(c + NST, true, MODE == MODE_STATE || own_out);
+                    COTT_STAMP_AT(4, c, 2);
                 }
                 if (MODE == MODE_STATE) continue;
                 if (!wait_or_abort(edone_bar(c), edone_par(c), abort_flag)) { alive = false; break; }
-                if (with_proj && !L::kProjInA && c + 1 < n_chunks) load_proj(c + 1);   // its buffer is free now
-                const uint32_t src = base + s * L::kStage + L::kOffOut;
+                COTT_STAMP_AT(4, c, 3);
+                if (with_proj && !L::kProjInA) {                // the tile buffer of chunk c is free now
+                    if (proj2) { if (c + 2 < n_chunks) load_proj(c + 2); }
+                    else if (c + 1 < n_chunks) load_proj(c + 1);
+                }
+                const uint32_t src = own_out ? base + out_off(c) : base + s * L::kStage + L::kOffOut;
 #pragma unroll
                 for (int hh = 0; hh < NH; ++hh)
                     tma_store_3d(&tmO, src + hh * 16384, hh * 64, chunk_row(c), bh);
                 tma_store_commit();
-                if (more) {
+                COTT_STAMP_AT(4, c, 4);
+                if (out_pair) {
+                    // The previous chunk's store has read its buffer: the epilogue of the
+                    // chunk after this one may fill it again.
+                    if (c >= 1) { tma_store_wait_read1(); mbar_arrive(bar_out_free + 8 * ((c - 1) & 1)); }
+                } else if (own_out) {
+                    tma_store_wait_read0();                      // one buffer: the next epilogue waits for this
+                    mbar_arrive(bar_out_free);
+                } else if (more) {
                     tma_store_wait_read0();
                     issue_loads(c + NST, !split_refill, true);
                 }
+                COTT_STAMP_AT(4, c, 5);
             }
             if (MODE != MODE_STATE) tma_store_wait_all0();
         }
@@ -661,30 +759,36 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             }
             fence_proxy_async();
         };
-        // Row norms of chunk c: the contraction-side operand is normalised in place; the X
-        // row scale (times c) is left in rx_buf[c % NRX] for the output epilogue.
-        auto norm_phase = [&](int c) {
+        // Row norms of chunk c, in two parts that either worker group can run: the
+        // contraction-side operand is normalised in place (the scores wait for this part); the
+        // X row scale (times c) is left in rx_buf[c % NRX] for the output epilogue.
+        auto norm_tile = [&](int c) {
             const int s = c % NST;
             if (!wait(bar_full + 8 * s, (c / NST) & 1)) return;
-            uint8_t* st = gbase + s * L::kStage;
-            if (L::kHasX) {
-                float rx = cfac;
-                if (kXNorm) {
-                    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll
-                    for (int j = 0; j < NC; j += 2) {
-                        sumsq8(*reinterpret_cast<const uint4*>(tile_h_ptr(st + L::kOffX, j)), a0, a1);
-                        sumsq8(*reinterpret_cast<const uint4*>(tile_h_ptr(st + L::kOffX, j + 1)), a2, a3);
-                    }
-                    rx = cfac / fmaxf(sqrtf(pair_sum((a0 + a1) + (a2 + a3))), kEps);
-                }
-                if (nhalf == 0) rx_buf[(c % NRX) * 128 + nrow] = rx;
-            }
+            COTT_STAMP_AT(1, c - 1, 7);
             // In the split causal walk Bv arrives on its own barrier and is normalised later.
             if (L::kHasAB && !(L::kSplitB && kNormBv))
-                normalise_half_row(st + (kNormBv ? L::kOffB : L::kOffA));
+                normalise_half_row(gbase + s * L::kStage + (kNormBv ? L::kOffB : L::kOffA));
             mbar_arrive(bar_a_ready + 8 * s);
         };
+        auto x_scale = [&](int c) {
+            if (!L::kHasX) return;
+            const int s = c % NST;
+            float rx = cfac;
+            if (kXNorm) {
+                if (!wait(bar_full + 8 * s, (c / NST) & 1)) return;
+                const uint8_t* xt = gbase + s * L::kStage + L::kOffX;
+                float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+                for (int j = 0; j < NC; j += 2) {
+                    sumsq8(*reinterpret_cast<const uint4*>(tile_h_ptr(const_cast<uint8_t*>(xt), j)), a0, a1);
+                    sumsq8(*reinterpret_cast<const uint4*>(tile_h_ptr(const_cast<uint8_t*>(xt), j + 1)), a2, a3);
+                }
+                rx = cfac / fmaxf(sqrtf(pair_sum((a0 + a1) + (a2 + a3))), kEps);
+            }
+            if (nhalf == 0) rx_buf[(c % NRX) * 128 + nrow] = rx;
+        };
+        auto norm_phase = [&](int c) { norm_tile(c); if (alive) x_scale(c); };
         // Split causal walk, Bv is the normalised operand (dQ^ and dK^ streams).
         auto norm_b = [&](int c) {
             const int s = c % NST;
@@ -712,15 +816,17 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             if (alive) wait(sfull_bar(n_chunks - 1), sfull_par(n_chunks - 1));
         } else if (grp == 0) {
             // -------------------------------------------------------------- group P
+            if (kTileNormInP) norm_tile(0);
+            if (kXScaleInP) x_scale(0);
             for (int c = 0; MODE == MODE_CAUSAL && c < n_chunks && alive; ++c) {
                 // Masked scores -> bf16 operand P~ in tensor memory.  Forward: row i keeps
                 // columns j <= i (diagonal kept, Eq. 6); backward in time: j >= i.  Per
                 // 32 x 32 block (row block q, column block cb) the mask is all-keep, all-zero
                 // or, on the diagonal, a triangle; the first two cases are warp-uniform.
-                COTT_STAMP(0);
+                COTT_STAMP_AT(0, c, 0);
                 if (!wait(bar_p_full, c & 1)) break;
                 tc_fence_after();
-                COTT_STAMP(1);
+                COTT_STAMP_AT(0, c, 1);
 #pragma unroll 1
                 for (int sbk = 0; sbk < 2; ++sbk) {
                     const int cb = 2 * hf + sbk;
@@ -747,18 +853,21 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
                         pk[j] = pack_bf16(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
-                    tmem_st16(tmem + lane_base + colPt + cb * 16, pk);
+                    tmem_st16(tmem + lane_base + colPt(c) + cb * 16, pk);
                 }
                 tmem_wait_st();
-                COTT_STAMP(2);
+                COTT_STAMP_AT(0, c, 2);
                 tc_fence_before();
                 mbar_arrive(bar_pt_ready);
+                // The next chunk's scores wait for its normalised tile: before the state copy.
+                if (kTileNormInP && c + 1 < n_chunks) { norm_tile(c + 1); if (!alive) break; }
                 // bf16 copy of the updated state for the next chunk's X State product.
                 if (c + 1 < n_chunks) {
                     if (!wait(sfull_bar(c), sfull_par(c))) break;
                     // A single copy is still being read by this chunk's X State product.
                     if (L::kSbBufs == 1 && !wait(ofull_bar(c), ofull_par(c))) break;
                     tc_fence_after();
+                    COTT_STAMP_AT(0, c, 3);
 #pragma unroll 1
                     for (int pc = 0; pc < NPIECE; ++pc) {
                         uint32_t r[32];
@@ -769,23 +878,34 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     fence_proxy_async();
                     tc_fence_before();
                     mbar_arrive(sb_bar(c));
+                    COTT_STAMP_AT(0, c, 4);
                 }
-                COTT_STAMP(3);
+                if (kXScaleInP && c + 1 < n_chunks) { x_scale(c + 1); if (!alive) break; }
             }
         } else {
             // -------------------------------------------------------------- group O
-            norm_phase(0);
+            if (!kTileNormInP) norm_tile(0);
+            if (!kXScaleInP && alive) x_scale(0);
             if (L::kSplitB && kNormBv && alive) norm_b(0);
             for (int c = 0; c < n_chunks && alive; ++c) {
                 const int s = c % NST;
                 uint8_t* st = gbase + s * L::kStage;
-                COTT_STAMP(0);
-                if (c + 1 < n_chunks) { norm_phase(c + 1); if (!alive) break; }
-                COTT_STAMP(1);
+                COTT_STAMP_AT(1, c, 0);
+                if (c + 1 < n_chunks) {
+                    if (!kTileNormInP) norm_tile(c + 1);
+                    if (!kXScaleInP && alive) x_scale(c + 1);
+                    if (!alive) break;
+                }
+                COTT_STAMP_AT(1, c, 1);
                 // ---- output epilogue of chunk c: accumulator -> bf16 rows in the staging slot
                 if (!wait(ofull_bar(c), ofull_par(c))) break;
+                // The X scales of this chunk were written by threads of this group during the
+                // previous iteration, before their arrival on that chunk's epilogue barrier;
+                // with two output accumulators nothing else orders those writes before the
+                // read below.
+                if (own_out && !kXScaleInP && c >= 1 && !wait(edone_bar(c - 1), edone_par(c - 1))) break;
                 tc_fence_after();
-                COTT_STAMP(2);
+                COTT_STAMP_AT(1, c, 2);
                 const uint32_t tO = tmem + lane_base + colO0 + (c % kOBufs) * D + hf * HW;
                 const float rx = rx_buf[(c % NRX) * 128 + arow];
                 uint32_t r[HW];
@@ -796,13 +916,13 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 tc_fence_before();
                 mbar_arrive(bar_o_free + 8 * (c & 1));
                 float coef = 0.f, rp = 1.f;
-                const uint8_t* proj = L::kProjInA ? (st + L::kOffA) : (gbase + L::kOffProj);
+                const uint8_t* proj = L::kProjInA ? (st + L::kOffA) : (gbase + proj_off(c));
                 auto proj_chunk = [&](int i) {       // 8 raw values next to accumulator columns hf*HW + i ..
                     const int col = hf * HW + i;
                     return *reinterpret_cast<const uint4*>(proj + (col >> 6) * 16384 + swz(arow, (col & 63) >> 3));
                 };
                 if (with_proj) {
-                    if (!wait(bar_proj, c & 1)) break;
+                    if (!wait(proj_bar(c), proj_par(c))) break;
                     // Per-row <p, acc> and ||p||^2: each of the two column-half threads sums its
                     // part; the parts meet in shared memory.
                     float2* xch = reinterpret_cast<float2*>(L::kProjInA ? (st + L::kOffX)
@@ -836,10 +956,20 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 }
                 // Scale, (project,) round to bf16, stage for the TMA store.  The staging slot is
                 // the Bv slot, which the state update (issued behind P~ Bv) still reads: wait for it.
-                COTT_STAMP(3);
-                if (MODE == MODE_CAUSAL && !wait(sfull_bar(c), sfull_par(c))) break;
-                COTT_STAMP(4);
-                uint8_t* so = st + L::kOffOut;
+                COTT_STAMP_AT(1, c, 3);
+                if (own_out) {
+                    // Nothing else waits for the last state update: it must not be in flight
+                    // when the CTA gives back its tensor memory.
+                    if (c + 1 == n_chunks && !wait(sfull_bar(c), sfull_par(c))) break;
+                }
+                if (out_pair) {
+                    // own buffer of this chunk parity: the store of chunk c - 2 has read it
+                    if (c >= 2 && !wait(bar_out_free + 8 * (c & 1), ((c >> 1) & 1) ^ 1)) break;
+                } else if (own_out) {
+                    if (c >= 1 && !wait(bar_out_free, (c - 1) & 1)) break;   // the one buffer: store of chunk c - 1
+                } else if (MODE == MODE_CAUSAL && !wait(sfull_bar(c), sfull_par(c))) break;
+                COTT_STAMP_AT(1, c, 4);
+                uint8_t* so = own_out ? gbase + out_off(c) : st + L::kOffOut;
 #pragma unroll
                 for (int i = 0; i < HW; i += 8) {
                     const int col = hf * HW + i;
@@ -863,11 +993,10 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 }
                 fence_proxy_async();
                 mbar_arrive(edone_bar(c));
-                COTT_STAMP(5);
+                COTT_STAMP_AT(1, c, 5);
                 // Bv of the next chunk lands last; normalise it (when it is the one) after this
                 // chunk's epilogue, before the tensor core needs it.
                 if (L::kSplitB && kNormBv && c + 1 < n_chunks) { norm_b(c + 1); if (!alive) break; }
-                COTT_STAMP(6);
             }
         }
 
@@ -958,10 +1087,6 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             p.status[2] = (int)blockIdx.x | (MODE << 24) | (STREAM << 28);
         }
     }
-#ifdef COTT_TIMING
-    if (D == 64 && STREAM == COTT_STAMP_STREAM && MODE == MODE_CAUSAL && blockIdx.x == 0 && tid < 42)
-        reinterpret_cast<long long*>(p.status)[1 + tid] = stamps[tid];
-#endif
     if (is_ctrl) tmem_dealloc(tmem, kTmemCols);
 }
 
@@ -1098,3 +1223,10 @@ cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cuda
 }
 
 }  // namespace cott
+
+#ifdef COTT_TIMING
+// Debug build only: copies the 160 timestamps (5 roles x 4 chunks x 8 slots) to the host.
+extern "C" int cott_debug_stamps(long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, cott::g_cott_stamps, sizeof(long long) * 160);
+}
+#endif
