@@ -534,6 +534,24 @@ def test_shape_sweep_forward_backward(case):
     gate_dm(dm, rm, 1e-4 if f32 else 1e-2, dm_condition(rv, c["v"], c["m"], None), DM_COND_F32 if f32 else DM_COND_BF16)
 
 
+@pytest.mark.parametrize("N", [128, 129, 256, 257, 384, 513])
+@pytest.mark.parametrize("pair", ["1", "0"])
+def test_chunk_count_boundaries_d64(N, pair, monkeypatch):
+    """One to five chunks per walk at d = 64, where the ring of three stages, the two raw-row
+    buffers of the gradient epilogues and the output buffers start, wrap and drain: forward and
+    all gradients against the definition, with the dK and dV streams side by side and one after
+    the other."""
+    monkeypatch.setenv("COTT_PAIR", pair)
+    c = synth.make_qkv(2, 20, N, 64, torch.bfloat16, 5400 + N, with_do=True)
+    q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
+    o = cott.fwd(q, k, v, m, causal=True)
+    gate(o, oracle.fwd_quadratic(c["q"], c["k"], c["v"], c["m"], None, True), torch.bfloat16)
+    dq, dk, dv, dm = cott.bwd(q, k, v, d_o, m, causal=True)
+    rq, rk, rv, rm = oracle.bwd_quadratic(c["q"], c["k"], c["v"], c["d_o"], c["m"], None, True)
+    gate(dq, rq, torch.bfloat16); gate(dk, rk, torch.bfloat16); gate(dv, rv, torch.bfloat16)
+    gate_dm(dm, rm, 1e-2, dm_condition(rv, c["v"], c["m"], None), DM_COND_BF16)
+
+
 @pytest.mark.parametrize("dtype,d", [(torch.bfloat16, 128), (torch.bfloat16, 64), (torch.float32, 32)])
 def test_short_blocks_many_heads(dtype, d):
     """More (b,h) pairs than SMs and blocks of a few tokens (the shape of tokens between decode
