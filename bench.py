@@ -36,10 +36,10 @@ L2_FLUSH_BYTES = 256 << 20  # larger than the 126 MB L2
 # token-heads of the captured launch); keyed by (d, causal).  Missing key: no capture yet.
 #   (64, causal):  mean of the four walk launches of a C4 step, 141.4 MB / 262144 token-heads
 #                  (profiles/tc_walk_kernel_c4_d64.md)
-#   (128, causal): forward walk at B=1 H=16 N=16384, 253.4 MB / 262144 token-heads
+#   (128, causal): forward walk at B=1 H=16 N=16384, 252.5 MB / 262144 token-heads
 #                  (profiles/tc_walk_kernel_c5_n16384_d128.md); traffic grows with the number
 #                  of tokens, so the figure is scaled to the launch that was timed.
-KERNEL_DRAM_TRAFFIC = {(64, True): 539.0, (128, True): 967.0}
+KERNEL_DRAM_TRAFFIC = {(64, True): 539.0, (128, True): 963.0}
 
 
 def load_peaks():
