@@ -201,7 +201,7 @@ static cott_status run_tc_stream(TcWalkArgs t, const Plan& p, int B, int H, int 
         TcWalkArgs a = t;
         a.group = p.group / split; a.n_groups = p.n_groups * split;
         a.mode = 0; a.x = nullptr; a.proj = nullptr; a.out = nullptr; a.init = nullptr;
-        a.state_out = states; a.dm_partial = nullptr; a.epilogue = EPI_PLAIN;
+        a.state_out = states; a.dm_partial = nullptr; a.dm_out = nullptr; a.epilogue = EPI_PLAIN;
         t.clear_status = 0;              // the state pass, launched first, does it
         a.reverse = t.reverse ? 0 : 1;   // chunk order opposite to the walk's: L2 reuse of its tiles
         if (causal && !total_out) {
@@ -326,8 +326,13 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
         // dV': backward in time with (K, Q^, dO); rows scale by c / ||k||; <dV', V> for dm
         TcWalkArgs tv = t;
         tv.x = k; tv.a = q; tv.bv = d_o; tv.proj = v; tv.out = dv;
-        tv.norm_bv = 0; tv.x_norm = 1; tv.epilogue = EPI_DV; tv.reverse = 1; tv.dm_partial = dm_partial;
-        tv.dm_out = dm;                  // finalised by the last CTA of the dV' walk
+        tv.norm_bv = 0; tv.x_norm = 1; tv.epilogue = EPI_DV; tv.reverse = 1;
+        // dm: sum over rows of <dV'_j, v_j>, which equals the sum over rows of <q^_i, dQ^_i>.
+        // The causal dQ^ walk forms the latter in its projection epilogue, so it carries the
+        // sum and its last CTA finalises dm; the bidirectional read-out keeps it in the dV' stream.
+        TcWalkArgs& tdm = causal ? tq : tv;
+        tdm.dm_partial = dm_partial;
+        tdm.dm_out = dm;
         if (ss) {
             struct TagScope { ~TagScope() { g_prof_cur_tag = 0; } } tag_scope;
             // Everything that follows a cross-stream event wait is a plain launch.

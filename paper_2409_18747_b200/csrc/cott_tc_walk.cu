@@ -332,7 +332,14 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     constexpr bool kNormBv = STREAM == S_DQ || STREAM == S_DK;
     constexpr bool kXNorm = STREAM == S_FWD || STREAM == S_DV;
     constexpr bool kReverse = STREAM == S_DK || STREAM == S_DV;
-    constexpr int kEpi = STREAM == S_FWD ? EPI_PLAIN : (STREAM == S_DV ? EPI_DV : EPI_PROJ);
+    // The causal dV' walk has a plain epilogue: the sum over rows of <dV'_j, v_j> that dm needs
+    // equals the sum over rows of <q^_i, dQ^_i> (both are the sum over i >= j of
+    // (q^_i . k^_j)(dO_i . v_j)), and the dQ^ walk's projection epilogue already forms
+    // <q_i, dQ^_i> for every row, so that walk accumulates it and the dV' walk needs neither
+    // the raw v rows nor the per-row exchange.
+    constexpr bool kDmFromDq = MODE == MODE_CAUSAL;
+    constexpr int kEpi = STREAM == S_FWD ? EPI_PLAIN
+                       : (STREAM == S_DV ? (kDmFromDq ? EPI_PLAIN : EPI_DV) : EPI_PROJ);
     constexpr bool with_proj = (MODE != MODE_STATE) && (kEpi != EPI_PLAIN);
     const bool is_ctrl = warp == kWorkerWarps;
     const bool is_store = warp == kWorkerWarps + 1;
@@ -532,8 +539,8 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     // the d = 64 causal walk.  Group O is the busy one (it has the epilogue), so: the forward
     // walk gives the X scales to group P; the gradient walks, whose epilogues are longer and
     // whose scores leave group P idle most of the time, give it the tile.
-    constexpr bool kTileNormInP = own_out && STREAM != S_FWD;
-    constexpr bool kXScaleInP = own_out && STREAM == S_FWD;
+    constexpr bool kTileNormInP = own_out && kEpi != EPI_PLAIN;
+    constexpr bool kXScaleInP = own_out && kEpi == EPI_PLAIN;
     // Where the normalised operand is Bv (dQ^ and dK^ streams) the scores need only the raw X
     // and A tiles: they are issued as soon as the tiles have landed, and the normalisation is
     // waited for before P~ Bv and the state update.
@@ -950,6 +957,8 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                         const float nrm = sqrtf(ss);
                         rp = 1.0f / fmaxf(nrm, kEps);
                         coef = nrm > kEps ? dp * rx * rp * rp : 0.f;
+                        // <q^_i, dQ^_i> of the unscaled accumulator, once per row (see kDmFromDq)
+                        if (STREAM == S_DQ && kDmFromDq && hf == 0) dm_acc += dp * rp;
                     } else if (hf == 0) {
                         dm_acc += dp * rx / cfac;  // <dV', v> with dV' = (rx / c) * acc, once per row
                     }
@@ -1127,7 +1136,8 @@ bool make_tile_map(CUtensorMap* map, const void* ptr, int BH, int N, int d) {
 template <int D, int MODE, int STREAM>
 cudaError_t launch_mode(const CUtensorMap* tm, const TcWalkParams& p, int BH, cudaStream_t st) {
     auto kern = tc_walk_kernel<D, MODE, STREAM>;
-    constexpr bool with_proj = (MODE != MODE_STATE) && (STREAM != S_FWD);
+    // (the causal dV' walk has a plain epilogue, like the forward walk)
+    constexpr bool with_proj = (MODE != MODE_STATE) && (STREAM != S_FWD) && !(MODE == MODE_CAUSAL && STREAM == S_DV);
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
