@@ -1053,7 +1053,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     if (MODE != MODE_STATE && p.dm_partial != nullptr) {
         int* last_flag = reinterpret_cast<int*>(&dm_red[15]);
         if (tid == 0) {
-            // Fixed-order reduction of <dV', V> over the CTA (the first-half warps of group O hold sums).
+            // Fixed-order reduction of the CTA's dm term (the first-half warps of group O hold sums).
             if (!*abort_flag)
                 p.dm_partial[(size_t)bh * p.n_groups + g] = (dm_red[8] + dm_red[9]) + (dm_red[10] + dm_red[11]);
             *last_flag = 0;
@@ -1064,22 +1064,28 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         }
         __syncthreads();
         if (*last_flag) {
-            // Every CTA's partial sum is visible: dm_h = sum_b dc/dm(b,h) * sum_g <dV', V>_{b,h,g},
-            // dc/dm = -ln(s_b) sigma(m_h) (1 - sigma(m_h)) c_{b,h}; fixed order, so deterministic.
+            // Every CTA's partial sum is visible: dm_h = sum_b dc/dm(b,h) * sum_g T_{b,h,g}, T the
+            // sum over rows of <dV', V> (equally of <q^, dQ^>), dc/dm = -ln(s_b) sigma(m_h)
+            // (1 - sigma(m_h)) c_{b,h}; fixed order, so deterministic.
             __threadfence();
+            // One warp per head; lane l takes the (b, g) pairs l, l + 32, ... and the lanes meet
+            // in a butterfly: the loads of a head go out together instead of one after the
+            // other (this tail is the end of the last kernel of a backward call).
             const int n_b = (int)gridDim.x / (p.n_groups * p.H);
-            for (int hh = tid; hh < p.H; hh += kTcThreads) {
+            const int per = n_b * p.n_groups;
+            for (int hh = warp; hh < p.H; hh += kTcThreads / 32) {
                 const float sg = 1.0f / (1.0f + expf(-p.m[hh]));
-                float total = 0.f;
-                for (int bb = 0; bb < n_b; ++bb) {
+                float part = 0.f;
+                for (int i = lane; i < per; i += 32) {
+                    const int bb = i / p.n_groups, gg = i - bb * p.n_groups;
                     const float sb2 = p.seq_len ? p.seq_len[bb] : (p.seq_len_scalar > 0.f ? p.seq_len_scalar : (float)p.N);
                     const float ls = logf(sb2);
-                    float acc = 0.f;
-                    for (int gg = 0; gg < p.n_groups; ++gg)
-                        acc += __ldcg(&p.dm_partial[((size_t)bb * p.H + hh) * p.n_groups + gg]);
-                    total += acc * (-ls * sg * (1.0f - sg) * expf(-sg * ls));
+                    part += __ldcg(&p.dm_partial[((size_t)bb * p.H + hh) * p.n_groups + gg]) *
+                            (-ls * sg * (1.0f - sg) * expf(-sg * ls));
                 }
-                p.dm_out[hh] = total;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+                if (lane == 0) p.dm_out[hh] = part;
             }
             if (tid == 0) p.status[4] = 0;
         }
