@@ -34,12 +34,12 @@ L2_FLUSH_BYTES = 256 << 20  # larger than the 126 MB L2
 # DRAM bytes (read + write) per token-head of one causal-walk launch, from the ncu captures
 # summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum divided by the
 # token-heads of the captured launch); keyed by (d, causal).  Missing key: no capture yet.
-#   (64, causal):  mean of the four walk launches of a C4 step, 141.4 MB / 262144 token-heads
+#   (64, causal):  mean of the four walk launches of a C4 step, 131.8 MB / 262144 token-heads
 #                  (profiles/tc_walk_kernel_c4_d64.md)
 #   (128, causal): forward walk at B=1 H=16 N=16384, 252.5 MB / 262144 token-heads
 #                  (profiles/tc_walk_kernel_c5_n16384_d128.md); traffic grows with the number
 #                  of tokens, so the figure is scaled to the launch that was timed.
-KERNEL_DRAM_TRAFFIC = {(64, True): 539.0, (128, True): 963.0}
+KERNEL_DRAM_TRAFFIC = {(64, True): 503.0, (128, True): 963.0}
 
 
 def load_peaks():
@@ -489,9 +489,11 @@ def run_ours(args, w):
     plan = cott.query_plan(cott.cott.OP_BWD if w.get("bwd") else cott.cott.OP_FWD, dt_code, B, H, max(N, 1), d,
                            w["causal"]) if not w.get("decode") else {"path": 0, "group": 1, "chunk": 1}
     if walk_ms:
-        # walk launches per step: forward reads 3 tensors and writes 1; each gradient stream
-        # reads 4 (x, a, bv and the raw rows of its epilogue) and writes 1
-        per_launch = [4 * th] + ([5 * th] * 3 if w.get("bwd") else [])
+        # walk launches per step: forward reads 3 tensors and writes 1; the dQ and dK streams
+        # read 4 (x, a, bv and the raw rows of their projection epilogue) and write 1; the
+        # causal dV stream has a plain epilogue (3 in, 1 out), the bidirectional one reads the
+        # raw v rows as well
+        per_launch = [4 * th] + ([5 * th, 5 * th, (4 if w["causal"] else 5) * th] if w.get("bwd") else [])
         alg = sum(per_launch) / len(per_launch)
         dom_ms = statistics.mean(walk_ms)
         kernel = f"tc_walk_kernel<{d},{1 if w['causal'] else 2}> (tcgen05 chunk walk), mean of {len(walk_ms)} launches"
