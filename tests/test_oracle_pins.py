@@ -210,6 +210,31 @@ def test_gradient_invariants():
         assert dm[h] == pytest.approx((do[0, h] * o[0, h]).sum() * (-math.log(24.0)) * sg * (1 - sg), rel=1e-11)
 
 
+def test_dm_sum_by_query_rows_equals_sum_by_value_rows():
+    """The identity the causal tensor-core backward relies on for dm, written out with numpy:
+    with dV'_j = sum_{i>=j} (q^_i.k^_j) dO_i and dQ^_i = sum_{j<=i} (dO_i.v_j) k^_j (both without
+    the factor c), sum_j <dV'_j, v_j> = sum_i <q^_i, dQ^_i>, and dm_h of the oracle is that sum
+    times dc/dm.  Bidirectional: the same with full sums."""
+    N, d = 19, 6
+    q, k, v, do = (rnd((N, d), i) for i in (61, 62, 63, 64))
+    k[5] = 0.0                                   # a zero key row takes the clamped branch
+    qh = q / np.maximum(np.linalg.norm(q, axis=-1, keepdims=True), 1e-12)
+    kh = k / np.maximum(np.linalg.norm(k, axis=-1, keepdims=True), 1e-12)
+    for causal in (True, False):
+        mask = np.tril(np.ones((N, N))) if causal else np.ones((N, N))
+        p = (qh @ kh.T) * mask                   # [i, j]
+        dvp = p.T @ do                           # dV'
+        dqh = ((do @ v.T) * mask) @ kh           # dQ^
+        by_value_rows = (dvp * v).sum()
+        by_query_rows = (qh * dqh).sum()
+        assert by_query_rows == pytest.approx(by_value_rows, rel=1e-12)
+        m, s = np.array([0.4]), np.array([float(N)])
+        dm = oracle.bwd_quadratic(q[None, None], k[None, None], v[None, None], do[None, None], m, s, causal)[3]
+        sg = 1 / (1 + math.exp(-m[0]))
+        dcdm = -math.log(float(N)) * sg * (1 - sg) * float(N) ** (-sg)
+        assert dm[0] == pytest.approx(by_query_rows * dcdm, rel=1e-10)
+
+
 # ---------------------------------------------------------------- finite differences
 @pytest.mark.parametrize("causal", [True, False])
 def test_finite_differences(causal):
