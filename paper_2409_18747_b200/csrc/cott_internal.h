@@ -79,8 +79,10 @@ struct TcWalkArgs {
     // the workspace header (a wait that gives up writes them two seconds later at the earliest),
     // which saves a separate memset in front of every call.
     int clear_status;
-    // EPI_DV: when set, the CTA that finishes last turns the [BH, n_groups] partial sums of
-    // <dV', V> into dm[H] (fixed summation order), so no separate launch is needed.
+    // On the stream that carries the dm sum (dm_partial set: the dQ^ walk of a causal call,
+    // the dV' read-out of a bidirectional one): when set, the CTA that finishes last turns the
+    // [BH, n_groups] partial sums into dm[H] (fixed summation order), so no separate launch
+    // is needed.
     float* dm_out;
     // Causal walk of a single group: `init` is a caller's state (it contains c and is divided
     // by c on the way in), and the state after the last token goes to state_final, times c.

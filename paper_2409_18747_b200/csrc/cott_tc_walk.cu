@@ -39,8 +39,8 @@ struct TcWalkParams {
                             // states, to be summed here over the groups before (after, when
                             // time runs backward; all, for the read-out) this one
     float* state_out;       // MODE_STATE: [BH, n_groups, d*d] partial states (unscaled)
-    float* dm_partial;      // EPI_DV: [BH, n_groups]
-    float* dm_out;          // EPI_DV: dm[H], written by the CTA that finishes last (or NULL)
+    float* dm_partial;      // the stream that carries the dm sum: [BH, n_groups]
+    float* dm_out;          // that stream: dm[H], written by the CTA that finishes last (or NULL)
     int init_has_scale;     // init is a caller's state (contains c): divide by c on the way in
     float* state_final;     // causal walk, one group: [BH, d*d] state after the last token, times c (or NULL)
     int* status;            // workspace status word
@@ -60,9 +60,9 @@ enum { MODE_STATE = 0, MODE_CAUSAL = 1, MODE_READOUT = 2 };
 // walk is sensitive to instruction-cache misses: ncu showed 'no instruction' as the top stall
 // of the d = 128 causal walk when all variants shared one body).
 //   S_FWD: X rows normalised in the epilogue, A normalised in shared memory, plain store
-//   S_DQ : Bv normalised, projection epilogue
+//   S_DQ : Bv normalised, projection epilogue (the causal walk also sums <q^, dQ^> for dm)
 //   S_DK : as S_DQ, time reversed
-//   S_DV : as S_FWD, time reversed, scale + <dV', V> epilogue
+//   S_DV : as S_FWD, time reversed (the read-out form adds the <dV', V> sums for dm)
 enum { S_FWD = 0, S_DQ = 1, S_DK = 2, S_DV = 3 };
 
 constexpr int kWorkerWarps = 16;                      // row-worker warps (4 per TMEM lane quadrant)
