@@ -115,6 +115,34 @@ cott_status cott_fwd(const void* q, const void* k, const void* v, void* o, float
                      void* stream);
 
 /*
+ * Element strides of a tensor of logical shape [B,H,N,d] whose rows (the d elements of one
+ * token of one head) are contiguous: distance between consecutive batch items, heads and
+ * tokens.  Dense [B,H,N,d] is {H*N*d, N*d, d}; [B,N,H,d], the layout a projection GEMM leaves,
+ * is {N*H*d, d, H*d}; q inside a fused [B,N,3,H,d] projection output is {N*3*H*d, d, 3*H*d}
+ * (k and v start H*d and 2*H*d elements later).  Every stride must be >= d and a multiple of
+ * 16 bytes; the tensor's first element must be 16-byte aligned.
+ */
+typedef struct cott_strides {
+    long long batch;
+    long long head;
+    long long token;
+} cott_strides;
+
+/*
+ * cott_fwd on tensors that are not dense [B,H,N,d] (no transpose pass before the attention):
+ *   qkv_strides : strides shared by q, k and v (NULL: dense)
+ *   o_strides   : strides of o (NULL: dense)
+ * Everything else as for cott_fwd.  On the tensor-core path (bf16, d 64 or 128) the strides must
+ * also be expressible as a 4-D tiled tensor map (each stride a multiple of the next smaller
+ * one, as in the three layouts above); COTT_ERR_UNSUPPORTED or COTT_ERR_CUDA otherwise.
+ */
+cott_status cott_fwd_strided(const void* q, const void* k, const void* v, void* o, float* state_out,
+                             int B, int H, int N, int d, int causal, cott_dtype dt,
+                             const cott_strides* qkv_strides, const cott_strides* o_strides,
+                             const cott_scale_params* sp, void* workspace, size_t workspace_bytes,
+                             void* stream);
+
+/*
  * Causal forward over one SEGMENT of a longer sequence (chunked prefill; blocks of several
  * tokens between decode steps): the running state of Eq. 8 carried across calls.
  *   state_in  : NULL (the sequence starts here) or fp32 [B,H,d,d], the state left by the previous
@@ -152,6 +180,21 @@ cott_status cott_bwd(const void* q, const void* k, const void* v, const void* d_
                      void* dk, void* dv, float* dm, int B, int H, int N, int d, int causal,
                      cott_dtype dt, const cott_scale_params* sp, void* workspace,
                      size_t workspace_bytes, void* stream);
+
+/*
+ * cott_bwd on tensors that are not dense [B,H,N,d]:
+ *   qkv_strides  : strides shared by q, k and v (NULL: dense)
+ *   do_strides   : strides of d_o (NULL: dense)
+ *   dqkv_strides : strides shared by dq, dk and dv (NULL: dense), e.g. the three slices of a
+ *                  fused gradient buffer
+ * Everything else, and the conditions on the strides, as for cott_bwd and cott_fwd_strided.
+ */
+cott_status cott_bwd_strided(const void* q, const void* k, const void* v, const void* d_o, void* dq,
+                             void* dk, void* dv, float* dm, int B, int H, int N, int d, int causal,
+                             cott_dtype dt, const cott_strides* qkv_strides,
+                             const cott_strides* do_strides, const cott_strides* dqkv_strides,
+                             const cott_scale_params* sp, void* workspace, size_t workspace_bytes,
+                             void* stream);
 
 /*
  * One recurrent decode step, Eq. 8:  S <- S + k^ (c v)^T ;  o = S^T q^  (update, then read).

@@ -66,6 +66,12 @@ def _load():
     lib.cott_fwd.restype = ci
     lib.cott_fwd.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci,
                              ctypes.POINTER(_ScaleParams), vp, cs, vp]
+    lib.cott_fwd_strided.restype = ci
+    lib.cott_fwd_strided.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, vp, vp,
+                                     ctypes.POINTER(_ScaleParams), vp, cs, vp]
+    lib.cott_bwd_strided.restype = ci
+    lib.cott_bwd_strided.argtypes = [vp] * 8 + [ci, ci, ci, ci, ci, ci, vp, vp, vp,
+                                                 ctypes.POINTER(_ScaleParams), vp, cs, vp]
     lib.cott_fwd_stateful.restype = ci
     lib.cott_fwd_stateful.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci,
                                       ctypes.POINTER(_ScaleParams), vp, cs, vp]
@@ -102,6 +108,34 @@ def _check_dev(*ts):
             raise RuntimeError("libcott needs CUDA tensors (there is no CPU path)")
         if not t.is_contiguous():
             raise ValueError("libcott needs contiguous tensors")
+
+
+class _Strides(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_longlong), ("head", ctypes.c_longlong), ("token", ctypes.c_longlong)]
+
+
+def _check_rows(*ts):
+    """[B,H,N,d] CUDA tensors with contiguous rows; any strides over batch, head and token."""
+    for t in ts:
+        if not t.is_cuda:
+            raise RuntimeError("libcott needs CUDA tensors (there is no CPU path)")
+        if t.dim() != 4 or (t.shape[3] > 1 and t.stride(3) != 1):
+            raise ValueError("libcott needs [B,H,N,d] tensors whose last dimension is contiguous")
+
+
+def _strides_of(*ts):
+    """ctypes strides shared by the given tensors (None when they are dense [B,H,N,d])."""
+    st = tuple(ts[0].stride()[:3])
+    for t in ts[1:]:
+        if tuple(t.stride()[:3]) != st:
+            raise ValueError("tensors of one group (q,k,v / dq,dk,dv) must share their strides")
+    if all(t.is_contiguous() for t in ts):
+        return None
+    return _Strides(st[0], st[1], st[2])
+
+
+def _ref(s):
+    return ctypes.byref(s) if s is not None else None
 
 
 def _stream_ptr(stream) -> int:
@@ -142,21 +176,27 @@ def _workspace(op, dt, B, H, N, d, causal, device, workspace):
 
 def fwd(q, k, v, m, seq_len=None, causal=True, return_state=False, out=None, workspace=None,
         stream=None):
-    """cott_fwd.  ``seq_len``: None (s_b = N), a float, or a float32 ``[B]`` CUDA tensor.
-    Returns ``o`` or ``(o, state[B,H,d,d] fp32)``."""
-    _check_dev(q, k, v, m, seq_len if isinstance(seq_len, torch.Tensor) else None)
+    """cott_fwd / cott_fwd_strided.  q, k, v: ``[B,H,N,d]`` tensors with contiguous rows and
+    common strides -- dense, a ``[B,N,H,d]`` buffer seen through ``permute(0,2,1,3)``, or the
+    slices of a fused projection output; no copy is made.  ``seq_len``: None (s_b = N), a float,
+    or a float32 ``[B]`` CUDA tensor.  Returns ``o`` (laid out like q when q is dense in
+    memory, else dense ``[B,H,N,d]``; or ``out``) or ``(o, state[B,H,d,d] fp32)``."""
+    _check_rows(q, k, v)
+    _check_dev(m, seq_len if isinstance(seq_len, torch.Tensor) else None)
     B, H, N, d = q.shape
     dt = _dt(q)
     o = torch.empty_like(q) if out is None else out
+    _check_rows(o)
+    s_qkv, s_o = _strides_of(q, k, v), _strides_of(o)
     state = torch.empty((B, H, d, d), dtype=torch.float32, device=q.device) if return_state else None
     ws, ws_bytes = _workspace(OP_FWD, dt, B, H, N, d, causal, q.device, workspace)
     sp = _scale(m, seq_len)
-    rc = _load().cott_fwd(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
-                          state.data_ptr() if state is not None else None, B, H, N, d,
-                          int(bool(causal)), dt, ctypes.byref(sp), ws.data_ptr(), ws_bytes,
-                          _stream_ptr(stream))
+    rc = _load().cott_fwd_strided(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
+                                  state.data_ptr() if state is not None else None, B, H, N, d,
+                                  int(bool(causal)), dt, _ref(s_qkv), _ref(s_o), ctypes.byref(sp),
+                                  ws.data_ptr(), ws_bytes, _stream_ptr(stream))
     if rc != 0:
-        raise CottError(rc, "cott_fwd")
+        raise CottError(rc, "cott_fwd_strided")
     return (o, state) if return_state else o
 
 
@@ -200,21 +240,26 @@ def fwd_noalloc(q, k, v, m, seq_len=None, causal=True, out=None, stream=None):
     return o
 
 
-def bwd(q, k, v, d_o, m, seq_len=None, causal=True, workspace=None, stream=None):
-    """cott_bwd.  Returns ``(dq, dk, dv, dm[H] fp32)``."""
-    _check_dev(q, k, v, d_o, m, seq_len if isinstance(seq_len, torch.Tensor) else None)
+def bwd(q, k, v, d_o, m, seq_len=None, causal=True, workspace=None, stream=None, out=None):
+    """cott_bwd / cott_bwd_strided.  q, k, v (common strides) and d_o as for ``fwd``; ``out``:
+    optional ``(dq, dk, dv)`` tensors with common strides (e.g. the slices of a fused gradient
+    buffer), else they are allocated like q.  Returns ``(dq, dk, dv, dm[H] fp32)``."""
+    _check_rows(q, k, v, d_o)
+    _check_dev(m, seq_len if isinstance(seq_len, torch.Tensor) else None)
     B, H, N, d = q.shape
     dt = _dt(q)
-    dq, dk, dv = torch.empty_like(q), torch.empty_like(q), torch.empty_like(q)
+    dq, dk, dv = (torch.empty_like(q), torch.empty_like(q), torch.empty_like(q)) if out is None else out
+    _check_rows(dq, dk, dv)
+    s_qkv, s_do, s_dqkv = _strides_of(q, k, v), _strides_of(d_o), _strides_of(dq, dk, dv)
     dm = torch.empty((H,), dtype=torch.float32, device=q.device)
     ws, ws_bytes = _workspace(OP_BWD, dt, B, H, N, d, causal, q.device, workspace)
     sp = _scale(m, seq_len)
-    rc = _load().cott_bwd(q.data_ptr(), k.data_ptr(), v.data_ptr(), d_o.data_ptr(), dq.data_ptr(),
-                          dk.data_ptr(), dv.data_ptr(), dm.data_ptr(), B, H, N, d,
-                          int(bool(causal)), dt, ctypes.byref(sp), ws.data_ptr(), ws_bytes,
-                          _stream_ptr(stream))
+    rc = _load().cott_bwd_strided(q.data_ptr(), k.data_ptr(), v.data_ptr(), d_o.data_ptr(),
+                                  dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), dm.data_ptr(), B, H, N,
+                                  d, int(bool(causal)), dt, _ref(s_qkv), _ref(s_do), _ref(s_dqkv),
+                                  ctypes.byref(sp), ws.data_ptr(), ws_bytes, _stream_ptr(stream))
     if rc != 0:
-        raise CottError(rc, "cott_bwd")
+        raise CottError(rc, "cott_bwd_strided")
     return dq, dk, dv, dm
 
 

@@ -137,6 +137,32 @@ static cott_status check_scale(const cott_scale_params* sp) {
     return COTT_OK;
 }
 
+// Layouts of the tensors of one call: q, k, v share one, o (forward) / dO (backward) has one,
+// dq, dk, dv share one.  All zero: dense [B,H,N,d].
+struct CallLayouts {
+    RowLayout qkv, o, dqkv;
+    const void* q; const void* k; const void* v; const void* o_or_do;
+    RowLayout of(const void* ptr) const {
+        if (ptr == q || ptr == k || ptr == v) return qkv;
+        if (ptr == o_or_do) return o;
+        return dqkv;
+    }
+    template <class Args> void assign(Args& a) const {
+        a.lx = of(a.x); a.la = of(a.a); a.lbv = of(a.bv); a.lproj = of(a.proj);
+        a.lout = (a.out == o_or_do) ? o : dqkv;
+    }
+};
+static RowLayout to_layout(const cott_strides* s) {
+    return s ? RowLayout{s->batch, s->head, s->token} : RowLayout{0, 0, 0};
+}
+// Element strides the kernels can address: rows of d contiguous elements, 16-byte aligned.
+static bool layout_ok(const cott_strides* s, int d, cott_dtype dt) {
+    if (!s) return true;
+    const long long q = 16 / (long long)dtype_size(dt);
+    return s->batch >= d && s->head >= d && s->token >= d && s->batch % q == 0 && s->head % q == 0 &&
+           s->token % q == 0;
+}
+
 static WalkArgs base_walk(const cott_scale_params* sp, int H, int N, const Plan& p) {
     WalkArgs w;
     memset(&w, 0, sizeof(w));
@@ -230,7 +256,9 @@ static cott_status run_tc_stream(TcWalkArgs t, const Plan& p, int B, int H, int 
 static cott_status fwd_impl(const void* q, const void* k, const void* v, void* o, float* state_out,
                             int B, int H, int N, int d, int causal, cott_dtype dt,
                             const cott_scale_params* sp, void* ws, const Plan& p,
-                            cudaStream_t st, const float* state_in = nullptr) {
+                            cudaStream_t st, const float* state_in = nullptr,
+                            const cott_strides* s_qkv = nullptr, const cott_strides* s_o = nullptr) {
+    const CallLayouts lay{to_layout(s_qkv), to_layout(s_o), RowLayout{0, 0, 0}, q, k, v, o};
     // The tensor-core path clears the status words in its first kernel.
     if (p.path != 1) COTT_CUDA(cudaMemsetAsync(ws, 0, kWsHeaderBytes, st));
     float* states = reinterpret_cast<float*>(static_cast<char*>(ws) + kWsHeaderBytes);
@@ -238,6 +266,7 @@ static cott_status fwd_impl(const void* q, const void* k, const void* v, void* o
         TcWalkArgs t;
         memset(&t, 0, sizeof(t));
         t.x = q; t.a = k; t.bv = v; t.out = o;
+        lay.assign(t);
         t.norm_bv = 0; t.x_norm = 1; t.epilogue = EPI_PLAIN; t.reverse = 0;
         t.clear_status = 1;
         return run_tc_stream(t, p, B, H, N, d, causal, sp, static_cast<int*>(ws), states,
@@ -245,6 +274,7 @@ static cott_status fwd_impl(const void* q, const void* k, const void* v, void* o
     }
     WalkArgs w = base_walk(sp, H, N, p);
     w.x = q; w.a = k; w.bv = v; w.out = o;
+    lay.assign(w);
     w.mode_x = ROW_NORM; w.mode_a = ROW_NORM; w.mode_b = ROW_SCALE;
     w.epilogue = EPI_PLAIN; w.reverse = 0;
     return run_stream(w, p, B * H, d, dt, causal, states, state_out, st, state_in);
@@ -284,7 +314,9 @@ static SideStreams* side_streams() {
 static cott_status bwd_impl(const void* q, const void* k, const void* v, const void* d_o, void* dq,
                             void* dk, void* dv, float* dm, int B, int H, int N, int d, int causal,
                             cott_dtype dt, const cott_scale_params* sp, void* ws, const Plan& p,
-                            cudaStream_t st) {
+                            cudaStream_t st, const cott_strides* s_qkv = nullptr,
+                            const cott_strides* s_do = nullptr, const cott_strides* s_dqkv = nullptr) {
+    const CallLayouts lay{to_layout(s_qkv), to_layout(s_do), to_layout(s_dqkv), q, k, v, d_o};
     // The tensor-core path clears the status words in its first kernel.
     if (p.path != 1) COTT_CUDA(cudaMemsetAsync(ws, 0, kWsHeaderBytes, st));
     char* base = static_cast<char*>(ws) + kWsHeaderBytes;
@@ -330,6 +362,7 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
         // dm: sum over rows of <dV'_j, v_j>, which equals the sum over rows of <q^_i, dQ^_i>.
         // The causal dQ^ walk forms the latter in its projection epilogue, so it carries the
         // sum and its last CTA finalises dm; the bidirectional read-out keeps it in the dV' stream.
+        lay.assign(tq); lay.assign(tk); lay.assign(tv);
         TcWalkArgs& tdm = causal ? tq : tv;
         tdm.dm_partial = dm_partial;
         tdm.dm_out = dm;
@@ -373,6 +406,7 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
     {   // dQ^_t = S_t dO_t : the forward walk with (dO, V', K^) in the roles of (Q, K, V)
         WalkArgs w = base_walk(sp, H, N, p);
         w.x = d_o; w.a = v; w.bv = k; w.proj = q; w.out = dq;
+        lay.assign(w);
         w.mode_x = ROW_RAW; w.mode_a = ROW_SCALE; w.mode_b = ROW_NORM;
         w.epilogue = EPI_PROJ; w.reverse = 0;
         if ((rc = run_stream(w, p, BH, d, dt, causal, st0, nullptr, st)) != COTT_OK) return rc;
@@ -380,6 +414,7 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
     {   // dK^_j = R_j v'_j : running sum of dO_t q^_t^T accumulated backward in time
         WalkArgs w = base_walk(sp, H, N, p);
         w.x = v; w.a = d_o; w.bv = q; w.proj = k; w.out = dk;
+        lay.assign(w);
         w.mode_x = ROW_SCALE; w.mode_a = ROW_RAW; w.mode_b = ROW_NORM;
         w.epilogue = EPI_PROJ; w.reverse = 1;
         if ((rc = run_stream(w, p, BH, d, dt, causal, st1, nullptr, st)) != COTT_OK) return rc;
@@ -387,6 +422,7 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
     {   // dV'_j = R_j^T k^_j, dV = c dV', and <dV', V> for dm
         WalkArgs w = base_walk(sp, H, N, p);
         w.x = k; w.a = q; w.bv = d_o; w.proj = v; w.out = dv;
+        lay.assign(w);
         w.mode_x = ROW_NORM; w.mode_a = ROW_NORM; w.mode_b = ROW_RAW;
         w.epilogue = EPI_DV; w.reverse = 1; w.dm_partial = dm_partial;
         if ((rc = run_stream(w, p, BH, d, dt, causal, st2, nullptr, st)) != COTT_OK) return rc;
@@ -482,7 +518,17 @@ cott_status cott_fwd(const void* q, const void* k, const void* v, void* o, float
                      int B, int H, int N, int d, int causal, cott_dtype dt,
                      const cott_scale_params* sp, void* workspace, size_t workspace_bytes,
                      void* stream) {
+    return cott_fwd_strided(q, k, v, o, state_out, B, H, N, d, causal, dt, nullptr, nullptr, sp,
+                            workspace, workspace_bytes, stream);
+}
+
+cott_status cott_fwd_strided(const void* q, const void* k, const void* v, void* o, float* state_out,
+                             int B, int H, int N, int d, int causal, cott_dtype dt,
+                             const cott_strides* qkv_strides, const cott_strides* o_strides,
+                             const cott_scale_params* sp, void* workspace, size_t workspace_bytes,
+                             void* stream) {
     if (!q || !k || !v || !o || B < 1 || H < 1 || N < 1) return COTT_ERR_INVALID_ARG;
+    if (!layout_ok(qkv_strides, d, dt) || !layout_ok(o_strides, d, dt)) return COTT_ERR_UNSUPPORTED;
     if (check_scale(sp) != COTT_OK) return COTT_ERR_INVALID_ARG;
     if (o == q || o == k || o == v) return COTT_ERR_INVALID_ARG;
     if (!sp->seq_len && sp->seq_len_scalar > 0.f && sp->seq_len_scalar < 1.f)
@@ -496,7 +542,7 @@ cott_status cott_fwd(const void* q, const void* k, const void* v, void* o, float
         workspace_bytes < workspace_bytes_impl(COTT_OP_FWD, p, B, H, d))
         return COTT_ERR_WORKSPACE;
     return fwd_impl(q, k, v, o, state_out, B, H, N, d, causal, dt, sp, workspace, p,
-                    static_cast<cudaStream_t>(stream));
+                    static_cast<cudaStream_t>(stream), nullptr, qkv_strides, o_strides);
 }
 
 cott_status cott_fwd_stateful(const void* q, const void* k, const void* v, void* o,
@@ -525,8 +571,20 @@ cott_status cott_bwd(const void* q, const void* k, const void* v, const void* d_
                      void* dk, void* dv, float* dm, int B, int H, int N, int d, int causal,
                      cott_dtype dt, const cott_scale_params* sp, void* workspace,
                      size_t workspace_bytes, void* stream) {
+    return cott_bwd_strided(q, k, v, d_o, dq, dk, dv, dm, B, H, N, d, causal, dt, nullptr, nullptr,
+                            nullptr, sp, workspace, workspace_bytes, stream);
+}
+
+cott_status cott_bwd_strided(const void* q, const void* k, const void* v, const void* d_o, void* dq,
+                             void* dk, void* dv, float* dm, int B, int H, int N, int d, int causal,
+                             cott_dtype dt, const cott_strides* qkv_strides,
+                             const cott_strides* do_strides, const cott_strides* dqkv_strides,
+                             const cott_scale_params* sp, void* workspace, size_t workspace_bytes,
+                             void* stream) {
     if (!q || !k || !v || !d_o || !dq || !dk || !dv || !dm || B < 1 || H < 1 || N < 1)
         return COTT_ERR_INVALID_ARG;
+    if (!layout_ok(qkv_strides, d, dt) || !layout_ok(do_strides, d, dt) || !layout_ok(dqkv_strides, d, dt))
+        return COTT_ERR_UNSUPPORTED;
     if (check_scale(sp) != COTT_OK) return COTT_ERR_INVALID_ARG;
     const void* ins[4] = {q, k, v, d_o};
     void* outs[3] = {dq, dk, dv};
@@ -547,7 +605,7 @@ cott_status cott_bwd(const void* q, const void* k, const void* v, const void* d_
         workspace_bytes < workspace_bytes_impl(COTT_OP_BWD, p, B, H, d))
         return COTT_ERR_WORKSPACE;
     return bwd_impl(q, k, v, d_o, dq, dk, dv, dm, B, H, N, d, causal, dt, sp, workspace, p,
-                    static_cast<cudaStream_t>(stream));
+                    static_cast<cudaStream_t>(stream), qkv_strides, do_strides, dqkv_strides);
 }
 
 cott_status cott_decode_step(const void* q, const void* k, const void* v, float* state, void* o,

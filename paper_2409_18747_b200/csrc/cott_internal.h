@@ -24,6 +24,16 @@ enum Epilogue : int {
     EPI_DV = 2      // multiply by c, and accumulate <row, proj row> for dm (proj = raw v)
 };
 
+// Where the rows of a [B,H,N,d] tensor sit in memory: element strides of the batch, head and
+// token index; the d elements of a row are contiguous.  All zero means dense [B,H,N,d].
+struct RowLayout {
+    long long sb, sh, sn;
+};
+inline RowLayout resolve_layout(const RowLayout& l, int H, int N, int d) {
+    if (l.sb == 0 && l.sh == 0 && l.sn == 0) return RowLayout{(long long)H * N * d, (long long)N * d, (long long)d};
+    return l;
+}
+
 // How the scan kernel combines the per-group partial states.
 enum ScanMode : int { SCAN_PREFIX = 0, SCAN_SUFFIX = 1, SCAN_TOTAL = 2 };
 
@@ -34,6 +44,7 @@ enum ScanMode : int { SCAN_PREFIX = 0, SCAN_SUFFIX = 1, SCAN_TOTAL = 2 };
 struct WalkArgs {
     const void* x; const void* a; const void* bv; const void* proj;
     void* out;
+    RowLayout lx, la, lbv, lproj, lout;   // layouts of the five tensors (all zero: dense)
     const float* init;   // [BH, n_groups, d*d] or NULL (zero initial state)
     float* final_state;  // NULL, or [BH, n_groups, d*d] (final_grouped) / [BH, d*d] (one group)
     int final_grouped;
@@ -58,6 +69,7 @@ cudaError_t launch_scan(float* states, float* total_out, int BH, int n_groups, i
 struct TcWalkArgs {
     int mode;
     const void* x; const void* a; const void* bv; const void* proj; void* out;
+    RowLayout lx, la, lbv, lproj, lout;   // layouts of the five tensors (all zero: dense)
     const float* init; float* state_out; float* dm_partial; int* status;
     const float* m; const float* seq_len; float seq_len_scalar;
     int group; int n_groups;

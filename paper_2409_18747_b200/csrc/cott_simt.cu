@@ -54,16 +54,17 @@ __device__ __forceinline__ float warp_sum(float v) {
     return v;
 }
 
-// Stage rows [t0, t0+kTile) of one [N,D] slice as fp32; rows outside [lo,hi) become zero.
+// Stage rows [t0, t0+kTile) of one (b,h) slice (rows `sn` elements apart) as fp32; rows outside
+// [lo,hi) become zero.
 template <int D, typename T>
-__device__ __forceinline__ void stage_tile(float (*dst)[D], const T* src, int t0, int lo, int hi,
-                                           int tid) {
+__device__ __forceinline__ void stage_tile(float (*dst)[D], const T* src, long long sn, int t0, int lo,
+                                           int hi, int tid) {
     constexpr int V4 = D / 4;
     for (int i = tid; i < kTile * V4; i += kThreads) {
         int r = i / V4, c4 = i % V4;
         int t = t0 + r;
         float f[4] = {0.f, 0.f, 0.f, 0.f};
-        if (t >= lo && t < hi) load4<T>(src + (size_t)t * D + c4 * 4, f);
+        if (t >= lo && t < hi) load4<T>(src + (size_t)t * sn + c4 * 4, f);
         *reinterpret_cast<float4*>(&dst[r][c4 * 4]) = make_float4(f[0], f[1], f[2], f[3]);
     }
 }
@@ -101,12 +102,13 @@ __global__ void __launch_bounds__(kThreads) walk_kernel(WalkArgs w) {
     const int b = bh / w.H, h = bh % w.H;
     const int lo = g * w.group;
     const int hi = min(w.N, lo + w.group);
-    const size_t slice = (size_t)bh * w.N * D;
-    const T* X = static_cast<const T*>(w.x) + slice;
-    const T* A = static_cast<const T*>(w.a) + slice;
-    const T* Bv = static_cast<const T*>(w.bv) + slice;
-    const T* P = w.proj ? static_cast<const T*>(w.proj) + slice : nullptr;
-    T* O = w.out ? static_cast<T*>(w.out) + slice : nullptr;
+    // (the launcher has resolved the layouts: strides are never all zero here)
+    auto slice = [&](const RowLayout& l) { return (size_t)b * l.sb + (size_t)h * l.sh; };
+    const T* X = static_cast<const T*>(w.x) + slice(w.lx);
+    const T* A = static_cast<const T*>(w.a) + slice(w.la);
+    const T* Bv = static_cast<const T*>(w.bv) + slice(w.lbv);
+    const T* P = w.proj ? static_cast<const T*>(w.proj) + slice(w.lproj) : nullptr;
+    T* O = w.out ? static_cast<T*>(w.out) + slice(w.lout) : nullptr;
 
     const float s_b = w.seq_len ? w.seq_len[b]
                                 : (w.seq_len_scalar > 0.f ? w.seq_len_scalar : (float)w.N);
@@ -129,9 +131,9 @@ __global__ void __launch_bounds__(kThreads) walk_kernel(WalkArgs w) {
         const int tile_idx = w.reverse ? (n_tiles - 1 - it) : it;
         const int t0 = lo + tile_idx * kTile;
         __syncthreads();  // previous tile fully consumed
-        stage_tile<D, T>(xs, X, t0, lo, hi, tid);
-        stage_tile<D, T>(as, A, t0, lo, hi, tid);
-        stage_tile<D, T>(bs, Bv, t0, lo, hi, tid);
+        stage_tile<D, T>(xs, X, w.lx.sn, t0, lo, hi, tid);
+        stage_tile<D, T>(as, A, w.la.sn, t0, lo, hi, tid);
+        stage_tile<D, T>(bs, Bv, w.lbv.sn, t0, lo, hi, tid);
         __syncthreads();
         treat_rows<D>(xs, w.mode_x, c, warp, lane);
         treat_rows<D>(as, w.mode_a, c, warp, lane);
@@ -170,7 +172,7 @@ __global__ void __launch_bounds__(kThreads) walk_kernel(WalkArgs w) {
             for (int sp = 1; sp < NSPLIT; ++sp) v += part[r][sp][e];
             part[r][0][e] = v;
         }
-        if (w.epilogue != EPI_PLAIN) stage_tile<D, T>(xs, P, t0, lo, hi, tid);  // xs is dead now
+        if (w.epilogue != EPI_PLAIN) stage_tile<D, T>(xs, P, w.lproj.sn, t0, lo, hi, tid);  // xs is dead now
         __syncthreads();
         // Epilogue: one warp per row.
         for (int r = warp; r < kTile; r += kThreads / 32) {
@@ -200,7 +202,7 @@ __global__ void __launch_bounds__(kThreads) walk_kernel(WalkArgs w) {
             __syncwarp();
             for (int e4 = lane; e4 < D / 4; e4 += 32) {
                 float f[4] = {row[e4 * 4], row[e4 * 4 + 1], row[e4 * 4 + 2], row[e4 * 4 + 3]};
-                store4<T>(O + (size_t)t * D + e4 * 4, f);
+                store4<T>(O + (size_t)t * w.lout.sn + e4 * 4, f);
             }
         }
     }
@@ -403,7 +405,11 @@ cudaError_t launch_decode_t(const void* q, const void* k, const void* v, float* 
 
 }  // namespace
 
-cudaError_t launch_walk_simt(const WalkArgs& w, int BH, int d, cott_dtype dt, cudaStream_t st) {
+cudaError_t launch_walk_simt(const WalkArgs& w0, int BH, int d, cott_dtype dt, cudaStream_t st) {
+    WalkArgs w = w0;   // resolve "all zero = dense [B,H,N,d]" once, on the host
+    w.lx = resolve_layout(w0.lx, w0.H, w0.N, d); w.la = resolve_layout(w0.la, w0.H, w0.N, d);
+    w.lbv = resolve_layout(w0.lbv, w0.H, w0.N, d); w.lproj = resolve_layout(w0.lproj, w0.H, w0.N, d);
+    w.lout = resolve_layout(w0.lout, w0.H, w0.N, d);
     return dt == COTT_F32 ? launch_walk_t<float>(w, BH, d, st)
                           : launch_walk_t<__nv_bfloat16>(w, BH, d, st);
 }

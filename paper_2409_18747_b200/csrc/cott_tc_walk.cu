@@ -51,6 +51,8 @@ struct TcWalkParams {
     int clear_status;                   // first kernel of a call: CTA 0 zeroes the status words
     int wait_limit_kcycles;             // bound of every wait, in units of 1024 SM cycles
     int debug_drop_commit;              // test hook: the scores of chunk 1 are never reported complete
+    int head_first_mask;                // bit i: in tensor map i (X, A, Bv, raw rows, Out) the head index
+                                        // comes before the token index (its stride is the smaller one)
 };
 
 enum { MODE_STATE = 0, MODE_CAUSAL = 1, MODE_READOUT = 2 };
@@ -385,9 +387,13 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     auto chunk_row = [&](int c) { return tok0 + (backward ? (n_chunks - 1 - c) : c) * kChunk; };
 
     // TMA loads (issued by single threads of the control and the store warp).
-    auto load_tile = [&](uint32_t dst, const CUtensorMap* tm, uint32_t bar, int row) {
+    // The tensor maps are 4-D (column, then head and token ordered by stride, then batch), so
+    // that [B,H,N,d], [B,N,H,d] and rows inside a fused projection output are read in place.
+    auto load_tile = [&](uint32_t dst, const CUtensorMap* tm, uint32_t bar, int row, int which) {
+        const bool hf = (p.head_first_mask >> which) & 1;   // head index before the token index
+        const int c1 = hf ? h : row, c2 = hf ? row : h;
 #pragma unroll
-        for (int hh = 0; hh < NH; ++hh) tma_load_3d(dst + hh * 16384, tm, bar, hh * 64, row, bh);
+        for (int hh = 0; hh < NH; ++hh) tma_load_4d(dst + hh * 16384, tm, bar, hh * 64, c1, c2, b);
     };
     // Loads of chunk c: part 1 = X and A, part 2 = Bv (X alone in the read-out pass).
     auto issue_loads = [&](int c, bool part1, bool part2) {
@@ -397,12 +403,12 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         if (L::kSplitB) {
             if (part1) {
                 mbar_expect_tx(bar, 2 * L::kTile);
-                load_tile(stage_x(s), &tmX, bar, row);
-                load_tile(stage_a(s), &tmA, bar, row);
+                load_tile(stage_x(s), &tmX, bar, row, 0);
+                load_tile(stage_a(s), &tmA, bar, row, 1);
             }
             if (part2) {
                 mbar_expect_tx(bar_full_b + 8 * s, L::kTile);
-                load_tile(stage_b(s), &tmB, bar_full_b + 8 * s, row);
+                load_tile(stage_b(s), &tmB, bar_full_b + 8 * s, row, 2);
             }
         } else {
             // One barrier for the stage, two arrivals: each part arms its own byte count
@@ -411,14 +417,14 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             if (part1) {
                 mbar_expect_tx(bar, kPart1Tiles * L::kTile);
                 if (L::kHasAB) {
-                    if (L::kHasX) load_tile(stage_x(s), &tmX, bar, row);
-                    load_tile(stage_a(s), &tmA, bar, row);
+                    if (L::kHasX) load_tile(stage_x(s), &tmX, bar, row, 0);
+                    load_tile(stage_a(s), &tmA, bar, row, 1);
                 }
             }
             if (part2) {
                 mbar_expect_tx(bar, L::kTile);
-                if (L::kHasAB) load_tile(stage_b(s), &tmB, bar, row);
-                else load_tile(stage_x(s), &tmX, bar, row);
+                if (L::kHasAB) load_tile(stage_b(s), &tmB, bar, row, 2);
+                else load_tile(stage_x(s), &tmX, bar, row, 0);
             }
         }
     };
@@ -431,7 +437,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                                             : base + ((two && (c & 1)) ? L::kOffOutBuf + L::kTile : L::kOffProj);
         const uint32_t pbar = two ? bar_proj + 8 * (c & 1) : bar_proj;
         mbar_expect_tx(pbar, L::kTile);
-        load_tile(proj_u, &tmP, pbar, chunk_row(c));
+        load_tile(proj_u, &tmP, pbar, chunk_row(c), 3);
     };
     // Every kernel but the first of a library call follows a kernel of the same call, which
     // writes none of the tensors loaded here: its first tiles are requested before the wait
@@ -699,8 +705,11 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 }
                 const uint32_t src = own_out ? base + out_off(c) : base + s * L::kStage + L::kOffOut;
 #pragma unroll
-                for (int hh = 0; hh < NH; ++hh)
-                    tma_store_3d(&tmO, src + hh * 16384, hh * 64, chunk_row(c), bh);
+                for (int hh = 0; hh < NH; ++hh) {
+                    const bool hfo = (p.head_first_mask >> 4) & 1;
+                    const int row = chunk_row(c);
+                    tma_store_4d(&tmO, src + hh * 16384, hh * 64, hfo ? h : row, hfo ? row : h, b);
+                }
                 tma_store_commit();
                 COTT_STAMP_AT(4, c, 4);
                 if (out_pair) {
@@ -1124,16 +1133,25 @@ EncodeTiledFn get_encode() {
     return fn;
 }
 
-// Tensor map over a contiguous [BH, N, d] bf16 tensor: box = 128 rows x 64 columns of one
-// (b,h) slice, 128-byte swizzle; rows past N read as zero and are not written.
-bool make_tile_map(CUtensorMap* map, const void* ptr, int BH, int N, int d) {
+// Tensor map over a bf16 tensor of logical shape [B,H,N,d] with element strides (sb, sh, sn)
+// and contiguous rows: 4-D, the head and token dimensions ordered by stride (dense [B,H,N,d]:
+// token first; [B,N,H,d] or rows inside a fused projection output: head first); box = 128
+// tokens x 64 columns of one (b,h), 128-byte swizzle; rows past N read as zero and are not
+// written.  *head_first tells the kernel the order of the two middle coordinates.
+bool make_tile_map(CUtensorMap* map, const void* ptr, int B, int H, int N, int d, const RowLayout& lay,
+                   bool* head_first) {
     EncodeTiledFn enc = get_encode();
     if (!enc) return false;
-    cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)BH};
-    cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)N * d * 2};
-    cuuint32_t box[3] = {64, (cuuint32_t)kChunk, 1};
-    cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides,
+    const RowLayout l = resolve_layout(lay, H, N, d);
+    if (l.sn < d || l.sh < d || l.sb < d || (l.sn & 7) || (l.sh & 7) || (l.sb & 7)) return false;
+    const bool hf = l.sh < l.sn;
+    *head_first = hf;
+    cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)(hf ? H : N), (cuuint64_t)(hf ? N : H), (cuuint64_t)B};
+    cuuint64_t strides[3] = {(cuuint64_t)(hf ? l.sh : l.sn) * 2, (cuuint64_t)(hf ? l.sn : l.sh) * 2,
+                             (cuuint64_t)l.sb * 2};
+    cuuint32_t box[4] = {64, hf ? 1u : (cuuint32_t)kChunk, hf ? (cuuint32_t)kChunk : 1u, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides,
                      box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
@@ -1199,12 +1217,20 @@ cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cuda
     const int BH = B * H;
     // Unused operands still need a valid map: point them at a tensor that exists.
     const void* any = a.x ? a.x : a.a;
+    const RowLayout any_l = a.x ? a.lx : a.la;
     const void* ptrs[5] = {a.x ? a.x : any, a.a ? a.a : any, a.bv ? a.bv : any,
                            a.proj ? a.proj : any, a.out ? a.out : any};
+    const RowLayout lays[5] = {a.x ? a.lx : any_l, a.a ? a.la : any_l, a.bv ? a.lbv : any_l,
+                               a.proj ? a.lproj : any_l, a.out ? a.lout : any_l};
     CUtensorMap tm[5];
-    for (int i = 0; i < 5; ++i)
-        if (!make_tile_map(&tm[i], ptrs[i], BH, N, d)) return cudaErrorInvalidValue;
+    int head_first_mask = 0;
+    for (int i = 0; i < 5; ++i) {
+        bool hf = false;
+        if (!make_tile_map(&tm[i], ptrs[i], B, H, N, d, lays[i], &hf)) return cudaErrorInvalidValue;
+        head_first_mask |= (hf ? 1 : 0) << i;
+    }
     TcWalkParams p;
+    p.head_first_mask = head_first_mask;
     p.init = a.init; p.state_out = a.state_out; p.dm_partial = a.dm_partial; p.dm_out = a.dm_out; p.status = a.status;
     p.init_has_scale = a.init_has_scale; p.state_final = a.state_final;
     p.m = a.m; p.seq_len = a.seq_len; p.seq_len_scalar = a.seq_len_scalar;

@@ -600,3 +600,63 @@ def test_bounded_wait_runs_out_and_reports(monkeypatch, force_group):
     o = cott.fwd(q, k, v, m, causal=True, workspace=ws)
     assert cott.cott.last_async_status(ws) == 0
     gate(o, oracle.fwd_quadratic(c["q"], c["k"], c["v"], c["m"], None, True), torch.bfloat16)
+
+
+# ------------------------------------------------------------------ tensors that are not dense [B,H,N,d]
+def _as_bnhd(x):
+    """The same values stored as [B,N,H,d], seen as [B,H,N,d] (what a projection GEMM leaves)."""
+    return x.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+
+
+@pytest.mark.parametrize("dtype,d", [(torch.bfloat16, 64), (torch.bfloat16, 128), (torch.float32, 32)])
+@pytest.mark.parametrize("causal", [True, False])
+def test_strided_layouts_match_dense(dtype, d, causal):
+    """[B,N,H,d] storage and the slices of a fused [B,N,3,H,d] projection output, read and
+    written in place: bit-identical to the same call on dense [B,H,N,d] copies (the arithmetic
+    does not depend on where the rows sit), forward, exported state and all gradients; and the
+    dense result itself against the definition."""
+    B, H, N = 2, 5, 333
+    c = synth.make_qkv(B, H, N, d, dtype, 5600 + d, with_do=True)
+    q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
+    o_ref, st_ref = cott.fwd(q, k, v, m, causal=causal, return_state=True)
+    g_ref = cott.bwd(q, k, v, d_o, m, causal=causal)
+    gate(o_ref, oracle.fwd_quadratic(c["q"], c["k"], c["v"], c["m"], None, causal), dtype)
+
+    # (1) [B,N,H,d] storage for everything, outputs included (empty_like keeps the strides)
+    qb, kb, vb, dob = (_as_bnhd(x) for x in (q, k, v, d_o))
+    assert not qb.is_contiguous()
+    o1, st1 = cott.fwd(qb, kb, vb, m, causal=causal, return_state=True)
+    assert o1.stride() == qb.stride()
+    assert torch.equal(o1, o_ref) and torch.equal(st1, st_ref)
+    g1 = cott.bwd(qb, kb, vb, dob, m, causal=causal)
+    for a, b in zip(g1, g_ref):
+        assert torch.equal(a, b)
+
+    # (2) fused projection output [B,N,3,H,d]; gradients into a fused buffer of the same shape;
+    #     o and dO dense [B,H,N,d]
+    fused = torch.stack([x.permute(0, 2, 1, 3) for x in (q, k, v)], dim=2).contiguous()   # [B,N,3,H,d]
+    qf, kf, vf = (fused[:, :, i].permute(0, 2, 1, 3) for i in range(3))
+    assert qf.stride() == (N * 3 * H * d, d, 3 * H * d, 1)
+    o2 = cott.fwd(qf, kf, vf, m, causal=causal, out=torch.empty_like(q))
+    assert torch.equal(o2, o_ref)
+    gfused = torch.full_like(fused, float("nan"))
+    outs = tuple(gfused[:, :, i].permute(0, 2, 1, 3) for i in range(3))
+    g2 = cott.bwd(qf, kf, vf, d_o, m, causal=causal, out=outs)
+    for a, b in zip(g2[:3], g_ref[:3]):
+        assert torch.equal(a, b)
+    assert torch.equal(g2[3], g_ref[3])
+    assert torch.isfinite(gfused.float()).all()          # every element of the fused buffer was written
+
+
+def test_strided_argument_checks():
+    """Strides the kernels cannot address are refused, not mis-read: rows that are not
+    contiguous, token strides that are not a multiple of 16 bytes."""
+    c = synth.make_qkv(1, 2, 64, 64, torch.bfloat16, 5700)
+    q, k, v, m = (dev(c[x]) for x in ("q", "k", "v", "m"))
+    with pytest.raises(ValueError):
+        cott.fwd(q.transpose(2, 3), k.transpose(2, 3), v.transpose(2, 3), m)      # rows not contiguous
+    wide = torch.zeros((1, 2, 64, 68), dtype=torch.bfloat16, device="cuda")       # token stride 136 bytes
+    with pytest.raises(cott.CottError):
+        cott.fwd(wide[..., :64], wide[..., :64], wide[..., :64], m, out=torch.empty_like(q))
+    with pytest.raises(ValueError):
+        cott.fwd(q, _as_bnhd(k), v, m)                                            # q, k, v must share strides
