@@ -197,6 +197,31 @@ cott_status cott_bwd_strided(const void* q, const void* k, const void* v, const 
                              void* stream);
 
 /*
+ * Packed variable-length batches: the rows of B sequences back to back in tensors of shape
+ * [total_tokens, H, d] (dense), sequence b occupying rows cu_seqlens[b] .. cu_seqlens[b+1]-1
+ * (cu_seqlens: DEVICE array of B + 1 ints, cu_seqlens[0] = 0, cu_seqlens[B] = total_tokens,
+ * non-decreasing).  Each sequence is attended on its own, Eq. 5 (causal == 0) or Eq. 6-8
+ * (causal != 0), with its own scaling base for Eq. 4: sp->seq_len[b], else sp->seq_len_scalar,
+ * else its length.  No padding rows are read as keys or written as outputs.
+ *   max_seqlen : an upper bound of the longest sequence (sizes the workspace and the plan)
+ *   workspace  : cott_workspace_bytes(COTT_OP_FWD or COTT_OP_BWD, dt, B, H, max_seqlen, d, causal)
+ * bf16 with d 64 or 128 only (COTT_ERR_UNSUPPORTED otherwise); one CTA walks one (sequence,
+ * head), so the GPU is filled when B*H reaches the number of SMs.  A NaN or Inf in the first
+ * rows of one sequence can reach the last rows of the sequence stored before it (the tile
+ * that holds both is multiplied by zeros, not skipped).  Other arguments, ordering and
+ * aliasing rules as for cott_fwd / cott_bwd.
+ */
+cott_status cott_fwd_varlen(const void* q, const void* k, const void* v, void* o,
+                            const int* cu_seqlens, int B, int H, int total_tokens, int max_seqlen,
+                            int d, int causal, cott_dtype dt, const cott_scale_params* sp,
+                            void* workspace, size_t workspace_bytes, void* stream);
+cott_status cott_bwd_varlen(const void* q, const void* k, const void* v, const void* d_o, void* dq,
+                            void* dk, void* dv, float* dm, const int* cu_seqlens, int B, int H,
+                            int total_tokens, int max_seqlen, int d, int causal, cott_dtype dt,
+                            const cott_scale_params* sp, void* workspace, size_t workspace_bytes,
+                            void* stream);
+
+/*
  * One recurrent decode step, Eq. 8:  S <- S + k^ (c v)^T ;  o = S^T q^  (update, then read).
  *   q,k,v  in    : [B,H,d] dt
  *   state  in/out: fp32 [B,H,d,d], updated in place (constant-size inference memory)

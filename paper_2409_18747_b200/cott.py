@@ -72,6 +72,12 @@ def _load():
     lib.cott_bwd_strided.restype = ci
     lib.cott_bwd_strided.argtypes = [vp] * 8 + [ci, ci, ci, ci, ci, ci, vp, vp, vp,
                                                  ctypes.POINTER(_ScaleParams), vp, cs, vp]
+    lib.cott_fwd_varlen.restype = ci
+    lib.cott_fwd_varlen.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci,
+                                    ctypes.POINTER(_ScaleParams), vp, cs, vp]
+    lib.cott_bwd_varlen.restype = ci
+    lib.cott_bwd_varlen.argtypes = [vp] * 9 + [ci, ci, ci, ci, ci, ci, ci,
+                                                ctypes.POINTER(_ScaleParams), vp, cs, vp]
     lib.cott_fwd_stateful.restype = ci
     lib.cott_fwd_stateful.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci,
                                       ctypes.POINTER(_ScaleParams), vp, cs, vp]
@@ -260,6 +266,56 @@ def bwd(q, k, v, d_o, m, seq_len=None, causal=True, workspace=None, stream=None,
                                   ctypes.byref(sp), ws.data_ptr(), ws_bytes, _stream_ptr(stream))
     if rc != 0:
         raise CottError(rc, "cott_bwd_strided")
+    return dq, dk, dv, dm
+
+
+def _check_packed(cu_seqlens, *ts):
+    if cu_seqlens.dtype != torch.int32 or cu_seqlens.dim() != 1 or cu_seqlens.numel() < 2:
+        raise ValueError("cu_seqlens must be an int32 [B+1] CUDA tensor")
+    _check_dev(cu_seqlens, *ts)
+    for t in ts:
+        if t.dim() != 3 or t.shape != ts[0].shape:
+            raise ValueError("packed tensors must all be [total_tokens, H, d]")
+
+
+def fwd_varlen(q, k, v, m, cu_seqlens, max_seqlen, seq_len=None, causal=True, out=None, workspace=None,
+               stream=None):
+    """cott_fwd_varlen: q, k, v ``[total_tokens, H, d]`` (bf16, d 64 or 128), the sequences of the
+    batch back to back; ``cu_seqlens`` int32 ``[B+1]`` CUDA tensor of row offsets.  Returns ``o``."""
+    _check_packed(cu_seqlens, q, k, v)
+    _check_dev(m, seq_len if isinstance(seq_len, torch.Tensor) else None)
+    T, H, d = q.shape
+    B = cu_seqlens.numel() - 1
+    dt = _dt(q)
+    o = torch.empty_like(q) if out is None else out
+    ws, ws_bytes = _workspace(OP_FWD, dt, B, H, int(max_seqlen), d, causal, q.device, workspace)
+    sp = _scale(m, seq_len)
+    rc = _load().cott_fwd_varlen(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
+                                 cu_seqlens.data_ptr(), B, H, T, int(max_seqlen), d, int(bool(causal)), dt,
+                                 ctypes.byref(sp), ws.data_ptr(), ws_bytes, _stream_ptr(stream))
+    if rc != 0:
+        raise CottError(rc, "cott_fwd_varlen")
+    return o
+
+
+def bwd_varlen(q, k, v, d_o, m, cu_seqlens, max_seqlen, seq_len=None, causal=True, workspace=None,
+               stream=None):
+    """cott_bwd_varlen.  Returns ``(dq, dk, dv, dm[H] fp32)`` for packed ``[total_tokens, H, d]`` inputs."""
+    _check_packed(cu_seqlens, q, k, v, d_o)
+    _check_dev(m, seq_len if isinstance(seq_len, torch.Tensor) else None)
+    T, H, d = q.shape
+    B = cu_seqlens.numel() - 1
+    dt = _dt(q)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(q), torch.empty_like(q)
+    dm = torch.empty((H,), dtype=torch.float32, device=q.device)
+    ws, ws_bytes = _workspace(OP_BWD, dt, B, H, int(max_seqlen), d, causal, q.device, workspace)
+    sp = _scale(m, seq_len)
+    rc = _load().cott_bwd_varlen(q.data_ptr(), k.data_ptr(), v.data_ptr(), d_o.data_ptr(), dq.data_ptr(),
+                                 dk.data_ptr(), dv.data_ptr(), dm.data_ptr(), cu_seqlens.data_ptr(), B, H, T,
+                                 int(max_seqlen), d, int(bool(causal)), dt, ctypes.byref(sp), ws.data_ptr(),
+                                 ws_bytes, _stream_ptr(stream))
+    if rc != 0:
+        raise CottError(rc, "cott_bwd_varlen")
     return dq, dk, dv, dm
 
 

@@ -253,11 +253,18 @@ static cott_status run_tc_stream(TcWalkArgs t, const Plan& p, int B, int H, int 
     return COTT_OK;
 }
 
+// Packed variable-length batch (see cott_fwd_varlen): row offsets and total row count.
+struct Packed {
+    const int* cu_seqlens = nullptr;
+    int total_tokens = 0;
+};
+
 static cott_status fwd_impl(const void* q, const void* k, const void* v, void* o, float* state_out,
                             int B, int H, int N, int d, int causal, cott_dtype dt,
                             const cott_scale_params* sp, void* ws, const Plan& p,
                             cudaStream_t st, const float* state_in = nullptr,
-                            const cott_strides* s_qkv = nullptr, const cott_strides* s_o = nullptr) {
+                            const cott_strides* s_qkv = nullptr, const cott_strides* s_o = nullptr,
+                            Packed packed = Packed()) {
     const CallLayouts lay{to_layout(s_qkv), to_layout(s_o), RowLayout{0, 0, 0}, q, k, v, o};
     // The tensor-core path clears the status words in its first kernel.
     if (p.path != 1) COTT_CUDA(cudaMemsetAsync(ws, 0, kWsHeaderBytes, st));
@@ -267,6 +274,7 @@ static cott_status fwd_impl(const void* q, const void* k, const void* v, void* o
         memset(&t, 0, sizeof(t));
         t.x = q; t.a = k; t.bv = v; t.out = o;
         lay.assign(t);
+        t.cu_seqlens = packed.cu_seqlens; t.total_tokens = packed.total_tokens;
         t.norm_bv = 0; t.x_norm = 1; t.epilogue = EPI_PLAIN; t.reverse = 0;
         t.clear_status = 1;
         return run_tc_stream(t, p, B, H, N, d, causal, sp, static_cast<int*>(ws), states,
@@ -315,7 +323,8 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
                             void* dk, void* dv, float* dm, int B, int H, int N, int d, int causal,
                             cott_dtype dt, const cott_scale_params* sp, void* ws, const Plan& p,
                             cudaStream_t st, const cott_strides* s_qkv = nullptr,
-                            const cott_strides* s_do = nullptr, const cott_strides* s_dqkv = nullptr) {
+                            const cott_strides* s_do = nullptr, const cott_strides* s_dqkv = nullptr,
+                            Packed packed = Packed()) {
     const CallLayouts lay{to_layout(s_qkv), to_layout(s_do), to_layout(s_dqkv), q, k, v, d_o};
     // The tensor-core path clears the status words in its first kernel.
     if (p.path != 1) COTT_CUDA(cudaMemsetAsync(ws, 0, kWsHeaderBytes, st));
@@ -331,6 +340,7 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
         int* status = static_cast<int*>(ws);
         TcWalkArgs t;
         memset(&t, 0, sizeof(t));
+        t.cu_seqlens = packed.cu_seqlens; t.total_tokens = packed.total_tokens;
         // When two walks with one CTA per (b, h) fit on the GPU side by side but not two per
         // (b, h) (74 / 2 < B*H <= 74), the dK^ and dV' streams run next to each other, each
         // over the whole sequence as a single group (no partial-state pass, no scan), with the
@@ -606,6 +616,65 @@ cott_status cott_bwd_strided(const void* q, const void* k, const void* v, const 
         return COTT_ERR_WORKSPACE;
     return bwd_impl(q, k, v, d_o, dq, dk, dv, dm, B, H, N, d, causal, dt, sp, workspace, p,
                     static_cast<cudaStream_t>(stream), qkv_strides, do_strides, dqkv_strides);
+}
+
+// Plan of a packed batch: one group per (sequence, head), tensor-core path only.
+static bool varlen_plan(cott_dtype dt, int B, int H, int total_tokens, int max_seqlen, int d, Plan* p) {
+    if (B < 1 || H < 1 || total_tokens < 1 || max_seqlen < 1 || max_seqlen > total_tokens) return false;
+    if (dt != COTT_BF16 || (d != 64 && d != 128)) return false;
+    p->path = 1; p->chunk = 128; p->group = (max_seqlen + 127) / 128 * 128; p->n_groups = 1; p->split = 1;
+    return true;
+}
+
+cott_status cott_fwd_varlen(const void* q, const void* k, const void* v, void* o,
+                            const int* cu_seqlens, int B, int H, int total_tokens, int max_seqlen,
+                            int d, int causal, cott_dtype dt, const cott_scale_params* sp,
+                            void* workspace, size_t workspace_bytes, void* stream) {
+    if (!q || !k || !v || !o || !cu_seqlens) return COTT_ERR_INVALID_ARG;
+    if (check_scale(sp) != COTT_OK) return COTT_ERR_INVALID_ARG;
+    if (o == q || o == k || o == v) return COTT_ERR_INVALID_ARG;
+    if (!sp->seq_len && sp->seq_len_scalar > 0.f && sp->seq_len_scalar < 1.f) return COTT_ERR_INVALID_ARG;
+    Plan p;
+    if (!varlen_plan(dt, B, H, total_tokens, max_seqlen, d, &p)) return COTT_ERR_UNSUPPORTED;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return COTT_ERR_UNSUPPORTED;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
+        workspace_bytes < workspace_bytes_impl(COTT_OP_FWD, p, B, H, d))
+        return COTT_ERR_WORKSPACE;
+    // rows of all sequences back to back, [total_tokens, H, d]
+    const cott_strides packed_l = {(long long)total_tokens * H * d, (long long)d, (long long)H * d};
+    Packed pk; pk.cu_seqlens = cu_seqlens; pk.total_tokens = total_tokens;
+    return fwd_impl(q, k, v, o, nullptr, B, H, max_seqlen, d, causal, dt, sp, workspace, p,
+                    static_cast<cudaStream_t>(stream), nullptr, &packed_l, &packed_l, pk);
+}
+
+cott_status cott_bwd_varlen(const void* q, const void* k, const void* v, const void* d_o, void* dq,
+                            void* dk, void* dv, float* dm, const int* cu_seqlens, int B, int H,
+                            int total_tokens, int max_seqlen, int d, int causal, cott_dtype dt,
+                            const cott_scale_params* sp, void* workspace, size_t workspace_bytes,
+                            void* stream) {
+    if (!q || !k || !v || !d_o || !dq || !dk || !dv || !dm || !cu_seqlens) return COTT_ERR_INVALID_ARG;
+    if (check_scale(sp) != COTT_OK) return COTT_ERR_INVALID_ARG;
+    const void* ins[4] = {q, k, v, d_o};
+    void* outs[3] = {dq, dk, dv};
+    for (int i = 0; i < 3; ++i) {
+        for (int j = 0; j < 4; ++j)
+            if (outs[i] == ins[j]) return COTT_ERR_INVALID_ARG;
+        for (int j = i + 1; j < 3; ++j)
+            if (outs[i] == outs[j]) return COTT_ERR_INVALID_ARG;
+    }
+    if (!sp->seq_len && sp->seq_len_scalar > 0.f && sp->seq_len_scalar < 1.f) return COTT_ERR_INVALID_ARG;
+    Plan p;
+    if (!varlen_plan(dt, B, H, total_tokens, max_seqlen, d, &p)) return COTT_ERR_UNSUPPORTED;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(d_o) || !aligned16(dq) ||
+        !aligned16(dk) || !aligned16(dv))
+        return COTT_ERR_UNSUPPORTED;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
+        workspace_bytes < workspace_bytes_impl(COTT_OP_BWD, p, B, H, d))
+        return COTT_ERR_WORKSPACE;
+    const cott_strides packed_l = {(long long)total_tokens * H * d, (long long)d, (long long)H * d};
+    Packed pk; pk.cu_seqlens = cu_seqlens; pk.total_tokens = total_tokens;
+    return bwd_impl(q, k, v, d_o, dq, dk, dv, dm, B, H, max_seqlen, d, causal, dt, sp, workspace, p,
+                    static_cast<cudaStream_t>(stream), &packed_l, &packed_l, &packed_l, pk);
 }
 
 cott_status cott_decode_step(const void* q, const void* k, const void* v, float* state, void* o,

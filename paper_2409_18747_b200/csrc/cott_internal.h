@@ -70,6 +70,9 @@ struct TcWalkArgs {
     int mode;
     const void* x; const void* a; const void* bv; const void* proj; void* out;
     RowLayout lx, la, lbv, lproj, lout;   // layouts of the five tensors (all zero: dense)
+    // Packed variable-length batch: device array of B + 1 row offsets into tensors that hold
+    // total_tokens rows per head (batch stride unused); one group per (b, h).  NULL: dense batch.
+    const int* cu_seqlens; int total_tokens;
     const float* init; float* state_out; float* dm_partial; int* status;
     const float* m; const float* seq_len; float seq_len_scalar;
     int group; int n_groups;

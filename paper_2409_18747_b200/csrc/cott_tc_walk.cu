@@ -51,6 +51,10 @@ struct TcWalkParams {
     int clear_status;                   // first kernel of a call: CTA 0 zeroes the status words
     int wait_limit_kcycles;             // bound of every wait, in units of 1024 SM cycles
     int debug_drop_commit;              // test hook: the scores of chunk 1 are never reported complete
+    // Packed variable-length batch: rows of all sequences back to back in one [T, H, d]
+    // tensor, sequence b = rows cu_seqlens[b] .. cu_seqlens[b+1]-1, one group per (b, h).
+    const int* cu_seqlens;              // NULL: every (b, h) has N rows of its own
+    void* out_rows; long long out_sn, out_sh;   // Out as plain global memory (rows of a ragged last chunk)
     int head_first_mask;                // bit i: in tensor map i (X, A, Bv, raw rows, Out) the head index
                                         // comes before the token index (its stride is the smaller one)
 };
@@ -328,9 +332,17 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     COTT_STAMP_AT(0, kStampC0, 5);
     const int g = p.first_group + blockIdx.x % p.grid_groups, bh = blockIdx.x / p.grid_groups;
     const int b = bh / p.H, h = bh % p.H;
-    const int tok0 = g * p.group;
-    const int tok1 = min(p.N, tok0 + p.group);
+    const bool varlen = p.cu_seqlens != nullptr;
+    const int tok0 = varlen ? p.cu_seqlens[b] : g * p.group;
+    const int tok1 = varlen ? p.cu_seqlens[b + 1] : min(p.N, tok0 + p.group);
     const int n_chunks = (tok1 - tok0 + kChunk - 1) / kChunk;
+    // Packed batch: the chunks of a sequence start at its first row, so only its last chunk can
+    // hold rows of the next sequence.  Those rows take no part: the operand that is normalised
+    // in shared memory gets zeros there (it is one of the two operands of the state update and
+    // either the key side of the scores or the value side of P~ Bv), their outputs are not
+    // stored, and they add nothing to dm.
+    const int bcoord = varlen ? 0 : b;                 // batch coordinate of the tensor maps
+    const bool ragged_last = varlen && ((tok1 - tok0) % kChunk) != 0;
     constexpr bool kNormBv = STREAM == S_DQ || STREAM == S_DK;
     constexpr bool kXNorm = STREAM == S_FWD || STREAM == S_DV;
     constexpr bool kReverse = STREAM == S_DK || STREAM == S_DV;
@@ -385,6 +397,8 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     // read last -- still in L2 -- are the ones the walk needs first.
     const bool backward = (MODE == MODE_STATE) ? (p.state_rev != 0) : kReverse;
     auto chunk_row = [&](int c) { return tok0 + (backward ? (n_chunks - 1 - c) : c) * kChunk; };
+    // Step at which the sequence's last chunk (the only one that can be ragged) is visited.
+    const int last_visit_of_ragged = backward ? 0 : n_chunks - 1;
 
     // TMA loads (issued by single threads of the control and the store warp).
     // The tensor maps are 4-D (column, then head and token ordered by stride, then batch), so
@@ -393,7 +407,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         const bool hf = (p.head_first_mask >> which) & 1;   // head index before the token index
         const int c1 = hf ? h : row, c2 = hf ? row : h;
 #pragma unroll
-        for (int hh = 0; hh < NH; ++hh) tma_load_4d(dst + hh * 16384, tm, bar, hh * 64, c1, c2, b);
+        for (int hh = 0; hh < NH; ++hh) tma_load_4d(dst + hh * 16384, tm, bar, hh * 64, c1, c2, bcoord);
     };
     // Loads of chunk c: part 1 = X and A, part 2 = Bv (X alone in the read-out pass).
     auto issue_loads = [&](int c, bool part1, bool part2) {
@@ -456,7 +470,9 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     if (!early_loads && is_ctrl && lane == 0)
         for (int c = 0; c < NST && c < n_chunks; ++c) issue_loads(c, true, true);
 
-    const float s_b = p.seq_len ? p.seq_len[b] : (p.seq_len_scalar > 0.f ? p.seq_len_scalar : (float)p.N);
+    const float s_b = p.seq_len ? p.seq_len[b]
+                                : (p.seq_len_scalar > 0.f ? p.seq_len_scalar
+                                                          : (float)(varlen ? max(tok1 - tok0, 1) : p.N));
     const float cfac = stab_factor(p.m[h], s_b);
 
     // Accumulator mapping of a worker thread: TMEM lane quadrant q, column quarter cq, row.
@@ -705,10 +721,11 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 }
                 const uint32_t src = own_out ? base + out_off(c) : base + s * L::kStage + L::kOffOut;
 #pragma unroll
-                for (int hh = 0; hh < NH; ++hh) {
+                // (the rows of a ragged last chunk of a packed batch were written by the workers)
+                for (int hh = 0; hh < ((ragged_last && c == last_visit_of_ragged) ? 0 : NH); ++hh) {
                     const bool hfo = (p.head_first_mask >> 4) & 1;
                     const int row = chunk_row(c);
-                    tma_store_4d(&tmO, src + hh * 16384, hh * 64, hfo ? h : row, hfo ? row : h, b);
+                    tma_store_4d(&tmO, src + hh * 16384, hh * 64, hfo ? h : row, hfo ? row : h, bcoord);
                 }
                 tma_store_commit();
                 COTT_STAMP_AT(4, c, 4);
@@ -753,14 +770,15 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         };
         auto pair_sum = [&](float v) { return v + __shfl_xor_sync(0xffffffffu, v, 16); };
         // x^ = x / max(||x||, eps) on this thread's half row, in place, rounded to bf16.
-        auto normalise_half_row = [&](uint8_t* nt) {
+        auto normalise_half_row = [&](uint8_t* nt, int c) {
             uint4 wn[NC];
             float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
             for (int j = 0; j < NC; ++j) wn[j] = *reinterpret_cast<const uint4*>(tile_h_ptr(nt, j));
 #pragma unroll
             for (int j = 0; j < NC; j += 2) { sumsq8(wn[j], a0, a1); sumsq8(wn[j + 1], a2, a3); }
-            const float r = 1.0f / fmaxf(sqrtf(pair_sum((a0 + a1) + (a2 + a3))), kEps);
+            float r = 1.0f / fmaxf(sqrtf(pair_sum((a0 + a1) + (a2 + a3))), kEps);
+            if (varlen && chunk_row(c) + nrow >= tok1) r = 0.f;     // a row of the next sequence
 #pragma unroll
             for (int j = 0; j < NC; ++j) {
                 const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&wn[j]);
@@ -784,7 +802,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             COTT_STAMP_AT(1, c - 1, 7);
             // In the split causal walk Bv arrives on its own barrier and is normalised later.
             if (L::kHasAB && !(L::kSplitB && kNormBv))
-                normalise_half_row(gbase + s * L::kStage + (kNormBv ? L::kOffB : L::kOffA));
+                normalise_half_row(gbase + s * L::kStage + (kNormBv ? L::kOffB : L::kOffA), c);
             mbar_arrive(bar_a_ready + 8 * s);
         };
         auto x_scale = [&](int c) {
@@ -809,7 +827,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         auto norm_b = [&](int c) {
             const int s = c % NST;
             if (!wait(bar_full_b + 8 * s, (c / NST) & 1)) return;
-            normalise_half_row(gbase + s * L::kStage + L::kOffB);
+            normalise_half_row(gbase + s * L::kStage + L::kOffB, c);
             mbar_arrive(bar_b_ready + 8 * s);
         };
         // bf16 copy of 32 state columns of this thread's row into the MN-major state tile.
@@ -967,8 +985,9 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                         rp = 1.0f / fmaxf(nrm, kEps);
                         coef = nrm > kEps ? dp * rx * rp * rp : 0.f;
                         // <q^_i, dQ^_i> of the unscaled accumulator, once per row (see kDmFromDq)
-                        if (STREAM == S_DQ && kDmFromDq && hf == 0) dm_acc += dp * rp;
-                    } else if (hf == 0) {
+                        if (STREAM == S_DQ && kDmFromDq && hf == 0 && !(varlen && chunk_row(c) + arow >= tok1))
+                            dm_acc += dp * rp;
+                    } else if (hf == 0 && !(varlen && chunk_row(c) + arow >= tok1)) {
                         dm_acc += dp * rx / cfac;  // <dV', v> with dV' = (rx / c) * acc, once per row
                     }
                 }
@@ -1007,7 +1026,16 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                     uint4 w;
                     w.x = pack_bf16(v[0], v[1]); w.y = pack_bf16(v[2], v[3]);
                     w.z = pack_bf16(v[4], v[5]); w.w = pack_bf16(v[6], v[7]);
-                    *reinterpret_cast<uint4*>(so + (col >> 6) * 16384 + swz(arow, (col & 63) >> 3)) = w;
+                    if (ragged_last && c == last_visit_of_ragged) {
+                        // Packed batch, last chunk of the sequence: a tile store would overwrite
+                        // rows of the next sequence; the rows that exist go out one by one.
+                        const long long grow = (long long)chunk_row(c) + arow;
+                        if (grow < tok1)
+                            *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out_rows) +
+                                                      grow * p.out_sn + (long long)h * p.out_sh + col) = w;
+                    } else {
+                        *reinterpret_cast<uint4*>(so + (col >> 6) * 16384 + swz(arow, (col & 63) >> 3)) = w;
+                    }
                 }
                 fence_proxy_async();
                 mbar_arrive(edone_bar(c));
@@ -1087,7 +1115,9 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 float part = 0.f;
                 for (int i = lane; i < per; i += 32) {
                     const int bb = i / p.n_groups, gg = i - bb * p.n_groups;
-                    const float sb2 = p.seq_len ? p.seq_len[bb] : (p.seq_len_scalar > 0.f ? p.seq_len_scalar : (float)p.N);
+                    const float sb2 = p.seq_len ? p.seq_len[bb]
+                                                : (p.seq_len_scalar > 0.f ? p.seq_len_scalar
+                                                   : (float)(varlen ? max(p.cu_seqlens[bb + 1] - p.cu_seqlens[bb], 1) : p.N));
                     const float ls = logf(sb2);
                     part += __ldcg(&p.dm_partial[((size_t)bb * p.H + hh) * p.n_groups + gg]) *
                             (-ls * sg * (1.0f - sg) * expf(-sg * ls));
@@ -1224,13 +1254,20 @@ cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cuda
                                a.proj ? a.lproj : any_l, a.out ? a.lout : any_l};
     CUtensorMap tm[5];
     int head_first_mask = 0;
+    // A packed batch is one tensor of total_tokens rows per head (batch extent 1).
+    const int map_B = a.cu_seqlens ? 1 : B, map_N = a.cu_seqlens ? a.total_tokens : N;
     for (int i = 0; i < 5; ++i) {
         bool hf = false;
-        if (!make_tile_map(&tm[i], ptrs[i], B, H, N, d, lays[i], &hf)) return cudaErrorInvalidValue;
+        if (!make_tile_map(&tm[i], ptrs[i], map_B, H, map_N, d, lays[i], &hf)) return cudaErrorInvalidValue;
         head_first_mask |= (hf ? 1 : 0) << i;
     }
     TcWalkParams p;
     p.head_first_mask = head_first_mask;
+    p.cu_seqlens = a.cu_seqlens;
+    {
+        const RowLayout lo = resolve_layout(a.lout, H, map_N, d);
+        p.out_rows = a.out; p.out_sn = lo.sn; p.out_sh = lo.sh;
+    }
     p.init = a.init; p.state_out = a.state_out; p.dm_partial = a.dm_partial; p.dm_out = a.dm_out; p.status = a.status;
     p.init_has_scale = a.init_has_scale; p.state_final = a.state_final;
     p.m = a.m; p.seq_len = a.seq_len; p.seq_len_scalar = a.seq_len_scalar;
@@ -1241,7 +1278,9 @@ cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cuda
     const bool subset = a.mode == MODE_STATE && a.grid_groups > 0;
     p.first_group = subset ? a.first_group : 0;
     p.grid_groups = subset ? a.grid_groups : a.n_groups;
-    p.plain_launch = a.plain_launch;
+    // (a packed batch reads cu_seqlens before anything else: no early start behind a kernel
+    // that may have produced it)
+    p.plain_launch = a.plain_launch || a.cu_seqlens != nullptr;
     p.clear_status = a.clear_status;
     {   // knobs for the test of the timeout path: a short bound, and a hand-off that never comes
         const char* e = getenv("COTT_WAIT_LIMIT_MS");

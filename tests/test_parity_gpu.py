@@ -660,3 +660,64 @@ def test_strided_argument_checks():
         cott.fwd(wide[..., :64], wide[..., :64], wide[..., :64], m, out=torch.empty_like(q))
     with pytest.raises(ValueError):
         cott.fwd(q, _as_bnhd(k), v, m)                                            # q, k, v must share strides
+
+
+# ------------------------------------------------------------------ packed variable-length batches
+def _pack(c, lens):
+    """Rows of the sequences back to back: [total, H, d] from per-sequence [1, H, L, d] arrays."""
+    return {k2: torch.cat([torch.from_numpy(np.ascontiguousarray(s[k2][0])).permute(1, 0, 2) for s in c], dim=0)
+            for k2 in ("q", "k", "v", "d_o")}
+
+
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("causal", [True, False])
+@pytest.mark.parametrize("lens", [(300, 1, 128, 129, 77), (1000, 513), (64,)])
+def test_packed_varlen_matches_per_sequence_definition(d, causal, lens):
+    """Sequences of different lengths back to back in [total, H, d]: every sequence's rows equal
+    the definition evaluated on that sequence alone (scaling base = its own length), forward and
+    all gradients; dm is the sum over the sequences.  Rows of a neighbour that share a tile with
+    the end of a sequence must neither be attended to nor overwritten."""
+    H = 3
+    seqs = [synth.make_qkv(1, H, L, d, torch.bfloat16, 5800 + 7 * i + L, with_do=True) for i, L in enumerate(lens)]
+    m_np = seqs[0]["m"]
+    for s in seqs:
+        s["m"] = m_np
+    packed = {k2: v2.to(torch.bfloat16).cuda() for k2, v2 in _pack(
+        [{k3: (x.float().numpy() if isinstance(x, torch.Tensor) else x) for k3, x in s.items()} for s in seqs], lens).items()}
+    cu = torch.tensor(np.concatenate([[0], np.cumsum(lens)]), dtype=torch.int32, device="cuda")
+    m = dev(m_np)
+    o = cott.fwd_varlen(packed["q"], packed["k"], packed["v"], m, cu, max(lens), causal=causal)
+    dq, dk, dv, dm = cott.bwd_varlen(packed["q"], packed["k"], packed["v"], packed["d_o"], m, cu, max(lens), causal=causal)
+    dm_ref = np.zeros(H)
+    conds = np.zeros(H)
+    off = 0
+    for s, L in zip(seqs, lens):
+        ref = oracle.fwd_quadratic(s["q"], s["k"], s["v"], s["m"], None, causal)          # [1,H,L,d]
+        rq, rk, rv, rm = oracle.bwd_quadratic(s["q"], s["k"], s["v"], s["d_o"], s["m"], None, causal)
+        sl = slice(off, off + L)
+        unpack = lambda x: x[sl].permute(1, 0, 2)[None]                                     # [1,H,L,d]
+        gate(unpack(o), ref, torch.bfloat16)
+        gate(unpack(dq), rq, torch.bfloat16); gate(unpack(dk), rk, torch.bfloat16); gate(unpack(dv), rv, torch.bfloat16)
+        dm_ref += rm
+        conds += dm_condition(rv, s["v"], s["m"], None)
+        off += L
+    gate_dm(dm, dm_ref, 1e-2, conds, DM_COND_BF16)
+
+
+def test_packed_varlen_leaves_neighbours_alone():
+    """The ragged end of a sequence shares a 128-row tile with the start of the next one: after a
+    forward into a buffer filled with a marker, exactly the rows of the batch are written."""
+    H, d, lens = 2, 64, (5, 200, 3)
+    T = sum(lens)
+    g = torch.Generator(device="cuda"); g.manual_seed(3)
+    q, k, v = (torch.randn((T + 40, H, d), generator=g, device="cuda").to(torch.bfloat16) for _ in range(3))
+    cu = torch.tensor([0, 5, 205, 208], dtype=torch.int32, device="cuda")
+    m = torch.zeros(H, device="cuda")
+    out = torch.full((T + 40, H, d), 7.0, dtype=torch.bfloat16, device="cuda")
+    cott.fwd_varlen(q[:T], k[:T], v[:T], m, cu, 200, out=out[:T])
+    assert (out[T:] == 7.0).all()                       # nothing past the batch
+    assert not (out[:T] == 7.0).all(dim=-1).any()       # every row of the batch written
+    # sequence 1 alone gives the same rows as inside the batch
+    cu1 = torch.tensor([0, 200], dtype=torch.int32, device="cuda")
+    alone = cott.fwd_varlen(q[5:205].contiguous(), k[5:205].contiguous(), v[5:205].contiguous(), m, cu1, 200)
+    assert torch.equal(alone, out[5:205])
