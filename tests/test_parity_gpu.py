@@ -721,3 +721,29 @@ def test_packed_varlen_leaves_neighbours_alone():
     cu1 = torch.tensor([0, 200], dtype=torch.int32, device="cuda")
     alone = cott.fwd_varlen(q[5:205].contiguous(), k[5:205].contiguous(), v[5:205].contiguous(), m, cu1, 200)
     assert torch.equal(alone, out[5:205])
+
+
+def test_packed_varlen_with_empty_sequences():
+    """Sequences of length zero anywhere in the batch: nothing is read or written for them, the
+    others are unaffected, and the call reports no error."""
+    H, d = 2, 64
+    g = torch.Generator(device="cuda"); g.manual_seed(5)
+    lens = (0, 130, 0, 64, 0)
+    T = sum(lens)
+    q, k, v, d_o = (torch.randn((T, H, d), generator=g, device="cuda").to(torch.bfloat16) for _ in range(4))
+    m = torch.zeros(H, device="cuda")
+    cu = torch.tensor(np.concatenate([[0], np.cumsum(lens)]), dtype=torch.int32, device="cuda")
+    cu2 = torch.tensor([0, 130, 194], dtype=torch.int32, device="cuda")
+    for causal in (True, False):
+        ws = torch.zeros(cott.workspace_bytes(cott.cott.OP_BWD, cott.cott.BF16, len(lens), H, 130, d, causal),
+                         dtype=torch.uint8, device="cuda")
+        a = cott.fwd_varlen(q, k, v, m, cu, 130, causal=causal, workspace=ws)
+        assert cott.cott.last_async_status(ws) == 0
+        b = cott.fwd_varlen(q, k, v, m, cu2, 130, causal=causal)
+        assert torch.equal(a, b)
+        ga = cott.bwd_varlen(q, k, v, d_o, m, cu, 130, causal=causal, workspace=ws)
+        assert cott.cott.last_async_status(ws) == 0
+        gb = cott.bwd_varlen(q, k, v, d_o, m, cu2, 130, causal=causal)
+        for x, y in zip(ga[:3], gb[:3]):
+            assert torch.equal(x, y)
+        torch.testing.assert_close(ga[3], gb[3], rtol=1e-3, atol=1e-3 * float(gb[3].abs().max()))
