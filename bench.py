@@ -55,6 +55,12 @@ WORKLOADS = {
     "c4": dict(name="C4 causal fwd+bwd", B=4, H=16, N=4096, d=64, causal=True, bwd=True),
     "c3": dict(name="C3 causal fwd", B=8, H=12, N=1024, d=64, causal=True, bwd=False),
     "c2": dict(name="C2 bidirectional fwd", B=32, H=12, N=512, d=64, causal=False, bwd=False),
+    # C4 with every tensor stored [B,N,H,d] (what a projection GEMM leaves), read in place
+    "c4-bnhd": dict(name="C4 causal fwd+bwd, tensors stored [B,N,H,d]", B=4, H=16, N=4096, d=64, causal=True,
+                    bwd=True, layout="bnhd"),
+    # packed variable-length batch: 64 sequences of 512..2048 tokens (seeded), no padding rows
+    "varlen": dict(name="packed varlen causal fwd+bwd, 64 sequences of 512..2048 tokens", B=64, H=16, N=2048,
+                   d=128, causal=True, bwd=True, varlen=True),
 }
 
 
@@ -73,7 +79,7 @@ def algorithmic_bytes(w: dict) -> dict:
     """Bytes the method must move per step (bf16 I/O): forward reads q,k,v and writes o
     (4 tensors), backward reads q,k,v,dO and writes dq,dk,dv (7 tensors); a decode step
     reads and writes the fp32 state once."""
-    th = w["B"] * w["H"] * w["N"] * w["d"] * 2
+    th = w.get("rows", w["B"] * w["N"]) * w["H"] * w["d"] * 2
     if w.get("decode"):
         st = w["B"] * w["H"] * w["d"] * w["d"] * 4
         return {"fwd": 2 * st + 4 * w["B"] * w["H"] * w["d"] * 2, "bwd": 0}
@@ -321,9 +327,27 @@ def run_ours(args, w):
         fwd_call = lambda: cott.decode_step(q, k, v, state, m, 8192.0, out=o)
         bwd_call = None
         tokens_per_step = B
+    elif w.get("varlen"):
+        import numpy as np
+        lens = np.random.RandomState(2024).randint(N // 4, N + 1, size=B)
+        lens[0] = N
+        T = int(lens.sum())
+        w["rows"] = T
+        cu = torch.tensor(np.concatenate([[0], np.cumsum(lens)]), dtype=torch.int32, device=dev)
+        q, k, v, d_o = mk(T, H, d), mk(T, H, d), mk(T, H, d), mk(T, H, d)
+        o = torch.empty_like(q)
+        ws_f = torch.empty(cott.workspace_bytes(cott.cott.OP_FWD, dt_code, B, H, N, d, True), dtype=torch.uint8, device=dev)
+        ws_b = torch.empty(cott.workspace_bytes(cott.cott.OP_BWD, dt_code, B, H, N, d, True), dtype=torch.uint8, device=dev)
+        fwd_call = lambda: cott.fwd_varlen(q, k, v, m, cu, N, causal=True, out=o, workspace=ws_f)
+        bwd_call = lambda: cott.bwd_varlen(q, k, v, d_o, m, cu, N, causal=True, workspace=ws_b)
+        tokens_per_step = T
     else:
-        q, k, v = mk(B, H, N, d), mk(B, H, N, d), mk(B, H, N, d)
-        d_o = mk(B, H, N, d) if w["bwd"] else None
+        if w.get("layout") == "bnhd":
+            mk4 = lambda: mk(B, N, H, d).permute(0, 2, 1, 3)     # [B,H,N,d] view of [B,N,H,d] storage
+        else:
+            mk4 = lambda: mk(B, H, N, d)
+        q, k, v = mk4(), mk4(), mk4()
+        d_o = mk4() if w["bwd"] else None
         o = torch.empty_like(q)
         ws_f = torch.empty(cott.workspace_bytes(cott.cott.OP_FWD, dt_code, B, H, N, d, w["causal"]),
                            dtype=torch.uint8, device=dev)
@@ -393,7 +417,7 @@ def run_ours(args, w):
 
     # ---- end to end: host buffers in, host buffers out, through cott_fwd_bwd_host
     e2e = None
-    if w.get("bwd") and not w.get("decode"):
+    if w.get("bwd") and not w.get("decode") and not w.get("varlen") and not w.get("layout"):
         host_in = [t.cpu().pin_memory() for t in (q, k, v, d_o)]
         host_m = m.cpu().pin_memory()
         host_out = [torch.empty_like(host_in[0]).pin_memory() for _ in range(4)]
@@ -485,9 +509,12 @@ def run_ours(args, w):
     if rank != 0:
         return
     ab = algorithmic_bytes(w)
-    th = B * H * N * d * 2                      # bytes of one [B,H,N,d] bf16 tensor
+    th = w.get("rows", B * N) * H * d * 2       # bytes of one bf16 tensor of the step
     plan = cott.query_plan(cott.cott.OP_BWD if w.get("bwd") else cott.cott.OP_FWD, dt_code, B, H, max(N, 1), d,
                            w["causal"]) if not w.get("decode") else {"path": 0, "group": 1, "chunk": 1}
+    if w.get("varlen"):
+        plan = {"path": 1, "group": (N + 127) // 128 * 128, "chunk": 128, "groups": "one per (sequence, head)",
+                "rows": w["rows"], "padded_rows": B * N}
     if walk_ms:
         # walk launches per step: forward reads 3 tensors and writes 1; the dQ and dK streams
         # read 4 (x, a, bv and the raw rows of their projection epilogue) and write 1; the
@@ -498,7 +525,7 @@ def run_ours(args, w):
         dom_ms = statistics.mean(walk_ms)
         kernel = f"tc_walk_kernel<{d},{1 if w['causal'] else 2}> (tcgen05 chunk walk), mean of {len(walk_ms)} launches"
         traffic = KERNEL_DRAM_TRAFFIC.get((d, bool(w["causal"])), None)
-        traffic = traffic * (B * H * N) if traffic else None
+        traffic = traffic * (w.get("rows", B * N) * H) if traffic else None
     else:
         alg = ab["fwd"]
         dom_ms = statistics.mean(fwd_ms)
