@@ -370,12 +370,11 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
         tv.x = k; tv.a = q; tv.bv = d_o; tv.proj = v; tv.out = dv;
         tv.norm_bv = 0; tv.x_norm = 1; tv.epilogue = EPI_DV; tv.reverse = 1;
         // dm: sum over rows of <dV'_j, v_j>, which equals the sum over rows of <q^_i, dQ^_i>.
-        // The causal dQ^ walk forms the latter in its projection epilogue, so it carries the
-        // sum and its last CTA finalises dm; the bidirectional read-out keeps it in the dV' stream.
+        // The dQ^ stream forms the latter in its projection epilogue, so it carries the sum and
+        // its last CTA finalises dm.
+        tq.dm_partial = dm_partial;
+        tq.dm_out = dm;
         lay.assign(tq); lay.assign(tk); lay.assign(tv);
-        TcWalkArgs& tdm = causal ? tq : tv;
-        tdm.dm_partial = dm_partial;
-        tdm.dm_out = dm;
         if (ss) {
             struct TagScope { ~TagScope() { g_prof_cur_tag = 0; } } tag_scope;
             // Everything that follows a cross-stream event wait is a plain launch.

@@ -94,8 +94,8 @@ struct TcWalkArgs {
     // the workspace header (a wait that gives up writes them two seconds later at the earliest),
     // which saves a separate memset in front of every call.
     int clear_status;
-    // On the stream that carries the dm sum (dm_partial set: the dQ^ walk of a causal call,
-    // the dV' read-out of a bidirectional one): when set, the CTA that finishes last turns the
+    // On the stream that carries the dm sum (dm_partial set: the dQ^ stream of the tensor-core
+    // path): when set, the CTA that finishes last turns the
     // [BH, n_groups] partial sums into dm[H] (fixed summation order), so no separate launch
     // is needed.
     float* dm_out;

@@ -66,9 +66,9 @@ enum { MODE_STATE = 0, MODE_CAUSAL = 1, MODE_READOUT = 2 };
 // walk is sensitive to instruction-cache misses: ncu showed 'no instruction' as the top stall
 // of the d = 128 causal walk when all variants shared one body).
 //   S_FWD: X rows normalised in the epilogue, A normalised in shared memory, plain store
-//   S_DQ : Bv normalised, projection epilogue (the causal walk also sums <q^, dQ^> for dm)
+//   S_DQ : Bv normalised, projection epilogue, also sums <q^, dQ^> for dm
 //   S_DK : as S_DQ, time reversed
-//   S_DV : as S_FWD, time reversed (the read-out form adds the <dV', V> sums for dm)
+//   S_DV : as S_FWD, time reversed
 enum { S_FWD = 0, S_DQ = 1, S_DK = 2, S_DV = 3 };
 
 constexpr int kWorkerWarps = 16;                      // row-worker warps (4 per TMEM lane quadrant)
@@ -346,14 +346,12 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     constexpr bool kNormBv = STREAM == S_DQ || STREAM == S_DK;
     constexpr bool kXNorm = STREAM == S_FWD || STREAM == S_DV;
     constexpr bool kReverse = STREAM == S_DK || STREAM == S_DV;
-    // The causal dV' walk has a plain epilogue: the sum over rows of <dV'_j, v_j> that dm needs
-    // equals the sum over rows of <q^_i, dQ^_i> (both are the sum over i >= j of
-    // (q^_i . k^_j)(dO_i . v_j)), and the dQ^ walk's projection epilogue already forms
-    // <q_i, dQ^_i> for every row, so that walk accumulates it and the dV' walk needs neither
+    // The dV' stream has a plain epilogue: the sum over rows of <dV'_j, v_j> that dm needs
+    // equals the sum over rows of <q^_i, dQ^_i> (both are the sum over the attended pairs (i, j)
+    // of (q^_i . k^_j)(dO_i . v_j)), and the dQ^ stream's projection epilogue already forms
+    // <q_i, dQ^_i> for every row, so that stream accumulates it and the dV' stream needs neither
     // the raw v rows nor the per-row exchange.
-    constexpr bool kDmFromDq = MODE == MODE_CAUSAL;
-    constexpr int kEpi = STREAM == S_FWD ? EPI_PLAIN
-                       : (STREAM == S_DV ? (kDmFromDq ? EPI_PLAIN : EPI_DV) : EPI_PROJ);
+    constexpr int kEpi = (STREAM == S_FWD || STREAM == S_DV) ? EPI_PLAIN : EPI_PROJ;
     constexpr bool with_proj = (MODE != MODE_STATE) && (kEpi != EPI_PLAIN);
     const bool is_ctrl = warp == kWorkerWarps;
     const bool is_store = warp == kWorkerWarps + 1;
@@ -984,11 +982,9 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                         const float nrm = sqrtf(ss);
                         rp = 1.0f / fmaxf(nrm, kEps);
                         coef = nrm > kEps ? dp * rx * rp * rp : 0.f;
-                        // <q^_i, dQ^_i> of the unscaled accumulator, once per row (see kDmFromDq)
-                        if (STREAM == S_DQ && kDmFromDq && hf == 0 && !(varlen && chunk_row(c) + arow >= tok1))
+                        // <q^_i, dQ^_i> of the unscaled accumulator, once per row (see kEpi)
+                        if (STREAM == S_DQ && hf == 0 && !(varlen && chunk_row(c) + arow >= tok1))
                             dm_acc += dp * rp;
-                    } else if (hf == 0 && !(varlen && chunk_row(c) + arow >= tok1)) {
-                        dm_acc += dp * rx / cfac;  // <dV', v> with dV' = (rx / c) * acc, once per row
                     }
                 }
                 // Scale, (project,) round to bf16, stage for the TMA store.  The staging slot is
@@ -1190,8 +1186,8 @@ bool make_tile_map(CUtensorMap* map, const void* ptr, int B, int H, int N, int d
 template <int D, int MODE, int STREAM>
 cudaError_t launch_mode(const CUtensorMap* tm, const TcWalkParams& p, int BH, cudaStream_t st) {
     auto kern = tc_walk_kernel<D, MODE, STREAM>;
-    // (the causal dV' walk has a plain epilogue, like the forward walk)
-    constexpr bool with_proj = (MODE != MODE_STATE) && (STREAM != S_FWD) && !(MODE == MODE_CAUSAL && STREAM == S_DV);
+    // (the dV' stream has a plain epilogue, like the forward pass)
+    constexpr bool with_proj = (MODE != MODE_STATE) && (STREAM == S_DQ || STREAM == S_DK);
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
