@@ -268,7 +268,10 @@ template <> __device__ __forceinline__ void tmem_stq<16>(uint32_t taddr, const u
 // (output stores, stage refills, epilogue-tile loads), of warp 18 the state-update thread
 // (State += A^T Bv in the causal walk).  The roles meet only through mbarriers, every wait
 // bounded.
-template <int D, int MODE, int STREAM>
+// VARLEN (packed variable-length batch) is a compile-time property as well: the walk is
+// sensitive to its instruction footprint and register count, and the dense instances were
+// measurably slower (C5 N=131072: 577 us against 515 us) with the packed-batch code in them.
+template <int D, int MODE, int STREAM, bool VARLEN>
 __global__ void __launch_bounds__(kTcThreads, 1)
 tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmA,
                const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmP,
@@ -332,7 +335,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     COTT_STAMP_AT(0, kStampC0, 5);
     const int g = p.first_group + blockIdx.x % p.grid_groups, bh = blockIdx.x / p.grid_groups;
     const int b = bh / p.H, h = bh % p.H;
-    const bool varlen = p.cu_seqlens != nullptr;
+    constexpr bool varlen = VARLEN;
     const int tok0 = varlen ? p.cu_seqlens[b] : g * p.group;
     const int tok1 = varlen ? p.cu_seqlens[b + 1] : min(p.N, tok0 + p.group);
     const int n_chunks = (tok1 - tok0 + kChunk - 1) / kChunk;
@@ -1183,9 +1186,9 @@ bool make_tile_map(CUtensorMap* map, const void* ptr, int B, int H, int N, int d
     return r == CUDA_SUCCESS;
 }
 
-template <int D, int MODE, int STREAM>
-cudaError_t launch_mode(const CUtensorMap* tm, const TcWalkParams& p, int BH, cudaStream_t st) {
-    auto kern = tc_walk_kernel<D, MODE, STREAM>;
+template <int D, int MODE, int STREAM, bool VARLEN>
+cudaError_t launch_mode_v(const CUtensorMap* tm, const TcWalkParams& p, int BH, cudaStream_t st) {
+    auto kern = tc_walk_kernel<D, MODE, STREAM, VARLEN>;
     // (the dV' stream has a plain epilogue, like the forward pass)
     constexpr bool with_proj = (MODE != MODE_STATE) && (STREAM == S_DQ || STREAM == S_DK);
     static bool configured = false;
@@ -1213,6 +1216,12 @@ cudaError_t launch_mode(const CUtensorMap* tm, const TcWalkParams& p, int BH, cu
     profile_end_launch(prof, st);
     note_launch();
     return le != cudaSuccess ? le : cudaGetLastError();
+}
+
+template <int D, int MODE, int STREAM>
+cudaError_t launch_mode(const CUtensorMap* tm, const TcWalkParams& p, int BH, cudaStream_t st) {
+    return p.cu_seqlens ? launch_mode_v<D, MODE, STREAM, true>(tm, p, BH, st)
+                        : launch_mode_v<D, MODE, STREAM, false>(tm, p, BH, st);
 }
 
 template <int D>
