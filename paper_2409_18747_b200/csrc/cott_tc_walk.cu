@@ -743,7 +743,9 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 }
                 COTT_STAMP_AT(4, c, 5);
             }
-            if (MODE != MODE_STATE) tma_store_wait_all0();
+            // (the stream that carries the dm sum drains its stores after the dm tail instead,
+            // so that the tail runs while the last store is still on its way)
+            if (MODE != MODE_STATE && p.dm_partial == nullptr) tma_store_wait_all0();
         }
     } else {
         // ------------------------------------------------------------------ row workers
@@ -806,11 +808,22 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 normalise_half_row(gbase + s * L::kStage + (kNormBv ? L::kOffB : L::kOffA), c);
             mbar_arrive(bar_a_ready + 8 * s);
         };
+        // Only streams whose X rows are normalised keep a scale per row; the others use c itself.
+        // Ordering of these shared-memory writes before the epilogue that reads them (other
+        // threads, other row mapping): when group P computes the scales, through its arrival on
+        // the masked-scores barrier of the same chunk.  When group O does: with a single output
+        // accumulator (d = 128) the scales of chunk c + 1 are written during iteration c, before
+        // the thread's arrival on `o_free` of chunk c, which X State of chunk c + 1 and hence
+        // its epilogue wait for -- so they may follow the tile's normalisation, off the path to
+        // the chunk's scores; chunk 0 has no such arrival and gets a barrier of the group
+        // instead.  With two accumulators `o_free` of chunk c does not gate chunk c + 1: there
+        // the scales come BEFORE the normalisation, whose arrival on `a_ready` the chunk's MMAs
+        // and hence its epilogue follow.
         auto x_scale = [&](int c) {
-            if (!L::kHasX) return;
+            if (!L::kHasX || !kXNorm) return;
             const int s = c % NST;
             float rx = cfac;
-            if (kXNorm) {
+            {
                 if (!wait(bar_full + 8 * s, (c / NST) & 1)) return;
                 const uint8_t* xt = gbase + s * L::kStage + L::kOffX;
                 float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
@@ -823,7 +836,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             }
             if (nhalf == 0) rx_buf[(c % NRX) * 128 + nrow] = rx;
         };
-        auto norm_phase = [&](int c) { norm_tile(c); if (alive) x_scale(c); };
+        auto norm_phase = [&](int c) { x_scale(c); if (alive) norm_tile(c); };
         // Split causal walk, Bv is the normalised operand (dQ^ and dK^ streams).
         auto norm_b = [&](int c) {
             const int s = c % NST;
@@ -919,30 +932,39 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             }
         } else {
             // -------------------------------------------------------------- group O
-            if (!kTileNormInP) norm_tile(0);
-            if (!kXScaleInP && alive) x_scale(0);
+            if (kOBufs == 1) {
+                if (!kTileNormInP) norm_tile(0);
+                if (!kXScaleInP && alive) x_scale(0);
+                // Chunk 0 has no earlier arrival of this group between these writes and the
+                // epilogue that reads them: the group meets once here.  Every thread of the
+                // group gets here exactly once (the waits above are bounded and return).
+                if (kXNorm && !kXScaleInP) asm volatile("bar.sync 1, %0;" ::"n"(kGroupThreads) : "memory");
+            } else {
+                if (!kXScaleInP) x_scale(0);
+                if (!kTileNormInP && alive) norm_tile(0);
+            }
             if (L::kSplitB && kNormBv && alive) norm_b(0);
             for (int c = 0; c < n_chunks && alive; ++c) {
                 const int s = c % NST;
                 uint8_t* st = gbase + s * L::kStage;
                 COTT_STAMP_AT(1, c, 0);
                 if (c + 1 < n_chunks) {
-                    if (!kTileNormInP) norm_tile(c + 1);
-                    if (!kXScaleInP && alive) x_scale(c + 1);
+                    if (kOBufs == 1) {
+                        if (!kTileNormInP) norm_tile(c + 1);
+                        if (!kXScaleInP && alive) x_scale(c + 1);
+                    } else {
+                        if (!kXScaleInP) x_scale(c + 1);
+                        if (!kTileNormInP && alive) norm_tile(c + 1);
+                    }
                     if (!alive) break;
                 }
                 COTT_STAMP_AT(1, c, 1);
                 // ---- output epilogue of chunk c: accumulator -> bf16 rows in the staging slot
                 if (!wait(ofull_bar(c), ofull_par(c))) break;
-                // The X scales of this chunk were written by threads of this group during the
-                // previous iteration, before their arrival on that chunk's epilogue barrier;
-                // with two output accumulators nothing else orders those writes before the
-                // read below.
-                if (own_out && !kXScaleInP && c >= 1 && !wait(edone_bar(c - 1), edone_par(c - 1))) break;
                 tc_fence_after();
                 COTT_STAMP_AT(1, c, 2);
                 const uint32_t tO = tmem + lane_base + colO0 + (c % kOBufs) * D + hf * HW;
-                const float rx = rx_buf[(c % NRX) * 128 + arow];
+                const float rx = kXNorm ? rx_buf[(c % NRX) * 128 + arow] : cfac;
                 uint32_t r[HW];
 #pragma unroll
                 for (int pc = 0; pc < NPIECE; ++pc)
@@ -1128,6 +1150,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             if (tid == 0) p.status[4] = 0;
         }
     }
+    if (MODE != MODE_STATE && p.dm_partial != nullptr && is_store && lane == 0) tma_store_wait_all0();
     if (*abort_flag) {
         // A wait gave up.  Before the CTA's shared memory and tensor memory go away, give the
         // copies and MMAs still in flight time to land (they need microseconds; nothing here
