@@ -34,12 +34,12 @@ L2_FLUSH_BYTES = 256 << 20  # larger than the 126 MB L2
 # DRAM bytes (read + write) per token-head of one causal-walk launch, from the ncu captures
 # summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum divided by the
 # token-heads of the captured launch); keyed by (d, causal).  Missing key: no capture yet.
-#   (64, causal):  mean of the four walk launches of a C4 step, 132.9 MB / 262144 token-heads
+#   (64, causal):  mean of the four walk launches of a C4 step, 132.1 MB / 262144 token-heads
 #                  (profiles/tc_walk_kernel_c4_d64.md)
-#   (128, causal): forward walk at B=1 H=16 N=16384, 252.5 MB / 262144 token-heads
+#   (128, causal): forward walk at B=1 H=16 N=16384, 251.7 MB / 262144 token-heads
 #                  (profiles/tc_walk_kernel_c5_n16384_d128.md); traffic grows with the number
 #                  of tokens, so the figure is scaled to the launch that was timed.
-KERNEL_DRAM_TRAFFIC = {(64, True): 507.0, (128, True): 963.0}
+KERNEL_DRAM_TRAFFIC = {(64, True): 504.0, (128, True): 960.0}
 
 
 def load_peaks():
