@@ -77,6 +77,37 @@ def test_argument_validation_returns_before_any_launch():
                         ctypes.byref(sp), a, 1 << 24, null) == -1
 
 
+def test_strided_and_packed_entry_points_validate_on_the_host():
+    """cott_*_strided and cott_*_varlen refuse strides and shapes they cannot address before
+    anything is launched (fake addresses, never dereferenced)."""
+    lib = cott._load()
+    sp = cott._ScaleParams()
+    sp.m, sp.seq_len, sp.seq_len_scalar = 256, None, 0.0
+    a, null = 4096, None
+    S = cott._Strides
+    ok = S(16 * 2 * 64, 64, 2 * 64)           # [B,N,H,d] with H=2, d=64, N=16
+    args = (a, a, a, a + 65536, null, 1, 2, 16, 64, 1, cott.BF16)
+    tail = (ctypes.byref(sp), a, 1 << 20, null)
+    # token stride not a multiple of 16 bytes / smaller than a row
+    assert lib.cott_fwd_strided(*args, ctypes.byref(S(4096, 64, 132)), None, *tail) == -2
+    assert lib.cott_fwd_strided(*args, ctypes.byref(S(4096, 64, 32)), None, *tail) == -2
+    assert lib.cott_fwd_strided(*args, None, ctypes.byref(S(4096, 8, 128)), *tail) == -2
+    # good strides get as far as the workspace check
+    assert lib.cott_fwd_strided(*args, ctypes.byref(ok), ctypes.byref(ok), ctypes.byref(sp), null, 0, null) == -3
+    bargs = (a, a, a, a, a + 65536, a + 131072, a + 196608, a, 1, 2, 16, 64, 1, cott.BF16)
+    assert lib.cott_bwd_strided(*bargs, None, None, ctypes.byref(S(4096, 64, 130)), ctypes.byref(sp), a, 1 << 24, null) == -2
+    assert lib.cott_bwd_strided(*bargs, ctypes.byref(ok), None, ctypes.byref(ok), ctypes.byref(sp), null, 0, null) == -3
+    # packed batches: NULL cu_seqlens, fp32 or d = 32 (tensor-core path only), max_seqlen > total
+    v = (a, a, a, a + 65536)
+    assert lib.cott_fwd_varlen(*v, null, 2, 2, 100, 60, 64, 1, cott.BF16, *tail) == -1
+    assert lib.cott_fwd_varlen(*v, a, 2, 2, 100, 60, 64, 1, cott.F32, *tail) == -2
+    assert lib.cott_fwd_varlen(*v, a, 2, 2, 100, 60, 32, 1, cott.BF16, *tail) == -2
+    assert lib.cott_fwd_varlen(*v, a, 2, 2, 100, 200, 64, 1, cott.BF16, *tail) == -2
+    assert lib.cott_fwd_varlen(*v, a, 2, 2, 100, 60, 64, 1, cott.BF16, ctypes.byref(sp), null, 0, null) == -3
+    assert lib.cott_bwd_varlen(a, a, a, a, a + 65536, a + 131072, a + 196608, a, null, 2, 2, 100, 60, 64, 1,
+                               cott.BF16, ctypes.byref(sp), a, 1 << 24, null) == -1
+
+
 def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(cott, "_lib", None)
     monkeypatch.setattr(cott, "_LIB_PATH", "/nonexistent/libcott.so")

@@ -747,3 +747,30 @@ def test_packed_varlen_with_empty_sequences():
         for x, y in zip(ga[:3], gb[:3]):
             assert torch.equal(x, y)
         torch.testing.assert_close(ga[3], gb[3], rtol=1e-3, atol=1e-3 * float(gb[3].abs().max()))
+
+
+def test_packed_varlen_with_given_scaling_bases():
+    """Per-sequence scaling bases passed by the caller (sp->seq_len) instead of the lengths."""
+    H, d, lens = 2, 64, (150, 260)
+    bases = np.array([512.0, 1024.0])
+    seqs = [synth.make_qkv(1, H, L, d, torch.bfloat16, 5900 + L, with_do=True) for L in lens]
+    for s_ in seqs:
+        s_["m"] = seqs[0]["m"]
+    cat = lambda key: torch.cat([s_[key][0].permute(1, 0, 2) for s_ in seqs], dim=0).contiguous().cuda()
+    q, k, v, d_o = (cat(x) for x in ("q", "k", "v", "d_o"))
+    cu = torch.tensor([0, 150, 410], dtype=torch.int32, device="cuda")
+    m = dev(seqs[0]["m"])
+    sl = torch.tensor(bases, dtype=torch.float32, device="cuda")
+    o = cott.fwd_varlen(q, k, v, m, cu, 260, seq_len=sl)
+    dq, dk, dv, dm = cott.bwd_varlen(q, k, v, d_o, m, cu, 260, seq_len=sl)
+    off, dm_ref, conds = 0, np.zeros(H), np.zeros(H)
+    for s_, L, base in zip(seqs, lens, bases):
+        sb = np.array([base])
+        ref = oracle.fwd_quadratic(s_["q"], s_["k"], s_["v"], s_["m"], sb, True)
+        rq, rk, rv, rm = oracle.bwd_quadratic(s_["q"], s_["k"], s_["v"], s_["d_o"], s_["m"], sb, True)
+        un = lambda x: x[off:off + L].permute(1, 0, 2)[None]
+        gate(un(o), ref, torch.bfloat16)
+        gate(un(dq), rq, torch.bfloat16); gate(un(dk), rk, torch.bfloat16); gate(un(dv), rv, torch.bfloat16)
+        dm_ref += rm; conds += dm_condition(rv, s_["v"], s_["m"], sb)
+        off += L
+    gate_dm(dm, dm_ref, 1e-2, conds, DM_COND_BF16)
