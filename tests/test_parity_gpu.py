@@ -774,3 +774,36 @@ def test_packed_varlen_with_given_scaling_bases():
         dm_ref += rm; conds += dm_condition(rv, s_["v"], s_["m"], sb)
         off += L
     gate_dm(dm, dm_ref, 1e-2, conds, DM_COND_BF16)
+
+
+_FIRST_CALL_SCRIPT = r"""
+import sys, torch
+sys.path.insert(0, sys.argv[1])
+import paper_2409_18747_b200 as cott
+from paper_2409_18747_b200 import synth
+bad = 0
+for (B, H, N, d, causal) in ((2, 5, 333, 128, False), (2, 5, 333, 128, True), (2, 5, 333, 64, False)):
+    c = synth.make_qkv(B, H, N, d, torch.bfloat16, 6000 + d, with_do=True)
+    q, k, v, d_o, m = (c[x].cuda() for x in ("q", "k", "v", "d_o", "m"))
+    runs = []
+    for _ in range(4):
+        o = cott.fwd(q, k, v, m, causal=causal)
+        runs.append((o,) + tuple(cott.bwd(q, k, v, d_o, m, causal=causal)))
+    torch.cuda.synchronize()
+    bad += sum(not torch.equal(x, y) for r in runs[:-1] for x, y in zip(r, runs[-1]))
+print("MISMATCH" if bad else "SAME")
+"""
+
+
+def test_first_calls_of_a_fresh_process_equal_later_ones():
+    """The first launches of a process run with cold instruction caches and skewed warps: a
+    hand-off that is only ordered by luck shows there first (this caught row scales read before
+    they were written).  Six fresh processes; in each, every call must equal the last one bit for bit."""
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    for _ in range(6):
+        out = subprocess.run([sys.executable, "-c", _FIRST_CALL_SCRIPT, root], capture_output=True, text=True,
+                             timeout=300)
+        assert out.returncode == 0, out.stderr[-2000:]
+        assert out.stdout.strip().endswith("SAME"), out.stdout[-500:]
