@@ -160,6 +160,13 @@ cott_status cott_fwd_stateful(const void* q, const void* k, const void* v, void*
                               cott_dtype dt, const cott_scale_params* sp, void* workspace,
                               size_t workspace_bytes, void* stream);
 
+/* cott_fwd_stateful on tensors that are not dense [B,H,N,d]; strides as for cott_fwd_strided. */
+cott_status cott_fwd_stateful_strided(const void* q, const void* k, const void* v, void* o,
+                                      const float* state_in, float* state_out, int B, int H, int N,
+                                      int d, cott_dtype dt, const cott_strides* qkv_strides,
+                                      const cott_strides* o_strides, const cott_scale_params* sp,
+                                      void* workspace, size_t workspace_bytes, void* stream);
+
 /*
  * Backward pass of cott_fwd for L = sum(d_o * O): the gradient formulas printed after Eq. 7
  * (dQ^ = (dO V'^T . M) K^, dK^ = (dO V'^T . M)^T Q^, dV' = (Q^ K^^T . M)^T dO; M all-ones when

@@ -78,6 +78,9 @@ def _load():
     lib.cott_bwd_varlen.restype = ci
     lib.cott_bwd_varlen.argtypes = [vp] * 9 + [ci, ci, ci, ci, ci, ci, ci,
                                                 ctypes.POINTER(_ScaleParams), vp, cs, vp]
+    lib.cott_fwd_stateful_strided.restype = ci
+    lib.cott_fwd_stateful_strided.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, vp, vp,
+                                              ctypes.POINTER(_ScaleParams), vp, cs, vp]
     lib.cott_fwd_stateful.restype = ci
     lib.cott_fwd_stateful.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci,
                                       ctypes.POINTER(_ScaleParams), vp, cs, vp]
@@ -212,7 +215,8 @@ def fwd_stateful(q, k, v, m, seq_len, state_in=None, return_state=True, out=None
     (fp32 ``[B,H,d,d]`` or None) is the state the previous segment (or a decode step) left;
     ``seq_len`` (a float >= 1 or a float32 ``[B]`` CUDA tensor) is the scaling base of the WHOLE
     sequence and must be the same for all its segments.  Returns ``(o, state)`` or ``o``."""
-    _check_dev(q, k, v, m, state_in, seq_len if isinstance(seq_len, torch.Tensor) else None)
+    _check_rows(q, k, v)
+    _check_dev(m, state_in, seq_len if isinstance(seq_len, torch.Tensor) else None)
     if seq_len is None:
         raise ValueError("fwd_stateful needs the scaling base of the whole sequence")
     B, H, N, d = q.shape
@@ -221,14 +225,17 @@ def fwd_stateful(q, k, v, m, seq_len, state_in=None, return_state=True, out=None
         raise ValueError("state_in must be float32 [B,H,d,d]")
     o = torch.empty_like(q) if out is None else out
     state = torch.empty((B, H, d, d), dtype=torch.float32, device=q.device) if return_state else None
+    _check_rows(o)
+    s_qkv, s_o = _strides_of(q, k, v), _strides_of(o)
     ws, ws_bytes = _workspace(OP_FWD, dt, B, H, N, d, True, q.device, workspace)
     sp = _scale(m, seq_len)
-    rc = _load().cott_fwd_stateful(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
-                                   state_in.data_ptr() if state_in is not None else None,
-                                   state.data_ptr() if state is not None else None, B, H, N, d, dt,
-                                   ctypes.byref(sp), ws.data_ptr(), ws_bytes, _stream_ptr(stream))
+    rc = _load().cott_fwd_stateful_strided(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
+                                           state_in.data_ptr() if state_in is not None else None,
+                                           state.data_ptr() if state is not None else None, B, H, N, d, dt,
+                                           _ref(s_qkv), _ref(s_o), ctypes.byref(sp), ws.data_ptr(), ws_bytes,
+                                           _stream_ptr(stream))
     if rc != 0:
-        raise CottError(rc, "cott_fwd_stateful")
+        raise CottError(rc, "cott_fwd_stateful_strided")
     return (o, state) if return_state else o
 
 

@@ -558,7 +558,17 @@ cott_status cott_fwd_stateful(const void* q, const void* k, const void* v, void*
                               const float* state_in, float* state_out, int B, int H, int N, int d,
                               cott_dtype dt, const cott_scale_params* sp, void* workspace,
                               size_t workspace_bytes, void* stream) {
+    return cott_fwd_stateful_strided(q, k, v, o, state_in, state_out, B, H, N, d, dt, nullptr, nullptr, sp,
+                                     workspace, workspace_bytes, stream);
+}
+
+cott_status cott_fwd_stateful_strided(const void* q, const void* k, const void* v, void* o,
+                                      const float* state_in, float* state_out, int B, int H, int N,
+                                      int d, cott_dtype dt, const cott_strides* qkv_strides,
+                                      const cott_strides* o_strides, const cott_scale_params* sp,
+                                      void* workspace, size_t workspace_bytes, void* stream) {
     if (!q || !k || !v || !o || B < 1 || H < 1 || N < 1) return COTT_ERR_INVALID_ARG;
+    if (!layout_ok(qkv_strides, d, dt) || !layout_ok(o_strides, d, dt)) return COTT_ERR_UNSUPPORTED;
     if (check_scale(sp) != COTT_OK) return COTT_ERR_INVALID_ARG;
     if (o == q || o == k || o == v) return COTT_ERR_INVALID_ARG;
     if (state_in && state_in == state_out) return COTT_ERR_INVALID_ARG;
@@ -573,7 +583,7 @@ cott_status cott_fwd_stateful(const void* q, const void* k, const void* v, void*
         workspace_bytes < workspace_bytes_impl(COTT_OP_FWD, p, B, H, d))
         return COTT_ERR_WORKSPACE;
     return fwd_impl(q, k, v, o, state_out, B, H, N, d, 1, dt, sp, workspace, p,
-                    static_cast<cudaStream_t>(stream), state_in);
+                    static_cast<cudaStream_t>(stream), state_in, qkv_strides, o_strides);
 }
 
 cott_status cott_bwd(const void* q, const void* k, const void* v, const void* d_o, void* dq,

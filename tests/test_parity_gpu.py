@@ -807,3 +807,23 @@ def test_first_calls_of_a_fresh_process_equal_later_ones():
                              timeout=300)
         assert out.returncode == 0, out.stderr[-2000:]
         assert out.stdout.strip().endswith("SAME"), out.stdout[-500:]
+
+
+@pytest.mark.parametrize("dtype,d", [(torch.bfloat16, 64), (torch.float32, 32)])
+def test_stateful_segments_on_strided_tensors(dtype, d):
+    """cott_fwd_stateful_strided: segments cut out of [B,N,H,d] storage (views, no copies) give
+    the same rows and the same final state, bit for bit, as contiguous copies of the segments."""
+    B, H, N = 2, 3, 700
+    c = synth.make_qkv(B, H, N, d, dtype, 6100 + d)
+    q, k, v, m = (dev(c[x]) for x in ("q", "k", "v", "m"))
+    qb, kb, vb = (_as_bnhd(x) for x in (q, k, v))
+    cuts = [0, 130, 131, 512, 700]
+    st_a = st_b = None
+    for a, b in zip(cuts[:-1], cuts[1:]):
+        seg = lambda x: x[:, :, a:b]
+        oa, st_a = cott.fwd_stateful(seg(q).contiguous(), seg(k).contiguous(), seg(v).contiguous(), m, float(N),
+                                     state_in=st_a)
+        ob, st_b = cott.fwd_stateful(seg(qb), seg(kb), seg(vb), m, float(N), state_in=st_b,
+                                     out=torch.empty_like(oa))
+        assert not seg(qb).is_contiguous()
+        assert torch.equal(oa, ob) and torch.equal(st_a, st_b)
