@@ -8,8 +8,9 @@
  *
  * Symbols: B batch, H heads, N sequence length, d per-head dimension (one d for
  * keys and values).  q,k,v,o,d_o,dq,dk,dv are contiguous row-major [B,H,N,d] in
- * the I/O dtype `dt`; decode tensors are [B,H,d]; `m`, `seq_len`, `state`, `dm`
- * are always fp32.
+ * the I/O dtype `dt` (the *_strided entry points take other strides, the *_varlen
+ * ones sequences of different lengths packed into [total_tokens,H,d]); decode
+ * tensors are [B,H,d]; `m`, `seq_len`, `state`, `dm` are always fp32.
  *
  * What is computed (paper equations):
  *   x^      = x / max(||x||_2, 1e-12)            row normalisation of Q and K (Eq. 2, Eq. 3)
