@@ -525,6 +525,10 @@ def run_ours(args, w):
         dom_ms = statistics.mean(walk_ms)
         kernel = f"tc_walk_kernel<{d},{1 if w['causal'] else 2}> (tcgen05 chunk walk), mean of {len(walk_ms)} launches"
         traffic = KERNEL_DRAM_TRAFFIC.get((d, bool(w["causal"])), None)
+        if w.get("varlen"):
+            # mean of the four walk launches of a step of this workload, 1468 MB / 1255520
+            # token-heads (profiles/tc_walk_kernel_varlen_d128.md)
+            traffic = 1169.0
         traffic = traffic * (w.get("rows", B * N) * H) if traffic else None
     else:
         alg = ab["fwd"]
