@@ -70,11 +70,29 @@ const char* cott_last_cuda_error(void);
 unsigned long long cott_launch_count(void);
 
 /*
+ * Process-wide switches for tests and measurements (none is needed in use).  Each starts from
+ * an environment variable that is read once, on first use, and can be changed at any time
+ * with cott_set_option (takes effect for calls issued afterwards; not synchronised with calls
+ * in flight on other host threads).  Names (environment variable, default):
+ *   "force_group"        (COTT_FORCE_GROUP, 0)        tokens per sequence group; 0 = the plan's choice
+ *   "force_path"         (COTT_FORCE_PATH, 1)         0 = bf16 d = 64 / 128 through the fp32-accumulating SIMT kernels
+ *   "pair"               (COTT_PAIR, 1)               0 = gradient streams one after the other where they would run side by side
+ *   "fused_bwd"          (COTT_FUSED_BWD, 1)          0 = causal d = 64 backward as three role-swapped walks instead of one fused walk
+ *   "wait_limit_ms"      (COTT_WAIT_LIMIT_MS, 2000)   bound of every device-side wait
+ *   "wait_limit_kcycles" (COTT_WAIT_LIMIT_KCYCLES, -1) the same bound in units of 1024 SM cycles; negative = use the millisecond
+ *                        value; 0 = every wait that is not met within a few polls gives up (the timeout test)
+ * cott_set_option returns COTT_ERR_INVALID_ARG for an unknown name; cott_get_option returns -1.
+ * No paper passage: library plumbing.
+ */
+cott_status cott_set_option(const char* name, long long value);
+long long cott_get_option(const char* name);
+
+/*
  * Per-launch timing of the tensor-core walk kernels, for benchmarks.  cott_profile_enable(n)
  * with n > 0 starts recording a pair of library-owned CUDA events around each of the next n
  * (at most 256) walk-kernel launches; n <= 0 stops.  cott_profile_read waits for the recorded
  * launches and writes their durations in milliseconds to ms[] and their kind to kinds[]
- * (0 = partial-state pass, 1 = causal walk, 2 = read-out; 17 = a causal walk that ran side by
+ * (0 = partial-state pass, 1 = causal walk, 2 = read-out, 3 = fused causal backward walk; 17 = a causal walk that ran side by
  * side with a sibling walk of the same size on another stream of the library, in which case
  * its ms is half of the span the pair occupied, first start to last end); both are host
  * arrays of `cap` entries.  Returns the number of entries written, or -1 on a CUDA error.  Not thread-safe

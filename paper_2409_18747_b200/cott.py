@@ -97,6 +97,10 @@ def _load():
     lib.cott_fwd_noalloc.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ctypes.POINTER(_ScaleParams), vp]
     lib.cott_last_async_status.restype = ci
     lib.cott_last_async_status.argtypes = [vp, vp]
+    lib.cott_set_option.restype = ci
+    lib.cott_set_option.argtypes = [ctypes.c_char_p, ctypes.c_longlong]
+    lib.cott_get_option.restype = ctypes.c_longlong
+    lib.cott_get_option.argtypes = [ctypes.c_char_p]
     _lib = lib
     return lib
 
@@ -158,6 +162,17 @@ def _scale(m: torch.Tensor, seq_len, scalar: float = 0.0) -> _ScaleParams:
     sp.seq_len = seq_len.data_ptr() if isinstance(seq_len, torch.Tensor) else None
     sp.seq_len_scalar = float(seq_len) if (seq_len is not None and not isinstance(seq_len, torch.Tensor)) else scalar
     return sp
+
+
+def set_option(name: str, value: int) -> None:
+    """cott_set_option: a process-wide switch for tests and measurements (see ``cott.h``)."""
+    rc = _load().cott_set_option(name.encode(), int(value))
+    if rc != 0:
+        raise CottError(rc, f"cott_set_option({name})")
+
+
+def get_option(name: str) -> int:
+    return int(_load().cott_get_option(name.encode()))
 
 
 def workspace_bytes(op: int, dt: int, B: int, H: int, N: int, d: int, causal: bool) -> int:

@@ -4,6 +4,9 @@
 #include <stdlib.h>
 #include <string.h>
 #include <atomic>
+#include <mutex>
+#include <utility>
+#include <vector>
 #include "cott_internal.h"
 
 namespace cott {
@@ -47,9 +50,56 @@ static cott_status cuda_fail(cudaError_t e, const char* where) {
         if (e__ != cudaSuccess) return cuda_fail(e__, #expr);    \
     } while (0)
 
-static int env_int(const char* name, int dflt) {
-    const char* v = getenv(name);
-    return (v && *v) ? atoi(v) : dflt;
+// ---- options: process-wide switches for tests and measurements (none is needed in use).
+// Each starts from its environment variable, read once on first use, and can be changed with
+// cott_set_option.
+struct Option {
+    const char* name; const char* env; long long dflt;
+    std::atomic<long long> value;
+    std::once_flag once;
+    Option(const char* n, const char* e, long long d) : name(n), env(e), dflt(d), value(d) {}
+    long long get() {
+        std::call_once(once, [this] {
+            const char* v = getenv(env);
+            if (v && *v) value.store(atoll(v), std::memory_order_relaxed);
+        });
+        return value.load(std::memory_order_relaxed);
+    }
+    void set(long long v) { get(); value.store(v, std::memory_order_relaxed); }
+};
+static Option g_opt_force_group("force_group", "COTT_FORCE_GROUP", 0);     // tokens per sequence group (0: the plan's)
+static Option g_opt_force_path("force_path", "COTT_FORCE_PATH", 1);        // 0: bf16 d=64/128 through the fp32-accumulating SIMT kernels
+static Option g_opt_pair("pair", "COTT_PAIR", 1);                          // 0: gradient streams one after the other
+static Option g_opt_fused_bwd("fused_bwd", "COTT_FUSED_BWD", 1);           // 0: causal d=64 backward through the three role-swapped walks
+static Option g_opt_wait_ms("wait_limit_ms", "COTT_WAIT_LIMIT_MS", 2000);  // bound of every device-side wait
+static Option g_opt_wait_kc("wait_limit_kcycles", "COTT_WAIT_LIMIT_KCYCLES", -1);  // the same in units of 1024 SM cycles (< 0: use the ms value)
+static Option* const g_options[] = {&g_opt_force_group, &g_opt_force_path, &g_opt_pair, &g_opt_fused_bwd,
+                                    &g_opt_wait_ms, &g_opt_wait_kc};
+
+int option_force_group() { return (int)g_opt_force_group.get(); }
+int option_force_path() { return (int)g_opt_force_path.get(); }
+int option_pair() { return (int)g_opt_pair.get(); }
+int option_fused_bwd() { return (int)g_opt_fused_bwd.get(); }
+int wait_limit_kcycles() {
+    const long long kc = g_opt_wait_kc.get();
+    if (kc >= 0) return (int)(kc > 200000000 ? 200000000 : kc);
+    const long long ms = g_opt_wait_ms.get();
+    return (int)((ms < 1 ? 1 : (ms > 100000 ? 100000 : ms)) * 2000);   // <= 2 GHz
+}
+
+cudaError_t configure_smem_once(const void* func, int bytes) {
+    static std::mutex mu;
+    static std::vector<std::pair<const void*, int>> done;      // (kernel, device) pairs already configured
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> lock(mu);
+    for (const auto& it : done)
+        if (it.first == func && it.second == dev) return cudaSuccess;
+    e = cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e != cudaSuccess) return e;
+    done.emplace_back(func, dev);
+    return cudaSuccess;
 }
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -73,9 +123,9 @@ static bool make_plan(int op, cott_dtype dt, int B, int H, int N, int d, int cau
     if (d != 32 && d != 64 && d != 128) return false;
     if (dt != COTT_F32 && dt != COTT_BF16) return false;
     const long BH = (long)B * H;
-    const int forced = env_int("COTT_FORCE_GROUP", 0);
+    const int forced = option_force_group();
     const bool tc_ok = dt == COTT_BF16 && (d == 64 || d == 128);
-    p->path = (tc_ok && env_int("COTT_FORCE_PATH", 1) != 0) ? 1 : 0;
+    p->path = (tc_ok && option_force_path() != 0) ? 1 : 0;
     int group;
     if (p->path == 1) {
         // One CTA per (b,h) and group, one CTA per SM.  Measured on B200: fewer, longer
@@ -128,7 +178,7 @@ static size_t workspace_bytes_impl(int op, const Plan& p, int B, int H, int d) {
     size_t total = kWsHeaderBytes;
     if (op == COTT_OP_FWD) total += states_bytes(p, B, H, d);
     else if (op == COTT_OP_BWD)
-        total += 3 * states_bytes(p, B, H, d) + align_up((size_t)B * H * p.n_groups * 4, 256);
+        total += 3 * states_bytes(p, B, H, d) + 2 * align_up((size_t)B * H * p.n_groups * 4, 256);
     return total;
 }
 
@@ -334,6 +384,7 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
     float* st1 = reinterpret_cast<float*>(base + sb);
     float* st2 = reinterpret_cast<float*>(base + 2 * sb);
     float* dm_partial = reinterpret_cast<float*>(base + 3 * sb);
+    float* dm_partial2 = dm_partial + align_up((size_t)B * H * p.n_groups * 4, 256) / 4;
     const int BH = B * H;
     cott_status rc;
     if (p.path == 1) {
@@ -346,12 +397,30 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
         // over the whole sequence as a single group (no partial-state pass, no scan), with the
         // dQ^ stream's partial-state pass filling the SMs that are left; the dQ^ walk follows on
         // the whole GPU.  Each side stream then carries one tensor-core kernel per call.
+        if (causal && d == 64 && !packed.cu_seqlens && option_fused_bwd() != 0) {
+            // One walk forward in time gives all three gradients and the dm sum (cott_tc_bwd.cu).
+            // It keeps two running states: Sq = V^T K^ over earlier tokens, accumulated chunk by
+            // chunk, and R = Q^^T dO over later tokens, which starts at the sum over the group
+            // and everything after it and is taken down as the walk passes.  Before it, one
+            // state-only launch gives both partial states of every group.
+            TcBwdFusedArgs f;
+            memset(&f, 0, sizeof(f));
+            f.q = q; f.k = k; f.v = v; f.d_o = d_o; f.dq = dq; f.dk = dk; f.dv = dv;
+            f.l_qkv = lay.qkv; f.l_do = lay.o; f.l_dqkv = lay.dqkv;
+            f.sq_part = st0; f.r_part = st1;
+            f.dm_partial = dm_partial; f.dm_out = dm; f.status = status;
+            f.m = sp->m; f.seq_len = sp->seq_len; f.seq_len_scalar = sp->seq_len_scalar;
+            f.group = p.group; f.n_groups = p.n_groups;
+            COTT_CUDA(launch_tc_bwd_states(f, st0, st1, 1, B, H, N, st));
+            COTT_CUDA(launch_tc_bwd_fused(f, B, H, N, st));
+            return COTT_OK;
+        }
         SideStreams* ss = nullptr;
         Plan pp = p;                       // plan of the two side-by-side streams
         // (d = 64 only: at d = 128 two such walks running at the same time ended in a launch
         // failure once in a dozen calls, for a reason that reading the kernel has not shown;
         // one after the other the same kernels have run hundreds of thousands of times.)
-        if (causal && d == 64 && p.n_groups >= 2 && 2 * BH <= 148 && 74 / BH == 1 && env_int("COTT_PAIR", 1) != 0) {
+        if (causal && d == 64 && p.n_groups >= 2 && 2 * BH <= 148 && 74 / BH == 1 && option_pair() != 0) {
             pp.group = (N + 127) / 128 * 128;
             pp.n_groups = 1; pp.split = 1;
             ss = side_streams();
@@ -403,8 +472,14 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
             COTT_CUDA(cudaStreamWaitEvent(st, ss->join[1], 0));
             if ((rc = run_tc_stream(tq, p, B, H, N, d, causal, sp, status, st0, nullptr, st, true, false, false)) != COTT_OK) return rc;
         } else {
-            if ((rc = run_tc_stream(tq, p, B, H, N, d, causal, sp, status, st0, nullptr, st)) != COTT_OK) return rc;
+            // The dK^ stream goes first: it also sums the first-order term by which the dQ^
+            // stream's dm sum is off because that stream multiplies by k^ rounded to bf16; the
+            // dQ^ stream, second, adds the two parts when it finalises dm.
+            tk.clear_status = 1; tq.clear_status = 0;
+            tk.dm_partial = dm_partial2; tk.dm_out = nullptr;
+            tq.dm_extra = dm_partial2;
             if ((rc = run_tc_stream(tk, p, B, H, N, d, causal, sp, status, st1, nullptr, st)) != COTT_OK) return rc;
+            if ((rc = run_tc_stream(tq, p, B, H, N, d, causal, sp, status, st0, nullptr, st)) != COTT_OK) return rc;
             // The dV' state sum_t q^_t dO_t^T is the transpose of the dK^ stream's
             // sum_t dO_t q^_t^T, accumulated in the same direction: reuse those group states
             // instead of a third pass.
@@ -500,6 +575,20 @@ int cott_profile_read(float* ms, int* kinds, int cap) {
         }
     }
     return n;
+}
+
+cott_status cott_set_option(const char* name, long long value) {
+    if (!name) return COTT_ERR_INVALID_ARG;
+    for (Option* o : g_options)
+        if (strcmp(o->name, name) == 0) { o->set(value); return COTT_OK; }
+    return COTT_ERR_INVALID_ARG;
+}
+
+long long cott_get_option(const char* name) {
+    if (!name) return -1;
+    for (Option* o : g_options)
+        if (strcmp(o->name, name) == 0) return o->get();
+    return -1;
 }
 
 unsigned long long cott_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

@@ -1,5 +1,6 @@
 // Internal declarations shared by the translation units of libcott.
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
@@ -74,6 +75,7 @@ struct TcWalkArgs {
     // total_tokens rows per head (batch stride unused); one group per (b, h).  NULL: dense batch.
     const int* cu_seqlens; int total_tokens;
     const float* init; float* state_out; float* dm_partial; int* status;
+    const float* dm_extra;   // the stream that finalises dm: the [BH, n_groups] part another stream summed, or NULL
     const float* m; const float* seq_len; float seq_len_scalar;
     int group; int n_groups;
     int norm_bv; int x_norm; int epilogue; int reverse;
@@ -105,6 +107,41 @@ struct TcWalkArgs {
     float* state_final;
 };
 cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cudaStream_t st);
+
+// Fused causal backward at d = 64 (cott_tc_bwd.cu): one walk forward in time over every group
+// produces dq, dk, dv and the dm sum.  sq_part / r_part are the partial states of the groups
+// (V^T K^ and Q^^T dO), written by launch_tc_bwd_states: a group reads sq_part of the groups
+// before it and r_part of itself and the groups after it.
+struct TcBwdFusedArgs {
+    const void* q; const void* k; const void* v; const void* d_o;
+    void* dq; void* dk; void* dv;
+    RowLayout l_qkv, l_do, l_dqkv;
+    const float* sq_part; const float* r_part;
+    float* dm_partial; float* dm_out; int* status;
+    const float* m; const float* seq_len; float seq_len_scalar;
+    int group; int n_groups;
+    int plain_launch;
+};
+cudaError_t launch_tc_bwd_fused(const TcBwdFusedArgs& a, int B, int H, int N, cudaStream_t st);
+// Both partial states of every group in one launch (uses q, k, v, d_o, the layouts, group,
+// n_groups and status of `a`); clear_status: this is the first kernel of a library call.
+cudaError_t launch_tc_bwd_states(const TcBwdFusedArgs& a, float* sq_out, float* r_out, int clear_status, int B, int H,
+                                 int N, cudaStream_t st);
+
+// Tensor map over a bf16 tensor of logical shape [B,H,N,d] with the given row layout: box of
+// 128 tokens x 64 columns of one (b,h), 128-byte swizzle (see cott_tc_walk.cu).
+bool make_tile_map(CUtensorMap* map, const void* ptr, int B, int H, int N, int d, const RowLayout& lay,
+                   bool* head_first);
+
+// Opt-in to `bytes` of dynamic shared memory for a kernel, once per (kernel, device).
+cudaError_t configure_smem_once(const void* func, int bytes);
+
+// Library options (cott_set_option; environment variables give the defaults, read once).
+int option_force_group();
+int option_force_path();
+int option_pair();
+int option_fused_bwd();
+int wait_limit_kcycles();      // bound of every device-side wait, in units of 1024 SM cycles
 
 cudaError_t launch_dm_finalize(const float* dm_partial, float* dm, const float* m,
                                const float* seq_len, float seq_len_scalar, int B, int H,

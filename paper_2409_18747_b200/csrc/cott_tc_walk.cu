@@ -39,7 +39,8 @@ struct TcWalkParams {
                             // states, to be summed here over the groups before (after, when
                             // time runs backward; all, for the read-out) this one
     float* state_out;       // MODE_STATE: [BH, n_groups, d*d] partial states (unscaled)
-    float* dm_partial;      // the stream that carries the dm sum: [BH, n_groups]
+    float* dm_partial;      // a stream that carries a part of the dm sum: [BH, n_groups]
+    const float* dm_extra;  // the finalising stream: the other stream's [BH, n_groups] part, or NULL
     float* dm_out;          // that stream: dm[H], written by the CTA that finishes last (or NULL)
     int init_has_scale;     // init is a caller's state (contains c): divide by c on the way in
     float* state_final;     // causal walk, one group: [BH, d*d] state after the last token, times c (or NULL)
@@ -50,7 +51,9 @@ struct TcWalkParams {
     int plain_launch;                   // host side only: launch without programmatic serialization
     int clear_status;                   // first kernel of a call: CTA 0 zeroes the status words
     int wait_limit_kcycles;             // bound of every wait, in units of 1024 SM cycles
-    int debug_drop_commit;              // test hook: the scores of chunk 1 are never reported complete
+#ifdef COTT_TEST_HOOKS
+    int debug_drop_commit;              // test builds only: the scores of chunk 1 are never reported complete
+#endif
     // Packed variable-length batch: rows of all sequences back to back in one [T, H, d]
     // tensor, sequence b = rows cu_seqlens[b] .. cu_seqlens[b+1]-1, one group per (b, h).
     const int* cu_seqlens;              // NULL: every (b, h) has N rows of its own
@@ -216,7 +219,7 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, vol
     const long long t0 = clock64();   // SM cycle counter: far cheaper to read than the global timer
     for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 15u) == 0) {
+        if ((it & 15u) == 1) {
             if (*abort_flag) return false;
             // the limit (in units of 1024 SM cycles) sits three words behind the abort flag
             if (clock64() - t0 > ((long long)abort_flag[3] << 10)) {
@@ -587,7 +590,10 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 const int s = c % NST;
                 tc_fence_after();
                 issue_p<D>(tmem + colP, stage_x(s), stage_a(s));
-                if (!(p.debug_drop_commit && c == 1)) tc_commit(bar_p_full);
+                #ifdef COTT_TEST_HOOKS
+                if (!(p.debug_drop_commit && c == 1))
+#endif
+                tc_commit(bar_p_full);
             };
             auto batch1 = [&](int c, bool scores_issued) {
                 const int s = c % NST;
@@ -1010,6 +1016,27 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                         // <q^_i, dQ^_i> of the unscaled accumulator, once per row (see kEpi)
                         if (STREAM == S_DQ && hf == 0 && !(varlen && chunk_row(c) + arow >= tok1))
                             dm_acc += dp * rp;
+                        // The dQ^ stream's sum uses k^ rounded to bf16 (its Bv operand).  To first
+                        // order the sum with the exact k^ is larger by sum_j <k^_j - bf16(k^_j), dK^_j>,
+                        // and this stream has both factors: the raw k rows and the dK^ accumulator.
+                        // dm is a heavily cancelling sum, so this rounding is its largest error.
+                        if (STREAM == S_DK && p.dm_partial != nullptr && !(varlen && chunk_row(c) + arow >= tok1)) {
+                            const float rpe = nrm > kEps ? rp : 0.f;     // (a clamped row has no such term worth keeping)
+                            float c0 = 0.f, c1 = 0.f;
+#pragma unroll
+                            for (int i = 0; i < HW; i += 8) {
+                                const uint4 w = proj_chunk(i);
+                                const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&w);
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) {
+                                    const float2 f = __bfloat1622float2(e[j]);
+                                    const float kx = f.x * rpe, ky = f.y * rpe;
+                                    c0 = fmaf(kx - __bfloat162float(__float2bfloat16_rn(kx)), __uint_as_float(r[i + 2 * j]), c0);
+                                    c1 = fmaf(ky - __bfloat162float(__float2bfloat16_rn(ky)), __uint_as_float(r[i + 2 * j + 1]), c1);
+                                }
+                            }
+                            dm_acc += c0 + c1;
+                        }
                     }
                 }
                 // Scale, (project,) round to bf16, stage for the TMA store.  The staging slot is
@@ -1109,11 +1136,13 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     tc_fence_before();
     __syncthreads();
     if (MODE != MODE_STATE && p.dm_partial != nullptr) {
-        int* last_flag = reinterpret_cast<int*>(&dm_red[15]);
+        int* last_flag = reinterpret_cast<int*>(&dm_red[0]);
         if (tid == 0) {
-            // Fixed-order reduction of the CTA's dm term (the first-half warps of group O hold sums).
+            // Fixed-order reduction of the CTA's dm term (the warps of group O hold sums; in the
+            // dQ^ stream only its first half).
             if (!*abort_flag)
-                p.dm_partial[(size_t)bh * p.n_groups + g] = (dm_red[8] + dm_red[9]) + (dm_red[10] + dm_red[11]);
+                p.dm_partial[(size_t)bh * p.n_groups + g] = ((dm_red[8] + dm_red[9]) + (dm_red[10] + dm_red[11])) +
+                                                             ((dm_red[12] + dm_red[13]) + (dm_red[14] + dm_red[15]));
             *last_flag = 0;
             if (p.dm_out != nullptr) {
                 __threadfence();
@@ -1140,8 +1169,9 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                                                 : (p.seq_len_scalar > 0.f ? p.seq_len_scalar
                                                    : (float)(varlen ? max(p.cu_seqlens[bb + 1] - p.cu_seqlens[bb], 1) : p.N));
                     const float ls = logf(sb2);
-                    part += __ldcg(&p.dm_partial[((size_t)bb * p.H + hh) * p.n_groups + gg]) *
-                            (-ls * sg * (1.0f - sg) * expf(-sg * ls));
+                    const size_t idx = ((size_t)bb * p.H + hh) * p.n_groups + gg;
+                    const float t_bh = __ldcg(&p.dm_partial[idx]) + (p.dm_extra ? __ldcg(&p.dm_extra[idx]) : 0.f);
+                    part += t_bh * (-ls * sg * (1.0f - sg) * expf(-sg * ls));
                 }
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
@@ -1172,18 +1202,19 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 EncodeTiledFn get_encode() {
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
+    // (initialised once, thread-safe: a function-local static)
+    static const EncodeTiledFn fn = []() -> EncodeTiledFn {
         void* ptr = nullptr;
         cudaDriverEntryPointQueryResult qres;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) ==
                 cudaSuccess && qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(ptr);
-    }
+            return reinterpret_cast<EncodeTiledFn>(ptr);
+        return nullptr;
+    }();
     return fn;
 }
+
+}  // namespace
 
 // Tensor map over a bf16 tensor of logical shape [B,H,N,d] with element strides (sb, sh, sn)
 // and contiguous rows: 4-D, the head and token dimensions ordered by stride (dense [B,H,N,d]:
@@ -1209,17 +1240,16 @@ bool make_tile_map(CUtensorMap* map, const void* ptr, int B, int H, int N, int d
     return r == CUDA_SUCCESS;
 }
 
+namespace {
+
 template <int D, int MODE, int STREAM, bool VARLEN>
 cudaError_t launch_mode_v(const CUtensorMap* tm, const TcWalkParams& p, int BH, cudaStream_t st) {
     auto kern = tc_walk_kernel<D, MODE, STREAM, VARLEN>;
     // (the dV' stream has a plain epilogue, like the forward pass)
     constexpr bool with_proj = (MODE != MODE_STATE) && (STREAM == S_DQ || STREAM == S_DK);
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             Smem<D, MODE>::dyn_bytes(with_proj));
+    {   // (per kernel and device: the attribute belongs to a function on one device)
+        cudaError_t e = configure_smem_once(reinterpret_cast<const void*>(kern), Smem<D, MODE>::dyn_bytes(with_proj));
         if (e != cudaSuccess) return e;
-        configured = true;
     }
     const int prof = profile_begin_launch(MODE, st);
     // Programmatic dependent launch: this kernel may start (allocate TMEM, set up barriers,
@@ -1296,7 +1326,7 @@ cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cuda
         const RowLayout lo = resolve_layout(a.lout, H, map_N, d);
         p.out_rows = a.out; p.out_sn = lo.sn; p.out_sh = lo.sh;
     }
-    p.init = a.init; p.state_out = a.state_out; p.dm_partial = a.dm_partial; p.dm_out = a.dm_out; p.status = a.status;
+    p.init = a.init; p.state_out = a.state_out; p.dm_partial = a.dm_partial; p.dm_extra = a.dm_extra; p.dm_out = a.dm_out; p.status = a.status;
     p.init_has_scale = a.init_has_scale; p.state_final = a.state_final;
     p.m = a.m; p.seq_len = a.seq_len; p.seq_len_scalar = a.seq_len_scalar;
     p.H = H; p.N = N; p.group = a.group; p.n_groups = a.n_groups;
@@ -1310,13 +1340,13 @@ cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cuda
     // that may have produced it)
     p.plain_launch = a.plain_launch || a.cu_seqlens != nullptr;
     p.clear_status = a.clear_status;
-    {   // knobs for the test of the timeout path: a short bound, and a hand-off that never comes
-        const char* e = getenv("COTT_WAIT_LIMIT_MS");
-        const long ms = (e && *e) ? atol(e) : kWaitLimitMsDefault;
-        p.wait_limit_kcycles = (int)((ms < 1 ? 1 : (ms > 100000 ? 100000 : ms)) * 2000);   // <= 2 GHz
-        e = getenv("COTT_DEBUG_DROP_COMMIT");
+    p.wait_limit_kcycles = wait_limit_kcycles();
+#ifdef COTT_TEST_HOOKS
+    {   // test builds only: a hand-off that never comes (the scores of chunk 1 are never reported complete)
+        const char* e = getenv("COTT_DEBUG_DROP_COMMIT");
         p.debug_drop_commit = (e && *e == '1') ? 1 : 0;
     }
+#endif
     if (p.first_group < 0 || p.first_group + p.grid_groups > a.n_groups) return cudaErrorInvalidValue;
     // The four combinations of roles the library uses, as compile-time kernel variants.
     int kind;

@@ -7,6 +7,7 @@ import ctypes
 import pytest
 import torch
 
+import oracle
 import paper_2409_18747_b200 as cott
 from paper_2409_18747_b200 import synth
 from _metrics import norm_max_err
@@ -26,6 +27,9 @@ def test_noalloc_matches_cott_fwd_twice_in_a_row():
         torch.cuda.synchronize()
         assert norm_max_err(got, want.double().cpu().numpy()) <= 1e-2   # the bf16 gate of the parity tests
         assert torch.equal(got, want)                                    # same kernels, same order: same bits
+        # and against the definition itself (fp64 oracle), so that this file stands on its own
+        ref = oracle.fwd_quadratic(case["q"], case["k"], case["v"], case["m"], None, causal)
+        assert norm_max_err(got, ref) <= 1e-2
 
 
 def test_noalloc_rejects_problems_beyond_its_scratch():
