@@ -25,7 +25,18 @@
  * All calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL is
  * the legacy default stream).  The returned status covers argument validation and
  * launch errors only.  Calls are thread-safe as long as concurrent calls use
- * different workspaces.  Outputs must not alias inputs.
+ * different workspaces.  Outputs must not share bytes with inputs or with each other:
+ * equal pointers, dense tensors whose byte ranges meet, and equally strided tensors
+ * (slices of one buffer) whose rows meet are refused with COTT_ERR_INVALID_ARG.
+ *
+ * State the library keeps (everything else lives in the caller's buffers):
+ *   - per host thread and device, three CUDA streams and five events used by cott_bwd
+ *     (gradient streams side by side) and cott_fwd_bwd_host (copies in both directions),
+ *     created on first use; cott_shutdown() destroys the calling thread's;
+ *   - the options of cott_set_option, a launch counter and, while cott_profile_enable is
+ *     on, up to 512 timing events (process-wide);
+ *   - per (kernel, device), the fact that the shared-memory opt-in has been made;
+ *   - the 8 MiB scratch array of cott_fwd_noalloc.
  */
 #ifndef COTT_H_
 #define COTT_H_
@@ -78,6 +89,7 @@ unsigned long long cott_launch_count(void);
  *   "force_path"         (COTT_FORCE_PATH, 1)         0 = bf16 d = 64 / 128 through the fp32-accumulating SIMT kernels
  *   "pair"               (COTT_PAIR, 1)               0 = gradient streams one after the other where they would run side by side
  *   "fused_bwd"          (COTT_FUSED_BWD, 1)          0 = causal d = 64 backward as three role-swapped walks instead of one fused walk
+ *   "host_slices"        (COTT_HOST_SLICES, 8)        most slices cott_fwd_bwd_host cuts a batch into (1 .. 16)
  *   "wait_limit_ms"      (COTT_WAIT_LIMIT_MS, 2000)   bound of every device-side wait
  *   "wait_limit_kcycles" (COTT_WAIT_LIMIT_KCYCLES, -1) the same bound in units of 1024 SM cycles; negative = use the millisecond
  *                        value; 0 = every wait that is not met within a few polls gives up (the timeout test)
@@ -262,15 +274,22 @@ cott_status cott_decode_step(const void* q, const void* k, const void* v, float*
 
 /*
  * Training step with HOST buffers (end-to-end path): copies q,k,v,d_o from host memory to the
- * device arena, runs cott_fwd then cott_bwd, and copies o,dq,dk,dv,dm back.  The call is ordered
- * on `stream` as a whole; inside, o travels back on a stream of the library while d_o comes in
- * (the link is full duplex), joined into `stream` before the call's last copy.
+ * device arena, runs cott_fwd then cott_bwd, and copies o,dq,dk,dv,dm back.  The batch goes
+ * through in at most 8 slices (option "host_slices") that are contiguous in [B,H,N,d] -- several whole batch items
+ * each, or, when the batch is small, a batch item's heads in equal groups
+ * (cott_host_step_slicing tells which) --, each a cott_fwd and a cott_bwd call of its own on
+ * `stream` with the scaling base s_b = N unless seq_len_host is given: while one slice is computed, the inputs of the next come in and the results
+ * of the one before go back on two streams of the library (the link is full duplex), joined
+ * into `stream` before the call returns its last copy.  Every row of o, dq, dk, dv equals what
+ * the device calls give for its slice; dm (a sum over the batch) is the sum of the slices' dm
+ * in slice order.
  *   *_host  : host pointers ([B,H,N,d] dt; dm_host fp32 [H]); pinned memory makes the copies
  *             asynchronous.  m_host fp32 [H], seq_len_host fp32 [B] or NULL (s_b = N).
  *   arena   : device scratch of at least cott_host_step_arena_bytes() bytes, 256-B aligned.
  * The caller synchronises `stream` before reading the host outputs.
  */
 size_t cott_host_step_arena_bytes(cott_dtype dt, int B, int H, int N, int d, int causal);
+cott_status cott_host_step_slicing(int B, int H, int* items_per_slice, int* heads_per_slice, int* n_slices);
 cott_status cott_fwd_bwd_host(const void* q_host, const void* k_host, const void* v_host,
                               const void* d_o_host, void* o_host, void* dq_host, void* dk_host,
                               void* dv_host, float* dm_host, const float* m_host,
@@ -298,6 +317,19 @@ size_t cott_fwd_noalloc_max_bytes(void);
 cott_status cott_fwd_noalloc(const void* q, const void* k, const void* v, void* o, int B, int H,
                              int N, int d, int causal, cott_dtype dt, const cott_scale_params* sp,
                              void* stream);
+
+/*
+ * The same for cott_fwd_noalloc, whose scratch (and status word) is inside the library.
+ * No paper passage: library plumbing.
+ */
+cott_status cott_fwd_noalloc_status(void* stream);
+
+/*
+ * Destroys the CUDA streams and events the library created for the calling host thread (on
+ * every device it used) and the profiling events; they are created again on demand.  Call it
+ * when no library call of this thread is in flight.  No paper passage: library plumbing.
+ */
+cott_status cott_shutdown(void);
 
 /*
  * Synchronises `stream`, then reads the status word the last call using `workspace` left

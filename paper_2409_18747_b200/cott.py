@@ -6,7 +6,9 @@ allocated here with torch because the library itself never allocates.
 """
 from __future__ import annotations
 
+import contextlib
 import ctypes
+import functools
 import os
 
 import torch
@@ -90,6 +92,8 @@ def _load():
     lib.cott_decode_step.argtypes = [vp] * 5 + [ci, ci, ci, ci, ctypes.POINTER(_ScaleParams), vp]
     lib.cott_host_step_arena_bytes.restype = cs
     lib.cott_host_step_arena_bytes.argtypes = [ci] * 6
+    lib.cott_host_step_slicing.restype = ci
+    lib.cott_host_step_slicing.argtypes = [ci, ci, ctypes.POINTER(ci), ctypes.POINTER(ci), ctypes.POINTER(ci)]
     lib.cott_fwd_bwd_host.restype = ci
     lib.cott_fwd_bwd_host.argtypes = [vp] * 11 + [ci] * 6 + [vp, cs, vp]
     lib.cott_fwd_noalloc_max_bytes.restype = cs
@@ -97,12 +101,29 @@ def _load():
     lib.cott_fwd_noalloc.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ctypes.POINTER(_ScaleParams), vp]
     lib.cott_last_async_status.restype = ci
     lib.cott_last_async_status.argtypes = [vp, vp]
+    lib.cott_fwd_noalloc_status.restype = ci
+    lib.cott_fwd_noalloc_status.argtypes = [vp]
+    lib.cott_shutdown.restype = ci
     lib.cott_set_option.restype = ci
     lib.cott_set_option.argtypes = [ctypes.c_char_p, ctypes.c_longlong]
     lib.cott_get_option.restype = ctypes.c_longlong
     lib.cott_get_option.argtypes = [ctypes.c_char_p]
     _lib = lib
     return lib
+
+
+def _on_call_stream(fn):
+    """Runs a binding call with its ``stream`` argument (if any) as torch's current stream, so
+    that every tensor the binding allocates (outputs, workspace) belongs to the stream the
+    kernels run on: the caching allocator then cannot hand such a block to work on another
+    stream while libcott kernels still use it."""
+    @functools.wraps(fn)
+    def wrapped(*args, **kwargs):
+        stream = kwargs.get("stream")
+        ctx = torch.cuda.stream(stream) if stream is not None else contextlib.nullcontext()
+        with ctx:
+            return fn(*args, **kwargs)
+    return wrapped
 
 
 def _dt(t: torch.Tensor) -> int:
@@ -164,6 +185,19 @@ def _scale(m: torch.Tensor, seq_len, scalar: float = 0.0) -> _ScaleParams:
     return sp
 
 
+def fwd_noalloc_status(stream=None) -> int:
+    """cott_fwd_noalloc_status: synchronises the stream and returns the status the last
+    ``fwd_noalloc`` call left (0, or -5 after a device-side wait gave up)."""
+    return int(_load().cott_fwd_noalloc_status(_stream_ptr(stream)))
+
+
+def shutdown() -> None:
+    """cott_shutdown: destroys the streams and events the library created for this thread."""
+    rc = _load().cott_shutdown()
+    if rc != 0:
+        raise CottError(rc, "cott_shutdown")
+
+
 def set_option(name: str, value: int) -> None:
     """cott_set_option: a process-wide switch for tests and measurements (see ``cott.h``)."""
     rc = _load().cott_set_option(name.encode(), int(value))
@@ -198,6 +232,7 @@ def _workspace(op, dt, B, H, N, d, causal, device, workspace):
     return workspace, workspace.numel()
 
 
+@_on_call_stream
 def fwd(q, k, v, m, seq_len=None, causal=True, return_state=False, out=None, workspace=None,
         stream=None):
     """cott_fwd / cott_fwd_strided.  q, k, v: ``[B,H,N,d]`` tensors with contiguous rows and
@@ -224,6 +259,7 @@ def fwd(q, k, v, m, seq_len=None, causal=True, return_state=False, out=None, wor
     return (o, state) if return_state else o
 
 
+@_on_call_stream
 def fwd_stateful(q, k, v, m, seq_len, state_in=None, return_state=True, out=None, workspace=None,
                  stream=None):
     """cott_fwd_stateful: causal forward over one segment of a longer sequence.  ``state_in``
@@ -254,6 +290,7 @@ def fwd_stateful(q, k, v, m, seq_len, state_in=None, return_state=True, out=None
     return (o, state) if return_state else o
 
 
+@_on_call_stream
 def fwd_noalloc(q, k, v, m, seq_len=None, causal=True, out=None, stream=None):
     """cott_fwd_noalloc: the forward pass on the library's built-in 8 MiB scratch, for callers
     that cannot supply a workspace.  Raises CottError(-3) when the problem needs more."""
@@ -268,6 +305,7 @@ def fwd_noalloc(q, k, v, m, seq_len=None, causal=True, out=None, stream=None):
     return o
 
 
+@_on_call_stream
 def bwd(q, k, v, d_o, m, seq_len=None, causal=True, workspace=None, stream=None, out=None):
     """cott_bwd / cott_bwd_strided.  q, k, v (common strides) and d_o as for ``fwd``; ``out``:
     optional ``(dq, dk, dv)`` tensors with common strides (e.g. the slices of a fused gradient
@@ -300,6 +338,7 @@ def _check_packed(cu_seqlens, *ts):
             raise ValueError("packed tensors must all be [total_tokens, H, d]")
 
 
+@_on_call_stream
 def fwd_varlen(q, k, v, m, cu_seqlens, max_seqlen, seq_len=None, causal=True, out=None, workspace=None,
                stream=None):
     """cott_fwd_varlen: q, k, v ``[total_tokens, H, d]`` (bf16, d 64 or 128), the sequences of the
@@ -320,6 +359,7 @@ def fwd_varlen(q, k, v, m, cu_seqlens, max_seqlen, seq_len=None, causal=True, ou
     return o
 
 
+@_on_call_stream
 def bwd_varlen(q, k, v, d_o, m, cu_seqlens, max_seqlen, seq_len=None, causal=True, workspace=None,
                stream=None):
     """cott_bwd_varlen.  Returns ``(dq, dk, dv, dm[H] fp32)`` for packed ``[total_tokens, H, d]`` inputs."""
@@ -341,6 +381,7 @@ def bwd_varlen(q, k, v, d_o, m, cu_seqlens, max_seqlen, seq_len=None, causal=Tru
     return dq, dk, dv, dm
 
 
+@_on_call_stream
 def decode_step(q, k, v, state, m, seq_len, out=None, stream=None):
     """cott_decode_step.  q,k,v ``[B,H,d]``; ``state`` fp32 ``[B,H,d,d]`` updated in place;
     ``seq_len`` a float (>= 1) or a float32 ``[B]`` CUDA tensor.  Returns ``o [B,H,d]``."""
@@ -358,6 +399,7 @@ def decode_step(q, k, v, state, m, seq_len, out=None, stream=None):
     return o
 
 
+@_on_call_stream
 def fwd_bwd_host(q, k, v, d_o, m, o, dq, dk, dv, dm, causal=True, seq_len=None, arena=None,
                  stream=None):
     """cott_fwd_bwd_host: every tensor argument is a HOST tensor (pinned for async copies);
@@ -379,6 +421,15 @@ def fwd_bwd_host(q, k, v, d_o, m, o, dq, dk, dv, dm, causal=True, seq_len=None, 
     if rc != 0:
         raise CottError(rc, "cott_fwd_bwd_host")
     return arena
+
+
+def host_step_slicing(B: int, H: int) -> dict:
+    """cott_host_step_slicing: how ``fwd_bwd_host`` cuts a batch into slices."""
+    a, b, c = ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
+    rc = _load().cott_host_step_slicing(B, H, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c))
+    if rc != 0:
+        raise CottError(rc, "cott_host_step_slicing")
+    return {"items": a.value, "heads": b.value, "n": c.value}
 
 
 def launch_count() -> int:

@@ -73,8 +73,9 @@ static Option g_opt_pair("pair", "COTT_PAIR", 1);                          // 0:
 static Option g_opt_fused_bwd("fused_bwd", "COTT_FUSED_BWD", 1);           // 0: causal d=64 backward through the three role-swapped walks
 static Option g_opt_wait_ms("wait_limit_ms", "COTT_WAIT_LIMIT_MS", 2000);  // bound of every device-side wait
 static Option g_opt_wait_kc("wait_limit_kcycles", "COTT_WAIT_LIMIT_KCYCLES", -1);  // the same in units of 1024 SM cycles (< 0: use the ms value)
+static Option g_opt_host_slices("host_slices", "COTT_HOST_SLICES", 8);     // slices of the host-buffer step (1 .. 16)
 static Option* const g_options[] = {&g_opt_force_group, &g_opt_force_path, &g_opt_pair, &g_opt_fused_bwd,
-                                    &g_opt_wait_ms, &g_opt_wait_kc};
+                                    &g_opt_wait_ms, &g_opt_wait_kc, &g_opt_host_slices};
 
 int option_force_group() { return (int)g_opt_force_group.get(); }
 int option_force_path() { return (int)g_opt_force_path.get(); }
@@ -213,6 +214,58 @@ static bool layout_ok(const cott_strides* s, int d, cott_dtype dt) {
            s->token % q == 0;
 }
 
+// Do two tensors of logical shape [B,H,N,d] share bytes?  Each is a set of rows of d elements.
+// The test answers "yes" only when it can prove it: (1) equal base addresses; (2) both tensors
+// dense in memory (their dimensions merge into one contiguous block): the byte ranges decide;
+// (3) both with the same strides, every stride a multiple of the smallest one above the merged
+// innermost block (slices of one fused buffer, [B,N,H,d] storage): the rows of both sit on one
+// lattice and the offset between the bases decides.  Anything else passes.
+struct Extent {
+    long long block;     // elements of the contiguous innermost block after merging dimensions
+    long long step;      // smallest stride above that block (0: the tensor is one block)
+    bool lattice;        // every larger stride is a multiple of `step`
+    long long span;      // elements from the first to one past the last
+};
+static Extent extent_of(const cott_strides* st, int B, int H, int N, int d) {
+    long long ext[3] = {B, H, N};
+    long long str[3] = {st ? st->batch : (long long)H * N * d, st ? st->head : (long long)N * d, st ? st->token : (long long)d};
+    // sort the three outer dimensions by stride (extent-1 dimensions do not matter)
+    for (int i = 0; i < 3; ++i)
+        for (int j = i + 1; j < 3; ++j)
+            if (str[j] < str[i]) { long long t = str[i]; str[i] = str[j]; str[j] = t; t = ext[i]; ext[i] = ext[j]; ext[j] = t; }
+    Extent e;
+    e.block = d; e.step = 0; e.lattice = true; e.span = d;
+    for (int i = 0; i < 3; ++i) {
+        if (ext[i] == 1) continue;
+        if (e.step == 0 && str[i] == e.block) e.block *= ext[i];          // contiguous with what is below: merge
+        else if (e.step == 0) e.step = str[i];
+        else if (str[i] % e.step != 0) e.lattice = false;
+    }
+    e.span = d;
+    for (int i = 0; i < 3; ++i) e.span += (ext[i] - 1) * str[i];
+    return e;
+}
+static bool same_strides(const cott_strides* a, const cott_strides* b) {
+    if (!a || !b) return a == b;
+    return a->batch == b->batch && a->head == b->head && a->token == b->token;
+}
+static bool tensors_overlap(const void* pa, const cott_strides* sa, const void* pb, const cott_strides* sb2,
+                            int B, int H, int N, int d, cott_dtype dt) {
+    if (pa == pb) return true;
+    const long long es = (long long)dtype_size(dt);
+    const Extent a = extent_of(sa, B, H, N, d), b = extent_of(sb2, B, H, N, d);
+    const long long a0 = (long long)reinterpret_cast<uintptr_t>(pa), b0 = (long long)reinterpret_cast<uintptr_t>(pb);
+    const bool ranges = a0 < b0 + b.span * es && b0 < a0 + a.span * es;
+    if (!ranges) return false;
+    if (a.step == 0 && b.step == 0) return true;                          // two dense blocks whose ranges meet
+    if (same_strides(sa, sb2) && a.lattice && a.step > 0) {
+        long long delta = ((b0 - a0) / es) % a.step;                       // (bases are element-aligned)
+        if (delta < 0) delta += a.step;
+        return delta < a.block || a.step - delta < a.block;
+    }
+    return false;
+}
+
 static WalkArgs base_walk(const cott_scale_params* sp, int H, int N, const Plan& p) {
     WalkArgs w;
     memset(&w, 0, sizeof(w));
@@ -341,13 +394,19 @@ static cott_status fwd_impl(const void* q, const void* k, const void* v, void* o
 // Side streams and events for launches of one call that run next to each other on the GPU:
 // one set per host thread and device (two calls from different threads must not share events),
 // created on the first call that needs them and kept until the process ends.
+constexpr int kHostSlices = 16;    // the host-buffer step moves and computes the batch in at most this many slices
 struct SideStreams {
     bool ready = false;
-    cudaStream_t s[3];            // [0], [1]: gradient streams of cott_bwd; [2]: copies of the host step
+    cudaStream_t s[3];            // [0], [1]: gradient streams of cott_bwd, copy streams of the host step; [2]: spare
     cudaEvent_t fork, join[3], fork_copy;
+    cudaEvent_t slice_in[kHostSlices], slice_out[kHostSlices];   // host step: inputs of a slice landed / its results are ready
 };
-static SideStreams* side_streams() {
+static SideStreams* side_streams_table() {
     static thread_local SideStreams per_device[64];
+    return per_device;
+}
+static SideStreams* side_streams() {
+    SideStreams* per_device = side_streams_table();
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
     SideStreams& ss = per_device[dev];
@@ -364,6 +423,10 @@ static SideStreams* side_streams() {
         }
         if (cudaEventCreateWithFlags(&ss.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
         if (cudaEventCreateWithFlags(&ss.fork_copy, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        for (int i = 0; i < kHostSlices; ++i) {
+            if (cudaEventCreateWithFlags(&ss.slice_in[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+            if (cudaEventCreateWithFlags(&ss.slice_out[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        }
         ss.ready = true;
     }
     return &ss;
@@ -628,7 +691,10 @@ cott_status cott_fwd_strided(const void* q, const void* k, const void* v, void* 
     if (!q || !k || !v || !o || B < 1 || H < 1 || N < 1) return COTT_ERR_INVALID_ARG;
     if (!layout_ok(qkv_strides, d, dt) || !layout_ok(o_strides, d, dt)) return COTT_ERR_UNSUPPORTED;
     if (check_scale(sp) != COTT_OK) return COTT_ERR_INVALID_ARG;
-    if (o == q || o == k || o == v) return COTT_ERR_INVALID_ARG;
+    if (d >= 1 && (tensors_overlap(o, o_strides, q, qkv_strides, B, H, N, d, dt) ||
+                   tensors_overlap(o, o_strides, k, qkv_strides, B, H, N, d, dt) ||
+                   tensors_overlap(o, o_strides, v, qkv_strides, B, H, N, d, dt)))
+        return COTT_ERR_INVALID_ARG;
     if (!sp->seq_len && sp->seq_len_scalar > 0.f && sp->seq_len_scalar < 1.f)
         return COTT_ERR_INVALID_ARG;
     Plan p;
@@ -659,7 +725,10 @@ cott_status cott_fwd_stateful_strided(const void* q, const void* k, const void* 
     if (!q || !k || !v || !o || B < 1 || H < 1 || N < 1) return COTT_ERR_INVALID_ARG;
     if (!layout_ok(qkv_strides, d, dt) || !layout_ok(o_strides, d, dt)) return COTT_ERR_UNSUPPORTED;
     if (check_scale(sp) != COTT_OK) return COTT_ERR_INVALID_ARG;
-    if (o == q || o == k || o == v) return COTT_ERR_INVALID_ARG;
+    if (d >= 1 && (tensors_overlap(o, o_strides, q, qkv_strides, B, H, N, d, dt) ||
+                   tensors_overlap(o, o_strides, k, qkv_strides, B, H, N, d, dt) ||
+                   tensors_overlap(o, o_strides, v, qkv_strides, B, H, N, d, dt)))
+        return COTT_ERR_INVALID_ARG;
     if (state_in && state_in == state_out) return COTT_ERR_INVALID_ARG;
     // the scaling base must be the caller's (the same for every segment of a sequence)
     if (!sp->seq_len && !(sp->seq_len_scalar >= 1.f)) return COTT_ERR_INVALID_ARG;
@@ -694,13 +763,16 @@ cott_status cott_bwd_strided(const void* q, const void* k, const void* v, const 
     if (!layout_ok(qkv_strides, d, dt) || !layout_ok(do_strides, d, dt) || !layout_ok(dqkv_strides, d, dt))
         return COTT_ERR_UNSUPPORTED;
     if (check_scale(sp) != COTT_OK) return COTT_ERR_INVALID_ARG;
-    const void* ins[4] = {q, k, v, d_o};
-    void* outs[3] = {dq, dk, dv};
-    for (int i = 0; i < 3; ++i) {
-        for (int j = 0; j < 4; ++j)
-            if (outs[i] == ins[j]) return COTT_ERR_INVALID_ARG;
-        for (int j = i + 1; j < 3; ++j)
-            if (outs[i] == outs[j]) return COTT_ERR_INVALID_ARG;
+    {
+        const void* ins[4] = {q, k, v, d_o};
+        const cott_strides* in_st[4] = {qkv_strides, qkv_strides, qkv_strides, do_strides};
+        void* outs[3] = {dq, dk, dv};
+        for (int i = 0; i < 3 && d >= 1; ++i) {
+            for (int j = 0; j < 4; ++j)
+                if (tensors_overlap(outs[i], dqkv_strides, ins[j], in_st[j], B, H, N, d, dt)) return COTT_ERR_INVALID_ARG;
+            for (int j = i + 1; j < 3; ++j)
+                if (tensors_overlap(outs[i], dqkv_strides, outs[j], dqkv_strides, B, H, N, d, dt)) return COTT_ERR_INVALID_ARG;
+        }
     }
     if (!sp->seq_len && sp->seq_len_scalar > 0.f && sp->seq_len_scalar < 1.f)
         return COTT_ERR_INVALID_ARG;
@@ -790,22 +862,55 @@ cott_status cott_decode_step(const void* q, const void* k, const void* v, float*
     return COTT_OK;
 }
 
-// Arena layout of the host-buffer training step: 8 tensors, m, seq_len, dm, workspace.
+// The host-buffer training step cuts the batch into at most kHostSlices slices that are
+// contiguous in [B,H,N,d]: several whole batch items each, or -- when the batch is small -- a
+// batch item's heads in equal groups.
+struct HostSlicing {
+    int items;     // batch items per slice (head_groups == 1)
+    int heads;     // heads per slice
+    int n;         // number of slices
+};
+static HostSlicing host_step_slicing(int B, int H) {
+    HostSlicing s;
+    long long want = g_opt_host_slices.get();
+    const int max_slices = (int)(want < 1 ? 1 : (want > kHostSlices ? kHostSlices : want));
+    if (B >= max_slices) {
+        s.items = (B + max_slices - 1) / max_slices; s.heads = H; s.n = (B + s.items - 1) / s.items;
+        return s;
+    }
+    int groups = 1;                                   // head groups per batch item: the largest divisor of H that fits
+    for (int g = 1; g <= H; ++g)
+        if (H % g == 0 && (long long)B * g <= max_slices) groups = g;
+    s.items = 1; s.heads = H / groups; s.n = B * groups;
+    return s;
+}
+
+// Arena layout: 8 tensors, m, seq_len, dm, per-batch-item dm, workspace (for one slice at a time).
 static size_t host_step_layout(cott_dtype dt, int B, int H, int N, int d, int causal,
                                size_t* tensor_bytes, size_t* ws_bytes) {
     const size_t tb = align_up((size_t)B * H * N * d * dtype_size(dt), 256);
-    const size_t wf = cott_workspace_bytes(COTT_OP_FWD, dt, B, H, N, d, causal);
-    const size_t wb = cott_workspace_bytes(COTT_OP_BWD, dt, B, H, N, d, causal);
+    const HostSlicing sl = host_step_slicing(B, H);
+    const size_t wf = cott_workspace_bytes(COTT_OP_FWD, dt, sl.items, sl.heads, N, d, causal);
+    const size_t wb = cott_workspace_bytes(COTT_OP_BWD, dt, sl.items, sl.heads, N, d, causal);
     if (wf == (size_t)-1 || wb == (size_t)-1) return (size_t)-1;
     const size_t wsz = align_up(wf > wb ? wf : wb, 256);
     if (tensor_bytes) *tensor_bytes = tb;
     if (ws_bytes) *ws_bytes = wsz;
-    return 8 * tb + 3 * align_up((size_t)(B > H ? B : H) * 4, 256) + wsz;
+    return 8 * tb + 3 * align_up((size_t)(B > H ? B : H) * 4, 256) + align_up((size_t)B * H * 4, 256) + wsz;
 }
 
 size_t cott_host_step_arena_bytes(cott_dtype dt, int B, int H, int N, int d, int causal) {
     if (B < 1 || H < 1 || N < 1) return (size_t)-1;
     return host_step_layout(dt, B, H, N, d, causal, nullptr, nullptr);
+}
+
+cott_status cott_host_step_slicing(int B, int H, int* items_per_slice, int* heads_per_slice, int* n_slices) {
+    if (B < 1 || H < 1) return COTT_ERR_INVALID_ARG;
+    const HostSlicing sl = host_step_slicing(B, H);
+    if (items_per_slice) *items_per_slice = sl.items;
+    if (heads_per_slice) *heads_per_slice = sl.heads;
+    if (n_slices) *n_slices = sl.n;
+    return COTT_OK;
 }
 
 cott_status cott_fwd_bwd_host(const void* q_host, const void* k_host, const void* v_host,
@@ -823,42 +928,94 @@ cott_status cott_fwd_bwd_host(const void* q_host, const void* k_host, const void
         return COTT_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     char* p = static_cast<char*>(arena);
-    void* dq_ = p;           void* dk_ = p + tb;      void* dv_ = p + 2 * tb;
-    void* q_ = p + 3 * tb;   void* k_ = p + 4 * tb;   void* v_ = p + 5 * tb;
-    void* do_ = p + 6 * tb;  void* o_ = p + 7 * tb;
+    char* dq_ = p;           char* dk_ = p + tb;      char* dv_ = p + 2 * tb;
+    char* q_ = p + 3 * tb;   char* k_ = p + 4 * tb;   char* v_ = p + 5 * tb;
+    char* do_ = p + 6 * tb;  char* o_ = p + 7 * tb;
     const size_t small = align_up((size_t)(B > H ? B : H) * 4, 256);
     float* m_ = reinterpret_cast<float*>(p + 8 * tb);
     float* sl_ = reinterpret_cast<float*>(p + 8 * tb + small);
     float* dm_ = reinterpret_cast<float*>(p + 8 * tb + 2 * small);
-    void* ws = p + 8 * tb + 3 * small;
-    const size_t nbytes = (size_t)B * H * N * d * dtype_size(dt);
-    COTT_CUDA(cudaMemcpyAsync(q_, q_host, nbytes, cudaMemcpyHostToDevice, st));
-    COTT_CUDA(cudaMemcpyAsync(k_, k_host, nbytes, cudaMemcpyHostToDevice, st));
-    COTT_CUDA(cudaMemcpyAsync(v_, v_host, nbytes, cudaMemcpyHostToDevice, st));
-    COTT_CUDA(cudaMemcpyAsync(m_, m_host, (size_t)H * 4, cudaMemcpyHostToDevice, st));
-    if (seq_len_host)
-        COTT_CUDA(cudaMemcpyAsync(sl_, seq_len_host, (size_t)B * 4, cudaMemcpyHostToDevice, st));
-    cott_scale_params sp;
-    sp.m = m_; sp.seq_len = seq_len_host ? sl_ : nullptr; sp.seq_len_scalar = 0.f;
-    cott_status rc = cott_fwd(q_, k_, v_, o_, nullptr, B, H, N, d, causal, dt, &sp, ws, wsz, stream);
-    if (rc != COTT_OK) return rc;
-    // The link is full duplex: o goes back to the host on a side stream while dO comes in.
+    float* dm_parts = reinterpret_cast<float*>(p + 8 * tb + 3 * small);           // [B or n_slices][H]
+    void* ws = p + 8 * tb + 3 * small + align_up((size_t)B * H * 4, 256);
+    // While slice i is computed on the caller's stream, the inputs of slice i + 1 come in on one
+    // library stream and the results of slice i - 1 go back on another: the link is full
+    // duplex, and both directions stay busy.  Each slice is a cott_fwd and a cott_bwd call of
+    // its own; dm, a sum over the batch, is summed over the slices in slice order.
     SideStreams* ss = side_streams();
-    if (ss) {
-        COTT_CUDA(cudaEventRecord(ss->fork_copy, st));
-        COTT_CUDA(cudaStreamWaitEvent(ss->s[2], ss->fork_copy, 0));
-        COTT_CUDA(cudaMemcpyAsync(o_host, o_, nbytes, cudaMemcpyDeviceToHost, ss->s[2]));
-        COTT_CUDA(cudaEventRecord(ss->join[2], ss->s[2]));
+    if (!ss) return COTT_ERR_CUDA;
+    const HostSlicing sl = host_step_slicing(B, H);
+    const int groups = H / sl.heads;                                // head groups per batch item
+    const size_t head_bytes = (size_t)N * d * dtype_size(dt);       // one (b, h) of one tensor
+    cudaStream_t s_in = ss->s[0], s_out = ss->s[1];
+    COTT_CUDA(cudaEventRecord(ss->fork_copy, st));                  // the arena is free once the caller's earlier work is done
+    COTT_CUDA(cudaStreamWaitEvent(s_in, ss->fork_copy, 0));
+    COTT_CUDA(cudaStreamWaitEvent(s_out, ss->fork_copy, 0));
+    COTT_CUDA(cudaMemcpyAsync(m_, m_host, (size_t)H * 4, cudaMemcpyHostToDevice, s_in));
+    if (seq_len_host)
+        COTT_CUDA(cudaMemcpyAsync(sl_, seq_len_host, (size_t)B * 4, cudaMemcpyHostToDevice, s_in));
+    auto slice_of = [&](int i, int* b0, int* nb, int* h0) {
+        if (groups == 1) { *b0 = i * sl.items; *nb = (*b0 + sl.items <= B ? sl.items : B - *b0); *h0 = 0; }
+        else { *b0 = i / groups; *nb = 1; *h0 = (i % groups) * sl.heads; }
+    };
+    for (int i = 0; i < sl.n; ++i) {
+        int b0, nb, h0;
+        slice_of(i, &b0, &nb, &h0);
+        const size_t off = ((size_t)b0 * H + h0) * head_bytes, nbytes = (size_t)nb * sl.heads * head_bytes;
+        COTT_CUDA(cudaMemcpyAsync(q_ + off, static_cast<const char*>(q_host) + off, nbytes, cudaMemcpyHostToDevice, s_in));
+        COTT_CUDA(cudaMemcpyAsync(k_ + off, static_cast<const char*>(k_host) + off, nbytes, cudaMemcpyHostToDevice, s_in));
+        COTT_CUDA(cudaMemcpyAsync(v_ + off, static_cast<const char*>(v_host) + off, nbytes, cudaMemcpyHostToDevice, s_in));
+        COTT_CUDA(cudaMemcpyAsync(do_ + off, static_cast<const char*>(d_o_host) + off, nbytes, cudaMemcpyHostToDevice, s_in));
+        COTT_CUDA(cudaEventRecord(ss->slice_in[i], s_in));
     }
-    COTT_CUDA(cudaMemcpyAsync(do_, d_o_host, nbytes, cudaMemcpyHostToDevice, st));
-    rc = cott_bwd(q_, k_, v_, do_, dq_, dk_, dv_, dm_, B, H, N, d, causal, dt, &sp, ws, wsz, stream);
-    if (rc != COTT_OK) return rc;
-    if (ss) COTT_CUDA(cudaStreamWaitEvent(st, ss->join[2], 0));
-    else COTT_CUDA(cudaMemcpyAsync(o_host, o_, nbytes, cudaMemcpyDeviceToHost, st));
-    COTT_CUDA(cudaMemcpyAsync(dq_host, dq_, nbytes, cudaMemcpyDeviceToHost, st));
-    COTT_CUDA(cudaMemcpyAsync(dk_host, dk_, nbytes, cudaMemcpyDeviceToHost, st));
-    COTT_CUDA(cudaMemcpyAsync(dv_host, dv_, nbytes, cudaMemcpyDeviceToHost, st));
+    for (int i = 0; i < sl.n; ++i) {
+        int b0, nb, h0;
+        slice_of(i, &b0, &nb, &h0);
+        const size_t off = ((size_t)b0 * H + h0) * head_bytes, nbytes = (size_t)nb * sl.heads * head_bytes;
+        cott_scale_params sp;
+        sp.m = m_ + h0; sp.seq_len = seq_len_host ? sl_ + b0 : nullptr; sp.seq_len_scalar = (float)N;
+        // (whole batch items per slice: one dm row per slice; head groups: one row per batch item)
+        float* dm_slice = dm_parts + (size_t)(groups == 1 ? i : b0) * H + h0;
+        COTT_CUDA(cudaStreamWaitEvent(st, ss->slice_in[i], 0));
+        cott_status rc = cott_fwd(q_ + off, k_ + off, v_ + off, o_ + off, nullptr, nb, sl.heads, N, d, causal, dt, &sp, ws, wsz, stream);
+        if (rc != COTT_OK) return rc;
+        rc = cott_bwd(q_ + off, k_ + off, v_ + off, do_ + off, dq_ + off, dk_ + off, dv_ + off, dm_slice,
+                      nb, sl.heads, N, d, causal, dt, &sp, ws, wsz, stream);
+        if (rc != COTT_OK) return rc;
+        COTT_CUDA(cudaEventRecord(ss->slice_out[i], st));
+        COTT_CUDA(cudaStreamWaitEvent(s_out, ss->slice_out[i], 0));
+        COTT_CUDA(cudaMemcpyAsync(static_cast<char*>(o_host) + off, o_ + off, nbytes, cudaMemcpyDeviceToHost, s_out));
+        COTT_CUDA(cudaMemcpyAsync(static_cast<char*>(dq_host) + off, dq_ + off, nbytes, cudaMemcpyDeviceToHost, s_out));
+        COTT_CUDA(cudaMemcpyAsync(static_cast<char*>(dk_host) + off, dk_ + off, nbytes, cudaMemcpyDeviceToHost, s_out));
+        COTT_CUDA(cudaMemcpyAsync(static_cast<char*>(dv_host) + off, dv_ + off, nbytes, cudaMemcpyDeviceToHost, s_out));
+    }
+    COTT_CUDA(launch_sum_slices(dm_parts, dm_, groups == 1 ? sl.n : B, H, st));
     COTT_CUDA(cudaMemcpyAsync(dm_host, dm_, (size_t)H * 4, cudaMemcpyDeviceToHost, st));
+    COTT_CUDA(cudaEventRecord(ss->join[2], s_out));
+    COTT_CUDA(cudaStreamWaitEvent(st, ss->join[2], 0));
+    return COTT_OK;
+}
+
+cott_status cott_shutdown(void) {
+    // The side streams and events of THIS host thread on every device it used, and the
+    // profiling events.  Other threads' sets stay until the process ends.
+    int cur = 0;
+    cudaGetDevice(&cur);
+    SideStreams* all = side_streams_table();
+    for (int dev = 0; dev < 64; ++dev) {
+        SideStreams& ss = all[dev];
+        if (!ss.ready) continue;
+        if (cudaSetDevice(dev) != cudaSuccess) continue;
+        for (int i = 0; i < 3; ++i) { cudaStreamSynchronize(ss.s[i]); cudaStreamDestroy(ss.s[i]); cudaEventDestroy(ss.join[i]); }
+        cudaEventDestroy(ss.fork); cudaEventDestroy(ss.fork_copy);
+        for (int i = 0; i < kHostSlices; ++i) { cudaEventDestroy(ss.slice_in[i]); cudaEventDestroy(ss.slice_out[i]); }
+        ss.ready = false;
+    }
+    cudaSetDevice(cur);
+    g_prof_n.store(-1);
+    if (g_prof_created) {
+        for (int i = 0; i < 2 * kProfMax; ++i) cudaEventDestroy(g_prof_ev[i]);
+        g_prof_created = false;
+    }
     return COTT_OK;
 }
 

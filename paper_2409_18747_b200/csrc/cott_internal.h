@@ -146,6 +146,7 @@ int wait_limit_kcycles();      // bound of every device-side wait, in units of 1
 cudaError_t launch_dm_finalize(const float* dm_partial, float* dm, const float* m,
                                const float* seq_len, float seq_len_scalar, int B, int H,
                                int n_groups, int N, cudaStream_t st);
+cudaError_t launch_sum_slices(const float* parts, float* out, int n, int H, cudaStream_t st);
 cudaError_t launch_decode(const void* q, const void* k, const void* v, float* state, void* o,
                           int B, int H, int d, cott_dtype dt, const float* m,
                           const float* seq_len, float seq_len_scalar, cudaStream_t st);

@@ -58,4 +58,10 @@ cott_status cott_fwd_noalloc(const void* q, const void* k, const void* v, void* 
     return cott_fwd(q, k, v, o, nullptr, B, H, N, d, causal, dt, sp, ws, kScratchBytes, stream);
 }
 
+cott_status cott_fwd_noalloc_status(void* stream) {
+    void* ws = nullptr;
+    if (scratch_address(&ws) != cudaSuccess) return COTT_ERR_CUDA;
+    return cott_last_async_status(ws, stream);
+}
+
 }  // extern "C"

@@ -425,6 +425,21 @@ cudaError_t launch_scan(float* states, float* total_out, int BH, int n_groups, i
     return cudaGetLastError();
 }
 
+// out[h] = sum over the n slices of parts[i][h], in slice order (deterministic).
+__global__ void sum_slices_kernel(const float* parts, float* out, int n, int H) {
+    const int h = blockIdx.x * blockDim.x + threadIdx.x;
+    if (h >= H) return;
+    float acc = 0.f;
+    for (int i = 0; i < n; ++i) acc += parts[(size_t)i * H + h];
+    out[h] = acc;
+}
+
+cudaError_t launch_sum_slices(const float* parts, float* out, int n, int H, cudaStream_t st) {
+    sum_slices_kernel<<<(H + 127) / 128, 128, 0, st>>>(parts, out, n, H);
+    note_launch();
+    return cudaGetLastError();
+}
+
 cudaError_t launch_dm_finalize(const float* dm_partial, float* dm, const float* m,
                                const float* seq_len, float seq_len_scalar, int B, int H,
                                int n_groups, int N, cudaStream_t st) {

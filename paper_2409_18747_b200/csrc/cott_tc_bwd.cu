@@ -100,6 +100,12 @@ __device__ long long g_bwd_stamps[8 * 4 * 8];
 __device__ long long g_bwd_cta[256 * 4];   // per CTA: global-timer ns at entry, after the prologue, after the walk, at exit
 __device__ __forceinline__ long long gtime_ns() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
 #define CSTAMP(slot) do { if (threadIdx.x == 0 && blockIdx.x < 256) g_bwd_cta[blockIdx.x * 4 + (slot)] = gtime_ns(); } while (0)
+__device__ long long g_state_stamps[3 * 16 * 4];   // state kernel, CTA 0: role (worker, mma, copy) x chunk x slot
+#define SSTAMP(role, cc, slot)                                                                     \
+    do {                                                                                           \
+        if (blockIdx.x == 0 && (cc) < 16 && ((role) == 0 ? threadIdx.x == 0 : true))              \
+            g_state_stamps[((role) * 16 + (cc)) * 4 + (slot)] = clock64();                        \
+    } while (0)
 #define BSTAMP(role, cc, slot)                                                                     \
     do {                                                                                           \
         if (blockIdx.x == 0 && (cc) >= COTT_STAMP_C0 && (cc) < COTT_STAMP_C0 + 4 &&               \
@@ -109,6 +115,7 @@ __device__ __forceinline__ long long gtime_ns() { long long t; asm volatile("mov
 #else
 #define BSTAMP(role, cc, slot) do {} while (0)
 #define CSTAMP(slot) do {} while (0)
+#define SSTAMP(role, cc, slot) do {} while (0)
 #endif
 
 // K-major operand of 64 columns: K step kk (16 elements) advances the address by 32 bytes.
@@ -935,10 +942,11 @@ tc_bwd_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 
     if (is_copy) {
         if (lane == 0) {
-            for (int c = 0; c < kStStages && c < n_chunks; ++c) issue_loads(c);
+            for (int c = 0; c < kStStages && c < n_chunks; ++c) { issue_loads(c); SSTAMP(2, c, 0); }
             for (int c = 0; c + kStStages < n_chunks; ++c) {
                 if (!wait_or_abort(bar(S_UFULL, c), par(c), abort_flag)) break;
                 issue_loads(c + kStStages);
+                SSTAMP(2, c + kStStages, 0);
             }
         }
     } else if (is_mma) {
@@ -946,6 +954,7 @@ tc_bwd_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             for (int c = 0; c < n_chunks; ++c) {
                 const uint32_t st = stage(c);
                 if (!wait_or_abort(bar(S_NREADY, c), par(c), abort_flag)) break;
+                SSTAMP(1, c, 0);
                 tc_fence_after();
                 constexpr uint32_t idesc = instr_desc_bf16(128, 128, true, true);
                 const uint32_t al = smem_desc_lo(st + L::kOffV, 16384), bl = smem_desc_lo(st + L::kOffK, 16384);
@@ -960,7 +969,9 @@ tc_bwd_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         bool alive = n_chunks > 0;
         const int q4 = warp & 3, hw = warp >> 2, row = q4 * 32 + lane;
         for (int c = 0; c < n_chunks && alive; ++c) {
+            SSTAMP(0, c, 0);
             if (!wait_or_abort(bar(S_FULL, c), par(c), abort_flag)) { alive = false; break; }
+            SSTAMP(0, c, 1);
             if (hw == 1 && !need_sq) { mbar_arrive(bar(S_NREADY, c)); continue; }
             uint8_t* tile = gbase + (c % kStStages) * L::kStage + (hw == 0 ? L::kOffQ : L::kOffK);
             uint4 w[8];
@@ -992,6 +1003,7 @@ tc_bwd_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             }
             fence_proxy_async();
             mbar_arrive(bar(S_NREADY, c));
+            SSTAMP(0, c, 2);
         }
         if (alive && wait_or_abort(bar(S_UFULL, n_chunks - 1), par(n_chunks - 1), abort_flag)) {
             // the group's partial states, fp32: rows 0-63 -> Sq, rows 64-127 -> R (32 columns per thread)
@@ -1100,6 +1112,9 @@ cudaError_t launch_tc_bwd_states(const TcBwdFusedArgs& a, float* sq_out, float* 
 // Debug build only: copies the 256 stamps (8 roles x 4 chunks x 8 slots) to the host.
 extern "C" int cott_debug_bwd_stamps(long long* out) {
     return (int)cudaMemcpyFromSymbol(out, cott::g_bwd_stamps, sizeof(long long) * 256);
+}
+extern "C" int cott_debug_state_stamps(long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, cott::g_state_stamps, sizeof(long long) * 192);
 }
 extern "C" int cott_debug_bwd_cta(long long* out) {
     return (int)cudaMemcpyFromSymbol(out, cott::g_bwd_cta, sizeof(long long) * 1024);

@@ -108,6 +108,64 @@ def test_strided_and_packed_entry_points_validate_on_the_host():
                                cott.BF16, ctypes.byref(sp), a, 1 << 24, null) == -1
 
 
+def test_outputs_that_share_bytes_with_other_tensors_are_refused():
+    """Aliasing is decided by the bytes the tensors cover, not by pointer equality: dense
+    tensors whose ranges meet and equally strided tensors whose rows meet are refused, while
+    the interleaved slices of one fused buffer (ranges meet, rows do not) are accepted."""
+    lib = cott._load()
+    sp = cott._ScaleParams()
+    sp.m, sp.seq_len, sp.seq_len_scalar = 256, None, 0.0
+    a, null = 1 << 20, None
+    B, H, N, d = 1, 2, 16, 64
+    nbytes = B * H * N * d * 2
+    tail = (ctypes.byref(sp), null, 0, null)          # valid calls stop at the workspace check (-3)
+    f = lambda o: lib.cott_fwd(a, a + nbytes, a + 2 * nbytes, o, null, B, H, N, d, 1, cott.BF16, *tail)
+    assert f(a + 3 * nbytes) == -3                     # disjoint
+    assert f(a + 2 * nbytes + 128) == -1               # o starts inside v
+    assert f(a - 256) == -1                            # o ends inside q
+    assert f(a + nbytes - 16) == -1                    # straddles q and k
+    g = lambda dq, dk, dv: lib.cott_bwd(a, a + nbytes, a + 2 * nbytes, a + 3 * nbytes, dq, dk, dv, a + 64 * nbytes,
+                                        B, H, N, d, 1, cott.BF16, *tail)
+    assert g(a + 4 * nbytes, a + 5 * nbytes, a + 6 * nbytes) == -3
+    assert g(a + 4 * nbytes, a + 4 * nbytes + 256, a + 6 * nbytes) == -1      # dk starts inside dq
+    assert g(a + 3 * nbytes + 512, a + 5 * nbytes, a + 6 * nbytes) == -1      # dq overlaps dO
+    # slices of a fused [B,N,3,H,d] buffer: q, k, v interleaved per token; gradients likewise
+    S = cott._Strides
+    fused = S(N * 3 * H * d, d, 3 * H * d)
+    row = H * d * 2
+    base_in, base_out = a, a + (1 << 22)
+    ok = lib.cott_bwd_strided(base_in, base_in + row, base_in + 2 * row, a + (1 << 23),
+                              base_out, base_out + row, base_out + 2 * row, a + (1 << 24), B, H, N, d, 1, cott.BF16,
+                              ctypes.byref(fused), None, ctypes.byref(fused), *tail)
+    assert ok == -3
+    bad = lib.cott_bwd_strided(base_in, base_in + row, base_in + 2 * row, a + (1 << 23),
+                               base_out, base_out + row - 64, base_out + 2 * row, a + (1 << 24), B, H, N, d, 1, cott.BF16,
+                               ctypes.byref(fused), None, ctypes.byref(fused), *tail)
+    assert bad == -1                                    # dk's rows run into dq's
+    same = lib.cott_bwd_strided(base_in, base_in + row, base_in + 2 * row, a + (1 << 23),
+                                base_in + row, base_out + row, base_out + 2 * row, a + (1 << 24), B, H, N, d, 1, cott.BF16,
+                                ctypes.byref(fused), None, ctypes.byref(fused), *tail)
+    assert same == -1                                   # dq is the k slice
+
+
+def test_options_and_shutdown_are_host_only():
+    assert cott.get_option("fused_bwd") in (0, 1, 2)
+    old = cott.get_option("force_group")
+    cott.set_option("force_group", 384)
+    assert cott.get_option("force_group") == 384
+    assert cott.query_plan(cott.OP_FWD, cott.BF16, 1, 2, 4096, 64, True)["group"] == 384
+    cott.set_option("force_group", old)
+    try:
+        cott.set_option("no_such_option", 1)
+    except cott.CottError as e:
+        assert e.status == -1
+    else:
+        raise AssertionError("unknown option names must be refused")
+    assert cott.get_option("no_such_option") == -1
+    cott.shutdown()          # nothing created yet on a machine without a GPU: still fine
+    cott.shutdown()
+
+
 def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(cott, "_lib", None)
     monkeypatch.setattr(cott, "_LIB_PATH", "/nonexistent/libcott.so")

@@ -423,8 +423,33 @@ def test_decode_matches_longer_forward(dtype, d):
     assert norm_max_err(state, ref_state) <= state_tol(dtype, d)
 
 
+def test_calls_on_a_stream_that_is_not_current():
+    """Outputs and workspace the binding allocates belong to the stream the kernels run on (the
+    caching allocator must not recycle them for work on the current stream meanwhile); results
+    equal the call on the current stream, also after the library's own streams were destroyed
+    and created again (cott_shutdown)."""
+    c = synth.make_config(4, B=2, N=1024)
+    q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
+    want_o = cott.fwd(q, k, v, m, causal=True)
+    want_g = cott.bwd(q, k, v, d_o, m, causal=True)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    for _ in range(3):
+        o = cott.fwd(q, k, v, m, causal=True, stream=side)
+        junk = [torch.randn(1 << 22, device="cuda") for _ in range(4)]     # allocator pressure on the current stream
+        g = cott.bwd(q, k, v, d_o, m, causal=True, stream=side)
+        del junk
+    side.synchronize()
+    assert torch.equal(o, want_o) and all(torch.equal(a, b) for a, b in zip(g, want_g))
+    cott.cott.shutdown()
+    g2 = cott.bwd(q, k, v, d_o, m, causal=True)
+    torch.cuda.synchronize()
+    assert all(torch.equal(a, b) for a, b in zip(g2, want_g))
+
+
 # ------------------------------------------------------------------ host-buffer entry point
-def test_fwd_bwd_host_matches_device_calls():
+def test_fwd_bwd_host_matches_the_oracle():
     c = synth.make_config(4, B=1, N=512)
     host = {x: c[x].pin_memory() for x in ("q", "k", "v", "d_o", "m")}
     outs = {x: torch.empty_like(c["q"]).pin_memory() for x in ("o", "dq", "dk", "dv")}
@@ -432,11 +457,51 @@ def test_fwd_bwd_host_matches_device_calls():
     cott.fwd_bwd_host(host["q"], host["k"], host["v"], host["d_o"], host["m"], outs["o"], outs["dq"],
                       outs["dk"], outs["dv"], dm, causal=True)
     torch.cuda.synchronize()
-    q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
-    o = cott.fwd(q, k, v, m, causal=True)
-    dq, dk, dv, dm2 = cott.bwd(q, k, v, d_o, m, causal=True)
-    assert torch.equal(outs["o"], o.cpu()) and torch.equal(outs["dq"], dq.cpu())
-    assert torch.equal(outs["dk"], dk.cpu()) and torch.equal(outs["dv"], dv.cpu()) and torch.equal(dm, dm2.cpu())
+    ref_o = oracle.fwd_quadratic(c["q"], c["k"], c["v"], c["m"], None, True)
+    rq, rk, rv, rm = oracle.bwd_quadratic(c["q"], c["k"], c["v"], c["d_o"], c["m"], None, True)
+    gate(outs["o"], ref_o, torch.bfloat16)
+    gate(outs["dq"], rq, torch.bfloat16); gate(outs["dk"], rk, torch.bfloat16); gate(outs["dv"], rv, torch.bfloat16)
+    gate_dm(dm, rm, 1e-2, dm_condition(rv, c["v"], c["m"], None), DM_COND_BF16)
+
+
+@pytest.mark.parametrize("B", [3, 20])
+def test_fwd_bwd_host_slices_match_device_calls_per_slice(B):
+    """The host step runs the batch in slices (B = 3: sixteen heads in four groups per batch item;
+    B = 20: two batch items per slice), copies in both directions overlapping the compute; every
+    slice's rows equal the device calls on that slice bit for bit, dm is the sum of the slices'
+    dm in slice order; two calls in a row on one arena agree."""
+    N = 640 if B == 3 else 256
+    c = synth.make_config(4, B=B, N=N)
+    H = 16
+    sl = cott.cott.host_step_slicing(B, H)
+    assert sl["n"] <= 16 and (sl["items"] == 1 or sl["heads"] == H)
+    host = {x: c[x].pin_memory() for x in ("q", "k", "v", "d_o", "m")}
+    outs = {x: torch.empty_like(c["q"]).pin_memory() for x in ("o", "dq", "dk", "dv")}
+    dm = torch.empty(H, dtype=torch.float32).pin_memory()
+    m = dev(c["m"])
+    arena = None
+    for _ in range(2):
+        for t in outs.values():
+            t.fill_(float("nan"))
+        arena = cott.fwd_bwd_host(host["q"], host["k"], host["v"], host["d_o"], host["m"], outs["o"], outs["dq"],
+                                  outs["dk"], outs["dv"], dm, causal=True, arena=arena)
+        torch.cuda.synchronize()
+        dm_rows = []
+        for b0 in range(0, B, sl["items"]):
+            row = torch.zeros(H, dtype=torch.float32, device="cuda")
+            for h0 in range(0, H, sl["heads"]):
+                cut = (slice(b0, b0 + sl["items"]), slice(h0, h0 + sl["heads"]))
+                q, k, v, d_o = (dev(c[x][cut].contiguous()) for x in ("q", "k", "v", "d_o"))
+                o = cott.fwd(q, k, v, m[cut[1]].contiguous(), seq_len=float(N), causal=True)
+                dq, dk, dv, dm_s = cott.bwd(q, k, v, d_o, m[cut[1]].contiguous(), seq_len=float(N), causal=True)
+                for name, t in (("o", o), ("dq", dq), ("dk", dk), ("dv", dv)):
+                    assert torch.equal(outs[name][cut], t.cpu()), (name, b0, h0)
+                row[cut[1]] = dm_s
+            dm_rows.append(row)
+        dm_sum = torch.zeros(H, dtype=torch.float32, device="cuda")
+        for row in dm_rows:
+            dm_sum = dm_sum + row
+        assert torch.equal(dm, dm_sum.cpu())
 
 
 # ------------------------------------------------------------------ library services

@@ -30,6 +30,7 @@ def test_noalloc_matches_cott_fwd_twice_in_a_row():
         # and against the definition itself (fp64 oracle), so that this file stands on its own
         ref = oracle.fwd_quadratic(case["q"], case["k"], case["v"], case["m"], None, causal)
         assert norm_max_err(got, ref) <= 1e-2
+        assert cott.cott.fwd_noalloc_status() == 0                       # no device-side wait gave up
 
 
 def test_noalloc_rejects_problems_beyond_its_scratch():
