@@ -71,16 +71,18 @@ static Option g_opt_force_group("force_group", "COTT_FORCE_GROUP", 0);     // to
 static Option g_opt_force_path("force_path", "COTT_FORCE_PATH", 1);        // 0: bf16 d=64/128 through the fp32-accumulating SIMT kernels
 static Option g_opt_pair("pair", "COTT_PAIR", 1);                          // 0: gradient streams one after the other
 static Option g_opt_fused_bwd("fused_bwd", "COTT_FUSED_BWD", 1);           // 0: causal d=64 backward through the three role-swapped walks
+static Option g_opt_fused_bidir("fused_bidir", "COTT_FUSED_BIDIR", 1);     // 0: bidirectional d=64 forward as state pass + read-out
 static Option g_opt_wait_ms("wait_limit_ms", "COTT_WAIT_LIMIT_MS", 2000);  // bound of every device-side wait
 static Option g_opt_wait_kc("wait_limit_kcycles", "COTT_WAIT_LIMIT_KCYCLES", -1);  // the same in units of 1024 SM cycles (< 0: use the ms value)
 static Option g_opt_host_slices("host_slices", "COTT_HOST_SLICES", 8);     // slices of the host-buffer step (1 .. 16)
 static Option* const g_options[] = {&g_opt_force_group, &g_opt_force_path, &g_opt_pair, &g_opt_fused_bwd,
-                                    &g_opt_wait_ms, &g_opt_wait_kc, &g_opt_host_slices};
+                                    &g_opt_wait_ms, &g_opt_wait_kc, &g_opt_host_slices, &g_opt_fused_bidir};
 
 int option_force_group() { return (int)g_opt_force_group.get(); }
 int option_force_path() { return (int)g_opt_force_path.get(); }
 int option_pair() { return (int)g_opt_pair.get(); }
 int option_fused_bwd() { return (int)g_opt_fused_bwd.get(); }
+int option_fused_bidir() { return (int)g_opt_fused_bidir.get(); }
 int wait_limit_kcycles() {
     const long long kc = g_opt_wait_kc.get();
     if (kc >= 0) return (int)(kc > 200000000 ? 200000000 : kc);
@@ -372,6 +374,14 @@ static cott_status fwd_impl(const void* q, const void* k, const void* v, void* o
     // The tensor-core path clears the status words in its first kernel.
     if (p.path != 1) COTT_CUDA(cudaMemsetAsync(ws, 0, kWsHeaderBytes, st));
     float* states = reinterpret_cast<float*>(static_cast<char*>(ws) + kWsHeaderBytes);
+    if (p.path == 1 && !causal && d == 64 && p.n_groups == 1 && !packed.cu_seqlens && !state_in &&
+        option_fused_bidir() != 0) {
+        // One CTA per (b, h) streams k, v into the d x d state and then q through it: one launch,
+        // every tensor touched once.
+        COTT_CUDA(launch_tc_bidir_fwd(q, k, v, o, lay.qkv, lay.o, state_out, static_cast<int*>(ws), sp->m, sp->seq_len,
+                                      sp->seq_len_scalar, B, H, N, st));
+        return COTT_OK;
+    }
     if (p.path == 1) {
         TcWalkArgs t;
         memset(&t, 0, sizeof(t));

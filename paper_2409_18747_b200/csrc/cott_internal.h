@@ -128,6 +128,12 @@ cudaError_t launch_tc_bwd_fused(const TcBwdFusedArgs& a, int B, int H, int N, cu
 cudaError_t launch_tc_bwd_states(const TcBwdFusedArgs& a, float* sq_out, float* r_out, int clear_status, int B, int H,
                                  int N, cudaStream_t st);
 
+// Bidirectional forward at d = 64 in one launch, one CTA per (b, h) (cott_tc_bidir.cu); it is
+// the first (and only) kernel of its call and clears the status words itself.
+cudaError_t launch_tc_bidir_fwd(const void* q, const void* k, const void* v, void* o, const RowLayout& l_qkv,
+                                const RowLayout& l_o, float* state_out, int* status, const float* m, const float* seq_len,
+                                float seq_len_scalar, int B, int H, int N, cudaStream_t st);
+
 // Tensor map over a bf16 tensor of logical shape [B,H,N,d] with the given row layout: box of
 // 128 tokens x 64 columns of one (b,h), 128-byte swizzle (see cott_tc_walk.cu).
 bool make_tile_map(CUtensorMap* map, const void* ptr, int B, int H, int N, int d, const RowLayout& lay,
@@ -141,6 +147,7 @@ int option_force_group();
 int option_force_path();
 int option_pair();
 int option_fused_bwd();
+int option_fused_bidir();
 int wait_limit_kcycles();      // bound of every device-side wait, in units of 1024 SM cycles
 
 cudaError_t launch_dm_finalize(const float* dm_partial, float* dm, const float* m,

@@ -25,10 +25,12 @@
 #include <stdlib.h>
 #include "cott_internal.h"
 #include "cott_sm100.cuh"
+#include "cott_tc_common.cuh"
 
 namespace cott {
 
 using namespace sm100;
+using namespace tc;
 
 namespace {
 
@@ -57,7 +59,7 @@ struct L {
     static constexpr int kOffCtl = kOffStK + kTile;
     // control block: mbarriers (first 512 bytes), tensor-memory slot, abort flag and wait
     // limit, reciprocal row norms of the two stages, dm scratch
-    static constexpr int kOffTmemSlot = 512, kOffAbort = 516;
+    static constexpr int kOffTmemSlot = kCtlTmemSlot, kOffAbort = kCtlAbort;
     static constexpr int kOffRq = 1024;                      // float2 [2][128]: 1 / max(||q||, eps), 1 if not clamped
     static constexpr int kOffRk = kOffRq + 2 * kC * 8;
     static constexpr int kOffDmRed = kOffRk + 2 * kC * 8;    // float [32]
@@ -77,17 +79,6 @@ struct BwdParams {
     int head_first_mask;     // bit i: in tensor map i (q, k, v, dO, dq, dk, dv) the head index comes before the token index
 };
 
-constexpr uint32_t kDescHi = smem_desc_hi(1024);
-#ifndef COTT_POLL_SLEEP_NS
-#define COTT_POLL_SLEEP_NS 0
-#endif
-#ifndef COTT_WAIT_SLEEP_NS
-#define COTT_WAIT_SLEEP_NS 0
-#endif
-#ifndef COTT_WAIT_HINT_NS
-#define COTT_WAIT_HINT_NS 1000
-#endif
-constexpr uint32_t kWaitHintNs = COTT_WAIT_HINT_NS;   // a waiting thread may be parked this long per try
 
 #ifdef COTT_TIMING
 // Debug build only: SM-clock stamps of CTA 0, chunks kStampC0 .. + 3, eight slots for each of
@@ -172,49 +163,6 @@ __device__ __forceinline__ void issue_update(uint32_t tS, uint32_t vq, uint32_t 
     const uint32_t al = smem_desc_lo(vq, 16384), bl = smem_desc_lo(kdo, 16384);
 #pragma unroll
     for (int kk = 0; kk < kC / 16; ++kk) mma_ss_w(tS, al + kk * 128u, kDescHi, bl + kk * 128u, kDescHi, idesc, 1u);
-}
-
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-
-// Bounded wait that also gives up as soon as any thread of the CTA has given up.  The thread
-// that gives up first leaves a record of where: bit 31 set, warp index in bits 16-20, byte
-// offset of the barrier inside the barrier block in bits 4-13, parity in bit 0.
-// (The loop is a function of its own, not inlined: the kernel has some seventy waits, and its
-// code must stay small enough for the instruction caches -- eight roles run different code on
-// one SM at the same time.)
-__device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    const long long t0 = clock64();
-    for (uint32_t it = 1;; ++it) {
-        if (kWaitHintNs ? mbar_try_wait_hint(bar, parity, kWaitHintNs) : mbar_try_wait(bar, parity)) return true;
-#if COTT_WAIT_SLEEP_NS > 0
-        __nanosleep(COTT_WAIT_SLEEP_NS);      // a waiting warp must not take issue slots from the working ones
-#endif
-        if ((it & 15u) == 1) {
-            if (*abort_flag) return false;
-            // the limit (in units of 1024 SM cycles) sits three words behind the abort flag
-            if (clock64() - t0 > ((long long)abort_flag[3] << 10)) {
-                const uint32_t bars = (uint32_t)__cvta_generic_to_shared((const void*)abort_flag) - (uint32_t)L::kOffAbort;
-                const uint32_t where = 0x80000000u | ((threadIdx.x >> 5) << 16) | (((bar - bars) & 0x3FFu) << 4) | (parity & 1u);
-                atomicCAS(const_cast<int*>(abort_flag), 0, (int)where);
-                return false;
-            }
-        }
-    }
-}
-__device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    if (mbar_try_wait(bar, parity)) return true;
-    return wait_slow(bar, parity, abort_flag);
-}
-
-__device__ __forceinline__ uint4 pack8(const uint32_t* r) {
-    uint4 w;
-    w.x = pack_bf16(__uint_as_float(r[0]), __uint_as_float(r[1]));
-    w.y = pack_bf16(__uint_as_float(r[2]), __uint_as_float(r[3]));
-    w.z = pack_bf16(__uint_as_float(r[4]), __uint_as_float(r[5]));
-    w.w = pack_bf16(__uint_as_float(r[6]), __uint_as_float(r[7]));
-    return w;
 }
 
 // Thread roles.  Warps 0-15 are row workers (warp w owns TMEM lanes / tile rows

@@ -702,6 +702,29 @@ def test_chunk_count_boundaries_d64(N, pair, option):
     gate_dm(dm, rm, 1e-2, dm_condition(rv, c["v"], c["m"], None), DM_COND_BF16)
 
 
+@pytest.mark.parametrize("N", [1, 127, 128, 129, 256, 300, 384, 513, 640, 897, 1100])
+@pytest.mark.parametrize("fused", [1, 0])
+def test_chunk_count_boundaries_bidirectional_d64(N, fused, option, force_group):
+    """One to nine chunks through the one-launch bidirectional forward (two stages of (k, v)
+    pairs, four q slots, two output tiles: every ring starts, wraps and drains, with an odd and
+    an even number of chunks and a ragged last one) and through the two-launch form it replaces:
+    rows and the exported state against the definition."""
+    option("fused_bidir", fused)
+    force_group(4096)
+    c = synth.make_qkv(3, 7, N, 64, torch.bfloat16, 5500 + N)
+    q, k, v, m = (dev(c[x]) for x in ("q", "k", "v", "m"))
+    cott.cott.profile_enable(8)
+    o, st = cott.fwd(q, k, v, m, causal=False, return_state=True)
+    kinds = [kd for kd, _ in cott.cott.profile_read()]
+    cott.cott.profile_enable(0)
+    assert kinds == ([4] if fused else [0, 2])             # one launch / state pass + read-out
+    gate(o, oracle.fwd_quadratic(c["q"], c["k"], c["v"], c["m"], None, False), torch.bfloat16)
+    _, ref_state = oracle.fwd_bidir_assoc(c["q"], c["k"], c["v"], c["m"], None)
+    assert norm_max_err(st, ref_state) <= state_tol(torch.bfloat16, 64)
+    o2 = cott.fwd(q, k, v, m, causal=False)
+    assert torch.equal(o2, o)
+
+
 @pytest.mark.parametrize("dtype,d", [(torch.bfloat16, 128), (torch.bfloat16, 64), (torch.float32, 32)])
 def test_short_blocks_many_heads(dtype, d):
     """More (b,h) pairs than SMs and blocks of a few tokens (the shape of tokens between decode
@@ -728,21 +751,22 @@ def test_short_blocks_many_heads(dtype, d):
 
 
 # ------------------------------------------------------------------ a wait that runs out
-@pytest.mark.parametrize("op", ["fwd", "bwd"])
+@pytest.mark.parametrize("op", ["fwd", "bwd", "bidir"])
 def test_bounded_wait_runs_out_and_reports(op, option, force_group):
     """Every device-side wait has a bound.  With the bound set to zero a wait gives up unless
     its hand-off is there within a few polls -- and the first tiles of a kernel cannot come
     from memory that fast, so a wait is certain to run out.  The kernel then reports where,
     lets its copies in flight land, frees its tensor memory and returns; the context stays
     usable and the next call is correct.  (No GPU fault is involved: the kernels end normally.)"""
-    force_group(512)
+    causal = op != "bidir"
+    force_group(512 if causal else 4096)
     c = synth.make_qkv(1, 2, 1024, 64, torch.bfloat16, 5400, with_do=True)
     q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
-    code = cott.cott.OP_FWD if op == "fwd" else cott.cott.OP_BWD
-    ws = torch.zeros(cott.workspace_bytes(code, cott.cott.BF16, 1, 2, 1024, 64, True),
+    code = cott.cott.OP_BWD if op == "bwd" else cott.cott.OP_FWD
+    ws = torch.zeros(cott.workspace_bytes(code, cott.cott.BF16, 1, 2, 1024, 64, causal),
                      dtype=torch.uint8, device="cuda")
-    call = (lambda: cott.fwd(q, k, v, m, causal=True, workspace=ws)) if op == "fwd" else \
-           (lambda: cott.bwd(q, k, v, d_o, m, causal=True, workspace=ws))
+    call = (lambda: cott.bwd(q, k, v, d_o, m, causal=True, workspace=ws)) if op == "bwd" else \
+           (lambda: cott.fwd(q, k, v, m, causal=causal, workspace=ws))
     option("wait_limit_kcycles", 0)
     call()
     assert cott.cott.last_async_status(ws) == -5                 # COTT_ERR_TIMEOUT
@@ -752,8 +776,8 @@ def test_bounded_wait_runs_out_and_reports(op, option, force_group):
     option("wait_limit_kcycles", -1)
     out = call()
     assert cott.cott.last_async_status(ws) == 0
-    if op == "fwd":
-        gate(out, oracle.fwd_quadratic(c["q"], c["k"], c["v"], c["m"], None, True), torch.bfloat16)
+    if op != "bwd":
+        gate(out, oracle.fwd_quadratic(c["q"], c["k"], c["v"], c["m"], None, causal), torch.bfloat16)
     else:
         rq, rk, rv, _ = oracle.bwd_quadratic(c["q"], c["k"], c["v"], c["d_o"], c["m"], None, True)
         gate(out[0], rq, torch.bfloat16); gate(out[1], rk, torch.bfloat16); gate(out[2], rv, torch.bfloat16)
