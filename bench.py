@@ -35,7 +35,11 @@ L2_FLUSH_BYTES = 256 << 20  # larger than the 126 MB L2
 # by ALL launches of one step of a workload class, keyed by (d, causal, backward included).
 # A constant from a committed capture, not a measurement of this run: the JSON line says so.
 # Missing key: no capture of that class.
-STEP_DRAM_TRAFFIC = {}
+STEP_DRAM_TRAFFIC = {
+    (64, True, True): 1704.6,     # C4 step: 446.8 MB over 262 144 token-heads (method's bytes: 1408)
+    (64, False, False): 403.1,    # C2 forward: 79.3 MB over 196 608 token-heads (method's bytes: 512;
+                                  # a third of the output is still in L2 when the kernel ends)
+}
 
 
 def load_peaks():
@@ -80,6 +84,40 @@ def algorithmic_bytes(w: dict) -> dict:
         st = w["B"] * w["H"] * w["d"] * w["d"] * 4
         return {"fwd": 2 * st + 4 * w["B"] * w["H"] * w["d"] * 2, "bwd": 0}
     return {"fwd": 4 * th, "bwd": 7 * th if w["bwd"] else 0}
+
+
+def roofline_record(w: dict, peaks: dict, kernels_ms: float, kernel: str, fwd_ms: float,
+                    bwd_ms: float | None, step_ms: float) -> dict:
+    """The `roofline` object of the JSON line.  Bytes are the METHOD's (forward 8d and backward
+    14d per token-head in bf16: every tensor of the step once, whatever this implementation
+    re-reads); `frac` = those bytes / the summed duration of the step's kernel launches / the
+    copy bandwidth; `calls` holds the same bytes over whole calls (launch gaps and the small
+    scan and finalise kernels included)."""
+    ab = algorithmic_bytes(w)
+    alg = ab["fwd"] + ab["bwd"]
+    d = w["d"]
+    per_th = STEP_DRAM_TRAFFIC.get((d, bool(w["causal"]), bool(w.get("bwd"))))
+    if w.get("decode") or w.get("varlen"):
+        per_th = None
+    traffic = per_th * (w.get("rows", w["B"] * w["N"]) * w["H"]) if per_th else None
+    achieved = alg / (kernels_ms * 1e-3) / 1e9
+    frac_of = lambda nbytes, ms: nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]
+    rec = {
+        "bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+        "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
+        "algorithmic_bytes": alg,
+        "algorithmic_bytes_per_token_head": {"fwd": 8 * d, "bwd": 14 * d if w.get("bwd") else 0},
+        "ms": kernels_ms, "frac_of_nominal_8TBs": achieved / 8000.0,
+        "traffic": traffic,
+        "traffic_source": "ncu capture summarised under profiles/ (a constant, not measured in this run)",
+        "traffic_over_algorithmic": (traffic / alg) if traffic else None,
+        "goal": "causal forward at long N >= 0.60 of the measured copy bandwidth (peak above)",
+        "calls": {"fwd": {"ms": fwd_ms, "frac": frac_of(ab["fwd"], fwd_ms)},
+                  "step": {"ms": step_ms, "frac": frac_of(alg, step_ms)}},
+    }
+    if bwd_ms is not None:
+        rec["calls"]["bwd"] = {"ms": bwd_ms, "frac": frac_of(ab["bwd"], bwd_ms)}
+    return rec
 
 
 class ClockSampler:
@@ -524,26 +562,8 @@ def run_ours(args, w):
     else:
         dom_ms = statistics.mean(fwd_ms)
         kernel = "decode_kernel (fp32 SIMT, two CTAs per (b,h))" if w.get("decode") else "cott_fwd call (fp32 SIMT path)"
-    per_th = STEP_DRAM_TRAFFIC.get((d, bool(w["causal"]), bool(w.get("bwd"))))
-    traffic = per_th * (w.get("rows", B * N) * H) if per_th else None
-    achieved = alg / (dom_ms * 1e-3) / 1e9
-    roofline = {
-        "bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-        "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
-        "algorithmic_bytes": alg, "algorithmic_bytes_per_token_head": {"fwd": 8 * d, "bwd": 14 * d if w.get("bwd") else 0},
-        "ms": dom_ms, "frac_of_nominal_8TBs": achieved / 8000.0,
-        "traffic": traffic, "traffic_source": "ncu capture summarised under profiles/ (a constant, not measured in this run)",
-        "traffic_over_algorithmic": (traffic / alg) if traffic else None,
-        "goal": "causal forward at long N >= 0.60 of the measured copy bandwidth (peak above)",
-    }
-    # whole calls (launch gaps, scan and finalise kernels included), against the same bytes
-    fwd_mean = statistics.mean(fwd_ms)
-    frac_of = lambda nbytes, ms: nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]
-    roofline["calls"] = {"fwd": {"ms": fwd_mean, "frac": frac_of(ab["fwd"], fwd_mean)},
-                         "step": {"ms": step_ms_local, "frac": frac_of(alg, step_ms_local)}}
-    if bwd_call is not None:
-        bwd_mean = statistics.mean(bwd_ms)
-        roofline["calls"]["bwd"] = {"ms": bwd_mean, "frac": frac_of(ab["bwd"], bwd_mean)}
+    roofline = roofline_record(w, peaks, dom_ms, kernel, statistics.mean(fwd_ms),
+                               statistics.mean(bwd_ms) if bwd_call is not None else None, step_ms_local)
     extra = {"step_ms_unflushed_back_to_back": unflushed_ms}
     extra.update(loop_detail)
 

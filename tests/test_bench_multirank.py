@@ -37,3 +37,28 @@ def test_single_rank_is_identity():
     assert bench.dist_env()[1] >= 1
     ab = bench.algorithmic_bytes(bench.get_workload("c4"))
     assert ab["fwd"] == 4 * 4 * 16 * 4096 * 64 * 2 and ab["bwd"] == 7 * 4 * 16 * 4096 * 64 * 2
+
+
+def test_roofline_counts_the_methods_bytes_only():
+    """The roofline object divides the method's bytes (4 tensors forward, 7 backward, each once)
+    by the summed kernel time -- not the bytes the implementation chooses to re-read -- and
+    reports the whole-call fractions and the captured DRAM traffic next to it."""
+    sys.path.insert(0, ROOT)
+    import bench
+    w = bench.get_workload("c4")
+    peaks = {"hbm_gbs": 6550.7, "bf16_tflops": 1646.4, "source": "measured"}
+    tensor = 4 * 16 * 4096 * 64 * 2
+    r = bench.roofline_record(w, peaks, kernels_ms=0.1452, kernel="k", fwd_ms=0.050, bwd_ms=0.100, step_ms=0.150)
+    assert r["algorithmic_bytes"] == 11 * tensor
+    assert r["algorithmic_bytes_per_token_head"] == {"fwd": 8 * 64, "bwd": 14 * 64}
+    assert abs(r["frac"] - 11 * tensor / 0.1452e-3 / 1e9 / 6550.7) < 1e-12
+    assert abs(r["frac_of_nominal_8TBs"] - 11 * tensor / 0.1452e-3 / 1e9 / 8000.0) < 1e-12
+    assert abs(r["calls"]["fwd"]["frac"] - 4 * tensor / 0.050e-3 / 1e9 / 6550.7) < 1e-12
+    assert abs(r["calls"]["bwd"]["frac"] - 7 * tensor / 0.100e-3 / 1e9 / 6550.7) < 1e-12
+    assert abs(r["calls"]["step"]["frac"] - 11 * tensor / 0.150e-3 / 1e9 / 6550.7) < 1e-12
+    assert r["bound"] == "hbm" and r["peak"] == 6550.7 and r["peak_source"] == "measured"
+    # DRAM traffic from the committed capture: above the method's bytes (re-reads), below 1.5x
+    assert 1.0 < r["traffic_over_algorithmic"] < 1.5 and "not measured in this run" in r["traffic_source"]
+    # a forward-only workload counts four tensors and has no backward entry
+    r2 = bench.roofline_record(bench.get_workload("c2"), peaks, 0.03, "k", 0.034, None, 0.034)
+    assert r2["algorithmic_bytes"] == 4 * 32 * 12 * 512 * 64 * 2 and "bwd" not in r2["calls"]
