@@ -453,7 +453,11 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         constexpr bool two = L::kOutBufs > 0 && !L::kProjInA;   // two tile buffers (see below)
         const uint32_t proj_u = L::kProjInA ? stage_a(c % NST)
                                             : base + ((two && (c & 1)) ? L::kOffOutBuf + L::kTile : L::kOffProj);
-        const uint32_t pbar = two ? bar_proj + 8 * (c & 1) : bar_proj;
+        // One barrier per chunk parity wherever the tile of chunk c + 1 can be requested before
+        // the epilogue of chunk c has seen its own: arming a barrier whose phase still waits for
+        // bytes would be a second arrival on a count of one.  (In the A slot the request follows
+        // the state update of c + 1, which only follows the epilogue of c - 1.)
+        const uint32_t pbar = (two || L::kProjInA) ? bar_proj + 8 * (c & 1) : bar_proj;
         mbar_expect_tx(pbar, L::kTile);
         load_tile(proj_u, &tmP, pbar, chunk_row(c), 3);
     };
@@ -571,8 +575,9 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     // and A tiles: they are issued as soon as the tiles have landed, and the normalisation is
     // waited for before P~ Bv and the state update.
     constexpr bool kScoresOnFull = own_out && kNormBv;
-    auto proj_bar = [&](int c) { return proj2 ? bar_proj + 8 * (c & 1) : bar_proj; };
-    auto proj_par = [&](int c) { return (uint32_t)((proj2 ? (c >> 1) : c) & 1); };
+    constexpr bool proj_bar2 = proj2 || (with_proj && L::kProjInA);     // barrier per chunk parity (see load_proj)
+    auto proj_bar = [&](int c) { return proj_bar2 ? bar_proj + 8 * (c & 1) : bar_proj; };
+    auto proj_par = [&](int c) { return (uint32_t)((proj_bar2 ? (c >> 1) : c) & 1); };
     auto proj_off = [&](int c) { return (proj2 && (c & 1)) ? L::kOffOutBuf + L::kTile : L::kOffProj; };
     auto out_off = [&](int c) { return L::kOffOutBuf + (out_pair ? (c & 1) * L::kTile : 0); };
 
