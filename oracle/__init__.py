@@ -60,84 +60,87 @@ def _p(a: np.ndarray):
 
 def _prep(q, k, v, m, s):
     q, k, v, m = _f64(q), _f64(k), _f64(v), _f64(m).reshape(-1)
-    B, H, N, d = q.shape
-    assert k.shape == q.shape and v.shape == q.shape and m.shape == (H,)
+    B, H, N, dk = q.shape
+    dv = v.shape[-1]
+    assert k.shape == q.shape and v.shape == (B, H, N, dv) and m.shape == (H,)
     s = np.full((B,), float(N)) if s is None else _f64(s).reshape(-1)
     assert s.shape == (B,) and (s >= 1.0).all()
-    return q, k, v, m, s, B, H, N, d
+    return q, k, v, m, s, B, H, N, dk, dv
 
 
 def fwd_quadratic(q, k, v, m, s=None, causal=True) -> np.ndarray:
-    """Eq. 3/4 (bidirectional) or Eq. 6 (causal, diagonal kept): the definition."""
-    q, k, v, m, s, B, H, N, d = _prep(q, k, v, m, s)
-    o = np.empty_like(q)
+    """Eq. 3/4 (bidirectional) or Eq. 6 (causal, diagonal kept): the definition.
+    q, k ``[B,H,N,dk]``, v ``[B,H,N,dv]``; returns o ``[B,H,N,dv]``."""
+    q, k, v, m, s, B, H, N, dk, dv = _prep(q, k, v, m, s)
+    o = np.empty_like(v)
     _load().oracle_fwd_quadratic(_p(q), _p(k), _p(v), _p(m), _p(s), _p(o), B, H,
-                                 ctypes.c_long(N), d, int(bool(causal)))
+                                 ctypes.c_long(N), dk, dv, int(bool(causal)))
     return o
 
 
 def fwd_rows(q, k, v, m, rows, s=None, causal=True) -> np.ndarray:
-    """The definition on selected rows only; returns ``[B,H,len(rows),d]``."""
-    q, k, v, m, s, B, H, N, d = _prep(q, k, v, m, s)
+    """The definition on selected rows only; returns ``[B,H,len(rows),dv]``."""
+    q, k, v, m, s, B, H, N, dk, dv = _prep(q, k, v, m, s)
     rows = np.ascontiguousarray(np.asarray(rows, dtype=np.int64))
     assert rows.ndim == 1 and (rows >= 0).all() and (rows < N).all()
-    out = np.empty((B, H, len(rows), d))
+    out = np.empty((B, H, len(rows), dv))
     _load().oracle_fwd_rows(_p(q), _p(k), _p(v), _p(m), _p(s), _p(rows), len(rows), _p(out), B, H,
-                            ctypes.c_long(N), d, int(bool(causal)))
+                            ctypes.c_long(N), dk, dv, int(bool(causal)))
     return out
 
 
 def fwd_recurrent(q, k, v, m, s=None):
-    """Eq. 8 recurrence (causal).  Returns ``(o, final_state[B,H,d,d])``."""
-    q, k, v, m, s, B, H, N, d = _prep(q, k, v, m, s)
-    o = np.empty_like(q)
-    st = np.empty((B, H, d, d))
+    """Eq. 8 recurrence (causal).  Returns ``(o, final_state[B,H,dk,dv])``."""
+    q, k, v, m, s, B, H, N, dk, dv = _prep(q, k, v, m, s)
+    o = np.empty_like(v)
+    st = np.empty((B, H, dk, dv))
     _load().oracle_fwd_recurrent(_p(q), _p(k), _p(v), _p(m), _p(s), _p(o), _p(st), B, H,
-                                 ctypes.c_long(N), d)
+                                 ctypes.c_long(N), dk, dv)
     return o, st
 
 
 def fwd_bidir_assoc(q, k, v, m, s=None):
-    """Eq. 5 right-hand side.  Returns ``(o, state[B,H,d,d])``."""
-    q, k, v, m, s, B, H, N, d = _prep(q, k, v, m, s)
-    o = np.empty_like(q)
-    st = np.empty((B, H, d, d))
+    """Eq. 5 right-hand side.  Returns ``(o, state[B,H,dk,dv])``."""
+    q, k, v, m, s, B, H, N, dk, dv = _prep(q, k, v, m, s)
+    o = np.empty_like(v)
+    st = np.empty((B, H, dk, dv))
     _load().oracle_fwd_bidir_assoc(_p(q), _p(k), _p(v), _p(m), _p(s), _p(o), _p(st), B, H,
-                                   ctypes.c_long(N), d)
+                                   ctypes.c_long(N), dk, dv)
     return o, st
 
 
 def bwd_quadratic(q, k, v, d_o, m, s=None, causal=True):
     """Gradients of sum(dO*O) w.r.t. raw q,k,v and m.  Returns (dq,dk,dv,dm)."""
-    q, k, v, m, s, B, H, N, d = _prep(q, k, v, m, s)
+    q, k, v, m, s, B, H, N, dk, dv = _prep(q, k, v, m, s)
     d_o = _f64(d_o)
-    assert d_o.shape == q.shape
-    dq, dk, dv = np.empty_like(q), np.empty_like(q), np.empty_like(q)
+    assert d_o.shape == v.shape
+    dq, dk_, dv_ = np.empty_like(q), np.empty_like(q), np.empty_like(v)
     dm = np.empty((H,))
-    _load().oracle_bwd_quadratic(_p(q), _p(k), _p(v), _p(d_o), _p(m), _p(s), _p(dq), _p(dk),
-                                 _p(dv), _p(dm), B, H, ctypes.c_long(N), d, int(bool(causal)))
-    return dq, dk, dv, dm
+    _load().oracle_bwd_quadratic(_p(q), _p(k), _p(v), _p(d_o), _p(m), _p(s), _p(dq), _p(dk_),
+                                 _p(dv_), _p(dm), B, H, ctypes.c_long(N), dk, dv, int(bool(causal)))
+    return dq, dk_, dv_, dm
 
 
 def bwd_recurrent(q, k, v, d_o, m, s=None):
     """Causal backward via forward / reverse running sums.  Returns (dq,dk,dv,dm)."""
-    q, k, v, m, s, B, H, N, d = _prep(q, k, v, m, s)
+    q, k, v, m, s, B, H, N, dk, dv = _prep(q, k, v, m, s)
     d_o = _f64(d_o)
-    assert d_o.shape == q.shape
-    dq, dk, dv = np.empty_like(q), np.empty_like(q), np.empty_like(q)
+    assert d_o.shape == v.shape
+    dq, dk_, dv_ = np.empty_like(q), np.empty_like(q), np.empty_like(v)
     dm = np.empty((H,))
-    _load().oracle_bwd_recurrent(_p(q), _p(k), _p(v), _p(d_o), _p(m), _p(s), _p(dq), _p(dk),
-                                 _p(dv), _p(dm), B, H, ctypes.c_long(N), d)
-    return dq, dk, dv, dm
+    _load().oracle_bwd_recurrent(_p(q), _p(k), _p(v), _p(d_o), _p(m), _p(s), _p(dq), _p(dk_),
+                                 _p(dv_), _p(dm), B, H, ctypes.c_long(N), dk, dv)
+    return dq, dk_, dv_, dm
 
 
 def decode_step(q, k, v, m, s, state):
-    """One Eq. 8 step.  q,k,v ``[B,H,d]``; ``state`` ``[B,H,d,d]`` float64 numpy,
-    updated IN PLACE; ``s`` ``[B]`` or a scalar.  Returns o ``[B,H,d]``."""
+    """One Eq. 8 step.  q,k ``[B,H,dk]``, v ``[B,H,dv]``; ``state`` ``[B,H,dk,dv]`` float64 numpy,
+    updated IN PLACE; ``s`` ``[B]`` or a scalar.  Returns o ``[B,H,dv]``."""
     q, k, v, m = _f64(q), _f64(k), _f64(v), _f64(m).reshape(-1)
-    B, H, d = q.shape
+    B, H, dk = q.shape
+    dv = v.shape[-1]
     s = np.full((B,), float(s)) if np.isscalar(s) else _f64(s).reshape(-1)
-    assert state.dtype == np.float64 and state.flags.c_contiguous and state.shape == (B, H, d, d)
-    o = np.empty_like(q)
-    _load().oracle_decode_step(_p(q), _p(k), _p(v), _p(m), _p(s), _p(state), _p(o), B, H, d)
+    assert state.dtype == np.float64 and state.flags.c_contiguous and state.shape == (B, H, dk, dv)
+    o = np.empty_like(v)
+    _load().oracle_decode_step(_p(q), _p(k), _p(v), _p(m), _p(s), _p(state), _p(o), B, H, dk, dv)
     return o

@@ -7,8 +7,11 @@
  * the smoke check and the benchmark's cpu_baseline / reference arm use it.
  *
  * Notation (letters of the workload description, not the paper's):
- *   B batch, H heads, N sequence length, d per-head dimension.
- *   All tensors are contiguous row-major [B,H,N,d] doubles; m is [H];
+ *   B batch, H heads, N sequence length; dk, dv the per-head sizes of keys /
+ *   queries and of values / outputs (the paper's d_H_key and d_H_value of
+ *   section 2.1; most workloads have dk = dv = d).
+ *   q, k are contiguous row-major [B,H,N,dk] doubles, v, o, dO [B,H,N,dv];
+ *   states are [B,H,dk,dv]; m is [H];
  *   s is [B] (the "sequence length" scaling base of Eq. 4, one number per
  *   batch item, >= 1).
  *
@@ -82,25 +85,26 @@ static double dot(const double* x, const double* y, int d) {
  *   o_t = sum_{j in allowed(t)} (q^_t . k^_j) * c * v_j
  * --------------------------------------------------------------------- */
 void oracle_fwd_quadratic(const double* q, const double* k, const double* v, const double* m,
-                          const double* s, double* o, int B, int H, long N, int d, int causal) {
+                          const double* s, double* o, int B, int H, long N, int dk, int dv,
+                          int causal) {
 #pragma omp parallel for schedule(dynamic)
     for (long bh = 0; bh < (long)B * H; ++bh) {
         int b = (int)(bh / H), h = (int)(bh % H);
-        const double *Q = q + bh * N * d, *K = k + bh * N * d, *V = v + bh * N * d;
-        double* O = o + bh * N * d;
-        double* qh = malloc(sizeof(double) * N * d);
-        double* kh = malloc(sizeof(double) * N * d);
-        double* vp = malloc(sizeof(double) * N * d);
-        normalise_rows(Q, qh, NULL, N, d);
-        normalise_rows(K, kh, NULL, N, d);
+        const double *Q = q + bh * N * dk, *K = k + bh * N * dk, *V = v + bh * N * dv;
+        double* O = o + bh * N * dv;
+        double* qh = malloc(sizeof(double) * N * dk);
+        double* kh = malloc(sizeof(double) * N * dk);
+        double* vp = malloc(sizeof(double) * N * dv);
+        normalise_rows(Q, qh, NULL, N, dk);
+        normalise_rows(K, kh, NULL, N, dk);
         double c = stab_factor(s[b], m[h]);
-        for (long i = 0; i < N * d; ++i) vp[i] = V[i] * c;
+        for (long i = 0; i < N * dv; ++i) vp[i] = V[i] * c;
         for (long t = 0; t < N; ++t) {
-            for (int e = 0; e < d; ++e) O[t * d + e] = 0.0;
+            for (int e = 0; e < dv; ++e) O[t * dv + e] = 0.0;
             long jend = causal ? t + 1 : N; /* mask: ones on and below the diagonal */
             for (long j = 0; j < jend; ++j) {
-                double score = dot(qh + t * d, kh + j * d, d);
-                for (int e = 0; e < d; ++e) O[t * d + e] += score * vp[j * d + e];
+                double score = dot(qh + t * dk, kh + j * dk, dk);
+                for (int e = 0; e < dv; ++e) O[t * dv + e] += score * vp[j * dv + e];
             }
         }
         free(qh); free(kh); free(vp);
@@ -108,27 +112,27 @@ void oracle_fwd_quadratic(const double* q, const double* k, const double* v, con
 }
 
 /* The same definition evaluated only on the listed rows (for very long N).
- * rows[r] in [0,N); out is [B,H,nrows,d]. */
+ * rows[r] in [0,N); out is [B,H,nrows,dv]. */
 void oracle_fwd_rows(const double* q, const double* k, const double* v, const double* m,
                      const double* s, const long* rows, int nrows, double* out, int B, int H,
-                     long N, int d, int causal) {
+                     long N, int dk, int dv, int causal) {
 #pragma omp parallel for schedule(dynamic) collapse(2)
     for (long bh = 0; bh < (long)B * H; ++bh) {
         for (int r = 0; r < nrows; ++r) {
             int b = (int)(bh / H), h = (int)(bh % H);
-            const double *Q = q + bh * N * d, *K = k + bh * N * d, *V = v + bh * N * d;
+            const double *Q = q + bh * N * dk, *K = k + bh * N * dk, *V = v + bh * N * dv;
             long t = rows[r];
             double c = stab_factor(s[b], m[h]);
-            double* qh = malloc(sizeof(double) * d);
-            double* kh = malloc(sizeof(double) * d);
-            normalise_rows(Q + t * d, qh, NULL, 1, d);
-            double* O = out + (bh * nrows + r) * d;
-            for (int e = 0; e < d; ++e) O[e] = 0.0;
+            double* qh = malloc(sizeof(double) * dk);
+            double* kh = malloc(sizeof(double) * dk);
+            normalise_rows(Q + t * dk, qh, NULL, 1, dk);
+            double* O = out + (bh * nrows + r) * dv;
+            for (int e = 0; e < dv; ++e) O[e] = 0.0;
             long jend = causal ? t + 1 : N;
             for (long j = 0; j < jend; ++j) {
-                normalise_rows(K + j * d, kh, NULL, 1, d);
-                double score = dot(qh, kh, d);
-                for (int e = 0; e < d; ++e) O[e] += score * (V[j * d + e] * c);
+                normalise_rows(K + j * dk, kh, NULL, 1, dk);
+                double score = dot(qh, kh, dk);
+                for (int e = 0; e < dv; ++e) O[e] += score * (V[j * dv + e] * c);
             }
             free(qh); free(kh);
         }
@@ -139,65 +143,65 @@ void oracle_fwd_rows(const double* q, const double* k, const double* v, const do
  * Forward, recurrent form (Eq. 7 read as the recurrence of Eq. 8):
  *   S_0 = 0;  S_t = S_{t-1} + k^_t (c v_t)^T;  o_t = S_t^T q^_t.
  * The state is kept as [d_key][d_value] (the paper's H_t transposed).
- * state_out (may be NULL) receives S_N, [B,H,d,d].
+ * state_out (may be NULL) receives S_N, [B,H,dk,dv].
  * --------------------------------------------------------------------- */
 void oracle_fwd_recurrent(const double* q, const double* k, const double* v, const double* m,
                           const double* s, double* o, double* state_out, int B, int H, long N,
-                          int d) {
+                          int dk, int dv) {
 #pragma omp parallel for schedule(dynamic)
     for (long bh = 0; bh < (long)B * H; ++bh) {
         int b = (int)(bh / H), h = (int)(bh % H);
-        const double *Q = q + bh * N * d, *K = k + bh * N * d, *V = v + bh * N * d;
-        double* O = o + bh * N * d;
-        double* S = calloc((size_t)d * d, sizeof(double));
-        double* qh = malloc(sizeof(double) * d);
-        double* kh = malloc(sizeof(double) * d);
+        const double *Q = q + bh * N * dk, *K = k + bh * N * dk, *V = v + bh * N * dv;
+        double* O = o + bh * N * dv;
+        double* S = calloc((size_t)dk * dv, sizeof(double));
+        double* qh = malloc(sizeof(double) * dk);
+        double* kh = malloc(sizeof(double) * dk);
         double c = stab_factor(s[b], m[h]);
         for (long t = 0; t < N; ++t) {
-            normalise_rows(Q + t * d, qh, NULL, 1, d);
-            normalise_rows(K + t * d, kh, NULL, 1, d);
-            for (int a = 0; a < d; ++a)
-                for (int e = 0; e < d; ++e) S[a * d + e] += kh[a] * (V[t * d + e] * c);
-            for (int e = 0; e < d; ++e) {
+            normalise_rows(Q + t * dk, qh, NULL, 1, dk);
+            normalise_rows(K + t * dk, kh, NULL, 1, dk);
+            for (int a = 0; a < dk; ++a)
+                for (int e = 0; e < dv; ++e) S[a * dv + e] += kh[a] * (V[t * dv + e] * c);
+            for (int e = 0; e < dv; ++e) {
                 double acc = 0.0;
-                for (int a = 0; a < d; ++a) acc += qh[a] * S[a * d + e];
-                O[t * d + e] = acc;
+                for (int a = 0; a < dk; ++a) acc += qh[a] * S[a * dv + e];
+                O[t * dv + e] = acc;
             }
         }
-        if (state_out) memcpy(state_out + bh * d * d, S, sizeof(double) * d * d);
+        if (state_out) memcpy(state_out + bh * dk * dv, S, sizeof(double) * dk * dv);
         free(S); free(qh); free(kh);
     }
 }
 
 /* ------------------------------------------------------------------------
  * Bidirectional forward through the re-association of Eq. 5:
- *   S = K^^T (cV)  (d x d),   O = Q^ S.     state_out may be NULL.
+ *   S = K^^T (cV)  (dk x dv),   O = Q^ S.     state_out may be NULL.
  * --------------------------------------------------------------------- */
 void oracle_fwd_bidir_assoc(const double* q, const double* k, const double* v, const double* m,
                             const double* s, double* o, double* state_out, int B, int H, long N,
-                            int d) {
+                            int dk, int dv) {
 #pragma omp parallel for schedule(dynamic)
     for (long bh = 0; bh < (long)B * H; ++bh) {
         int b = (int)(bh / H), h = (int)(bh % H);
-        const double *Q = q + bh * N * d, *K = k + bh * N * d, *V = v + bh * N * d;
-        double* O = o + bh * N * d;
-        double* S = calloc((size_t)d * d, sizeof(double));
-        double* xh = malloc(sizeof(double) * d);
+        const double *Q = q + bh * N * dk, *K = k + bh * N * dk, *V = v + bh * N * dv;
+        double* O = o + bh * N * dv;
+        double* S = calloc((size_t)dk * dv, sizeof(double));
+        double* xh = malloc(sizeof(double) * dk);
         double c = stab_factor(s[b], m[h]);
         for (long j = 0; j < N; ++j) {
-            normalise_rows(K + j * d, xh, NULL, 1, d);
-            for (int a = 0; a < d; ++a)
-                for (int e = 0; e < d; ++e) S[a * d + e] += xh[a] * (V[j * d + e] * c);
+            normalise_rows(K + j * dk, xh, NULL, 1, dk);
+            for (int a = 0; a < dk; ++a)
+                for (int e = 0; e < dv; ++e) S[a * dv + e] += xh[a] * (V[j * dv + e] * c);
         }
         for (long t = 0; t < N; ++t) {
-            normalise_rows(Q + t * d, xh, NULL, 1, d);
-            for (int e = 0; e < d; ++e) {
+            normalise_rows(Q + t * dk, xh, NULL, 1, dk);
+            for (int e = 0; e < dv; ++e) {
                 double acc = 0.0;
-                for (int a = 0; a < d; ++a) acc += xh[a] * S[a * d + e];
-                O[t * d + e] = acc;
+                for (int a = 0; a < dk; ++a) acc += xh[a] * S[a * dv + e];
+                O[t * dv + e] = acc;
             }
         }
-        if (state_out) memcpy(state_out + bh * d * d, S, sizeof(double) * d * d);
+        if (state_out) memcpy(state_out + bh * dk * dv, S, sizeof(double) * dk * dv);
         free(S); free(xh);
     }
 }
@@ -221,14 +225,14 @@ static void normalise_backward_row(const double* xh, double nrm, const double* d
 static double chain_to_raw(const double* qh, const double* kh, const double* nq, const double* nk,
                            const double* V, const double* dqh, const double* dkh,
                            const double* dvp, double* dQ, double* dK, double* dV, double c,
-                           double s, double m, long N, int d) {
+                           double s, double m, long N, int dk, int dv) {
     double dLdc = 0.0;
     for (long t = 0; t < N; ++t) {
-        normalise_backward_row(qh + t * d, nq[t], dqh + t * d, dQ + t * d, d);
-        normalise_backward_row(kh + t * d, nk[t], dkh + t * d, dK + t * d, d);
-        for (int e = 0; e < d; ++e) {
-            dV[t * d + e] = c * dvp[t * d + e];
-            dLdc += dvp[t * d + e] * V[t * d + e];
+        normalise_backward_row(qh + t * dk, nq[t], dqh + t * dk, dQ + t * dk, dk);
+        normalise_backward_row(kh + t * dk, nk[t], dkh + t * dk, dK + t * dk, dk);
+        for (int e = 0; e < dv; ++e) {
+            dV[t * dv + e] = c * dvp[t * dv + e];
+            dLdc += dvp[t * dv + e] * V[t * dv + e];
         }
     }
     double sg = sigmoid(m);
@@ -243,38 +247,38 @@ static double chain_to_raw(const double* qh, const double* kh, const double* nq,
  * followed by the chain rule to raw q,k,v and m.  dm is [H], overwritten.
  * --------------------------------------------------------------------- */
 void oracle_bwd_quadratic(const double* q, const double* k, const double* v, const double* d_o,
-                          const double* m, const double* s, double* dq, double* dk, double* dv,
-                          double* dm, int B, int H, long N, int d, int causal) {
+                          const double* m, const double* s, double* dq, double* dk_out, double* dv_out,
+                          double* dm, int B, int H, long N, int dk, int dv, int causal) {
     double* dm_bh = calloc((size_t)B * H, sizeof(double));
 #pragma omp parallel for schedule(dynamic)
     for (long bh = 0; bh < (long)B * H; ++bh) {
         int b = (int)(bh / H), h = (int)(bh % H);
-        const double *Q = q + bh * N * d, *K = k + bh * N * d, *V = v + bh * N * d;
-        const double* dO = d_o + bh * N * d;
-        size_t nd = (size_t)N * d;
-        double *qh = malloc(sizeof(double) * nd), *kh = malloc(sizeof(double) * nd);
-        double *vp = malloc(sizeof(double) * nd);
+        const double *Q = q + bh * N * dk, *K = k + bh * N * dk, *V = v + bh * N * dv;
+        const double* dO = d_o + bh * N * dv;
+        size_t nk_ = (size_t)N * dk, nv_ = (size_t)N * dv;
+        double *qh = malloc(sizeof(double) * nk_), *kh = malloc(sizeof(double) * nk_);
+        double *vp = malloc(sizeof(double) * nv_);
         double *nq = malloc(sizeof(double) * N), *nk = malloc(sizeof(double) * N);
-        double *dqh = calloc(nd, sizeof(double)), *dkh = calloc(nd, sizeof(double));
-        double* dvp = calloc(nd, sizeof(double));
-        normalise_rows(Q, qh, nq, N, d);
-        normalise_rows(K, kh, nk, N, d);
+        double *dqh = calloc(nk_, sizeof(double)), *dkh = calloc(nk_, sizeof(double));
+        double* dvp = calloc(nv_, sizeof(double));
+        normalise_rows(Q, qh, nq, N, dk);
+        normalise_rows(K, kh, nk, N, dk);
         double c = stab_factor(s[b], m[h]);
-        for (size_t i = 0; i < nd; ++i) vp[i] = V[i] * c;
+        for (size_t i = 0; i < nv_; ++i) vp[i] = V[i] * c;
         for (long t = 0; t < N; ++t) {
             long jend = causal ? t + 1 : N;
             for (long j = 0; j < jend; ++j) {
-                double g = dot(dO + t * d, vp + j * d, d);      /* G[t][j]          */
-                double p = dot(qh + t * d, kh + j * d, d);      /* (Q^K^^T.M)[t][j] */
-                for (int a = 0; a < d; ++a) {
-                    dqh[t * d + a] += g * kh[j * d + a];
-                    dkh[j * d + a] += g * qh[t * d + a];
-                    dvp[j * d + a] += p * dO[t * d + a];
+                double g = dot(dO + t * dv, vp + j * dv, dv);   /* G[t][j]          */
+                double p = dot(qh + t * dk, kh + j * dk, dk);   /* (Q^K^^T.M)[t][j] */
+                for (int a = 0; a < dk; ++a) {
+                    dqh[t * dk + a] += g * kh[j * dk + a];
+                    dkh[j * dk + a] += g * qh[t * dk + a];
                 }
+                for (int e = 0; e < dv; ++e) dvp[j * dv + e] += p * dO[t * dv + e];
             }
         }
-        dm_bh[bh] = chain_to_raw(qh, kh, nq, nk, V, dqh, dkh, dvp, dq + bh * N * d,
-                                 dk + bh * N * d, dv + bh * N * d, c, s[b], m[h], N, d);
+        dm_bh[bh] = chain_to_raw(qh, kh, nq, nk, V, dqh, dkh, dvp, dq + bh * N * dk,
+                                 dk_out + bh * N * dk, dv_out + bh * N * dv, c, s[b], m[h], N, dk, dv);
         free(qh); free(kh); free(vp); free(nq); free(nk); free(dqh); free(dkh); free(dvp);
     }
     for (int h = 0; h < H; ++h) {
@@ -287,48 +291,48 @@ void oracle_bwd_quadratic(const double* q, const double* k, const double* v, con
 /* ------------------------------------------------------------------------
  * Causal backward in the running-sum form the paper describes: dQ^ uses the
  * forward cumulative state, dK^ and dV' use a cumulative sum that runs
- * backward in time:
+ * backward in time (both sums are dk x dv):
  *   S_t = sum_{j<=t} k^_j v'_j^T ,  dq^_t = S_t do_t
  *   R_j = sum_{t>=j} q^_t do_t^T ,  dk^_j = R_j v'_j ,  dv'_j = R_j^T k^_j
  * --------------------------------------------------------------------- */
 void oracle_bwd_recurrent(const double* q, const double* k, const double* v, const double* d_o,
-                          const double* m, const double* s, double* dq, double* dk, double* dv,
-                          double* dm, int B, int H, long N, int d) {
+                          const double* m, const double* s, double* dq, double* dk_out, double* dv_out,
+                          double* dm, int B, int H, long N, int dk, int dv) {
     double* dm_bh = calloc((size_t)B * H, sizeof(double));
 #pragma omp parallel for schedule(dynamic)
     for (long bh = 0; bh < (long)B * H; ++bh) {
         int b = (int)(bh / H), h = (int)(bh % H);
-        const double *Q = q + bh * N * d, *K = k + bh * N * d, *V = v + bh * N * d;
-        const double* dO = d_o + bh * N * d;
-        size_t nd = (size_t)N * d;
-        double *qh = malloc(sizeof(double) * nd), *kh = malloc(sizeof(double) * nd);
-        double *vp = malloc(sizeof(double) * nd);
+        const double *Q = q + bh * N * dk, *K = k + bh * N * dk, *V = v + bh * N * dv;
+        const double* dO = d_o + bh * N * dv;
+        size_t nk_ = (size_t)N * dk, nv_ = (size_t)N * dv;
+        double *qh = malloc(sizeof(double) * nk_), *kh = malloc(sizeof(double) * nk_);
+        double *vp = malloc(sizeof(double) * nv_);
         double *nq = malloc(sizeof(double) * N), *nk = malloc(sizeof(double) * N);
-        double *dqh = malloc(sizeof(double) * nd), *dkh = malloc(sizeof(double) * nd);
-        double* dvp = malloc(sizeof(double) * nd);
-        double* S = calloc((size_t)d * d, sizeof(double));
-        normalise_rows(Q, qh, nq, N, d);
-        normalise_rows(K, kh, nk, N, d);
+        double *dqh = malloc(sizeof(double) * nk_), *dkh = malloc(sizeof(double) * nk_);
+        double* dvp = malloc(sizeof(double) * nv_);
+        double* S = calloc((size_t)dk * dv, sizeof(double));
+        normalise_rows(Q, qh, nq, N, dk);
+        normalise_rows(K, kh, nk, N, dk);
         double c = stab_factor(s[b], m[h]);
-        for (size_t i = 0; i < nd; ++i) vp[i] = V[i] * c;
+        for (size_t i = 0; i < nv_; ++i) vp[i] = V[i] * c;
         for (long t = 0; t < N; ++t) { /* forward in time */
-            for (int a = 0; a < d; ++a)
-                for (int e = 0; e < d; ++e) S[a * d + e] += kh[t * d + a] * vp[t * d + e];
-            for (int a = 0; a < d; ++a) dqh[t * d + a] = dot(S + a * d, dO + t * d, d);
+            for (int a = 0; a < dk; ++a)
+                for (int e = 0; e < dv; ++e) S[a * dv + e] += kh[t * dk + a] * vp[t * dv + e];
+            for (int a = 0; a < dk; ++a) dqh[t * dk + a] = dot(S + a * dv, dO + t * dv, dv);
         }
-        memset(S, 0, sizeof(double) * d * d); /* now R */
+        memset(S, 0, sizeof(double) * dk * dv); /* now R */
         for (long j = N - 1; j >= 0; --j) { /* backward in time */
-            for (int a = 0; a < d; ++a)
-                for (int e = 0; e < d; ++e) S[a * d + e] += qh[j * d + a] * dO[j * d + e];
-            for (int a = 0; a < d; ++a) dkh[j * d + a] = dot(S + a * d, vp + j * d, d);
-            for (int e = 0; e < d; ++e) {
+            for (int a = 0; a < dk; ++a)
+                for (int e = 0; e < dv; ++e) S[a * dv + e] += qh[j * dk + a] * dO[j * dv + e];
+            for (int a = 0; a < dk; ++a) dkh[j * dk + a] = dot(S + a * dv, vp + j * dv, dv);
+            for (int e = 0; e < dv; ++e) {
                 double acc = 0.0;
-                for (int a = 0; a < d; ++a) acc += S[a * d + e] * kh[j * d + a];
-                dvp[j * d + e] = acc;
+                for (int a = 0; a < dk; ++a) acc += S[a * dv + e] * kh[j * dk + a];
+                dvp[j * dv + e] = acc;
             }
         }
-        dm_bh[bh] = chain_to_raw(qh, kh, nq, nk, V, dqh, dkh, dvp, dq + bh * N * d,
-                                 dk + bh * N * d, dv + bh * N * d, c, s[b], m[h], N, d);
+        dm_bh[bh] = chain_to_raw(qh, kh, nq, nk, V, dqh, dkh, dvp, dq + bh * N * dk,
+                                 dk_out + bh * N * dk, dv_out + bh * N * dv, c, s[b], m[h], N, dk, dv);
         free(qh); free(kh); free(vp); free(nq); free(nk); free(dqh); free(dkh); free(dvp); free(S);
     }
     for (int h = 0; h < H; ++h) {
@@ -341,25 +345,25 @@ void oracle_bwd_recurrent(const double* q, const double* k, const double* v, con
 /* ------------------------------------------------------------------------
  * One step of the recurrence of Eq. 8 on a caller-held state (in place):
  *   S <- S + k^ (c v)^T ;  o = S^T q^      (update first, then observe)
- * q,k,v,o are [B,H,d]; state is [B,H,d,d]; s is [B].
+ * q,k are [B,H,dk]; v,o [B,H,dv]; state is [B,H,dk,dv]; s is [B].
  * --------------------------------------------------------------------- */
 void oracle_decode_step(const double* q, const double* k, const double* v, const double* m,
-                        const double* s, double* state, double* o, int B, int H, int d) {
+                        const double* s, double* state, double* o, int B, int H, int dk, int dv) {
 #pragma omp parallel for schedule(dynamic)
     for (long bh = 0; bh < (long)B * H; ++bh) {
         int b = (int)(bh / H), h = (int)(bh % H);
-        double* S = state + bh * d * d;
-        double* qh = malloc(sizeof(double) * d);
-        double* kh = malloc(sizeof(double) * d);
-        normalise_rows(q + bh * d, qh, NULL, 1, d);
-        normalise_rows(k + bh * d, kh, NULL, 1, d);
+        double* S = state + bh * dk * dv;
+        double* qh = malloc(sizeof(double) * dk);
+        double* kh = malloc(sizeof(double) * dk);
+        normalise_rows(q + bh * dk, qh, NULL, 1, dk);
+        normalise_rows(k + bh * dk, kh, NULL, 1, dk);
         double c = stab_factor(s[b], m[h]);
-        for (int a = 0; a < d; ++a)
-            for (int e = 0; e < d; ++e) S[a * d + e] += kh[a] * (v[bh * d + e] * c);
-        for (int e = 0; e < d; ++e) {
+        for (int a = 0; a < dk; ++a)
+            for (int e = 0; e < dv; ++e) S[a * dv + e] += kh[a] * (v[bh * dv + e] * c);
+        for (int e = 0; e < dv; ++e) {
             double acc = 0.0;
-            for (int a = 0; a < d; ++a) acc += qh[a] * S[a * d + e];
-            o[bh * d + e] = acc;
+            for (int a = 0; a < dk; ++a) acc += qh[a] * S[a * dv + e];
+            o[bh * dv + e] = acc;
         }
         free(qh); free(kh);
     }

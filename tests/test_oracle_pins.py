@@ -289,3 +289,116 @@ def test_prefill_then_decode_equals_longer_forward():
         np.testing.assert_allclose(o, full[:, :, t], rtol=1e-11, atol=1e-12)
     _, st_full = oracle.fwd_recurrent(q, k, v, m, s)
     np.testing.assert_allclose(st, st_full, rtol=1e-12, atol=1e-13)
+
+
+# ------------------------------------------------------------------ different key and value sizes
+def _frac(x):
+    from fractions import Fraction
+    return np.array([[float(Fraction(e)) for e in row] for row in x])
+
+
+@pytest.fixture(scope="module")
+def hand_rect():
+    with open(os.path.join(HERE, "golden", "hand_example_dk2_dv3.json")) as f:
+        return json.load(f)
+
+
+def test_hand_example_with_different_key_and_value_sizes(hand_rect):
+    """d_key = 2, d_value = 3 (section 2.1 of the paper lets them differ): every tensor of the
+    forward, the final state and all gradients against fractions worked out by hand."""
+    g = hand_rect
+    t4 = lambda x: np.array(x, dtype=np.float64)[None, None]
+    q, k, v, d_o = t4(g["Q"]), t4(g["K"]), t4(g["V"]), t4(g["dO"])
+    m, s = np.array(g["m"]), np.array(g["s"])
+    tol = dict(rtol=0, atol=1e-14)
+    np.testing.assert_allclose(oracle.fwd_quadratic(q, k, v, m, s, True)[0, 0], _frac(g["O_causal"]), **tol)
+    np.testing.assert_allclose(oracle.fwd_quadratic(q, k, v, m, s, False)[0, 0], _frac(g["O_bidirectional"]), **tol)
+    o, st = oracle.fwd_recurrent(q, k, v, m, s)
+    assert st.shape == (1, 1, 2, 3)
+    np.testing.assert_allclose(o[0, 0], _frac(g["O_causal"]), **tol)
+    np.testing.assert_allclose(st[0, 0], _frac(g["state_final"]), **tol)
+    o, st = oracle.fwd_bidir_assoc(q, k, v, m, s)
+    np.testing.assert_allclose(o[0, 0], _frac(g["O_bidirectional"]), **tol)
+    np.testing.assert_allclose(st[0, 0], _frac(g["state_final"]), **tol)
+    np.testing.assert_allclose(oracle.fwd_rows(q, k, v, m, [1], s, True)[0, 0, 0], _frac(g["O_causal"])[1], **tol)
+    from fractions import Fraction
+    dm_ref = float(Fraction(g["dm_causal_over_ln4"])) * np.log(4.0)
+    for bwd in (oracle.bwd_quadratic, oracle.bwd_recurrent):
+        dq, dk, dv, dm = bwd(q, k, v, d_o, m, s)
+        np.testing.assert_allclose(dq[0, 0], _frac(g["dQ_causal"]), **tol)
+        np.testing.assert_allclose(dk[0, 0], _frac(g["dK_causal"]), **tol)
+        np.testing.assert_allclose(dv[0, 0], _frac(g["dV_causal"]), **tol)
+        np.testing.assert_allclose(dm[0], dm_ref, rtol=1e-13)
+    # one decode step per token reproduces the rows and the state
+    state = np.zeros((1, 1, 2, 3))
+    for t in range(2):
+        o_t = oracle.decode_step(q[:, :, t], k[:, :, t], v[:, :, t], m, s, state)
+        np.testing.assert_allclose(o_t[0, 0], _frac(g["O_causal"])[t], **tol)
+    np.testing.assert_allclose(state[0, 0], _frac(g["state_final"]), **tol)
+
+
+@pytest.mark.parametrize("dk,dv", [(3, 7), (8, 5), (16, 4)])
+@pytest.mark.parametrize("causal", [True, False])
+def test_unequal_sizes_are_the_square_problem_with_zero_columns(dk, dv, causal):
+    """Zero columns change no norm, no score and no product: the dk x dv problem embedded in a
+    square one of size max(dk, dv) by zero-padding q, k (or v, dO) must give the same outputs
+    and gradients, zeros in the padded columns -- which ties the rectangular code to the
+    square case every other pin covers.  The padded dq, dk columns are exactly zero only for
+    unclamped rows (all rows here)."""
+    B, H, N, D = 2, 2, 19, max(dk, dv)
+    q, k = rnd((B, H, N, dk), 71), rnd((B, H, N, dk), 72)
+    v, d_o = rnd((B, H, N, dv), 73), rnd((B, H, N, dv), 74)
+    m, s = rnd((H,), 75), np.array([7.0, 30.0])
+    pad = lambda x: np.concatenate([x, np.zeros(x.shape[:-1] + (D - x.shape[-1],))], axis=-1)
+    o = oracle.fwd_quadratic(q, k, v, m, s, causal)
+    o_sq = oracle.fwd_quadratic(pad(q), pad(k), pad(v), m, s, causal)
+    np.testing.assert_allclose(o_sq[..., :dv], o, rtol=1e-13, atol=1e-13)
+    assert np.all(o_sq[..., dv:] == 0.0)
+    got = oracle.bwd_quadratic(q, k, v, d_o, m, s, causal)
+    ref = oracle.bwd_quadratic(pad(q), pad(k), pad(v), pad(d_o), m, s, causal)
+    for g_, r_, w in zip(got[:3], ref[:3], (dk, dk, dv)):
+        np.testing.assert_allclose(r_[..., :w], g_, rtol=1e-12, atol=1e-12)
+        assert w == D or np.abs(r_[..., w:]).max() == 0.0
+    np.testing.assert_allclose(got[3], ref[3], rtol=1e-12)
+    if causal:
+        o_r, st = oracle.fwd_recurrent(q, k, v, m, s)
+        _, st_sq = oracle.fwd_recurrent(pad(q), pad(k), pad(v), m, s)
+        np.testing.assert_allclose(o_r, o, rtol=1e-12, atol=1e-12)
+        np.testing.assert_allclose(st_sq[:, :, :dk, :dv], st, rtol=1e-13, atol=1e-13)
+        rec = oracle.bwd_recurrent(q, k, v, d_o, m, s)
+        for a, b in zip(rec, got):
+            np.testing.assert_allclose(a, b, rtol=1e-10, atol=1e-10)
+    else:
+        o_a, st = oracle.fwd_bidir_assoc(q, k, v, m, s)
+        np.testing.assert_allclose(o_a, o, rtol=1e-12, atol=1e-12)
+        assert st.shape == (B, H, dk, dv)
+
+
+@pytest.mark.parametrize("causal", [True, False])
+def test_unequal_sizes_numpy_and_finite_differences(causal):
+    """dk = 5, dv = 3 against the masked-GEMM form in numpy, and the gradients against central
+    differences of the forward definition."""
+    B, H, N, dk, dv = 1, 2, 9, 5, 3
+    q, k = rnd((B, H, N, dk), 81), rnd((B, H, N, dk), 82)
+    v, d_o = rnd((B, H, N, dv), 83), rnd((B, H, N, dv), 84)
+    m, s = rnd((H,), 85), np.array([11.0])
+    np.testing.assert_allclose(oracle.fwd_quadratic(q, k, v, m, s, causal), numpy_forward(q, k, v, m, s, causal),
+                               rtol=1e-12, atol=1e-12)
+    dq, dk_, dv_, dm = oracle.bwd_quadratic(q, k, v, d_o, m, s, causal)
+    loss = lambda q_, k_, v_, m_: float((oracle.fwd_quadratic(q_, k_, v_, m_, s, causal) * d_o).sum())
+    eps = 1e-6
+    r = np.random.default_rng(86)
+    for name, x, g in (("q", q, dq), ("k", k, dk_), ("v", v, dv_)):
+        for _ in range(6):
+            idx = tuple(r.integers(0, n) for n in x.shape)
+            xp, xm = x.copy(), x.copy()
+            xp[idx] += eps; xm[idx] -= eps
+            args_p = {"q": (xp, k, v), "k": (q, xp, v), "v": (q, k, xp)}[name]
+            args_m = {"q": (xm, k, v), "k": (q, xm, v), "v": (q, k, xm)}[name]
+            fd = (loss(*args_p, m) - loss(*args_m, m)) / (2 * eps)
+            assert abs(fd - g[idx]) <= 1e-6 * max(1.0, abs(fd)), (name, idx, fd, g[idx])
+    for h in range(H):
+        mp, mm = m.copy(), m.copy()
+        mp[h] += eps; mm[h] -= eps
+        fd = (loss(q, k, v, mp) - loss(q, k, v, mm)) / (2 * eps)
+        assert abs(fd - dm[h]) <= 1e-6 * max(1.0, abs(fd))
