@@ -50,7 +50,7 @@ extern "C" {
 typedef enum {
     COTT_OK = 0,
     COTT_ERR_INVALID_ARG = -1, /* NULL required pointer, non-positive size, s < 1, aliasing      */
-    COTT_ERR_UNSUPPORTED = -2, /* d not in {32,64,128}, unknown dtype, pointer not 16-B aligned  */
+    COTT_ERR_UNSUPPORTED = -2, /* head size, dtype or alignment the kernels do not cover         */
     COTT_ERR_WORKSPACE = -3,   /* workspace NULL or smaller than cott_workspace_bytes()          */
     COTT_ERR_CUDA = -4,        /* a CUDA runtime / driver call failed (see cott_last_cuda_error) */
     COTT_ERR_TIMEOUT = -5      /* a bounded device-side wait expired (reported asynchronously)   */
@@ -273,6 +273,45 @@ cott_status cott_bwd_varlen(const void* q, const void* k, const void* v, const v
 cott_status cott_decode_step(const void* q, const void* k, const void* v, float* state, void* o,
                              int B, int H, int d, cott_dtype dt, const cott_scale_params* sp,
                              void* stream);
+
+/*
+ * Head sizes.  The paper's section 2.1 gives keys / queries and values sizes of their own
+ * (d_H_key, d_H_value); every call above takes one `d` for both.  The *_dkdv calls below take
+ * the two separately:
+ *   q, k (and dq, dk)     : [B,H,N,d_k]        v, o, dO (and dv) : [B,H,N,d_v]
+ *   states                : fp32 [B,H,d_k,d_v]  (S = sum_j k^_j (c v_j)^T)
+ * What is supported (either form of call):
+ *   bf16: any d_k, d_v that are multiples of 8 up to 128 (rows of 16 bytes) -- tensor-core
+ *         kernels of size 64 (both <= 64) or 128, the tiles zero-filled beyond the real
+ *         columns, which changes no norm, score or product; a caller's state passes through a
+ *         padded copy in the workspace (cott_workspace_bytes_dkdv accounts for it);
+ *   fp32: d_k = d_v in {32, 64, 128};
+ *   decode step: additionally any d_k, d_v up to 1024 that are multiples of 16 bytes.
+ * Packed (varlen) batches and cott_fwd_noalloc keep d in {64, 128}; cott_fwd_bwd_host takes one d.
+ * Strides: q and k share `qk_strides`, v has `v_strides`, o / dO `o_strides` / `do_strides`,
+ * dq and dk share `dqk_strides`, dv has `dv_strides` (NULL: dense for that tensor's own width;
+ * with d_k == d_v a NULL v_strides / dv_strides means "as q and k" / "as dq and dk").
+ * cott_fwd_dkdv is cott_fwd, cott_fwd_strided and cott_fwd_stateful in one: state_in non-NULL
+ * makes it the stateful call (causal only, scaling base required, see cott_fwd_stateful).
+ * cott_query_plan_dkdv also reports the size the kernels run at (*kernel_d; NULL allowed).
+ */
+size_t cott_workspace_bytes_dkdv(int op, cott_dtype dt, int B, int H, int N, int d_k, int d_v, int causal);
+cott_status cott_query_plan_dkdv(int op, cott_dtype dt, int B, int H, int N, int d_k, int d_v, int causal,
+                                 int* path, int* group, int* chunk, int* kernel_d);
+cott_status cott_fwd_dkdv(const void* q, const void* k, const void* v, void* o, const float* state_in,
+                          float* state_out, int B, int H, int N, int d_k, int d_v, int causal, cott_dtype dt,
+                          const cott_strides* qk_strides, const cott_strides* v_strides,
+                          const cott_strides* o_strides, const cott_scale_params* sp, void* workspace,
+                          size_t workspace_bytes, void* stream);
+cott_status cott_bwd_dkdv(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk,
+                          void* dv, float* dm, int B, int H, int N, int d_k, int d_v, int causal, cott_dtype dt,
+                          const cott_strides* qk_strides, const cott_strides* v_strides,
+                          const cott_strides* do_strides, const cott_strides* dqk_strides,
+                          const cott_strides* dv_strides, const cott_scale_params* sp, void* workspace,
+                          size_t workspace_bytes, void* stream);
+cott_status cott_decode_step_dkdv(const void* q, const void* k, const void* v, float* state, void* o,
+                                  int B, int H, int d_k, int d_v, cott_dtype dt, const cott_scale_params* sp,
+                                  void* stream);
 
 /*
  * Training step with HOST buffers (end-to-end path): copies q,k,v,d_o from host memory to the

@@ -65,6 +65,16 @@ def _load():
     lib.cott_workspace_bytes.argtypes = [ci, ci, ci, ci, ci, ci, ci]
     lib.cott_query_plan.restype = ci
     lib.cott_query_plan.argtypes = [ci] * 7 + [ctypes.POINTER(ci)] * 3
+    lib.cott_workspace_bytes_dkdv.restype = cs
+    lib.cott_workspace_bytes_dkdv.argtypes = [ci] * 8
+    lib.cott_query_plan_dkdv.restype = ci
+    lib.cott_query_plan_dkdv.argtypes = [ci] * 8 + [ctypes.POINTER(ci)] * 4
+    lib.cott_fwd_dkdv.restype = ci
+    lib.cott_fwd_dkdv.argtypes = [vp] * 6 + [ci] * 7 + [vp, vp, vp, ctypes.POINTER(_ScaleParams), vp, cs, vp]
+    lib.cott_bwd_dkdv.restype = ci
+    lib.cott_bwd_dkdv.argtypes = [vp] * 8 + [ci] * 7 + [vp] * 5 + [ctypes.POINTER(_ScaleParams), vp, cs, vp]
+    lib.cott_decode_step_dkdv.restype = ci
+    lib.cott_decode_step_dkdv.argtypes = [vp] * 5 + [ci] * 5 + [ctypes.POINTER(_ScaleParams), vp]
     lib.cott_fwd.restype = ci
     lib.cott_fwd.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci,
                              ctypes.POINTER(_ScaleParams), vp, cs, vp]
@@ -225,6 +235,48 @@ def query_plan(op: int, dt: int, B: int, H: int, N: int, d: int, causal: bool) -
     return {"path": path.value, "group": group.value, "chunk": chunk.value}
 
 
+def workspace_bytes_dkdv(op: int, dt: int, B: int, H: int, N: int, d_k: int, d_v: int, causal: bool) -> int:
+    n = _load().cott_workspace_bytes_dkdv(op, dt, B, H, N, d_k, d_v, int(bool(causal)))
+    if n == _SIZE_MAX:
+        raise CottError(-2, "cott_workspace_bytes_dkdv")
+    return int(n)
+
+
+def query_plan_dkdv(op: int, dt: int, B: int, H: int, N: int, d_k: int, d_v: int, causal: bool) -> dict:
+    path, group, chunk, kd = ctypes.c_int(), ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
+    rc = _load().cott_query_plan_dkdv(op, dt, B, H, N, d_k, d_v, int(bool(causal)), ctypes.byref(path),
+                                      ctypes.byref(group), ctypes.byref(chunk), ctypes.byref(kd))
+    if rc != 0:
+        raise CottError(rc, "cott_query_plan_dkdv")
+    return {"path": path.value, "group": group.value, "chunk": chunk.value, "kernel_d": kd.value}
+
+
+def _fwd_dkdv(q, k, v, m, seq_len, causal, state_in, return_state, out, workspace, stream):
+    """cott_fwd_dkdv: q, k ``[B,H,N,d_k]``, v ``[B,H,N,d_v]``; states ``[B,H,d_k,d_v]``."""
+    _check_rows(q, k, v)
+    _check_dev(m, state_in, seq_len if isinstance(seq_len, torch.Tensor) else None)
+    B, H, N, dk = q.shape
+    dv = v.shape[3]
+    dt = _dt(q)
+    if state_in is not None and (state_in.dtype != torch.float32 or tuple(state_in.shape) != (B, H, dk, dv)):
+        raise ValueError("state_in must be float32 [B,H,d_k,d_v]")
+    o = torch.empty_like(v) if out is None else out
+    _check_rows(o)
+    s_qk, s_v, s_o = _strides_of(q, k), _strides_of(v), _strides_of(o)
+    state = torch.empty((B, H, dk, dv), dtype=torch.float32, device=q.device) if return_state else None
+    need = workspace_bytes_dkdv(OP_FWD, dt, B, H, N, dk, dv, causal)
+    ws = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device) if workspace is None else workspace
+    sp = _scale(m, seq_len)
+    rc = _load().cott_fwd_dkdv(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
+                               state_in.data_ptr() if state_in is not None else None,
+                               state.data_ptr() if state is not None else None, B, H, N, dk, dv,
+                               int(bool(causal)), dt, _ref(s_qk), _ref(s_v), _ref(s_o), ctypes.byref(sp),
+                               ws.data_ptr(), ws.numel(), _stream_ptr(stream))
+    if rc != 0:
+        raise CottError(rc, "cott_fwd_dkdv")
+    return (o, state) if return_state else o
+
+
 def _workspace(op, dt, B, H, N, d, causal, device, workspace):
     need = workspace_bytes(op, dt, B, H, N, d, causal)
     if workspace is None:
@@ -240,6 +292,8 @@ def fwd(q, k, v, m, seq_len=None, causal=True, return_state=False, out=None, wor
     slices of a fused projection output; no copy is made.  ``seq_len``: None (s_b = N), a float,
     or a float32 ``[B]`` CUDA tensor.  Returns ``o`` (laid out like q when q is dense in
     memory, else dense ``[B,H,N,d]``; or ``out``) or ``(o, state[B,H,d,d] fp32)``."""
+    if v.shape[-1] != q.shape[-1]:      # different key and value sizes
+        return _fwd_dkdv(q, k, v, m, seq_len, causal, None, return_state, out, workspace, stream)
     _check_rows(q, k, v)
     _check_dev(m, seq_len if isinstance(seq_len, torch.Tensor) else None)
     B, H, N, d = q.shape
@@ -270,6 +324,10 @@ def fwd_stateful(q, k, v, m, seq_len, state_in=None, return_state=True, out=None
     _check_dev(m, state_in, seq_len if isinstance(seq_len, torch.Tensor) else None)
     if seq_len is None:
         raise ValueError("fwd_stateful needs the scaling base of the whole sequence")
+    if v.shape[-1] != q.shape[-1]:      # different key and value sizes
+        if state_in is None:
+            raise ValueError("with different key and value sizes a segment without a state is a plain fwd call")
+        return _fwd_dkdv(q, k, v, m, seq_len, True, state_in, return_state, out, workspace, stream)
     B, H, N, d = q.shape
     dt = _dt(q)
     if state_in is not None and (state_in.dtype != torch.float32 or tuple(state_in.shape) != (B, H, d, d)):
@@ -314,6 +372,22 @@ def bwd(q, k, v, d_o, m, seq_len=None, causal=True, workspace=None, stream=None,
     _check_dev(m, seq_len if isinstance(seq_len, torch.Tensor) else None)
     B, H, N, d = q.shape
     dt = _dt(q)
+    if v.shape[-1] != d:                # different key and value sizes: cott_bwd_dkdv
+        d_v = v.shape[-1]
+        dq, dk, dv = (torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)) if out is None else out
+        _check_rows(dq, dk, dv)
+        dm = torch.empty((H,), dtype=torch.float32, device=q.device)
+        need = workspace_bytes_dkdv(OP_BWD, dt, B, H, N, d, d_v, causal)
+        ws = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device) if workspace is None else workspace
+        sp = _scale(m, seq_len)
+        st = [_strides_of(q, k), _strides_of(v), _strides_of(d_o), _strides_of(dq, dk), _strides_of(dv)]
+        rc = _load().cott_bwd_dkdv(q.data_ptr(), k.data_ptr(), v.data_ptr(), d_o.data_ptr(), dq.data_ptr(),
+                                   dk.data_ptr(), dv.data_ptr(), dm.data_ptr(), B, H, N, d, d_v,
+                                   int(bool(causal)), dt, *[_ref(x) for x in st], ctypes.byref(sp),
+                                   ws.data_ptr(), ws.numel(), _stream_ptr(stream))
+        if rc != 0:
+            raise CottError(rc, "cott_bwd_dkdv")
+        return dq, dk, dv, dm
     dq, dk, dv = (torch.empty_like(q), torch.empty_like(q), torch.empty_like(q)) if out is None else out
     _check_rows(dq, dk, dv)
     s_qkv, s_do, s_dqkv = _strides_of(q, k, v), _strides_of(d_o), _strides_of(dq, dk, dv)
@@ -387,10 +461,17 @@ def decode_step(q, k, v, state, m, seq_len, out=None, stream=None):
     ``seq_len`` a float (>= 1) or a float32 ``[B]`` CUDA tensor.  Returns ``o [B,H,d]``."""
     _check_dev(q, k, v, state, m, seq_len if isinstance(seq_len, torch.Tensor) else None)
     B, H, d = q.shape
-    if state.dtype != torch.float32 or tuple(state.shape) != (B, H, d, d):
-        raise ValueError("state must be float32 [B,H,d,d]")
-    o = torch.empty_like(q) if out is None else out
+    d_v = v.shape[-1]
+    if state.dtype != torch.float32 or tuple(state.shape) != (B, H, d, d_v):
+        raise ValueError("state must be float32 [B,H,d_k,d_v]")
+    o = torch.empty_like(v) if out is None else out
     sp = _scale(m, seq_len)
+    if d_v != d:
+        rc = _load().cott_decode_step_dkdv(q.data_ptr(), k.data_ptr(), v.data_ptr(), state.data_ptr(), o.data_ptr(),
+                                           B, H, d, d_v, _dt(q), ctypes.byref(sp), _stream_ptr(stream))
+        if rc != 0:
+            raise CottError(rc, "cott_decode_step_dkdv")
+        return o
     rc = _load().cott_decode_step(q.data_ptr(), k.data_ptr(), v.data_ptr(), state.data_ptr(),
                                   o.data_ptr(), B, H, d, _dt(q), ctypes.byref(sp),
                                   _stream_ptr(stream))

@@ -116,19 +116,31 @@ struct Plan {
     int chunk;     // tokens per chunk inside a group
     int n_groups;
     int split;   // partial-state pass: parts per group when the walk sums the prefix itself
+    // Head sizes: dk columns in q, k (and dq, dk), dv in v, o, dO (and dv).  `d` is the size the
+    // kernels run at: dk = dv = d on the fp32-accumulating SIMT path; on the tensor-core path
+    // the smallest of 64 and 128 that holds both, the tiles zero-filled beyond the real columns
+    // (`padded`: a caller's state then goes through a [BH, d, d] copy in the workspace).
+    int d, dk, dv;
+    bool padded;
 };
 
 // Sequence groups give sequence-level parallelism when B*H alone cannot fill the GPU:
 // halve the group until there are enough CTAs, but never below a floor that keeps the
 // per-group state traffic (d*d fp32) small against the group's own q,k,v,o bytes.
-static bool make_plan(int op, cott_dtype dt, int B, int H, int N, int d, int causal, Plan* p) {
+static bool make_plan(int op, cott_dtype dt, int B, int H, int N, int dk, int dv, int causal, Plan* p) {
     if (B < 1 || H < 1 || N < 1) return false;
-    if (d != 32 && d != 64 && d != 128) return false;
     if (dt != COTT_F32 && dt != COTT_BF16) return false;
     const long BH = (long)B * H;
     const int forced = option_force_group();
-    const bool tc_ok = dt == COTT_BF16 && (d == 64 || d == 128);
-    p->path = (tc_ok && option_force_path() != 0) ? 1 : 0;
+    // Tensor cores: bf16, head sizes that are multiples of 8 (16-byte rows) up to 128.
+    const bool tc_ok = dt == COTT_BF16 && dk >= 8 && dv >= 8 && dk <= 128 && dv <= 128 && dk % 8 == 0 && dv % 8 == 0;
+    const bool simt_ok = dk == dv && (dk == 32 || dk == 64 || dk == 128);
+    if (!tc_ok && !simt_ok) return false;
+    p->path = (tc_ok && (option_force_path() != 0 || !simt_ok)) ? 1 : 0;
+    p->dk = dk; p->dv = dv;
+    p->d = p->path == 1 ? ((dk <= 64 && dv <= 64) ? 64 : 128) : dk;
+    p->padded = dk != p->d || dv != p->d;
+    const int d = p->d;
     int group;
     if (p->path == 1) {
         // One CTA per (b,h) and group, one CTA per SM.  Measured on B200: fewer, longer
@@ -177,9 +189,14 @@ static size_t states_bytes(const Plan& p, int B, int H, int d) {
     return align_up((size_t)B * H * p.n_groups * p.split * d * d * sizeof(float), 256);
 }
 
+// (padded head sizes: room for a caller's initial and final state in the kernels' size)
+static size_t padded_state_bytes(const Plan& p, int B, int H) {
+    return p.padded ? align_up((size_t)B * H * p.d * p.d * sizeof(float), 256) : 0;
+}
+
 static size_t workspace_bytes_impl(int op, const Plan& p, int B, int H, int d) {
     size_t total = kWsHeaderBytes;
-    if (op == COTT_OP_FWD) total += states_bytes(p, B, H, d);
+    if (op == COTT_OP_FWD) total += states_bytes(p, B, H, d) + 2 * padded_state_bytes(p, B, H);
     else if (op == COTT_OP_BWD)
         total += 3 * states_bytes(p, B, H, d) + 2 * align_up((size_t)B * H * p.n_groups * 4, 256);
     return total;
@@ -195,15 +212,25 @@ static cott_status check_scale(const cott_scale_params* sp) {
 struct CallLayouts {
     RowLayout qkv, o, dqkv;
     const void* q; const void* k; const void* v; const void* o_or_do;
+    // Different key and value sizes: v and dv may have layouts of their own (dense tensors of
+    // another width), and every tensor has its own column count.
+    RowLayout vl, dvl;
+    bool own_v = false;
+    const void* dv_ptr = nullptr;
+    int dk = 0, dv = 0;
     RowLayout of(const void* ptr) const {
+        if (ptr == v && own_v) return vl;
         if (ptr == q || ptr == k || ptr == v) return qkv;
         if (ptr == o_or_do) return o;
+        if (ptr == dv_ptr && own_v) return dvl;
         return dqkv;
     }
+    int width(const void* ptr) const { return (ptr == v || ptr == o_or_do || ptr == dv_ptr) ? dv : dk; }
     template <class Args> void assign(Args& a) const {
         a.lx = of(a.x); a.la = of(a.a); a.lbv = of(a.bv); a.lproj = of(a.proj);
-        a.lout = (a.out == o_or_do) ? o : dqkv;
+        a.lout = (a.out == o_or_do) ? o : of(a.out);
     }
+    void assign_widths(TcWalkArgs& a) const { a.d_xa = width(a.x ? a.x : a.a); a.d_bo = width(a.bv); }
 };
 static RowLayout to_layout(const cott_strides* s) {
     return s ? RowLayout{s->batch, s->head, s->token} : RowLayout{0, 0, 0};
@@ -252,10 +279,11 @@ static bool same_strides(const cott_strides* a, const cott_strides* b) {
     return a->batch == b->batch && a->head == b->head && a->token == b->token;
 }
 static bool tensors_overlap(const void* pa, const cott_strides* sa, const void* pb, const cott_strides* sb2,
-                            int B, int H, int N, int d, cott_dtype dt) {
+                            int B, int H, int N, int d, cott_dtype dt, int d_b = 0) {
     if (pa == pb) return true;
     const long long es = (long long)dtype_size(dt);
-    const Extent a = extent_of(sa, B, H, N, d), b = extent_of(sb2, B, H, N, d);
+    const Extent a = extent_of(sa, B, H, N, d);
+    const Extent b = extent_of(sb2, B, H, N, d_b > 0 ? d_b : d);
     const long long a0 = (long long)reinterpret_cast<uintptr_t>(pa), b0 = (long long)reinterpret_cast<uintptr_t>(pb);
     const bool ranges = a0 < b0 + b.span * es && b0 < a0 + a.span * es;
     if (!ranges) return false;
@@ -263,7 +291,8 @@ static bool tensors_overlap(const void* pa, const cott_strides* sa, const void* 
     if (same_strides(sa, sb2) && a.lattice && a.step > 0) {
         long long delta = ((b0 - a0) / es) % a.step;                       // (bases are element-aligned)
         if (delta < 0) delta += a.step;
-        return delta < a.block || a.step - delta < a.block;
+        // rows of a cover [0, a.block) of every period, rows of b [delta, delta + b.block)
+        return delta < a.block || a.step - delta < b.block;
     }
     return false;
 }
@@ -369,29 +398,51 @@ static cott_status fwd_impl(const void* q, const void* k, const void* v, void* o
                             const cott_scale_params* sp, void* ws, const Plan& p,
                             cudaStream_t st, const float* state_in = nullptr,
                             const cott_strides* s_qkv = nullptr, const cott_strides* s_o = nullptr,
-                            Packed packed = Packed()) {
-    const CallLayouts lay{to_layout(s_qkv), to_layout(s_o), RowLayout{0, 0, 0}, q, k, v, o};
+                            Packed packed = Packed(), const cott_strides* s_v = nullptr) {
+    // (d is the size the kernels run at, p.d; the tensors have p.dk and p.dv columns)
+    CallLayouts lay{to_layout(s_qkv), to_layout(s_o), RowLayout{0, 0, 0}, q, k, v, o};
+    lay.dk = p.dk; lay.dv = p.dv;
+    if (p.dk != p.dv || s_v) { lay.own_v = true; lay.vl = to_layout(s_v); }
     // The tensor-core path clears the status words in its first kernel.
     if (p.path != 1) COTT_CUDA(cudaMemsetAsync(ws, 0, kWsHeaderBytes, st));
     float* states = reinterpret_cast<float*>(static_cast<char*>(ws) + kWsHeaderBytes);
+    // Zero-padded head sizes: the kernels read and write states of their own size.
+    float* user_state_out = state_out;
+    if (p.padded && (state_in || state_out)) {
+        char* pad0 = static_cast<char*>(ws) + kWsHeaderBytes + states_bytes(p, B, H, d);
+        float* pad_in = reinterpret_cast<float*>(pad0);
+        float* pad_out = reinterpret_cast<float*>(pad0 + padded_state_bytes(p, B, H));
+        if (state_in) {
+            COTT_CUDA(launch_pad_state(state_in, pad_in, B * H, p.dk, p.dv, d, st));
+            state_in = pad_in;
+        }
+        if (state_out) state_out = pad_out;
+    }
+    auto finish = [&]() -> cott_status {
+        if (state_out != user_state_out)
+            COTT_CUDA(launch_unpad_state(state_out, user_state_out, B * H, p.dk, p.dv, d, st));
+        return COTT_OK;
+    };
     if (p.path == 1 && !causal && d == 64 && p.n_groups == 1 && !packed.cu_seqlens && !state_in &&
         option_fused_bidir() != 0) {
         // One CTA per (b, h) streams k, v into the d x d state and then q through it: one launch,
         // every tensor touched once.
-        COTT_CUDA(launch_tc_bidir_fwd(q, k, v, o, lay.qkv, lay.o, state_out, static_cast<int*>(ws), sp->m, sp->seq_len,
-                                      sp->seq_len_scalar, B, H, N, st));
-        return COTT_OK;
+        COTT_CUDA(launch_tc_bidir_fwd(q, k, v, o, lay.qkv, lay.of(v), lay.o, state_out, static_cast<int*>(ws), sp->m,
+                                      sp->seq_len, sp->seq_len_scalar, B, H, N, st, p.dk, p.dv));
+        return finish();
     }
     if (p.path == 1) {
         TcWalkArgs t;
         memset(&t, 0, sizeof(t));
         t.x = q; t.a = k; t.bv = v; t.out = o;
-        lay.assign(t);
+        lay.assign(t); lay.assign_widths(t);
         t.cu_seqlens = packed.cu_seqlens; t.total_tokens = packed.total_tokens;
         t.norm_bv = 0; t.x_norm = 1; t.epilogue = EPI_PLAIN; t.reverse = 0;
+        // (a padded initial state was staged by a kernel of this call: the walk is not the first)
         t.clear_status = 1;
-        return run_tc_stream(t, p, B, H, N, d, causal, sp, static_cast<int*>(ws), states,
-                             state_out, st, false, false, true, state_in);
+        cott_status rc = run_tc_stream(t, p, B, H, N, d, causal, sp, static_cast<int*>(ws), states,
+                                       state_out, st, false, false, true, state_in);
+        return rc != COTT_OK ? rc : finish();
     }
     WalkArgs w = base_walk(sp, H, N, p);
     w.x = q; w.a = k; w.bv = v; w.out = o;
@@ -447,8 +498,12 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
                             cott_dtype dt, const cott_scale_params* sp, void* ws, const Plan& p,
                             cudaStream_t st, const cott_strides* s_qkv = nullptr,
                             const cott_strides* s_do = nullptr, const cott_strides* s_dqkv = nullptr,
-                            Packed packed = Packed()) {
-    const CallLayouts lay{to_layout(s_qkv), to_layout(s_do), to_layout(s_dqkv), q, k, v, d_o};
+                            Packed packed = Packed(), const cott_strides* s_v = nullptr,
+                            const cott_strides* s_dv = nullptr) {
+    // (d is the size the kernels run at, p.d; the tensors have p.dk and p.dv columns)
+    CallLayouts lay{to_layout(s_qkv), to_layout(s_do), to_layout(s_dqkv), q, k, v, d_o};
+    lay.dk = p.dk; lay.dv = p.dv; lay.dv_ptr = dv;
+    if (p.dk != p.dv || s_v || s_dv) { lay.own_v = true; lay.vl = to_layout(s_v); lay.dvl = to_layout(s_dv); }
     // The tensor-core path clears the status words in its first kernel.
     if (p.path != 1) COTT_CUDA(cudaMemsetAsync(ws, 0, kWsHeaderBytes, st));
     char* base = static_cast<char*>(ws) + kWsHeaderBytes;
@@ -480,6 +535,7 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
             memset(&f, 0, sizeof(f));
             f.q = q; f.k = k; f.v = v; f.d_o = d_o; f.dq = dq; f.dk = dk; f.dv = dv;
             f.l_qkv = lay.qkv; f.l_do = lay.o; f.l_dqkv = lay.dqkv;
+            f.l_v = lay.of(v); f.l_dv = lay.of(dv); f.w_k = p.dk; f.w_v = p.dv;
             f.sq_part = st0; f.r_part = st1;
             f.dm_partial = dm_partial; f.dm_out = dm; f.status = status;
             f.m = sp->m; f.seq_len = sp->seq_len; f.seq_len_scalar = sp->seq_len_scalar;
@@ -517,6 +573,7 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
         tq.dm_partial = dm_partial;
         tq.dm_out = dm;
         lay.assign(tq); lay.assign(tk); lay.assign(tv);
+        lay.assign_widths(tq); lay.assign_widths(tk); lay.assign_widths(tv);
         if (ss) {
             struct TagScope { ~TagScope() { g_prof_cur_tag = 0; } } tag_scope;
             // Everything that follows a cross-stream event wait is a plain launch.
@@ -666,31 +723,78 @@ long long cott_get_option(const char* name) {
 
 unsigned long long cott_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
-size_t cott_workspace_bytes(int op, cott_dtype dt, int B, int H, int N, int d, int causal) {
+size_t cott_workspace_bytes_dkdv(int op, cott_dtype dt, int B, int H, int N, int d_k, int d_v, int causal) {
     if (op == COTT_OP_DECODE) return 0;
     if (op != COTT_OP_FWD && op != COTT_OP_BWD) return (size_t)-1;
     Plan p;
-    if (!make_plan(op, dt, B, H, N, d, causal, &p)) return (size_t)-1;
-    return workspace_bytes_impl(op, p, B, H, d);
+    if (!make_plan(op, dt, B, H, N, d_k, d_v, causal, &p)) return (size_t)-1;
+    return workspace_bytes_impl(op, p, B, H, p.d);
+}
+
+size_t cott_workspace_bytes(int op, cott_dtype dt, int B, int H, int N, int d, int causal) {
+    return cott_workspace_bytes_dkdv(op, dt, B, H, N, d, d, causal);
+}
+
+cott_status cott_query_plan_dkdv(int op, cott_dtype dt, int B, int H, int N, int d_k, int d_v, int causal,
+                                 int* path, int* group, int* chunk, int* kernel_d) {
+    Plan p;
+    if (op == COTT_OP_DECODE) { p.path = 0; p.group = 1; p.chunk = 1; p.d = d_k > d_v ? d_k : d_v; }
+    else if (!make_plan(op, dt, B, H, N, d_k, d_v, causal, &p)) return COTT_ERR_UNSUPPORTED;
+    if (path) *path = p.path;
+    if (group) *group = p.group;
+    if (chunk) *chunk = p.chunk;
+    if (kernel_d) *kernel_d = p.d;
+    return COTT_OK;
 }
 
 cott_status cott_query_plan(int op, cott_dtype dt, int B, int H, int N, int d, int causal,
                             int* path, int* group, int* chunk) {
+    return cott_query_plan_dkdv(op, dt, B, H, N, d, d, causal, path, group, chunk, nullptr);
+}
+
+// Validation and dispatch shared by every dense / strided forward entry point.
+static cott_status fwd_entry(const void* q, const void* k, const void* v, void* o, const float* state_in,
+                             float* state_out, int B, int H, int N, int d_k, int d_v, int causal, bool stateful,
+                             cott_dtype dt, const cott_strides* qk_strides, const cott_strides* v_strides,
+                             const cott_strides* o_strides, const cott_scale_params* sp, void* workspace,
+                             size_t workspace_bytes, void* stream) {
+    if (!q || !k || !v || !o || B < 1 || H < 1 || N < 1 || d_k < 1 || d_v < 1) return COTT_ERR_INVALID_ARG;
+    const cott_strides* vs = v_strides ? v_strides : (d_k == d_v ? qk_strides : nullptr);
+    if (!layout_ok(qk_strides, d_k, dt) || !layout_ok(vs, d_v, dt) || !layout_ok(o_strides, d_v, dt))
+        return COTT_ERR_UNSUPPORTED;
+    if (check_scale(sp) != COTT_OK) return COTT_ERR_INVALID_ARG;
+    if (tensors_overlap(o, o_strides, q, qk_strides, B, H, N, d_v, dt, d_k) ||
+        tensors_overlap(o, o_strides, k, qk_strides, B, H, N, d_v, dt, d_k) ||
+        tensors_overlap(o, o_strides, v, vs, B, H, N, d_v, dt, d_v))
+        return COTT_ERR_INVALID_ARG;
+    if (stateful) {
+        if (!causal) return COTT_ERR_INVALID_ARG;
+        if (state_in && state_in == state_out) return COTT_ERR_INVALID_ARG;
+        // the scaling base must be the caller's (the same for every segment of a sequence)
+        if (!sp->seq_len && !(sp->seq_len_scalar >= 1.f)) return COTT_ERR_INVALID_ARG;
+    } else {
+        if (state_in) return COTT_ERR_INVALID_ARG;
+        if (!sp->seq_len && sp->seq_len_scalar > 0.f && sp->seq_len_scalar < 1.f) return COTT_ERR_INVALID_ARG;
+    }
     Plan p;
-    if (op == COTT_OP_DECODE) { p.path = 0; p.group = 1; p.chunk = 1; }
-    else if (!make_plan(op, dt, B, H, N, d, causal, &p)) return COTT_ERR_UNSUPPORTED;
-    if (path) *path = p.path;
-    if (group) *group = p.group;
-    if (chunk) *chunk = p.chunk;
-    return COTT_OK;
+    if (!make_plan(COTT_OP_FWD, dt, B, H, N, d_k, d_v, causal, &p)) return COTT_ERR_UNSUPPORTED;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) ||
+        (state_in && !aligned16(state_in)) || (state_out && !aligned16(state_out)))
+        return COTT_ERR_UNSUPPORTED;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
+        workspace_bytes < workspace_bytes_impl(COTT_OP_FWD, p, B, H, p.d))
+        return COTT_ERR_WORKSPACE;
+    return fwd_impl(q, k, v, o, state_out, B, H, N, p.d, causal, dt, sp, workspace, p,
+                    static_cast<cudaStream_t>(stream), state_in, qk_strides, o_strides, Packed(),
+                    (d_k != d_v || v_strides) ? vs : nullptr);
 }
 
 cott_status cott_fwd(const void* q, const void* k, const void* v, void* o, float* state_out,
                      int B, int H, int N, int d, int causal, cott_dtype dt,
                      const cott_scale_params* sp, void* workspace, size_t workspace_bytes,
                      void* stream) {
-    return cott_fwd_strided(q, k, v, o, state_out, B, H, N, d, causal, dt, nullptr, nullptr, sp,
-                            workspace, workspace_bytes, stream);
+    return fwd_entry(q, k, v, o, nullptr, state_out, B, H, N, d, d, causal, false, dt, nullptr, nullptr, nullptr, sp,
+                     workspace, workspace_bytes, stream);
 }
 
 cott_status cott_fwd_strided(const void* q, const void* k, const void* v, void* o, float* state_out,
@@ -698,33 +802,16 @@ cott_status cott_fwd_strided(const void* q, const void* k, const void* v, void* 
                              const cott_strides* qkv_strides, const cott_strides* o_strides,
                              const cott_scale_params* sp, void* workspace, size_t workspace_bytes,
                              void* stream) {
-    if (!q || !k || !v || !o || B < 1 || H < 1 || N < 1) return COTT_ERR_INVALID_ARG;
-    if (!layout_ok(qkv_strides, d, dt) || !layout_ok(o_strides, d, dt)) return COTT_ERR_UNSUPPORTED;
-    if (check_scale(sp) != COTT_OK) return COTT_ERR_INVALID_ARG;
-    if (d >= 1 && (tensors_overlap(o, o_strides, q, qkv_strides, B, H, N, d, dt) ||
-                   tensors_overlap(o, o_strides, k, qkv_strides, B, H, N, d, dt) ||
-                   tensors_overlap(o, o_strides, v, qkv_strides, B, H, N, d, dt)))
-        return COTT_ERR_INVALID_ARG;
-    if (!sp->seq_len && sp->seq_len_scalar > 0.f && sp->seq_len_scalar < 1.f)
-        return COTT_ERR_INVALID_ARG;
-    Plan p;
-    if (!make_plan(COTT_OP_FWD, dt, B, H, N, d, causal, &p)) return COTT_ERR_UNSUPPORTED;
-    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) ||
-        (state_out && !aligned16(state_out)))
-        return COTT_ERR_UNSUPPORTED;
-    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
-        workspace_bytes < workspace_bytes_impl(COTT_OP_FWD, p, B, H, d))
-        return COTT_ERR_WORKSPACE;
-    return fwd_impl(q, k, v, o, state_out, B, H, N, d, causal, dt, sp, workspace, p,
-                    static_cast<cudaStream_t>(stream), nullptr, qkv_strides, o_strides);
+    return fwd_entry(q, k, v, o, nullptr, state_out, B, H, N, d, d, causal, false, dt, qkv_strides, nullptr, o_strides,
+                     sp, workspace, workspace_bytes, stream);
 }
 
 cott_status cott_fwd_stateful(const void* q, const void* k, const void* v, void* o,
                               const float* state_in, float* state_out, int B, int H, int N, int d,
                               cott_dtype dt, const cott_scale_params* sp, void* workspace,
                               size_t workspace_bytes, void* stream) {
-    return cott_fwd_stateful_strided(q, k, v, o, state_in, state_out, B, H, N, d, dt, nullptr, nullptr, sp,
-                                     workspace, workspace_bytes, stream);
+    return fwd_entry(q, k, v, o, state_in, state_out, B, H, N, d, d, 1, true, dt, nullptr, nullptr, nullptr, sp,
+                     workspace, workspace_bytes, stream);
 }
 
 cott_status cott_fwd_stateful_strided(const void* q, const void* k, const void* v, void* o,
@@ -732,34 +819,71 @@ cott_status cott_fwd_stateful_strided(const void* q, const void* k, const void* 
                                       int d, cott_dtype dt, const cott_strides* qkv_strides,
                                       const cott_strides* o_strides, const cott_scale_params* sp,
                                       void* workspace, size_t workspace_bytes, void* stream) {
-    if (!q || !k || !v || !o || B < 1 || H < 1 || N < 1) return COTT_ERR_INVALID_ARG;
-    if (!layout_ok(qkv_strides, d, dt) || !layout_ok(o_strides, d, dt)) return COTT_ERR_UNSUPPORTED;
-    if (check_scale(sp) != COTT_OK) return COTT_ERR_INVALID_ARG;
-    if (d >= 1 && (tensors_overlap(o, o_strides, q, qkv_strides, B, H, N, d, dt) ||
-                   tensors_overlap(o, o_strides, k, qkv_strides, B, H, N, d, dt) ||
-                   tensors_overlap(o, o_strides, v, qkv_strides, B, H, N, d, dt)))
+    return fwd_entry(q, k, v, o, state_in, state_out, B, H, N, d, d, 1, true, dt, qkv_strides, nullptr, o_strides, sp,
+                     workspace, workspace_bytes, stream);
+}
+
+cott_status cott_fwd_dkdv(const void* q, const void* k, const void* v, void* o, const float* state_in,
+                          float* state_out, int B, int H, int N, int d_k, int d_v, int causal, cott_dtype dt,
+                          const cott_strides* qk_strides, const cott_strides* v_strides,
+                          const cott_strides* o_strides, const cott_scale_params* sp, void* workspace,
+                          size_t workspace_bytes, void* stream) {
+    return fwd_entry(q, k, v, o, state_in, state_out, B, H, N, d_k, d_v, causal, state_in != nullptr, dt, qk_strides,
+                     v_strides, o_strides, sp, workspace, workspace_bytes, stream);
+}
+
+// Validation and dispatch shared by every dense / strided backward entry point.
+static cott_status bwd_entry(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk,
+                             void* dv, float* dm, int B, int H, int N, int d_k, int d_v, int causal, cott_dtype dt,
+                             const cott_strides* qk_strides, const cott_strides* v_strides,
+                             const cott_strides* do_strides, const cott_strides* dqk_strides,
+                             const cott_strides* dv_strides, const cott_scale_params* sp, void* workspace,
+                             size_t workspace_bytes, void* stream) {
+    if (!q || !k || !v || !d_o || !dq || !dk || !dv || !dm || B < 1 || H < 1 || N < 1 || d_k < 1 || d_v < 1)
         return COTT_ERR_INVALID_ARG;
-    if (state_in && state_in == state_out) return COTT_ERR_INVALID_ARG;
-    // the scaling base must be the caller's (the same for every segment of a sequence)
-    if (!sp->seq_len && !(sp->seq_len_scalar >= 1.f)) return COTT_ERR_INVALID_ARG;
+    const bool same = d_k == d_v;
+    const cott_strides* vs = v_strides ? v_strides : (same ? qk_strides : nullptr);
+    const cott_strides* dvs = dv_strides ? dv_strides : (same ? dqk_strides : nullptr);
+    if (!layout_ok(qk_strides, d_k, dt) || !layout_ok(vs, d_v, dt) || !layout_ok(do_strides, d_v, dt) ||
+        !layout_ok(dqk_strides, d_k, dt) || !layout_ok(dvs, d_v, dt))
+        return COTT_ERR_UNSUPPORTED;
+    if (check_scale(sp) != COTT_OK) return COTT_ERR_INVALID_ARG;
+    {
+        const void* ins[4] = {q, k, v, d_o};
+        const cott_strides* in_st[4] = {qk_strides, qk_strides, vs, do_strides};
+        const int in_d[4] = {d_k, d_k, d_v, d_v};
+        void* outs[3] = {dq, dk, dv};
+        const cott_strides* out_st[3] = {dqk_strides, dqk_strides, dvs};
+        const int out_d[3] = {d_k, d_k, d_v};
+        for (int i = 0; i < 3; ++i) {
+            for (int j = 0; j < 4; ++j)
+                if (tensors_overlap(outs[i], out_st[i], ins[j], in_st[j], B, H, N, out_d[i], dt, in_d[j])) return COTT_ERR_INVALID_ARG;
+            for (int j = i + 1; j < 3; ++j)
+                if (tensors_overlap(outs[i], out_st[i], outs[j], out_st[j], B, H, N, out_d[i], dt, out_d[j])) return COTT_ERR_INVALID_ARG;
+        }
+    }
+    if (!sp->seq_len && sp->seq_len_scalar > 0.f && sp->seq_len_scalar < 1.f)
+        return COTT_ERR_INVALID_ARG;
     Plan p;
-    if (!make_plan(COTT_OP_FWD, dt, B, H, N, d, 1, &p)) return COTT_ERR_UNSUPPORTED;
-    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) ||
-        (state_in && !aligned16(state_in)) || (state_out && !aligned16(state_out)))
+    if (!make_plan(COTT_OP_BWD, dt, B, H, N, d_k, d_v, causal, &p)) return COTT_ERR_UNSUPPORTED;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(d_o) || !aligned16(dq) ||
+        !aligned16(dk) || !aligned16(dv))
         return COTT_ERR_UNSUPPORTED;
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
-        workspace_bytes < workspace_bytes_impl(COTT_OP_FWD, p, B, H, d))
+        workspace_bytes < workspace_bytes_impl(COTT_OP_BWD, p, B, H, p.d))
         return COTT_ERR_WORKSPACE;
-    return fwd_impl(q, k, v, o, state_out, B, H, N, d, 1, dt, sp, workspace, p,
-                    static_cast<cudaStream_t>(stream), state_in, qkv_strides, o_strides);
+    const bool own_v = !same || v_strides || dv_strides;
+    return bwd_impl(q, k, v, d_o, dq, dk, dv, dm, B, H, N, p.d, causal, dt, sp, workspace, p,
+                    static_cast<cudaStream_t>(stream), qk_strides, do_strides, dqk_strides, Packed(),
+                    own_v ? vs : nullptr, own_v ? dvs : nullptr);
 }
 
 cott_status cott_bwd(const void* q, const void* k, const void* v, const void* d_o, void* dq,
                      void* dk, void* dv, float* dm, int B, int H, int N, int d, int causal,
                      cott_dtype dt, const cott_scale_params* sp, void* workspace,
                      size_t workspace_bytes, void* stream) {
-    return cott_bwd_strided(q, k, v, d_o, dq, dk, dv, dm, B, H, N, d, causal, dt, nullptr, nullptr,
-                            nullptr, sp, workspace, workspace_bytes, stream);
+    return bwd_entry(q, k, v, d_o, dq, dk, dv, dm, B, H, N, d, d, causal, dt, nullptr, nullptr, nullptr, nullptr,
+                     nullptr, sp, workspace, workspace_bytes, stream);
 }
 
 cott_status cott_bwd_strided(const void* q, const void* k, const void* v, const void* d_o, void* dq,
@@ -768,34 +892,18 @@ cott_status cott_bwd_strided(const void* q, const void* k, const void* v, const 
                              const cott_strides* do_strides, const cott_strides* dqkv_strides,
                              const cott_scale_params* sp, void* workspace, size_t workspace_bytes,
                              void* stream) {
-    if (!q || !k || !v || !d_o || !dq || !dk || !dv || !dm || B < 1 || H < 1 || N < 1)
-        return COTT_ERR_INVALID_ARG;
-    if (!layout_ok(qkv_strides, d, dt) || !layout_ok(do_strides, d, dt) || !layout_ok(dqkv_strides, d, dt))
-        return COTT_ERR_UNSUPPORTED;
-    if (check_scale(sp) != COTT_OK) return COTT_ERR_INVALID_ARG;
-    {
-        const void* ins[4] = {q, k, v, d_o};
-        const cott_strides* in_st[4] = {qkv_strides, qkv_strides, qkv_strides, do_strides};
-        void* outs[3] = {dq, dk, dv};
-        for (int i = 0; i < 3 && d >= 1; ++i) {
-            for (int j = 0; j < 4; ++j)
-                if (tensors_overlap(outs[i], dqkv_strides, ins[j], in_st[j], B, H, N, d, dt)) return COTT_ERR_INVALID_ARG;
-            for (int j = i + 1; j < 3; ++j)
-                if (tensors_overlap(outs[i], dqkv_strides, outs[j], dqkv_strides, B, H, N, d, dt)) return COTT_ERR_INVALID_ARG;
-        }
-    }
-    if (!sp->seq_len && sp->seq_len_scalar > 0.f && sp->seq_len_scalar < 1.f)
-        return COTT_ERR_INVALID_ARG;
-    Plan p;
-    if (!make_plan(COTT_OP_BWD, dt, B, H, N, d, causal, &p)) return COTT_ERR_UNSUPPORTED;
-    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(d_o) || !aligned16(dq) ||
-        !aligned16(dk) || !aligned16(dv))
-        return COTT_ERR_UNSUPPORTED;
-    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
-        workspace_bytes < workspace_bytes_impl(COTT_OP_BWD, p, B, H, d))
-        return COTT_ERR_WORKSPACE;
-    return bwd_impl(q, k, v, d_o, dq, dk, dv, dm, B, H, N, d, causal, dt, sp, workspace, p,
-                    static_cast<cudaStream_t>(stream), qkv_strides, do_strides, dqkv_strides);
+    return bwd_entry(q, k, v, d_o, dq, dk, dv, dm, B, H, N, d, d, causal, dt, qkv_strides, nullptr, do_strides,
+                     dqkv_strides, nullptr, sp, workspace, workspace_bytes, stream);
+}
+
+cott_status cott_bwd_dkdv(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk,
+                          void* dv, float* dm, int B, int H, int N, int d_k, int d_v, int causal, cott_dtype dt,
+                          const cott_strides* qk_strides, const cott_strides* v_strides,
+                          const cott_strides* do_strides, const cott_strides* dqk_strides,
+                          const cott_strides* dv_strides, const cott_scale_params* sp, void* workspace,
+                          size_t workspace_bytes, void* stream) {
+    return bwd_entry(q, k, v, d_o, dq, dk, dv, dm, B, H, N, d_k, d_v, causal, dt, qk_strides, v_strides, do_strides,
+                     dqk_strides, dv_strides, sp, workspace, workspace_bytes, stream);
 }
 
 // Plan of a packed batch: one group per (sequence, head), tensor-core path only.
@@ -803,6 +911,7 @@ static bool varlen_plan(cott_dtype dt, int B, int H, int total_tokens, int max_s
     if (B < 1 || H < 1 || total_tokens < 1 || max_seqlen < 1 || max_seqlen > total_tokens) return false;
     if (dt != COTT_BF16 || (d != 64 && d != 128)) return false;
     p->path = 1; p->chunk = 128; p->group = (max_seqlen + 127) / 128 * 128; p->n_groups = 1; p->split = 1;
+    p->d = p->dk = p->dv = d; p->padded = false;
     return true;
 }
 
@@ -857,19 +966,32 @@ cott_status cott_bwd_varlen(const void* q, const void* k, const void* v, const v
                     static_cast<cudaStream_t>(stream), &packed_l, &packed_l, &packed_l, pk);
 }
 
+cott_status cott_decode_step_dkdv(const void* q, const void* k, const void* v, float* state, void* o,
+                                  int B, int H, int d_k, int d_v, cott_dtype dt, const cott_scale_params* sp,
+                                  void* stream) {
+    if (!q || !k || !v || !state || !o || B < 1 || H < 1 || d_k < 1 || d_v < 1) return COTT_ERR_INVALID_ARG;
+    if (check_scale(sp) != COTT_OK) return COTT_ERR_INVALID_ARG;
+    if (!sp->seq_len && !(sp->seq_len_scalar >= 1.f)) return COTT_ERR_INVALID_ARG;
+    if (dt != COTT_F32 && dt != COTT_BF16) return COTT_ERR_UNSUPPORTED;
+    const bool tuned = d_k == d_v && (d_k == 32 || d_k == 64 || d_k == 128);
+    // other sizes: rows of 16 bytes at least (as in the forward), at most 1024 columns
+    const int q16 = 16 / (int)dtype_size(dt);
+    if (!tuned && (d_k % q16 != 0 || d_v % q16 != 0 || d_k > 1024 || d_v > 1024)) return COTT_ERR_UNSUPPORTED;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(state) || !aligned16(o))
+        return COTT_ERR_UNSUPPORTED;
+    if (tuned)
+        COTT_CUDA(launch_decode(q, k, v, state, o, B, H, d_k, dt, sp->m, sp->seq_len,
+                                sp->seq_len_scalar, static_cast<cudaStream_t>(stream)));
+    else
+        COTT_CUDA(launch_decode_generic(q, k, v, state, o, B, H, d_k, d_v, dt, sp->m, sp->seq_len,
+                                        sp->seq_len_scalar, static_cast<cudaStream_t>(stream)));
+    return COTT_OK;
+}
+
 cott_status cott_decode_step(const void* q, const void* k, const void* v, float* state, void* o,
                              int B, int H, int d, cott_dtype dt, const cott_scale_params* sp,
                              void* stream) {
-    if (!q || !k || !v || !state || !o || B < 1 || H < 1) return COTT_ERR_INVALID_ARG;
-    if (check_scale(sp) != COTT_OK) return COTT_ERR_INVALID_ARG;
-    if (!sp->seq_len && !(sp->seq_len_scalar >= 1.f)) return COTT_ERR_INVALID_ARG;
-    if (d != 32 && d != 64 && d != 128) return COTT_ERR_UNSUPPORTED;
-    if (dt != COTT_F32 && dt != COTT_BF16) return COTT_ERR_UNSUPPORTED;
-    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(state) || !aligned16(o))
-        return COTT_ERR_UNSUPPORTED;
-    COTT_CUDA(launch_decode(q, k, v, state, o, B, H, d, dt, sp->m, sp->seq_len,
-                            sp->seq_len_scalar, static_cast<cudaStream_t>(stream)));
-    return COTT_OK;
+    return cott_decode_step_dkdv(q, k, v, state, o, B, H, d, d, dt, sp, stream);
 }
 
 // The host-buffer training step cuts the batch into at most kHostSlices slices that are

@@ -105,6 +105,11 @@ struct TcWalkArgs {
     // by c on the way in), and the state after the last token goes to state_final, times c.
     int init_has_scale;
     float* state_final;
+    // Columns the tensors really have, when fewer than the kernel's d: x and a have d_xa, bv,
+    // the raw rows and out have d_bo (0: d).  The tensor maps get the real extents -- tiles are
+    // zero-filled beyond them on the way in and clipped on the way out -- and everything else
+    // (states, workspace) keeps the kernel's d.  Zero columns change no norm, score or product.
+    int d_xa; int d_bo;
 };
 cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cudaStream_t st);
 
@@ -116,11 +121,13 @@ struct TcBwdFusedArgs {
     const void* q; const void* k; const void* v; const void* d_o;
     void* dq; void* dk; void* dv;
     RowLayout l_qkv, l_do, l_dqkv;
+    RowLayout l_v, l_dv;      // v and dv (their own when the value size differs from the key size)
     const float* sq_part; const float* r_part;
     float* dm_partial; float* dm_out; int* status;
     const float* m; const float* seq_len; float seq_len_scalar;
     int group; int n_groups;
     int plain_launch;
+    int w_k, w_v;   // real columns of q, k, dq, dk and of v, dO, dv when fewer than 64 (0: 64)
 };
 cudaError_t launch_tc_bwd_fused(const TcBwdFusedArgs& a, int B, int H, int N, cudaStream_t st);
 // Both partial states of every group in one launch (uses q, k, v, d_o, the layouts, group,
@@ -131,8 +138,8 @@ cudaError_t launch_tc_bwd_states(const TcBwdFusedArgs& a, float* sq_out, float* 
 // Bidirectional forward at d = 64 in one launch, one CTA per (b, h) (cott_tc_bidir.cu); it is
 // the first (and only) kernel of its call and clears the status words itself.
 cudaError_t launch_tc_bidir_fwd(const void* q, const void* k, const void* v, void* o, const RowLayout& l_qkv,
-                                const RowLayout& l_o, float* state_out, int* status, const float* m, const float* seq_len,
-                                float seq_len_scalar, int B, int H, int N, cudaStream_t st);
+                                const RowLayout& l_v, const RowLayout& l_o, float* state_out, int* status, const float* m, const float* seq_len,
+                                float seq_len_scalar, int B, int H, int N, cudaStream_t st, int dk = 0, int dv = 0);
 
 // Tensor map over a bf16 tensor of logical shape [B,H,N,d] with the given row layout: box of
 // 128 tokens x 64 columns of one (b,h), 128-byte swizzle (see cott_tc_walk.cu).
@@ -154,6 +161,13 @@ cudaError_t launch_dm_finalize(const float* dm_partial, float* dm, const float* 
                                const float* seq_len, float seq_len_scalar, int B, int H,
                                int n_groups, int N, cudaStream_t st);
 cudaError_t launch_sum_slices(const float* parts, float* out, int n, int H, cudaStream_t st);
+// Caller-visible states [BH, dk, dv] <-> the kernels' padded [BH, d, d] (zero outside).
+cudaError_t launch_pad_state(const float* src, float* dst, int BH, int dk, int dv, int d, cudaStream_t st);
+cudaError_t launch_unpad_state(const float* src, float* dst, int BH, int dk, int dv, int d, cudaStream_t st);
+// Decode step for head sizes the specialised kernel does not cover (any dk, dv multiples of 4 / 8).
+cudaError_t launch_decode_generic(const void* q, const void* k, const void* v, float* state, void* o,
+                                  int B, int H, int dk, int dv, cott_dtype dt, const float* m,
+                                  const float* seq_len, float seq_len_scalar, cudaStream_t st);
 cudaError_t launch_decode(const void* q, const void* k, const void* v, float* state, void* o,
                           int B, int H, int d, cott_dtype dt, const float* m,
                           const float* seq_len, float seq_len_scalar, cudaStream_t st);

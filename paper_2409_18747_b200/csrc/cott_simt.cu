@@ -449,6 +449,107 @@ cudaError_t launch_dm_finalize(const float* dm_partial, float* dm, const float* 
     return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------------------------
+// Head sizes the tensor-core kernels run zero-padded (dk, dv <= their d): a caller's state
+// [BH, dk, dv] enters and leaves through a padded [BH, d, d] copy in the workspace.
+__global__ void pad_state_kernel(const float* __restrict__ src, float* __restrict__ dst, int dk, int dv, int d) {
+    const size_t bh = blockIdx.y;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < d * d; i += gridDim.x * blockDim.x) {
+        const int r = i / d, c = i - r * d;
+        dst[bh * d * d + i] = (r < dk && c < dv) ? src[bh * dk * dv + (size_t)r * dv + c] : 0.f;
+    }
+}
+__global__ void unpad_state_kernel(const float* __restrict__ src, float* __restrict__ dst, int dk, int dv, int d) {
+    const size_t bh = blockIdx.y;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < dk * dv; i += gridDim.x * blockDim.x) {
+        const int r = i / dv, c = i - r * dv;
+        dst[bh * dk * dv + i] = src[bh * d * d + (size_t)r * d + c];
+    }
+}
+cudaError_t launch_pad_state(const float* src, float* dst, int BH, int dk, int dv, int d, cudaStream_t st) {
+    dim3 grid((unsigned)((d * d + 1023) / 1024), (unsigned)BH);
+    pad_state_kernel<<<grid, 256, 0, st>>>(src, dst, dk, dv, d);
+    note_launch();
+    return cudaGetLastError();
+}
+cudaError_t launch_unpad_state(const float* src, float* dst, int BH, int dk, int dv, int d, cudaStream_t st) {
+    dim3 grid((unsigned)((dk * dv + 1023) / 1024), (unsigned)BH);
+    unpad_state_kernel<<<grid, 256, 0, st>>>(src, dst, dk, dv, d);
+    note_launch();
+    return cudaGetLastError();
+}
+
+// One step of Eq. 8 for any head sizes (dk keys, dv values, dv a multiple of 4): one CTA per
+// (b, h); thread t owns the four state columns 4 (t % (dv/4)) .. +3 of the rows
+// t / (dv/4), + 256 / (dv/4), ...: 128-bit state loads and stores, coalesced along a row; the
+// per-column partial sums of o meet in shared memory.
+//   S <- S + k^ (c v)^T ;  o = S^T q^      (update first, then observe)
+template <typename T>
+__global__ void __launch_bounds__(256) decode_generic_kernel(const T* __restrict__ q, const T* __restrict__ k,
+                                                             const T* __restrict__ v, float* __restrict__ state,
+                                                             T* __restrict__ o, int H, int dk, int dv,
+                                                             const float* __restrict__ m, const float* __restrict__ seq_len,
+                                                             float seq_len_scalar) {
+    extern __shared__ float sm[];            // q^ [dk] | k^ [dk] | c v [dv] | partial o [slices][dv] | 2 norms
+    float* qh = sm; float* kh = sm + dk; float* cv = kh + dk; float* part = cv + dv;
+    const size_t bh = blockIdx.x;
+    const int b = (int)(bh / H), h = (int)(bh % H), tid = threadIdx.x;
+    const int cgs = dv / 4, slices = 256 / cgs;          // column groups, row slices (>= 1 since dv <= 1024)
+    __shared__ float red[2][8];
+    float sq = 0.f, sk = 0.f;
+    for (int i = tid; i < dk; i += 256) {
+        const float a = to_f32(q[bh * dk + i]), c2 = to_f32(k[bh * dk + i]);
+        qh[i] = a; kh[i] = c2; sq = fmaf(a, a, sq); sk = fmaf(c2, c2, sk);
+    }
+    for (int off = 16; off; off >>= 1) { sq += __shfl_xor_sync(0xffffffffu, sq, off); sk += __shfl_xor_sync(0xffffffffu, sk, off); }
+    if ((tid & 31) == 0) { red[0][tid >> 5] = sq; red[1][tid >> 5] = sk; }
+    const float s_b = seq_len ? seq_len[b] : seq_len_scalar;
+    const float cfac = stab_factor(m[h], s_b);
+    for (int i = tid; i < dv; i += 256) cv[i] = cfac * to_f32(v[bh * dv + i]);
+    __syncthreads();
+    float nq = 0.f, nk = 0.f;
+    for (int w = 0; w < 8; ++w) { nq += red[0][w]; nk += red[1][w]; }
+    const float rq = 1.0f / fmaxf(sqrtf(nq), kEps), rk = 1.0f / fmaxf(sqrtf(nk), kEps);
+    const int cg = tid % cgs, sl = tid / cgs;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (sl < slices) {
+        const float4 vv = *reinterpret_cast<const float4*>(cv + 4 * cg);
+        float4* S = reinterpret_cast<float4*>(state + bh * (size_t)dk * dv) + cg;
+        for (int r = sl; r < dk; r += slices) {
+            float4 x = S[(size_t)r * cgs];
+            const float kr = kh[r] * rk, qr = qh[r] * rq;
+            x.x = fmaf(kr, vv.x, x.x); x.y = fmaf(kr, vv.y, x.y); x.z = fmaf(kr, vv.z, x.z); x.w = fmaf(kr, vv.w, x.w);
+            S[(size_t)r * cgs] = x;
+            acc.x = fmaf(qr, x.x, acc.x); acc.y = fmaf(qr, x.y, acc.y); acc.z = fmaf(qr, x.z, acc.z); acc.w = fmaf(qr, x.w, acc.w);
+        }
+        *reinterpret_cast<float4*>(part + (size_t)sl * dv + 4 * cg) = acc;
+    }
+    __syncthreads();
+    for (int i = tid; i < dv; i += 256) {
+        float a = 0.f;
+        for (int s2 = 0; s2 < slices; ++s2) a += part[(size_t)s2 * dv + i];
+        o[bh * dv + i] = from_f32<T>(a);
+    }
+}
+
+cudaError_t launch_decode_generic(const void* q, const void* k, const void* v, float* state, void* o,
+                                  int B, int H, int dk, int dv, cott_dtype dt, const float* m,
+                                  const float* seq_len, float seq_len_scalar, cudaStream_t st) {
+    if (dk < 1 || dv < 4 || (dv & 3) || dv > 1024 || dk > 1024) return cudaErrorInvalidValue;
+    const int cgs = dv / 4, slices = 256 / cgs;
+    const size_t smem = sizeof(float) * ((size_t)2 * dk + dv + (size_t)slices * dv);
+    const unsigned BH = (unsigned)(B * H);
+    if (dt == COTT_F32)
+        decode_generic_kernel<float><<<BH, 256, smem, st>>>((const float*)q, (const float*)k, (const float*)v, state,
+                                                            (float*)o, H, dk, dv, m, seq_len, seq_len_scalar);
+    else
+        decode_generic_kernel<__nv_bfloat16><<<BH, 256, smem, st>>>((const __nv_bfloat16*)q, (const __nv_bfloat16*)k,
+                                                                    (const __nv_bfloat16*)v, state, (__nv_bfloat16*)o, H,
+                                                                    dk, dv, m, seq_len, seq_len_scalar);
+    note_launch();
+    return cudaGetLastError();
+}
+
 cudaError_t launch_decode(const void* q, const void* k, const void* v, float* state, void* o,
                           int B, int H, int d, cott_dtype dt, const float* m,
                           const float* seq_len, float seq_len_scalar, cudaStream_t st) {

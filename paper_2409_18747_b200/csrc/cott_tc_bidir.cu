@@ -304,16 +304,18 @@ tc_bidir_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 }  // namespace
 
 cudaError_t launch_tc_bidir_fwd(const void* q, const void* k, const void* v, void* o, const RowLayout& l_qkv,
-                                const RowLayout& l_o, float* state_out, int* status, const float* m, const float* seq_len,
-                                float seq_len_scalar, int B, int H, int N, cudaStream_t st) {
+                                const RowLayout& l_v, const RowLayout& l_o, float* state_out, int* status, const float* m, const float* seq_len,
+                                float seq_len_scalar, int B, int H, int N, cudaStream_t st, int dk, int dv) {
     const void* ptrs[4] = {q, k, v, o};
-    const RowLayout lays[4] = {l_qkv, l_qkv, l_qkv, l_o};
+    const RowLayout lays[4] = {l_qkv, l_qkv, l_v, l_o};
+    // real column counts (<= 64): tiles are zero-filled beyond them and stores clipped
+    const int dims[4] = {dk > 0 ? dk : kD, dk > 0 ? dk : kD, dv > 0 ? dv : kD, dv > 0 ? dv : kD};
     CUtensorMap tm[4];
     BidirParams p;
     p.head_first_mask = 0;
     for (int i = 0; i < 4; ++i) {
         bool hf = false;
-        if (!make_tile_map(&tm[i], ptrs[i], B, H, N, kD, lays[i], &hf)) return cudaErrorInvalidValue;
+        if (dims[i] > kD || !make_tile_map(&tm[i], ptrs[i], B, H, N, dims[i], lays[i], &hf)) return cudaErrorInvalidValue;
         p.head_first_mask |= (hf ? 1 : 0) << i;
     }
     p.state_out = state_out; p.status = status; p.m = m; p.seq_len = seq_len; p.seq_len_scalar = seq_len_scalar;

@@ -984,13 +984,17 @@ tc_bwd_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 
 cudaError_t launch_tc_bwd_fused(const TcBwdFusedArgs& a, int B, int H, int N, cudaStream_t st) {
     const void* ptrs[7] = {a.q, a.k, a.v, a.d_o, a.dq, a.dk, a.dv};
-    const RowLayout lays[7] = {a.l_qkv, a.l_qkv, a.l_qkv, a.l_do, a.l_dqkv, a.l_dqkv, a.l_dqkv};
+    const RowLayout lays[7] = {a.l_qkv, a.l_qkv, a.l_v, a.l_do, a.l_dqkv, a.l_dqkv, a.l_dv};
+    // real column counts (<= 64): tiles are zero-filled beyond them and stores clipped
+    const int wk = a.w_k > 0 ? a.w_k : kD, wv = a.w_v > 0 ? a.w_v : kD;
+    const int dims[7] = {wk, wk, wv, wv, wk, wk, wv};
+    if (wk > kD || wv > kD) return cudaErrorInvalidValue;
     CUtensorMap tm[7];
     BwdParams p;
     p.head_first_mask = 0;
     for (int i = 0; i < 7; ++i) {
         bool hf = false;
-        if (!make_tile_map(&tm[i], ptrs[i], B, H, N, kD, lays[i], &hf)) return cudaErrorInvalidValue;
+        if (!make_tile_map(&tm[i], ptrs[i], B, H, N, dims[i], lays[i], &hf)) return cudaErrorInvalidValue;
         p.head_first_mask |= (hf ? 1 : 0) << i;
     }
     p.sq_part = a.sq_part; p.r_part = a.r_part; p.dm_partial = a.dm_partial; p.dm_out = a.dm_out;
@@ -1019,13 +1023,16 @@ cudaError_t launch_tc_bwd_fused(const TcBwdFusedArgs& a, int B, int H, int N, cu
 cudaError_t launch_tc_bwd_states(const TcBwdFusedArgs& a, float* sq_out, float* r_out, int clear_status, int B, int H,
                                  int N, cudaStream_t st) {
     const void* ptrs[4] = {a.q, a.k, a.v, a.d_o};
-    const RowLayout lays[4] = {a.l_qkv, a.l_qkv, a.l_qkv, a.l_do};
+    const RowLayout lays[4] = {a.l_qkv, a.l_qkv, a.l_v, a.l_do};
+    const int wk = a.w_k > 0 ? a.w_k : kD, wv = a.w_v > 0 ? a.w_v : kD;
+    const int dims[4] = {wk, wk, wv, wv};
+    if (wk > kD || wv > kD) return cudaErrorInvalidValue;
     CUtensorMap tm[4];
     StateParams p;
     p.head_first_mask = 0;
     for (int i = 0; i < 4; ++i) {
         bool hf = false;
-        if (!make_tile_map(&tm[i], ptrs[i], B, H, N, kD, lays[i], &hf)) return cudaErrorInvalidValue;
+        if (!make_tile_map(&tm[i], ptrs[i], B, H, N, dims[i], lays[i], &hf)) return cudaErrorInvalidValue;
         p.head_first_mask |= (hf ? 1 : 0) << i;
     }
     p.sq_out = sq_out; p.r_out = r_out; p.status = a.status;

@@ -60,6 +60,7 @@ struct TcWalkParams {
     void* out_rows; long long out_sn, out_sh;   // Out as plain global memory (rows of a ragged last chunk)
     int head_first_mask;                // bit i: in tensor map i (X, A, Bv, raw rows, Out) the head index
                                         // comes before the token index (its stride is the smaller one)
+    int d_out;                          // columns Out really has (<= d): boxes wholly beyond are not stored
 };
 
 enum { MODE_STATE = 0, MODE_CAUSAL = 1, MODE_READOUT = 2 };
@@ -735,6 +736,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
 #pragma unroll
                 // (the rows of a ragged last chunk of a packed batch were written by the workers)
                 for (int hh = 0; hh < ((ragged_last && c == last_visit_of_ragged) ? 0 : NH); ++hh) {
+                    if (hh * 64 >= p.d_out) break;
                     const bool hfo = (p.head_first_mask >> 4) & 1;
                     const int row = chunk_row(c);
                     tma_store_4d(&tmO, src + hh * 16384, hh * 64, hfo ? h : row, hfo ? row : h, bcoord);
@@ -1319,14 +1321,19 @@ cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cuda
     int head_first_mask = 0;
     // A packed batch is one tensor of total_tokens rows per head (batch extent 1).
     const int map_B = a.cu_seqlens ? 1 : B, map_N = a.cu_seqlens ? a.total_tokens : N;
+    const int d_xa = a.d_xa > 0 ? a.d_xa : d, d_bo = a.d_bo > 0 ? a.d_bo : d;
+    if (d_xa > d || d_bo > d || (a.cu_seqlens && (d_xa != d || d_bo != d))) return cudaErrorInvalidValue;
+    // (an unused operand's map points at x or a)
+    const int dims[5] = {d_xa, d_xa, a.bv ? d_bo : d_xa, a.proj ? d_bo : d_xa, a.out ? d_bo : d_xa};
     for (int i = 0; i < 5; ++i) {
         bool hf = false;
-        if (!make_tile_map(&tm[i], ptrs[i], map_B, H, map_N, d, lays[i], &hf)) return cudaErrorInvalidValue;
+        if (!make_tile_map(&tm[i], ptrs[i], map_B, H, map_N, dims[i], lays[i], &hf)) return cudaErrorInvalidValue;
         head_first_mask |= (hf ? 1 : 0) << i;
     }
     TcWalkParams p;
     p.head_first_mask = head_first_mask;
     p.cu_seqlens = a.cu_seqlens;
+    p.d_out = d_bo;
     {
         const RowLayout lo = resolve_layout(a.lout, H, map_N, d);
         p.out_rows = a.out; p.out_sn = lo.sn; p.out_sh = lo.sh;

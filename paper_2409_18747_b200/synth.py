@@ -38,12 +38,14 @@ def normal(shape, dtype, gen: torch.Generator) -> torch.Tensor:
     return torch.randn(shape, generator=gen, dtype=torch.float32).to(dtype)
 
 
-def make_qkv(B, H, N, d, dtype, seed, row_lognormal=False, zero_k_frac=0.0, with_do=False):
-    """Returns a dict with q,k,v (and d_o) ``[B,H,N,d]`` in ``dtype`` and m ``[H]`` fp32."""
+def make_qkv(B, H, N, d, dtype, seed, row_lognormal=False, zero_k_frac=0.0, with_do=False, d_v=None):
+    """Returns a dict with q,k,v (and d_o) ``[B,H,N,d]`` in ``dtype`` and m ``[H]`` fp32.
+    ``d_v``: value size when it differs from the key size d (v and d_o are ``[B,H,N,d_v]``)."""
     g = _gen(seed)
+    d_v = d if d_v is None else d_v
     q = torch.randn((B, H, N, d), generator=g, dtype=torch.float32)
     k = torch.randn((B, H, N, d), generator=g, dtype=torch.float32)
-    v = torch.randn((B, H, N, d), generator=g, dtype=torch.float32)
+    v = torch.randn((B, H, N, d_v), generator=g, dtype=torch.float32)
     m = torch.randn((H,), generator=g, dtype=torch.float32)
     if row_lognormal:  # exercises the normalisation: rows of wildly different length
         q = q * torch.exp(torch.randn((B, H, N, 1), generator=g, dtype=torch.float32))
@@ -56,7 +58,7 @@ def make_qkv(B, H, N, d, dtype, seed, row_lognormal=False, zero_k_frac=0.0, with
                 k[b, h, idx, :] = 0.0
     out = {"q": q.to(dtype), "k": k.to(dtype), "v": v.to(dtype), "m": m}
     if with_do:
-        out["d_o"] = torch.randn((B, H, N, d), generator=g, dtype=torch.float32).to(dtype)
+        out["d_o"] = torch.randn((B, H, N, d_v), generator=g, dtype=torch.float32).to(dtype)
     return out
 
 

@@ -42,7 +42,23 @@ def test_workspace_and_plan_are_host_only():
             assert 256 <= wf <= wb < (8 << 30)
     assert cott.workspace_bytes(cott.OP_DECODE, cott.BF16, 64, 16, 1, 128, True) == 0
     lib = cott._load()
-    assert lib.cott_workspace_bytes(0, cott.BF16, 1, 1, 16, 48, 1) == ctypes.c_size_t(-1).value  # d unsupported
+    assert lib.cott_workspace_bytes(0, cott.BF16, 1, 1, 16, 44, 1) == ctypes.c_size_t(-1).value  # rows not of 16 bytes
+    assert lib.cott_workspace_bytes(0, cott.BF16, 1, 1, 16, 136, 1) == ctypes.c_size_t(-1).value  # d beyond 128
+    assert lib.cott_workspace_bytes(0, cott.F32, 1, 1, 16, 48, 1) == ctypes.c_size_t(-1).value  # fp32: 32, 64, 128 only
+    # bf16 head sizes that are multiples of 8 run zero-padded in the next kernel size: the same
+    # group states plus room for a caller's state in that size, in and out
+    lib.cott_workspace_bytes_dkdv.restype = ctypes.c_size_t
+    w64 = lib.cott_workspace_bytes(0, cott.BF16, 1, 1, 16, 64, 1)
+    assert lib.cott_workspace_bytes(0, cott.BF16, 1, 1, 16, 48, 1) == w64 + 2 * 64 * 64 * 4
+    assert lib.cott_workspace_bytes_dkdv(0, cott.BF16, 1, 1, 16, 64, 64, 1) == w64
+    w128 = lib.cott_workspace_bytes(0, cott.BF16, 1, 1, 16, 128, 1)
+    assert lib.cott_workspace_bytes_dkdv(0, cott.BF16, 1, 1, 16, 64, 128, 1) == w128 + 2 * 128 * 128 * 4
+    assert lib.cott_workspace_bytes_dkdv(0, cott.F32, 1, 1, 16, 32, 64, 1) == ctypes.c_size_t(-1).value
+    kd = ctypes.c_int()
+    assert lib.cott_query_plan_dkdv(0, cott.BF16, 1, 1, 16, 32, 96, 1, None, None, None, ctypes.byref(kd)) == 0
+    assert kd.value == 128
+    assert lib.cott_query_plan_dkdv(0, cott.BF16, 1, 1, 16, 32, 40, 1, None, None, None, ctypes.byref(kd)) == 0
+    assert kd.value == 64
     assert lib.cott_workspace_bytes(0, cott.BF16, 0, 1, 16, 64, 1) == ctypes.c_size_t(-1).value
 
 
@@ -59,7 +75,7 @@ def test_argument_validation_returns_before_any_launch():
     # output aliases an input
     assert lib.cott_fwd(a, a, a, a, null, 1, 1, 16, 64, 1, cott.BF16, ctypes.byref(sp), a, 1 << 20, null) == -1
     # unsupported head dimension, misaligned pointer
-    assert lib.cott_fwd(a, a, a, a + 65536, null, 1, 1, 16, 48, 1, cott.BF16, ctypes.byref(sp), a, 1 << 20, null) == -2
+    assert lib.cott_fwd(a, a, a, a + 65536, null, 1, 1, 16, 44, 1, cott.BF16, ctypes.byref(sp), a, 1 << 20, null) == -2
     assert lib.cott_fwd(a + 2, a, a, a + 65536, null, 1, 1, 16, 64, 1, cott.BF16, ctypes.byref(sp), a, 1 << 20, null) == -2
     # workspace missing / too small
     assert lib.cott_fwd(a, a, a, a + 65536, null, 1, 1, 16, 64, 1, cott.BF16, ctypes.byref(sp), null, 0, null) == -3
@@ -146,6 +162,31 @@ def test_outputs_that_share_bytes_with_other_tensors_are_refused():
                                 base_in + row, base_out + row, base_out + 2 * row, a + (1 << 24), B, H, N, d, 1, cott.BF16,
                                 ctypes.byref(fused), None, ctypes.byref(fused), *tail)
     assert same == -1                                   # dq is the k slice
+
+
+def test_slices_of_different_widths_in_one_buffer():
+    """Key and value sizes of their own (48 and 80 columns): q, k, v as column slices of one
+    [B,N,H,176] buffer do not meet although their ranges interleave; a dv slice that starts
+    inside dk's columns does."""
+    lib = cott._load()
+    sp = cott._ScaleParams()
+    sp.m, sp.seq_len, sp.seq_len_scalar = 256, None, 0.0
+    a, g0, null = 1 << 20, 1 << 24, None
+    B, H, N, dk, dv = 1, 2, 16, 48, 80
+    W = 2 * dk + dv
+    S = cott._Strides
+    fused = S(N * H * W, W, H * W)
+    tail = (ctypes.byref(sp), null, 0, null)                       # valid calls stop at the workspace check (-3)
+    call = lambda dq, dk_, dv_: lib.cott_bwd_dkdv(a, a + 2 * dk, a + 4 * dk, 1 << 26, dq, dk_, dv_, 1 << 27, B, H, N,
+                                                  dk, dv, 1, cott.BF16, ctypes.byref(fused), ctypes.byref(fused), None,
+                                                  ctypes.byref(fused), ctypes.byref(fused), *tail)
+    assert call(g0, g0 + 2 * dk, g0 + 4 * dk) == -3                # dq | dk | dv side by side in each row
+    assert call(g0, g0 + 2 * dk, g0 + 4 * dk - 32) == -1           # dv starts 16 columns inside dk
+    assert call(g0, g0 + 2 * dk - 16, g0 + 4 * dk) == -1           # dk starts inside dq
+    assert call(a + 4 * dk + 2 * dv - 16, g0 + 2 * dk, g0 + 4 * dk) == -1   # dq starts inside v's last columns
+    f = lambda o: lib.cott_fwd_dkdv(a, a + 2 * dk, a + 4 * dk, o, null, null, B, H, N, dk, dv, 1, cott.BF16,
+                                    ctypes.byref(fused), ctypes.byref(fused), None, *tail)
+    assert f(g0) == -3 and f(a) == -1                              # dense o elsewhere / o at q's address
 
 
 def test_options_and_shutdown_are_host_only():
