@@ -146,6 +146,14 @@ cudaError_t launch_tc_bidir_fwd(const void* q, const void* k, const void* v, voi
 bool make_tile_map(CUtensorMap* map, const void* ptr, int B, int H, int N, int d, const RowLayout& lay,
                    bool* head_first);
 
+bool make_rows_map(CUtensorMap* map, const void* ptr, long long rows, int d, int box_rows);
+
+// Forward for sequences of at most 128 tokens in dense [B,H,N,d] tensors (cott_tc_short.cu): the
+// quadratic form, several sequences per 128-row tile, no state; the only kernel of its call.
+cudaError_t launch_tc_short_fwd(const void* q, const void* k, const void* v, void* o, int* status, const float* m,
+                                const float* seq_len, float seq_len_scalar, int B, int H, int N, int d, int dk, int dv,
+                                int causal, cudaStream_t st);
+
 // Opt-in to `bytes` of dynamic shared memory for a kernel, once per (kernel, device).
 cudaError_t configure_smem_once(const void* func, int bytes);
 
@@ -155,6 +163,7 @@ int option_force_path();
 int option_pair();
 int option_fused_bwd();
 int option_fused_bidir();
+int option_short_fwd();
 int wait_limit_kcycles();      // bound of every device-side wait, in units of 1024 SM cycles
 
 cudaError_t launch_dm_finalize(const float* dm_partial, float* dm, const float* m,

@@ -1247,6 +1247,21 @@ bool make_tile_map(CUtensorMap* map, const void* ptr, int B, int H, int N, int d
     return r == CUDA_SUCCESS;
 }
 
+// Tensor map over `rows` contiguous rows of d bf16 values (a dense [B,H,N,d] tensor seen as one
+// list of rows): box = box_rows rows x 64 columns, 128-byte swizzle, coordinates (column, row, 0, 0).
+bool make_rows_map(CUtensorMap* map, const void* ptr, long long rows, int d, int box_rows) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc || rows < 1 || d < 8 || (d & 7) || box_rows < 1 || box_rows > 256) return false;
+    cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)rows, 1, 1};
+    cuuint64_t strides[3] = {(cuuint64_t)d * 2, (cuuint64_t)rows * d * 2, (cuuint64_t)rows * d * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides,
+                     box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 namespace {
 
 template <int D, int MODE, int STREAM, bool VARLEN>

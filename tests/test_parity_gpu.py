@@ -710,6 +710,7 @@ def test_chunk_count_boundaries_bidirectional_d64(N, fused, option, force_group)
     an even number of chunks and a ragged last one) and through the two-launch form it replaces:
     rows and the exported state against the definition."""
     option("fused_bidir", fused)
+    option("short_fwd", 0)           # (N <= 128 without a state export would take the short-sequence kernel)
     force_group(4096)
     c = synth.make_qkv(3, 7, N, 64, torch.bfloat16, 5500 + N)
     q, k, v, m = (dev(c[x]) for x in ("q", "k", "v", "m"))
@@ -723,6 +724,39 @@ def test_chunk_count_boundaries_bidirectional_d64(N, fused, option, force_group)
     assert norm_max_err(st, ref_state) <= state_tol(torch.bfloat16, 64)
     o2 = cott.fwd(q, k, v, m, causal=False)
     assert torch.equal(o2, o)
+
+
+# ------------------------------------------------------------------ short sequences
+@pytest.mark.parametrize("N", [1, 2, 7, 16, 33, 64, 65, 100, 128])
+@pytest.mark.parametrize("dk,dv", [(64, 64), (128, 128), (32, 96)])
+@pytest.mark.parametrize("causal", [True, False])
+def test_short_sequences_take_the_quadratic_side(N, dk, dv, causal, option):
+    """Sequences of at most 128 tokens in dense tensors: one launch of the quadratic form with
+    floor(128 / N) sequences of consecutive (b, h) pairs per tile and a block-diagonal mask --
+    no state.  21 pairs, so the last tile is partly empty; every row against the definition,
+    and the same call through the generic walk for comparison."""
+    B, H = 3, 7
+    c = synth.make_qkv(B, H, N, dk, torch.bfloat16, 6600 + N + dk, d_v=dv)
+    q, k, v, m = (dev(c[x]) for x in ("q", "k", "v", "m"))
+    s = torch.tensor([float(N), 50.0, 300.0], device="cuda")
+    ref = oracle.fwd_quadratic(c["q"], c["k"], c["v"], c["m"], s.cpu().numpy().astype(np.float64), causal)
+    cott.cott.profile_enable(8)
+    o = cott.fwd(q, k, v, m, seq_len=s, causal=causal)
+    kinds = [kd for kd, _ in cott.cott.profile_read()]
+    cott.cott.profile_enable(0)
+    assert kinds == [5]
+    gate(o, ref, torch.bfloat16)
+    option("short_fwd", 0)
+    o_walk = cott.fwd(q, k, v, m, seq_len=s, causal=causal)
+    gate(o_walk, ref, torch.bfloat16)
+    # neighbours in a tile do not leak into each other: changing one pair's rows changes only its output
+    if N <= 64:
+        option("short_fwd", 1)
+        k2 = k.clone(); k2[1, 2] = -k2[1, 2]
+        o2 = cott.fwd(q, k2, v, m, seq_len=s, causal=causal)
+        same = torch.ones((B, H), dtype=torch.bool); same[1, 2] = False
+        assert torch.equal(o2[same.cuda()], o[same.cuda()])
+        assert not torch.equal(o2[1, 2], o[1, 2])
 
 
 # ------------------------------------------------------------------ head sizes (d_key, d_value)
