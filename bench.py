@@ -90,9 +90,9 @@ def roofline_record(w: dict, peaks: dict, kernels_ms: float, kernel: str, fwd_ms
                     bwd_ms: float | None, step_ms: float) -> dict:
     """The `roofline` object of the JSON line.  Bytes are the METHOD's (forward 8d and backward
     14d per token-head in bf16: every tensor of the step once, whatever this implementation
-    re-reads); `frac` = those bytes / the summed duration of the step's kernel launches / the
-    copy bandwidth; `calls` holds the same bytes over whole calls (launch gaps and the small
-    scan and finalise kernels included)."""
+    re-reads); `frac` = those bytes / `kernels_ms` (the time the step's kernel launches take on
+    the launching stream) / the copy bandwidth; `calls` holds the same bytes over each whole
+    call."""
     ab = algorithmic_bytes(w)
     alg = ab["fwd"] + ab["bwd"]
     d = w["d"]
@@ -551,8 +551,8 @@ def run_ours(args, w):
                 "rows": w["rows"], "padded_rows": B * N}
     # Roofline of the step: the METHOD's bytes (forward: q, k, v in, o out = 8d per token-head;
     # backward: q, k, v, dO in, dq, dk, dv out = 14d; decode: the fp32 state in and out) over the
-    # summed duration of the step's tensor-core kernel launches, each timed with CUDA events on
-    # the stream it was launched on.  Tensors this implementation reads twice count once.
+    # time the step's kernel launches take, measured with CUDA events on the stream they are
+    # launched on.  Tensors this implementation reads twice count once.
     alg = ab["fwd"] + ab["bwd"]
     # The kernels of a step overlap (a kernel's prologue runs under its predecessor's tail), so
     # their time is the span of the step on the launching stream in the timed region; the
