@@ -165,7 +165,7 @@ typedef struct cott_strides {
  * cott_fwd on tensors that are not dense [B,H,N,d] (no transpose pass before the attention):
  *   qkv_strides : strides shared by q, k and v (NULL: dense)
  *   o_strides   : strides of o (NULL: dense)
- * Everything else as for cott_fwd.  On the tensor-core path (bf16, d 64 or 128) the strides must
+ * Everything else as for cott_fwd.  On the tensor-core path (bf16) the strides must
  * also be expressible as a 4-D tiled tensor map (each stride a multiple of the next smaller
  * one, as in the three layouts above); COTT_ERR_UNSUPPORTED or COTT_ERR_CUDA otherwise.
  */
@@ -245,7 +245,7 @@ cott_status cott_bwd_strided(const void* q, const void* k, const void* v, const 
  * else its length.  No padding rows are read as keys or written as outputs.
  *   max_seqlen : an upper bound of the longest sequence (sizes the workspace and the plan)
  *   workspace  : cott_workspace_bytes(COTT_OP_FWD or COTT_OP_BWD, dt, B, H, max_seqlen, d, causal)
- * bf16 with d 64 or 128 only (COTT_ERR_UNSUPPORTED otherwise); one CTA walks one (sequence,
+ * bf16 with d a multiple of 8 up to 128 only (COTT_ERR_UNSUPPORTED otherwise); one CTA walks one (sequence,
  * head), so the GPU is filled when B*H reaches the number of SMs.  A NaN or Inf in the first
  * rows of one sequence can reach the last rows of the sequence stored before it (the tile
  * that holds both is multiplied by zeros, not skipped).  Other arguments, ordering and
@@ -287,7 +287,8 @@ cott_status cott_decode_step(const void* q, const void* k, const void* v, float*
  *         padded copy in the workspace (cott_workspace_bytes_dkdv accounts for it);
  *   fp32: d_k = d_v in {32, 64, 128};
  *   decode step: additionally any d_k, d_v up to 1024 that are multiples of 16 bytes.
- * Packed (varlen) batches and cott_fwd_noalloc keep d in {64, 128}; cott_fwd_bwd_host takes one d.
+ * Packed (varlen) batches take one d (bf16, any multiple of 8 up to 128); cott_fwd_noalloc and
+ * cott_fwd_bwd_host take one d as well.
  * Strides: q and k share `qk_strides`, v has `v_strides`, o / dO `o_strides` / `do_strides`,
  * dq and dk share `dqk_strides`, dv has `dv_strides` (NULL: dense for that tensor's own width;
  * with d_k == d_v a NULL v_strides / dv_strides means "as q and k" / "as dq and dk").

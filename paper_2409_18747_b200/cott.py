@@ -415,7 +415,7 @@ def _check_packed(cu_seqlens, *ts):
 @_on_call_stream
 def fwd_varlen(q, k, v, m, cu_seqlens, max_seqlen, seq_len=None, causal=True, out=None, workspace=None,
                stream=None):
-    """cott_fwd_varlen: q, k, v ``[total_tokens, H, d]`` (bf16, d 64 or 128), the sequences of the
+    """cott_fwd_varlen: q, k, v ``[total_tokens, H, d]`` (bf16, d a multiple of 8 up to 128), the sequences of the
     batch back to back; ``cu_seqlens`` int32 ``[B+1]`` CUDA tensor of row offsets.  Returns ``o``."""
     _check_packed(cu_seqlens, q, k, v)
     _check_dev(m, seq_len if isinstance(seq_len, torch.Tensor) else None)

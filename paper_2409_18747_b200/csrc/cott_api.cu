@@ -927,9 +927,10 @@ cott_status cott_bwd_dkdv(const void* q, const void* k, const void* v, const voi
 // Plan of a packed batch: one group per (sequence, head), tensor-core path only.
 static bool varlen_plan(cott_dtype dt, int B, int H, int total_tokens, int max_seqlen, int d, Plan* p) {
     if (B < 1 || H < 1 || total_tokens < 1 || max_seqlen < 1 || max_seqlen > total_tokens) return false;
-    if (dt != COTT_BF16 || (d != 64 && d != 128)) return false;
+    // bf16, tensor cores: any head size that is a multiple of 8 up to 128 (zero-filled tiles)
+    if (dt != COTT_BF16 || d < 8 || d > 128 || d % 8 != 0) return false;
     p->path = 1; p->chunk = 128; p->group = (max_seqlen + 127) / 128 * 128; p->n_groups = 1; p->split = 1;
-    p->d = p->dk = p->dv = d; p->padded = false;
+    p->dk = p->dv = d; p->d = d <= 64 ? 64 : 128; p->padded = p->d != d;
     return true;
 }
 
@@ -945,12 +946,12 @@ cott_status cott_fwd_varlen(const void* q, const void* k, const void* v, void* o
     if (!varlen_plan(dt, B, H, total_tokens, max_seqlen, d, &p)) return COTT_ERR_UNSUPPORTED;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return COTT_ERR_UNSUPPORTED;
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
-        workspace_bytes < workspace_bytes_impl(COTT_OP_FWD, p, B, H, d))
+        workspace_bytes < workspace_bytes_impl(COTT_OP_FWD, p, B, H, p.d))
         return COTT_ERR_WORKSPACE;
     // rows of all sequences back to back, [total_tokens, H, d]
     const cott_strides packed_l = {(long long)total_tokens * H * d, (long long)d, (long long)H * d};
     Packed pk; pk.cu_seqlens = cu_seqlens; pk.total_tokens = total_tokens;
-    return fwd_impl(q, k, v, o, nullptr, B, H, max_seqlen, d, causal, dt, sp, workspace, p,
+    return fwd_impl(q, k, v, o, nullptr, B, H, max_seqlen, p.d, causal, dt, sp, workspace, p,
                     static_cast<cudaStream_t>(stream), nullptr, &packed_l, &packed_l, pk);
 }
 
@@ -976,11 +977,11 @@ cott_status cott_bwd_varlen(const void* q, const void* k, const void* v, const v
         !aligned16(dk) || !aligned16(dv))
         return COTT_ERR_UNSUPPORTED;
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
-        workspace_bytes < workspace_bytes_impl(COTT_OP_BWD, p, B, H, d))
+        workspace_bytes < workspace_bytes_impl(COTT_OP_BWD, p, B, H, p.d))
         return COTT_ERR_WORKSPACE;
     const cott_strides packed_l = {(long long)total_tokens * H * d, (long long)d, (long long)H * d};
     Packed pk; pk.cu_seqlens = cu_seqlens; pk.total_tokens = total_tokens;
-    return bwd_impl(q, k, v, d_o, dq, dk, dv, dm, B, H, max_seqlen, d, causal, dt, sp, workspace, p,
+    return bwd_impl(q, k, v, d_o, dq, dk, dv, dm, B, H, max_seqlen, p.d, causal, dt, sp, workspace, p,
                     static_cast<cudaStream_t>(stream), &packed_l, &packed_l, &packed_l, pk);
 }
 

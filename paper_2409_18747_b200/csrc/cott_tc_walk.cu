@@ -1085,7 +1085,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                         // Packed batch, last chunk of the sequence: a tile store would overwrite
                         // rows of the next sequence; the rows that exist go out one by one.
                         const long long grow = (long long)chunk_row(c) + arow;
-                        if (grow < tok1)
+                        if (grow < tok1 && col < p.d_out)
                             *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out_rows) +
                                                       grow * p.out_sn + (long long)h * p.out_sh + col) = w;
                     } else {
@@ -1337,7 +1337,7 @@ cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cuda
     // A packed batch is one tensor of total_tokens rows per head (batch extent 1).
     const int map_B = a.cu_seqlens ? 1 : B, map_N = a.cu_seqlens ? a.total_tokens : N;
     const int d_xa = a.d_xa > 0 ? a.d_xa : d, d_bo = a.d_bo > 0 ? a.d_bo : d;
-    if (d_xa > d || d_bo > d || (a.cu_seqlens && (d_xa != d || d_bo != d))) return cudaErrorInvalidValue;
+    if (d_xa > d || d_bo > d) return cudaErrorInvalidValue;
     // (an unused operand's map points at x or a)
     const int dims[5] = {d_xa, d_xa, a.bv ? d_bo : d_xa, a.proj ? d_bo : d_xa, a.out ? d_bo : d_xa};
     for (int i = 0; i < 5; ++i) {
@@ -1350,7 +1350,7 @@ cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cuda
     p.cu_seqlens = a.cu_seqlens;
     p.d_out = d_bo;
     {
-        const RowLayout lo = resolve_layout(a.lout, H, map_N, d);
+        const RowLayout lo = resolve_layout(a.lout, H, map_N, d_bo);
         p.out_rows = a.out; p.out_sn = lo.sn; p.out_sh = lo.sh;
     }
     p.init = a.init; p.state_out = a.state_out; p.dm_partial = a.dm_partial; p.dm_extra = a.dm_extra; p.dm_out = a.dm_out; p.status = a.status;

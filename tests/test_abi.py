@@ -113,11 +113,11 @@ def test_strided_and_packed_entry_points_validate_on_the_host():
     bargs = (a, a, a, a, a + 65536, a + 131072, a + 196608, a, 1, 2, 16, 64, 1, cott.BF16)
     assert lib.cott_bwd_strided(*bargs, None, None, ctypes.byref(S(4096, 64, 130)), ctypes.byref(sp), a, 1 << 24, null) == -2
     assert lib.cott_bwd_strided(*bargs, ctypes.byref(ok), None, ctypes.byref(ok), ctypes.byref(sp), null, 0, null) == -3
-    # packed batches: NULL cu_seqlens, fp32 or d = 32 (tensor-core path only), max_seqlen > total
+    # packed batches: NULL cu_seqlens, fp32 or rows that are not multiples of 16 bytes (tensor-core path only), max_seqlen > total
     v = (a, a, a, a + 65536)
     assert lib.cott_fwd_varlen(*v, null, 2, 2, 100, 60, 64, 1, cott.BF16, *tail) == -1
     assert lib.cott_fwd_varlen(*v, a, 2, 2, 100, 60, 64, 1, cott.F32, *tail) == -2
-    assert lib.cott_fwd_varlen(*v, a, 2, 2, 100, 60, 32, 1, cott.BF16, *tail) == -2
+    assert lib.cott_fwd_varlen(*v, a, 2, 2, 100, 60, 36, 1, cott.BF16, *tail) == -2
     assert lib.cott_fwd_varlen(*v, a, 2, 2, 100, 200, 64, 1, cott.BF16, *tail) == -2
     assert lib.cott_fwd_varlen(*v, a, 2, 2, 100, 60, 64, 1, cott.BF16, ctypes.byref(sp), null, 0, null) == -3
     assert lib.cott_bwd_varlen(a, a, a, a, a + 65536, a + 131072, a + 196608, a, null, 2, 2, 100, 60, 64, 1,

@@ -985,7 +985,7 @@ def _pack(c, lens):
             for k2 in ("q", "k", "v", "d_o")}
 
 
-@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("d", [64, 128, 32, 96])
 @pytest.mark.parametrize("causal", [True, False])
 @pytest.mark.parametrize("lens", [(300, 1, 128, 129, 77), (1000, 513), (64,)])
 def test_packed_varlen_matches_per_sequence_definition(d, causal, lens):
