@@ -7,7 +7,9 @@
 // fp32 rows are multiplied by c / max(||q||, eps) (the stabilisation factor of Eq. 4 and the
 // query's row norm), rounded to bf16 and stored.  Every tensor is read or written exactly once,
 // and nothing but the optional state export goes through global memory in between.
-// Two CTAs share an SM (about 106 KB of shared memory and 256 tensor-memory columns each).
+// Three CTAs share an SM (74 KB of shared memory and 128 tensor-memory columns each), so that a
+// batch of a few hundred (b, h) pairs is resident all at once and one CTA's load latency hides
+// behind the others' work; the output rows are staged in the q tile they were computed from.
 #include "cott_internal.h"
 #include "cott_sm100.cuh"
 #include "cott_tc_common.cuh"
@@ -28,8 +30,7 @@ constexpr int kThreads = (kWorkerWarps + 2) * 32;   // + product thread, copy th
 struct L {
     static constexpr int kSlots = 4;                        // ring of tile slots: (k, v) pairs in phase 1, q tiles in phase 2
     static constexpr int kOffSb = kSlots * kTile;           // bf16 copy of the state (64 x 64)
-    static constexpr int kOffOut = kOffSb + kD * kD * 2;    // [2] output staging tiles
-    static constexpr int kOffCtl = kOffOut + 2 * kTile;
+    static constexpr int kOffCtl = kOffSb + kD * kD * 2;
     static constexpr int kCtlBytes = 1024;                  // mbarriers, tensor-memory slot, abort flag and wait limit
     static constexpr int kDynBytes = kOffCtl + kCtlBytes + 1024;
 };
@@ -44,24 +45,24 @@ struct BidirParams {
     int head_first_mask;     // bit i: in tensor map i (q, k, v, o) the head index comes before the token index
 };
 
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 3)
 tc_bidir_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                     const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO, BidirParams p) {
-    // Tensor-memory columns: S 64 | O[2] 64 each.
+    // Tensor-memory columns: S 64 | O 64.
     constexpr uint32_t colS = 0, colO = 64;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* gbase = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t bars = base + L::kOffCtl;
     // Phase 1 (per chunk, pairs indexed by chunk parity): KV_FULL, K_READY, U_FULL.
-    // Phase 2 (per chunk, rings of four / two): Q_FULL[4], O_FULL[2], E_DONE[2], OUT_FREE[2], Q_READ[4].
+    // Phase 2 (per chunk): Q_FULL[4], Q_READ[4] and E_DONE[4] by tile slot, O_FULL[2] and O_DRAIN[2] by chunk parity.
     // A waiter may only ask for the phase that follows the last one it saw complete on the same
     // barrier: asking for one further ahead passes at once (a fresh barrier counts as having
     // completed an odd phase), and asking for one the barrier has left two or more behind
     // blocks until the next phase of that parity.  Hence PH1_DONE for "the whole state is
     // there": the row workers take alternate chunks and do not follow every U_FULL phase.
-    enum { B_KVFULL = 0, B_KREADY = 16, B_UFULL = 32, B_SBREADY = 48, B_PH1DONE = 56, B_QFULL = 64, B_OFULL = 96, B_EDONE = 112,
-           B_OUTFREE = 128, B_QREAD = 144 };
+    enum { B_KVFULL = 0, B_KREADY = 16, B_UFULL = 32, B_SBREADY = 48, B_PH1DONE = 56, B_QFULL = 64, B_OFULL = 96, B_ODRAIN = 112,
+           B_EDONE = 128, B_QREAD = 160 };
     const uint32_t tmem_slot = bars + kCtlTmemSlot;
     volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(gbase + L::kOffCtl + kCtlTmemSlot);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + L::kOffCtl + kCtlAbort);
@@ -72,7 +73,7 @@ tc_bidir_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const bool is_mma = warp == kWorkerWarps, is_copy = warp == kWorkerWarps + 1;
 
     if (is_mma) {
-        tmem_alloc(tmem_slot, 256);
+        tmem_alloc(tmem_slot, 128);
         tmem_relinquish();
     }
     if (tid == 0) {
@@ -81,12 +82,13 @@ tc_bidir_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             mbar_init(bars + B_KREADY + 8 * i, 128);
             mbar_init(bars + B_UFULL + 8 * i, 1);
             mbar_init(bars + B_OFULL + 8 * i, 1);
-            mbar_init(bars + B_EDONE + 8 * i, 256);
-            mbar_init(bars + B_OUTFREE + 8 * i, 1);
+            mbar_init(bars + B_ODRAIN + 8 * i, 256);
         }
         mbar_init(bars + B_SBREADY, 256);
         mbar_init(bars + B_PH1DONE, 1);
-        for (int i = 0; i < 4; ++i) { mbar_init(bars + B_QFULL + 8 * i, 1); mbar_init(bars + B_QREAD + 8 * i, 256); }
+        for (int i = 0; i < 4; ++i) {
+            mbar_init(bars + B_QFULL + 8 * i, 1); mbar_init(bars + B_EDONE + 8 * i, 256); mbar_init(bars + B_QREAD + 8 * i, 256);
+        }
         *abort_flag = 0;
         abort_flag[3] = p.wait_limit_kcycles;
         mbar_fence_init();
@@ -128,16 +130,20 @@ tc_bidir_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             }
             // phase 2: q of chunk c into slot c & 3, once the slot's last reader is done: a (k, v)
             // pair of phase 1 (the state update of the last chunk with that parity), then the
-            // row norms and the product of chunk c - 4
+            // store of the output rows of chunk c - 4, which were staged in the slot
+            auto store = [&](int e) {
+                const bool hfo = (p.head_first_mask >> 3) & 1;
+                tma_store_4d(&tmO, base + (uint32_t)(e & 3) * kTile, 0, hfo ? h : e * kC, hfo ? e * kC : h, b);
+                tma_store_commit();
+            };
             for (int c = 0; c < n_chunks && ok; ++c) {
                 if (c < 4) {
                     const int par = (c & 3) >> 1;                         // stage of phase 1 that used the slot
                     const int last = ((n_chunks - 1) & 1) == par ? n_chunks - 1 : n_chunks - 2;
                     if (last >= 0 && !wait_or_abort(bars + B_UFULL + 8 * par, par2(last), abort_flag)) { ok = false; break; }
                 } else {
-                    // (its product has completed: this thread saw the epilogue of chunk c - 4 done
-                    // when it stored that chunk's rows)
-                    if (!wait_or_abort(bars + B_QREAD + 8 * (c & 3), par4(c - 4), abort_flag)) { ok = false; break; }
+                    // stores issued so far: chunks 0 .. c - 3; all but the last must have read their tile
+                    tma_store_wait_read1();
                 }
                 const uint32_t fb = bars + B_QFULL + 8 * (c & 3);
                 mbar_expect_tx(fb, kTile);
@@ -145,19 +151,13 @@ tc_bidir_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 // the output rows of chunk c - 2, if staged meanwhile, go out between the loads
                 if (c >= 2) {
                     const int e = c - 2;
-                    if (!wait_or_abort(bars + B_EDONE + 8 * (e & 1), par2(e), abort_flag)) { ok = false; break; }
-                    const bool hfo = (p.head_first_mask >> 3) & 1;
-                    tma_store_4d(&tmO, base + L::kOffOut + (uint32_t)(e & 1) * kTile, 0, hfo ? h : e * kC, hfo ? e * kC : h, b);
-                    tma_store_commit();
-                    tma_store_wait_read0();
-                    mbar_arrive(bars + B_OUTFREE + 8 * (e & 1));
+                    if (!wait_or_abort(bars + B_EDONE + 8 * (e & 3), par4(e), abort_flag)) { ok = false; break; }
+                    store(e);
                 }
             }
             for (int e = (n_chunks >= 2 ? n_chunks - 2 : 0); e < n_chunks && ok; ++e) {
-                if (!wait_or_abort(bars + B_EDONE + 8 * (e & 1), par2(e), abort_flag)) break;
-                const bool hfo = (p.head_first_mask >> 3) & 1;
-                tma_store_4d(&tmO, base + L::kOffOut + (uint32_t)(e & 1) * kTile, 0, hfo ? h : e * kC, hfo ? e * kC : h, b);
-                tma_store_commit();
+                if (!wait_or_abort(bars + B_EDONE + 8 * (e & 3), par4(e), abort_flag)) break;
+                store(e);
             }
             tma_store_wait_all0();
         }
@@ -182,14 +182,14 @@ tc_bidir_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 for (int c = 0; c < n_chunks; ++c) {
                     // O = Q S: Q K-major, the bf16 state MN-major (its rows are the contraction index)
                     if (!wait_or_abort(bars + B_QFULL + 8 * (c & 3), par4(c), abort_flag)) break;
-                    // (the accumulator of this parity was drained by the epilogue of chunk c - 2)
-                    if (c >= 2 && !wait_or_abort(bars + B_EDONE + 8 * (c & 1), par2(c - 2), abort_flag)) break;
+                    // (the one accumulator was drained by the epilogue of the chunk before)
+                    if (c >= 1 && !wait_or_abort(bars + B_ODRAIN + 8 * ((c - 1) & 1), par2(c - 1), abort_flag)) break;
                     tc_fence_after();
                     constexpr uint32_t idesc = instr_desc_bf16(128, kD, false, true);
                     const uint32_t xl = smem_desc_lo(base + (uint32_t)(c & 3) * kTile, 16), sl = smem_desc_lo(base + L::kOffSb, kD * 128u);
 #pragma unroll
                     for (int kk = 0; kk < kD / 16; ++kk)
-                        mma_ss_w(tmem + colO + (c & 1) * 64, xl + kk * 2u, kDescHi, sl + kk * 128u, kDescHi, idesc, kk > 0);
+                        mma_ss_w(tmem + colO, xl + kk * 2u, kDescHi, sl + kk * 128u, kDescHi, idesc, kk > 0);
                     tc_commit(bars + B_OFULL + 8 * (c & 1));
                 }
             }
@@ -266,13 +266,18 @@ tc_bidir_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             }
             const float rx = cfac / fmaxf(sqrtf((a0 + a1) + (a2 + a3)), kEps);
             mbar_arrive(bars + B_QREAD + 8 * (c & 3));
+            // the product has read the q tile and filled the accumulator: drain it, then stage
+            // the rows where q was
             if (!wait(bars + B_OFULL + 8 * (c & 1), par2(c))) break;
-            if (c >= 2 && !wait(bars + B_OUTFREE + 8 * (c & 1), par2(c - 2))) break;
             tc_fence_after();
             uint32_t a[32];
-            tmem_ld32(tmem + lane_base + colO + (c & 1) * 64 + hw * 32, a);
+            tmem_ld32(tmem + lane_base + colO + hw * 32, a);
             tmem_wait_ld();
-            uint8_t* out = gbase + L::kOffOut + (c & 1) * kTile;
+            tc_fence_before();
+            mbar_arrive(bars + B_ODRAIN + 8 * (c & 1));
+            // (both threads of a row sum the whole q row: the other one must be done with it)
+            if (!wait(bars + B_QREAD + 8 * (c & 3), par4(c))) break;
+            uint8_t* out = gbase + (c & 3) * kTile;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 uint4 o;
@@ -283,8 +288,7 @@ tc_bidir_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 *reinterpret_cast<uint4*>(out + swz(row, hw * 4 + j)) = o;
             }
             fence_proxy_async();
-            tc_fence_before();
-            mbar_arrive(bars + B_EDONE + 8 * (c & 1));
+            mbar_arrive(bars + B_EDONE + 8 * (c & 3));
         }
     }
     tc_fence_before();
@@ -298,7 +302,7 @@ tc_bidir_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             p.status[2] = (int)blockIdx.x | (5 << 24);
         }
     }
-    if (is_mma) tmem_dealloc(tmem, 256);
+    if (is_mma) tmem_dealloc(tmem, 128);
 }
 
 }  // namespace
