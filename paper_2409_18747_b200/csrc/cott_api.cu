@@ -73,11 +73,12 @@ static Option g_opt_pair("pair", "COTT_PAIR", 1);                          // 0:
 static Option g_opt_fused_bwd("fused_bwd", "COTT_FUSED_BWD", 1);           // 0: causal d=64 backward through the three role-swapped walks
 static Option g_opt_fused_bidir("fused_bidir", "COTT_FUSED_BIDIR", 1);     // 0: bidirectional d=64 forward as state pass + read-out
 static Option g_opt_short_fwd("short_fwd", "COTT_SHORT_FWD", 1);           // 0: sequences of <= 128 tokens through the generic walk
+static Option g_opt_block_fwd("block_fwd", "COTT_BLOCK_FWD", 1);           // 0: blocks of <= 64 tokens on a state through the generic walk
 static Option g_opt_wait_ms("wait_limit_ms", "COTT_WAIT_LIMIT_MS", 2000);  // bound of every device-side wait
 static Option g_opt_wait_kc("wait_limit_kcycles", "COTT_WAIT_LIMIT_KCYCLES", -1);  // the same in units of 1024 SM cycles (< 0: use the ms value)
 static Option g_opt_host_slices("host_slices", "COTT_HOST_SLICES", 8);     // slices of the host-buffer step (1 .. 16)
 static Option* const g_options[] = {&g_opt_force_group, &g_opt_force_path, &g_opt_pair, &g_opt_fused_bwd,
-                                    &g_opt_wait_ms, &g_opt_wait_kc, &g_opt_host_slices, &g_opt_fused_bidir, &g_opt_short_fwd};
+                                    &g_opt_wait_ms, &g_opt_wait_kc, &g_opt_host_slices, &g_opt_fused_bidir, &g_opt_short_fwd, &g_opt_block_fwd};
 
 int option_force_group() { return (int)g_opt_force_group.get(); }
 int option_force_path() { return (int)g_opt_force_path.get(); }
@@ -85,6 +86,7 @@ int option_pair() { return (int)g_opt_pair.get(); }
 int option_fused_bwd() { return (int)g_opt_fused_bwd.get(); }
 int option_fused_bidir() { return (int)g_opt_fused_bidir.get(); }
 int option_short_fwd() { return (int)g_opt_short_fwd.get(); }
+int option_block_fwd() { return (int)g_opt_block_fwd.get(); }
 int wait_limit_kcycles() {
     const long long kc = g_opt_wait_kc.get();
     if (kc >= 0) return (int)(kc > 200000000 ? 200000000 : kc);
@@ -440,6 +442,13 @@ static cott_status fwd_impl(const void* q, const void* k, const void* v, void* o
         COTT_CUDA(launch_tc_short_fwd(q, k, v, o, static_cast<int*>(ws), sp->m, sp->seq_len, sp->seq_len_scalar, B, H, N,
                                       d, p.dk, p.dv, causal, st));
         return COTT_OK;
+    }
+    if (p.path == 1 && causal && N <= 64 && (state_in || state_out) && !packed.cu_seqlens && option_block_fwd() != 0) {
+        // A short block on a caller's state (multi-token decode, short prefill segments): one
+        // light kernel, several CTAs per SM (cott_tc_block.cu).
+        COTT_CUDA(launch_tc_block_fwd(q, k, v, o, lay.qkv, lay.of(v), lay.o, state_in, state_out, static_cast<int*>(ws),
+                                      sp->m, sp->seq_len, sp->seq_len_scalar, B, H, N, d, p.dk, p.dv, st));
+        return finish();
     }
     if (p.path == 1 && !causal && d == 64 && p.n_groups == 1 && !packed.cu_seqlens && !state_in &&
         option_fused_bidir() != 0) {

@@ -144,7 +144,7 @@ cudaError_t launch_tc_bidir_fwd(const void* q, const void* k, const void* v, voi
 // Tensor map over a bf16 tensor of logical shape [B,H,N,d] with the given row layout: box of
 // 128 tokens x 64 columns of one (b,h), 128-byte swizzle (see cott_tc_walk.cu).
 bool make_tile_map(CUtensorMap* map, const void* ptr, int B, int H, int N, int d, const RowLayout& lay,
-                   bool* head_first);
+                   bool* head_first, int box_rows = 128);
 
 bool make_rows_map(CUtensorMap* map, const void* ptr, long long rows, int d, int box_rows);
 
@@ -153,6 +153,13 @@ bool make_rows_map(CUtensorMap* map, const void* ptr, long long rows, int d, int
 cudaError_t launch_tc_short_fwd(const void* q, const void* k, const void* v, void* o, int* status, const float* m,
                                 const float* seq_len, float seq_len_scalar, int B, int H, int N, int d, int dk, int dv,
                                 int causal, cudaStream_t st);
+
+// A block of at most 64 tokens per (b, h) on a caller's state (cott_tc_block.cu): o and the new
+// state in one launch, the only kernel of its call.
+cudaError_t launch_tc_block_fwd(const void* q, const void* k, const void* v, void* o, const RowLayout& l_qk,
+                                const RowLayout& l_v, const RowLayout& l_o, const float* state_in, float* state_out,
+                                int* status, const float* m, const float* seq_len, float seq_len_scalar, int B, int H,
+                                int N, int d, int dk, int dv, cudaStream_t st);
 
 // Opt-in to `bytes` of dynamic shared memory for a kernel, once per (kernel, device).
 cudaError_t configure_smem_once(const void* func, int bytes);
@@ -164,6 +171,7 @@ int option_pair();
 int option_fused_bwd();
 int option_fused_bidir();
 int option_short_fwd();
+int option_block_fwd();
 int wait_limit_kcycles();      // bound of every device-side wait, in units of 1024 SM cycles
 
 cudaError_t launch_dm_finalize(const float* dm_partial, float* dm, const float* m,

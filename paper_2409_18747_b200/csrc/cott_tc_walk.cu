@@ -1229,7 +1229,7 @@ EncodeTiledFn get_encode() {
 // tokens x 64 columns of one (b,h), 128-byte swizzle; rows past N read as zero and are not
 // written.  *head_first tells the kernel the order of the two middle coordinates.
 bool make_tile_map(CUtensorMap* map, const void* ptr, int B, int H, int N, int d, const RowLayout& lay,
-                   bool* head_first) {
+                   bool* head_first, int box_rows) {
     EncodeTiledFn enc = get_encode();
     if (!enc) return false;
     const RowLayout l = resolve_layout(lay, H, N, d);
@@ -1239,7 +1239,7 @@ bool make_tile_map(CUtensorMap* map, const void* ptr, int B, int H, int N, int d
     cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)(hf ? H : N), (cuuint64_t)(hf ? N : H), (cuuint64_t)B};
     cuuint64_t strides[3] = {(cuuint64_t)(hf ? l.sh : l.sn) * 2, (cuuint64_t)(hf ? l.sn : l.sh) * 2,
                              (cuuint64_t)l.sb * 2};
-    cuuint32_t box[4] = {64, hf ? 1u : (cuuint32_t)kChunk, hf ? (cuuint32_t)kChunk : 1u, 1};
+    cuuint32_t box[4] = {64, hf ? 1u : (cuuint32_t)box_rows, hf ? (cuuint32_t)box_rows : 1u, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides,
                      box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,

@@ -759,6 +759,51 @@ def test_short_sequences_take_the_quadratic_side(N, dk, dv, causal, option):
         assert not torch.equal(o2[1, 2], o[1, 2])
 
 
+@pytest.mark.parametrize("T", [1, 5, 16, 33, 64])
+@pytest.mark.parametrize("dk,dv", [(128, 128), (64, 64), (96, 40)])
+def test_token_blocks_on_a_state(T, dk, dv, option):
+    """Blocks of at most 64 tokens on a caller-held state take a kernel of their own (several
+    CTAs per SM, the state read and written once): prefill 200 tokens, then three blocks of T
+    tokens; rows and the final [d_key, d_value] state against one long causal forward by the
+    definition; more (b, h) pairs than fit on the GPU at once."""
+    B, H, N0 = 5, 40, 200
+    N = N0 + 3 * T
+    c = synth.make_qkv(B, H, N, dk, torch.bfloat16, 6700 + T + dk, d_v=dv)
+    s = np.full((B,), float(N))
+    q, k, v, m = (dev(c[x]) for x in ("q", "k", "v", "m"))
+    seg = lambda x, a, b: x[:, :, a:b].contiguous()
+    o0, state = cott.fwd(seg(q, 0, N0), seg(k, 0, N0), seg(v, 0, N0), m, seq_len=float(N), causal=True, return_state=True)
+    rows = [o0]
+    for i in range(3):
+        a, b = N0 + i * T, N0 + (i + 1) * T
+        cott.cott.profile_enable(8)
+        o, state = cott.fwd_stateful(seg(q, a, b), seg(k, a, b), seg(v, a, b), m, float(N), state_in=state)
+        kinds = [kd for kd, _ in cott.cott.profile_read()]
+        cott.cott.profile_enable(0)
+        assert kinds == [6]
+        rows.append(o)
+    # a sample of (b, h) pairs through the oracle (the whole batch would take a minute)
+    pick = [(0, 0), (2, 17), (4, 39)]
+    sub = {x: np.stack([c[x][b_, h_].float().numpy() for b_, h_ in pick])[None] for x in ("q", "k", "v")}
+    msub = np.array([float(c["m"][h_]) for _, h_ in pick])
+    ref = oracle.fwd_quadratic(sub["q"], sub["k"], sub["v"], msub, np.array([float(N)]), True)[0]
+    _, ref_state = oracle.fwd_recurrent(sub["q"], sub["k"], sub["v"], msub, np.array([float(N)]))
+    got = torch.cat(rows, dim=2)
+    got_sub = torch.stack([got[b_, h_] for b_, h_ in pick])
+    gate(got_sub, ref, torch.bfloat16)
+    st_sub = torch.stack([state[b_, h_] for b_, h_ in pick])
+    assert norm_max_err(st_sub, ref_state[0]) <= state_tol(torch.bfloat16, max(dk, dv))
+    # the same blocks through the generic walk agree
+    option("block_fwd", 0)
+    o_w, st_w = cott.fwd_stateful(seg(q, N - T, N), seg(k, N - T, N), seg(v, N - T, N), m, float(N),
+                                  state_in=state.clone())
+    option("block_fwd", 1)
+    o_b, st_b = cott.fwd_stateful(seg(q, N - T, N), seg(k, N - T, N), seg(v, N - T, N), m, float(N),
+                                  state_in=state.clone())
+    assert norm_max_err(o_b, o_w.double().cpu().numpy()) <= TOL_BF16
+    assert norm_max_err(st_b, st_w.double().cpu().numpy()) <= 1e-3
+
+
 # ------------------------------------------------------------------ head sizes (d_key, d_value)
 HEAD_SIZES = [(32, 32), (96, 96), (64, 128), (128, 64), (32, 64), (40, 72), (8, 16), (128, 32), (72, 8)]
 
