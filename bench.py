@@ -37,7 +37,7 @@ L2_FLUSH_BYTES = 256 << 20  # larger than the 126 MB L2
 # Missing key: no capture of that class.
 STEP_DRAM_TRAFFIC = {
     (64, True, True): 1704.6,     # C4 step: 446.8 MB over 262 144 token-heads (method's bytes: 1408)
-    (64, False, False): 403.1,    # C2 forward: 79.3 MB over 196 608 token-heads (method's bytes: 512;
+    (64, False, False): 403.5,    # C2 forward: 79.3 MB over 196 608 token-heads (method's bytes: 512;
                                   # a third of the output is still in L2 when the kernel ends)
 }
 
