@@ -567,6 +567,14 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
             f.dm_partial = dm_partial; f.dm_out = dm; f.status = status;
             f.m = sp->m; f.seq_len = sp->seq_len; f.seq_len_scalar = sp->seq_len_scalar;
             f.group = p.group; f.n_groups = p.n_groups;
+            if (p.n_groups == 1 && N <= 128) {
+                // One chunk per (b, h): no state is ever read, the walk is the only launch.
+                f.sq_part = nullptr; f.r_part = nullptr;
+                COTT_CUDA(cudaMemsetAsync(ws, 0, kWsHeaderBytes, st));      // status words and the dm counter
+                f.plain_launch = 1;
+                COTT_CUDA(launch_tc_bwd_fused(f, B, H, N, st));
+                return COTT_OK;
+            }
             COTT_CUDA(launch_tc_bwd_states(f, st0, st1, 1, B, H, N, st));
             COTT_CUDA(launch_tc_bwd_fused(f, B, H, N, st));
             return COTT_OK;

@@ -77,6 +77,7 @@ struct BwdParams {
     int H; int N; int group; int n_groups;
     int wait_limit_kcycles;
     int head_first_mask;     // bit i: in tensor map i (q, k, v, dO, dq, dk, dv) the head index comes before the token index
+    int no_state;            // the whole sequence is one chunk: both states are zero wherever they are read, no update
 };
 
 
@@ -413,7 +414,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 if (c >= 1 && !wait_or_abort(bar(B_CLREADY, c - 1), par(c - 1), abort_flag)) break;
                 BSTAMP(6, c, 1);
                 tc_fence_after();
-                issue_update(tmem + colS, st + L::kOffV, st + L::kOffK);
+                if (!p.no_state) issue_update(tmem + colS, st + L::kOffV, st + L::kOffK);
                 tc_commit(bar(B_UFULL, c));
                 BSTAMP(6, c, 2);
             }
@@ -1001,6 +1002,10 @@ cudaError_t launch_tc_bwd_fused(const TcBwdFusedArgs& a, int B, int H, int N, cu
     p.status = a.status; p.m = a.m; p.seq_len = a.seq_len; p.seq_len_scalar = a.seq_len_scalar;
     p.H = H; p.N = N; p.group = a.group; p.n_groups = a.n_groups;
     p.wait_limit_kcycles = wait_limit_kcycles();
+    // One chunk per (b, h): nothing precedes it (Sq = 0) and nothing follows it (R = 0 once its own
+    // update is taken out again), so the states stay zero and no partial-state pass is needed.
+    p.no_state = (a.n_groups == 1 && N <= kC && !a.sq_part && !a.r_part) ? 1 : 0;
+    if (!p.no_state && !a.r_part) return cudaErrorInvalidValue;
     if (cudaError_t e = configure_smem_once(reinterpret_cast<const void*>(tc_bwd_fused_kernel), L::kDynBytes); e != cudaSuccess)
         return e;
     const int prof = profile_begin_launch(3, st);
