@@ -802,6 +802,13 @@ def test_token_blocks_on_a_state(T, dk, dv, option):
                                   state_in=state.clone())
     assert norm_max_err(o_b, o_w.double().cpu().numpy()) <= TOL_BF16
     assert norm_max_err(st_b, st_w.double().cpu().numpy()) <= 1e-3
+    # the block read in place from the long tensors (rows N - T .. N - 1 of every (b, h)) and
+    # written into a [B,T,H,d] buffer: bit-identical to the call on contiguous copies
+    out_bthd = torch.empty((B, T, H, dv), dtype=torch.bfloat16, device="cuda").permute(0, 2, 1, 3)
+    o_s, st_s = cott.fwd_stateful(q[:, :, N - T:], k[:, :, N - T:], v[:, :, N - T:], m, float(N),
+                                  state_in=state.clone(), out=out_bthd)
+    assert not q[:, :, N - T:].is_contiguous() or T == N
+    assert torch.equal(o_s, o_b) and torch.equal(st_s, st_b)
 
 
 # ------------------------------------------------------------------ head sizes (d_key, d_value)
