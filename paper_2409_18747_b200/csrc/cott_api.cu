@@ -552,7 +552,7 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
         // over the whole sequence as a single group (no partial-state pass, no scan), with the
         // dQ^ stream's partial-state pass filling the SMs that are left; the dQ^ walk follows on
         // the whole GPU.  Each side stream then carries one tensor-core kernel per call.
-        if (causal && d == 64 && !packed.cu_seqlens && option_fused_bwd() != 0) {
+        if (d == 64 && !packed.cu_seqlens && option_fused_bwd() != 0) {
             // One walk forward in time gives all three gradients and the dm sum (cott_tc_bwd.cu).
             // It keeps two running states: Sq = V^T K^ over earlier tokens, accumulated chunk by
             // chunk, and R = Q^^T dO over later tokens, which starts at the sum over the group
@@ -567,7 +567,8 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
             f.dm_partial = dm_partial; f.dm_out = dm; f.status = status;
             f.m = sp->m; f.seq_len = sp->seq_len; f.seq_len_scalar = sp->seq_len_scalar;
             f.group = p.group; f.n_groups = p.n_groups;
-            if (p.n_groups == 1 && N <= 128) {
+            f.bidir = causal ? 0 : 1;
+            if (causal && p.n_groups == 1 && N <= 128) {
                 // One chunk per (b, h): no state is ever read, the walk is the only launch.
                 f.sq_part = nullptr; f.r_part = nullptr;
                 COTT_CUDA(cudaMemsetAsync(ws, 0, kWsHeaderBytes, st));      // status words and the dm counter

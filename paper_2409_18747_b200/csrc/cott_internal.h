@@ -127,6 +127,7 @@ struct TcBwdFusedArgs {
     const float* m; const float* seq_len; float seq_len_scalar;
     int group; int n_groups;
     int plain_launch;
+    int bidir;      // 1: all-ones mask (bidirectional backward): both states are totals over the sequence
     int w_k, w_v;   // real columns of q, k, dq, dk and of v, dO, dv when fewer than 64 (0: 64)
 };
 cudaError_t launch_tc_bwd_fused(const TcBwdFusedArgs& a, int B, int H, int N, cudaStream_t st);

@@ -145,18 +145,20 @@ __device__ __forceinline__ void issue_pt_b(uint32_t tO, uint32_t tPt, uint32_t b
     for (int kk = 0; kk < kC / 16; ++kk) mma_ts_w(tO, tPt + kk * 8u, bl + kk * 128u, kDescHi, idesc, kk > 0);
 }
 // Out[128 x 64] += X[128 x 64] St[64 x 64], St read MN-major (its rows are the contraction index).
-__device__ __forceinline__ void issue_x_state(uint32_t tO, uint32_t x, uint32_t st) {
+__device__ __forceinline__ void issue_x_state(uint32_t tO, uint32_t x, uint32_t st, bool acc_first = true) {
     constexpr uint32_t idesc = instr_desc_bf16(128, kD, false, true);
     const uint32_t xl = smem_desc_lo(x, 16), sl = smem_desc_lo(st, kD * 128u);
 #pragma unroll
-    for (int kk = 0; kk < kD / 16; ++kk) mma_ss_w(tO, xl + kk * 2u, kDescHi, sl + kk * 128u, kDescHi, idesc, 1u);
+    for (int kk = 0; kk < kD / 16; ++kk)
+        mma_ss_w(tO, xl + kk * 2u, kDescHi, sl + kk * 128u, kDescHi, idesc, (acc_first || kk > 0) ? 1u : 0u);
 }
 // Out[128 x 64] += X[128 x 64] St^T, St read K-major (its columns are the contraction index).
-__device__ __forceinline__ void issue_x_state_t(uint32_t tO, uint32_t x, uint32_t st) {
+__device__ __forceinline__ void issue_x_state_t(uint32_t tO, uint32_t x, uint32_t st, bool acc_first = true) {
     constexpr uint32_t idesc = instr_desc_bf16(128, kD, false, false);
     const uint32_t xl = smem_desc_lo(x, 16), sl = smem_desc_lo(st, 16);
 #pragma unroll
-    for (int kk = 0; kk < kD / 16; ++kk) mma_ss_w(tO, xl + kk * 2u, kDescHi, sl + kk * 2u, kDescHi, idesc, 1u);
+    for (int kk = 0; kk < kD / 16; ++kk)
+        mma_ss_w(tO, xl + kk * 2u, kDescHi, sl + kk * 2u, kDescHi, idesc, (acc_first || kk > 0) ? 1u : 0u);
 }
 // State[128 x 128] += [V | Q^]^T [K^ | dO]: both operands MN-major, 128 wide (two tiles 16 KB apart).
 __device__ __forceinline__ void issue_update(uint32_t tS, uint32_t vq, uint32_t kdo) {
@@ -173,6 +175,13 @@ __device__ __forceinline__ void issue_update(uint32_t tS, uint32_t vq, uint32_t 
 // mbarriers, every wait bounded.  Every per-chunk barrier is a pair indexed by chunk parity:
 // the two-stage ring keeps all roles within one chunk of each other (the tiles of chunk c + 2
 // are requested only after every epilogue of chunk c), so a phase parity names one chunk.
+// BIDIR: the bidirectional backward (all-ones mask).  Both states are then totals over the whole
+// sequence -- S^T = V^T K^ and R = Q^^T dO, summed in the prologue from the partial states of ALL
+// groups -- and every chunk's rows are plain products with them,
+//     dQ^ = dO S^T ,   dK^ = V R^T ,   dV' = K^ R ,
+// so the score products, the masks, the state update and the per-chunk state copies fall away;
+// loads, row norms, epilogues, stores and the dm sum are those of the causal walk.
+template <bool BIDIR>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                     const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmDO,
@@ -297,7 +306,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 #pragma unroll
             for (int i = 0; i < 32; ++i) acc[i] = 0.f;
             const float* src = upper ? p.sq_part : p.r_part;
-            const int g_lo = upper ? 0 : g, g_hi = upper ? g : p.n_groups;
+            const int g_lo = BIDIR ? 0 : (upper ? 0 : g), g_hi = BIDIR ? p.n_groups : (upper ? g : p.n_groups);
             const size_t off = (size_t)(row & 63) * kD + (size_t)(wg & 1) * 32;
             if (src != nullptr) {
                 for (int gg = g_lo; gg < g_hi; ++gg) {
@@ -309,21 +318,25 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     }
                 }
             }
-            if (upper) {
+            if (upper || BIDIR) {
                 // Sq is what the first chunk reads before any update: its bf16 copy goes to the
-                // late-copy buffer
+                // late-copy buffer.  (Bidirectional: both totals are copied here, once: S^T to
+                // the late-copy buffer, R to the first early-copy buffer.)
 #pragma unroll
                 for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(acc[i]);
+                uint8_t* dst = gbase + (upper ? L::kOffLb : L::kOffEb);
 #pragma unroll
                 for (int i = 0; i < 32; i += 8)
-                    *reinterpret_cast<uint4*>(gbase + L::kOffLb + swz(row & 63, (uint32_t)((wg & 1) * 4 + (i >> 3)))) = pack8(&r[i]);
+                    *reinterpret_cast<uint4*>(dst + swz(row & 63, (uint32_t)((wg & 1) * 4 + (i >> 3)))) = pack8(&r[i]);
             } else {
 #pragma unroll
                 for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(-acc[i]);
             }
         }
-        tmem_st32(tmem + lane_base + colS + wg * 32, r);
-        tmem_wait_st();
+        if (!BIDIR) {
+            tmem_st32(tmem + lane_base + colS + wg * 32, r);
+            tmem_wait_st();
+        }
         fence_proxy_async();
     }
     tc_fence_before();
@@ -356,7 +369,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 mbar_arrive(bars + B_STQFREE);           // the tile may take the dv rows of the chunk
                 if (more) {
                     if (!wait_or_abort(bar(B_OVFULL, c), par(c), abort_flag)) break;
-                    if (!wait_or_abort(bar(B_UFULL, c), par(c), abort_flag)) break;
+                    if (!BIDIR && !wait_or_abort(bar(B_UFULL, c), par(c), abort_flag)) break;
                     mbar_expect_tx(fb, 4 * kTile);
                     coords(3, nrow, c1, c2); tma_load_4d(st + L::kOffDO, &tmDO, fb, 0, c1, c2, b);
                     coords(2, nrow, c1, c2); tma_load_4d(st + L::kOffV, &tmV, fb, 0, c1, c2, b);
@@ -381,7 +394,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
     } else if (is_score) {
         // ------------------------------------------------------------------ score thread
-        if (lane == 0) {
+        if (lane == 0 && !BIDIR) {
             for (int c = 0; c < n_chunks; ++c) {
                 const uint32_t st = stage(c);
                 if (!wait_or_abort(bar(B_FULL, c), par(c), abort_flag)) break;
@@ -404,7 +417,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
     } else if (is_upd) {
         // ------------------------------------------------------------------ state-update thread
-        if (lane == 0) {
+        if (lane == 0 && !BIDIR) {
             for (int c = 0; c < n_chunks; ++c) {
                 const uint32_t st = stage(c);
                 if (!wait_or_abort(bar(B_NREADY, c), par(c), abort_flag)) break;
@@ -421,7 +434,28 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
     } else if (is_out) {
         // ------------------------------------------------------------------ output-product thread
-        if (lane == 0) {
+        if (lane == 0 && BIDIR) {
+            // every chunk: three products of its rows with the two totals
+            const uint32_t st_t = base + L::kOffLb, rt = base + L::kOffEb;
+            for (int c = 0; c < n_chunks; ++c) {
+                const uint32_t st = stage(c);
+                const uint32_t tP1 = tmem + colP1 + (c & 1) * 128;
+                if (!wait_or_abort(bar(B_NREADY, c), par(c), abort_flag)) break;
+                // (the accumulators of this parity were drained by the epilogues of chunk c - 2,
+                // which the request for this chunk's tiles waited for)
+                tc_fence_after();
+                issue_x_state(tP1, st + L::kOffDO, st_t, false);          // dQ^ = dO S^T
+                tc_commit(bar(B_OQFULL, c));
+                issue_x_state_t(tP1 + 64, st + L::kOffV, rt, false);      // dK^ = V R^T
+                tc_commit(bar(B_OKFULL, c));
+                // the one dV' accumulator: drained by the epilogue of the chunk before
+                if (c >= 1 && !wait_or_abort(bar(B_OVFREE, c - 1), par(c - 1), abort_flag)) break;
+                tc_fence_after();
+                issue_x_state(tmem + colP2 + 64, st + L::kOffK, rt, false);   // dV' = K^ R
+                tc_commit(bar(B_OVFULL, c));
+            }
+        }
+        if (lane == 0 && !BIDIR) {
             const uint32_t gt = base + L::kOffG;
             for (int c = 0; c < n_chunks; ++c) {
                 const uint32_t st = stage(c);
@@ -517,7 +551,10 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 if (tid == 0) BSTAMP(3, c, 2);
             };
             normalise(0);
-            for (int c = 0; c < n_chunks && alive; ++c) {
+            if (BIDIR) {
+                for (int c = 1; c < n_chunks && alive; ++c) normalise(c);
+            }
+            for (int c = 0; !BIDIR && c < n_chunks && alive; ++c) {
                 // ---- G[i][j] = dO_i . v_j, kept for j <= i (diagonal kept, Eq. 6), rounded to bf16,
                 // into shared memory; this warp's half: column blocks 2 hw and 2 hw + 1.  Per
                 // 32 x 32 block (row block q4, column block cb) the mask is all-keep, all-zero or
@@ -814,6 +851,7 @@ struct StateParams {
     int clear_status;
     int wait_limit_kcycles;
     int head_first_mask;     // bit i: in tensor map i (q, k, v, dO) the head index comes before the token index
+    int all_sq;              // bidirectional backward: V^T K^ of the last group is read too
 };
 
 __global__ void __launch_bounds__(kStThreads, 1)
@@ -838,7 +876,7 @@ tc_bwd_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const bool is_mma = warp == 8, is_copy = warp == 9;
     // Nobody reads V^T K^ of the last group: its CTA leaves the v and k slots at zero (the product
     // then adds nothing to that block) and loads q and dO only.
-    const bool need_sq = g + 1 < p.n_groups;
+    const bool need_sq = p.all_sq || g + 1 < p.n_groups;
 
     if (is_mma) {
         tmem_alloc(tmem_slot, 128);
@@ -1004,9 +1042,10 @@ cudaError_t launch_tc_bwd_fused(const TcBwdFusedArgs& a, int B, int H, int N, cu
     p.wait_limit_kcycles = wait_limit_kcycles();
     // One chunk per (b, h): nothing precedes it (Sq = 0) and nothing follows it (R = 0 once its own
     // update is taken out again), so the states stay zero and no partial-state pass is needed.
-    p.no_state = (a.n_groups == 1 && N <= kC && !a.sq_part && !a.r_part) ? 1 : 0;
+    p.no_state = (!a.bidir && a.n_groups == 1 && N <= kC && !a.sq_part && !a.r_part) ? 1 : 0;
     if (!p.no_state && !a.r_part) return cudaErrorInvalidValue;
-    if (cudaError_t e = configure_smem_once(reinterpret_cast<const void*>(tc_bwd_fused_kernel), L::kDynBytes); e != cudaSuccess)
+    auto kern = a.bidir ? tc_bwd_fused_kernel<true> : tc_bwd_fused_kernel<false>;
+    if (cudaError_t e = configure_smem_once(reinterpret_cast<const void*>(kern), L::kDynBytes); e != cudaSuccess)
         return e;
     const int prof = profile_begin_launch(3, st);
     cudaLaunchConfig_t cfg = {};
@@ -1019,7 +1058,7 @@ cudaError_t launch_tc_bwd_fused(const TcBwdFusedArgs& a, int B, int H, int N, cu
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = a.plain_launch ? 0 : 1;
-    cudaError_t le = cudaLaunchKernelEx(&cfg, tc_bwd_fused_kernel, tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], tm[6], p);
+    cudaError_t le = cudaLaunchKernelEx(&cfg, kern, tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], tm[6], p);
     profile_end_launch(prof, st);
     note_launch();
     return le != cudaSuccess ? le : cudaGetLastError();
@@ -1043,6 +1082,7 @@ cudaError_t launch_tc_bwd_states(const TcBwdFusedArgs& a, float* sq_out, float* 
     p.sq_out = sq_out; p.r_out = r_out; p.status = a.status;
     p.H = H; p.N = N; p.group = a.group; p.n_groups = a.n_groups;
     p.clear_status = clear_status;
+    p.all_sq = a.bidir;
     p.wait_limit_kcycles = wait_limit_kcycles();
     constexpr int kBytes = kStStages * L::kStage + L::kCtlBytes + 1024;
     static_assert(kStStages * L::kStage <= L::kOffCtl, "the stage ring overlaps the control block");
