@@ -938,22 +938,31 @@ def test_short_blocks_many_heads(dtype, d):
 
 
 # ------------------------------------------------------------------ a wait that runs out
-@pytest.mark.parametrize("op", ["fwd", "bwd", "bidir"])
+@pytest.mark.parametrize("op", ["fwd", "bwd", "bidir", "bidir_bwd", "short", "block"])
 def test_bounded_wait_runs_out_and_reports(op, option, force_group):
     """Every device-side wait has a bound.  With the bound set to zero a wait gives up unless
     its hand-off is there within a few polls -- and the first tiles of a kernel cannot come
     from memory that fast, so a wait is certain to run out.  The kernel then reports where,
     lets its copies in flight land, frees its tensor memory and returns; the context stays
-    usable and the next call is correct.  (No GPU fault is involved: the kernels end normally.)"""
-    causal = op != "bidir"
+    usable and the next call is correct.  (No GPU fault is involved: the kernels end normally.)
+    One case per warp-specialised kernel: the generic walk, the fused backward (causal and
+    bidirectional instance), the bidirectional, the short-sequence and the block forward."""
+    causal = op not in ("bidir", "bidir_bwd")
     force_group(512 if causal else 4096)
-    c = synth.make_qkv(1, 2, 1024, 64, torch.bfloat16, 5400, with_do=True)
+    N = {"short": 64, "block": 16}.get(op, 1024)
+    c = synth.make_qkv(1, 2, N, 64, torch.bfloat16, 5400, with_do=True)
     q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
-    code = cott.cott.OP_BWD if op == "bwd" else cott.cott.OP_FWD
-    ws = torch.zeros(cott.workspace_bytes(code, cott.cott.BF16, 1, 2, 1024, 64, causal),
+    is_bwd = op in ("bwd", "bidir_bwd")
+    code = cott.cott.OP_BWD if is_bwd else cott.cott.OP_FWD
+    ws = torch.zeros(cott.workspace_bytes(code, cott.cott.BF16, 1, 2, N, 64, causal),
                      dtype=torch.uint8, device="cuda")
-    call = (lambda: cott.bwd(q, k, v, d_o, m, causal=True, workspace=ws)) if op == "bwd" else \
-           (lambda: cott.fwd(q, k, v, m, causal=causal, workspace=ws))
+    state0 = torch.zeros((1, 2, 64, 64), dtype=torch.float32, device="cuda")
+    if is_bwd:
+        call = lambda: cott.bwd(q, k, v, d_o, m, causal=causal, workspace=ws)
+    elif op == "block":
+        call = lambda: cott.fwd_stateful(q, k, v, m, float(N), state_in=state0, workspace=ws)[0]
+    else:
+        call = lambda: cott.fwd(q, k, v, m, causal=causal, workspace=ws)
     option("wait_limit_kcycles", 0)
     call()
     assert cott.cott.last_async_status(ws) == -5                 # COTT_ERR_TIMEOUT
@@ -963,10 +972,10 @@ def test_bounded_wait_runs_out_and_reports(op, option, force_group):
     option("wait_limit_kcycles", -1)
     out = call()
     assert cott.cott.last_async_status(ws) == 0
-    if op != "bwd":
+    if not is_bwd:
         gate(out, oracle.fwd_quadratic(c["q"], c["k"], c["v"], c["m"], None, causal), torch.bfloat16)
     else:
-        rq, rk, rv, _ = oracle.bwd_quadratic(c["q"], c["k"], c["v"], c["d_o"], c["m"], None, True)
+        rq, rk, rv, _ = oracle.bwd_quadratic(c["q"], c["k"], c["v"], c["d_o"], c["m"], None, causal)
         gate(out[0], rq, torch.bfloat16); gate(out[1], rk, torch.bfloat16); gate(out[2], rv, torch.bfloat16)
 
 
