@@ -245,7 +245,7 @@ cott_status cott_bwd_strided(const void* q, const void* k, const void* v, const 
  * else its length.  No padding rows are read as keys or written as outputs.
  *   max_seqlen : an upper bound of the longest sequence (sizes the workspace and the plan)
  *   workspace  : cott_workspace_bytes(COTT_OP_FWD or COTT_OP_BWD, dt, B, H, max_seqlen, d, causal)
- * bf16 with d a multiple of 8 up to 128 only (COTT_ERR_UNSUPPORTED otherwise); one CTA walks one (sequence,
+ * bf16 with d a multiple of 8 up to 128, or fp32 with d in {32, 64, 128} (COTT_ERR_UNSUPPORTED otherwise); one CTA walks one (sequence,
  * head), so the GPU is filled when B*H reaches the number of SMs.  A NaN or Inf in the first
  * rows of one sequence can reach the last rows of the sequence stored before it (the tile
  * that holds both is multiplied by zeros, not skipped).  Other arguments, ordering and

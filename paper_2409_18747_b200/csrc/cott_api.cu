@@ -472,6 +472,7 @@ static cott_status fwd_impl(const void* q, const void* k, const void* v, void* o
         return rc != COTT_OK ? rc : finish();
     }
     WalkArgs w = base_walk(sp, H, N, p);
+    w.cu_seqlens = packed.cu_seqlens;
     w.x = q; w.a = k; w.bv = v; w.out = o;
     lay.assign(w);
     w.mode_x = ROW_NORM; w.mode_a = ROW_NORM; w.mode_b = ROW_SCALE;
@@ -656,6 +657,7 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
     {   // dQ^_t = S_t dO_t : the forward walk with (dO, V', K^) in the roles of (Q, K, V)
         WalkArgs w = base_walk(sp, H, N, p);
         w.x = d_o; w.a = v; w.bv = k; w.proj = q; w.out = dq;
+        w.cu_seqlens = packed.cu_seqlens;
         lay.assign(w);
         w.mode_x = ROW_RAW; w.mode_a = ROW_SCALE; w.mode_b = ROW_NORM;
         w.epilogue = EPI_PROJ; w.reverse = 0;
@@ -664,6 +666,7 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
     {   // dK^_j = R_j v'_j : running sum of dO_t q^_t^T accumulated backward in time
         WalkArgs w = base_walk(sp, H, N, p);
         w.x = v; w.a = d_o; w.bv = q; w.proj = k; w.out = dk;
+        w.cu_seqlens = packed.cu_seqlens;
         lay.assign(w);
         w.mode_x = ROW_SCALE; w.mode_a = ROW_RAW; w.mode_b = ROW_NORM;
         w.epilogue = EPI_PROJ; w.reverse = 1;
@@ -672,13 +675,14 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
     {   // dV'_j = R_j^T k^_j, dV = c dV', and <dV', V> for dm
         WalkArgs w = base_walk(sp, H, N, p);
         w.x = k; w.a = q; w.bv = d_o; w.proj = v; w.out = dv;
+        w.cu_seqlens = packed.cu_seqlens;
         lay.assign(w);
         w.mode_x = ROW_NORM; w.mode_a = ROW_NORM; w.mode_b = ROW_RAW;
         w.epilogue = EPI_DV; w.reverse = 1; w.dm_partial = dm_partial;
         if ((rc = run_stream(w, p, BH, d, dt, causal, st2, nullptr, st)) != COTT_OK) return rc;
     }
     COTT_CUDA(launch_dm_finalize(dm_partial, dm, sp->m, sp->seq_len, sp->seq_len_scalar, B, H,
-                                 p.n_groups, N, st));
+                                 p.n_groups, N, st, packed.cu_seqlens));
     return COTT_OK;
 }
 
@@ -945,10 +949,15 @@ cott_status cott_bwd_dkdv(const void* q, const void* k, const void* v, const voi
 // Plan of a packed batch: one group per (sequence, head), tensor-core path only.
 static bool varlen_plan(cott_dtype dt, int B, int H, int total_tokens, int max_seqlen, int d, Plan* p) {
     if (B < 1 || H < 1 || total_tokens < 1 || max_seqlen < 1 || max_seqlen > total_tokens) return false;
-    // bf16, tensor cores: any head size that is a multiple of 8 up to 128 (zero-filled tiles)
-    if (dt != COTT_BF16 || d < 8 || d > 128 || d % 8 != 0) return false;
-    p->path = 1; p->chunk = 128; p->group = (max_seqlen + 127) / 128 * 128; p->n_groups = 1; p->split = 1;
-    p->dk = p->dv = d; p->d = d <= 64 ? 64 : 128; p->padded = p->d != d;
+    // bf16, tensor cores: any head size that is a multiple of 8 up to 128 (zero-filled tiles);
+    // fp32 (and bf16 with force_path = 0): the fp32-accumulating SIMT kernels at 32, 64, 128
+    const bool tc_ok = dt == COTT_BF16 && d >= 8 && d <= 128 && d % 8 == 0;
+    const bool simt_ok = (dt == COTT_F32 || dt == COTT_BF16) && (d == 32 || d == 64 || d == 128);
+    if (!tc_ok && !simt_ok) return false;
+    p->path = (tc_ok && (option_force_path() != 0 || !simt_ok)) ? 1 : 0;
+    p->chunk = p->path == 1 ? 128 : 16;
+    p->group = (max_seqlen + p->chunk - 1) / p->chunk * p->chunk; p->n_groups = 1; p->split = 1;
+    p->dk = p->dv = d; p->d = p->path == 1 ? (d <= 64 ? 64 : 128) : d; p->padded = p->d != d;
     return true;
 }
 

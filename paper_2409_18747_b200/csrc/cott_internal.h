@@ -54,6 +54,9 @@ struct WalkArgs {
     int H; int N; int group; int n_groups;
     int mode_x, mode_a, mode_b;
     int epilogue; int reverse; int update; int write_out;
+    // Packed variable-length batch: B + 1 row offsets into tensors of total rows per head
+    // (batch stride unused), one group per (sequence, head); NULL: dense batch.
+    const int* cu_seqlens;
 };
 
 cudaError_t launch_walk_simt(const WalkArgs& w, int BH, int d, cott_dtype dt, cudaStream_t st);
@@ -177,7 +180,7 @@ int wait_limit_kcycles();      // bound of every device-side wait, in units of 1
 
 cudaError_t launch_dm_finalize(const float* dm_partial, float* dm, const float* m,
                                const float* seq_len, float seq_len_scalar, int B, int H,
-                               int n_groups, int N, cudaStream_t st);
+                               int n_groups, int N, cudaStream_t st, const int* cu_seqlens = nullptr);
 cudaError_t launch_sum_slices(const float* parts, float* out, int n, int H, cudaStream_t st);
 // Caller-visible states [BH, dk, dv] <-> the kernels' padded [BH, d, d] (zero outside).
 cudaError_t launch_pad_state(const float* src, float* dst, int BH, int dk, int dv, int d, cudaStream_t st);

@@ -100,10 +100,11 @@ __global__ void __launch_bounds__(kThreads) walk_kernel(WalkArgs w) {
     const int g = blockIdx.x % w.n_groups;
     const int bh = blockIdx.x / w.n_groups;
     const int b = bh / w.H, h = bh % w.H;
-    const int lo = g * w.group;
-    const int hi = min(w.N, lo + w.group);
+    // (a packed batch: the rows of sequence b, one group)
+    const int lo = w.cu_seqlens ? w.cu_seqlens[b] : g * w.group;
+    const int hi = w.cu_seqlens ? w.cu_seqlens[b + 1] : min(w.N, lo + w.group);
     // (the launcher has resolved the layouts: strides are never all zero here)
-    auto slice = [&](const RowLayout& l) { return (size_t)b * l.sb + (size_t)h * l.sh; };
+    auto slice = [&](const RowLayout& l) { return (w.cu_seqlens ? (size_t)0 : (size_t)b * l.sb) + (size_t)h * l.sh; };
     const T* X = static_cast<const T*>(w.x) + slice(w.lx);
     const T* A = static_cast<const T*>(w.a) + slice(w.la);
     const T* Bv = static_cast<const T*>(w.bv) + slice(w.lbv);
@@ -111,7 +112,8 @@ __global__ void __launch_bounds__(kThreads) walk_kernel(WalkArgs w) {
     T* O = w.out ? static_cast<T*>(w.out) + slice(w.lout) : nullptr;
 
     const float s_b = w.seq_len ? w.seq_len[b]
-                                : (w.seq_len_scalar > 0.f ? w.seq_len_scalar : (float)w.N);
+                                : (w.seq_len_scalar > 0.f ? w.seq_len_scalar
+                                                          : (float)(w.cu_seqlens ? max(hi - lo, 1) : w.N));
     const float c = stab_factor(w.m[h], s_b);
 
     const int col = tid % D, split = tid / D, a0 = split * AR;
@@ -294,13 +296,15 @@ __global__ void __launch_bounds__(256) scan_kernel(float* __restrict__ states,
 // Fixed summation order (deterministic).
 __global__ void dm_finalize_kernel(const float* dm_partial, float* dm, const float* m,
                                    const float* seq_len, float seq_len_scalar, int B, int H,
-                                   int n_groups, int N) {
+                                   int n_groups, int N, const int* cu_seqlens) {
     const int h = blockIdx.x * blockDim.x + threadIdx.x;
     if (h >= H) return;
     const float sg = 1.0f / (1.0f + expf(-m[h]));
     float total = 0.f;
     for (int b = 0; b < B; ++b) {
-        const float s_b = seq_len ? seq_len[b] : (seq_len_scalar > 0.f ? seq_len_scalar : (float)N);
+        const float s_b = seq_len ? seq_len[b]
+                                  : (seq_len_scalar > 0.f ? seq_len_scalar
+                                                          : (float)(cu_seqlens ? max(cu_seqlens[b + 1] - cu_seqlens[b], 1) : N));
         const float ls = logf(s_b);
         const float c = expf(-sg * ls);
         float acc = 0.f;
@@ -442,9 +446,9 @@ cudaError_t launch_sum_slices(const float* parts, float* out, int n, int H, cuda
 
 cudaError_t launch_dm_finalize(const float* dm_partial, float* dm, const float* m,
                                const float* seq_len, float seq_len_scalar, int B, int H,
-                               int n_groups, int N, cudaStream_t st) {
+                               int n_groups, int N, cudaStream_t st, const int* cu_seqlens) {
     dm_finalize_kernel<<<(H + 127) / 128, 128, 0, st>>>(dm_partial, dm, m, seq_len,
-                                                        seq_len_scalar, B, H, n_groups, N);
+                                                        seq_len_scalar, B, H, n_groups, N, cu_seqlens);
     note_launch();
     return cudaGetLastError();
 }

@@ -116,7 +116,7 @@ def test_strided_and_packed_entry_points_validate_on_the_host():
     # packed batches: NULL cu_seqlens, fp32 or rows that are not multiples of 16 bytes (tensor-core path only), max_seqlen > total
     v = (a, a, a, a + 65536)
     assert lib.cott_fwd_varlen(*v, null, 2, 2, 100, 60, 64, 1, cott.BF16, *tail) == -1
-    assert lib.cott_fwd_varlen(*v, a, 2, 2, 100, 60, 64, 1, cott.F32, *tail) == -2
+    assert lib.cott_fwd_varlen(*v, a, 2, 2, 100, 60, 96, 1, cott.F32, *tail) == -2          # fp32: 32, 64, 128 only
     assert lib.cott_fwd_varlen(*v, a, 2, 2, 100, 60, 36, 1, cott.BF16, *tail) == -2
     assert lib.cott_fwd_varlen(*v, a, 2, 2, 100, 200, 64, 1, cott.BF16, *tail) == -2
     assert lib.cott_fwd_varlen(*v, a, 2, 2, 100, 60, 64, 1, cott.BF16, ctypes.byref(sp), null, 0, null) == -3

@@ -1081,6 +1081,32 @@ def test_packed_varlen_matches_per_sequence_definition(d, causal, lens):
     gate_dm(dm, dm_ref, 1e-2, conds, DM_COND_BF16)
 
 
+@pytest.mark.parametrize("causal", [True, False])
+def test_packed_varlen_fp32(causal):
+    """fp32 I/O of a packed batch (the fp32-accumulating SIMT kernels, d = 32): every sequence
+    against the definition evaluated on it alone at the fp32 gate; neighbours' rows untouched."""
+    H, d, lens = 3, 32, (70, 1, 16, 33)
+    seqs = [synth.make_qkv(1, H, L, d, torch.float32, 5900 + 7 * i + L, with_do=True) for i, L in enumerate(lens)]
+    m_np = seqs[0]["m"]
+    cat = lambda key: torch.cat([s[key][0].permute(1, 0, 2) for s in seqs], dim=0).contiguous().cuda()
+    q, k, v, d_o = (cat(x) for x in ("q", "k", "v", "d_o"))
+    cu = torch.tensor(np.concatenate([[0], np.cumsum(lens)]), dtype=torch.int32, device="cuda")
+    m = dev(m_np)
+    o = cott.fwd_varlen(q, k, v, m, cu, max(lens), causal=causal)
+    dq, dk, dv, dm = cott.bwd_varlen(q, k, v, d_o, m, cu, max(lens), causal=causal)
+    dm_ref, conds, off = np.zeros(H), np.zeros(H), 0
+    for s, L in zip(seqs, lens):
+        ref = oracle.fwd_quadratic(s["q"], s["k"], s["v"], m_np, None, causal)
+        rq, rk, rv, rm = oracle.bwd_quadratic(s["q"], s["k"], s["v"], s["d_o"], m_np, None, causal)
+        unpack = lambda x: x[off:off + L].permute(1, 0, 2)[None]
+        gate(unpack(o), ref, torch.float32)
+        gate(unpack(dq), rq, torch.float32); gate(unpack(dk), rk, torch.float32); gate(unpack(dv), rv, torch.float32)
+        dm_ref += rm
+        conds += dm_condition(rv, s["v"], m_np, None)
+        off += L
+    gate_dm(dm, dm_ref, 1e-4, conds, DM_COND_F32)
+
+
 def test_packed_varlen_leaves_neighbours_alone():
     """The ragged end of a sequence shares a 128-row tile with the start of the next one: after a
     forward into a buffer filled with a marker, exactly the rows of the batch are written."""
