@@ -766,7 +766,8 @@ def test_token_blocks_on_a_state(T, dk, dv, option):
     CTAs per SM, the state read and written once): prefill 200 tokens, then three blocks of T
     tokens; rows and the final [d_key, d_value] state against one long causal forward by the
     definition; more (b, h) pairs than fit on the GPU at once."""
-    B, H, N0 = 5, 40, 200
+    # (d = 128: more than two pairs per SM, which takes the persistent form of the kernel)
+    B, H, N0 = (10 if dk == 128 else 5), 40, 200
     N = N0 + 3 * T
     c = synth.make_qkv(B, H, N, dk, torch.bfloat16, 6700 + T + dk, d_v=dv)
     s = np.full((B,), float(N))
@@ -783,7 +784,7 @@ def test_token_blocks_on_a_state(T, dk, dv, option):
         assert kinds == [6]
         rows.append(o)
     # a sample of (b, h) pairs through the oracle (the whole batch would take a minute)
-    pick = [(0, 0), (2, 17), (4, 39)]
+    pick = [(0, 0), (2, 17), (4, 39), (B - 1, 38)]
     sub = {x: np.stack([c[x][b_, h_].float().numpy() for b_, h_ in pick])[None] for x in ("q", "k", "v")}
     msub = np.array([float(c["m"][h_]) for _, h_ in pick])
     ref = oracle.fwd_quadratic(sub["q"], sub["k"], sub["v"], msub, np.array([float(N)]), True)[0]
