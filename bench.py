@@ -390,7 +390,9 @@ def run_ours(args, w):
         if w["bwd"]:
             ws_b = torch.empty(cott.workspace_bytes(cott.cott.OP_BWD, dt_code, B, H, N, d, w["causal"]),
                                dtype=torch.uint8, device=dev)
-            bwd_call = lambda: cott.bwd(q, k, v, d_o, m, causal=w["causal"], workspace=ws_b)
+            # (a training step: the backward is given the forward call's workspace, whose partial
+            # states it reuses where the plan has any)
+            bwd_call = lambda: cott.bwd(q, k, v, d_o, m, causal=w["causal"], workspace=ws_b, fwd_workspace=ws_f)
         tokens_per_step = B * N
 
     def barrier():

@@ -278,6 +278,23 @@ cott_status cott_decode_step(const void* q, const void* k, const void* v, float*
                              void* stream);
 
 /*
+ * cott_bwd_strided for a training step: `fwd_workspace` is the workspace the cott_fwd /
+ * cott_fwd_strided call on the SAME q, k, v, scale parameters and options used (with
+ * state_out == NULL), not overwritten since.  Where that call left the per-group partial states
+ * K^^T V there (the causal tensor-core path at d <= 64 with two to eight groups), the backward
+ * reads them instead of streaming k and v once more for its own; everywhere else the pointer is
+ * ignored and the call is cott_bwd_strided.  The library cannot check that the workspace belongs
+ * to these tensors: passing another one gives wrong gradients, not an error.  NULL is allowed.
+ * It must not be the backward's own workspace.
+ */
+cott_status cott_bwd_after_fwd(const void* q, const void* k, const void* v, const void* d_o, void* dq,
+                               void* dk, void* dv, float* dm, int B, int H, int N, int d, int causal,
+                               cott_dtype dt, const cott_strides* qkv_strides,
+                               const cott_strides* do_strides, const cott_strides* dqkv_strides,
+                               const cott_scale_params* sp, const void* fwd_workspace, void* workspace,
+                               size_t workspace_bytes, void* stream);
+
+/*
  * Head sizes.  The paper's section 2.1 gives keys / queries and values sizes of their own
  * (d_H_key, d_H_value); every call above takes one `d` for both.  The *_dkdv calls below take
  * the two separately:

@@ -84,6 +84,9 @@ def _load():
     lib.cott_bwd_strided.restype = ci
     lib.cott_bwd_strided.argtypes = [vp] * 8 + [ci, ci, ci, ci, ci, ci, vp, vp, vp,
                                                  ctypes.POINTER(_ScaleParams), vp, cs, vp]
+    lib.cott_bwd_after_fwd.restype = ci
+    lib.cott_bwd_after_fwd.argtypes = [vp] * 8 + [ci, ci, ci, ci, ci, ci, vp, vp, vp,
+                                                   ctypes.POINTER(_ScaleParams), vp, vp, cs, vp]
     lib.cott_fwd_varlen.restype = ci
     lib.cott_fwd_varlen.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci,
                                     ctypes.POINTER(_ScaleParams), vp, cs, vp]
@@ -364,8 +367,10 @@ def fwd_noalloc(q, k, v, m, seq_len=None, causal=True, out=None, stream=None):
 
 
 @_on_call_stream
-def bwd(q, k, v, d_o, m, seq_len=None, causal=True, workspace=None, stream=None, out=None):
-    """cott_bwd / cott_bwd_strided.  q, k, v (common strides) and d_o as for ``fwd``; ``out``:
+def bwd(q, k, v, d_o, m, seq_len=None, causal=True, workspace=None, stream=None, out=None, fwd_workspace=None):
+    """cott_bwd / cott_bwd_strided; with ``fwd_workspace`` (the workspace tensor the forward call
+    on the same q, k, v used, untouched since) cott_bwd_after_fwd, which reuses what that call
+    left there.  q, k, v (common strides) and d_o as for ``fwd``; ``out``:
     optional ``(dq, dk, dv)`` tensors with common strides (e.g. the slices of a fused gradient
     buffer), else they are allocated like q.  Returns ``(dq, dk, dv, dm[H] fp32)``."""
     _check_rows(q, k, v, d_o)
@@ -394,6 +399,15 @@ def bwd(q, k, v, d_o, m, seq_len=None, causal=True, workspace=None, stream=None,
     dm = torch.empty((H,), dtype=torch.float32, device=q.device)
     ws, ws_bytes = _workspace(OP_BWD, dt, B, H, N, d, causal, q.device, workspace)
     sp = _scale(m, seq_len)
+    if fwd_workspace is not None:
+        rc = _load().cott_bwd_after_fwd(q.data_ptr(), k.data_ptr(), v.data_ptr(), d_o.data_ptr(),
+                                        dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), dm.data_ptr(), B, H, N,
+                                        d, int(bool(causal)), dt, _ref(s_qkv), _ref(s_do), _ref(s_dqkv),
+                                        ctypes.byref(sp), fwd_workspace.data_ptr(), ws.data_ptr(), ws_bytes,
+                                        _stream_ptr(stream))
+        if rc != 0:
+            raise CottError(rc, "cott_bwd_after_fwd")
+        return dq, dk, dv, dm
     rc = _load().cott_bwd_strided(q.data_ptr(), k.data_ptr(), v.data_ptr(), d_o.data_ptr(),
                                   dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), dm.data_ptr(), B, H, N,
                                   d, int(bool(causal)), dt, _ref(s_qkv), _ref(s_do), _ref(s_dqkv),

@@ -527,7 +527,7 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
                             cudaStream_t st, const cott_strides* s_qkv = nullptr,
                             const cott_strides* s_do = nullptr, const cott_strides* s_dqkv = nullptr,
                             Packed packed = Packed(), const cott_strides* s_v = nullptr,
-                            const cott_strides* s_dv = nullptr) {
+                            const cott_strides* s_dv = nullptr, const void* fwd_ws = nullptr) {
     // (d is the size the kernels run at, p.d; the tensors have p.dk and p.dv columns)
     CallLayouts lay{to_layout(s_qkv), to_layout(s_do), to_layout(s_dqkv), q, k, v, d_o};
     lay.dk = p.dk; lay.dv = p.dv; lay.dv_ptr = dv;
@@ -569,6 +569,13 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
             f.m = sp->m; f.seq_len = sp->seq_len; f.seq_len_scalar = sp->seq_len_scalar;
             f.group = p.group; f.n_groups = p.n_groups;
             f.bidir = causal ? 0 : 1;
+            // The forward call of the same q, k, v (no state in or out) left the partial states
+            // K^^T V of every group but the last in its workspace whenever its walk summed them
+            // itself: the transposes of what this walk needs, so the state pass skips k and v.
+            if (fwd_ws && causal && p.n_groups >= 2 && p.n_groups <= 8 && fused_scan_ok(p.n_groups, d, p.group)) {
+                f.sq_fwd = reinterpret_cast<const float*>(static_cast<const char*>(fwd_ws) + kWsHeaderBytes);
+                f.sq_fwd_split = p.split;
+            }
             if (causal && p.n_groups == 1 && N <= 128) {
                 // One chunk per (b, h): no state is ever read, the walk is the only launch.
                 f.sq_part = nullptr; f.r_part = nullptr;
@@ -878,8 +885,10 @@ static cott_status bwd_entry(const void* q, const void* k, const void* v, const 
                              const cott_strides* qk_strides, const cott_strides* v_strides,
                              const cott_strides* do_strides, const cott_strides* dqk_strides,
                              const cott_strides* dv_strides, const cott_scale_params* sp, void* workspace,
-                             size_t workspace_bytes, void* stream) {
+                             size_t workspace_bytes, void* stream, const void* fwd_workspace = nullptr) {
     if (!q || !k || !v || !d_o || !dq || !dk || !dv || !dm || B < 1 || H < 1 || N < 1 || d_k < 1 || d_v < 1)
+        return COTT_ERR_INVALID_ARG;
+    if (fwd_workspace && (fwd_workspace == workspace || (reinterpret_cast<uintptr_t>(fwd_workspace) & 255u)))
         return COTT_ERR_INVALID_ARG;
     const bool same = d_k == d_v;
     const cott_strides* vs = v_strides ? v_strides : (same ? qk_strides : nullptr);
@@ -915,7 +924,17 @@ static cott_status bwd_entry(const void* q, const void* k, const void* v, const 
     const bool own_v = !same || v_strides || dv_strides;
     return bwd_impl(q, k, v, d_o, dq, dk, dv, dm, B, H, N, p.d, causal, dt, sp, workspace, p,
                     static_cast<cudaStream_t>(stream), qk_strides, do_strides, dqk_strides, Packed(),
-                    own_v ? vs : nullptr, own_v ? dvs : nullptr);
+                    own_v ? vs : nullptr, own_v ? dvs : nullptr, fwd_workspace);
+}
+
+cott_status cott_bwd_after_fwd(const void* q, const void* k, const void* v, const void* d_o, void* dq,
+                               void* dk, void* dv, float* dm, int B, int H, int N, int d, int causal,
+                               cott_dtype dt, const cott_strides* qkv_strides,
+                               const cott_strides* do_strides, const cott_strides* dqkv_strides,
+                               const cott_scale_params* sp, const void* fwd_workspace, void* workspace,
+                               size_t workspace_bytes, void* stream) {
+    return bwd_entry(q, k, v, d_o, dq, dk, dv, dm, B, H, N, d, d, causal, dt, qkv_strides, nullptr, do_strides,
+                     dqkv_strides, nullptr, sp, workspace, workspace_bytes, stream, fwd_workspace);
 }
 
 cott_status cott_bwd(const void* q, const void* k, const void* v, const void* d_o, void* dq,

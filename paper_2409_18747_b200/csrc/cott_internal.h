@@ -130,6 +130,10 @@ struct TcBwdFusedArgs {
     const float* m; const float* seq_len; float seq_len_scalar;
     int group; int n_groups;
     int plain_launch;
+    // Causal walk: the partial states K^^T V the forward call of the same q, k, v left in its
+    // workspace ([BH, n_groups * sq_fwd_split, 64 * 64], unscaled; every group but the last): read
+    // transposed instead of sq_part, which the state pass then does not compute.  NULL: none.
+    const float* sq_fwd; int sq_fwd_split;
     int bidir;      // 1: all-ones mask (bidirectional backward): both states are totals over the sequence
     int w_k, w_v;   // real columns of q, k, dq, dk and of v, dO, dv when fewer than 64 (0: 64)
 };

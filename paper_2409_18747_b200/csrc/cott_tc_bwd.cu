@@ -78,6 +78,8 @@ struct BwdParams {
     int wait_limit_kcycles;
     int head_first_mask;     // bit i: in tensor map i (q, k, v, dO, dq, dk, dv) the head index comes before the token index
     int no_state;            // the whole sequence is one chunk: both states are zero wherever they are read, no update
+    const float* sq_fwd;     // the forward call's partial states K^^T V ([BH, n_groups * split, 64 * 64]) or NULL
+    int sq_fwd_split;
 };
 
 
@@ -308,7 +310,17 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             const float* src = upper ? p.sq_part : p.r_part;
             const int g_lo = BIDIR ? 0 : (upper ? 0 : g), g_hi = BIDIR ? p.n_groups : (upper ? g : p.n_groups);
             const size_t off = (size_t)(row & 63) * kD + (size_t)(wg & 1) * 32;
-            if (src != nullptr) {
+            if (!BIDIR && upper && p.sq_fwd != nullptr) {
+                // V^T K^ of the groups before this one is the transpose of what the forward call
+                // left: element (row, col) of Sq is element (col, row) of K^^T V.
+                const int parts = g * p.sq_fwd_split;
+                const float* sf = p.sq_fwd + (size_t)bh * p.n_groups * p.sq_fwd_split * kD * kD + (size_t)(wg & 1) * 32 * kD + (row & 63);
+                for (int pp = 0; pp < parts; ++pp) {
+                    const float* sg = sf + (size_t)pp * kD * kD;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) acc[i] += __ldg(sg + (size_t)i * kD);
+                }
+            } else if (src != nullptr) {
                 for (int gg = g_lo; gg < g_hi; ++gg) {
                     const float* sg = src + ((size_t)bh * p.n_groups + gg) * kD * kD + off;
 #pragma unroll
@@ -852,6 +864,7 @@ struct StateParams {
     int wait_limit_kcycles;
     int head_first_mask;     // bit i: in tensor map i (q, k, v, dO) the head index comes before the token index
     int all_sq;              // bidirectional backward: V^T K^ of the last group is read too
+    int no_sq;               // V^T K^ comes from the forward call's workspace: no group loads k and v
 };
 
 __global__ void __launch_bounds__(kStThreads, 1)
@@ -876,7 +889,7 @@ tc_bwd_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const bool is_mma = warp == 8, is_copy = warp == 9;
     // Nobody reads V^T K^ of the last group: its CTA leaves the v and k slots at zero (the product
     // then adds nothing to that block) and loads q and dO only.
-    const bool need_sq = p.all_sq || g + 1 < p.n_groups;
+    const bool need_sq = !p.no_sq && (p.all_sq || g + 1 < p.n_groups);
 
     if (is_mma) {
         tmem_alloc(tmem_slot, 128);
@@ -1040,6 +1053,7 @@ cudaError_t launch_tc_bwd_fused(const TcBwdFusedArgs& a, int B, int H, int N, cu
     p.status = a.status; p.m = a.m; p.seq_len = a.seq_len; p.seq_len_scalar = a.seq_len_scalar;
     p.H = H; p.N = N; p.group = a.group; p.n_groups = a.n_groups;
     p.wait_limit_kcycles = wait_limit_kcycles();
+    p.sq_fwd = a.bidir ? nullptr : a.sq_fwd; p.sq_fwd_split = a.sq_fwd_split > 0 ? a.sq_fwd_split : 1;
     // One chunk per (b, h): nothing precedes it (Sq = 0) and nothing follows it (R = 0 once its own
     // update is taken out again), so the states stay zero and no partial-state pass is needed.
     p.no_state = (!a.bidir && a.n_groups == 1 && N <= kC && !a.sq_part && !a.r_part) ? 1 : 0;
@@ -1083,6 +1097,7 @@ cudaError_t launch_tc_bwd_states(const TcBwdFusedArgs& a, float* sq_out, float* 
     p.H = H; p.N = N; p.group = a.group; p.n_groups = a.n_groups;
     p.clear_status = clear_status;
     p.all_sq = a.bidir;
+    p.no_sq = (!a.bidir && a.sq_fwd != nullptr) ? 1 : 0;
     p.wait_limit_kcycles = wait_limit_kcycles();
     constexpr int kBytes = kStStages * L::kStage + L::kCtlBytes + 1024;
     static_assert(kStStages * L::kStage <= L::kOffCtl, "the stage ring overlaps the control block");

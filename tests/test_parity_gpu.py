@@ -529,6 +529,29 @@ def test_profile_and_status_words():
     assert cott.cott.profile_read() == []                  # disabled
 
 
+@pytest.mark.parametrize("B,H,N", [(2, 20, 1024), (4, 16, 1000), (1, 64, 2048)])
+def test_backward_reuses_the_forward_calls_partial_states(B, H, N):
+    """A training step: the causal forward leaves the per-group partial states K^^T V in its
+    workspace, and cott_bwd_after_fwd reads them (transposed) instead of streaming k and v once
+    more.  Gradients against the definition, and against the plain backward call."""
+    c = synth.make_qkv(B, H, N, 64, torch.bfloat16, 4700 + N + H, with_do=True)
+    q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
+    plan = cott.cott.query_plan(cott.cott.OP_BWD, cott.cott.BF16, B, H, N, 64, True)
+    assert plan["group"] < N                                  # several groups per (b, h)
+    ws_f = torch.zeros(cott.workspace_bytes(cott.cott.OP_FWD, cott.cott.BF16, B, H, N, 64, True), dtype=torch.uint8, device="cuda")
+    o = cott.fwd(q, k, v, m, causal=True, workspace=ws_f)
+    gate(o, oracle.fwd_quadratic(c["q"], c["k"], c["v"], c["m"], None, True), torch.bfloat16)
+    n0 = cott.cott.launch_count()
+    got = cott.bwd(q, k, v, d_o, m, causal=True, fwd_workspace=ws_f)
+    assert cott.cott.launch_count() - n0 == 2                # state pass (q, dO only) + walk
+    rq, rk, rv, rm = oracle.bwd_quadratic(c["q"], c["k"], c["v"], c["d_o"], c["m"], None, True)
+    gate(got[0], rq, torch.bfloat16); gate(got[1], rk, torch.bfloat16); gate(got[2], rv, torch.bfloat16)
+    gate_dm(got[3], rm, 1e-2, dm_condition(rv, c["v"], c["m"], None), DM_COND_BF16)
+    plain = cott.bwd(q, k, v, d_o, m, causal=True)
+    for a, b in zip(got[:3], plain[:3]):
+        assert norm_max_err(a, b.double().cpu().numpy()) <= TOL_BF16  # the same sums in another order, each rounded to bf16 once
+
+
 def test_side_by_side_backward_matches_one_after_the_other(option):
     """B*H = 64: the dQ and dK streams run side by side, each over the whole sequence.  Same
     gradients (up to the rounding of a different grouping) as the three streams in sequence,
