@@ -381,7 +381,17 @@ static cott_status run_tc_stream(TcWalkArgs t, const Plan& p, int B, int H, int 
             a.grid_groups = (p.n_groups - 1) * split;
             a.first_group = t.reverse ? split : 0;
         }
-        COTT_CUDA(launch_tc_walk(a, B, H, N, d, st));
+        // The forward's pass at d = 64 (k normalised, v raw, forward in time) has a lighter kernel
+        // of its own: stages of two tiles, a ring twice as deep.
+        const bool light = d == 64 && !t.cu_seqlens && t.epilogue == EPI_PLAIN && t.x_norm && !t.norm_bv && !t.reverse &&
+                           option_fused_bwd() != 0;
+        if (light) {
+            COTT_CUDA(launch_tc_pair_states(a.a, a.bv, a.la, a.lbv, a.d_xa > 0 ? a.d_xa : d, a.d_bo > 0 ? a.d_bo : d, states,
+                                            status, a.clear_status, B, H, N, a.group, a.n_groups,
+                                            a.grid_groups > 0 ? a.grid_groups : a.n_groups, a.plain_launch, st));
+        } else {
+            COTT_CUDA(launch_tc_walk(a, B, H, N, d, st));
+        }
         const int mode = !causal ? SCAN_TOTAL : (t.reverse ? SCAN_SUFFIX : SCAN_PREFIX);
         if (!fused_scan)
             COTT_CUDA(launch_scan(states, total_out, B * H, p.n_groups, d, mode, st, sp->m, sp->seq_len,

@@ -143,6 +143,12 @@ cudaError_t launch_tc_bwd_fused(const TcBwdFusedArgs& a, int B, int H, int N, cu
 cudaError_t launch_tc_bwd_states(const TcBwdFusedArgs& a, float* sq_out, float* r_out, int clear_status, int B, int H,
                                  int N, cudaStream_t st);
 
+// Partial states A^^T B (A's rows normalised) of the first grid_groups groups of every (b, h) at
+// d <= 64, written to out[(bh * n_groups + g) * 64 * 64] (cott_tc_bwd.cu).
+cudaError_t launch_tc_pair_states(const void* a_rows, const void* b_rows, const RowLayout& l_a, const RowLayout& l_b,
+                                  int w_a, int w_b, float* out, int* status, int clear_status, int B, int H, int N,
+                                  int group, int n_groups, int grid_groups, int plain_launch, cudaStream_t st);
+
 // Bidirectional forward at d = 64 in one launch, one CTA per (b, h) (cott_tc_bidir.cu); it is
 // the first (and only) kernel of its call and clears the status words itself.
 cudaError_t launch_tc_bidir_fwd(const void* q, const void* k, const void* v, void* o, const RowLayout& l_qkv,

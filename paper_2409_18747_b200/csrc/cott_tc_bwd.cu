@@ -854,6 +854,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 // last to first, so that the tiles still in L2 afterwards are the ones the walk asks for first.
 constexpr int kStThreads = 10 * 32;
 constexpr int kStStages = 3;
+constexpr int kStStagesR = 6;       // when only Q^^T dO is needed: stages of two tiles, twice as many
 
 struct StateParams {
     float* sq_out;           // [BH, n_groups, 64 * 64]
@@ -865,8 +866,13 @@ struct StateParams {
     int head_first_mask;     // bit i: in tensor map i (q, k, v, dO) the head index comes before the token index
     int all_sq;              // bidirectional backward: V^T K^ of the last group is read too
     int no_sq;               // V^T K^ comes from the forward call's workspace: no group loads k and v
+    int grid_groups;         // groups 0 .. grid_groups - 1 of every (b, h) are computed (a causal forward never reads the last one's)
 };
 
+// RONLY: no group needs V^T K^ (the forward call's partial states serve): a stage holds q and dO
+// only, the product is the 64 x 64 Q^^T dO (rows 16 i .. 16 i + 15 of the result sit in lanes
+// 32 i .. 32 i + 15 of the accumulator), and the ring is twice as deep.
+template <bool RONLY>
 __global__ void __launch_bounds__(kStThreads, 1)
 tc_bwd_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                     const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmDO, StateParams p) {
@@ -874,29 +880,32 @@ tc_bwd_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* gbase = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t bars = base + L::kOffCtl;
-    enum { S_FULL = 0, S_NREADY = 32, S_UFULL = 64 };          // rings of three, indexed by chunk % 3
-    auto bar = [&](int which, int c) { return bars + which + 8 * (c % kStStages); };
-    auto par = [&](int c) { return (uint32_t)((c / kStStages) & 1); };
+    constexpr int NS = RONLY ? kStStagesR : kStStages;
+    constexpr uint32_t kSt = RONLY ? 2u * kTile : (uint32_t)L::kStage;     // bytes of a stage
+    constexpr uint32_t oQ = RONLY ? 0u : (uint32_t)L::kOffQ, oDO = RONLY ? (uint32_t)kTile : (uint32_t)L::kOffDO;
+    enum { S_FULL = 0, S_NREADY = 64, S_UFULL = 128 };         // rings of NS, indexed by chunk % NS
+    auto bar = [&](int which, int c) { return bars + which + 8 * (c % NS); };
+    auto par = [&](int c) { return (uint32_t)((c / NS) & 1); };
     const uint32_t tmem_slot = bars + L::kOffTmemSlot;
     volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(gbase + L::kOffCtl + L::kOffTmemSlot);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + L::kOffCtl + L::kOffAbort);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int g = blockIdx.x % p.n_groups, bh = blockIdx.x / p.n_groups;
+    const int g = blockIdx.x % p.grid_groups, bh = blockIdx.x / p.grid_groups;
     const int b = bh / p.H, h = bh % p.H;
     const int tok0 = g * p.group, tok1 = min(p.N, tok0 + p.group);
     const int n_chunks = (tok1 - tok0 + kC - 1) / kC;
     const bool is_mma = warp == 8, is_copy = warp == 9;
     // Nobody reads V^T K^ of the last group: its CTA leaves the v and k slots at zero (the product
     // then adds nothing to that block) and loads q and dO only.
-    const bool need_sq = !p.no_sq && (p.all_sq || g + 1 < p.n_groups);
+    const bool need_sq = !RONLY && !p.no_sq && (p.all_sq || g + 1 < p.n_groups);
 
     if (is_mma) {
         tmem_alloc(tmem_slot, 128);
         tmem_relinquish();
     }
     if (tid == 0) {
-        for (int i = 0; i < kStStages; ++i) {
+        for (int i = 0; i < NS; ++i) {
             mbar_init(bars + S_FULL + 8 * i, 1);
             mbar_init(bars + S_NREADY + 8 * i, 256);
             mbar_init(bars + S_UFULL + 8 * i, 1);
@@ -913,7 +922,7 @@ tc_bwd_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot_g;
-    auto stage = [&](int c) { return base + (uint32_t)(c % kStStages) * L::kStage; };
+    auto stage = [&](int c) { return base + (uint32_t)(c % NS) * kSt; };
     auto issue_loads = [&](int c) {
         const uint32_t fb = bar(S_FULL, c), st = stage(c);
         const int row = tok0 + (n_chunks - 1 - c) * kC;
@@ -922,11 +931,11 @@ tc_bwd_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             const bool hf = (p.head_first_mask >> which) & 1;
             tma_load_4d(dst, tm, fb, 0, hf ? h : row, hf ? row : h, b);
         };
-        load(st + L::kOffQ, &tmQ, 0);
-        load(st + L::kOffDO, &tmDO, 3);
+        load(st + oQ, &tmQ, 0);
+        load(st + oDO, &tmDO, 3);
         if (need_sq) { load(st + L::kOffK, &tmK, 1); load(st + L::kOffV, &tmV, 2); }
     };
-    if (!need_sq) {
+    if (!RONLY && !need_sq) {
         for (int i = tid; i < kStStages * 2 * (kTile / 16); i += kStThreads) {
             const int s3 = i / (2 * (kTile / 16)), r2 = i % (2 * (kTile / 16));
             const int off = s3 * L::kStage + (r2 < kTile / 16 ? L::kOffV : L::kOffK) + (r2 % (kTile / 16)) * 16;
@@ -942,11 +951,11 @@ tc_bwd_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 
     if (is_copy) {
         if (lane == 0) {
-            for (int c = 0; c < kStStages && c < n_chunks; ++c) { issue_loads(c); SSTAMP(2, c, 0); }
-            for (int c = 0; c + kStStages < n_chunks; ++c) {
+            for (int c = 0; c < NS && c < n_chunks; ++c) { issue_loads(c); SSTAMP(2, c, 0); }
+            for (int c = 0; c + NS < n_chunks; ++c) {
                 if (!wait_or_abort(bar(S_UFULL, c), par(c), abort_flag)) break;
-                issue_loads(c + kStStages);
-                SSTAMP(2, c + kStStages, 0);
+                issue_loads(c + NS);
+                SSTAMP(2, c + NS, 0);
             }
         }
     } else if (is_mma) {
@@ -956,8 +965,9 @@ tc_bwd_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 if (!wait_or_abort(bar(S_NREADY, c), par(c), abort_flag)) break;
                 SSTAMP(1, c, 0);
                 tc_fence_after();
-                constexpr uint32_t idesc = instr_desc_bf16(128, 128, true, true);
-                const uint32_t al = smem_desc_lo(st + L::kOffV, 16384), bl = smem_desc_lo(st + L::kOffK, 16384);
+                constexpr uint32_t idesc = RONLY ? instr_desc_bf16(64, 64, true, true) : instr_desc_bf16(128, 128, true, true);
+                const uint32_t al = smem_desc_lo(st + (RONLY ? oQ : (uint32_t)L::kOffV), 16384);
+                const uint32_t bl = smem_desc_lo(st + (RONLY ? oDO : (uint32_t)L::kOffK), 16384);
 #pragma unroll
                 for (int kk = 0; kk < kC / 16; ++kk)
                     mma_ss_w(tmem, al + kk * 128u, kDescHi, bl + kk * 128u, kDescHi, idesc, (c > 0 || kk > 0) ? 1u : 0u);
@@ -973,7 +983,7 @@ tc_bwd_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             if (!wait_or_abort(bar(S_FULL, c), par(c), abort_flag)) { alive = false; break; }
             SSTAMP(0, c, 1);
             if (hw == 1 && !need_sq) { mbar_arrive(bar(S_NREADY, c)); continue; }
-            uint8_t* tile = gbase + (c % kStStages) * L::kStage + (hw == 0 ? L::kOffQ : L::kOffK);
+            uint8_t* tile = gbase + (c % NS) * kSt + (hw == 0 ? oQ : (uint32_t)L::kOffK);
             uint4 w[8];
             float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
@@ -1010,13 +1020,17 @@ tc_bwd_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             tc_fence_after();
             const bool upper = row < 64;
             uint32_t r[32];
-            tmem_ld32(tmem + ((uint32_t)(q4 * 32) << 16) + (upper ? 0 : 64) + hw * 32, r);
+            tmem_ld32(tmem + ((uint32_t)(q4 * 32) << 16) + (RONLY ? 0 : (upper ? 0 : 64)) + hw * 32, r);
             tmem_wait_ld();
-            float* dst = (upper ? p.sq_out : p.r_out) + ((size_t)bh * p.n_groups + g) * kD * kD + (size_t)(row & 63) * kD + hw * 32;
+            // (the 64-row accumulator: lanes 0-15 of every quadrant hold rows 16 q4 .. 16 q4 + 15)
+            const int orow = RONLY ? q4 * 16 + (lane & 15) : (row & 63);
+            float* dst = ((upper && !RONLY) ? p.sq_out : p.r_out) + ((size_t)bh * p.n_groups + g) * kD * kD + (size_t)orow * kD + hw * 32;
+            if (!RONLY || lane < 16) {
 #pragma unroll
-            for (int i = 0; i < 32; i += 4)
-                *reinterpret_cast<float4*>(dst + i) = make_float4(__uint_as_float(r[i]), __uint_as_float(r[i + 1]),
-                                                                   __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+                for (int i = 0; i < 32; i += 4)
+                    *reinterpret_cast<float4*>(dst + i) = make_float4(__uint_as_float(r[i]), __uint_as_float(r[i + 1]),
+                                                                       __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+            }
         }
     }
     tc_fence_before();
@@ -1098,12 +1112,12 @@ cudaError_t launch_tc_bwd_states(const TcBwdFusedArgs& a, float* sq_out, float* 
     p.clear_status = clear_status;
     p.all_sq = a.bidir;
     p.no_sq = (!a.bidir && a.sq_fwd != nullptr) ? 1 : 0;
+    p.grid_groups = a.n_groups;
     p.wait_limit_kcycles = wait_limit_kcycles();
-    constexpr int kBytes = kStStages * L::kStage + L::kCtlBytes + 1024;
-    static_assert(kStStages * L::kStage <= L::kOffCtl, "the stage ring overlaps the control block");
-    if (cudaError_t e = configure_smem_once(reinterpret_cast<const void*>(tc_bwd_state_kernel), L::kOffCtl + L::kCtlBytes + 1024); e != cudaSuccess)
+    static_assert(kStStages * L::kStage <= L::kOffCtl && kStStagesR * 2 * kTile <= L::kOffCtl, "the stage ring overlaps the control block");
+    auto kern = p.no_sq ? tc_bwd_state_kernel<true> : tc_bwd_state_kernel<false>;
+    if (cudaError_t e = configure_smem_once(reinterpret_cast<const void*>(kern), L::kOffCtl + L::kCtlBytes + 1024); e != cudaSuccess)
         return e;
-    (void)kBytes;
     const int prof = profile_begin_launch(0, st);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(B * H * a.n_groups));
@@ -1115,7 +1129,48 @@ cudaError_t launch_tc_bwd_states(const TcBwdFusedArgs& a, float* sq_out, float* 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = a.plain_launch ? 0 : 1;
-    cudaError_t le = cudaLaunchKernelEx(&cfg, tc_bwd_state_kernel, tm[0], tm[1], tm[2], tm[3], p);
+    cudaError_t le = cudaLaunchKernelEx(&cfg, kern, tm[0], tm[1], tm[2], tm[3], p);
+    profile_end_launch(prof, st);
+    note_launch();
+    return le != cudaSuccess ? le : cudaGetLastError();
+}
+
+// Partial states A^^T B of groups 0 .. grid_groups - 1 of every (b, h), A's rows normalised
+// (the forward's K^^T V): the q / dO-only instance of the kernel above on another pair of tensors.
+cudaError_t launch_tc_pair_states(const void* a_rows, const void* b_rows, const RowLayout& l_a, const RowLayout& l_b,
+                                  int w_a, int w_b, float* out, int* status, int clear_status, int B, int H, int N,
+                                  int group, int n_groups, int grid_groups, int plain_launch, cudaStream_t st) {
+    if (w_a > kD || w_b > kD || grid_groups < 1 || grid_groups > n_groups) return cudaErrorInvalidValue;
+    const void* ptrs[4] = {a_rows, a_rows, b_rows, b_rows};            // (the k and v maps are not used)
+    const RowLayout lays[4] = {l_a, l_a, l_b, l_b};
+    const int dims[4] = {w_a, w_a, w_b, w_b};
+    CUtensorMap tm[4];
+    StateParams p;
+    p.head_first_mask = 0;
+    for (int i = 0; i < 4; ++i) {
+        bool hf = false;
+        if (!make_tile_map(&tm[i], ptrs[i], B, H, N, dims[i], lays[i], &hf)) return cudaErrorInvalidValue;
+        p.head_first_mask |= (hf ? 1 : 0) << i;
+    }
+    p.sq_out = nullptr; p.r_out = out; p.status = status;
+    p.H = H; p.N = N; p.group = group; p.n_groups = n_groups; p.grid_groups = grid_groups;
+    p.clear_status = clear_status; p.all_sq = 0; p.no_sq = 1;
+    p.wait_limit_kcycles = wait_limit_kcycles();
+    auto kern = tc_bwd_state_kernel<true>;
+    if (cudaError_t e = configure_smem_once(reinterpret_cast<const void*>(kern), L::kOffCtl + L::kCtlBytes + 1024); e != cudaSuccess)
+        return e;
+    const int prof = profile_begin_launch(0, st);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(B * H * grid_groups));
+    cfg.blockDim = dim3(kStThreads);
+    cfg.dynamicSmemBytes = L::kOffCtl + L::kCtlBytes + 1024;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = plain_launch ? 0 : 1;
+    cudaError_t le = cudaLaunchKernelEx(&cfg, kern, tm[0], tm[1], tm[2], tm[3], p);
     profile_end_launch(prof, st);
     note_launch();
     return le != cudaSuccess ? le : cudaGetLastError();
