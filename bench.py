@@ -36,7 +36,7 @@ L2_FLUSH_BYTES = 256 << 20  # larger than the 126 MB L2
 # A constant from a committed capture, not a measurement of this run: the JSON line says so.
 # Missing key: no capture of that class.
 STEP_DRAM_TRAFFIC = {
-    (64, True, True): 1704.6,     # C4 step: 446.8 MB over 262 144 token-heads (method's bytes: 1408)
+    (64, True, True): 1563.3,     # C4 step: 409.8 MB over 262 144 token-heads (method's bytes: 1408)
     (64, False, False): 403.5,    # C2 forward: 79.3 MB over 196 608 token-heads (method's bytes: 512;
                                   # a third of the output is still in L2 when the kernel ends)
 }
