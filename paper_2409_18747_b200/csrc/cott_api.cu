@@ -563,7 +563,7 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
         // over the whole sequence as a single group (no partial-state pass, no scan), with the
         // dQ^ stream's partial-state pass filling the SMs that are left; the dQ^ walk follows on
         // the whole GPU.  Each side stream then carries one tensor-core kernel per call.
-        if (d == 64 && !packed.cu_seqlens && option_fused_bwd() != 0) {
+        if (d == 64 && option_fused_bwd() != 0) {
             // One walk forward in time gives all three gradients and the dm sum (cott_tc_bwd.cu).
             // It keeps two running states: Sq = V^T K^ over earlier tokens, accumulated chunk by
             // chunk, and R = Q^^T dO over later tokens, which starts at the sum over the group
@@ -579,14 +579,15 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
             f.m = sp->m; f.seq_len = sp->seq_len; f.seq_len_scalar = sp->seq_len_scalar;
             f.group = p.group; f.n_groups = p.n_groups;
             f.bidir = causal ? 0 : 1;
+            f.cu_seqlens = packed.cu_seqlens; f.total_tokens = packed.total_tokens;
             // The forward call of the same q, k, v (no state in or out) left the partial states
             // K^^T V of every group but the last in its workspace whenever its walk summed them
             // itself: the transposes of what this walk needs, so the state pass skips k and v.
-            if (fwd_ws && causal && p.n_groups >= 2 && p.n_groups <= 8 && fused_scan_ok(p.n_groups, d, p.group)) {
+            if (fwd_ws && !packed.cu_seqlens && causal && p.n_groups >= 2 && p.n_groups <= 8 && fused_scan_ok(p.n_groups, d, p.group)) {
                 f.sq_fwd = reinterpret_cast<const float*>(static_cast<const char*>(fwd_ws) + kWsHeaderBytes);
                 f.sq_fwd_split = p.split;
             }
-            if (causal && p.n_groups == 1 && N <= 128) {
+            if (causal && !packed.cu_seqlens && p.n_groups == 1 && N <= 128) {
                 // One chunk per (b, h): no state is ever read, the walk is the only launch.
                 f.sq_part = nullptr; f.r_part = nullptr;
                 COTT_CUDA(cudaMemsetAsync(ws, 0, kWsHeaderBytes, st));      // status words and the dm counter

@@ -134,6 +134,9 @@ struct TcBwdFusedArgs {
     // workspace ([BH, n_groups * sq_fwd_split, 64 * 64], unscaled; every group but the last): read
     // transposed instead of sq_part, which the state pass then does not compute.  NULL: none.
     const float* sq_fwd; int sq_fwd_split;
+    // Packed variable-length batch: B + 1 row offsets into tensors of total_tokens rows per head, one
+    // group per (sequence, head); NULL: dense batch.
+    const int* cu_seqlens; int total_tokens;
     int bidir;      // 1: all-ones mask (bidirectional backward): both states are totals over the sequence
     int w_k, w_v;   // real columns of q, k, dq, dk and of v, dO, dv when fewer than 64 (0: 64)
 };

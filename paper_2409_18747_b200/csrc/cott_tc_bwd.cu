@@ -80,6 +80,12 @@ struct BwdParams {
     int no_state;            // the whole sequence is one chunk: both states are zero wherever they are read, no update
     const float* sq_fwd;     // the forward call's partial states K^^T V ([BH, n_groups * split, 64 * 64]) or NULL
     int sq_fwd_split;
+    // Packed variable-length batch (VARLEN instances): rows of all sequences back to back, sequence
+    // b = rows cu_seqlens[b] .. cu_seqlens[b + 1] - 1, one group per (sequence, head); the rows
+    // of a ragged last chunk leave as plain stores: dq, dk, dv as global memory with their
+    // token and head strides in elements.
+    const int* cu_seqlens;
+    void* out_rows[3]; long long out_sn[3], out_sh[3]; int out_w[3];
 };
 
 
@@ -183,7 +189,7 @@ __device__ __forceinline__ void issue_update(uint32_t tS, uint32_t vq, uint32_t 
 //     dQ^ = dO S^T ,   dK^ = V R^T ,   dV' = K^ R ,
 // so the score products, the masks, the state update and the per-chunk state copies fall away;
 // loads, row norms, epilogues, stores and the dm sum are those of the causal walk.
-template <bool BIDIR>
+template <bool BIDIR, bool VARLEN>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                     const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmDO,
@@ -213,9 +219,14 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     CSTAMP(0);
     const int g = blockIdx.x % p.n_groups, bh = blockIdx.x / p.n_groups;
-    const int b = bh / p.H, h = bh % p.H;
-    const int tok0 = g * p.group, tok1 = min(p.N, tok0 + p.group);
+    const int bseq = bh / p.H, h = bh % p.H;
+    const int b = VARLEN ? 0 : bseq;                   // batch coordinate of the tensor maps
+    const int tok0 = VARLEN ? p.cu_seqlens[bseq] : g * p.group;
+    const int tok1 = VARLEN ? p.cu_seqlens[bseq + 1] : min(p.N, tok0 + p.group);
     const int n_chunks = (tok1 - tok0 + kC - 1) / kC;
+    // (a packed batch: the last chunk of a sequence may hold rows of the next one -- they are made
+    // inert by normalising them to zero, and that chunk's output rows are stored one by one)
+    const bool ragged_last = VARLEN && ((tok1 - tok0) % kC) != 0;
     auto chunk_row = [&](int c) { return tok0 + c * kC; };
     const bool is_score = warp == kWorkerWarps, is_out = warp == kWorkerWarps + 1;
     const bool is_upd = warp == kWorkerWarps + 2, is_copy = warp == kWorkerWarps + 3;
@@ -286,7 +297,8 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-    const float s_b = p.seq_len ? p.seq_len[b] : (p.seq_len_scalar > 0.f ? p.seq_len_scalar : (float)p.N);
+    const float s_b = p.seq_len ? p.seq_len[bseq]
+                                : (p.seq_len_scalar > 0.f ? p.seq_len_scalar : (float)(VARLEN ? max(tok1 - tok0, 1) : p.N));
     const float cfac = stab_factor(p.m[h], s_b);
 
     const int wg = warp >> 2, q4 = warp & 3;
@@ -329,6 +341,31 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         acc[i] += v.x; acc[i + 1] += v.y; acc[i + 2] += v.z; acc[i + 3] += v.w;
                     }
                 }
+            }
+            if (BIDIR && g == 0) {
+                // dm of the bidirectional case needs no row sums at all: sum_i <q^_i, dO_i S^T> is
+                // the element-wise product of the two totals, <S, R>, formed here in fp32 from the
+                // partial states -- none of the bf16 roundings of the walk enters it.  The upper
+                // threads hold S^T (row b, 32 columns a), the lower ones R (row a, 32 columns b):
+                // S^T crosses over through the output staging tiles (unused until the first
+                // epilogue), rows padded to 65 words so that neither side has bank conflicts.
+                float* sT = reinterpret_cast<float*>(gbase + L::kOffStQ);
+                if (upper) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) sT[row * 65 + (wg & 1) * 32 + i] = acc[i];
+                }
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                if (!upper) {
+                    float t = 0.f;
+                    const int a_ = row & 63, b0 = (wg & 1) * 32;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) t = fmaf(acc[i], sT[(b0 + i) * 65 + a_], t);
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+                    if (lane == 0) dm_red[4 + (wg & 1) * 2 + (q4 & 1)] = t;
+                }
+            } else if (BIDIR && !upper && lane == 0) {
+                dm_red[4 + (wg & 1) * 2 + (q4 & 1)] = 0.f;
             }
             if (upper || BIDIR) {
                 // Sq is what the first chunk reads before any update: its bf16 copy goes to the
@@ -375,7 +412,8 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 int c1, c2;
                 if (!wait_or_abort(bar(B_EQDONE, c), par(c), abort_flag)) break;
                 BSTAMP(7, c, 0);
-                coords(4, trow, c1, c2); tma_store_4d(&tmDQ, base + L::kOffStQ, 0, c1, c2, b);
+                const bool by_rows = ragged_last && c == n_chunks - 1;      // the workers stored this chunk's rows themselves
+                if (!by_rows) { coords(4, trow, c1, c2); tma_store_4d(&tmDQ, base + L::kOffStQ, 0, c1, c2, b); }
                 tma_store_commit();
                 tma_store_wait_read0();
                 mbar_arrive(bars + B_STQFREE);           // the tile may take the dv rows of the chunk
@@ -389,12 +427,12 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     BSTAMP(7, c, 1);
                 }
                 if (!wait_or_abort(bar(B_EKDONE, c), par(c), abort_flag)) break;
-                coords(5, trow, c1, c2); tma_store_4d(&tmDK, base + L::kOffStK, 0, c1, c2, b);
+                if (!by_rows) { coords(5, trow, c1, c2); tma_store_4d(&tmDK, base + L::kOffStK, 0, c1, c2, b); }
                 tma_store_commit();
                 if (more) { coords(1, nrow, c1, c2); tma_load_4d(st + L::kOffK, &tmK, fb, 0, c1, c2, b); }
                 BSTAMP(7, c, 2);
                 if (!wait_or_abort(bar(B_EVDONE, c), par(c), abort_flag)) break;
-                coords(6, trow, c1, c2); tma_store_4d(&tmDV, base + L::kOffStQ, 0, c1, c2, b);
+                if (!by_rows) { coords(6, trow, c1, c2); tma_store_4d(&tmDV, base + L::kOffStQ, 0, c1, c2, b); }
                 tma_store_commit();
                 tma_store_wait_read1();
                 mbar_arrive(bars + B_STKFREE);
@@ -542,7 +580,8 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     }
                 }
                 const float nrm = sqrtf((a0 + a1) + (a2 + a3));
-                const float rn = 1.0f / fmaxf(nrm, kEps);
+                float rn = 1.0f / fmaxf(nrm, kEps);
+                if (VARLEN && chunk_row(c) + row >= tok1) rn = 0.f;      // a row of the next sequence
                 // x * rn in packed bf16 arithmetic with the scale split in two bf16 terms
                 // (rn = hi + lo to 2^-17): round(x hi + round(x lo)) is x rn rounded once, up to a
                 // second rounding of the small term -- two instructions per pair of elements
@@ -550,12 +589,40 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 const __nv_bfloat16 hi = __float2bfloat16_rn(rn);
                 const __nv_bfloat16 lo = __float2bfloat16_rn(rn - __bfloat162float(hi));
                 const __nv_bfloat162 hi2 = __halves2bfloat162(hi, hi), lo2 = __halves2bfloat162(lo, lo);
+                // Bidirectional: what the rounding of x^ to bf16 drops, x rn - x^, goes to the
+                // (unused) score buffer as 7-bit fixed point, for the first-order correction of dm in
+                // the projection epilogue: units of 2^-15 (|x rn - x^| <= 2^-9 since |x^| <= 1),
+                // formed in packed bf16 arithmetic as well (x hi - x^ is a difference of close
+                // values, exact before its one rounding).  In bf16, r + 192 = 128 + (r + 64) for
+                // |r| <= 63, so the low byte of the sum is r + 64.
+                uint8_t* res = gbase + L::kOffG + (c & 1) * 16384 + hw * 8192 + row * 64;
+                const __nv_bfloat16 sc15 = __float2bfloat16_rn(32768.f);
+                const __nv_bfloat162 hi2s = __hmul2(hi2, __halves2bfloat162(sc15, sc15)), lo2s = __hmul2(lo2, __halves2bfloat162(sc15, sc15));
+                const __nv_bfloat162 nsc = __halves2bfloat162(__float2bfloat16_rn(-32768.f), __float2bfloat16_rn(-32768.f));
+                const __nv_bfloat162 c63 = __halves2bfloat162(__float2bfloat16_rn(63.f), __float2bfloat16_rn(63.f));
+                const __nv_bfloat162 c192 = __halves2bfloat162(__float2bfloat16_rn(192.f), __float2bfloat16_rn(192.f));
+                uint32_t rb[4];
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     __nv_bfloat162* e = reinterpret_cast<__nv_bfloat162*>(&w[j]);
+                    uint32_t t[4];
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) e[i] = __hfma2(e[i], hi2, __hmul2(e[i], lo2));
+                    for (int i = 0; i < 4; ++i) {
+                        const __nv_bfloat162 x = e[i];
+                        e[i] = __hfma2(x, hi2, __hmul2(x, lo2));
+                        if (BIDIR) {
+                            __nv_bfloat162 r = __hfma2(x, lo2s, __hfma2(x, hi2s, __hmul2(e[i], nsc)));
+                            r = __hadd2(__hmin2(__hmax2(r, __hneg2(c63)), c63), c192);
+                            t[i] = *reinterpret_cast<const uint32_t*>(&r);
+                        }
+                    }
                     *reinterpret_cast<uint4*>(tile + swz(row, j)) = w[j];
+                    if (BIDIR) {
+                        rb[(j & 1) * 2] = __byte_perm(t[0], t[1], 0x6420);
+                        rb[(j & 1) * 2 + 1] = __byte_perm(t[2], t[3], 0x6420);
+                        if (j & 1)
+                            *reinterpret_cast<uint4*>(res + ((((j >> 1) ^ (row >> 1)) & 3) << 4)) = make_uint4(rb[0], rb[1], rb[2], rb[3]);
+                    }
                 }
                 (hw == 0 ? rq_buf : rk_buf)[(c & 1) * kC + row] = make_float2(rn, nrm > kEps ? 1.f : 0.f);
                 fence_proxy_async();
@@ -710,7 +777,11 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     const uint32_t tacc = tmem + lane_base + colP1 + (c & 1) * 128 + (isq ? 0 : 64);
                     const uint8_t* tile = stage_g(c) + off_tile;
                     const float2 rn = rn_buf[(c & 1) * kC + row];
+                    const uint8_t* res = gbase + L::kOffG + (c & 1) * 16384 + hw * 8192 + row * 64;
                     float d0 = 0.f, d1 = 0.f;
+                    __nv_bfloat162 ec[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) ec[i] = __halves2bfloat162(__float2bfloat16_rn(0.f), __float2bfloat16_rn(0.f));
 #pragma unroll 1
                     for (int hf = 0; hf < 2; ++hf) {
                         uint32_t a[32];
@@ -726,10 +797,34 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                                 d0 = fmaf(f.x, __uint_as_float(a[8 * j + 2 * i]), d0);
                                 d1 = fmaf(f.y, __uint_as_float(a[8 * j + 2 * i + 1]), d1);
                             }
+                            if (BIDIR) {
+                                // <x rn - x^, a>: the part of <x^, a> that the bf16 rounding of x^ lost,
+                                // in packed bf16 arithmetic (a correction: one percent of it is plenty).
+                                // Byte m of the residuals next to 0x43 is the bf16 number 128 + m.
+                                const uint2 rw = *reinterpret_cast<const uint2*>(res + ((((hf * 2 + (j >> 1)) ^ (row >> 1)) & 3) << 4) + (j & 1) * 8);
+                                const __nv_bfloat162 c192 = __halves2bfloat162(__float2bfloat16_rn(192.f), __float2bfloat16_rn(192.f));
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    const uint32_t word = i < 2 ? rw.x : rw.y;
+                                    const uint32_t pr = __byte_perm(word, 0x43434343u, (i & 1) ? 0x4342 : 0x4140);
+                                    const __nv_bfloat162 r = __hsub2(*reinterpret_cast<const __nv_bfloat162*>(&pr), c192);
+                                    const __nv_bfloat162 ab = __floats2bfloat162_rn(__uint_as_float(a[8 * j + 2 * i]), __uint_as_float(a[8 * j + 2 * i + 1]));
+                                    ec[i] = __hfma2(r, ab, ec[i]);
+                                }
+                            }
                         }
                     }
-                    const float dot = d0 + d1;
-                    if (isq) dm_acc += dot;    // <q^_i, dQ^_i> of the unscaled accumulator (rows past N are zero)
+                    float dot = d0 + d1;
+                    if (BIDIR) {
+                        // dm = <S, R> (formed in the prologue) + sum_i <dq^_i, dQ^_i> + sum_j <dk^_j, dK^_j>,
+                        // dx^ the rounding residuals: exact to second order in the bf16 roundings.
+                        const float2 s01 = __bfloat1622float2(__hadd2(ec[0], ec[1])), s23 = __bfloat1622float2(__hadd2(ec[2], ec[3]));
+                        const float corr = ((s01.x + s01.y) + (s23.x + s23.y)) * (1.f / 32768.f);
+                        dm_acc += corr;
+                        dot += corr;
+                    } else if (isq) {
+                        dm_acc += dot;    // <q^_i, dQ^_i> of the unscaled accumulator (rows past N are zero)
+                    }
                     // out = sc (a - coef x^), rounded to bf16 once
                     const float sc = cfac * rn.x, mc = -(dot * rn.y) * sc;
 #pragma unroll 1
@@ -749,7 +844,14 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                                 ow[i] = pack_bf16(fmaf(f.x, mc, __uint_as_float(a[8 * j + 2 * i]) * sc),
                                                   fmaf(f.y, mc, __uint_as_float(a[8 * j + 2 * i + 1]) * sc));
                             }
-                            *reinterpret_cast<uint4*>(out_tile + swz(row, hf * 4 + j)) = o;
+                            if (VARLEN && ragged_last && c == n_chunks - 1) {
+                                const long long grow = (long long)chunk_row(c) + row;
+                                if (grow < tok1 && (hf * 4 + j) * 8 < p.out_w[hw])
+                                    *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out_rows[hw]) + grow * p.out_sn[hw] +
+                                                              (long long)h * p.out_sh[hw] + (hf * 4 + j) * 8) = o;
+                            } else {
+                                *reinterpret_cast<uint4*>(out_tile + swz(row, hf * 4 + j)) = o;
+                            }
                         }
                     }
                 }
@@ -777,17 +879,24 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         o.y = pack_bf16(__uint_as_float(a[8 * j + 2]) * cfac, __uint_as_float(a[8 * j + 3]) * cfac);
                         o.z = pack_bf16(__uint_as_float(a[8 * j + 4]) * cfac, __uint_as_float(a[8 * j + 5]) * cfac);
                         o.w = pack_bf16(__uint_as_float(a[8 * j + 6]) * cfac, __uint_as_float(a[8 * j + 7]) * cfac);
-                        *reinterpret_cast<uint4*>(tile + swz(row, hw * 4 + j)) = o;
+                        if (VARLEN && ragged_last && c == n_chunks - 1) {
+                            const long long grow = (long long)chunk_row(c) + row;
+                            if (grow < tok1 && (hw * 4 + j) * 8 < p.out_w[2])
+                                *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out_rows[2]) + grow * p.out_sn[2] +
+                                                          (long long)h * p.out_sh[2] + (hw * 4 + j) * 8) = o;
+                        } else {
+                            *reinterpret_cast<uint4*>(tile + swz(row, hw * 4 + j)) = o;
+                        }
                     }
                 }
                 fence_proxy_async();
                 mbar_arrive(bar(B_EVDONE, c));
                 BSTAMP(1 + hw, c, 4);
             }
-            if (isq) {
+            if (isq || BIDIR) {
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) dm_acc += __shfl_xor_sync(0xffffffffu, dm_acc, o);
-                if (lane == 0) dm_red[q4] = dm_acc;
+                if (lane == 0) dm_red[(isq ? 0 : 12) + q4] = dm_acc;
             }
         }
     }
@@ -800,7 +909,10 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         if (tid == 0) {
             // Fixed-order reduction of the CTA's dm term.
             if (!*abort_flag)
-                p.dm_partial[(size_t)bh * p.n_groups + g] = (dm_red[0] + dm_red[1]) + (dm_red[2] + dm_red[3]);
+                p.dm_partial[(size_t)bh * p.n_groups + g] = BIDIR ? ((dm_red[4] + dm_red[5]) + (dm_red[6] + dm_red[7])) +
+                                                                          (((dm_red[0] + dm_red[1]) + (dm_red[2] + dm_red[3])) +
+                                                                           ((dm_red[12] + dm_red[13]) + (dm_red[14] + dm_red[15])))
+                                                                  : (dm_red[0] + dm_red[1]) + (dm_red[2] + dm_red[3]);
             __threadfence();
             *last_flag = atomicAdd(&p.status[4], 1) == (int)gridDim.x - 1;
         }
@@ -817,7 +929,9 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 float part = 0.f;
                 for (int i = lane; i < per; i += 32) {
                     const int bb = i / p.n_groups, gg = i - bb * p.n_groups;
-                    const float sb2 = p.seq_len ? p.seq_len[bb] : (p.seq_len_scalar > 0.f ? p.seq_len_scalar : (float)p.N);
+                    const float sb2 = p.seq_len ? p.seq_len[bb]
+                                                : (p.seq_len_scalar > 0.f ? p.seq_len_scalar
+                                                   : (float)(VARLEN ? max(p.cu_seqlens[bb + 1] - p.cu_seqlens[bb], 1) : p.N));
                     const float ls = logf(sb2);
                     part += __ldcg(&p.dm_partial[((size_t)bb * p.H + hh) * p.n_groups + gg]) *
                             (-ls * sg * (1.0f - sg) * expf(-sg * ls));
@@ -867,12 +981,13 @@ struct StateParams {
     int all_sq;              // bidirectional backward: V^T K^ of the last group is read too
     int no_sq;               // V^T K^ comes from the forward call's workspace: no group loads k and v
     int grid_groups;         // groups 0 .. grid_groups - 1 of every (b, h) are computed (a causal forward never reads the last one's)
+    const int* cu_seqlens;   // VARLEN instances: packed batch, one group per (sequence, head)
 };
 
 // RONLY: no group needs V^T K^ (the forward call's partial states serve): a stage holds q and dO
 // only, the product is the 64 x 64 Q^^T dO (rows 16 i .. 16 i + 15 of the result sit in lanes
 // 32 i .. 32 i + 15 of the accumulator), and the ring is twice as deep.
-template <bool RONLY>
+template <bool RONLY, bool VARLEN>
 __global__ void __launch_bounds__(kStThreads, 1)
 tc_bwd_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                     const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmDO, StateParams p) {
@@ -892,8 +1007,10 @@ tc_bwd_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = blockIdx.x % p.grid_groups, bh = blockIdx.x / p.grid_groups;
-    const int b = bh / p.H, h = bh % p.H;
-    const int tok0 = g * p.group, tok1 = min(p.N, tok0 + p.group);
+    const int bseq = bh / p.H, h = bh % p.H;
+    const int b = VARLEN ? 0 : bseq;                   // batch coordinate of the tensor maps
+    const int tok0 = VARLEN ? p.cu_seqlens[bseq] : g * p.group;
+    const int tok1 = VARLEN ? p.cu_seqlens[bseq + 1] : min(p.N, tok0 + p.group);
     const int n_chunks = (tok1 - tok0 + kC - 1) / kC;
     const bool is_mma = warp == 8, is_copy = warp == 9;
     // Nobody reads V^T K^ of the last group: its CTA leaves the v and k slots at zero (the product
@@ -999,7 +1116,9 @@ tc_bwd_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     a2 = fmaf(f1.x, f1.x, a2); a3 = fmaf(f1.y, f1.y, a3);
                 }
             }
-            const float rn = 1.0f / fmaxf(sqrtf((a0 + a1) + (a2 + a3)), kEps);
+            float rn = 1.0f / fmaxf(sqrtf((a0 + a1) + (a2 + a3)), kEps);
+            // (a packed batch: rows of the next sequence in a ragged chunk count for nothing)
+            if (VARLEN && tok0 + (n_chunks - 1 - c) * kC + row >= tok1) rn = 0.f;
             // (the same two-term packed scaling as in the walk: its q^, k^ must be the same bits)
             const __nv_bfloat16 hi = __float2bfloat16_rn(rn);
             const __nv_bfloat16 lo = __float2bfloat16_rn(rn - __bfloat162float(hi));
@@ -1058,11 +1177,19 @@ cudaError_t launch_tc_bwd_fused(const TcBwdFusedArgs& a, int B, int H, int N, cu
     CUtensorMap tm[7];
     BwdParams p;
     p.head_first_mask = 0;
+    // A packed batch is one tensor of total_tokens rows per head (batch extent 1).
+    const int map_B = a.cu_seqlens ? 1 : B, map_N = a.cu_seqlens ? a.total_tokens : N;
     for (int i = 0; i < 7; ++i) {
         bool hf = false;
-        if (!make_tile_map(&tm[i], ptrs[i], B, H, N, dims[i], lays[i], &hf)) return cudaErrorInvalidValue;
+        if (!make_tile_map(&tm[i], ptrs[i], map_B, H, map_N, dims[i], lays[i], &hf)) return cudaErrorInvalidValue;
         p.head_first_mask |= (hf ? 1 : 0) << i;
     }
+    p.cu_seqlens = a.cu_seqlens;
+    for (int i = 0; i < 3; ++i) {
+        const RowLayout lo = resolve_layout(lays[4 + i], H, map_N, dims[4 + i]);
+        p.out_rows[i] = const_cast<void*>(ptrs[4 + i]); p.out_sn[i] = lo.sn; p.out_sh[i] = lo.sh; p.out_w[i] = dims[4 + i];
+    }
+    if (a.cu_seqlens && a.n_groups != 1) return cudaErrorInvalidValue;
     p.sq_part = a.sq_part; p.r_part = a.r_part; p.dm_partial = a.dm_partial; p.dm_out = a.dm_out;
     p.status = a.status; p.m = a.m; p.seq_len = a.seq_len; p.seq_len_scalar = a.seq_len_scalar;
     p.H = H; p.N = N; p.group = a.group; p.n_groups = a.n_groups;
@@ -1072,7 +1199,8 @@ cudaError_t launch_tc_bwd_fused(const TcBwdFusedArgs& a, int B, int H, int N, cu
     // update is taken out again), so the states stay zero and no partial-state pass is needed.
     p.no_state = (!a.bidir && a.n_groups == 1 && N <= kC && !a.sq_part && !a.r_part) ? 1 : 0;
     if (!p.no_state && !a.r_part) return cudaErrorInvalidValue;
-    auto kern = a.bidir ? tc_bwd_fused_kernel<true> : tc_bwd_fused_kernel<false>;
+    auto kern = a.cu_seqlens ? (a.bidir ? tc_bwd_fused_kernel<true, true> : tc_bwd_fused_kernel<false, true>)
+                             : (a.bidir ? tc_bwd_fused_kernel<true, false> : tc_bwd_fused_kernel<false, false>);
     if (cudaError_t e = configure_smem_once(reinterpret_cast<const void*>(kern), L::kDynBytes); e != cudaSuccess)
         return e;
     const int prof = profile_begin_launch(3, st);
@@ -1102,11 +1230,14 @@ cudaError_t launch_tc_bwd_states(const TcBwdFusedArgs& a, float* sq_out, float* 
     CUtensorMap tm[4];
     StateParams p;
     p.head_first_mask = 0;
+    const int map_B = a.cu_seqlens ? 1 : B, map_N = a.cu_seqlens ? a.total_tokens : N;
     for (int i = 0; i < 4; ++i) {
         bool hf = false;
-        if (!make_tile_map(&tm[i], ptrs[i], B, H, N, dims[i], lays[i], &hf)) return cudaErrorInvalidValue;
+        if (!make_tile_map(&tm[i], ptrs[i], map_B, H, map_N, dims[i], lays[i], &hf)) return cudaErrorInvalidValue;
         p.head_first_mask |= (hf ? 1 : 0) << i;
     }
+    p.cu_seqlens = a.cu_seqlens;
+    if (a.cu_seqlens && a.n_groups != 1) return cudaErrorInvalidValue;
     p.sq_out = sq_out; p.r_out = r_out; p.status = a.status;
     p.H = H; p.N = N; p.group = a.group; p.n_groups = a.n_groups;
     p.clear_status = clear_status;
@@ -1115,7 +1246,8 @@ cudaError_t launch_tc_bwd_states(const TcBwdFusedArgs& a, float* sq_out, float* 
     p.grid_groups = a.n_groups;
     p.wait_limit_kcycles = wait_limit_kcycles();
     static_assert(kStStages * L::kStage <= L::kOffCtl && kStStagesR * 2 * kTile <= L::kOffCtl, "the stage ring overlaps the control block");
-    auto kern = p.no_sq ? tc_bwd_state_kernel<true> : tc_bwd_state_kernel<false>;
+    auto kern = a.cu_seqlens ? tc_bwd_state_kernel<false, true> : (p.no_sq ? tc_bwd_state_kernel<true, false> : tc_bwd_state_kernel<false, false>);
+    if (a.cu_seqlens) p.no_sq = 0;
     if (cudaError_t e = configure_smem_once(reinterpret_cast<const void*>(kern), L::kOffCtl + L::kCtlBytes + 1024); e != cudaSuccess)
         return e;
     const int prof = profile_begin_launch(0, st);
@@ -1154,9 +1286,9 @@ cudaError_t launch_tc_pair_states(const void* a_rows, const void* b_rows, const 
     }
     p.sq_out = nullptr; p.r_out = out; p.status = status;
     p.H = H; p.N = N; p.group = group; p.n_groups = n_groups; p.grid_groups = grid_groups;
-    p.clear_status = clear_status; p.all_sq = 0; p.no_sq = 1;
+    p.clear_status = clear_status; p.all_sq = 0; p.no_sq = 1; p.cu_seqlens = nullptr;
     p.wait_limit_kcycles = wait_limit_kcycles();
-    auto kern = tc_bwd_state_kernel<true>;
+    auto kern = tc_bwd_state_kernel<true, false>;
     if (cudaError_t e = configure_smem_once(reinterpret_cast<const void*>(kern), L::kOffCtl + L::kCtlBytes + 1024); e != cudaSuccess)
         return e;
     const int prof = profile_begin_launch(0, st);

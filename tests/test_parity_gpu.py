@@ -1150,6 +1150,39 @@ def test_packed_varlen_leaves_neighbours_alone():
     assert torch.equal(alone, out[5:205])
 
 
+@pytest.mark.parametrize("causal", [True, False])
+def test_packed_varlen_gradients_leave_neighbours_alone(causal, option):
+    """The one-launch backward of a packed batch (d = 64): the rows of a ragged last chunk leave as
+    plain stores, so every sequence's gradient rows are, bit for bit, those of the same sequence
+    passed alone -- nothing of a neighbour is overwritten or attended to -- and the two backward
+    paths (one launch / role-swapped walks) agree within the bf16 tolerance."""
+    H, d, lens = 2, 64, (5, 200, 3, 128, 131)
+    T = sum(lens)
+    g = torch.Generator(device="cuda"); g.manual_seed(11)
+    q, k, v, d_o = (torch.randn((T, H, d), generator=g, device="cuda").to(torch.bfloat16) for _ in range(4))
+    m = torch.randn((H,), generator=g, device="cuda")
+    cu = torch.tensor(np.concatenate([[0], np.cumsum(lens)]), dtype=torch.int32, device="cuda")
+    grads = cott.bwd_varlen(q, k, v, d_o, m, cu, max(lens), causal=causal)
+    dm_sum = torch.zeros_like(grads[3])
+    off = 0
+    for L in lens:
+        sl = slice(off, off + L)
+        cu1 = torch.tensor([0, L], dtype=torch.int32, device="cuda")
+        # (the scaling base of a sequence is its own length in both calls)
+        alone = cott.bwd_varlen(q[sl].contiguous(), k[sl].contiguous(), v[sl].contiguous(), d_o[sl].contiguous(),
+                                m, cu1, L, causal=causal)
+        for x, y in zip(grads[:3], alone[:3]):
+            assert torch.equal(x[sl], y)
+        dm_sum += alone[3]
+        off += L
+    torch.testing.assert_close(grads[3], dm_sum, rtol=1e-4, atol=1e-4 * float(dm_sum.abs().max()))
+    option("fused_bwd", 0)
+    walks = cott.bwd_varlen(q, k, v, d_o, m, cu, max(lens), causal=causal)
+    for x, y in zip(grads[:3], walks[:3]):
+        scale = float(y.float().abs().max())
+        assert float((x.float() - y.float()).abs().max()) <= TOL_BF16 * scale
+
+
 def test_packed_varlen_with_empty_sequences():
     """Sequences of length zero anywhere in the batch: nothing is read or written for them, the
     others are unaffected, and the call reports no error."""
