@@ -90,6 +90,7 @@ unsigned long long cott_launch_count(void);
  *   "pair"               (COTT_PAIR, 1)               0 = gradient streams one after the other where they would run side by side
  *   "fused_bwd"          (COTT_FUSED_BWD, 1)          0 = d = 64 backward (causal and bidirectional) as three role-swapped walks instead of one fused walk
  *   "fused_bidir"        (COTT_FUSED_BIDIR, 1)        0 = bidirectional d = 64 forward as a state pass and a read-out instead of one launch
+ *   "bidir_bwd"          (COTT_BIDIR_BWD, 1)          0 = bidirectional d = 64 backward with one group per (b, h) as a state pass and a walk instead of one launch
  *   "short_fwd"          (COTT_SHORT_FWD, 1)          0 = sequences of at most 128 tokens through the generic walk instead of the stateless kernel
  *   "block_fwd"          (COTT_BLOCK_FWD, 1)          0 = blocks of at most 64 tokens on a state through the generic walk instead of the block kernel
  *   "host_slices"        (COTT_HOST_SLICES, 8)        most slices cott_fwd_bwd_host cuts a batch into (1 .. 16)
@@ -109,7 +110,7 @@ long long cott_get_option(const char* name);
  * launches and writes their durations in milliseconds to ms[] and their kind to kinds[]
  * (0 = partial-state pass, 1 = causal walk, 2 = read-out, 3 = fused backward walk (causal or
  * bidirectional), 4 = one-launch bidirectional forward, 5 = short-sequence forward, 6 = token-block
- * forward on a state; 17 = a causal walk that ran side by
+ * forward on a state, 7 = one-launch bidirectional backward; 17 = a causal walk that ran side by
  * side with a sibling walk of the same size on another stream of the library, in which case
  * its ms is half of the span the pair occupied, first start to last end); both are host
  * arrays of `cap` entries.  Returns the number of entries written, or -1 on a CUDA error.  Not thread-safe

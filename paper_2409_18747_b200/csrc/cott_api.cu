@@ -72,19 +72,21 @@ static Option g_opt_force_path("force_path", "COTT_FORCE_PATH", 1);        // 0:
 static Option g_opt_pair("pair", "COTT_PAIR", 1);                          // 0: gradient streams one after the other
 static Option g_opt_fused_bwd("fused_bwd", "COTT_FUSED_BWD", 1);           // 0: causal d=64 backward through the three role-swapped walks
 static Option g_opt_fused_bidir("fused_bidir", "COTT_FUSED_BIDIR", 1);     // 0: bidirectional d=64 forward as state pass + read-out
+static Option g_opt_bidir_bwd("bidir_bwd", "COTT_BIDIR_BWD", 1);           // 0: bidirectional d=64 backward of one group per (b, h) as state pass + walk
 static Option g_opt_short_fwd("short_fwd", "COTT_SHORT_FWD", 1);           // 0: sequences of <= 128 tokens through the generic walk
 static Option g_opt_block_fwd("block_fwd", "COTT_BLOCK_FWD", 1);           // 0: blocks of <= 64 tokens on a state through the generic walk
 static Option g_opt_wait_ms("wait_limit_ms", "COTT_WAIT_LIMIT_MS", 2000);  // bound of every device-side wait
 static Option g_opt_wait_kc("wait_limit_kcycles", "COTT_WAIT_LIMIT_KCYCLES", -1);  // the same in units of 1024 SM cycles (< 0: use the ms value)
 static Option g_opt_host_slices("host_slices", "COTT_HOST_SLICES", 8);     // slices of the host-buffer step (1 .. 16)
 static Option* const g_options[] = {&g_opt_force_group, &g_opt_force_path, &g_opt_pair, &g_opt_fused_bwd,
-                                    &g_opt_wait_ms, &g_opt_wait_kc, &g_opt_host_slices, &g_opt_fused_bidir, &g_opt_short_fwd, &g_opt_block_fwd};
+                                    &g_opt_wait_ms, &g_opt_wait_kc, &g_opt_host_slices, &g_opt_fused_bidir, &g_opt_short_fwd, &g_opt_block_fwd, &g_opt_bidir_bwd};
 
 int option_force_group() { return (int)g_opt_force_group.get(); }
 int option_force_path() { return (int)g_opt_force_path.get(); }
 int option_pair() { return (int)g_opt_pair.get(); }
 int option_fused_bwd() { return (int)g_opt_fused_bwd.get(); }
 int option_fused_bidir() { return (int)g_opt_fused_bidir.get(); }
+int option_bidir_bwd() { return (int)g_opt_bidir_bwd.get(); }
 int option_short_fwd() { return (int)g_opt_short_fwd.get(); }
 int option_block_fwd() { return (int)g_opt_block_fwd.get(); }
 int wait_limit_kcycles() {
@@ -593,6 +595,15 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
                 COTT_CUDA(cudaMemsetAsync(ws, 0, kWsHeaderBytes, st));      // status words and the dm counter
                 f.plain_launch = 1;
                 COTT_CUDA(launch_tc_bwd_fused(f, B, H, N, st));
+                return COTT_OK;
+            }
+            if (!causal && p.n_groups == 1 && N <= 1024 && option_bidir_bwd() != 0) {
+                // One group per (b, h) of at most 1024 tokens: both state totals, the three gradients and
+                // dm in one launch (cott_tc_bidir_bwd.cu), nothing but q, k, v, dO read and dq, dk, dv
+                // written.  (A CTA walks its sequence twice with two tile pairs in flight: beyond
+                // eight chunks the two-launch form with its deeper rings is as fast or faster.)
+                COTT_CUDA(cudaMemsetAsync(ws, 0, kWsHeaderBytes, st));      // status words and the dm counter
+                COTT_CUDA(launch_tc_bidir_bwd(f, B, H, N, st));
                 return COTT_OK;
             }
             COTT_CUDA(launch_tc_bwd_states(f, st0, st1, 1, B, H, N, st));

@@ -141,6 +141,10 @@ struct TcBwdFusedArgs {
     int w_k, w_v;   // real columns of q, k, dq, dk and of v, dO, dv when fewer than 64 (0: 64)
 };
 cudaError_t launch_tc_bwd_fused(const TcBwdFusedArgs& a, int B, int H, int N, cudaStream_t st);
+// Bidirectional backward of one group per (b, h) (or per sequence and head of a packed batch) at
+// d <= 64 in one launch (cott_tc_bidir_bwd.cu): uses the tensors, layouts, widths, dm_partial
+// ([B * H] floats), dm_out, status (words 0-7 zero at launch), m, seq_len and cu_seqlens of `a`.
+cudaError_t launch_tc_bidir_bwd(const TcBwdFusedArgs& a, int B, int H, int N, cudaStream_t st);
 // Both partial states of every group in one launch (uses q, k, v, d_o, the layouts, group,
 // n_groups and status of `a`); clear_status: this is the first kernel of a library call.
 cudaError_t launch_tc_bwd_states(const TcBwdFusedArgs& a, float* sq_out, float* r_out, int clear_status, int B, int H,
@@ -187,6 +191,7 @@ int option_force_path();
 int option_pair();
 int option_fused_bwd();
 int option_fused_bidir();
+int option_bidir_bwd();
 int option_short_fwd();
 int option_block_fwd();
 int wait_limit_kcycles();      // bound of every device-side wait, in units of 1024 SM cycles

@@ -674,6 +674,50 @@ def test_bidirectional_backward_many_heads():
     torch.testing.assert_close(dm.double(), route2, rtol=5e-2, atol=5e-2 * float(route2.abs().max()))
 
 
+@pytest.mark.parametrize("one_launch", [1, 0])
+@pytest.mark.parametrize("shape", [(2, 3, 1, 64, 64), (2, 3, 127, 64, 64), (3, 5, 128, 64, 64), (2, 4, 129, 64, 64),
+                                   (2, 7, 640, 64, 64), (1, 3, 1024, 64, 64), (2, 3, 300, 32, 64), (2, 3, 300, 64, 40),
+                                   (2, 2, 200, 24, 16)])
+def test_bidirectional_backward_both_forms(shape, one_launch, option, force_group):
+    """The bidirectional backward at head sizes up to 64 with one group per (b, h): in one launch
+    (both state totals, then the gradient rows; dm from the element-wise product of the totals)
+    and as a state pass followed by the walk -- every gradient of both against the definition, dm at
+    the strict gate, on chunk-count boundaries, a ragged last chunk and key / value sizes of their
+    own."""
+    B, H, N, dk, dv = shape
+    c = synth.make_qkv(B, H, N, dk, torch.bfloat16, 6100 + N + dk + dv, with_do=True, d_v=dv)
+    q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
+    option("bidir_bwd", one_launch)
+    force_group(4096)
+    n0 = cott.cott.launch_count()
+    dq, dk_, dv_, dm = cott.bwd(q, k, v, d_o, m, causal=False)
+    assert cott.cott.launch_count() - n0 == (1 if one_launch else 2)
+    rq, rk, rv, rm = oracle.bwd_quadratic(c["q"], c["k"], c["v"], c["d_o"], c["m"], None, False)
+    gate(dq, rq, torch.bfloat16); gate(dk_, rk, torch.bfloat16); gate(dv_, rv, torch.bfloat16)
+    gate_dm(dm, rm, 1e-2, dm_condition(rv, c["v"], c["m"], None), DM_COND_BF16)
+
+
+def test_bidirectional_backward_one_launch_in_a_fused_buffer(force_group):
+    """The one-launch bidirectional backward reads q, k, v from a fused [B, N, 3, H, d] projection
+    output and writes dq, dk, dv into one: bit-identical to the dense call."""
+    B, H, N, d = 2, 4, 333, 64
+    c = synth.make_qkv(B, H, N, d, torch.bfloat16, 6200, with_do=True)
+    q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
+    force_group(4096)
+    n0 = cott.cott.launch_count()
+    want = cott.bwd(q, k, v, d_o, m, causal=False)
+    assert cott.cott.launch_count() - n0 == 1
+    fused = torch.stack([q.permute(0, 2, 1, 3), k.permute(0, 2, 1, 3), v.permute(0, 2, 1, 3)], dim=2).contiguous()   # [B,N,3,H,d]
+    qs, ks, vs = (fused[:, :, i].permute(0, 2, 1, 3) for i in range(3))
+    grads = torch.full_like(fused, 7.0)
+    outs = tuple(grads[:, :, i].permute(0, 2, 1, 3) for i in range(3))
+    d_o_bnhd = d_o.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    got = cott.bwd(qs, ks, vs, d_o_bnhd, m, causal=False, out=outs)
+    for x, y in zip(got[:3], want[:3]):
+        assert torch.equal(x, y)
+    torch.testing.assert_close(got[3], want[3], rtol=0, atol=0)
+
+
 # ------------------------------------------------------------------ seeded sweep over shapes
 def _sweep_cases():
     rng = np.random.RandomState(77)
@@ -962,7 +1006,7 @@ def test_short_blocks_many_heads(dtype, d):
 
 
 # ------------------------------------------------------------------ a wait that runs out
-@pytest.mark.parametrize("op", ["fwd", "bwd", "bidir", "bidir_bwd", "short", "block"])
+@pytest.mark.parametrize("op", ["fwd", "bwd", "bidir", "bidir_bwd", "bidir_bwd_walk", "short", "block"])
 def test_bounded_wait_runs_out_and_reports(op, option, force_group):
     """Every device-side wait has a bound.  With the bound set to zero a wait gives up unless
     its hand-off is there within a few polls -- and the first tiles of a kernel cannot come
@@ -970,13 +1014,16 @@ def test_bounded_wait_runs_out_and_reports(op, option, force_group):
     lets its copies in flight land, frees its tensor memory and returns; the context stays
     usable and the next call is correct.  (No GPU fault is involved: the kernels end normally.)
     One case per warp-specialised kernel: the generic walk, the fused backward (causal and
-    bidirectional instance), the bidirectional, the short-sequence and the block forward."""
-    causal = op not in ("bidir", "bidir_bwd")
+    bidirectional instance), the one-launch bidirectional backward, the bidirectional, the
+    short-sequence and the block forward."""
+    causal = op not in ("bidir", "bidir_bwd", "bidir_bwd_walk")
     force_group(512 if causal else 4096)
+    if op == "bidir_bwd_walk":
+        option("bidir_bwd", 0)
     N = {"short": 64, "block": 16}.get(op, 1024)
     c = synth.make_qkv(1, 2, N, 64, torch.bfloat16, 5400, with_do=True)
     q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
-    is_bwd = op in ("bwd", "bidir_bwd")
+    is_bwd = op in ("bwd", "bidir_bwd", "bidir_bwd_walk")
     code = cott.cott.OP_BWD if is_bwd else cott.cott.OP_FWD
     ws = torch.zeros(cott.workspace_bytes(code, cott.cott.BF16, 1, 2, N, 64, causal),
                      dtype=torch.uint8, device="cuda")
