@@ -17,7 +17,8 @@
 // rounding of q^ and k^ before the state products is the only rounding that enters dm; its
 // first-order terms, sum_i <q^_i - bf16(q^_i), dQ^_i> + sum_j <k^_j - bf16(k^_j), dK^_j>, are added
 // by the same threads.
-// Two CTAs share an SM (83 KB of shared memory, 256 tensor-memory columns each).
+// Two CTAs share an SM (113 KB of shared memory, 256 tensor-memory columns each): three tile pairs
+// are in flight per CTA.
 #include "cott_internal.h"
 #include "cott_sm100.cuh"
 #include "cott_tc_common.cuh"
@@ -33,17 +34,17 @@ constexpr int kC = 128;                 // tokens per chunk
 constexpr int kD = 64;
 constexpr int kTile = kC * kD * 2;      // one 128 x 64 bf16 tile
 constexpr int kWorkerWarps = 8;
-constexpr int kThreads = (kWorkerWarps + 2) * 32;   // + product thread, copy thread
+constexpr int kThreads = (kWorkerWarps + 3) * 32;   // + product thread, load thread, store thread
 
-// Two stages of two tiles.  Phase 1: stage 0 = (k, v), stage 1 = (q, dO); phase 2: stage 0 =
-// (dO, q), stage 1 = (v, k).  The items of a phase alternate between the stages.
+// Three stages of two tiles: a ring that the tile pairs of both phases go through in turn.
 struct L {
-    static constexpr int kOffSb = 4 * kTile;                // bf16 copy of S (64 x 64)
+    static constexpr int kStages = 3;
+    static constexpr int kOffSb = kStages * 2 * kTile;      // bf16 copy of S (64 x 64)
     static constexpr int kOffRb = kOffSb + kD * kD * 2;     // bf16 copy of R
     static constexpr int kOffCtl = kOffRb + kD * kD * 2;
     static constexpr int kOffDmRed = 640;                   // float [16] + a flag, inside the control block
     static constexpr int kCtlBytes = 1024;
-    static constexpr int kDynBytes = kOffCtl + kCtlBytes + 1024;
+    static constexpr int kDynBytes = kOffCtl + kCtlBytes;   // (no slack: the base must be aligned, see the kernel)
 };
 
 struct BidirBwdParams {
@@ -74,6 +75,15 @@ __device__ __forceinline__ void issue_x_state_t(uint32_t tO, uint32_t x, uint32_
     for (int kk = 0; kk < kD / 16; ++kk) mma_ss_w(tO, xl + kk * 2u, kDescHi, sl + kk * 2u, kDescHi, idesc, kk > 0 ? 1u : 0u);
 }
 
+#ifdef COTT_TIMING
+// Debug build only: SM-clock stamps of CTA 0 for the first 32 items: role (0, 1: first thread of the
+// two worker halves; 2: product, 3: load, 4: store thread) x item x slot.
+__device__ long long g_bb_stamps[5 * 32 * 4];
+#define BBSTAMP(role, g, slot) do { if (blockIdx.x == 0 && (g) < 32) g_bb_stamps[((role) * 32 + (g)) * 4 + (slot)] = clock64(); } while (0)
+#else
+#define BBSTAMP(role, g, slot) do { } while (0)
+#endif
+
 template <bool VARLEN>
 __global__ void __launch_bounds__(kThreads, 2)
 tc_bidir_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -83,46 +93,65 @@ tc_bidir_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     // Tensor-memory columns.  Phase 1: S 64 | R 64.  Phase 2: dQ^ [2] 64 each (chunk parity, over
     // S and R, which have been copied by then) | dK^ 64 | dV' 64.
     constexpr uint32_t colS = 0, colR = 64, colQ = 0, colK = 128, colV = 192;
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t* gbase = smem_raw + (base - smem_u32(smem_raw));
+    // Six tiles, two state copies and the control block are all of the 113 KB a CTA can have when
+    // two share an SM: there is no room to round the base up, so it must come aligned to the
+    // 1024 bytes of the swizzle pattern (checked below, reported as an error otherwise).
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t base = smem_u32(smem_raw);
+    uint8_t* gbase = smem_raw;
     const uint32_t bars = base + L::kOffCtl;
-    // Phase 1, by stage: FULL (tiles landed), READY (rows normalised), UFULL (product done, stage
-    // free); PH1DONE, SBREADY once.  Phase 2: FULLB and EDONE by stage; the dQ^ accumulators QFULL /
-    // QDRAIN by chunk parity; KFULL / KDRAIN for the dK^, dV' pair.
-    // A waiter may only ask for the phase that follows the last one it saw complete on the same
-    // barrier; every waiter below follows every phase of the barriers it uses.
-    enum { B_FULL = 0, B_READY = 16, B_UFULL = 32, B_PH1DONE = 48, B_SBREADY = 56, B_FULLB = 64, B_QFULL = 80,
-           B_QDRAIN = 96, B_KFULL = 112, B_KDRAIN = 120, B_EDONE = 128 };
+    // The tile pairs of both phases are one sequence of items: g = 0 .. 2 n - 1 are the (k, v)
+    // (even g) and (q, dO) (odd g) pairs of phase 1, g = 2 n .. 4 n - 1 the (dO, q) (even g - 2 n)
+    // and (v, k) (odd) pairs of phase 2; item g uses stage g % 3.
+    // By stage: FULL (tiles landed; both phases, so its phase parity is (g / 3) & 1), READY (rows
+    // normalised) and UFULL (product done, stage free) in phase 1, EDONE (gradient rows staged) in
+    // phase 2.  PH1DONE, SBREADY once; the dQ^ accumulators QFULL / QDRAIN by chunk parity; KFULL /
+    // KDRAIN for the dK^, dV' pair.
+    // A wait asks whether the barrier's current phase differs in parity from the one named: it is
+    // only meaningful while the barrier is less than two phases away from that one.  Hence every
+    // waiter follows every phase of a barrier it uses -- the row workers wait for the tiles of
+    // every item, also those the other half handles.
+    enum { B_FULL = 0, B_READY = 24, B_UFULL = 48, B_EDONE = 72, B_PH1DONE = 96, B_SBREADY = 104, B_QFULL = 112,
+           B_QDRAIN = 128, B_KFULL = 144, B_KDRAIN = 152, B_SFREE = 160 /* by stage: the stores have read the tiles */ };
     const uint32_t tmem_slot = bars + kCtlTmemSlot;
     volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(gbase + L::kOffCtl + kCtlTmemSlot);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + L::kOffCtl + kCtlAbort);
     float* dm_red = reinterpret_cast<float*>(gbase + L::kOffCtl + L::kOffDmRed);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (base & 1023u) {
+        if (tid == 0 && atomicCAS(p.status, 0, 1) == 0) {
+            p.status[1] = (int)0x80007FF0u;
+            p.status[2] = (int)blockIdx.x | (7 << 24);
+        }
+        return;
+    }
     const int bh = blockIdx.x, bseq = bh / p.H, h = bh % p.H;
     const int b = VARLEN ? 0 : bseq;                   // batch coordinate of the tensor maps
     const int tok0 = VARLEN ? p.cu_seqlens[bseq] : 0;
     const int tok1 = VARLEN ? p.cu_seqlens[bseq + 1] : p.N;
     const int n_chunks = (tok1 - tok0 + kC - 1) / kC;
+    const int n1 = 2 * n_chunks, n_items = 4 * n_chunks;
     // (a packed batch: the last chunk of a sequence may hold rows of the next one -- they are
     // normalised to zero in phase 1, and that chunk's gradient rows are stored one by one)
     const bool ragged_last = VARLEN && ((tok1 - tok0) % kC) != 0;
-    const bool is_mma = warp == kWorkerWarps, is_copy = warp == kWorkerWarps + 1;
+    const bool is_mma = warp == kWorkerWarps, is_copy = warp == kWorkerWarps + 1, is_store = warp == kWorkerWarps + 2;
 
     if (is_mma) {
         tmem_alloc(tmem_slot, 256);
         tmem_relinquish();
     }
     if (tid == 0) {
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < L::kStages; ++i) {
             mbar_init(bars + B_FULL + 8 * i, 1);
             mbar_init(bars + B_READY + 8 * i, 128);
             mbar_init(bars + B_UFULL + 8 * i, 1);
-            mbar_init(bars + B_FULLB + 8 * i, 1);
+            mbar_init(bars + B_EDONE + 8 * i, 128);
+            mbar_init(bars + B_SFREE + 8 * i, 1);
+        }
+        for (int i = 0; i < 2; ++i) {
             mbar_init(bars + B_QFULL + 8 * i, 1);
             mbar_init(bars + B_QDRAIN + 8 * i, 128);
-            mbar_init(bars + B_EDONE + 8 * i, 128);
         }
         mbar_init(bars + B_PH1DONE, 1);
         mbar_init(bars + B_SBREADY, 256);
@@ -136,6 +165,8 @@ tc_bidir_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     if (tid < 16) dm_red[tid] = 0.f;
     if (is_copy && lane == 0) {
         tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); tma_prefetch_desc(&tmDO);
+    }
+    if (is_store && lane == 0) {
         tma_prefetch_desc(&tmDQ); tma_prefetch_desc(&tmDK); tma_prefetch_desc(&tmDV);
     }
     tc_fence_before();
@@ -160,53 +191,65 @@ tc_bidir_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const float cfac = stab_factor(p.m[h], s_b);
     auto par = [&](int c) { return (uint32_t)(c & 1); };
     auto chunk_row = [&](int c) { return tok0 + c * kC; };
+    // item g: its stage, the parity of its phase on the stage's FULL / READY / UFULL barriers, and
+    // (phase 2) on the stage's EDONE barrier, whose first use is the first item >= 2 n on the stage
+    auto stage_of = [&](int g) { return g % L::kStages; };
+    auto fpar = [&](int g) { return (uint32_t)((g / L::kStages) & 1); };
+    auto epar = [&](int g) {
+        const int st = g % L::kStages, first = n1 + ((st - n1 % L::kStages) + L::kStages) % L::kStages;
+        return (uint32_t)(((g - first) / L::kStages) & 1);
+    };
+    auto stage_base = [&](int g) { return (uint32_t)(stage_of(g) * 2) * (uint32_t)kTile; };
 
     if (is_copy) {
-        // ------------------------------------------------------------------ copy thread
+        // ------------------------------------------------------------------ load thread
         if (lane == 0 && n_chunks > 0) {
-            bool ok = true;
-            // phase 1: item (c, s): stage s takes (k, v) (s = 0) or (q, dO) (s = 1) of chunk c once
-            // the product of chunk c - 1 on the same stage is done
-            for (int i = 0; i < 2 * n_chunks && ok; ++i) {
-                const int c = i >> 1, s = i & 1;
-                if (c >= 1 && !wait_or_abort(bars + B_UFULL + 8 * s, par(c - 1), abort_flag)) { ok = false; break; }
-                const uint32_t fb = bars + B_FULL + 8 * s, dst = base + (uint32_t)(2 * s) * kTile;
+            for (int g = 0; g < n_items; ++g) {
+                const int st = stage_of(g);
+                // the stage's previous item: its product (phase 1) or its stores (phase 2) must be done with the tiles
+                if (g >= L::kStages) {
+                    const int prev = g - L::kStages;
+                    if (!wait_or_abort(bars + (prev < n1 ? B_UFULL : B_SFREE) + 8 * st, prev < n1 ? fpar(prev) : epar(prev), abort_flag)) break;
+                }
+                const uint32_t fb = bars + B_FULL + 8 * st, dst = base + stage_base(g);
+                BBSTAMP(3, g, 0);
                 mbar_expect_tx(fb, 2 * kTile);
-                load(dst, s == 0 ? &tmK : &tmQ, s == 0 ? 1 : 0, fb, chunk_row(c));
-                load(dst + kTile, s == 0 ? &tmV : &tmDO, s == 0 ? 2 : 3, fb, chunk_row(c));
+                if (g < n1) {
+                    const int c = g >> 1, s = g & 1;       // (k, v) or (q, dO): the rows to normalise first
+                    load(dst, s == 0 ? &tmK : &tmQ, s == 0 ? 1 : 0, fb, chunk_row(c));
+                    load(dst + kTile, s == 0 ? &tmV : &tmDO, s == 0 ? 2 : 3, fb, chunk_row(c));
+                } else {
+                    const int j = g - n1, c = j >> 1, s = j & 1;   // (dO, q) or (v, k): the product's operand first
+                    load(dst, s == 0 ? &tmDO : &tmV, s == 0 ? 3 : 2, fb, chunk_row(c));
+                    load(dst + kTile, s == 0 ? &tmQ : &tmK, s == 0 ? 0 : 1, fb, chunk_row(c));
+                }
             }
-            // phase 2: item (c, s): stage 0 takes (dO, q), stage 1 (v, k).  The gradient rows of
-            // item (c - 1, s) were staged in the same tiles: they go out first.
-            auto store_item = [&](int c, int s) {
-                const int trow = chunk_row(c);
+        }
+    } else if (is_store) {
+        // ------------------------------------------------------------------ store thread
+        // The gradient rows of a phase-2 item are staged in its own tiles (dq over q; dk over k, dv
+        // over v); the stage is free for the next load once the stores have read them.  (A thread of
+        // its own: waiting for that read must not hold up the loads of the other stages.)
+        if (lane == 0 && n_chunks > 0) {
+            for (int g = n1; g < n_items; ++g) {
+                const int st = stage_of(g);
+                if (!wait_or_abort(bars + B_EDONE + 8 * st, epar(g), abort_flag)) break;
+                BBSTAMP(4, g, 0);
+                const int j = g - n1, c = j >> 1, trow = chunk_row(c);
+                const uint32_t sb = base + stage_base(g);
                 int c1, c2;
                 if (!(ragged_last && c == n_chunks - 1)) {      // (else the workers stored the rows themselves)
-                    if (s == 0) {
-                        coords(4, trow, c1, c2); tma_store_4d(&tmDQ, base + kTile, 0, c1, c2, b);
+                    if ((j & 1) == 0) {
+                        coords(4, trow, c1, c2); tma_store_4d(&tmDQ, sb + kTile, 0, c1, c2, b);
                     } else {
-                        coords(5, trow, c1, c2); tma_store_4d(&tmDK, base + 3 * kTile, 0, c1, c2, b);
-                        coords(6, trow, c1, c2); tma_store_4d(&tmDV, base + 2 * kTile, 0, c1, c2, b);
+                        coords(5, trow, c1, c2); tma_store_4d(&tmDK, sb + kTile, 0, c1, c2, b);
+                        coords(6, trow, c1, c2); tma_store_4d(&tmDV, sb, 0, c1, c2, b);
                     }
                 }
                 tma_store_commit();
-            };
-            for (int i = 0; i < 2 * n_chunks && ok; ++i) {
-                const int c = i >> 1, s = i & 1;
-                if (c == 0) {
-                    if (!wait_or_abort(bars + B_UFULL + 8 * s, par(n_chunks - 1), abort_flag)) { ok = false; break; }
-                } else {
-                    if (!wait_or_abort(bars + B_EDONE + 8 * s, par(c - 1), abort_flag)) { ok = false; break; }
-                    store_item(c - 1, s);
-                    tma_store_wait_read0();
-                }
-                const uint32_t fb = bars + B_FULLB + 8 * s, dst = base + (uint32_t)(2 * s) * kTile;
-                mbar_expect_tx(fb, 2 * kTile);
-                load(dst, s == 0 ? &tmDO : &tmV, s == 0 ? 3 : 2, fb, chunk_row(c));
-                load(dst + kTile, s == 0 ? &tmQ : &tmK, s == 0 ? 0 : 1, fb, chunk_row(c));
-            }
-            for (int s = 0; s < 2 && ok; ++s) {
-                if (!wait_or_abort(bars + B_EDONE + 8 * s, par(n_chunks - 1), abort_flag)) break;
-                store_item(n_chunks - 1, s);
+                tma_store_wait_read0();
+                BBSTAMP(4, g, 1);
+                mbar_arrive(bars + B_SFREE + 8 * st);
             }
             tma_store_wait_all0();
         }
@@ -214,46 +257,52 @@ tc_bidir_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         // ------------------------------------------------------------------ product thread
         if (lane == 0 && n_chunks > 0) {
             bool ok = true;
-            for (int i = 0; i < 2 * n_chunks; ++i) {
+            for (int g = 0; g < n1; ++g) {
                 // S (+)= K^^T V, R (+)= Q^^T dO: both operands MN-major (rows = tokens = contraction index)
-                const int c = i >> 1, s = i & 1;
-                if (!wait_or_abort(bars + B_READY + 8 * s, par(c), abort_flag)) { ok = false; break; }
+                const int c = g >> 1, s = g & 1, st = stage_of(g);
+                if (!wait_or_abort(bars + B_READY + 8 * st, fpar(g), abort_flag)) { ok = false; break; }
+                BBSTAMP(2, g, 0);
                 tc_fence_after();
                 constexpr uint32_t idesc = instr_desc_bf16(kD, kD, true, true);
-                const uint32_t at = base + (uint32_t)(2 * s) * kTile;
+                const uint32_t at = base + stage_base(g);
                 const uint32_t al = smem_desc_lo(at, 16384), bl = smem_desc_lo(at + kTile, 16384);
 #pragma unroll
                 for (int kk = 0; kk < kC / 16; ++kk)
                     mma_ss_w(tmem + (s == 0 ? colS : colR), al + kk * 128u, kDescHi, bl + kk * 128u, kDescHi, idesc, (c > 0 || kk > 0) ? 1u : 0u);
-                tc_commit(bars + B_UFULL + 8 * s);
-                if (i + 1 == 2 * n_chunks) tc_commit(bars + B_PH1DONE);
+                tc_commit(bars + B_UFULL + 8 * st);
+                BBSTAMP(2, g, 1);
+                if (g + 1 == n1) tc_commit(bars + B_PH1DONE);
             }
             if (ok && wait_or_abort(bars + B_SBREADY, 0u, abort_flag)) {
-                for (int i = 0; i < 2 * n_chunks; ++i) {
-                    const int c = i >> 1, s = i & 1;
-                    if (!wait_or_abort(bars + B_FULLB + 8 * s, par(c), abort_flag)) break;
+                for (int g = n1; g < n_items; ++g) {
+                    const int j = g - n1, c = j >> 1, s = j & 1;
+                    if (!wait_or_abort(bars + B_FULL + 8 * stage_of(g), fpar(g), abort_flag)) break;
+                    BBSTAMP(2, g, 0);
+                    const uint32_t sb = base + stage_base(g);
                     if (s == 0) {
                         // dQ^ = dO S^T into the accumulator of the chunk's parity (drained by chunk c - 2)
                         const int a = c & 1;
                         if (c >= 2 && !wait_or_abort(bars + B_QDRAIN + 8 * a, (uint32_t)(((c >> 1) - 1) & 1), abort_flag)) break;
                         tc_fence_after();
-                        issue_x_state_t(tmem + colQ + a * 64, base, base + L::kOffSb);
+                        issue_x_state_t(tmem + colQ + a * 64, sb, base + L::kOffSb);
                         tc_commit(bars + B_QFULL + 8 * a);
+                        BBSTAMP(2, g, 1);
                     } else {
                         // dK^ = V R^T, dV' = K R (raw k rows: their scale is applied to the product's rows)
                         if (c >= 1 && !wait_or_abort(bars + B_KDRAIN, par(c - 1), abort_flag)) break;
                         tc_fence_after();
-                        issue_x_state_t(tmem + colK, base + 2 * kTile, base + L::kOffRb);
-                        issue_x_state(tmem + colV, base + 3 * kTile, base + L::kOffRb);
+                        issue_x_state_t(tmem + colK, sb, base + L::kOffRb);
+                        issue_x_state(tmem + colV, sb + kTile, base + L::kOffRb);
                         tc_commit(bars + B_KFULL);
+                        BBSTAMP(2, g, 1);
                     }
                 }
             }
         }
     } else {
         // ------------------------------------------------------------------ row workers
-        // Eight warps: TMEM lane quadrant q4 = warp & 3, half hw = warp >> 2.  Half 0 serves stage 0
-        // of both phases (k rows, then the dq rows), half 1 stage 1 (q rows, then dk and dv).
+        // Eight warps: TMEM lane quadrant q4 = warp & 3, half hw = warp >> 2.  Half 0 serves the even
+        // items of both phases (k rows, then the dq rows), half 1 the odd ones (q rows, then dk and dv).
         bool alive = n_chunks > 0;
         auto wait = [&](uint32_t bar_, uint32_t parity) {
             if (alive && !wait_or_abort(bar_, parity, abort_flag)) alive = false;
@@ -261,10 +310,13 @@ tc_bidir_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         };
         const int q4 = warp & 3, hw = warp >> 2, row = q4 * 32 + lane;
         const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
-        // phase 1: a thread normalises one row of the first tile of its stage
-        for (int c = 0; c < n_chunks && alive; ++c) {
-            if (!wait(bars + B_FULL + 8 * hw, par(c))) break;
-            uint8_t* tile = gbase + (2 * hw) * kTile;
+        // phase 1: a thread normalises one row of the first tile of its items
+        for (int g = 0; g < n1 && alive; ++g) {
+            if (!wait(bars + B_FULL + 8 * stage_of(g), fpar(g))) break;
+            if ((g & 1) != hw) continue;
+            if ((tid & 127) == 0) BBSTAMP(hw, g, 0);
+            const int c = g >> 1;
+            uint8_t* tile = gbase + stage_base(g);
             uint4 w[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j) w[j] = *reinterpret_cast<const uint4*>(tile + swz(row, j));
@@ -277,7 +329,8 @@ tc_bidir_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 #pragma unroll
             for (int j = 0; j < 8; ++j) *reinterpret_cast<uint4*>(tile + swz(row, j)) = w[j];
             fence_proxy_async();
-            mbar_arrive(bars + B_READY + 8 * hw);
+            mbar_arrive(bars + B_READY + 8 * stage_of(g));
+            if ((tid & 127) == 0) BBSTAMP(hw, g, 2);
         }
         // the totals: fp32 in tensor memory (M = 64: row r sits in lane 32 (r / 16) + r % 16), bf16
         // copies into shared memory, and <S, R> for dm
@@ -330,17 +383,17 @@ tc_bidir_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&wj);
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
+                        // <x, a> with the raw row (times rn afterwards) and <bf16(x^), a>
                         const float2 x = __bfloat1622float2(e[i]);
                         const float2 xh = __bfloat1622float2(__hfma2(e[i], hi2, __hmul2(e[i], lo2)));
-                        const float x0 = x.x * rn, x1 = x.y * rn;
                         const float a0 = __uint_as_float(a[8 * j + 2 * i]), a1 = __uint_as_float(a[8 * j + 2 * i + 1]);
-                        d0 = fmaf(x0, a0, d0); d1 = fmaf(x1, a1, d1);
-                        e0 = fmaf(x0 - xh.x, a0, e0); e1 = fmaf(x1 - xh.y, a1, e1);
+                        d0 = fmaf(x.x, a0, d0); d1 = fmaf(x.y, a1, d1);
+                        e0 = fmaf(xh.x, a0, e0); e1 = fmaf(xh.y, a1, e1);
                     }
                 }
             }
-            const float dot = d0 + d1;
-            const float sc = cfac * rn, mc = clamped ? 0.f : -dot * sc;
+            const float dot = (d0 + d1) * rn;                       // <x^, a>
+            const float sc = cfac * rn, mc = (clamped ? 0.f : -dot * sc) * rn;   // (times rn: applied to the raw row)
 #pragma unroll 1
             for (int hf = 0; hf < 2; ++hf) {
                 uint32_t a[32];
@@ -355,8 +408,8 @@ tc_bidir_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const float2 x = __bfloat1622float2(e[i]);
-                        ow[i] = pack_bf16(fmaf(x.x * rn, mc, __uint_as_float(a[8 * j + 2 * i]) * sc),
-                                          fmaf(x.y * rn, mc, __uint_as_float(a[8 * j + 2 * i + 1]) * sc));
+                        ow[i] = pack_bf16(fmaf(x.x, mc, __uint_as_float(a[8 * j + 2 * i]) * sc),
+                                          fmaf(x.y, mc, __uint_as_float(a[8 * j + 2 * i + 1]) * sc));
                     }
                     if (VARLEN && ragged_last && c == n_chunks - 1) {
                         const long long grow = (long long)chunk_row(c) + row;
@@ -368,12 +421,15 @@ tc_bidir_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     }
                 }
             }
-            return e0 + e1;
+            return dot - (e0 + e1);                                 // <x^ - bf16(x^), a>
         };
-        for (int c = 0; c < n_chunks && alive; ++c) {
-            if (!wait(bars + B_FULLB + 8 * hw, par(c))) break;
+        for (int g = n1; g < n_items && alive; ++g) {
+            if (!wait(bars + B_FULL + 8 * stage_of(g), fpar(g))) break;
+            if (((g - n1) & 1) != hw) continue;
+            if ((tid & 127) == 0) BBSTAMP(hw, g, 0);
+            const int c = (g - n1) >> 1;
             // the raw q (half 0) or k (half 1) row, its norm
-            uint8_t* xt = gbase + (2 * hw + 1) * kTile;
+            uint8_t* xt = gbase + stage_base(g) + kTile;
             float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
             for (int j = 0; j < 8; j += 2) {
@@ -395,17 +451,19 @@ tc_bidir_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             if (hw == 0) {
                 const int a = c & 1;
                 if (!wait(bars + B_QFULL + 8 * a, (uint32_t)((c >> 1) & 1))) break;
+                if ((tid & 127) == 0) BBSTAMP(hw, g, 1);
                 tc_fence_after();
                 dm_acc += project(tmem + lane_base + colQ + a * 64, xt, rn, clamped, c, 0);
                 tc_fence_before();
                 mbar_arrive(bars + B_QDRAIN + 8 * a);
             } else {
                 if (!wait(bars + B_KFULL, par(c))) break;
+                if ((tid & 127) == 0) BBSTAMP(hw, g, 1);
                 tc_fence_after();
                 dm_acc += project(tmem + lane_base + colK, xt, rn, clamped, c, 1);
                 // dv = c K^ R: the rows of K R times c / max(||k||, eps), over the v rows (both
                 // products that read them are done)
-                uint8_t* vt = gbase + 2 * kTile;
+                uint8_t* vt = gbase + stage_base(g);
                 const float sc = cfac * rn;
 #pragma unroll 1
                 for (int hf = 0; hf < 2; ++hf) {
@@ -433,7 +491,8 @@ tc_bidir_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 mbar_arrive(bars + B_KDRAIN);
             }
             fence_proxy_async();
-            mbar_arrive(bars + B_EDONE + 8 * hw);
+            mbar_arrive(bars + B_EDONE + 8 * stage_of(g));
+            if ((tid & 127) == 0) BBSTAMP(hw, g, 2);
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) dm_acc += __shfl_xor_sync(0xffffffffu, dm_acc, o);
@@ -517,6 +576,10 @@ cudaError_t launch_tc_bidir_bwd(const TcBwdFusedArgs& a, int B, int H, int N, cu
     auto kern = a.cu_seqlens ? tc_bidir_bwd_kernel<true> : tc_bidir_bwd_kernel<false>;
     if (cudaError_t e = configure_smem_once(reinterpret_cast<const void*>(kern), L::kDynBytes); e != cudaSuccess)
         return e;
+    // Two CTAs of 113 KB fill an SM's shared memory: ask for the largest carve-out.
+    if (cudaError_t e = cudaFuncSetAttribute(reinterpret_cast<const void*>(kern), cudaFuncAttributePreferredSharedMemoryCarveout,
+                                             (int)cudaSharedmemCarveoutMaxShared); e != cudaSuccess)
+        return e;
     const int prof = profile_begin_launch(7, st);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(B * H));
@@ -535,3 +598,10 @@ cudaError_t launch_tc_bidir_bwd(const TcBwdFusedArgs& a, int B, int H, int N, cu
 }
 
 }  // namespace cott
+
+#ifdef COTT_TIMING
+// Debug build only: copies the stamps (5 roles x 32 items x 4 slots) to the host.
+extern "C" int cott_debug_bidir_bwd_stamps(long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, cott::g_bb_stamps, sizeof(long long) * 640);
+}
+#endif
