@@ -249,8 +249,9 @@ cott_status cott_bwd_strided(const void* q, const void* k, const void* v, const 
  * else its length.  No padding rows are read as keys or written as outputs.
  *   max_seqlen : an upper bound of the longest sequence (sizes the workspace and the plan)
  *   workspace  : cott_workspace_bytes(COTT_OP_FWD or COTT_OP_BWD, dt, B, H, max_seqlen, d, causal)
- * bf16 with d a multiple of 8 up to 128, or fp32 with d in {32, 64, 128} (COTT_ERR_UNSUPPORTED otherwise); one CTA walks one (sequence,
- * head), so the GPU is filled when B*H reaches the number of SMs.  A NaN or Inf in the first
+ * bf16 with d a multiple of 8 up to 128, or fp32 with d in {32, 64, 128} (COTT_ERR_UNSUPPORTED otherwise).  On the tensor-core
+ * path a sequence is cut into the groups the dense plan for N = max_seqlen uses (group g = its rows g * group .. + group - 1,
+ * as far as they exist), so a batch of few long sequences still fills the GPU; the fp32 kernels walk one (sequence, head) per CTA.  A NaN or Inf in the first
  * rows of one sequence can reach the last rows of the sequence stored before it (the tile
  * that holds both is multiplied by zeros, not skipped).  Other arguments, ordering and
  * aliasing rules as for cott_fwd / cott_bwd.

@@ -987,8 +987,8 @@ cott_status cott_bwd_dkdv(const void* q, const void* k, const void* v, const voi
                      dqk_strides, dv_strides, sp, workspace, workspace_bytes, stream);
 }
 
-// Plan of a packed batch: one group per (sequence, head), tensor-core path only.
-static bool varlen_plan(cott_dtype dt, int B, int H, int total_tokens, int max_seqlen, int d, Plan* p) {
+// Plan of a packed batch.
+static bool varlen_plan(int op, cott_dtype dt, int B, int H, int total_tokens, int max_seqlen, int d, int causal, Plan* p) {
     if (B < 1 || H < 1 || total_tokens < 1 || max_seqlen < 1 || max_seqlen > total_tokens) return false;
     // bf16, tensor cores: any head size that is a multiple of 8 up to 128 (zero-filled tiles);
     // fp32 (and bf16 with force_path = 0): the fp32-accumulating SIMT kernels at 32, 64, 128
@@ -999,6 +999,14 @@ static bool varlen_plan(cott_dtype dt, int B, int H, int total_tokens, int max_s
     p->chunk = p->path == 1 ? 128 : 16;
     p->group = (max_seqlen + p->chunk - 1) / p->chunk * p->chunk; p->n_groups = 1; p->split = 1;
     p->dk = p->dv = d; p->d = p->path == 1 ? (d <= 64 ? 64 : 128) : d; p->padded = p->d != d;
+    if (p->path == 1) {
+        // Tensor cores: the groups of the dense plan for sequences of max_seqlen tokens -- group g
+        // of a sequence is its rows g * group .. + group - 1, as far as they exist -- so that a
+        // batch of few long sequences still fills the GPU.  (No finer partition for the state pass.)
+        Plan dense;
+        if (!make_plan(op, dt, B, H, max_seqlen, d, d, causal, &dense) || dense.path != 1) return false;
+        p->group = dense.group; p->n_groups = dense.n_groups;
+    }
     return true;
 }
 
@@ -1011,7 +1019,7 @@ cott_status cott_fwd_varlen(const void* q, const void* k, const void* v, void* o
     if (o == q || o == k || o == v) return COTT_ERR_INVALID_ARG;
     if (!sp->seq_len && sp->seq_len_scalar > 0.f && sp->seq_len_scalar < 1.f) return COTT_ERR_INVALID_ARG;
     Plan p;
-    if (!varlen_plan(dt, B, H, total_tokens, max_seqlen, d, &p)) return COTT_ERR_UNSUPPORTED;
+    if (!varlen_plan(COTT_OP_FWD, dt, B, H, total_tokens, max_seqlen, d, causal, &p)) return COTT_ERR_UNSUPPORTED;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return COTT_ERR_UNSUPPORTED;
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
         workspace_bytes < workspace_bytes_impl(COTT_OP_FWD, p, B, H, p.d))
@@ -1040,7 +1048,7 @@ cott_status cott_bwd_varlen(const void* q, const void* k, const void* v, const v
     }
     if (!sp->seq_len && sp->seq_len_scalar > 0.f && sp->seq_len_scalar < 1.f) return COTT_ERR_INVALID_ARG;
     Plan p;
-    if (!varlen_plan(dt, B, H, total_tokens, max_seqlen, d, &p)) return COTT_ERR_UNSUPPORTED;
+    if (!varlen_plan(COTT_OP_BWD, dt, B, H, total_tokens, max_seqlen, d, causal, &p)) return COTT_ERR_UNSUPPORTED;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(d_o) || !aligned16(dq) ||
         !aligned16(dk) || !aligned16(dv))
         return COTT_ERR_UNSUPPORTED;

@@ -55,7 +55,7 @@ struct WalkArgs {
     int mode_x, mode_a, mode_b;
     int epilogue; int reverse; int update; int write_out;
     // Packed variable-length batch: B + 1 row offsets into tensors of total rows per head
-    // (batch stride unused), one group per (sequence, head); NULL: dense batch.
+    // (batch stride unused), every sequence cut into groups from its first row on; NULL: dense batch.
     const int* cu_seqlens;
 };
 

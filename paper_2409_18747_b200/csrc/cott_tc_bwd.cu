@@ -81,7 +81,7 @@ struct BwdParams {
     const float* sq_fwd;     // the forward call's partial states K^^T V ([BH, n_groups * split, 64 * 64]) or NULL
     int sq_fwd_split;
     // Packed variable-length batch (VARLEN instances): rows of all sequences back to back, sequence
-    // b = rows cu_seqlens[b] .. cu_seqlens[b + 1] - 1, one group per (sequence, head); the rows
+    // b = rows cu_seqlens[b] .. cu_seqlens[b + 1] - 1, cut into groups from its first row on; the rows
     // of a ragged last chunk leave as plain stores: dq, dk, dv as global memory with their
     // token and head strides in elements.
     const int* cu_seqlens;
@@ -221,9 +221,12 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const int g = blockIdx.x % p.n_groups, bh = blockIdx.x / p.n_groups;
     const int bseq = bh / p.H, h = bh % p.H;
     const int b = VARLEN ? 0 : bseq;                   // batch coordinate of the tensor maps
-    const int tok0 = VARLEN ? p.cu_seqlens[bseq] : g * p.group;
-    const int tok1 = VARLEN ? p.cu_seqlens[bseq + 1] : min(p.N, tok0 + p.group);
-    const int n_chunks = (tok1 - tok0 + kC - 1) / kC;
+    // (packed batch: group g of a sequence starts g groups behind its first row and may lie wholly
+    // behind its last one -- a CTA with nothing to do)
+    const int seq0 = VARLEN ? p.cu_seqlens[bseq] : 0, seq1 = VARLEN ? p.cu_seqlens[bseq + 1] : p.N;
+    const int tok0 = seq0 + g * p.group;
+    const int tok1 = min(seq1, tok0 + p.group);
+    const int n_chunks = tok1 > tok0 ? (tok1 - tok0 + kC - 1) / kC : 0;
     // (a packed batch: the last chunk of a sequence may hold rows of the next one -- they are made
     // inert by normalising them to zero, and that chunk's output rows are stored one by one)
     const bool ragged_last = VARLEN && ((tok1 - tok0) % kC) != 0;
@@ -298,7 +301,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     const float s_b = p.seq_len ? p.seq_len[bseq]
-                                : (p.seq_len_scalar > 0.f ? p.seq_len_scalar : (float)(VARLEN ? max(tok1 - tok0, 1) : p.N));
+                                : (p.seq_len_scalar > 0.f ? p.seq_len_scalar : (float)(VARLEN ? max(seq1 - seq0, 1) : p.N));
     const float cfac = stab_factor(p.m[h], s_b);
 
     const int wg = warp >> 2, q4 = warp & 3;
@@ -981,7 +984,7 @@ struct StateParams {
     int all_sq;              // bidirectional backward: V^T K^ of the last group is read too
     int no_sq;               // V^T K^ comes from the forward call's workspace: no group loads k and v
     int grid_groups;         // groups 0 .. grid_groups - 1 of every (b, h) are computed (a causal forward never reads the last one's)
-    const int* cu_seqlens;   // VARLEN instances: packed batch, one group per (sequence, head)
+    const int* cu_seqlens;   // VARLEN instances: packed batch
 };
 
 // RONLY: no group needs V^T K^ (the forward call's partial states serve): a stage holds q and dO
@@ -1009,9 +1012,9 @@ tc_bwd_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const int g = blockIdx.x % p.grid_groups, bh = blockIdx.x / p.grid_groups;
     const int bseq = bh / p.H, h = bh % p.H;
     const int b = VARLEN ? 0 : bseq;                   // batch coordinate of the tensor maps
-    const int tok0 = VARLEN ? p.cu_seqlens[bseq] : g * p.group;
-    const int tok1 = VARLEN ? p.cu_seqlens[bseq + 1] : min(p.N, tok0 + p.group);
-    const int n_chunks = (tok1 - tok0 + kC - 1) / kC;
+    const int tok0 = (VARLEN ? p.cu_seqlens[bseq] : 0) + g * p.group;
+    const int tok1 = min(VARLEN ? p.cu_seqlens[bseq + 1] : p.N, tok0 + p.group);
+    const int n_chunks = tok1 > tok0 ? (tok1 - tok0 + kC - 1) / kC : 0;
     const bool is_mma = warp == 8, is_copy = warp == 9;
     // Nobody reads V^T K^ of the last group: its CTA leaves the v and k slots at zero (the product
     // then adds nothing to that block) and loads q and dO only.
@@ -1134,6 +1137,14 @@ tc_bwd_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             mbar_arrive(bar(S_NREADY, c));
             SSTAMP(0, c, 2);
         }
+        if (VARLEN && n_chunks == 0) {
+            // A group behind the end of its sequence (packed batch): its partial states are zero.
+            const size_t slot = ((size_t)bh * p.n_groups + g) * kD * kD;
+            for (int i = tid; i < kD * kD / 4; i += 256) {
+                reinterpret_cast<float4*>(p.r_out + slot)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (!RONLY && p.sq_out != nullptr) reinterpret_cast<float4*>(p.sq_out + slot)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
         if (alive && wait_or_abort(bar(S_UFULL, n_chunks - 1), par(n_chunks - 1), abort_flag)) {
             // the group's partial states, fp32: rows 0-63 -> Sq, rows 64-127 -> R (32 columns per thread)
             tc_fence_after();
@@ -1189,7 +1200,6 @@ cudaError_t launch_tc_bwd_fused(const TcBwdFusedArgs& a, int B, int H, int N, cu
         const RowLayout lo = resolve_layout(lays[4 + i], H, map_N, dims[4 + i]);
         p.out_rows[i] = const_cast<void*>(ptrs[4 + i]); p.out_sn[i] = lo.sn; p.out_sh[i] = lo.sh; p.out_w[i] = dims[4 + i];
     }
-    if (a.cu_seqlens && a.n_groups != 1) return cudaErrorInvalidValue;
     p.sq_part = a.sq_part; p.r_part = a.r_part; p.dm_partial = a.dm_partial; p.dm_out = a.dm_out;
     p.status = a.status; p.m = a.m; p.seq_len = a.seq_len; p.seq_len_scalar = a.seq_len_scalar;
     p.H = H; p.N = N; p.group = a.group; p.n_groups = a.n_groups;
@@ -1237,7 +1247,6 @@ cudaError_t launch_tc_bwd_states(const TcBwdFusedArgs& a, float* sq_out, float* 
         p.head_first_mask |= (hf ? 1 : 0) << i;
     }
     p.cu_seqlens = a.cu_seqlens;
-    if (a.cu_seqlens && a.n_groups != 1) return cudaErrorInvalidValue;
     p.sq_out = sq_out; p.r_out = r_out; p.status = a.status;
     p.H = H; p.N = N; p.group = a.group; p.n_groups = a.n_groups;
     p.clear_status = clear_status;

@@ -340,9 +340,12 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     const int g = p.first_group + blockIdx.x % p.grid_groups, bh = blockIdx.x / p.grid_groups;
     const int b = bh / p.H, h = bh % p.H;
     constexpr bool varlen = VARLEN;
-    const int tok0 = varlen ? p.cu_seqlens[b] : g * p.group;
-    const int tok1 = varlen ? p.cu_seqlens[b + 1] : min(p.N, tok0 + p.group);
-    const int n_chunks = (tok1 - tok0 + kChunk - 1) / kChunk;
+    // (packed batch: group g of sequence b starts g groups behind the sequence's first row and may
+    // lie wholly behind its last one -- a CTA with nothing to do)
+    const int seq0 = varlen ? p.cu_seqlens[b] : 0, seq1 = varlen ? p.cu_seqlens[b + 1] : p.N;
+    const int tok0 = seq0 + g * p.group;
+    const int tok1 = min(seq1, tok0 + p.group);
+    const int n_chunks = tok1 > tok0 ? (tok1 - tok0 + kChunk - 1) / kChunk : 0;
     // Packed batch: the chunks of a sequence start at its first row, so only its last chunk can
     // hold rows of the next sequence.  Those rows take no part: the operand that is normalised
     // in shared memory gets zeros there (it is one of the two operands of the state update and
@@ -481,7 +484,7 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
 
     const float s_b = p.seq_len ? p.seq_len[b]
                                 : (p.seq_len_scalar > 0.f ? p.seq_len_scalar
-                                                          : (float)(varlen ? max(tok1 - tok0, 1) : p.N));
+                                                          : (float)(varlen ? max(seq1 - seq0, 1) : p.N));
     const float cfac = stab_factor(p.m[h], s_b);
 
     // Accumulator mapping of a worker thread: TMEM lane quadrant q, column quarter cq, row.
@@ -1101,6 +1104,11 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             }
         }
 
+        if (MODE == MODE_STATE && varlen && n_chunks == 0 && p.state_out != nullptr) {
+            // A group behind the end of its sequence: its partial state is zero.
+            float4* dst = reinterpret_cast<float4*>(p.state_out + ((size_t)bh * p.n_groups + g) * D * D);
+            for (int i = tid; i < D * D / 4; i += 16 * 32) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
         if (MODE == MODE_STATE && alive && p.state_out != nullptr) {
             // Partial state of this group, fp32, unscaled (every state update was waited for).
             tc_fence_after();

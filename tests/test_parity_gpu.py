@@ -1125,6 +1125,22 @@ def test_packed_varlen_matches_per_sequence_definition(d, causal, lens):
     the definition evaluated on that sequence alone (scaling base = its own length), forward and
     all gradients; dm is the sum over the sequences.  Rows of a neighbour that share a tile with
     the end of a sequence must neither be attended to nor overwritten."""
+    _check_packed_batch(d, causal, lens)
+
+
+@pytest.mark.parametrize("d", [64, 128, 96])
+@pytest.mark.parametrize("causal", [True, False])
+@pytest.mark.parametrize("group", [128, 256])
+def test_packed_varlen_with_several_groups_per_sequence(d, causal, group, force_group):
+    """A packed batch whose sequences are cut into groups (few long sequences would otherwise leave
+    most of the GPU idle): group g of a sequence is its rows g * group .. + group - 1 as far as
+    they exist, so sequences have different numbers of groups, some groups end ragged and the
+    shortest sequences leave whole groups empty.  Same checks as with one group per sequence."""
+    force_group(group)
+    _check_packed_batch(d, causal, (650, 1, 256, 257, 129, 900))
+
+
+def _check_packed_batch(d, causal, lens):
     H = 3
     seqs = [synth.make_qkv(1, H, L, d, torch.bfloat16, 5800 + 7 * i + L, with_do=True) for i, L in enumerate(lens)]
     m_np = seqs[0]["m"]
@@ -1198,13 +1214,14 @@ def test_packed_varlen_leaves_neighbours_alone():
 
 
 @pytest.mark.parametrize("causal", [True, False])
-def test_packed_varlen_gradients_leave_neighbours_alone(causal, option):
+def test_packed_varlen_gradients_leave_neighbours_alone(causal, option, force_group):
     """The one-launch backward of a packed batch (d = 64): the rows of a ragged last chunk leave as
     plain stores, so every sequence's gradient rows are, bit for bit, those of the same sequence
     passed alone -- nothing of a neighbour is overwritten or attended to -- and the two backward
     paths (one launch / role-swapped walks) agree within the bf16 tolerance."""
     H, d, lens = 2, 64, (5, 200, 3, 128, 131)
     T = sum(lens)
+    force_group(4096)        # (one group per sequence in both calls: the same kernel, the same bits)
     g = torch.Generator(device="cuda"); g.manual_seed(11)
     q, k, v, d_o = (torch.randn((T, H, d), generator=g, device="cuda").to(torch.bfloat16) for _ in range(4))
     m = torch.randn((H,), generator=g, device="cuda")
@@ -1230,9 +1247,13 @@ def test_packed_varlen_gradients_leave_neighbours_alone(causal, option):
         assert float((x.float() - y.float()).abs().max()) <= TOL_BF16 * scale
 
 
-def test_packed_varlen_with_empty_sequences():
+@pytest.mark.parametrize("group", [0, 128])
+def test_packed_varlen_with_empty_sequences(group, force_group):
     """Sequences of length zero anywhere in the batch: nothing is read or written for them, the
-    others are unaffected, and the call reports no error."""
+    others are unaffected, and the call reports no error -- with one group per sequence and with
+    several (every group of an empty sequence is empty)."""
+    if group:
+        force_group(group)
     H, d = 2, 64
     g = torch.Generator(device="cuda"); g.manual_seed(5)
     lens = (0, 130, 0, 64, 0)
