@@ -133,6 +133,34 @@ def bwd_recurrent(q, k, v, d_o, m, s=None):
     return dq, dk_, dv_, dm
 
 
+def fwd_segment(q, k, v, m, state_in, s=None):
+    """A segment of a longer causal sequence: Eq. 8 started from ``state_in [B,H,dk,dv]``.
+    Returns ``(o, state_out)``."""
+    q, k, v, m, s, B, H, N, dk, dv = _prep(q, k, v, m, s)
+    st_in = np.ascontiguousarray(_f64(state_in)).reshape(B, H, dk, dv)
+    o = np.empty_like(v)
+    st = np.empty((B, H, dk, dv))
+    _load().oracle_fwd_segment(_p(q), _p(k), _p(v), _p(m), _p(s), _p(st_in), _p(o), _p(st), B, H,
+                               ctypes.c_long(N), dk, dv)
+    return o, st
+
+
+def bwd_segment(q, k, v, d_o, m, state_in, d_state_out, s=None):
+    """Gradients of ``sum(dO*O) + sum(d_state_out*state_out)`` of a segment w.r.t. raw q, k, v,
+    ``state_in`` and m.  Returns ``(dq, dk, dv, d_state_in, dm)``."""
+    q, k, v, m, s, B, H, N, dk, dv = _prep(q, k, v, m, s)
+    d_o = _f64(d_o)
+    assert d_o.shape == v.shape
+    st_in = np.ascontiguousarray(_f64(state_in)).reshape(B, H, dk, dv)
+    d_st_out = np.ascontiguousarray(_f64(d_state_out)).reshape(B, H, dk, dv)
+    dq, dk_, dv_ = np.empty_like(q), np.empty_like(q), np.empty_like(v)
+    d_st_in = np.empty((B, H, dk, dv))
+    dm = np.empty((H,))
+    _load().oracle_bwd_segment(_p(q), _p(k), _p(v), _p(d_o), _p(st_in), _p(d_st_out), _p(m), _p(s),
+                               _p(dq), _p(dk_), _p(dv_), _p(d_st_in), _p(dm), B, H, ctypes.c_long(N), dk, dv)
+    return dq, dk_, dv_, d_st_in, dm
+
+
 def decode_step(q, k, v, m, s, state):
     """One Eq. 8 step.  q,k ``[B,H,dk]``, v ``[B,H,dv]``; ``state`` ``[B,H,dk,dv]`` float64 numpy,
     updated IN PLACE; ``s`` ``[B]`` or a scalar.  Returns o ``[B,H,dv]``."""

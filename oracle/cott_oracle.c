@@ -25,7 +25,8 @@
  * only distributes independent (b,h) pairs over host threads.
  *
  * Pins (see tests): hand-worked example, closed forms, numpy GEMM/tril
- * cross-check, finite differences, the identities between Eq. 6, 7/8 and 5.
+ * cross-check, finite differences, the identities between Eq. 6, 7/8 and 5;
+ * the segment forms against the whole-sequence definition they compose to.
  * Readings of the paper that no printed value pins (parity unpinned by the
  * paper itself): the gradient on the clamped (||x|| <= EPS) branch, and the
  * scaling base used by a decode step.
@@ -331,6 +332,105 @@ void oracle_bwd_recurrent(const double* q, const double* k, const double* v, con
                 dvp[j * dv + e] = acc;
             }
         }
+        dm_bh[bh] = chain_to_raw(qh, kh, nq, nk, V, dqh, dkh, dvp, dq + bh * N * dk,
+                                 dk_out + bh * N * dk, dv_out + bh * N * dv, c, s[b], m[h], N, dk, dv);
+        free(qh); free(kh); free(vp); free(nq); free(nk); free(dqh); free(dkh); free(dvp); free(S);
+    }
+    for (int h = 0; h < H; ++h) {
+        dm[h] = 0.0;
+        for (int b = 0; b < B; ++b) dm[h] += dm_bh[(long)b * H + h];
+    }
+    free(dm_bh);
+}
+
+/* ------------------------------------------------------------------------
+ * A segment of a longer causal sequence, forward: the recurrence of Eq. 8
+ * started from a caller-held state instead of zero,
+ *   S_0 = state_in;  S_t = S_{t-1} + k^_t (c v_t)^T;  o_t = S_t^T q^_t,
+ * state_out = S_N (may be NULL).  The state carries the factor c of the
+ * tokens it has absorbed, as the decode step's state does.
+ * --------------------------------------------------------------------- */
+void oracle_fwd_segment(const double* q, const double* k, const double* v, const double* m,
+                        const double* s, const double* state_in, double* o, double* state_out,
+                        int B, int H, long N, int dk, int dv) {
+#pragma omp parallel for schedule(dynamic)
+    for (long bh = 0; bh < (long)B * H; ++bh) {
+        int b = (int)(bh / H), h = (int)(bh % H);
+        const double *Q = q + bh * N * dk, *K = k + bh * N * dk, *V = v + bh * N * dv;
+        double* O = o + bh * N * dv;
+        double* S = malloc(sizeof(double) * dk * dv);
+        double* qh = malloc(sizeof(double) * dk);
+        double* kh = malloc(sizeof(double) * dk);
+        double c = stab_factor(s[b], m[h]);
+        memcpy(S, state_in + bh * dk * dv, sizeof(double) * dk * dv);
+        for (long t = 0; t < N; ++t) {
+            normalise_rows(Q + t * dk, qh, NULL, 1, dk);
+            normalise_rows(K + t * dk, kh, NULL, 1, dk);
+            for (int a = 0; a < dk; ++a)
+                for (int e = 0; e < dv; ++e) S[a * dv + e] += kh[a] * (V[t * dv + e] * c);
+            for (int e = 0; e < dv; ++e) {
+                double acc = 0.0;
+                for (int a = 0; a < dk; ++a) acc += qh[a] * S[a * dv + e];
+                O[t * dv + e] = acc;
+            }
+        }
+        if (state_out) memcpy(state_out + bh * dk * dv, S, sizeof(double) * dk * dv);
+        free(S); free(qh); free(kh);
+    }
+}
+
+/* ------------------------------------------------------------------------
+ * Backward of such a segment, for L = sum(dO (.) O) + sum(d_state_out (.)
+ * state_out), the running sums of the backward (see oracle_bwd_recurrent)
+ * started from what lies outside the segment: the forward sum from state_in,
+ * the reverse sum from d_state_out (the gradient that later tokens send into
+ * the state this segment hands on):
+ *   S_t = state_in + sum_{j<=t} k^_j v'_j^T ,           dq^_t = S_t do_t
+ *   R_j = d_state_out + sum_{t>=j} q^_t do_t^T ,        dk^_j = R_j v'_j ,  dv'_j = R_j^T k^_j
+ *   d_state_in = R_1
+ * state_in is an input of its own (its dependence on m through earlier tokens
+ * belongs to the segment that produced it), so c enters through v' = c v only
+ * and the chain to raw q, k, v and m is the common one.  dm is [H], overwritten.
+ * --------------------------------------------------------------------- */
+void oracle_bwd_segment(const double* q, const double* k, const double* v, const double* d_o,
+                        const double* state_in, const double* d_state_out, const double* m,
+                        const double* s, double* dq, double* dk_out, double* dv_out,
+                        double* d_state_in, double* dm, int B, int H, long N, int dk, int dv) {
+    double* dm_bh = calloc((size_t)B * H, sizeof(double));
+#pragma omp parallel for schedule(dynamic)
+    for (long bh = 0; bh < (long)B * H; ++bh) {
+        int b = (int)(bh / H), h = (int)(bh % H);
+        const double *Q = q + bh * N * dk, *K = k + bh * N * dk, *V = v + bh * N * dv;
+        const double* dO = d_o + bh * N * dv;
+        size_t nk_ = (size_t)N * dk, nv_ = (size_t)N * dv;
+        double *qh = malloc(sizeof(double) * nk_), *kh = malloc(sizeof(double) * nk_);
+        double *vp = malloc(sizeof(double) * nv_);
+        double *nq = malloc(sizeof(double) * N), *nk = malloc(sizeof(double) * N);
+        double *dqh = malloc(sizeof(double) * nk_), *dkh = malloc(sizeof(double) * nk_);
+        double* dvp = malloc(sizeof(double) * nv_);
+        double* S = malloc(sizeof(double) * dk * dv);
+        normalise_rows(Q, qh, nq, N, dk);
+        normalise_rows(K, kh, nk, N, dk);
+        double c = stab_factor(s[b], m[h]);
+        for (size_t i = 0; i < nv_; ++i) vp[i] = V[i] * c;
+        memcpy(S, state_in + bh * dk * dv, sizeof(double) * dk * dv);
+        for (long t = 0; t < N; ++t) { /* forward in time */
+            for (int a = 0; a < dk; ++a)
+                for (int e = 0; e < dv; ++e) S[a * dv + e] += kh[t * dk + a] * vp[t * dv + e];
+            for (int a = 0; a < dk; ++a) dqh[t * dk + a] = dot(S + a * dv, dO + t * dv, dv);
+        }
+        memcpy(S, d_state_out + bh * dk * dv, sizeof(double) * dk * dv); /* now R */
+        for (long j = N - 1; j >= 0; --j) { /* backward in time */
+            for (int a = 0; a < dk; ++a)
+                for (int e = 0; e < dv; ++e) S[a * dv + e] += qh[j * dk + a] * dO[j * dv + e];
+            for (int a = 0; a < dk; ++a) dkh[j * dk + a] = dot(S + a * dv, vp + j * dv, dv);
+            for (int e = 0; e < dv; ++e) {
+                double acc = 0.0;
+                for (int a = 0; a < dk; ++a) acc += S[a * dv + e] * kh[j * dk + a];
+                dvp[j * dv + e] = acc;
+            }
+        }
+        memcpy(d_state_in + bh * dk * dv, S, sizeof(double) * dk * dv);
         dm_bh[bh] = chain_to_raw(qh, kh, nq, nk, V, dqh, dkh, dvp, dq + bh * N * dk,
                                  dk_out + bh * N * dk, dv_out + bh * N * dv, c, s[b], m[h], N, dk, dv);
         free(qh); free(kh); free(vp); free(nq); free(nk); free(dqh); free(dkh); free(dvp); free(S);

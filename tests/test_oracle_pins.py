@@ -402,3 +402,88 @@ def test_unequal_sizes_numpy_and_finite_differences(causal):
         mp[h] += eps; mm[h] -= eps
         fd = (loss(q, k, v, mp) - loss(q, k, v, mm)) / (2 * eps)
         assert abs(fd - dm[h]) <= 1e-6 * max(1.0, abs(fd))
+
+
+# ---------------------------------------------------------------- segments of a longer sequence
+def _segment_case(seed, B=2, H=3, N=37, dk=6, dv=5):
+    q, k = rnd((B, H, N, dk), seed), rnd((B, H, N, dk), seed + 1)
+    v, do = rnd((B, H, N, dv), seed + 2), rnd((B, H, N, dv), seed + 3)
+    m, s = rnd((H,), seed + 4), np.full((B,), float(N))
+    return q, k, v, do, m, s
+
+
+def test_segment_forward_composes_to_the_whole_sequence():
+    """Eq. 8 started from a caller's state: with a zero state it is the recurrence from zero; cut
+    anywhere, two segments give the outputs and the final state of the quadratic definition of the
+    whole sequence (the scaling base belongs to the whole sequence)."""
+    q, k, v, _, m, s = _segment_case(700)
+    B, H, N, dk = q.shape
+    dv = v.shape[-1]
+    zero = np.zeros((B, H, dk, dv))
+    o0, st0 = oracle.fwd_segment(q, k, v, m, zero, s)
+    o_rec, st_rec = oracle.fwd_recurrent(q, k, v, m, s)
+    assert np.array_equal(o0, o_rec) and np.array_equal(st0, st_rec)
+    whole = oracle.fwd_quadratic(q, k, v, m, s, True)
+    for cut in (1, 16, N - 1):
+        o1, st1 = oracle.fwd_segment(q[:, :, :cut], k[:, :, :cut], v[:, :, :cut], m, zero, s)
+        o2, st2 = oracle.fwd_segment(q[:, :, cut:], k[:, :, cut:], v[:, :, cut:], m, st1, s)
+        np.testing.assert_allclose(np.concatenate([o1, o2], axis=2), whole, rtol=1e-12, atol=1e-13)
+        np.testing.assert_allclose(st2, st_rec, rtol=1e-12, atol=1e-13)
+
+
+def test_segment_backward_reduces_and_composes():
+    """Backward of a segment.  (1) With a zero incoming state and no gradient into the outgoing one
+    it is the quadratic definition's backward, and the gradient of the incoming state is
+    sum_t q^_t dO_t^T (numpy).  (2) Chained over two segments -- the second one's d_state_in is the
+    first one's d_state_out -- the gradients are those of the whole sequence, dm the sum."""
+    q, k, v, do, m, s = _segment_case(710)
+    B, H, N, dk = q.shape
+    dv = v.shape[-1]
+    zero = np.zeros((B, H, dk, dv))
+    rq, rk, rv, rm = oracle.bwd_quadratic(q, k, v, do, m, s, True)
+    dq, dk_, dv_, dst, dm = oracle.bwd_segment(q, k, v, do, m, zero, zero, s)
+    for got, want in ((dq, rq), (dk_, rk), (dv_, rv), (dm, rm)):
+        np.testing.assert_allclose(got, want, rtol=1e-11, atol=1e-12)
+    qh = q / np.maximum(np.linalg.norm(q, axis=-1, keepdims=True), 1e-12)
+    np.testing.assert_allclose(dst, np.einsum("bhta,bhte->bhae", qh, do), rtol=1e-12, atol=1e-13)
+    for cut in (1, 20, N - 1):
+        a, b = slice(0, cut), slice(cut, N)
+        _, st1 = oracle.fwd_segment(q[:, :, a], k[:, :, a], v[:, :, a], m, zero, s)
+        g2 = oracle.bwd_segment(q[:, :, b], k[:, :, b], v[:, :, b], do[:, :, b], m, st1, zero, s)
+        g1 = oracle.bwd_segment(q[:, :, a], k[:, :, a], v[:, :, a], do[:, :, a], m, zero, g2[3], s)
+        for i, want in enumerate((rq, rk, rv)):
+            np.testing.assert_allclose(np.concatenate([g1[i], g2[i]], axis=2), want, rtol=1e-11, atol=1e-12)
+        np.testing.assert_allclose(g1[4] + g2[4], rm, rtol=1e-11, atol=1e-12)
+
+
+def test_segment_backward_finite_differences():
+    """Central differences of L = <dO, O> + <d_state_out, state_out> through the segment forward
+    (itself pinned above) in entries of state_in, q, k, v and in m."""
+    q, k, v, do, m, s = _segment_case(720, B=1, H=2, N=9, dk=4, dv=3)
+    B, H, N, dk = q.shape
+    dv = v.shape[-1]
+    st_in, d_st_out = rnd((B, H, dk, dv), 730), rnd((B, H, dk, dv), 731)
+    s = np.array([64.0])
+
+    def loss(q_, k_, v_, m_, st_):
+        o, st = oracle.fwd_segment(q_, k_, v_, m_, st_, s)
+        return float((do * o).sum() + (d_st_out * st).sum())
+
+    dq, dk_, dv_, dst, dm = oracle.bwd_segment(q, k, v, do, m, st_in, d_st_out, s)
+    eps = 1e-6
+    rng = np.random.default_rng(740)
+    for name, arr, grad in (("q", q, dq), ("k", k, dk_), ("v", v, dv_), ("state_in", st_in, dst)):
+        for _ in range(6):
+            idx = tuple(int(rng.integers(0, n)) for n in arr.shape)
+            args = {"q": q, "k": k, "v": v, "state_in": st_in}
+            hi, lo = arr.copy(), arr.copy()
+            hi[idx] += eps; lo[idx] -= eps
+            up = dict(args); up[name] = hi
+            dn = dict(args); dn[name] = lo
+            fd = (loss(up["q"], up["k"], up["v"], m, up["state_in"]) - loss(dn["q"], dn["k"], dn["v"], m, dn["state_in"])) / (2 * eps)
+            assert grad[idx] == pytest.approx(fd, rel=1e-6, abs=1e-8), (name, idx)
+    for h in range(H):
+        mh, ml = m.copy(), m.copy()
+        mh[h] += eps; ml[h] -= eps
+        fd = (loss(q, k, v, mh, st_in) - loss(q, k, v, ml, st_in)) / (2 * eps)
+        assert dm[h] == pytest.approx(fd, rel=1e-6, abs=1e-8)
