@@ -297,6 +297,34 @@ cott_status cott_bwd_after_fwd(const void* q, const void* k, const void* v, cons
                                size_t workspace_bytes, void* stream);
 
 /*
+ * Backward of cott_fwd_stateful: the gradients of one SEGMENT of a longer causal sequence (training
+ * through chunked prefill).  For L = sum(dO (.) O) + sum(d_state_out (.) state_out) of the segment,
+ * the running sums of the backward described after Eq. 7 start from what lies outside it: the
+ * forward sum from state_in, the reverse sum from d_state_out,
+ *     dq^_t = S_t dO_t ,                      S_t = state_in + sum_{j<=t} k^_j (c v_j)^T
+ *     dk^_j = R_j (c v_j) ,  dv'_j = R_j^T k^_j ,  R_j = d_state_out + sum_{t>=j} q^_t dO_t^T
+ *     d_state_in = R_1
+ * followed by the chain rule through Eq. 2-4 as in cott_bwd.
+ *   state_in    : NULL (zero) or fp32 [B,H,d_k,d_v], what cott_fwd_stateful was given
+ *   d_state_out : NULL (zero) or fp32 [B,H,d_k,d_v], the gradient of the state the segment handed on
+ *                 (the d_state_in of the next segment's backward; NULL for the last one)
+ *   d_state_in  : NULL or fp32 [B,H,d_k,d_v], receives the gradient of state_in; not one of the
+ *                 other two buffers
+ *   dm          : this segment's part of the gradient of m (state_in counts as an input of its
+ *                 own: its dependence on m belongs to the segment that produced it, which sees it
+ *                 through d_state_in); the parts of all segments add up to the dm of the sequence
+ * Run over the segments last to first, with the caller's scaling base (sp->seq_len or
+ * sp->seq_len_scalar >= 1, the same for every segment), the calls give the gradients of one
+ * cott_bwd over the whole sequence.  Dense [B,H,N,d] tensors; bf16 with d_k, d_v multiples of 8 up
+ * to 64 (the one-walk backward of the tensor-core path): COTT_ERR_UNSUPPORTED otherwise.
+ * workspace: cott_workspace_bytes_dkdv(COTT_OP_BWD, dt, B, H, N, d_k, d_v, 1).
+ */
+cott_status cott_bwd_stateful(const void* q, const void* k, const void* v, const void* d_o,
+                              const float* state_in, const float* d_state_out, void* dq, void* dk, void* dv,
+                              float* d_state_in, float* dm, int B, int H, int N, int d_k, int d_v, cott_dtype dt,
+                              const cott_scale_params* sp, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Head sizes.  The paper's section 2.1 gives keys / queries and values sizes of their own
  * (d_H_key, d_H_value); every call above takes one `d` for both.  The *_dkdv calls below take
  * the two separately:

@@ -208,11 +208,15 @@ static size_t padded_state_bytes(const Plan& p, int B, int H) {
     return p.padded ? align_up((size_t)B * H * p.d * p.d * sizeof(float), 256) : 0;
 }
 
+// (backward of a segment: the caller's two states and the one it gets back, in the kernels' size)
+static size_t segment_state_bytes(int B, int H, int d) { return align_up((size_t)B * H * d * d * sizeof(float), 256); }
+
 static size_t workspace_bytes_impl(int op, const Plan& p, int B, int H, int d) {
     size_t total = kWsHeaderBytes;
     if (op == COTT_OP_FWD) total += states_bytes(p, B, H, d) + 2 * padded_state_bytes(p, B, H);
     else if (op == COTT_OP_BWD)
-        total += 3 * states_bytes(p, B, H, d) + 2 * align_up((size_t)B * H * p.n_groups * 4, 256);
+        total += 3 * states_bytes(p, B, H, d) + 2 * align_up((size_t)B * H * p.n_groups * 4, 256) +
+                 3 * segment_state_bytes(B, H, d);
     return total;
 }
 
@@ -411,6 +415,15 @@ static cott_status run_tc_stream(TcWalkArgs t, const Plan& p, int B, int H, int 
     return COTT_OK;
 }
 
+// Backward of a segment of a longer causal sequence (cott_bwd_stateful): the caller's fp32
+// [B,H,d_k,d_v] states; state_in / d_state_out NULL = zero, d_state_in NULL = not wanted.
+struct Segment {
+    bool on = false;
+    const float* state_in = nullptr;
+    const float* d_state_out = nullptr;
+    float* d_state_in = nullptr;
+};
+
 // Packed variable-length batch (see cott_fwd_varlen): row offsets and total row count.
 struct Packed {
     const int* cu_seqlens = nullptr;
@@ -539,7 +552,8 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
                             cudaStream_t st, const cott_strides* s_qkv = nullptr,
                             const cott_strides* s_do = nullptr, const cott_strides* s_dqkv = nullptr,
                             Packed packed = Packed(), const cott_strides* s_v = nullptr,
-                            const cott_strides* s_dv = nullptr, const void* fwd_ws = nullptr) {
+                            const cott_strides* s_dv = nullptr, const void* fwd_ws = nullptr,
+                            Segment seg = Segment()) {
     // (d is the size the kernels run at, p.d; the tensors have p.dk and p.dv columns)
     CallLayouts lay{to_layout(s_qkv), to_layout(s_do), to_layout(s_dqkv), q, k, v, d_o};
     lay.dk = p.dk; lay.dv = p.dv; lay.dv_ptr = dv;
@@ -588,6 +602,24 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
             if (fwd_ws && !packed.cu_seqlens && causal && p.n_groups >= 2 && p.n_groups <= 8 && fused_scan_ok(p.n_groups, d, p.group)) {
                 f.sq_fwd = reinterpret_cast<const float*>(static_cast<const char*>(fwd_ws) + kWsHeaderBytes);
                 f.sq_fwd_split = p.split;
+            }
+            if (seg.on) {
+                // A segment: the states enter and leave through copies of the kernels' size behind
+                // the other regions of the workspace (zero where the caller passed none).
+                char* sbase = base + 3 * sb + 2 * align_up((size_t)B * H * p.n_groups * 4, 256);
+                const size_t ssb = segment_state_bytes(B, H, d);
+                float* s_in = reinterpret_cast<float*>(sbase);
+                float* ds_out = reinterpret_cast<float*>(sbase + ssb);
+                float* ds_in = reinterpret_cast<float*>(sbase + 2 * ssb);
+                if (seg.state_in) COTT_CUDA(launch_pad_state(seg.state_in, s_in, BH, p.dk, p.dv, d, st));
+                if (seg.d_state_out) COTT_CUDA(launch_pad_state(seg.d_state_out, ds_out, BH, p.dk, p.dv, d, st));
+                f.state_in = seg.state_in ? s_in : nullptr;
+                f.d_state_out = seg.d_state_out ? ds_out : nullptr;
+                f.d_state_in = seg.d_state_in ? ds_in : nullptr;
+                COTT_CUDA(launch_tc_bwd_states(f, st0, st1, 1, B, H, N, st));
+                COTT_CUDA(launch_tc_bwd_fused(f, B, H, N, st));
+                if (seg.d_state_in) COTT_CUDA(launch_unpad_state(ds_in, seg.d_state_in, BH, p.dk, p.dv, d, st));
+                return COTT_OK;
             }
             if (causal && !packed.cu_seqlens && p.n_groups == 1 && N <= 128) {
                 // One chunk per (b, h): no state is ever read, the walk is the only launch.
@@ -907,7 +939,8 @@ static cott_status bwd_entry(const void* q, const void* k, const void* v, const 
                              const cott_strides* qk_strides, const cott_strides* v_strides,
                              const cott_strides* do_strides, const cott_strides* dqk_strides,
                              const cott_strides* dv_strides, const cott_scale_params* sp, void* workspace,
-                             size_t workspace_bytes, void* stream, const void* fwd_workspace = nullptr) {
+                             size_t workspace_bytes, void* stream, const void* fwd_workspace = nullptr,
+                             Segment seg = Segment()) {
     if (!q || !k || !v || !d_o || !dq || !dk || !dv || !dm || B < 1 || H < 1 || N < 1 || d_k < 1 || d_v < 1)
         return COTT_ERR_INVALID_ARG;
     if (fwd_workspace && (fwd_workspace == workspace || (reinterpret_cast<uintptr_t>(fwd_workspace) & 255u)))
@@ -944,9 +977,29 @@ static cott_status bwd_entry(const void* q, const void* k, const void* v, const 
         workspace_bytes < workspace_bytes_impl(COTT_OP_BWD, p, B, H, p.d))
         return COTT_ERR_WORKSPACE;
     const bool own_v = !same || v_strides || dv_strides;
+    if (seg.on) {
+        // A segment needs the caller's scaling base (the same for every segment of a sequence), is
+        // causal, and runs through the one-walk backward of the tensor-core path at sizes up to 64.
+        if (!causal || (!sp->seq_len && !(sp->seq_len_scalar >= 1.f))) return COTT_ERR_INVALID_ARG;
+        if (p.path != 1 || p.d != 64 || option_fused_bwd() == 0) return COTT_ERR_UNSUPPORTED;
+        if ((seg.state_in && !aligned16(seg.state_in)) || (seg.d_state_out && !aligned16(seg.d_state_out)) ||
+            (seg.d_state_in && !aligned16(seg.d_state_in)))
+            return COTT_ERR_UNSUPPORTED;
+        if (seg.d_state_in && (seg.d_state_in == seg.state_in || seg.d_state_in == seg.d_state_out)) return COTT_ERR_INVALID_ARG;
+    }
     return bwd_impl(q, k, v, d_o, dq, dk, dv, dm, B, H, N, p.d, causal, dt, sp, workspace, p,
                     static_cast<cudaStream_t>(stream), qk_strides, do_strides, dqk_strides, Packed(),
-                    own_v ? vs : nullptr, own_v ? dvs : nullptr, fwd_workspace);
+                    own_v ? vs : nullptr, own_v ? dvs : nullptr, fwd_workspace, seg);
+}
+
+cott_status cott_bwd_stateful(const void* q, const void* k, const void* v, const void* d_o,
+                              const float* state_in, const float* d_state_out, void* dq, void* dk, void* dv,
+                              float* d_state_in, float* dm, int B, int H, int N, int d_k, int d_v, cott_dtype dt,
+                              const cott_scale_params* sp, void* workspace, size_t workspace_bytes, void* stream) {
+    Segment seg;
+    seg.on = true; seg.state_in = state_in; seg.d_state_out = d_state_out; seg.d_state_in = d_state_in;
+    return bwd_entry(q, k, v, d_o, dq, dk, dv, dm, B, H, N, d_k, d_v, 1, dt, nullptr, nullptr, nullptr, nullptr,
+                     nullptr, sp, workspace, workspace_bytes, stream, nullptr, seg);
 }
 
 cott_status cott_bwd_after_fwd(const void* q, const void* k, const void* v, const void* d_o, void* dq,

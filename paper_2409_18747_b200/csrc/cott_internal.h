@@ -137,6 +137,10 @@ struct TcBwdFusedArgs {
     // Packed variable-length batch: B + 1 row offsets into tensors of total_tokens rows per head, one
     // group per (sequence, head); NULL: dense batch.
     const int* cu_seqlens; int total_tokens;
+    // Segment of a longer causal sequence (cott_bwd_stateful; all NULL otherwise): fp32 [BH, 64, 64]
+    // in the kernels' size -- the incoming state (it contains c), the gradient of the outgoing
+    // state, and where the gradient of the incoming state goes.
+    const float* state_in; const float* d_state_out; float* d_state_in;
     int bidir;      // 1: all-ones mask (bidirectional backward): both states are totals over the sequence
     int w_k, w_v;   // real columns of q, k, dq, dk and of v, dO, dv when fewer than 64 (0: 64)
 };

@@ -86,6 +86,13 @@ struct BwdParams {
     // token and head strides in elements.
     const int* cu_seqlens;
     void* out_rows[3]; long long out_sn[3], out_sh[3]; int out_w[3];
+    // A segment of a longer causal sequence (all three NULL otherwise), fp32 [BH, 64, 64] in the
+    // [key][value] layout of a caller's state: what earlier tokens left in the running state of
+    // Eq. 8 (it contains c), the gradient that later tokens send into the state this segment hands
+    // on, and where the gradient of state_in goes.  The dm sum is then taken over the value rows,
+    // <dV'_j, v_j>, which sees d_state_out and does not see state_in.
+    const float* state_in; const float* d_state_out; float* d_state_in;
+    int dm_by_v;
 };
 
 
@@ -345,6 +352,29 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     }
                 }
             }
+            if (!BIDIR) {
+                // Segment of a longer sequence: Sq starts from the caller's state (its transpose,
+                // without the factor c the state carries), R from the gradient of the outgoing state.
+                const float* extra = upper ? p.state_in : p.d_state_out;
+                if (extra != nullptr) {
+                    const float* eb = extra + (size_t)bh * kD * kD;
+                    const float f = upper ? 1.0f / cfac : 1.0f;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const int col = (wg & 1) * 32 + i;
+                        // upper: Sq[row = value index][col = key index] = state_in[col][row] / c;
+                        // lower: R[row = key index][col = value index] = d_state_out[row][col]
+                        acc[i] += f * (upper ? __ldg(eb + (size_t)col * kD + (row & 63)) : __ldg(eb + (size_t)(row & 63) * kD + col));
+                    }
+                }
+                // the first group's R is the sum over the whole segment plus d_state_out: d_state_in
+                if (!upper && g == 0 && p.d_state_in != nullptr) {
+                    float* db = p.d_state_in + (size_t)bh * kD * kD + (size_t)(row & 63) * kD + (wg & 1) * 32;
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4)
+                        *reinterpret_cast<float4*>(db + i) = make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
+                }
+            }
             if (BIDIR && g == 0) {
                 // dm of the bidirectional case needs no row sums at all: sum_i <q^_i, dO_i S^T> is
                 // the element-wise product of the two totals, <S, R>, formed here in fp32 from the
@@ -425,7 +455,8 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     if (!BIDIR && !wait_or_abort(bar(B_UFULL, c), par(c), abort_flag)) break;
                     mbar_expect_tx(fb, 4 * kTile);
                     coords(3, nrow, c1, c2); tma_load_4d(st + L::kOffDO, &tmDO, fb, 0, c1, c2, b);
-                    coords(2, nrow, c1, c2); tma_load_4d(st + L::kOffV, &tmV, fb, 0, c1, c2, b);
+                    // (dm over the value rows: the dV epilogue still reads the v tile)
+                    if (!p.dm_by_v) { coords(2, nrow, c1, c2); tma_load_4d(st + L::kOffV, &tmV, fb, 0, c1, c2, b); }
                     coords(0, nrow, c1, c2); tma_load_4d(st + L::kOffQ, &tmQ, fb, 0, c1, c2, b);
                     BSTAMP(7, c, 1);
                 }
@@ -435,6 +466,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 if (more) { coords(1, nrow, c1, c2); tma_load_4d(st + L::kOffK, &tmK, fb, 0, c1, c2, b); }
                 BSTAMP(7, c, 2);
                 if (!wait_or_abort(bar(B_EVDONE, c), par(c), abort_flag)) break;
+                if (more && p.dm_by_v) { coords(2, nrow, c1, c2); tma_load_4d(st + L::kOffV, &tmV, fb, 0, c1, c2, b); }
                 if (!by_rows) { coords(6, trow, c1, c2); tma_store_4d(&tmDV, base + L::kOffStQ, 0, c1, c2, b); }
                 tma_store_commit();
                 tma_store_wait_read1();
@@ -825,7 +857,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         const float corr = ((s01.x + s01.y) + (s23.x + s23.y)) * (1.f / 32768.f);
                         dm_acc += corr;
                         dot += corr;
-                    } else if (isq) {
+                    } else if (isq && !p.dm_by_v) {
                         dm_acc += dot;    // <q^_i, dQ^_i> of the unscaled accumulator (rows past N are zero)
                     }
                     // out = sc (a - coef x^), rounded to bf16 once
@@ -875,6 +907,24 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     tc_fence_before();
                     mbar_arrive(bar(B_OVFREE, c));     // the P columns may take the next chunk's scores
                     uint8_t* tile = gbase + L::kOffStQ;
+                    if (!BIDIR && p.dm_by_v && (long long)chunk_row(c) + row < tok1) {
+                        // dm of a segment: <dV'_j, v_j> of the unscaled accumulator with the raw v row
+                        // (the copy thread keeps the v tile until this epilogue is done)
+                        const uint8_t* vt = stage_g(c) + L::kOffV;
+                        float t0 = 0.f, t1 = 0.f;
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint4 w = *reinterpret_cast<const uint4*>(vt + swz(row, hw * 4 + j));
+                            const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&w);
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const float2 f = __bfloat1622float2(e[i]);
+                                t0 = fmaf(f.x, __uint_as_float(a[8 * j + 2 * i]), t0);
+                                t1 = fmaf(f.y, __uint_as_float(a[8 * j + 2 * i + 1]), t1);
+                            }
+                        }
+                        dm_acc += t0 + t1;
+                    }
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         uint4 o;
@@ -896,7 +946,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 mbar_arrive(bar(B_EVDONE, c));
                 BSTAMP(1 + hw, c, 4);
             }
-            if (isq || BIDIR) {
+            if (isq || BIDIR || p.dm_by_v) {
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) dm_acc += __shfl_xor_sync(0xffffffffu, dm_acc, o);
                 if (lane == 0) dm_red[(isq ? 0 : 12) + q4] = dm_acc;
@@ -915,7 +965,8 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 p.dm_partial[(size_t)bh * p.n_groups + g] = BIDIR ? ((dm_red[4] + dm_red[5]) + (dm_red[6] + dm_red[7])) +
                                                                           (((dm_red[0] + dm_red[1]) + (dm_red[2] + dm_red[3])) +
                                                                            ((dm_red[12] + dm_red[13]) + (dm_red[14] + dm_red[15])))
-                                                                  : (dm_red[0] + dm_red[1]) + (dm_red[2] + dm_red[3]);
+                                                                  : ((dm_red[0] + dm_red[1]) + (dm_red[2] + dm_red[3])) +
+                                                                        (p.dm_by_v ? (dm_red[12] + dm_red[13]) + (dm_red[14] + dm_red[15]) : 0.f);
             __threadfence();
             *last_flag = atomicAdd(&p.status[4], 1) == (int)gridDim.x - 1;
         }
@@ -1201,13 +1252,16 @@ cudaError_t launch_tc_bwd_fused(const TcBwdFusedArgs& a, int B, int H, int N, cu
         p.out_rows[i] = const_cast<void*>(ptrs[4 + i]); p.out_sn[i] = lo.sn; p.out_sh[i] = lo.sh; p.out_w[i] = dims[4 + i];
     }
     p.sq_part = a.sq_part; p.r_part = a.r_part; p.dm_partial = a.dm_partial; p.dm_out = a.dm_out;
+    const bool segment = !a.bidir && (a.state_in || a.d_state_out || a.d_state_in);
+    p.state_in = a.bidir ? nullptr : a.state_in; p.d_state_out = a.bidir ? nullptr : a.d_state_out;
+    p.d_state_in = a.bidir ? nullptr : a.d_state_in; p.dm_by_v = segment ? 1 : 0;
     p.status = a.status; p.m = a.m; p.seq_len = a.seq_len; p.seq_len_scalar = a.seq_len_scalar;
     p.H = H; p.N = N; p.group = a.group; p.n_groups = a.n_groups;
     p.wait_limit_kcycles = wait_limit_kcycles();
     p.sq_fwd = a.bidir ? nullptr : a.sq_fwd; p.sq_fwd_split = a.sq_fwd_split > 0 ? a.sq_fwd_split : 1;
     // One chunk per (b, h): nothing precedes it (Sq = 0) and nothing follows it (R = 0 once its own
     // update is taken out again), so the states stay zero and no partial-state pass is needed.
-    p.no_state = (!a.bidir && a.n_groups == 1 && N <= kC && !a.sq_part && !a.r_part) ? 1 : 0;
+    p.no_state = (!a.bidir && !segment && a.n_groups == 1 && N <= kC && !a.sq_part && !a.r_part) ? 1 : 0;
     if (!p.no_state && !a.r_part) return cudaErrorInvalidValue;
     auto kern = a.cu_seqlens ? (a.bidir ? tc_bwd_fused_kernel<true, true> : tc_bwd_fused_kernel<false, true>)
                              : (a.bidir ? tc_bwd_fused_kernel<true, false> : tc_bwd_fused_kernel<false, false>);

@@ -1005,6 +1005,78 @@ def test_short_blocks_many_heads(dtype, d):
     gate(o0, ref[:, :, :9], dtype)
 
 
+# ------------------------------------------------------------------ backward of segments
+@pytest.mark.parametrize("shape", [(2, 3, 200, 64, 64, 0), (1, 2, 1000, 64, 64, 256), (2, 2, 77, 32, 64, 0),
+                                   (1, 3, 300, 48, 24, 128), (2, 2, 128, 64, 64, 0)])
+def test_segment_backward_matches_the_definition(shape, force_group):
+    """cott_bwd_stateful on a segment with a caller's incoming state and a gradient flowing into the
+    outgoing one: dq, dk, dv, the gradient of the incoming state and dm against the definition
+    (states scaled like a real history: state_in from a forward over earlier tokens), with one and
+    with several groups, key / value sizes of their own, a single chunk."""
+    B, H, N, dk, dv, group = shape
+    if group:
+        force_group(group)
+    hist = synth.make_qkv(B, H, 150, dk, torch.bfloat16, 6300 + N, d_v=dv)
+    c = synth.make_qkv(B, H, N, dk, torch.bfloat16, 6400 + N + dk + dv, with_do=True, d_v=dv)
+    c["m"] = hist["m"]
+    s = np.full((B,), float(N + 150))
+    zero = np.zeros((B, H, dk, dv))
+    _, st_in = oracle.fwd_segment(hist["q"], hist["k"], hist["v"], hist["m"], zero, s)
+    d_st_out = np.random.default_rng(6500 + N).standard_normal((B, H, dk, dv)) * 0.5
+    rq, rk, rv, rst, rm = oracle.bwd_segment(c["q"], c["k"], c["v"], c["d_o"], c["m"], st_in, d_st_out, s)
+    q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
+    f32 = lambda a: torch.tensor(a, dtype=torch.float32, device="cuda")
+    dq, dk_, dv_, dst, dm = cott.bwd_stateful(q, k, v, d_o, m, float(N + 150), state_in=f32(st_in), d_state_out=f32(d_st_out))
+    gate(dq, rq, torch.bfloat16); gate(dk_, rk, torch.bfloat16); gate(dv_, rv, torch.bfloat16)
+    assert norm_max_err(dst, rst) <= TOL_STATE_TC    # (q^ enters the sum rounded to bf16, like every tensor-core state)
+    gate_dm(dm, rm, 1e-2, dm_condition(rv, c["v"], c["m"], s), DM_COND_BF16)
+    # without states it is the plain causal backward
+    a = cott.bwd_stateful(q, k, v, d_o, m, float(N + 150), return_d_state=False)
+    b = cott.bwd(q, k, v, d_o, m, seq_len=float(N + 150), causal=True)
+    for x, y in zip(a[:3], b[:3]):
+        assert float((x.float() - y.float()).abs().max()) <= TOL_BF16 * float(y.float().abs().max())
+
+
+def test_segment_backwards_chain_to_the_whole_sequence():
+    """Three segments forward (cott_fwd_stateful), then backward last to first with the state
+    gradients handed on: the gradients of one backward over the whole sequence (the definition),
+    dm the sum of the segments' parts."""
+    B, H, N, d = 2, 4, 900, 64
+    cuts = [(0, 256), (256, 600), (600, 900)]
+    c = synth.make_qkv(B, H, N, d, torch.bfloat16, 6600, with_do=True)
+    q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
+    seg = lambda x, a, b: x[:, :, a:b].contiguous()
+    states = [None]
+    for a, b in cuts:
+        _, st = cott.fwd_stateful(seg(q, a, b), seg(k, a, b), seg(v, a, b), m, float(N), state_in=states[-1])
+        states.append(st)
+    d_state = None
+    grads = []
+    dm = torch.zeros(H, device="cuda")
+    for (a, b), st_in in reversed(list(zip(cuts, states[:-1]))):
+        g = cott.bwd_stateful(seg(q, a, b), seg(k, a, b), seg(v, a, b), seg(d_o, a, b), m, float(N),
+                              state_in=st_in, d_state_out=d_state)
+        grads.append(g[:3])
+        d_state = g[3]
+        dm += g[4]
+    grads.reverse()
+    rq, rk, rv, rm = oracle.bwd_quadratic(c["q"], c["k"], c["v"], c["d_o"], c["m"], None, True)
+    for i, ref in enumerate((rq, rk, rv)):
+        gate(torch.cat([g[i] for g in grads], dim=2), ref, torch.bfloat16)
+    gate_dm(dm, rm, 1e-2, dm_condition(rv, c["v"], c["m"], None), DM_COND_BF16)
+
+
+def test_segment_backward_refuses_what_it_does_not_cover():
+    c = synth.make_qkv(1, 2, 64, 128, torch.bfloat16, 6700, with_do=True)
+    q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
+    with pytest.raises(cott.CottError):
+        cott.bwd_stateful(q, k, v, d_o, m, 64.0)                     # d = 128: not built
+    c = synth.make_qkv(1, 2, 64, 64, torch.bfloat16, 6701, with_do=True)
+    q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
+    with pytest.raises(cott.CottError):
+        cott.bwd_stateful(q, k, v, d_o, m, None)                     # no scaling base
+
+
 # ------------------------------------------------------------------ a wait that runs out
 @pytest.mark.parametrize("op", ["fwd", "bwd", "bidir", "bidir_bwd", "bidir_bwd_walk", "short", "block"])
 def test_bounded_wait_runs_out_and_reports(op, option, force_group):
