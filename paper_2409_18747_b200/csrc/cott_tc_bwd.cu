@@ -196,7 +196,10 @@ __device__ __forceinline__ void issue_update(uint32_t tS, uint32_t vq, uint32_t 
 //     dQ^ = dO S^T ,   dK^ = V R^T ,   dV' = K^ R ,
 // so the score products, the masks, the state update and the per-chunk state copies fall away;
 // loads, row norms, epilogues, stores and the dm sum are those of the causal walk.
-template <bool BIDIR, bool VARLEN>
+// SEG: a segment of a longer causal sequence (cott_bwd_stateful): the running states start from
+// the caller's, and dm is summed over the value rows.  An instance of its own, so that the plain
+// causal walk carries none of it.
+template <bool BIDIR, bool VARLEN, bool SEG = false>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                     const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmDO,
@@ -352,7 +355,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     }
                 }
             }
-            if (!BIDIR) {
+            if constexpr (SEG) {
                 // Segment of a longer sequence: Sq starts from the caller's state (its transpose,
                 // without the factor c the state carries), R from the gradient of the outgoing state.
                 const float* extra = upper ? p.state_in : p.d_state_out;
@@ -456,7 +459,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     mbar_expect_tx(fb, 4 * kTile);
                     coords(3, nrow, c1, c2); tma_load_4d(st + L::kOffDO, &tmDO, fb, 0, c1, c2, b);
                     // (dm over the value rows: the dV epilogue still reads the v tile)
-                    if (!p.dm_by_v) { coords(2, nrow, c1, c2); tma_load_4d(st + L::kOffV, &tmV, fb, 0, c1, c2, b); }
+                    if (!SEG) { coords(2, nrow, c1, c2); tma_load_4d(st + L::kOffV, &tmV, fb, 0, c1, c2, b); }
                     coords(0, nrow, c1, c2); tma_load_4d(st + L::kOffQ, &tmQ, fb, 0, c1, c2, b);
                     BSTAMP(7, c, 1);
                 }
@@ -466,7 +469,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 if (more) { coords(1, nrow, c1, c2); tma_load_4d(st + L::kOffK, &tmK, fb, 0, c1, c2, b); }
                 BSTAMP(7, c, 2);
                 if (!wait_or_abort(bar(B_EVDONE, c), par(c), abort_flag)) break;
-                if (more && p.dm_by_v) { coords(2, nrow, c1, c2); tma_load_4d(st + L::kOffV, &tmV, fb, 0, c1, c2, b); }
+                if (more && SEG) { coords(2, nrow, c1, c2); tma_load_4d(st + L::kOffV, &tmV, fb, 0, c1, c2, b); }
                 if (!by_rows) { coords(6, trow, c1, c2); tma_store_4d(&tmDV, base + L::kOffStQ, 0, c1, c2, b); }
                 tma_store_commit();
                 tma_store_wait_read1();
@@ -857,7 +860,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         const float corr = ((s01.x + s01.y) + (s23.x + s23.y)) * (1.f / 32768.f);
                         dm_acc += corr;
                         dot += corr;
-                    } else if (isq && !p.dm_by_v) {
+                    } else if (isq && !SEG) {
                         dm_acc += dot;    // <q^_i, dQ^_i> of the unscaled accumulator (rows past N are zero)
                     }
                     // out = sc (a - coef x^), rounded to bf16 once
@@ -907,7 +910,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     tc_fence_before();
                     mbar_arrive(bar(B_OVFREE, c));     // the P columns may take the next chunk's scores
                     uint8_t* tile = gbase + L::kOffStQ;
-                    if (!BIDIR && p.dm_by_v && (long long)chunk_row(c) + row < tok1) {
+                    if (SEG && (long long)chunk_row(c) + row < tok1) {
                         // dm of a segment: <dV'_j, v_j> of the unscaled accumulator with the raw v row
                         // (the copy thread keeps the v tile until this epilogue is done)
                         const uint8_t* vt = stage_g(c) + L::kOffV;
@@ -946,7 +949,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 mbar_arrive(bar(B_EVDONE, c));
                 BSTAMP(1 + hw, c, 4);
             }
-            if (isq || BIDIR || p.dm_by_v) {
+            if (isq || BIDIR || SEG) {
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) dm_acc += __shfl_xor_sync(0xffffffffu, dm_acc, o);
                 if (lane == 0) dm_red[(isq ? 0 : 12) + q4] = dm_acc;
@@ -966,7 +969,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                                                                           (((dm_red[0] + dm_red[1]) + (dm_red[2] + dm_red[3])) +
                                                                            ((dm_red[12] + dm_red[13]) + (dm_red[14] + dm_red[15])))
                                                                   : ((dm_red[0] + dm_red[1]) + (dm_red[2] + dm_red[3])) +
-                                                                        (p.dm_by_v ? (dm_red[12] + dm_red[13]) + (dm_red[14] + dm_red[15]) : 0.f);
+                                                                        (SEG ? (dm_red[12] + dm_red[13]) + (dm_red[14] + dm_red[15]) : 0.f);
             __threadfence();
             *last_flag = atomicAdd(&p.status[4], 1) == (int)gridDim.x - 1;
         }
@@ -1263,8 +1266,10 @@ cudaError_t launch_tc_bwd_fused(const TcBwdFusedArgs& a, int B, int H, int N, cu
     // update is taken out again), so the states stay zero and no partial-state pass is needed.
     p.no_state = (!a.bidir && !segment && a.n_groups == 1 && N <= kC && !a.sq_part && !a.r_part) ? 1 : 0;
     if (!p.no_state && !a.r_part) return cudaErrorInvalidValue;
-    auto kern = a.cu_seqlens ? (a.bidir ? tc_bwd_fused_kernel<true, true> : tc_bwd_fused_kernel<false, true>)
-                             : (a.bidir ? tc_bwd_fused_kernel<true, false> : tc_bwd_fused_kernel<false, false>);
+    if (segment && a.cu_seqlens) return cudaErrorInvalidValue;
+    auto kern = segment ? tc_bwd_fused_kernel<false, false, true>
+                        : a.cu_seqlens ? (a.bidir ? tc_bwd_fused_kernel<true, true> : tc_bwd_fused_kernel<false, true>)
+                                       : (a.bidir ? tc_bwd_fused_kernel<true, false> : tc_bwd_fused_kernel<false, false>);
     if (cudaError_t e = configure_smem_once(reinterpret_cast<const void*>(kern), L::kDynBytes); e != cudaSuccess)
         return e;
     const int prof = profile_begin_launch(3, st);
