@@ -314,12 +314,14 @@ def test_zero_query_rows_and_clamped_gradient():
 
 @pytest.mark.parametrize("d", [64, 128])
 @pytest.mark.parametrize("causal", [True, False])
-def test_clamped_gradient_on_tensor_core_path(d, causal, force_group):
+@pytest.mark.parametrize("group", [256, 4096])
+def test_clamped_gradient_on_tensor_core_path(d, causal, group, force_group):
     """bf16 through the tcgen05 kernels with one exactly-zero query row and one exactly-zero key
     row (in different chunks and groups): the forward gives a zero output row for the zero
     query; the gradient of a clamped row is the derivative of the clamped formula, dx = dx^ / eps
-    (order 1e12), compared relatively; every other row passes the usual gate."""
-    force_group(256)
+    (order 1e12), compared relatively; every other row passes the usual gate.  With several groups
+    per (b, h) and with one (at d = 64 the one-launch bidirectional kernels)."""
+    force_group(group)
     B, H, N = 1, 2, 700
     c = synth.make_qkv(B, H, N, d, torch.bfloat16, 4250 + d, with_do=True)
     c["q"][0, 0, 131] = 0.0
