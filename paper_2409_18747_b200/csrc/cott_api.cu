@@ -715,6 +715,29 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
         }
         return COTT_OK;
     }
+    // A segment of a longer sequence (cott_bwd_stateful): every stream's running sum starts from
+    // what lies outside the segment.  The dQ^ stream's sum is the caller's state transposed (these
+    // states contain c, as the caller's does), the dK^ stream's the transposed gradient of the
+    // outgoing state, the dV' stream's that gradient itself -- and its total is the gradient of
+    // the incoming state.  dm is summed over the value rows here, which is what a segment needs.
+    const float* seg_q = nullptr; const float* seg_k = nullptr; const float* seg_v = nullptr;
+    float* seg_total = nullptr;
+    if (seg.on) {
+        char* sbase = base + 3 * sb + 2 * align_up((size_t)B * H * p.n_groups * 4, 256);
+        const size_t ssb = segment_state_bytes(B, H, d);
+        if (seg.state_in) {
+            float* tbuf = reinterpret_cast<float*>(sbase);
+            COTT_CUDA(launch_transpose_state(seg.state_in, tbuf, BH, d, st));
+            seg_q = tbuf;
+        }
+        if (seg.d_state_out) {
+            float* tbuf = reinterpret_cast<float*>(sbase + ssb);
+            COTT_CUDA(launch_transpose_state(seg.d_state_out, tbuf, BH, d, st));
+            seg_k = tbuf;
+            seg_v = seg.d_state_out;
+        }
+        seg_total = seg.d_state_in;
+    }
     {   // dQ^_t = S_t dO_t : the forward walk with (dO, V', K^) in the roles of (Q, K, V)
         WalkArgs w = base_walk(sp, H, N, p);
         w.x = d_o; w.a = v; w.bv = k; w.proj = q; w.out = dq;
@@ -722,7 +745,7 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
         lay.assign(w);
         w.mode_x = ROW_RAW; w.mode_a = ROW_SCALE; w.mode_b = ROW_NORM;
         w.epilogue = EPI_PROJ; w.reverse = 0;
-        if ((rc = run_stream(w, p, BH, d, dt, causal, st0, nullptr, st)) != COTT_OK) return rc;
+        if ((rc = run_stream(w, p, BH, d, dt, causal, st0, nullptr, st, seg_q)) != COTT_OK) return rc;
     }
     {   // dK^_j = R_j v'_j : running sum of dO_t q^_t^T accumulated backward in time
         WalkArgs w = base_walk(sp, H, N, p);
@@ -731,7 +754,7 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
         lay.assign(w);
         w.mode_x = ROW_SCALE; w.mode_a = ROW_RAW; w.mode_b = ROW_NORM;
         w.epilogue = EPI_PROJ; w.reverse = 1;
-        if ((rc = run_stream(w, p, BH, d, dt, causal, st1, nullptr, st)) != COTT_OK) return rc;
+        if ((rc = run_stream(w, p, BH, d, dt, causal, st1, nullptr, st, seg_k)) != COTT_OK) return rc;
     }
     {   // dV'_j = R_j^T k^_j, dV = c dV', and <dV', V> for dm
         WalkArgs w = base_walk(sp, H, N, p);
@@ -740,7 +763,7 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
         lay.assign(w);
         w.mode_x = ROW_NORM; w.mode_a = ROW_NORM; w.mode_b = ROW_RAW;
         w.epilogue = EPI_DV; w.reverse = 1; w.dm_partial = dm_partial;
-        if ((rc = run_stream(w, p, BH, d, dt, causal, st2, nullptr, st)) != COTT_OK) return rc;
+        if ((rc = run_stream(w, p, BH, d, dt, causal, st2, seg_total, st, seg_v)) != COTT_OK) return rc;
     }
     COTT_CUDA(launch_dm_finalize(dm_partial, dm, sp->m, sp->seq_len, sp->seq_len_scalar, B, H,
                                  p.n_groups, N, st, packed.cu_seqlens));
@@ -981,7 +1004,14 @@ static cott_status bwd_entry(const void* q, const void* k, const void* v, const 
         // A segment needs the caller's scaling base (the same for every segment of a sequence), is
         // causal, and runs through the one-walk backward of the tensor-core path at sizes up to 64.
         if (!causal || (!sp->seq_len && !(sp->seq_len_scalar >= 1.f))) return COTT_ERR_INVALID_ARG;
-        if (p.path != 1 || p.d != 64 || option_fused_bwd() == 0) return COTT_ERR_UNSUPPORTED;
+        // Tensor cores: the one-walk backward at sizes up to 64.  Everything else the fp32-accumulating
+        // kernels cover (fp32, and bf16 at 128, with equal key and value sizes) goes through them, with
+        // the groups of the plan as it stands (the workspace was sized for it).
+        if (p.path == 1 && (p.d != 64 || option_fused_bwd() == 0)) {
+            if (!(d_k == d_v && (d_k == 32 || d_k == 64 || d_k == 128))) return COTT_ERR_UNSUPPORTED;
+            p.path = 0; p.chunk = 16; p.d = d_k; p.padded = false; p.split = 1;
+        }
+        if (qk_strides || v_strides || do_strides || dqk_strides || dv_strides) return COTT_ERR_UNSUPPORTED;
         if ((seg.state_in && !aligned16(seg.state_in)) || (seg.d_state_out && !aligned16(seg.d_state_out)) ||
             (seg.d_state_in && !aligned16(seg.d_state_in)))
             return COTT_ERR_UNSUPPORTED;

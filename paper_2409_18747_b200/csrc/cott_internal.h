@@ -205,6 +205,7 @@ cudaError_t launch_dm_finalize(const float* dm_partial, float* dm, const float* 
                                int n_groups, int N, cudaStream_t st, const int* cu_seqlens = nullptr);
 cudaError_t launch_sum_slices(const float* parts, float* out, int n, int H, cudaStream_t st);
 // Caller-visible states [BH, dk, dv] <-> the kernels' padded [BH, d, d] (zero outside).
+cudaError_t launch_transpose_state(const float* src, float* dst, int BH, int d, cudaStream_t st);
 cudaError_t launch_pad_state(const float* src, float* dst, int BH, int dk, int dv, int d, cudaStream_t st);
 cudaError_t launch_unpad_state(const float* src, float* dst, int BH, int dk, int dv, int d, cudaStream_t st);
 // Decode step for head sizes the specialised kernel does not cover (any dk, dv multiples of 4 / 8).

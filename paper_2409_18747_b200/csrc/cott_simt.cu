@@ -470,6 +470,20 @@ __global__ void unpad_state_kernel(const float* __restrict__ src, float* __restr
         dst[bh * dk * dv + i] = src[bh * d * d + (size_t)r * d + c];
     }
 }
+// dst[bh][c][r] = src[bh][r][c] for square d x d states.
+__global__ void transpose_state_kernel(const float* __restrict__ src, float* __restrict__ dst, int d) {
+    const size_t bh = blockIdx.y;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < d * d; i += gridDim.x * blockDim.x) {
+        const int r = i / d, c = i - r * d;
+        dst[bh * d * d + (size_t)c * d + r] = src[bh * d * d + i];
+    }
+}
+cudaError_t launch_transpose_state(const float* src, float* dst, int BH, int d, cudaStream_t st) {
+    dim3 grid((unsigned)((d * d + 1023) / 1024), (unsigned)BH);
+    transpose_state_kernel<<<grid, 256, 0, st>>>(src, dst, d);
+    note_launch();
+    return cudaGetLastError();
+}
 cudaError_t launch_pad_state(const float* src, float* dst, int BH, int dk, int dv, int d, cudaStream_t st) {
     dim3 grid((unsigned)((d * d + 1023) / 1024), (unsigned)BH);
     pad_state_kernel<<<grid, 256, 0, st>>>(src, dst, dk, dv, d);

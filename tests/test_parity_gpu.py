@@ -1068,11 +1068,39 @@ def test_segment_backwards_chain_to_the_whole_sequence():
     gate_dm(dm, rm, 1e-2, dm_condition(rv, c["v"], c["m"], None), DM_COND_BF16)
 
 
+@pytest.mark.parametrize("case", [(torch.float32, 32, 150, 0), (torch.float32, 64, 300, 64), (torch.float32, 128, 90, 0),
+                                  (torch.bfloat16, 128, 400, 128)])
+def test_segment_backward_through_the_fp32_accumulating_kernels(case, force_group):
+    """cott_bwd_stateful where the one-walk tensor-core backward does not reach: fp32 I/O, and
+    bf16 at head size 128 -- three running-sum walks whose sums start from the caller's state, the
+    transposed gradient of the outgoing state and that gradient itself."""
+    dtype, d, N, group = case
+    if group:
+        force_group(group)
+    B, H = 2, 3
+    hist = synth.make_qkv(B, H, 100, d, dtype, 6800 + d)
+    c = synth.make_qkv(B, H, N, d, dtype, 6810 + d + N, with_do=True)
+    c["m"] = hist["m"]
+    s = np.full((B,), float(N + 100))
+    _, st_in = oracle.fwd_segment(hist["q"], hist["k"], hist["v"], hist["m"], np.zeros((B, H, d, d)), s)
+    d_st_out = np.random.default_rng(6820 + d).standard_normal((B, H, d, d)) * 0.5
+    rq, rk, rv, rst, rm = oracle.bwd_segment(c["q"], c["k"], c["v"], c["d_o"], c["m"], st_in, d_st_out, s)
+    q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
+    f32 = lambda a: torch.tensor(a, dtype=torch.float32, device="cuda")
+    dq, dk_, dv_, dst, dm = cott.bwd_stateful(q, k, v, d_o, m, float(N + 100), state_in=f32(st_in), d_state_out=f32(d_st_out))
+    gate(dq, rq, dtype); gate(dk_, rk, dtype); gate(dv_, rv, dtype)
+    assert norm_max_err(dst, rst) <= (TOL_STATE_F32 if dtype == torch.float32 else TOL_STATE_TC)
+    if dtype == torch.float32:
+        gate_dm(dm, rm, 1e-4, dm_condition(rv, c["v"], c["m"], s), DM_COND_F32)
+    else:
+        gate_dm(dm, rm, 1e-2, dm_condition(rv, c["v"], c["m"], s), DM_COND_BF16)
+
+
 def test_segment_backward_refuses_what_it_does_not_cover():
-    c = synth.make_qkv(1, 2, 64, 128, torch.bfloat16, 6700, with_do=True)
+    c = synth.make_qkv(1, 2, 64, 96, torch.bfloat16, 6700, with_do=True)
     q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
     with pytest.raises(cott.CottError):
-        cott.bwd_stateful(q, k, v, d_o, m, 64.0)                     # d = 128: not built
+        cott.bwd_stateful(q, k, v, d_o, m, 64.0)                     # bf16 between 64 and 128: not built
     c = synth.make_qkv(1, 2, 64, 64, torch.bfloat16, 6701, with_do=True)
     q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
     with pytest.raises(cott.CottError):
