@@ -24,7 +24,11 @@
  *
  * All calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL is
  * the legacy default stream).  The returned status covers argument validation and
- * launch errors only.  Calls are thread-safe as long as concurrent calls use
+ * launch errors only.  cott_fwd*, cott_bwd* and cott_decode_step* with caller-owned outputs
+ * and workspaces put only kernel launches and memsets on the stream (and, where gradient streams
+ * run side by side, event-ordered work on the library's streams): once each kernel has been
+ * launched at least once on the device, such calls can be captured in a CUDA graph and
+ * replayed.  Calls are thread-safe as long as concurrent calls use
  * different workspaces.  Outputs must not share bytes with inputs or with each other:
  * equal pointers, dense tensors whose byte ranges meet, and equally strided tensors
  * (slices of one buffer) whose rows meet are refused with COTT_ERR_INVALID_ARG.

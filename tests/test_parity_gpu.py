@@ -1007,6 +1007,45 @@ def test_short_blocks_many_heads(dtype, d):
     gate(o0, ref[:, :, :9], dtype)
 
 
+# ------------------------------------------------------------------ stream capture
+@pytest.mark.parametrize("causal", [True, False])
+def test_a_training_step_can_be_captured_in_a_cuda_graph(causal):
+    """cott_fwd and cott_bwd with caller-owned outputs and workspaces issue only kernels (and one
+    memset) on the caller's stream: captured once in a CUDA graph and replayed, the step gives the
+    bits of the eager calls."""
+    B, H, N, d = 2, 6, 1500, 64
+    c = synth.make_qkv(B, H, N, d, torch.bfloat16, 6900, with_do=True)
+    q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
+    o = torch.empty_like(q)
+    outs = tuple(torch.empty_like(q) for _ in range(3))
+    wf = torch.zeros(cott.workspace_bytes(cott.cott.OP_FWD, cott.cott.BF16, B, H, N, d, causal), dtype=torch.uint8, device="cuda")
+    wb = torch.zeros(cott.workspace_bytes(cott.cott.OP_BWD, cott.cott.BF16, B, H, N, d, causal), dtype=torch.uint8, device="cuda")
+
+    def step():
+        cott.fwd(q, k, v, m, causal=causal, out=o, workspace=wf)
+        return cott.bwd(q, k, v, d_o, m, causal=causal, out=outs, workspace=wb)
+
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        for _ in range(2):
+            step()                       # (first calls configure the kernels: outside the capture)
+    torch.cuda.synchronize()
+    ref = [t.clone() for t in step()] + [o.clone()]
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        res = step()
+    torch.cuda.synchronize()
+    for t in outs + (o,):
+        t.zero_()
+    res[3].zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    for got, want in zip(list(res) + [o], ref):
+        assert torch.equal(got, want)
+    assert cott.cott.last_async_status(wf) == 0 and cott.cott.last_async_status(wb) == 0
+
+
 # ------------------------------------------------------------------ backward of segments
 @pytest.mark.parametrize("shape", [(2, 3, 200, 64, 64, 0), (1, 2, 1000, 64, 64, 256), (2, 2, 77, 32, 64, 0),
                                    (1, 3, 300, 48, 24, 128), (2, 2, 128, 64, 64, 0)])
