@@ -252,7 +252,8 @@ cott_status cott_bwd_strided(const void* q, const void* k, const void* v, const 
  * (causal != 0), with its own scaling base for Eq. 4: sp->seq_len[b], else sp->seq_len_scalar,
  * else its length.  No padding rows are read as keys or written as outputs.
  *   max_seqlen : an upper bound of the longest sequence (sizes the workspace and the plan)
- *   workspace  : cott_workspace_bytes(COTT_OP_FWD or COTT_OP_BWD, dt, B, H, max_seqlen, d, causal)
+ *   workspace  : cott_workspace_bytes_varlen(COTT_OP_FWD or COTT_OP_BWD, dt, B, H, total_tokens, max_seqlen, d, causal),
+ *                or at least cott_workspace_bytes(op, dt, B, H, max_seqlen, d, causal)
  * bf16 with d a multiple of 8 up to 128, or fp32 with d in {32, 64, 128} (COTT_ERR_UNSUPPORTED otherwise).  On the tensor-core
  * path a sequence is cut into the groups the dense plan for N = max_seqlen uses (group g = its rows g * group .. + group - 1,
  * as far as they exist), so a batch of few long sequences still fills the GPU; the fp32 kernels walk one (sequence, head) per CTA.  A NaN or Inf in the first
@@ -260,6 +261,17 @@ cott_status cott_bwd_strided(const void* q, const void* k, const void* v, const 
  * that holds both is multiplied by zeros, not skipped).  Other arguments, ordering and
  * aliasing rules as for cott_fwd / cott_bwd.
  */
+/*
+ * Workspace of cott_fwd_varlen / cott_bwd_varlen with room for the finer groups the library uses
+ * when the sum of the lengths is well below B * max_seqlen (a few long sequences among short ones:
+ * the group size then follows total_tokens, so that all groups of the batch still make about one
+ * wave of CTAs).  A workspace of cott_workspace_bytes(op, dt, B, H, max_seqlen, d, causal) bytes
+ * works as well: where that is less than the finer groups need, the calls use the groups of the
+ * dense plan for max_seqlen tokens.
+ */
+size_t cott_workspace_bytes_varlen(int op, cott_dtype dt, int B, int H, int total_tokens, int max_seqlen,
+                                   int d, int causal);
+
 cott_status cott_fwd_varlen(const void* q, const void* k, const void* v, void* o,
                             const int* cu_seqlens, int B, int H, int total_tokens, int max_seqlen,
                             int d, int causal, cott_dtype dt, const cott_scale_params* sp,

@@ -8,5 +8,5 @@ library or a missing GPU raises.
 from . import cott  # noqa: F401
 from .cott import (  # noqa: F401
     CottError, bwd, bwd_stateful, bwd_varlen, decode_step, fwd, fwd_bwd_host, fwd_noalloc, fwd_stateful, fwd_varlen,
-    library_path, query_plan, workspace_bytes,
+    library_path, query_plan, workspace_bytes, workspace_bytes_varlen,
 )

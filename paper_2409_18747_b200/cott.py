@@ -67,6 +67,8 @@ def _load():
     lib.cott_query_plan.argtypes = [ci] * 7 + [ctypes.POINTER(ci)] * 3
     lib.cott_workspace_bytes_dkdv.restype = cs
     lib.cott_workspace_bytes_dkdv.argtypes = [ci] * 8
+    lib.cott_workspace_bytes_varlen.restype = cs
+    lib.cott_workspace_bytes_varlen.argtypes = [ci] * 8
     lib.cott_query_plan_dkdv.restype = ci
     lib.cott_query_plan_dkdv.argtypes = [ci] * 8 + [ctypes.POINTER(ci)] * 4
     lib.cott_fwd_dkdv.restype = ci
@@ -289,6 +291,22 @@ def _workspace(op, dt, B, H, N, d, causal, device, workspace):
     return workspace, workspace.numel()
 
 
+def workspace_bytes_varlen(op, dt, B, H, total_tokens, max_seqlen, d, causal=True) -> int:
+    """cott_workspace_bytes_varlen: the workspace of a packed batch with room for groups sized by the
+    total token count."""
+    n = int(_load().cott_workspace_bytes_varlen(op, dt, B, H, int(total_tokens), int(max_seqlen), d, int(bool(causal))))
+    if n == _SIZE_MAX:
+        raise CottError(-2, "cott_workspace_bytes_varlen")
+    return n
+
+
+def _workspace_varlen(op, dt, B, H, T, max_seqlen, d, causal, device, workspace):
+    if workspace is None:
+        workspace = torch.empty(max(workspace_bytes_varlen(op, dt, B, H, T, max_seqlen, d, causal), 256),
+                                dtype=torch.uint8, device=device)
+    return workspace, workspace.numel()
+
+
 @_on_call_stream
 def fwd(q, k, v, m, seq_len=None, causal=True, return_state=False, out=None, workspace=None,
         stream=None):
@@ -439,7 +457,7 @@ def fwd_varlen(q, k, v, m, cu_seqlens, max_seqlen, seq_len=None, causal=True, ou
     B = cu_seqlens.numel() - 1
     dt = _dt(q)
     o = torch.empty_like(q) if out is None else out
-    ws, ws_bytes = _workspace(OP_FWD, dt, B, H, int(max_seqlen), d, causal, q.device, workspace)
+    ws, ws_bytes = _workspace_varlen(OP_FWD, dt, B, H, T, int(max_seqlen), d, causal, q.device, workspace)
     sp = _scale(m, seq_len)
     rc = _load().cott_fwd_varlen(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
                                  cu_seqlens.data_ptr(), B, H, T, int(max_seqlen), d, int(bool(causal)), dt,
@@ -460,7 +478,7 @@ def bwd_varlen(q, k, v, d_o, m, cu_seqlens, max_seqlen, seq_len=None, causal=Tru
     dt = _dt(q)
     dq, dk, dv = torch.empty_like(q), torch.empty_like(q), torch.empty_like(q)
     dm = torch.empty((H,), dtype=torch.float32, device=q.device)
-    ws, ws_bytes = _workspace(OP_BWD, dt, B, H, int(max_seqlen), d, causal, q.device, workspace)
+    ws, ws_bytes = _workspace_varlen(OP_BWD, dt, B, H, T, int(max_seqlen), d, causal, q.device, workspace)
     sp = _scale(m, seq_len)
     rc = _load().cott_bwd_varlen(q.data_ptr(), k.data_ptr(), v.data_ptr(), d_o.data_ptr(), dq.data_ptr(),
                                  dk.data_ptr(), dv.data_ptr(), dm.data_ptr(), cu_seqlens.data_ptr(), B, H, T,

@@ -855,6 +855,18 @@ size_t cott_workspace_bytes_dkdv(int op, cott_dtype dt, int B, int H, int N, int
     return workspace_bytes_impl(op, p, B, H, p.d);
 }
 
+static bool varlen_plan(int op, cott_dtype dt, int B, int H, int total_tokens, int max_seqlen, int d, int causal, Plan* p,
+                        size_t room);
+
+size_t cott_workspace_bytes_varlen(int op, cott_dtype dt, int B, int H, int total_tokens, int max_seqlen, int d, int causal) {
+    if (op != COTT_OP_FWD && op != COTT_OP_BWD) return (size_t)-1;
+    Plan coarse, fine;
+    if (!varlen_plan(op, dt, B, H, total_tokens, max_seqlen, d, causal, &coarse, 0)) return (size_t)-1;
+    if (!varlen_plan(op, dt, B, H, total_tokens, max_seqlen, d, causal, &fine, (size_t)-1)) return (size_t)-1;
+    const size_t a = workspace_bytes_impl(op, coarse, B, H, coarse.d), b = workspace_bytes_impl(op, fine, B, H, fine.d);
+    return a > b ? a : b;
+}
+
 size_t cott_workspace_bytes(int op, cott_dtype dt, int B, int H, int N, int d, int causal) {
     return cott_workspace_bytes_dkdv(op, dt, B, H, N, d, d, causal);
 }
@@ -1071,7 +1083,9 @@ cott_status cott_bwd_dkdv(const void* q, const void* k, const void* v, const voi
 }
 
 // Plan of a packed batch.
-static bool varlen_plan(int op, cott_dtype dt, int B, int H, int total_tokens, int max_seqlen, int d, int causal, Plan* p) {
+// `room`: bytes of workspace the caller has (0: the plan that the dense workspace query covers).
+static bool varlen_plan(int op, cott_dtype dt, int B, int H, int total_tokens, int max_seqlen, int d, int causal, Plan* p,
+                        size_t room) {
     if (B < 1 || H < 1 || total_tokens < 1 || max_seqlen < 1 || max_seqlen > total_tokens) return false;
     // bf16, tensor cores: any head size that is a multiple of 8 up to 128 (zero-filled tiles);
     // fp32 (and bf16 with force_path = 0): the fp32-accumulating SIMT kernels at 32, 64, 128
@@ -1089,6 +1103,21 @@ static bool varlen_plan(int op, cott_dtype dt, int B, int H, int total_tokens, i
         Plan dense;
         if (!make_plan(op, dt, B, H, max_seqlen, d, d, causal, &dense) || dense.path != 1) return false;
         p->group = dense.group; p->n_groups = dense.n_groups;
+        // That plan sizes the groups as if every sequence had max_seqlen tokens.  The lengths are on
+        // the device, but their sum is known: about total / G + B groups per head exist, and one
+        // wave holds 148 / H of them -- a smaller G when the batch is skewed (a few long sequences
+        // among short ones), as long as the caller's workspace has room for the states of
+        // max_seqlen / G groups per sequence (cott_workspace_bytes_varlen asks for it).
+        const long per_head = 148 / H - B;
+        if (option_force_group() <= 0 && per_head >= 1) {
+            long g = ((long)total_tokens + per_head - 1) / per_head;
+            g = (g + 127) / 128 * 128;
+            if (g < p->group) {
+                Plan fine = *p;
+                fine.group = (int)g; fine.n_groups = (max_seqlen + fine.group - 1) / fine.group;
+                if (room == (size_t)-1 || workspace_bytes_impl(op, fine, B, H, fine.d) <= room) *p = fine;
+            }
+        }
     }
     return true;
 }
@@ -1102,7 +1131,7 @@ cott_status cott_fwd_varlen(const void* q, const void* k, const void* v, void* o
     if (o == q || o == k || o == v) return COTT_ERR_INVALID_ARG;
     if (!sp->seq_len && sp->seq_len_scalar > 0.f && sp->seq_len_scalar < 1.f) return COTT_ERR_INVALID_ARG;
     Plan p;
-    if (!varlen_plan(COTT_OP_FWD, dt, B, H, total_tokens, max_seqlen, d, causal, &p)) return COTT_ERR_UNSUPPORTED;
+    if (!varlen_plan(COTT_OP_FWD, dt, B, H, total_tokens, max_seqlen, d, causal, &p, workspace ? workspace_bytes : 0)) return COTT_ERR_UNSUPPORTED;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return COTT_ERR_UNSUPPORTED;
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
         workspace_bytes < workspace_bytes_impl(COTT_OP_FWD, p, B, H, p.d))
@@ -1131,7 +1160,7 @@ cott_status cott_bwd_varlen(const void* q, const void* k, const void* v, const v
     }
     if (!sp->seq_len && sp->seq_len_scalar > 0.f && sp->seq_len_scalar < 1.f) return COTT_ERR_INVALID_ARG;
     Plan p;
-    if (!varlen_plan(COTT_OP_BWD, dt, B, H, total_tokens, max_seqlen, d, causal, &p)) return COTT_ERR_UNSUPPORTED;
+    if (!varlen_plan(COTT_OP_BWD, dt, B, H, total_tokens, max_seqlen, d, causal, &p, workspace ? workspace_bytes : 0)) return COTT_ERR_UNSUPPORTED;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(d_o) || !aligned16(dq) ||
         !aligned16(dk) || !aligned16(dv))
         return COTT_ERR_UNSUPPORTED;

@@ -1281,6 +1281,43 @@ def test_packed_varlen_with_several_groups_per_sequence(d, causal, group, force_
     _check_packed_batch(d, causal, (650, 1, 256, 257, 129, 900))
 
 
+@pytest.mark.parametrize("d", [64, 128])
+def test_packed_varlen_skewed_batch_uses_finer_groups(d):
+    """One long sequence among short ones: with the workspace of cott_workspace_bytes_varlen the
+    group size follows the total token count (more, shorter groups than the dense plan for
+    max_seqlen), with the dense query's workspace the dense groups -- both against the definition,
+    and the finer partition launches more CTAs for the long sequence (a different launch count is
+    not required, equal results within the bf16 tolerance are)."""
+    H, lens = 8, (3000, 200, 129, 64)
+    seqs = [synth.make_qkv(1, H, L, d, torch.bfloat16, 7000 + L, with_do=True) for L in lens]
+    for s_ in seqs:
+        s_["m"] = seqs[0]["m"]
+    cat = lambda key: torch.cat([s_[key][0].permute(1, 0, 2) for s_ in seqs], dim=0).contiguous().cuda()
+    q, k, v, d_o = (cat(x) for x in ("q", "k", "v", "d_o"))
+    cu = torch.tensor(np.concatenate([[0], np.cumsum(lens)]), dtype=torch.int32, device="cuda")
+    m = dev(seqs[0]["m"])
+    B, T, Lmax = len(lens), sum(lens), max(lens)
+    results = []
+    for fine in (True, False):
+        size = (lambda op: cott.workspace_bytes_varlen(op, cott.cott.BF16, B, H, T, Lmax, d, True)) if fine else \
+               (lambda op: cott.workspace_bytes(op, cott.cott.BF16, B, H, Lmax, d, True))
+        wf = torch.zeros(size(cott.cott.OP_FWD), dtype=torch.uint8, device="cuda")
+        wb = torch.zeros(size(cott.cott.OP_BWD), dtype=torch.uint8, device="cuda")
+        o = cott.fwd_varlen(q, k, v, m, cu, Lmax, causal=True, workspace=wf)
+        g = cott.bwd_varlen(q, k, v, d_o, m, cu, Lmax, causal=True, workspace=wb)
+        assert cott.cott.last_async_status(wf) == 0 and cott.cott.last_async_status(wb) == 0
+        results.append((o,) + tuple(g))
+    off = 0
+    for s_, L in zip(seqs, lens):
+        ref = oracle.fwd_quadratic(s_["q"], s_["k"], s_["v"], s_["m"], None, True)
+        rq, rk, rv, _ = oracle.bwd_quadratic(s_["q"], s_["k"], s_["v"], s_["d_o"], s_["m"], None, True)
+        un = lambda x: x[off:off + L].permute(1, 0, 2)[None]
+        for r in results:
+            gate(un(r[0]), ref, torch.bfloat16)
+            gate(un(r[1]), rq, torch.bfloat16); gate(un(r[2]), rk, torch.bfloat16); gate(un(r[3]), rv, torch.bfloat16)
+        off += L
+
+
 def _check_packed_batch(d, causal, lens):
     H = 3
     seqs = [synth.make_qkv(1, H, L, d, torch.bfloat16, 5800 + 7 * i + L, with_do=True) for i, L in enumerate(lens)]
