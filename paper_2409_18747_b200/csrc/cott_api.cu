@@ -475,12 +475,13 @@ static cott_status fwd_impl(const void* q, const void* k, const void* v, void* o
                                       sp->m, sp->seq_len, sp->seq_len_scalar, B, H, N, d, p.dk, p.dv, st));
         return finish();
     }
-    if (p.path == 1 && !causal && d == 64 && p.n_groups == 1 && !packed.cu_seqlens && !state_in &&
+    if (p.path == 1 && !causal && d == 64 && p.n_groups == 1 && !(packed.cu_seqlens && state_out) && !state_in &&
         option_fused_bidir() != 0) {
-        // One CTA per (b, h) streams k, v into the d x d state and then q through it: one launch,
-        // every tensor touched once.
+        // One CTA per (b, h) -- or per (sequence, head) of a packed batch -- streams k, v into the
+        // d x d state and then q through it: one launch, every tensor touched once.
         COTT_CUDA(launch_tc_bidir_fwd(q, k, v, o, lay.qkv, lay.of(v), lay.o, state_out, static_cast<int*>(ws), sp->m,
-                                      sp->seq_len, sp->seq_len_scalar, B, H, N, st, p.dk, p.dv));
+                                      sp->seq_len, sp->seq_len_scalar, B, H, N, st, p.dk, p.dv, packed.cu_seqlens,
+                                      packed.total_tokens));
         return finish();
     }
     if (p.path == 1) {

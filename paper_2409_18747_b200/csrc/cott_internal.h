@@ -164,7 +164,8 @@ cudaError_t launch_tc_pair_states(const void* a_rows, const void* b_rows, const 
 // the first (and only) kernel of its call and clears the status words itself.
 cudaError_t launch_tc_bidir_fwd(const void* q, const void* k, const void* v, void* o, const RowLayout& l_qkv,
                                 const RowLayout& l_v, const RowLayout& l_o, float* state_out, int* status, const float* m, const float* seq_len,
-                                float seq_len_scalar, int B, int H, int N, cudaStream_t st, int dk = 0, int dv = 0);
+                                float seq_len_scalar, int B, int H, int N, cudaStream_t st, int dk = 0, int dv = 0,
+                                const int* cu_seqlens = nullptr, int total_tokens = 0);
 
 // Tensor map over a bf16 tensor of logical shape [B,H,N,d] with the given row layout: box of
 // 128 tokens x 64 columns of one (b,h), 128-byte swizzle (see cott_tc_walk.cu).

@@ -43,8 +43,16 @@ struct BidirParams {
     int clear_status;
     int wait_limit_kcycles;
     int head_first_mask;     // bit i: in tensor map i (q, k, v, o) the head index comes before the token index
+    // Packed variable-length batch (NULL: dense): every tensor is [1, H, total_tokens, d], sequence
+    // b = rows cu_seqlens[b] .. cu_seqlens[b + 1] - 1, one CTA per (sequence, head).  The k rows of
+    // the next sequence in a ragged last chunk are normalised to zero (they then add nothing to
+    // the state), and that chunk's output rows leave as plain stores: o as global memory with its
+    // token and head strides in elements.
+    const int* cu_seqlens;
+    void* out_rows; long long out_sn, out_sh; int out_w;
 };
 
+template <bool VARLEN>
 __global__ void __launch_bounds__(kThreads, 3)
 tc_bidir_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                     const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO, BidirParams p) {
@@ -68,8 +76,13 @@ tc_bidir_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + L::kOffCtl + kCtlAbort);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int bh = blockIdx.x, b = bh / p.H, h = bh % p.H;
-    const int n_chunks = (p.N + kC - 1) / kC;
+    const int bh = blockIdx.x, bseq = bh / p.H, h = bh % p.H;
+    const int b = VARLEN ? 0 : bseq;                   // batch coordinate of the tensor maps
+    const int tok0 = VARLEN ? p.cu_seqlens[bseq] : 0;
+    const int tok1 = VARLEN ? p.cu_seqlens[bseq + 1] : p.N;
+    const int n_chunks = (tok1 - tok0 + kC - 1) / kC;
+    const bool ragged_last = VARLEN && ((tok1 - tok0) % kC) != 0;
+    auto chunk_row = [&](int c) { return tok0 + c * kC; };
     const bool is_mma = warp == kWorkerWarps, is_copy = warp == kWorkerWarps + 1;
 
     if (is_mma) {
@@ -111,7 +124,8 @@ tc_bidir_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (p.clear_status && blockIdx.x == 0 && tid < 8) p.status[tid] = 0;
 
-    const float s_b = p.seq_len ? p.seq_len[b] : (p.seq_len_scalar > 0.f ? p.seq_len_scalar : (float)p.N);
+    const float s_b = p.seq_len ? p.seq_len[bseq]
+                                : (p.seq_len_scalar > 0.f ? p.seq_len_scalar : (float)(VARLEN ? max(tok1 - tok0, 1) : p.N));
     const float cfac = stab_factor(p.m[h], s_b);
     auto par2 = [&](int c) { return (uint32_t)((c >> 1) & 1); };
     auto par4 = [&](int c) { return (uint32_t)((c >> 2) & 1); };
@@ -125,15 +139,17 @@ tc_bidir_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 if (c >= 2 && !wait_or_abort(bars + B_UFULL + 8 * (c & 1), par2(c - 2), abort_flag)) { ok = false; break; }
                 const uint32_t fb = bars + B_KVFULL + 8 * (c & 1), dst = base + (uint32_t)(2 * (c & 1)) * kTile;
                 mbar_expect_tx(fb, 2 * kTile);
-                load(dst, &tmK, 1, fb, c * kC);
-                load(dst + kTile, &tmV, 2, fb, c * kC);
+                load(dst, &tmK, 1, fb, chunk_row(c));
+                load(dst + kTile, &tmV, 2, fb, chunk_row(c));
             }
             // phase 2: q of chunk c into slot c & 3, once the slot's last reader is done: a (k, v)
             // pair of phase 1 (the state update of the last chunk with that parity), then the
             // store of the output rows of chunk c - 4, which were staged in the slot
             auto store = [&](int e) {
                 const bool hfo = (p.head_first_mask >> 3) & 1;
-                tma_store_4d(&tmO, base + (uint32_t)(e & 3) * kTile, 0, hfo ? h : e * kC, hfo ? e * kC : h, b);
+                // (the rows of a ragged last chunk of a packed batch were stored by the workers)
+                if (!(ragged_last && e == n_chunks - 1))
+                    tma_store_4d(&tmO, base + (uint32_t)(e & 3) * kTile, 0, hfo ? h : chunk_row(e), hfo ? chunk_row(e) : h, b);
                 tma_store_commit();
             };
             for (int c = 0; c < n_chunks && ok; ++c) {
@@ -147,7 +163,7 @@ tc_bidir_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 }
                 const uint32_t fb = bars + B_QFULL + 8 * (c & 3);
                 mbar_expect_tx(fb, kTile);
-                load(base + (uint32_t)(c & 3) * kTile, &tmQ, 0, fb, c * kC);
+                load(base + (uint32_t)(c & 3) * kTile, &tmQ, 0, fb, chunk_row(c));
                 // the output rows of chunk c - 2, if staged meanwhile, go out between the loads
                 if (c >= 2) {
                     const int e = c - 2;
@@ -213,6 +229,10 @@ tc_bidir_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             for (int j = 0; j < 8; ++j) w[j] = *reinterpret_cast<const uint4*>(tile + swz(row, j));
             float rn;
             normalise_row64(w, kEps, &rn);
+            if (VARLEN && chunk_row(c) + row >= tok1) {          // a row of the next sequence
+#pragma unroll
+                for (int j = 0; j < 8; ++j) w[j] = make_uint4(0u, 0u, 0u, 0u);
+            }
 #pragma unroll
             for (int j = 0; j < 8; ++j) *reinterpret_cast<uint4*>(tile + swz(row, j)) = w[j];
             fence_proxy_async();
@@ -285,7 +305,14 @@ tc_bidir_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 o.y = pack_bf16(__uint_as_float(a[8 * j + 2]) * rx, __uint_as_float(a[8 * j + 3]) * rx);
                 o.z = pack_bf16(__uint_as_float(a[8 * j + 4]) * rx, __uint_as_float(a[8 * j + 5]) * rx);
                 o.w = pack_bf16(__uint_as_float(a[8 * j + 6]) * rx, __uint_as_float(a[8 * j + 7]) * rx);
-                *reinterpret_cast<uint4*>(out + swz(row, hw * 4 + j)) = o;
+                if (VARLEN && ragged_last && c == n_chunks - 1) {
+                    const long long grow = (long long)chunk_row(c) + row;
+                    if (grow < tok1 && (hw * 4 + j) * 8 < p.out_w)
+                        *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out_rows) + grow * p.out_sn + (long long)h * p.out_sh +
+                                                  (hw * 4 + j) * 8) = o;
+                } else {
+                    *reinterpret_cast<uint4*>(out + swz(row, hw * 4 + j)) = o;
+                }
             }
             fence_proxy_async();
             mbar_arrive(bars + B_EDONE + 8 * (c & 3));
@@ -309,7 +336,8 @@ tc_bidir_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 
 cudaError_t launch_tc_bidir_fwd(const void* q, const void* k, const void* v, void* o, const RowLayout& l_qkv,
                                 const RowLayout& l_v, const RowLayout& l_o, float* state_out, int* status, const float* m, const float* seq_len,
-                                float seq_len_scalar, int B, int H, int N, cudaStream_t st, int dk, int dv) {
+                                float seq_len_scalar, int B, int H, int N, cudaStream_t st, int dk, int dv,
+                                const int* cu_seqlens, int total_tokens) {
     const void* ptrs[4] = {q, k, v, o};
     const RowLayout lays[4] = {l_qkv, l_qkv, l_v, l_o};
     // real column counts (<= 64): tiles are zero-filled beyond them and stores clipped
@@ -317,15 +345,24 @@ cudaError_t launch_tc_bidir_fwd(const void* q, const void* k, const void* v, voi
     CUtensorMap tm[4];
     BidirParams p;
     p.head_first_mask = 0;
+    // A packed batch is one tensor of total_tokens rows per head (batch extent 1).
+    const int map_B = cu_seqlens ? 1 : B, map_N = cu_seqlens ? total_tokens : N;
     for (int i = 0; i < 4; ++i) {
         bool hf = false;
-        if (dims[i] > kD || !make_tile_map(&tm[i], ptrs[i], B, H, N, dims[i], lays[i], &hf)) return cudaErrorInvalidValue;
+        if (dims[i] > kD || !make_tile_map(&tm[i], ptrs[i], map_B, H, map_N, dims[i], lays[i], &hf)) return cudaErrorInvalidValue;
         p.head_first_mask |= (hf ? 1 : 0) << i;
     }
+    p.cu_seqlens = cu_seqlens;
+    {
+        const RowLayout lo = resolve_layout(l_o, H, map_N, dims[3]);
+        p.out_rows = o; p.out_sn = lo.sn; p.out_sh = lo.sh; p.out_w = dims[3];
+    }
+    if (cu_seqlens && state_out) return cudaErrorInvalidValue;
     p.state_out = state_out; p.status = status; p.m = m; p.seq_len = seq_len; p.seq_len_scalar = seq_len_scalar;
     p.H = H; p.N = N; p.clear_status = 1;
     p.wait_limit_kcycles = wait_limit_kcycles();
-    if (cudaError_t e = configure_smem_once(reinterpret_cast<const void*>(tc_bidir_fwd_kernel), L::kDynBytes); e != cudaSuccess)
+    auto kern = cu_seqlens ? tc_bidir_fwd_kernel<true> : tc_bidir_fwd_kernel<false>;
+    if (cudaError_t e = configure_smem_once(reinterpret_cast<const void*>(kern), L::kDynBytes); e != cudaSuccess)
         return e;
     const int prof = profile_begin_launch(4, st);
     cudaLaunchConfig_t cfg = {};
@@ -337,8 +374,8 @@ cudaError_t launch_tc_bidir_fwd(const void* q, const void* k, const void* v, voi
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    cudaError_t le = cudaLaunchKernelEx(&cfg, tc_bidir_fwd_kernel, tm[0], tm[1], tm[2], tm[3], p);
+    cfg.numAttrs = cu_seqlens ? 0 : 1;      // (a packed batch reads cu_seqlens before anything else: a plain launch)
+    cudaError_t le = cudaLaunchKernelEx(&cfg, kern, tm[0], tm[1], tm[2], tm[3], p);
     profile_end_launch(prof, st);
     note_launch();
     return le != cudaSuccess ? le : cudaGetLastError();

@@ -1391,6 +1391,34 @@ def test_packed_varlen_leaves_neighbours_alone():
     assert torch.equal(alone, out[5:205])
 
 
+@pytest.mark.parametrize("d", [64, 40])
+def test_packed_varlen_bidirectional_forward_in_one_launch(d, force_group):
+    """A packed bidirectional batch with one group per sequence goes through the one-launch forward
+    kernel (d <= 64): every sequence against the definition, exactly the rows of the batch written
+    (ragged ends share tiles with the next sequence), an empty sequence in the middle."""
+    H, lens = 3, (5, 200, 0, 129, 128, 511)
+    force_group(4096)
+    seqs = [synth.make_qkv(1, H, L, d, torch.bfloat16, 7100 + L) if L else None for L in lens]
+    m_np = seqs[0]["m"]
+    cat = lambda key: torch.cat([s_[key][0].permute(1, 0, 2) for s_ in seqs if s_ is not None], dim=0).contiguous().cuda()
+    q, k, v = (cat(x) for x in ("q", "k", "v"))
+    T = sum(lens)
+    cu = torch.tensor(np.concatenate([[0], np.cumsum(lens)]), dtype=torch.int32, device="cuda")
+    out = torch.full((T + 40, H, d), 7.0, dtype=torch.bfloat16, device="cuda")
+    n0 = cott.cott.launch_count()
+    cott.fwd_varlen(q, k, v, dev(m_np), cu, max(lens), causal=False, out=out[:T])
+    assert cott.cott.launch_count() - n0 == 1
+    assert (out[T:] == 7.0).all()
+    assert not (out[:T] == 7.0).all(dim=-1).any()
+    off = 0
+    for s_, L in zip(seqs, lens):
+        if s_ is None:
+            continue
+        ref = oracle.fwd_quadratic(s_["q"], s_["k"], s_["v"], m_np, None, False)
+        gate(out[off:off + L].permute(1, 0, 2)[None], ref, torch.bfloat16)
+        off += L
+
+
 @pytest.mark.parametrize("causal", [True, False])
 def test_packed_varlen_gradients_leave_neighbours_alone(causal, option, force_group):
     """The one-launch backward of a packed batch (d = 64): the rows of a ragged last chunk leave as
