@@ -6,7 +6,7 @@ forward + backward, bf16 I/O with fp32 state, B=4 H=16 N=4096 d=64, synthetic N(
 tensors.  A step is one cott_fwd followed by one cott_bwd over one batch.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload c4|c2|c2-train|c3|c5:<N>|decode|c4-bnhd|varlen]
+                    [--workload c4|c2|c2-train|c3|c3-train|c5:<N>|decode|c4-bnhd|varlen]
 
 Prints ONE JSON line.  `value` is tokens/s with inputs resident in HBM; `e2e` is the same
 metric through the host-buffer entry point (host<->device copies inside the timed region);
@@ -54,6 +54,8 @@ def load_peaks():
 WORKLOADS = {
     "c4": dict(name="C4 causal fwd+bwd", B=4, H=16, N=4096, d=64, causal=True, bwd=True),
     "c3": dict(name="C3 causal fwd", B=8, H=12, N=1024, d=64, causal=True, bwd=False),
+    # C3 with its backward: one training step of a GPT-2-small attention layer
+    "c3-train": dict(name="C3 causal fwd+bwd", B=8, H=12, N=1024, d=64, causal=True, bwd=True),
     "c2": dict(name="C2 bidirectional fwd", B=32, H=12, N=512, d=64, causal=False, bwd=False),
     # the same shape with its backward: one training step of a BERT-base attention layer
     "c2-train": dict(name="C2 bidirectional fwd+bwd", B=32, H=12, N=512, d=64, causal=False, bwd=True),
