@@ -39,6 +39,8 @@ STEP_DRAM_TRAFFIC = {
     (64, True, True): 1563.3,     # C4 step: 409.8 MB over 262 144 token-heads (method's bytes: 1408)
     (64, False, False): 403.5,    # C2 forward: 79.3 MB over 196 608 token-heads (method's bytes: 512;
                                   # a third of the output is still in L2 when the kernel ends)
+    (64, False, True): 1160.3,    # C2 forward + backward: 79.3 + 148.8 MB (method's bytes: 1408; the backward's
+                                  # second pass over its inputs is served by L2, part of the gradients still there)
 }
 
 
