@@ -6,7 +6,7 @@ forward + backward, bf16 I/O with fp32 state, B=4 H=16 N=4096 d=64, synthetic N(
 tensors.  A step is one cott_fwd followed by one cott_bwd over one batch.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload c4|c2|c2-train|c3|c3-train|c5:<N>|decode|c4-bnhd|varlen]
+                    [--workload c4|c2|c2-train|c3|c3-train|c5:<N>|decode|c4-bnhd|varlen|varlen-small]
 
 Prints ONE JSON line.  `value` is tokens/s with inputs resident in HBM; `e2e` is the same
 metric through the host-buffer entry point (host<->device copies inside the timed region);
@@ -67,6 +67,9 @@ WORKLOADS = {
     # packed variable-length batch: 64 sequences of 512..2048 tokens (seeded), no padding rows
     "varlen": dict(name="packed varlen causal fwd+bwd, 64 sequences of 512..2048 tokens", B=64, H=16, N=2048,
                    d=128, causal=True, bwd=True, varlen=True),
+    # a quarter of it (0.65 GB of tensors, still several L2s): the case multi-counter profiler captures run on
+    "varlen-small": dict(name="packed varlen causal fwd+bwd, 16 sequences of 512..2048 tokens", B=16, H=16, N=2048,
+                         d=128, causal=True, bwd=True, varlen=True),
 }
 
 
@@ -555,7 +558,7 @@ def run_ours(args, w):
     plan = cott.query_plan(cott.cott.OP_BWD if w.get("bwd") else cott.cott.OP_FWD, dt_code, B, H, max(N, 1), d,
                            w["causal"]) if not w.get("decode") else {"path": 0, "group": 1, "chunk": 1}
     if w.get("varlen"):
-        plan = {"path": 1, "group": (N + 127) // 128 * 128, "chunk": 128, "groups": "one per (sequence, head)",
+        plan = {"path": 1, "chunk": 128, "groups": "the dense plan's for max_seqlen, or finer by the total token count",
                 "rows": w["rows"], "padded_rows": B * N}
     # Roofline of the step: the METHOD's bytes (forward: q, k, v in, o out = 8d per token-head;
     # backward: q, k, v, dO in, dq, dk, dv out = 14d; decode: the fp32 state in and out) over the

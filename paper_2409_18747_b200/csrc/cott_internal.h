@@ -75,7 +75,8 @@ struct TcWalkArgs {
     const void* x; const void* a; const void* bv; const void* proj; void* out;
     RowLayout lx, la, lbv, lproj, lout;   // layouts of the five tensors (all zero: dense)
     // Packed variable-length batch: device array of B + 1 row offsets into tensors that hold
-    // total_tokens rows per head (batch stride unused); one group per (b, h).  NULL: dense batch.
+    // total_tokens rows per head (batch stride unused); every sequence cut into groups from its first
+    // row on.  NULL: dense batch.
     const int* cu_seqlens; int total_tokens;
     const float* init; float* state_out; float* dm_partial; int* status;
     const float* dm_extra;   // the stream that finalises dm: the [BH, n_groups] part another stream summed, or NULL

@@ -51,11 +51,8 @@ struct TcWalkParams {
     int plain_launch;                   // host side only: launch without programmatic serialization
     int clear_status;                   // first kernel of a call: CTA 0 zeroes the status words
     int wait_limit_kcycles;             // bound of every wait, in units of 1024 SM cycles
-#ifdef COTT_TEST_HOOKS
-    int debug_drop_commit;              // test builds only: the scores of chunk 1 are never reported complete
-#endif
     // Packed variable-length batch: rows of all sequences back to back in one [T, H, d]
-    // tensor, sequence b = rows cu_seqlens[b] .. cu_seqlens[b+1]-1, one group per (b, h).
+    // tensor, sequence b = rows cu_seqlens[b] .. cu_seqlens[b+1]-1, cut into groups from its first row on.
     const int* cu_seqlens;              // NULL: every (b, h) has N rows of its own
     void* out_rows; long long out_sn, out_sh;   // Out as plain global memory (rows of a ragged last chunk)
     int head_first_mask;                // bit i: in tensor map i (X, A, Bv, raw rows, Out) the head index
@@ -599,9 +596,6 @@ tc_walk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 const int s = c % NST;
                 tc_fence_after();
                 issue_p<D>(tmem + colP, stage_x(s), stage_a(s));
-                #ifdef COTT_TEST_HOOKS
-                if (!(p.debug_drop_commit && c == 1))
-#endif
                 tc_commit(bar_p_full);
             };
             auto batch1 = [&](int c, bool scores_issued) {
@@ -1376,12 +1370,6 @@ cudaError_t launch_tc_walk(const TcWalkArgs& a, int B, int H, int N, int d, cuda
     p.plain_launch = a.plain_launch || a.cu_seqlens != nullptr;
     p.clear_status = a.clear_status;
     p.wait_limit_kcycles = wait_limit_kcycles();
-#ifdef COTT_TEST_HOOKS
-    {   // test builds only: a hand-off that never comes (the scores of chunk 1 are never reported complete)
-        const char* e = getenv("COTT_DEBUG_DROP_COMMIT");
-        p.debug_drop_commit = (e && *e == '1') ? 1 : 0;
-    }
-#endif
     if (p.first_group < 0 || p.first_group + p.grid_groups > a.n_groups) return cudaErrorInvalidValue;
     // The four combinations of roles the library uses, as compile-time kernel variants.
     int kind;
