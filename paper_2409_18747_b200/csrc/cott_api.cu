@@ -645,10 +645,11 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
         }
         SideStreams* ss = nullptr;
         Plan pp = p;                       // plan of the two side-by-side streams
-        // (d = 64 only: at d = 128 two such walks running at the same time ended in a launch
-        // failure once in a dozen calls, for a reason that reading the kernel has not shown;
-        // one after the other the same kernels have run hundreds of thousands of times.)
-        if (causal && d == 64 && p.n_groups >= 2 && 2 * BH <= 148 && 74 / BH == 1 && option_pair() != 0) {
+        // (d = 64 only: at d = 128 two such walks running at the same time once ended in launch
+        // failures -- a transaction barrier of the raw-row tile was re-armed before its phase had
+        // completed; it has one barrier per chunk parity since -- and the concurrent form has not
+        // been switched on again there.)
+        if (causal && !seg.on && d == 64 && p.n_groups >= 2 && 2 * BH <= 148 && 74 / BH == 1 && option_pair() != 0) {
             pp.group = (N + 127) / 128 * 128;
             pp.n_groups = 1; pp.split = 1;
             ss = side_streams();
@@ -673,6 +674,50 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
         tq.dm_out = dm;
         lay.assign(tq); lay.assign(tk); lay.assign(tv);
         lay.assign_widths(tq); lay.assign_widths(tk); lay.assign_widths(tv);
+        if (seg.on) {
+            // A segment at head size 128 (cott_bwd_stateful) through the three walks.  Each stream's
+            // running sum starts from what lies outside the segment, in that stream's layout and
+            // scale (the walks divide an initial state by c, as they do with a caller's forward
+            // state): the dQ^ stream from state_in^T, the dK^ stream from c d_state_out^T; the dV'
+            // stream reuses the dK^ stream's scanned states (with one group, where nothing is
+            // shared, it starts from c d_state_out).  The totals of the first two give
+            // d_state_in and the two terms by which the dm sum over the query rows is off
+            // (segment_finish_kernel); dm is finalised after that.
+            char* sbase = base + 3 * sb + 2 * align_up((size_t)B * H * p.n_groups * 4, 256);
+            const size_t ssb = segment_state_bytes(B, H, d);
+            float* b_q = reinterpret_cast<float*>(sbase);
+            float* b_k = reinterpret_cast<float*>(sbase + ssb);
+            float* tk_tot = reinterpret_cast<float*>(sbase + 2 * ssb);
+            float* tq_tot = st2;           // (the third states region is free: dV' has no state pass of its own)
+            float* b_v = st0;              // (one group: no stream has a state pass, the regions are free)
+            const bool one = p.n_groups == 1;
+            if (seg.state_in)
+                COTT_CUDA(launch_state_prep(seg.state_in, b_q, BH, d, 1, 0, sp->m, sp->seq_len, sp->seq_len_scalar, H, N, st));
+            if (seg.d_state_out) {
+                COTT_CUDA(launch_state_prep(seg.d_state_out, b_k, BH, d, 1, 1, sp->m, sp->seq_len, sp->seq_len_scalar, H, N, st));
+                if (one) COTT_CUDA(launch_state_prep(seg.d_state_out, b_v, BH, d, 0, 1, sp->m, sp->seq_len, sp->seq_len_scalar, H, N, st));
+            }
+            tk.clear_status = 1; tq.clear_status = 0;
+            tk.dm_partial = dm_partial2; tk.dm_out = nullptr;
+            tq.dm_partial = dm_partial; tq.dm_out = nullptr; tq.dm_extra = nullptr;
+            if ((rc = run_tc_stream(tk, p, B, H, N, d, causal, sp, status, st1, tk_tot, st, false, false, true,
+                                    seg.d_state_out ? b_k : nullptr)) != COTT_OK) return rc;
+            if ((rc = run_tc_stream(tq, p, B, H, N, d, causal, sp, status, one ? st1 : st0, tq_tot, st, false, false, true,
+                                    seg.state_in ? b_q : nullptr)) != COTT_OK) return rc;
+            if (one) {
+                if ((rc = run_tc_stream(tv, p, B, H, N, d, causal, sp, status, st1, nullptr, st, false, false, true,
+                                        seg.d_state_out ? b_v : nullptr)) != COTT_OK) return rc;
+            } else {
+                // (the states were scanned by the dK^ stream's scan launch: the non-null last
+                // argument keeps this call from summing them itself)
+                if ((rc = run_tc_stream(tv, p, B, H, N, d, causal, sp, status, st1, nullptr, st, true, false, true, b_k)) != COTT_OK)
+                    return rc;
+            }
+            COTT_CUDA(launch_segment_finish(seg.state_in, seg.d_state_out, tq_tot, tk_tot, seg.d_state_in, dm_partial, dm_partial2,
+                                            BH, p.n_groups, d, sp->m, sp->seq_len, sp->seq_len_scalar, H, N, st));
+            COTT_CUDA(launch_dm_finalize(dm_partial, dm, sp->m, sp->seq_len, sp->seq_len_scalar, B, H, p.n_groups, N, st, nullptr));
+            return COTT_OK;
+        }
         if (ss) {
             struct TagScope { ~TagScope() { g_prof_cur_tag = 0; } } tag_scope;
             // Everything that follows a cross-stream event wait is a plain launch.
@@ -1017,10 +1062,12 @@ static cott_status bwd_entry(const void* q, const void* k, const void* v, const 
         // A segment needs the caller's scaling base (the same for every segment of a sequence), is
         // causal, and runs through the one-walk backward of the tensor-core path at sizes up to 64.
         if (!causal || (!sp->seq_len && !(sp->seq_len_scalar >= 1.f))) return COTT_ERR_INVALID_ARG;
-        // Tensor cores: the one-walk backward at sizes up to 64.  Everything else the fp32-accumulating
-        // kernels cover (fp32, and bf16 at 128, with equal key and value sizes) goes through them, with
-        // the groups of the plan as it stands (the workspace was sized for it).
-        if (p.path == 1 && (p.d != 64 || option_fused_bwd() == 0)) {
+        // Tensor cores: the one-walk backward at sizes up to 64, the three walks at 128.  Everything
+        // else the fp32-accumulating kernels cover (equal key and value sizes of 32, 64 or 128) goes
+        // through them, with the groups of the plan as it stands (the workspace was sized for it).
+        const bool tc_fused = p.path == 1 && p.d == 64 && option_fused_bwd() != 0;
+        const bool tc_walks = p.path == 1 && p.d == 128 && d_k == 128 && d_v == 128 && option_force_path() != 0;
+        if (p.path == 1 && !tc_fused && !tc_walks) {
             if (!(d_k == d_v && (d_k == 32 || d_k == 64 || d_k == 128))) return COTT_ERR_UNSUPPORTED;
             p.path = 0; p.chunk = 16; p.d = d_k; p.padded = false; p.split = 1;
         }

@@ -208,6 +208,11 @@ cudaError_t launch_dm_finalize(const float* dm_partial, float* dm, const float* 
 cudaError_t launch_sum_slices(const float* parts, float* out, int n, int H, cudaStream_t st);
 // Caller-visible states [BH, dk, dv] <-> the kernels' padded [BH, d, d] (zero outside).
 cudaError_t launch_transpose_state(const float* src, float* dst, int BH, int d, cudaStream_t st);
+cudaError_t launch_state_prep(const float* src, float* dst, int BH, int d, int transpose, int scale_mode, const float* m,
+                              const float* seq_len, float seq_len_scalar, int H, int N, cudaStream_t st);
+cudaError_t launch_segment_finish(const float* state_in, const float* d_state_out, const float* tq_total, const float* tk_total,
+                                  float* d_state_in, float* dm_partial, const float* fold, int BH, int n_groups, int d,
+                                  const float* m, const float* seq_len, float seq_len_scalar, int H, int N, cudaStream_t st);
 cudaError_t launch_pad_state(const float* src, float* dst, int BH, int dk, int dv, int d, cudaStream_t st);
 cudaError_t launch_unpad_state(const float* src, float* dst, int BH, int dk, int dv, int d, cudaStream_t st);
 // Decode step for head sizes the specialised kernel does not cover (any dk, dv multiples of 4 / 8).

@@ -484,6 +484,81 @@ cudaError_t launch_transpose_state(const float* src, float* dst, int BH, int d, 
     note_launch();
     return cudaGetLastError();
 }
+// dst = src (transposed if asked) times c[b,h] (scale_mode 1), divided by it (2) or as is (0):
+// a caller's square state brought into the layout and scale a tensor-core stream starts from.
+__global__ void state_prep_kernel(const float* __restrict__ src, float* __restrict__ dst, int d, int transpose, int scale_mode,
+                                  const float* m, const float* seq_len, float seq_len_scalar, int H, int N) {
+    const size_t bh = blockIdx.y;
+    float f = 1.f;
+    if (scale_mode) {
+        const float s_b = seq_len ? seq_len[bh / H] : (seq_len_scalar > 0.f ? seq_len_scalar : (float)N);
+        const float c = stab_factor(m[bh % H], s_b);
+        f = scale_mode == 1 ? c : 1.0f / c;
+    }
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < d * d; i += gridDim.x * blockDim.x) {
+        const int r = i / d, c2 = i - r * d;
+        dst[bh * d * d + (transpose ? (size_t)c2 * d + r : (size_t)i)] = src[bh * d * d + i] * f;
+    }
+}
+cudaError_t launch_state_prep(const float* src, float* dst, int BH, int d, int transpose, int scale_mode, const float* m,
+                              const float* seq_len, float seq_len_scalar, int H, int N, cudaStream_t st) {
+    dim3 grid((unsigned)((d * d + 1023) / 1024), (unsigned)BH);
+    state_prep_kernel<<<grid, 256, 0, st>>>(src, dst, d, transpose, scale_mode, m, seq_len, seq_len_scalar, H, N);
+    note_launch();
+    return cudaGetLastError();
+}
+
+// Backward of a segment through the three tensor-core walks: what the streams' totals give.
+//   tq_total [d_v][d_k] = state_in^T + c V^T K^        (the dQ^ stream's final sum, scaled)
+//   tk_total [d_v][d_k] = c (d_state_out + Q^^T dO)^T  (the dK^ stream's)
+// With S = K^^T V and R = Q^^T dO of the segment:
+//   d_state_in = d_state_out + R = tk_total^T / c
+//   the dm sum over the query rows, <q^_i, dQ^_i>, contains q^_i^T (state_in / c) dO_i, which is no
+//   derivative with respect to c, and lacks <d_state_out, S>:  T = T_q - <state_in / c, R> + <d_state_out, S>.
+// One CTA per (b, h); the correction (and the dK^ stream's partial sums `fold`, if any) is added to
+// dm_partial[bh * n_groups], which the dm finaliser sums afterwards.
+__global__ void __launch_bounds__(256) segment_finish_kernel(const float* __restrict__ state_in, const float* __restrict__ d_state_out,
+                                                             const float* __restrict__ tq_total, const float* __restrict__ tk_total,
+                                                             float* __restrict__ d_state_in, float* dm_partial, const float* fold,
+                                                             int n_groups, int d, const float* m, const float* seq_len,
+                                                             float seq_len_scalar, int H, int N) {
+    const size_t bh = blockIdx.x;
+    const float s_b = seq_len ? seq_len[bh / H] : (seq_len_scalar > 0.f ? seq_len_scalar : (float)N);
+    const float ic = 1.0f / stab_factor(m[bh % H], s_b);
+    const size_t o = bh * (size_t)d * d;
+    float acc = 0.f;
+    for (int i = threadIdx.x; i < d * d; i += blockDim.x) {
+        const int a = i / d, b = i - a * d;                    // element [a][b] of a [d_k][d_v] state
+        const size_t t = o + (size_t)b * d + a;                // its place in a transposed total
+        const float dsi = tk_total[t] * ic;                    // d_state_out + R
+        const float dso = d_state_out ? d_state_out[o + i] : 0.f;
+        const float sin = state_in ? state_in[o + i] : 0.f;
+        if (d_state_in) d_state_in[o + i] = dsi;
+        const float r = dsi - dso, sl = (tq_total[t] - sin) * ic;
+        acc += dso * sl - sin * ic * r;
+    }
+    __shared__ float red[8];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float t = 0.f;
+        for (int w = 0; w < 8; ++w) t += red[w];
+        float f = 0.f;
+        if (fold) for (int g = 0; g < n_groups; ++g) f += fold[bh * n_groups + g];
+        dm_partial[bh * n_groups] += t + f;
+    }
+}
+cudaError_t launch_segment_finish(const float* state_in, const float* d_state_out, const float* tq_total, const float* tk_total,
+                                  float* d_state_in, float* dm_partial, const float* fold, int BH, int n_groups, int d,
+                                  const float* m, const float* seq_len, float seq_len_scalar, int H, int N, cudaStream_t st) {
+    segment_finish_kernel<<<(unsigned)BH, 256, 0, st>>>(state_in, d_state_out, tq_total, tk_total, d_state_in, dm_partial, fold,
+                                                        n_groups, d, m, seq_len, seq_len_scalar, H, N);
+    note_launch();
+    return cudaGetLastError();
+}
+
 cudaError_t launch_pad_state(const float* src, float* dst, int BH, int dk, int dv, int d, cudaStream_t st) {
     dim3 grid((unsigned)((d * d + 1023) / 1024), (unsigned)BH);
     pad_state_kernel<<<grid, 256, 0, st>>>(src, dst, dk, dv, d);

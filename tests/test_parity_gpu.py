@@ -1078,11 +1078,12 @@ def test_segment_backward_matches_the_definition(shape, force_group):
         assert float((x.float() - y.float()).abs().max()) <= TOL_BF16 * float(y.float().abs().max())
 
 
-def test_segment_backwards_chain_to_the_whole_sequence():
+@pytest.mark.parametrize("d", [64, 128])
+def test_segment_backwards_chain_to_the_whole_sequence(d):
     """Three segments forward (cott_fwd_stateful), then backward last to first with the state
     gradients handed on: the gradients of one backward over the whole sequence (the definition),
     dm the sum of the segments' parts."""
-    B, H, N, d = 2, 4, 900, 64
+    B, H, N = 2, 4, 900
     cuts = [(0, 256), (256, 600), (600, 900)]
     c = synth.make_qkv(B, H, N, d, torch.bfloat16, 6600, with_do=True)
     q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
@@ -1107,15 +1108,21 @@ def test_segment_backwards_chain_to_the_whole_sequence():
     gate_dm(dm, rm, 1e-2, dm_condition(rv, c["v"], c["m"], None), DM_COND_BF16)
 
 
-@pytest.mark.parametrize("case", [(torch.float32, 32, 150, 0), (torch.float32, 64, 300, 64), (torch.float32, 128, 90, 0),
-                                  (torch.bfloat16, 128, 400, 128)])
-def test_segment_backward_through_the_fp32_accumulating_kernels(case, force_group):
-    """cott_bwd_stateful where the one-walk tensor-core backward does not reach: fp32 I/O, and
-    bf16 at head size 128 -- three running-sum walks whose sums start from the caller's state, the
-    transposed gradient of the outgoing state and that gradient itself."""
-    dtype, d, N, group = case
+@pytest.mark.parametrize("case", [(torch.float32, 32, 150, 0, 1), (torch.float32, 64, 300, 64, 1), (torch.float32, 128, 90, 0, 1),
+                                  (torch.bfloat16, 128, 400, 128, 0),
+                                  (torch.bfloat16, 128, 400, 128, 1), (torch.bfloat16, 128, 1000, 4096, 1), (torch.bfloat16, 128, 130, 0, 1)])
+def test_segment_backward_through_three_walks(case, force_group, option):
+    """cott_bwd_stateful where the one-walk tensor-core backward does not reach -- three running-sum
+    walks whose sums start from the caller's state (transposed), the transposed gradient of the
+    outgoing state and that gradient itself: the fp32-accumulating kernels for fp32 I/O (and, with
+    force_path = 0, bf16), the tensor-core walks for bf16 at head size 128 (several groups, one
+    group, a ragged second chunk), where the totals of two streams give the gradient of the
+    incoming state and correct the dm sum."""
+    dtype, d, N, group, tensor_cores = case
     if group:
         force_group(group)
+    if not tensor_cores:
+        option("force_path", 0)
     B, H = 2, 3
     hist = synth.make_qkv(B, H, 100, d, dtype, 6800 + d)
     c = synth.make_qkv(B, H, N, d, dtype, 6810 + d + N, with_do=True)
