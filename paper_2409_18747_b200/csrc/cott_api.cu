@@ -612,14 +612,19 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
                 float* s_in = reinterpret_cast<float*>(sbase);
                 float* ds_out = reinterpret_cast<float*>(sbase + ssb);
                 float* ds_in = reinterpret_cast<float*>(sbase + 2 * ssb);
-                if (seg.state_in) COTT_CUDA(launch_pad_state(seg.state_in, s_in, BH, p.dk, p.dv, d, st));
-                if (seg.d_state_out) COTT_CUDA(launch_pad_state(seg.d_state_out, ds_out, BH, p.dk, p.dv, d, st));
-                f.state_in = seg.state_in ? s_in : nullptr;
-                f.d_state_out = seg.d_state_out ? ds_out : nullptr;
-                f.d_state_in = seg.d_state_in ? ds_in : nullptr;
+                if (!p.padded) {
+                    // (states of the kernels' own size: read and written where the caller has them)
+                    f.state_in = seg.state_in; f.d_state_out = seg.d_state_out; f.d_state_in = seg.d_state_in;
+                } else {
+                    if (seg.state_in) COTT_CUDA(launch_pad_state(seg.state_in, s_in, BH, p.dk, p.dv, d, st));
+                    if (seg.d_state_out) COTT_CUDA(launch_pad_state(seg.d_state_out, ds_out, BH, p.dk, p.dv, d, st));
+                    f.state_in = seg.state_in ? s_in : nullptr;
+                    f.d_state_out = seg.d_state_out ? ds_out : nullptr;
+                    f.d_state_in = seg.d_state_in ? ds_in : nullptr;
+                }
                 COTT_CUDA(launch_tc_bwd_states(f, st0, st1, 1, B, H, N, st));
                 COTT_CUDA(launch_tc_bwd_fused(f, B, H, N, st));
-                if (seg.d_state_in) COTT_CUDA(launch_unpad_state(ds_in, seg.d_state_in, BH, p.dk, p.dv, d, st));
+                if (p.padded && seg.d_state_in) COTT_CUDA(launch_unpad_state(ds_in, seg.d_state_in, BH, p.dk, p.dv, d, st));
                 return COTT_OK;
             }
             if (causal && !packed.cu_seqlens && p.n_groups == 1 && N <= 128) {
