@@ -332,9 +332,9 @@ cott_status cott_bwd_after_fwd(const void* q, const void* k, const void* v, cons
  * Run over the segments last to first, with the caller's scaling base (sp->seq_len or
  * sp->seq_len_scalar >= 1, the same for every segment), the calls give the gradients of one
  * cott_bwd over the whole sequence.  Dense [B,H,N,d] tensors.  bf16 with d_k, d_v multiples of 8 up
- * to 64: the one-walk backward of the tensor-core path.  bf16 with d_k = d_v = 128: the three
- * tensor-core walks.  fp32 with d_k = d_v in {32, 64, 128}: three running-sum walks of the
- * fp32-accumulating kernels.  COTT_ERR_UNSUPPORTED otherwise.
+ * to 64: the one-walk backward of the tensor-core path.  bf16 with larger sizes (multiples of 8 up
+ * to 128): the three tensor-core walks.  fp32 with d_k = d_v in {32, 64, 128}: three running-sum
+ * walks of the fp32-accumulating kernels.  COTT_ERR_UNSUPPORTED otherwise.
  * workspace: cott_workspace_bytes_dkdv(COTT_OP_BWD, dt, B, H, N, d_k, d_v, 1).
  */
 cott_status cott_bwd_stateful(const void* q, const void* k, const void* v, const void* d_o,

@@ -216,7 +216,7 @@ static size_t workspace_bytes_impl(int op, const Plan& p, int B, int H, int d) {
     if (op == COTT_OP_FWD) total += states_bytes(p, B, H, d) + 2 * padded_state_bytes(p, B, H);
     else if (op == COTT_OP_BWD)
         total += 3 * states_bytes(p, B, H, d) + 2 * align_up((size_t)B * H * p.n_groups * 4, 256) +
-                 3 * segment_state_bytes(B, H, d);
+                 (p.padded ? 6 : 3) * segment_state_bytes(B, H, d);
     return total;
 }
 
@@ -696,11 +696,19 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
             float* tq_tot = st2;           // (the third states region is free: dV' has no state pass of its own)
             float* b_v = st0;              // (one group: no stream has a state pass, the regions are free)
             const bool one = p.n_groups == 1;
-            if (seg.state_in)
-                COTT_CUDA(launch_state_prep(seg.state_in, b_q, BH, d, 1, 0, sp->m, sp->seq_len, sp->seq_len_scalar, H, N, st));
-            if (seg.d_state_out) {
-                COTT_CUDA(launch_state_prep(seg.d_state_out, b_k, BH, d, 1, 1, sp->m, sp->seq_len, sp->seq_len_scalar, H, N, st));
-                if (one) COTT_CUDA(launch_state_prep(seg.d_state_out, b_v, BH, d, 0, 1, sp->m, sp->seq_len, sp->seq_len_scalar, H, N, st));
+            // (smaller head sizes: the caller's states enter and leave through zero-padded copies)
+            const float* s_in = seg.state_in; const float* ds_out = seg.d_state_out; float* ds_in = seg.d_state_in;
+            if (p.padded) {
+                float* pad = reinterpret_cast<float*>(sbase + 3 * ssb);
+                if (seg.state_in) { COTT_CUDA(launch_pad_state(seg.state_in, pad, BH, p.dk, p.dv, d, st)); s_in = pad; }
+                if (seg.d_state_out) { COTT_CUDA(launch_pad_state(seg.d_state_out, pad + ssb / 4, BH, p.dk, p.dv, d, st)); ds_out = pad + ssb / 4; }
+                if (seg.d_state_in) ds_in = pad + 2 * (ssb / 4);
+            }
+            if (s_in)
+                COTT_CUDA(launch_state_prep(s_in, b_q, BH, d, 1, 0, sp->m, sp->seq_len, sp->seq_len_scalar, H, N, st));
+            if (ds_out) {
+                COTT_CUDA(launch_state_prep(ds_out, b_k, BH, d, 1, 1, sp->m, sp->seq_len, sp->seq_len_scalar, H, N, st));
+                if (one) COTT_CUDA(launch_state_prep(ds_out, b_v, BH, d, 0, 1, sp->m, sp->seq_len, sp->seq_len_scalar, H, N, st));
             }
             tk.clear_status = 1; tq.clear_status = 0;
             tk.dm_partial = dm_partial2; tk.dm_out = nullptr;
@@ -718,8 +726,9 @@ static cott_status bwd_impl(const void* q, const void* k, const void* v, const v
                 if ((rc = run_tc_stream(tv, p, B, H, N, d, causal, sp, status, st1, nullptr, st, true, false, true, b_k)) != COTT_OK)
                     return rc;
             }
-            COTT_CUDA(launch_segment_finish(seg.state_in, seg.d_state_out, tq_tot, tk_tot, seg.d_state_in, dm_partial, dm_partial2,
+            COTT_CUDA(launch_segment_finish(s_in, ds_out, tq_tot, tk_tot, ds_in, dm_partial, dm_partial2,
                                             BH, p.n_groups, d, sp->m, sp->seq_len, sp->seq_len_scalar, H, N, st));
+            if (p.padded && seg.d_state_in) COTT_CUDA(launch_unpad_state(ds_in, seg.d_state_in, BH, p.dk, p.dv, d, st));
             COTT_CUDA(launch_dm_finalize(dm_partial, dm, sp->m, sp->seq_len, sp->seq_len_scalar, B, H, p.n_groups, N, st, nullptr));
             return COTT_OK;
         }
@@ -1071,7 +1080,7 @@ static cott_status bwd_entry(const void* q, const void* k, const void* v, const 
         // else the fp32-accumulating kernels cover (equal key and value sizes of 32, 64 or 128) goes
         // through them, with the groups of the plan as it stands (the workspace was sized for it).
         const bool tc_fused = p.path == 1 && p.d == 64 && option_fused_bwd() != 0;
-        const bool tc_walks = p.path == 1 && p.d == 128 && d_k == 128 && d_v == 128 && option_force_path() != 0;
+        const bool tc_walks = p.path == 1 && p.d == 128;
         if (p.path == 1 && !tc_fused && !tc_walks) {
             if (!(d_k == d_v && (d_k == 32 || d_k == 64 || d_k == 128))) return COTT_ERR_UNSUPPORTED;
             p.path = 0; p.chunk = 16; p.d = d_k; p.padded = false; p.split = 1;

@@ -1142,11 +1142,35 @@ def test_segment_backward_through_three_walks(case, force_group, option):
         gate_dm(dm, rm, 1e-2, dm_condition(rv, c["v"], c["m"], s), DM_COND_BF16)
 
 
-def test_segment_backward_refuses_what_it_does_not_cover():
-    c = synth.make_qkv(1, 2, 64, 96, torch.bfloat16, 6700, with_do=True)
+@pytest.mark.parametrize("sizes", [(96, 96, 300, 128), (64, 128, 500, 4096), (128, 40, 260, 0), (72, 88, 130, 0)])
+def test_segment_backward_head_sizes_above_64(sizes, force_group):
+    """cott_bwd_stateful at bf16 head sizes that run in the kernels of size 128 (zero-filled
+    tiles): the caller's [d_k, d_v] states enter and leave through padded copies."""
+    dk, dv, N, group = sizes
+    if group:
+        force_group(group)
+    B, H = 2, 3
+    hist = synth.make_qkv(B, H, 90, dk, torch.bfloat16, 6850 + dk, d_v=dv)
+    c = synth.make_qkv(B, H, N, dk, torch.bfloat16, 6860 + dk + dv, with_do=True, d_v=dv)
+    c["m"] = hist["m"]
+    s = np.full((B,), float(N + 90))
+    _, st_in = oracle.fwd_segment(hist["q"], hist["k"], hist["v"], hist["m"], np.zeros((B, H, dk, dv)), s)
+    d_st_out = np.random.default_rng(6870 + dk).standard_normal((B, H, dk, dv)) * 0.5
+    rq, rk, rv, rst, rm = oracle.bwd_segment(c["q"], c["k"], c["v"], c["d_o"], c["m"], st_in, d_st_out, s)
     q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
+    f32 = lambda a: torch.tensor(a, dtype=torch.float32, device="cuda")
+    dq, dk_, dv_, dst, dm = cott.bwd_stateful(q, k, v, d_o, m, float(N + 90), state_in=f32(st_in), d_state_out=f32(d_st_out))
+    gate(dq, rq, torch.bfloat16); gate(dk_, rk, torch.bfloat16); gate(dv_, rv, torch.bfloat16)
+    assert norm_max_err(dst, rst) <= TOL_STATE_TC
+    gate_dm(dm, rm, 1e-2, dm_condition(rv, c["v"], c["m"], s), DM_COND_BF16)
+
+
+def test_segment_backward_refuses_what_it_does_not_cover():
+    c = synth.make_qkv(1, 2, 64, 32, torch.float32, 6700, with_do=True)
+    q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
+    wide = torch.zeros((1, 2, 64, 48), dtype=torch.float32, device="cuda")
     with pytest.raises(cott.CottError):
-        cott.bwd_stateful(q, k, v, d_o, m, 64.0)                     # bf16 between 64 and 128: not built
+        cott.bwd_stateful(wide, wide.clone(), wide.clone(), wide.clone(), m, 64.0)   # fp32 covers 32 / 64 / 128 only
     c = synth.make_qkv(1, 2, 64, 64, torch.bfloat16, 6701, with_do=True)
     q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
     with pytest.raises(cott.CottError):
