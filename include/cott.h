@@ -331,7 +331,7 @@ cott_status cott_bwd_after_fwd(const void* q, const void* k, const void* v, cons
  *                 through d_state_in); the parts of all segments add up to the dm of the sequence
  * Run over the segments last to first, with the caller's scaling base (sp->seq_len or
  * sp->seq_len_scalar >= 1, the same for every segment), the calls give the gradients of one
- * cott_bwd over the whole sequence.  Dense [B,H,N,d] tensors.  bf16 with d_k, d_v multiples of 8 up
+ * cott_bwd over the whole sequence.  bf16 with d_k, d_v multiples of 8 up
  * to 64: the one-walk backward of the tensor-core path.  bf16 with larger sizes (multiples of 8 up
  * to 128): the three tensor-core walks.  fp32 with d_k = d_v in {32, 64, 128}: three running-sum
  * walks of the fp32-accumulating kernels.  COTT_ERR_UNSUPPORTED otherwise.
@@ -341,6 +341,15 @@ cott_status cott_bwd_stateful(const void* q, const void* k, const void* v, const
                               const float* state_in, const float* d_state_out, void* dq, void* dk, void* dv,
                               float* d_state_in, float* dm, int B, int H, int N, int d_k, int d_v, cott_dtype dt,
                               const cott_scale_params* sp, void* workspace, size_t workspace_bytes, void* stream);
+
+/* cott_bwd_stateful on tensors that are not dense [B,H,N,d]; strides as for cott_bwd_dkdv (the states stay dense). */
+cott_status cott_bwd_stateful_strided(const void* q, const void* k, const void* v, const void* d_o,
+                                      const float* state_in, const float* d_state_out, void* dq, void* dk, void* dv,
+                                      float* d_state_in, float* dm, int B, int H, int N, int d_k, int d_v, cott_dtype dt,
+                                      const cott_strides* qk_strides, const cott_strides* v_strides,
+                                      const cott_strides* do_strides, const cott_strides* dqk_strides,
+                                      const cott_strides* dv_strides, const cott_scale_params* sp, void* workspace,
+                                      size_t workspace_bytes, void* stream);
 
 /*
  * Head sizes.  The paper's section 2.1 gives keys / queries and values sizes of their own

@@ -100,6 +100,8 @@ def _load():
                                               ctypes.POINTER(_ScaleParams), vp, cs, vp]
     lib.cott_bwd_stateful.restype = ci
     lib.cott_bwd_stateful.argtypes = [vp] * 11 + [ci] * 6 + [ctypes.POINTER(_ScaleParams), vp, cs, vp]
+    lib.cott_bwd_stateful_strided.restype = ci
+    lib.cott_bwd_stateful_strided.argtypes = [vp] * 11 + [ci] * 6 + [vp] * 5 + [ctypes.POINTER(_ScaleParams), vp, cs, vp]
     lib.cott_fwd_stateful.restype = ci
     lib.cott_fwd_stateful.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci,
                                       ctypes.POINTER(_ScaleParams), vp, cs, vp]
@@ -491,12 +493,13 @@ def bwd_varlen(q, k, v, d_o, m, cu_seqlens, max_seqlen, seq_len=None, causal=Tru
 
 @_on_call_stream
 def bwd_stateful(q, k, v, d_o, m, seq_len, state_in=None, d_state_out=None, return_d_state=True,
-                 workspace=None, stream=None):
+                 workspace=None, stream=None, out=None):
     """cott_bwd_stateful: the backward of one segment of a longer causal sequence.  ``state_in``
     (fp32 ``[B,H,d_k,d_v]`` or None = zero) is what ``fwd_stateful`` was given for the segment,
     ``d_state_out`` (same shape, or None = zero) the gradient of the state it handed on (the
-    ``d_state_in`` of the next segment's backward); ``seq_len`` as for ``fwd_stateful``.  Returns
-    ``(dq, dk, dv, d_state_in, dm)`` (``d_state_in`` is None when not asked for)."""
+    ``d_state_in`` of the next segment's backward); ``seq_len`` as for ``fwd_stateful``; tensors and
+    ``out`` as for ``bwd`` (strides are picked up).  Returns ``(dq, dk, dv, d_state_in, dm)``
+    (``d_state_in`` is None when not asked for)."""
     _check_rows(q, k, v, d_o)
     _check_dev(m, state_in, d_state_out, seq_len if isinstance(seq_len, torch.Tensor) else None)
     B, H, N, d = q.shape
@@ -505,22 +508,23 @@ def bwd_stateful(q, k, v, d_o, m, seq_len, state_in=None, d_state_out=None, retu
     for t in (state_in, d_state_out):
         if t is not None and (t.dtype != torch.float32 or tuple(t.shape) != (B, H, d, d_v) or not t.is_contiguous()):
             raise ValueError("states must be contiguous float32 [B,H,d_k,d_v]")
-    for t in (q, k, v, d_o):
-        if not t.is_contiguous():
-            raise ValueError("cott_bwd_stateful takes dense [B,H,N,d] tensors")
-    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    dq, dk, dv = (torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)) if out is None else out
+    _check_rows(dq, dk, dv)
+    same = d == d_v
+    st = [_strides_of(q, k, v) if same else _strides_of(q, k), None if same else _strides_of(v), _strides_of(d_o),
+          _strides_of(dq, dk, dv) if same else _strides_of(dq, dk), None if same else _strides_of(dv)]
     dm = torch.empty((H,), dtype=torch.float32, device=q.device)
     d_state_in = torch.empty((B, H, d, d_v), dtype=torch.float32, device=q.device) if return_d_state else None
     need = workspace_bytes_dkdv(OP_BWD, dt, B, H, N, d, d_v, True)
     ws = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device) if workspace is None else workspace
     sp = _scale(m, seq_len)
     ptr = lambda t: 0 if t is None else t.data_ptr()
-    rc = _load().cott_bwd_stateful(q.data_ptr(), k.data_ptr(), v.data_ptr(), d_o.data_ptr(), ptr(state_in),
-                                   ptr(d_state_out), dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), ptr(d_state_in),
-                                   dm.data_ptr(), B, H, N, d, d_v, dt, ctypes.byref(sp), ws.data_ptr(), ws.numel(),
-                                   _stream_ptr(stream))
+    rc = _load().cott_bwd_stateful_strided(q.data_ptr(), k.data_ptr(), v.data_ptr(), d_o.data_ptr(), ptr(state_in),
+                                           ptr(d_state_out), dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), ptr(d_state_in),
+                                           dm.data_ptr(), B, H, N, d, d_v, dt, *[_ref(x) for x in st], ctypes.byref(sp),
+                                           ws.data_ptr(), ws.numel(), _stream_ptr(stream))
     if rc != 0:
-        raise CottError(rc, "cott_bwd_stateful")
+        raise CottError(rc, "cott_bwd_stateful_strided")
     return dq, dk, dv, d_state_in, dm
 
 

@@ -1085,7 +1085,6 @@ static cott_status bwd_entry(const void* q, const void* k, const void* v, const 
             if (!(d_k == d_v && (d_k == 32 || d_k == 64 || d_k == 128))) return COTT_ERR_UNSUPPORTED;
             p.path = 0; p.chunk = 16; p.d = d_k; p.padded = false; p.split = 1;
         }
-        if (qk_strides || v_strides || do_strides || dqk_strides || dv_strides) return COTT_ERR_UNSUPPORTED;
         if ((seg.state_in && !aligned16(seg.state_in)) || (seg.d_state_out && !aligned16(seg.d_state_out)) ||
             (seg.d_state_in && !aligned16(seg.d_state_in)))
             return COTT_ERR_UNSUPPORTED;
@@ -1096,14 +1095,25 @@ static cott_status bwd_entry(const void* q, const void* k, const void* v, const 
                     own_v ? vs : nullptr, own_v ? dvs : nullptr, fwd_workspace, seg);
 }
 
+cott_status cott_bwd_stateful_strided(const void* q, const void* k, const void* v, const void* d_o,
+                                      const float* state_in, const float* d_state_out, void* dq, void* dk, void* dv,
+                                      float* d_state_in, float* dm, int B, int H, int N, int d_k, int d_v, cott_dtype dt,
+                                      const cott_strides* qk_strides, const cott_strides* v_strides,
+                                      const cott_strides* do_strides, const cott_strides* dqk_strides,
+                                      const cott_strides* dv_strides, const cott_scale_params* sp, void* workspace,
+                                      size_t workspace_bytes, void* stream) {
+    Segment seg;
+    seg.on = true; seg.state_in = state_in; seg.d_state_out = d_state_out; seg.d_state_in = d_state_in;
+    return bwd_entry(q, k, v, d_o, dq, dk, dv, dm, B, H, N, d_k, d_v, 1, dt, qk_strides, v_strides, do_strides, dqk_strides,
+                     dv_strides, sp, workspace, workspace_bytes, stream, nullptr, seg);
+}
+
 cott_status cott_bwd_stateful(const void* q, const void* k, const void* v, const void* d_o,
                               const float* state_in, const float* d_state_out, void* dq, void* dk, void* dv,
                               float* d_state_in, float* dm, int B, int H, int N, int d_k, int d_v, cott_dtype dt,
                               const cott_scale_params* sp, void* workspace, size_t workspace_bytes, void* stream) {
-    Segment seg;
-    seg.on = true; seg.state_in = state_in; seg.d_state_out = d_state_out; seg.d_state_in = d_state_in;
-    return bwd_entry(q, k, v, d_o, dq, dk, dv, dm, B, H, N, d_k, d_v, 1, dt, nullptr, nullptr, nullptr, nullptr,
-                     nullptr, sp, workspace, workspace_bytes, stream, nullptr, seg);
+    return cott_bwd_stateful_strided(q, k, v, d_o, state_in, d_state_out, dq, dk, dv, d_state_in, dm, B, H, N, d_k, d_v, dt,
+                                     nullptr, nullptr, nullptr, nullptr, nullptr, sp, workspace, workspace_bytes, stream);
 }
 
 cott_status cott_bwd_after_fwd(const void* q, const void* k, const void* v, const void* d_o, void* dq,

@@ -1165,6 +1165,27 @@ def test_segment_backward_head_sizes_above_64(sizes, force_group):
     gate_dm(dm, rm, 1e-2, dm_condition(rv, c["v"], c["m"], s), DM_COND_BF16)
 
 
+@pytest.mark.parametrize("dtype,d", [(torch.bfloat16, 64), (torch.bfloat16, 128), (torch.float32, 32)])
+def test_segment_backward_strided_matches_dense(dtype, d):
+    """cott_bwd_stateful_strided: q, k, v, dO stored [B,N,H,d] and gradients written into a fused
+    [B,N,3,H,d] buffer give the bits of the dense call."""
+    B, H, N = 2, 5, 333
+    c = synth.make_qkv(B, H, N, d, dtype, 6950 + d, with_do=True)
+    q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
+    g = torch.Generator(device="cuda"); g.manual_seed(9)
+    st_in = torch.randn((B, H, d, d), generator=g, device="cuda")
+    d_st_out = torch.randn((B, H, d, d), generator=g, device="cuda")
+    want = cott.bwd_stateful(q, k, v, d_o, m, 1000.0, state_in=st_in, d_state_out=d_st_out)
+    qs, ks, vs, dos = (_as_bnhd(x) for x in (q, k, v, d_o))
+    grads = torch.full((B, N, 3, H, d), 7.0, dtype=dtype, device="cuda")
+    outs = tuple(grads[:, :, i].permute(0, 2, 1, 3) for i in range(3))
+    got = cott.bwd_stateful(qs, ks, vs, dos, m, 1000.0, state_in=st_in, d_state_out=d_st_out, out=outs)
+    for x, y in zip(got[:3], want[:3]):
+        assert torch.equal(x, y)
+    assert torch.equal(got[3], want[3])
+    torch.testing.assert_close(got[4], want[4], rtol=0, atol=0)
+
+
 def test_segment_backward_refuses_what_it_does_not_cover():
     c = synth.make_qkv(1, 2, 64, 32, torch.float32, 6700, with_do=True)
     q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
