@@ -659,10 +659,12 @@ def test_repeated_calls_are_bit_identical(shape):
     assert all(torch.isfinite(x.float()).all() for x in first)
 
 
-def test_bidirectional_backward_many_heads():
-    """Bidirectional gradients at a BERT-like shape with more (b,h) pairs than SMs: one group of
-    four chunks per CTA through the read-out form of every gradient stream."""
-    B, H, N, d = 13, 12, 512, 64
+@pytest.mark.parametrize("B", [13, 32])
+def test_bidirectional_backward_many_heads(B):
+    """Bidirectional gradients at the BERT-base shape (B = 32: config 2 at full size, as bench.py's
+    c2-train times it) and with a ragged number of (b, h) pairs: more pairs than CTA slots, one
+    group of four chunks per CTA through the one-launch backward."""
+    H, N, d = 12, 512, 64
     c = synth.make_qkv(B, H, N, d, torch.bfloat16, 5100, with_do=True)
     q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
     dq, dk, dv, dm = cott.bwd(q, k, v, d_o, m, causal=False)
