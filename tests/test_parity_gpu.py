@@ -140,6 +140,30 @@ def test_config3_causal_bf16_zero_keys():
     assert torch.equal(o2, o)
 
 
+def test_config3_backward_bf16_zero_keys():
+    """Config 3 at full size with its backward (bench.py's c3-train: the GPT-2-small attention
+    training step; 5 % of the key rows are exactly zero, so the clamped branch of the chain rule
+    runs inside the one-walk backward): all gradients of the first batch item against the
+    quadratic definition, the clamped key rows relative to their own size."""
+    c = synth.make_config(3)
+    B, H, N, d = c["q"].shape
+    d_o = torch.randn(c["v"].shape, generator=torch.Generator().manual_seed(1003)).to(torch.bfloat16)
+    dq, dk, dv, dm = cott.bwd(dev(c["q"]), dev(c["k"]), dev(c["v"]), dev(d_o), dev(c["m"]), causal=True)
+    sub = slice(0, 1)
+    rq, rk, rv, _ = oracle.bwd_quadratic(c["q"][sub], c["k"][sub], c["v"][sub], d_o[sub], c["m"], np.full((1,), float(N)), True)
+    zero = (c["k"][sub].float().abs().sum(-1) == 0)                 # [1,H,N]
+    assert zero.any()
+    gate(dq[sub], rq, torch.bfloat16)
+    gate(dv[sub], rv, torch.bfloat16)
+    keep = ~zero
+    gate(dk[sub].cpu()[keep], rk[keep.numpy()], torch.bfloat16)
+    # a clamped row's gradient is dk^ / eps: compare row by row on its own scale
+    got_z, ref_z = dk[sub].cpu()[zero].double().numpy(), rk[zero.numpy()]
+    err = np.abs(got_z - ref_z).max(axis=-1) / np.abs(ref_z).max(axis=-1)
+    assert err.max() <= TOL_BF16, f"clamped key rows: {err.max():.3e}"
+    assert torch.isfinite(dm).all()
+
+
 def test_config4_causal_fwd_bwd_bf16():
     c = synth.make_config(4)
     q, k, v, d_o, m = (dev(c[x]) for x in ("q", "k", "v", "d_o", "m"))
